@@ -1,0 +1,187 @@
+"""The five benchmark programs as plain data (relations, rules, loaded facts).
+
+A ``Program`` is only a description: which relations exist, which rules derive
+them and which arrays are loaded.  It is handed unchanged to the CUDA binding
+and (in tests) to the CPU oracle; it performs no evaluation itself.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+from . import synth
+
+MAXPLUS, MINPLUS, LOGSUMEXP, SUMPROD = "maxplus", "minplus", "logsumexp", "sumprod"
+
+
+@dataclass(frozen=True)
+class Const:
+    value: int
+
+
+@dataclass(frozen=True)
+class Var:
+    """Column pattern ``column == mul * var + add`` (mul > 0)."""
+    var: int
+    mul: int = 1
+    add: int = 0
+
+
+@dataclass(frozen=True)
+class Affine:
+    """Head column ``c0 + sum(coef[v] * v)``."""
+    c0: int = 0
+    coef: Tuple[Tuple[int, int], ...] = ()      # ((var, coefficient), ...)
+
+
+def V(v: int) -> Affine:
+    return Affine(0, ((v, 1),))
+
+
+@dataclass(frozen=True)
+class Atom:
+    rel: str
+    args: Tuple[object, ...]
+
+
+@dataclass(frozen=True)
+class Rule:
+    head: str
+    head_exprs: Tuple[Affine, ...]
+    atoms: Tuple[Atom, ...]
+    emit_count: bool = False
+
+
+@dataclass
+class Program:
+    name: str
+    relations: Dict[str, Tuple[int, str]]                     # name -> (arity, semiring)
+    rules: List[Rule]
+    facts: Dict[str, Tuple[List[np.ndarray], Optional[np.ndarray]]] = field(default_factory=dict)
+    outputs: Sequence[str] = ()
+    info: Dict[str, object] = field(default_factory=dict)
+
+
+# ----------------------------------------------------------------------------
+
+def closure_program(src, dst, tag, semiring=MAXPLUS, name="closure") -> Program:
+    """path(x,y) :- edge(x,y).  path(x,z) :- path(x,y), edge(y,z)."""
+    return Program(
+        name=name,
+        relations={"edge": (2, semiring), "path": (2, semiring)},
+        rules=[
+            Rule("path", (V(0), V(1)), (Atom("edge", (Var(0), Var(1))),)),
+            Rule("path", (V(0), V(2)), (Atom("path", (Var(0), Var(1))), Atom("edge", (Var(1), Var(2))))),
+        ],
+        facts={"edge": ([np.ascontiguousarray(src, np.int32), np.ascontiguousarray(dst, np.int32)],
+                        None if tag is None else np.ascontiguousarray(tag, np.float32))},
+        outputs=("path",),
+    )
+
+
+def sssp_program(src, dst, w, source=0, semiring=MINPLUS, name="sssp") -> Program:
+    """dist(s) = 0 loaded as a fact.  dist(y) :- dist(x), edge(x,y)."""
+    return Program(
+        name=name,
+        relations={"edge": (2, semiring), "dist": (1, semiring)},
+        rules=[Rule("dist", (V(1),), (Atom("dist", (Var(0),)), Atom("edge", (Var(0), Var(1)))))],
+        facts={"edge": ([np.ascontiguousarray(src, np.int32), np.ascontiguousarray(dst, np.int32)],
+                        np.ascontiguousarray(w, np.float32)),
+               "dist": ([np.asarray([source], np.int32)], np.zeros(1, np.float32))},
+        outputs=("dist",),
+    )
+
+
+def reach_program(src, dst, w, sources, semiring=MINPLUS, name="reach") -> Program:
+    """reach(s,s) :- src(s).  reach(s,z) :- reach(s,y), edge(y,z)."""
+    return Program(
+        name=name,
+        relations={"edge": (2, semiring), "src": (1, semiring), "reach": (2, semiring)},
+        rules=[
+            Rule("reach", (V(0), V(0)), (Atom("src", (Var(0),)),)),
+            Rule("reach", (V(0), V(2)), (Atom("reach", (Var(0), Var(1))), Atom("edge", (Var(1), Var(2))))),
+        ],
+        facts={"edge": ([np.ascontiguousarray(src, np.int32), np.ascontiguousarray(dst, np.int32)],
+                        np.ascontiguousarray(w, np.float32)),
+               "src": ([np.ascontiguousarray(sources, np.int32)], None)},
+        outputs=("reach",),
+    )
+
+
+def triangle_program(src, dst, w, name="triangles") -> Program:
+    """tri_agg(x, count) :- e(x,y), e(y,z), e(z,x); tag = logsumexp of (w_xy + w_yz) + w_zx."""
+    return Program(
+        name=name,
+        relations={"e": (2, LOGSUMEXP), "tri_agg": (2, LOGSUMEXP)},
+        rules=[Rule("tri_agg", (V(0),),
+                    (Atom("e", (Var(0), Var(1))), Atom("e", (Var(1), Var(2))), Atom("e", (Var(2), Var(0)))),
+                    emit_count=True)],
+        facts={"e": ([np.ascontiguousarray(src, np.int32), np.ascontiguousarray(dst, np.int32)],
+                     np.ascontiguousarray(w, np.float32))},
+        outputs=("tri_agg",),
+    )
+
+
+def digits_program(log_tags: np.ndarray, name="digits") -> Program:
+    """sum(p, a+b) :- digit(2p, a), digit(2p+1, b), logsumexp per (p, a+b).
+
+    ``log_tags`` is [2B, 10]; digit(i, d) carries log_tags[i, d]."""
+    n_img = log_tags.shape[0]
+    img = np.repeat(np.arange(n_img, dtype=np.int32), 10)
+    dig = np.tile(np.arange(10, dtype=np.int32), n_img)
+    return Program(
+        name=name,
+        relations={"digit": (2, LOGSUMEXP), "sum": (2, LOGSUMEXP)},
+        rules=[Rule("sum", (V(0), Affine(0, ((1, 1), (2, 1)))),
+                    (Atom("digit", (Var(0, 2, 0), Var(1))), Atom("digit", (Var(0, 2, 1), Var(2)))))],
+        facts={"digit": ([img, dig], np.ascontiguousarray(log_tags.reshape(-1), np.float32))},
+        outputs=("sum",),
+    )
+
+
+# ----------------------------------------------------------------------------
+# the five configurations, with a size knob each
+# ----------------------------------------------------------------------------
+
+def config1(n_nodes=1000, n_edges=4000) -> Program:
+    seed = synth.SEED_BASE + 1
+    s, d = synth.uniform_digraph(n_nodes, n_edges, seed)
+    t = synth.log_prob_tags(n_edges, seed)
+    p = closure_program(s, d, t, MAXPLUS, name=f"closure_n{n_nodes}_m{n_edges}")
+    p.info.update(n_nodes=n_nodes, n_edges=n_edges)
+    return p
+
+
+def config2(scale=20, edge_factor=16) -> Program:
+    seed = synth.SEED_BASE + 2
+    s, d, w = synth.rmat_graph(scale, edge_factor, seed, "u1_10")
+    p = sssp_program(s, d, w, 0, MINPLUS, name=f"sssp_rmat{scale}")
+    p.info.update(scale=scale, n_nodes=1 << scale, n_edges=int(s.size))
+    return p
+
+
+def config3(scale=18, edge_factor=16) -> Program:
+    seed = synth.SEED_BASE + 3
+    s, d, w = synth.rmat_graph(scale, edge_factor, seed, "n01")
+    p = triangle_program(s, d, w, name=f"triangles_rmat{scale}")
+    p.info.update(scale=scale, n_nodes=1 << scale, n_edges=int(s.size))
+    return p
+
+
+def config4(n_pairs=65536) -> Program:
+    seed = synth.SEED_BASE + 4
+    lt = synth.digit_log_tags(2 * n_pairs, seed)
+    p = digits_program(lt, name=f"digits_B{n_pairs}")
+    p.info.update(n_pairs=n_pairs)
+    return p
+
+
+def config5(scale=22, edge_factor=16, n_sources=64) -> Program:
+    seed = synth.SEED_BASE + 5
+    s, d, w = synth.rmat_graph(scale, edge_factor, seed, "u1_10")
+    srcs = np.sort(synth.distinct_sources(1 << scale, n_sources, seed))
+    p = reach_program(s, d, w, srcs, MINPLUS, name=f"reach_rmat{scale}_s{n_sources}")
+    p.info.update(scale=scale, n_nodes=1 << scale, n_edges=int(s.size), n_sources=n_sources)
+    return p
