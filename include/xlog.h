@@ -1,0 +1,180 @@
+/* xlog.h -- C ABI of the B200 tagged-Datalog fixpoint engine.
+ *
+ * The library evaluates Datalog-style rules bottom-up over GPU-resident relations
+ * whose tuples carry an fp32 tag from a semiring, with the semi-naive loop of the
+ * paper's Algorithm 1 ("Semi-naive evaluation on GPU"): join the delta with the
+ * full relation, project the head, combine tags per head key, remove what the full
+ * relation already holds (keeping strict tag improvements) and merge, until
+ * nothing changes.  Relational steps follow the paper's kernel table ("Relational
+ * kernels": join, sort, groupby, dedup, set_ops, scan, pack); head aggregates are
+ * those of "Aggregations and constraints" (count, sum, min, max, logsumexp).
+ *
+ * Conventions
+ *   - every function returns an xlog_status, never throws, never aborts; outputs
+ *     are untouched on failure; xlog_last_error() gives a message;
+ *   - pointers are HOST pointers unless a parameter says xlog_memspace or "device";
+ *   - the caller owns every buffer it passes in (arena, inputs, outputs); the
+ *     context owns what it carves from the arena; nothing is freed across the
+ *     boundary; the library calls no cudaMalloc for relation data;
+ *   - all device work is issued on the stream given at context creation and every
+ *     entry point is stream-synchronous on return;
+ *   - a context is not thread-safe; there is no process-wide state
+ *     (Section "Crate architecture": no runtime singleton).
+ *   - keys are int32 and must be >= 0 (dense ids, Section "Reversible symbols").
+ */
+#ifndef XLOG_H
+#define XLOG_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define XLOG_MAX_ARITY 4
+#define XLOG_MAX_ATOMS 3
+#define XLOG_MAX_VARS  8
+
+/* Typed outcomes (Section "GPU residency model": RESOURCE_EXHAUSTED for bytes,
+ * CAPACITY_EXCEEDED for counts, CONVERGENCE_FAILURE for the iteration limit). */
+typedef enum {
+  XLOG_OK = 0,
+  XLOG_ERR_INVALID_ARGUMENT = 1,
+  XLOG_ERR_INVALID_VALUE = 2,        /* NaN tag, tag equal to the semiring zero, negative key */
+  XLOG_ERR_UNSUPPORTED = 3,          /* plan shape; non-idempotent oplus inside a recursive component */
+  XLOG_ERR_RESOURCE_EXHAUSTED = 4,   /* arena bytes */
+  XLOG_ERR_CAPACITY_EXCEEDED = 5,    /* key bits > 64, count > INT32_MAX, head value outside [0, 2^31) */
+  XLOG_ERR_CONVERGENCE_FAILURE = 6,  /* iteration cap reached */
+  XLOG_ERR_BUFFER_TOO_SMALL = 7,
+  XLOG_ERR_INVALID_STATE = 8,        /* derived relations poisoned by an earlier failure */
+  XLOG_ERR_CUDA = 9,
+  XLOG_ERR_INTERNAL = 10
+} xlog_status;
+
+/* (oplus, otimes, zero, one): MAXPLUS (max,+,-inf,0)  MINPLUS (min,+,+inf,0)
+ * LOGSUMEXP (logaddexp,+,-inf,0)  SUMPROD (+,*,0,1). */
+typedef enum { XLOG_SR_MAXPLUS = 0, XLOG_SR_MINPLUS = 1, XLOG_SR_LOGSUMEXP = 2, XLOG_SR_SUMPROD = 3 } xlog_semiring;
+typedef enum { XLOG_MEM_HOST = 0, XLOG_MEM_DEVICE = 1 } xlog_memspace;
+
+typedef struct xlog_ctx xlog_ctx;
+typedef int32_t xlog_rel;      /* relation handle, valid for the context that made it */
+typedef int32_t xlog_rule;     /* rule handle */
+
+typedef struct {
+  uint32_t struct_size;            /* sizeof(xlog_config) */
+  int32_t  device;                 /* CUDA device ordinal the arena lives on */
+  void*    stream;                 /* cudaStream_t, may be NULL (default stream) */
+  void*    arena;                  /* DEVICE memory, >= 256-byte aligned, owned by the caller, must outlive the ctx */
+  uint64_t arena_bytes;
+  int64_t  max_iterations;         /* per recursive component; <= 0 means 2^20 */
+  uint64_t candidate_chunk_bytes;  /* upper bound on one batch of join candidates; 0 = bounded by the arena only */
+  uint32_t flags;                  /* XLOG_FLAG_* */
+} xlog_config;
+
+#define XLOG_FLAG_CHECK_INVARIANTS 1u  /* after every load/merge verify keys strictly increase (slow, for tests) */
+
+/* ---- context --------------------------------------------------------------- */
+xlog_status xlog_ctx_create(const xlog_config* cfg, xlog_ctx** out);
+xlog_status xlog_ctx_destroy(xlog_ctx* ctx);          /* frees host state and the pinned control block only */
+const char* xlog_last_error(const xlog_ctx* ctx);     /* owned by ctx, valid until the next call on it */
+
+/* ---- relations (Section "Type system": typed columnar predicates) ------------ */
+/* arity 1..XLOG_MAX_ARITY.  The packed key of a row (all columns, bit widths taken
+ * from the column maxima) must fit 64 bits, else CAPACITY_EXCEEDED at load/fixpoint. */
+xlog_status xlog_relation_create(xlog_ctx* ctx, int32_t arity, xlog_semiring sr, const char* name, xlog_rel* out);
+
+/* Replace the relation's facts by n rows given column-major: cols[c][i], tags[i]
+ * (tags == NULL loads the semiring one).  COPIES the data (space says where cols/tags
+ * live), sorts lexicographically, combines rows with equal keys by oplus, canonicalises
+ * -0.0 to +0.0, stores int32 columns + fp32 tag column-major.  Rejects negative keys,
+ * NaN tags and (except SUMPROD) tags equal to the semiring zero with INVALID_VALUE.
+ * Any load drops all derived tuples of the context (as xlog_ctx_reset_idb). */
+xlog_status xlog_relation_load(xlog_ctx* ctx, xlog_rel rel, const int32_t* const* cols, const float* tags,
+                               int64_t n, xlog_memspace space);
+
+xlog_status xlog_relation_size(xlog_ctx* ctx, xlog_rel rel, int64_t* n);
+
+/* Copy the relation out in ascending lexicographic key order.  cols_out[c] and
+ * tags_out each hold `capacity` elements in `space`; BUFFER_TOO_SMALL if n > capacity. */
+xlog_status xlog_relation_read(xlog_ctx* ctx, xlog_rel rel, int32_t* const* cols_out, float* tags_out,
+                               int64_t capacity, int64_t* n_out, xlog_memspace space);
+
+/* Zero-copy DEVICE pointers to the stored columns (Section "Zero-copy
+ * interoperability"); borrowed, valid until the relation next changes. */
+xlog_status xlog_relation_view(xlog_ctx* ctx, xlog_rel rel, const int32_t** cols /*[arity]*/, const float** tags, int64_t* n);
+
+/* ---- rules: a compiled conjunctive plan ---------------------------------------
+ * Each atom argument is a constant or an affine pattern  column == mul*var + add
+ * (mul > 0; rows that do not divide evenly do not match).  Equal var ids are join
+ * keys.  Head column c is  c0 + sum_v coef[v]*var_v  evaluated in int64; a value
+ * outside [0, 2^31) fails the fixpoint with CAPACITY_EXCEEDED.  The head tag is
+ * the otimes-product of the atom tags in atom order, combined per head key with the
+ * HEAD relation's oplus.  emit_count_column appends the number of bindings of the
+ * group as a trailing int32 head column (the paper's count is a head column:
+ * Listing 7), so the head relation's arity is n_head_cols + 1.
+ * Supported shapes: 1 atom; 2 atoms joined on one variable, the second side looked
+ * up through a sorted index on that column, its other columns plain variables;
+ * the 3-atom directed triangle  h(x..) :- e(x,y), e(y,z), e(z,x)  evaluated as a
+ * fused intersect-and-aggregate (Section "Worst-case-optimal joins").  Anything
+ * else: UNSUPPORTED.  Which atoms are recursive is derived from the strongly
+ * connected components of the relation dependency graph. */
+typedef enum { XLOG_ARG_CONST = 0, XLOG_ARG_VAR = 1 } xlog_arg_kind;
+typedef struct { int32_t kind; int32_t var; int32_t mul; int32_t add; /* CONST: add is the value */ } xlog_arg;
+typedef struct { xlog_rel rel; xlog_arg args[XLOG_MAX_ARITY]; } xlog_atom;
+typedef struct { int64_t c0; int32_t coef[XLOG_MAX_VARS]; } xlog_expr;
+typedef struct {
+  uint32_t  struct_size;           /* sizeof(xlog_plan) */
+  xlog_rel  head_rel;
+  int32_t   n_head_cols;
+  xlog_expr head[XLOG_MAX_ARITY];
+  int32_t   n_atoms;
+  xlog_atom atoms[XLOG_MAX_ATOMS];
+  int32_t   emit_count_column;
+} xlog_plan;
+
+xlog_status xlog_rule_add(xlog_ctx* ctx, const xlog_plan* plan, xlog_rule* out);   /* validates and copies */
+
+/* ---- evaluation ------------------------------------------------------------- */
+/* Terminal receipt: status, counters and timing, never tuple data (Section
+ * "GPU-Native Symbolic Substrate"). */
+typedef struct {
+  uint32_t struct_size;            /* sizeof(xlog_receipt), set by the caller */
+  int32_t  status;
+  int64_t  strata;                 /* components evaluated */
+  int64_t  iterations;             /* join rounds over all components, seed rounds included */
+  int64_t  derived_tuples;         /* sum over rule heads of rows - loaded facts */
+  int64_t  candidates;             /* join outputs before aggregation */
+  int64_t  unique_candidates;      /* after reduce-by-key */
+  int64_t  new_tuples;
+  int64_t  improved_tags;
+  int64_t  h2d_bytes, d2h_bytes;   /* control traffic of this call (counters only) */
+  int64_t  kernel_launches;
+  int64_t  peak_arena_bytes;
+  double   device_ms;              /* CUDA-event time of the whole call on the ctx stream */
+} xlog_receipt;
+
+/* Evaluate all rules to the least fixpoint, strata in dependency order
+ * (Algorithm 1; non-recursive components evaluate each rule once).  On failure
+ * the derived relations are poisoned: every later call that needs them returns
+ * INVALID_STATE until xlog_ctx_reset_idb ("partial counters do not turn it into
+ * a result", Section "Current limitations").  receipt may be NULL. */
+xlog_status xlog_fixpoint(xlog_ctx* ctx, xlog_receipt* receipt);
+
+/* Drop all derived tuples; loaded facts and their join indices stay. */
+xlog_status xlog_ctx_reset_idb(xlog_ctx* ctx);
+
+/* Gradient of a non-recursive LOGSUMEXP (or SUMPROD) rule after a successful
+ * fixpoint (the quantity the paper obtains by circuit backward, Section
+ * "End-to-end training").  grad_head: DEVICE, one float per head row in stored
+ * order.  grad_atoms[j]: DEVICE, one float per row of atom j's relation in stored
+ * order; each distinct buffer is zero-filled first, then
+ *   LOGSUMEXP:  grad_j[row] += g[h] * exp(sum_i tag_i - out[h])
+ *   SUMPROD:    grad_j[row] += g[h] * prod_{i != j} tag_i
+ * Passing the same pointer for two atoms of one relation yields the sum. */
+xlog_status xlog_rule_backward(xlog_ctx* ctx, xlog_rule rule, const float* grad_head, float* const* grad_atoms);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* XLOG_H */

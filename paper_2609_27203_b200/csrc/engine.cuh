@@ -1,0 +1,353 @@
+// Host-side engine state and the typed building blocks the fixpoint driver composes:
+// sort, reduce-by-key, merge, join evaluation.  Everything here issues work on the context's
+// stream and sub-allocates from the caller's arena.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <functional>
+#include <set>
+#include <string>
+#include <vector>
+
+#include "../../include/xlog.h"
+#include "arena.h"
+#include "common.cuh"
+#include "join.cuh"
+#include "relops.cuh"
+#include "scan.cuh"
+#include "sort.cuh"
+
+namespace xlog {
+
+struct Fail {
+  xlog_status st;
+  std::string msg;
+};
+[[noreturn]] inline void fail(xlog_status st, const std::string& m) { throw Fail{st, m}; }
+
+#define XLOG_CUDA(expr)                                                                            \
+  do {                                                                                             \
+    cudaError_t e__ = (expr);                                                                      \
+    if (e__ != cudaSuccess) fail(XLOG_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); \
+  } while (0)
+
+constexpr int kCtrlSlots = 64;          // uint64 control words mirrored to pinned host memory
+constexpr int kSlotErr = 0;
+
+struct Ctx;
+
+// Arena allocation with scope lifetime.
+struct DevBuf {
+  Ctx* c = nullptr;
+  void* p = nullptr;
+  size_t bytes = 0;
+  DevBuf() {}
+  DevBuf(Ctx* ctx, size_t n);
+  DevBuf(const DevBuf&) = delete;
+  DevBuf& operator=(const DevBuf&) = delete;
+  DevBuf(DevBuf&& o) noexcept { *this = std::move(o); }
+  DevBuf& operator=(DevBuf&& o) noexcept {
+    if (this != &o) { reset(); c = o.c; p = o.p; bytes = o.bytes; o.p = nullptr; o.bytes = 0; }
+    return *this;
+  }
+  ~DevBuf() { reset(); }
+  void reset();
+  template <typename T> T* as() const { return reinterpret_cast<T*>(p); }
+};
+
+struct Index {                          // sorted access path on one column of a relation
+  bool valid = false;
+  int64_t domain = 0;                   // offsets has domain + 1 entries
+  DevBuf off;
+  int n_other = 0;
+  int other_src[kMaxArity - 1] = {0, 0, 0};     // original column of each non-probed column
+  const int32_t* other[kMaxArity - 1] = {nullptr, nullptr, nullptr};
+  const float* tags = nullptr;
+  DevBuf own_cols[kMaxArity - 1];       // owned storage when the index is a permuted copy
+  DevBuf own_tags;
+};
+
+struct Relation {
+  int arity = 0, sr = 0;
+  std::string name;
+  // loaded facts: packed keys sorted ascending, unique
+  KeyLayout layout{};
+  int key_bytes = 4;
+  int32_t col_max[kMaxArity] = {0, 0, 0, 0};
+  DevBuf fact_keys, fact_tags;
+  uint32_t n_facts = 0;
+  // current contents; alias the facts until something is derived
+  DevBuf cur_keys, cur_tags;
+  bool cur_owned = false;
+  uint32_t n = 0;
+  // column-major int32 view of the current contents
+  DevBuf cols[kMaxArity];
+  bool soa_valid = false;
+  Index idx[kMaxArity];
+  bool is_head = false;
+
+  const void* keys() const { return cur_owned ? cur_keys.p : fact_keys.p; }
+  float* tags() const { return reinterpret_cast<float*>(cur_owned ? cur_tags.p : fact_tags.p); }
+};
+
+struct JoinShape {                      // how a two-atom rule is evaluated with `outer` as the scanned side
+  bool ok = false;
+  int outer = 0, inner = 1;
+  int probe_col = 0;                    // column of the inner atom that is looked up
+  int probe_var = 0, probe_mul = 1, probe_add = 0;
+};
+
+struct RuleC {
+  xlog_plan plan;
+  int kind = 0;                         // 1: one atom, 2: two-atom join, 3: directed triangle
+  JoinShape shape[2];                   // indexed by the outer atom
+};
+
+struct Ctx {
+  int device = 0;
+  cudaStream_t stream = nullptr;
+  Arena arena;
+  int64_t max_iter = 1 << 20;
+  size_t chunk_bytes = 0;
+  uint32_t flags = 0;
+  std::string err;
+  std::vector<Relation*> rels;
+  std::vector<RuleC> rules;
+  bool idb_dirty = false, poisoned = false, evaluated = false;
+  uint64_t* d_ctrl = nullptr;
+  uint64_t* h_ctrl = nullptr;
+  int64_t launches = 0, d2h_bytes = 0, h2d_bytes = 0;
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  // receipt counters of the running fixpoint
+  int64_t r_candidates = 0, r_unique = 0, r_new = 0, r_improved = 0, r_iterations = 0, r_strata = 0;
+};
+
+inline DevBuf::DevBuf(Ctx* ctx, size_t n) : c(ctx), bytes(n) {
+  p = ctx->arena.alloc(n);
+  if (!p) {
+    char m[160];
+    snprintf(m, sizeof m, "arena exhausted: need %zu bytes, %zu of %zu in use, largest free block %zu", n,
+             ctx->arena.in_use(), ctx->arena.capacity(), ctx->arena.largest_free());
+    fail(XLOG_ERR_RESOURCE_EXHAUSTED, m);
+  }
+}
+inline void DevBuf::reset() {
+  if (p && c) c->arena.release(p);
+  p = nullptr; bytes = 0;
+}
+
+inline void check_launch(Ctx* c, const char* what) {
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) fail(XLOG_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
+  ++c->launches;
+}
+#define XLOG_LAUNCH(ctx, kern, grid, block, smem, ...)                   \
+  do {                                                                   \
+    kern<<<(grid), (block), (smem), (ctx)->stream>>>(__VA_ARGS__);       \
+    check_launch((ctx), #kern);                                          \
+  } while (0)
+
+inline unsigned grid_for(uint64_t n, int block, int cap = kSMs * 16) {
+  const uint64_t g = (n + block - 1) / block;
+  return (unsigned)std::max<uint64_t>(1, std::min<uint64_t>(g, (uint64_t)cap));
+}
+
+// Copy the control block to pinned host memory and wait: the bounded control read of an iteration.
+inline void sync_ctrl(Ctx* c) {
+  XLOG_CUDA(cudaMemcpyAsync(c->h_ctrl, c->d_ctrl, kCtrlSlots * sizeof(uint64_t), cudaMemcpyDeviceToHost, c->stream));
+  XLOG_CUDA(cudaStreamSynchronize(c->stream));
+  c->d2h_bytes += kCtrlSlots * sizeof(uint64_t);
+  const uint32_t e = (uint32_t)c->h_ctrl[kSlotErr];
+  if (e) {
+    XLOG_CUDA(cudaMemsetAsync(c->d_ctrl, 0, sizeof(uint64_t), c->stream));
+    if (e & kErrNegativeKey) fail(XLOG_ERR_INVALID_VALUE, "negative key");
+    if (e & kErrBadTag) fail(XLOG_ERR_INVALID_VALUE, "tag is NaN or the semiring zero");
+    if (e & kErrHeadRange) fail(XLOG_ERR_CAPACITY_EXCEEDED, "head column value outside the relation's key range [0, 2^31)");
+    if (e & kErrCountOverflow) fail(XLOG_ERR_CAPACITY_EXCEEDED, "count exceeds INT32_MAX");
+    if (e & kErrNotSorted) fail(XLOG_ERR_INTERNAL, "invariant violated: keys not strictly increasing");
+    fail(XLOG_ERR_INTERNAL, "device error flag set");
+  }
+}
+inline uint32_t* ctrl_u32(Ctx* c, int slot) { return reinterpret_cast<uint32_t*>(c->d_ctrl + slot); }
+inline void zero_ctrl(Ctx* c, int slot, int n = 1) {
+  XLOG_CUDA(cudaMemsetAsync(c->d_ctrl + slot, 0, n * sizeof(uint64_t), c->stream));
+}
+
+inline int bit_length(int64_t v) { int b = 0; while (v > 0) { ++b; v >>= 1; } return std::max(b, 1); }
+
+inline KeyLayout make_layout(int arity, const int32_t* col_max) {
+  KeyLayout L{};
+  L.arity = arity;
+  int bits[kMaxArity], total = 0;
+  for (int c = 0; c < arity; ++c) { bits[c] = bit_length(col_max[c]); total += bits[c]; }
+  int sh = total;
+  for (int c = 0; c < arity; ++c) { sh -= bits[c]; L.shift[c] = sh; L.mask[c] = (uint32_t)((1ull << bits[c]) - 1); }
+  L.total_bits = total;
+  return L;
+}
+inline bool same_layout(const KeyLayout& a, const KeyLayout& b) {
+  if (a.arity != b.arity || a.total_bits != b.total_bits) return false;
+  for (int c = 0; c < a.arity; ++c) if (a.shift[c] != b.shift[c] || a.mask[c] != b.mask[c]) return false;
+  return true;
+}
+
+// ---------------------------------------------------------------------------------
+// typed building blocks
+// ---------------------------------------------------------------------------------
+
+template <typename T>
+inline void scan_exclusive_u32_inplace(Ctx* c, uint32_t* v, uint64_t n, uint32_t* spine /* >= tiles entries */) {
+  if (n == 0) return;
+  const unsigned tiles = (unsigned)((n + kScanTile - 1) / kScanTile);
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), tiles, kScanBlock, 0, v, (int64_t)n, spine);
+  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, spine, (int64_t)tiles, (uint32_t*)nullptr);
+  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), tiles, kScanBlock, 0, v, (int64_t)n, spine, v);
+}
+
+// Sort n (key, tag) pairs on key bits [0, nbits).  On return keys/tags point at the sorted data
+// (either the original buffers or the alternates).
+template <typename K>
+inline void sort_pairs(Ctx* c, K*& keys, float*& tags, K*& keys_alt, float*& tags_alt, uint64_t n, int nbits) {
+  if (n <= 1) return;
+  const SortPlan p = make_sort_plan<K>(n, nbits);
+  if (p.passes == 0) return;
+  DevBuf hist(c, p.hist_entries * 4), spine(c, (p.scan_tiles + 1) * 4);
+  for (int pass = 0; pass < p.passes; ++pass) {
+    const int shift = pass * p.bits_per_pass;
+    const int nb = std::min(p.bits_per_pass, nbits - shift);
+    if (nb <= 0) break;
+    const int nbins = 1 << nb;
+    XLOG_LAUNCH(c, (k_sort_hist<K>), (p.ntiles + kHistGroup - 1) / kHistGroup, kSortBlock, 0, keys, (uint32_t)n, shift, nbins,
+                p.ntiles, hist.as<uint32_t>());
+    scan_exclusive_u32_inplace<uint32_t>(c, hist.as<uint32_t>(), (uint64_t)nbins * p.ntiles, spine.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_sort_scatter<K>), p.ntiles, kSortBlock, sort_scatter_smem<K>(), keys,
+                reinterpret_cast<const uint32_t*>(tags), keys_alt, reinterpret_cast<uint32_t*>(tags_alt), (uint32_t)n, shift,
+                nbins, p.ntiles, hist.as<uint32_t>());
+    std::swap(keys, keys_alt);
+    std::swap(tags, tags_alt);
+  }
+}
+
+// Sorted unique (key, tag) list in arena buffers of exact size.
+struct KeyTags {
+  DevBuf keys, tags;
+  uint32_t n = 0;
+  DevBuf head_pos;                      // optional: row index of each group head in the reduced input (+ sentinel n)
+};
+
+constexpr int kSlotA = 8, kSlotB = 9, kSlotC = 10, kSlotD = 11;
+
+// Reduce-by-key of a sorted list into caller-provided buffers of capacity n (typically the idle
+// half of the sort's double buffer, so nothing is allocated while the candidates are alive).
+// One control read returns the number of groups.  head_pos (optional, filled when
+// want_head_pos) gets the row index of each group's first row plus a sentinel n, so that a
+// group's size is head_pos[u+1] - head_pos[u].
+template <typename K, typename Op>
+inline uint32_t reduce_by_key_t(Ctx* c, const K* keys, const float* tags, uint32_t n, K* out_keys, float* out_tags,
+                                DevBuf* head_pos) {
+  if (n == 0) return 0;
+  typedef typename Op::A A;
+  const unsigned tiles = (n + kRbkTile - 1) / kRbkTile;
+  DevBuf heads(c, (size_t)tiles * 4), tails(c, (size_t)tiles * sizeof(A)), carry(c, (size_t)tiles * sizeof(A));
+  XLOG_LAUNCH(c, (k_rbk_tiles<K, Op>), tiles, kRbkBlock, 0, keys, tags, n, heads.as<uint32_t>(), tails.as<A>());
+  XLOG_LAUNCH(c, (k_rbk_spine<Op>), 1, 1024, 0, heads.as<uint32_t>(), tails.as<A>(), carry.as<A>(), tiles, ctrl_u32(c, kSlotA));
+  sync_ctrl(c);
+  const uint32_t u = (uint32_t)c->h_ctrl[kSlotA];
+  uint32_t* hp = nullptr;
+  if (head_pos) { *head_pos = DevBuf(c, ((size_t)u + 1) * 4); hp = head_pos->as<uint32_t>(); }
+  XLOG_LAUNCH(c, (k_rbk_emit<K, Op>), tiles, kRbkBlock, 0, keys, tags, n, heads.as<uint32_t>(), carry.as<A>(), out_keys, out_tags, hp);
+  if (hp) XLOG_CUDA(cudaMemcpyAsync(hp + u, &n, 4, cudaMemcpyHostToDevice, c->stream));
+  XLOG_CUDA(cudaStreamSynchronize(c->stream));           // scratch is released on return
+  return u;
+}
+template <typename K>
+inline uint32_t reduce_by_key(Ctx* c, int sr, const K* keys, const float* tags, uint32_t n, K* out_keys, float* out_tags,
+                              DevBuf* head_pos = nullptr) {
+  switch (sr) {
+    case XLOG_SR_MAXPLUS: return reduce_by_key_t<K, OpMax>(c, keys, tags, n, out_keys, out_tags, head_pos);
+    case XLOG_SR_MINPLUS: return reduce_by_key_t<K, OpMin>(c, keys, tags, n, out_keys, out_tags, head_pos);
+    case XLOG_SR_LOGSUMEXP: return reduce_by_key_t<K, OpLse>(c, keys, tags, n, out_keys, out_tags, head_pos);
+    default: return reduce_by_key_t<K, OpSum>(c, keys, tags, n, out_keys, out_tags, head_pos);
+  }
+}
+
+// Sort + reduce the first n pairs of (k0,t0) using (k1,t1) as the second half of the double
+// buffer; releases both and returns the groups in exact-size buffers.
+template <typename K>
+inline KeyTags sort_reduce(Ctx* c, int sr, DevBuf& k0, DevBuf& t0, DevBuf& k1, DevBuf& t1, uint64_t n, int nbits, bool want_head_pos) {
+  KeyTags out;
+  K* ka = k0.as<K>(); K* kb = k1.as<K>();
+  float* ta = t0.as<float>(); float* tb = t1.as<float>();
+  sort_pairs<K>(c, ka, ta, kb, tb, n, nbits);
+  out.n = reduce_by_key<K>(c, sr, ka, ta, (uint32_t)n, kb, tb, want_head_pos ? &out.head_pos : nullptr);
+  // the sorted input is no longer needed: free it, then move the groups into exact-size storage
+  const bool sorted_in_0 = (void*)ka == k0.p;
+  (sorted_in_0 ? k0 : k1).reset();
+  (sorted_in_0 ? t0 : t1).reset();
+  out.keys = DevBuf(c, (size_t)std::max(out.n, 1u) * sizeof(K));
+  out.tags = DevBuf(c, (size_t)std::max(out.n, 1u) * 4);
+  if (out.n) {
+    XLOG_CUDA(cudaMemcpyAsync(out.keys.p, kb, (size_t)out.n * sizeof(K), cudaMemcpyDeviceToDevice, c->stream));
+    XLOG_CUDA(cudaMemcpyAsync(out.tags.p, tb, (size_t)out.n * 4, cudaMemcpyDeviceToDevice, c->stream));
+    XLOG_CUDA(cudaStreamSynchronize(c->stream));
+  }
+  k0.reset(); t0.reset(); k1.reset(); t1.reset();
+  return out;
+}
+
+// Merge A (reduced candidates) into B (full): returns full' and, if want_delta, delta'.
+// If no key of A is new, B's tags are updated in place and full' stays empty (n_new == 0).
+struct MergeResult {
+  KeyTags full, delta;
+  uint32_t n_new = 0, n_improved = 0;
+  bool in_place = false;
+};
+template <typename K, typename Op>
+inline MergeResult merge_t(Ctx* c, const K* A, const float* TA, uint32_t na, const K* B, float* TB, uint32_t nb, bool want_delta,
+                           bool allow_in_place) {
+  MergeResult r;
+  const uint64_t total = (uint64_t)na + nb;
+  const unsigned tiles = (unsigned)((total + kMrgTile - 1) / kMrgTile);
+  if (tiles == 0) return r;
+  DevBuf a_start(c, ((size_t)tiles + 1) * 4), nf(c, (size_t)tiles * 4), nd(c, (size_t)tiles * 4);
+  XLOG_LAUNCH(c, (k_merge_partition<K>), (tiles + 1 + 255) / 256, 256, 0, A, na, B, nb, tiles, a_start.as<uint32_t>());
+  XLOG_LAUNCH(c, (k_merge<K, Op, false>), tiles, kMrgBlock, 0, A, TA, na, B, TB, nb, a_start.as<uint32_t>(), nf.as<uint32_t>(),
+              nd.as<uint32_t>(), (K*)nullptr, (float*)nullptr, (K*)nullptr, (float*)nullptr, 0);
+  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, nf.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotB));
+  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, nd.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotC));
+  sync_ctrl(c);
+  const uint32_t tot_f = (uint32_t)c->h_ctrl[kSlotB], tot_d = (uint32_t)c->h_ctrl[kSlotC];
+  r.n_new = tot_f - nb;
+  r.n_improved = tot_d - r.n_new;
+  r.in_place = allow_in_place && r.n_new == 0;
+  if (r.in_place && tot_d == 0) return r;             // nothing new, nothing improved
+  if (!r.in_place) {
+    r.full.n = tot_f;
+    r.full.keys = DevBuf(c, (size_t)tot_f * sizeof(K));
+    r.full.tags = DevBuf(c, (size_t)tot_f * 4);
+  }
+  // delta buffers are always written by the emit kernel (they are small); size >= 1 keeps pointers valid
+  r.delta.n = tot_d;
+  r.delta.keys = DevBuf(c, (size_t)std::max(tot_d, 1u) * sizeof(K));
+  r.delta.tags = DevBuf(c, (size_t)std::max(tot_d, 1u) * 4);
+  XLOG_LAUNCH(c, (k_merge<K, Op, true>), tiles, kMrgBlock, 0, A, TA, na, B, TB, nb, a_start.as<uint32_t>(), nf.as<uint32_t>(),
+              nd.as<uint32_t>(), r.full.keys.as<K>(), r.full.tags.as<float>(), r.delta.keys.as<K>(), r.delta.tags.as<float>(),
+              r.in_place ? 1 : 0);
+  if (!want_delta) { r.delta.keys.reset(); r.delta.tags.reset(); r.delta.n = 0; }
+  return r;
+}
+template <typename K>
+inline MergeResult merge(Ctx* c, int sr, const K* A, const float* TA, uint32_t na, const K* B, float* TB, uint32_t nb,
+                         bool want_delta, bool allow_in_place) {
+  switch (sr) {
+    case XLOG_SR_MAXPLUS: return merge_t<K, OpMax>(c, A, TA, na, B, TB, nb, want_delta, allow_in_place);
+    case XLOG_SR_MINPLUS: return merge_t<K, OpMin>(c, A, TA, na, B, TB, nb, want_delta, allow_in_place);
+    case XLOG_SR_LOGSUMEXP: return merge_t<K, OpLse>(c, A, TA, na, B, TB, nb, want_delta, false);
+    default: return merge_t<K, OpSum>(c, A, TA, na, B, TB, nb, want_delta, false);
+  }
+}
+
+}  // namespace xlog

@@ -1,0 +1,169 @@
+// Join of an outer relation (the delta, or a full relation in the seed round) with an indexed
+// inner relation, fused with head projection and the otimes of the tags (paper kernel table:
+// `join`, count -> scan -> materialise; Algorithm 1 lines 5-6; RIR `Project`).
+//
+// The paper's join is a chained hash join over FNV-1a hashes.  Here the inner side is a sorted
+// column store with an offsets array over its probed column (keys are dense ids), so a probe is
+// two offset reads, and materialisation is tiled by OUTPUT position: every block produces the
+// same number of candidates no matter how skewed the degrees are.
+#pragma once
+#include "common.cuh"
+
+namespace xlog {
+
+struct ArgSpec { int kind; int var; int mul; int add; };      // kind 0: constant `add`; 1: column == mul*var + add
+
+struct JoinSpec {
+  // outer side: packed keys + tags
+  KeyLayout outer;
+  ArgSpec outer_args[kMaxArity];
+  // inner side (absent for one-atom rules): offsets over the probed column, the other columns, tags
+  int has_inner;
+  int probe_var, probe_mul, probe_add;                        // probed value = probe_mul * var + probe_add
+  int64_t inner_domain;                                       // offsets has inner_domain + 1 entries
+  const uint32_t* inner_off;
+  int inner_free;                                             // number of non-probed inner columns
+  const int32_t* inner_col[kMaxArity - 1];
+  int inner_var[kMaxArity - 1];                               // variable bound by each non-probed column (pattern var + add)
+  int inner_add[kMaxArity - 1];
+  const float* inner_tag;
+  // head
+  KeyLayout head;
+  int64_t head_c0[kMaxArity];
+  int32_t head_coef[kMaxArity][kMaxVars];
+  int times;                                                  // otimes: 0 = add, 1 = multiply
+};
+
+// Decode an outer row into variable values; false if a constant / repeated variable /
+// divisibility test fails.
+template <typename KO>
+__device__ __forceinline__ bool bind_outer(const JoinSpec& S, KO key, int64_t* var) {
+  bool ok = true;
+  bool bound[kMaxVars];
+#pragma unroll
+  for (int v = 0; v < kMaxVars; ++v) { bound[v] = false; var[v] = 0; }
+#pragma unroll
+  for (int c = 0; c < kMaxArity; ++c) {
+    if (c < S.outer.arity) {
+      const int64_t val = key_col<KO>(S.outer, key, c);
+      const ArgSpec a = S.outer_args[c];
+      if (a.kind == 0) ok = ok && val == a.add;
+      else {
+        const int64_t d = val - a.add;
+        const int64_t q = d / a.mul;
+        const bool divides = q * a.mul == d;
+#pragma unroll
+        for (int v = 0; v < kMaxVars; ++v)
+          if (v == a.var) {
+            if (bound[v]) ok = ok && divides && var[v] == q;
+            else { ok = ok && divides; var[v] = q; bound[v] = true; }
+          }
+      }
+    }
+  }
+  return ok;
+}
+
+// One thread per outer row: degree (number of inner matches) and the first matching inner row.
+template <typename KO>
+__global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
+                                                    uint32_t* __restrict__ deg, uint32_t* __restrict__ first) {
+  const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_outer) return;
+  int64_t var[kMaxVars];
+  uint32_t d = 0, lo = 0;
+  if (bind_outer<KO>(S, okeys[i], var)) {
+    if (!S.has_inner) d = 1;
+    else {
+      int64_t pv = 0;
+#pragma unroll
+      for (int v = 0; v < kMaxVars; ++v) if (v == S.probe_var) pv = var[v];
+      pv = pv * S.probe_mul + S.probe_add;
+      if (pv >= 0 && pv < S.inner_domain) {
+        lo = S.inner_off[pv];
+        d = S.inner_off[pv + 1] - lo;
+      }
+    }
+  }
+  deg[i] = d;
+  first[i] = lo;
+}
+
+constexpr int kExpBlock = 256;
+constexpr int kExpItems = 8;
+constexpr int kExpTile = kExpBlock * kExpItems;       // candidates per block
+constexpr int kExpRows = 2048;                        // outer-row starts staged in shared memory
+
+// Block b writes candidates [out_lo + b*kExpTile, ...).  `start` is the exclusive scan of
+// `deg` (global candidate index of each outer row's first match).
+template <typename KO, typename KH>
+__global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, const float* __restrict__ otags,
+                                                           uint32_t n_outer, const uint64_t* __restrict__ start,
+                                                           const uint32_t* __restrict__ first, uint64_t out_lo, uint64_t out_hi,
+                                                           KH* __restrict__ ckeys, float* __restrict__ ctags,
+                                                           uint32_t* __restrict__ err) {
+  __shared__ uint64_t sstart[kExpRows + 1];
+  __shared__ uint32_t srow[2];
+  const uint64_t t_lo = out_lo + (uint64_t)blockIdx.x * kExpTile;
+  const uint64_t t_hi = min(t_lo + kExpTile, out_hi);
+  if (t_lo >= t_hi) return;
+  // outer rows covering this tile: r_lo = last row with start <= t_lo, r_hi = last row with start < t_hi
+  if (threadIdx.x < 2) {
+    const uint64_t target = threadIdx.x == 0 ? t_lo : t_hi - 1;
+    uint32_t lo = 0, hi = n_outer;                    // upper_bound(start, target) - 1
+    while (lo < hi) {
+      const uint32_t mid = lo + ((hi - lo) >> 1);
+      if (start[mid] <= target) lo = mid + 1; else hi = mid;
+    }
+    srow[threadIdx.x] = lo - 1;
+  }
+  __syncthreads();
+  const uint32_t r_lo = srow[0], r_hi = srow[1];
+  const uint32_t nrows = r_hi - r_lo + 1;
+  const bool staged = nrows <= kExpRows;
+  if (staged) for (uint32_t i = threadIdx.x; i < nrows; i += kExpBlock) sstart[i] = start[r_lo + i];
+  __syncthreads();
+
+  uint32_t e = 0;
+  for (uint64_t p = t_lo + threadIdx.x; p < t_hi; p += kExpBlock) {
+    // row = last row in [r_lo, r_hi] with start <= p   (rows of degree 0 share a start and are skipped)
+    uint32_t lo = 0, hi = nrows;
+    if (staged) {
+      while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (sstart[mid] <= p) lo = mid + 1; else hi = mid; }
+    } else {
+      while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (start[r_lo + mid] <= p) lo = mid + 1; else hi = mid; }
+    }
+    const uint32_t row = r_lo + lo - 1;
+    const uint32_t j = (uint32_t)(p - (staged ? sstart[lo - 1] : start[row]));
+    int64_t var[kMaxVars];
+    bind_outer<KO>(S, okeys[row], var);
+    float tag = otags[row];
+    if (S.has_inner) {
+      const uint32_t ir = first[row] + j;
+#pragma unroll
+      for (int c = 0; c < kMaxArity - 1; ++c)
+        if (c < S.inner_free) {
+          const int64_t val = (int64_t)S.inner_col[c][ir] - S.inner_add[c];
+#pragma unroll
+          for (int v = 0; v < kMaxVars; ++v) if (v == S.inner_var[c]) var[v] = val;
+        }
+      const float it = S.inner_tag[ir];
+      tag = S.times ? tag * it : tag + it;
+    }
+    KH key = 0;
+#pragma unroll
+    for (int c = 0; c < kMaxArity; ++c)
+      if (c < S.head.arity) {
+        int64_t h = S.head_c0[c];
+#pragma unroll
+        for (int v = 0; v < kMaxVars; ++v) h += (int64_t)S.head_coef[c][v] * var[v];
+        if (h < 0 || h > (int64_t)S.head.mask[c]) { e |= kErrHeadRange; h = 0; }
+        key |= (KH)(uint32_t)h << S.head.shift[c];
+      }
+    ckeys[p - out_lo] = key;
+    ctags[p - out_lo] = tag;
+  }
+  if (e) atomicOr(err, e);
+}
+
+}  // namespace xlog

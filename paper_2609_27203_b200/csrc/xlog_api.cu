@@ -1,0 +1,857 @@
+// C ABI of the engine (see include/xlog.h) and the host-side fixpoint driver.
+#include "engine.cuh"
+#include "triangle.cuh"
+#include "backward.cuh"
+
+using namespace xlog;
+
+struct xlog_ctx : public xlog::Ctx {};
+
+namespace {
+
+template <typename F>
+xlog_status guarded(xlog_ctx* c, F&& f) {
+  if (!c) return XLOG_ERR_INVALID_ARGUMENT;
+  try {
+    cudaSetDevice(c->device);
+    f();
+    c->err.clear();
+    return XLOG_OK;
+  } catch (const Fail& e) {
+    c->err = e.msg;
+    return e.st;
+  } catch (const std::exception& e) {
+    c->err = e.what();
+    return XLOG_ERR_INTERNAL;
+  }
+}
+
+Relation& rel_of(Ctx* c, xlog_rel r) {
+  if (r < 0 || r >= (int)c->rels.size()) fail(XLOG_ERR_INVALID_ARGUMENT, "bad relation handle");
+  return *c->rels[r];
+}
+
+float one_of(int sr) { return sr == XLOG_SR_SUMPROD ? 1.f : 0.f; }
+
+#define DISPATCH_K(key_bytes, ...)                        \
+  do {                                                    \
+    if ((key_bytes) == 4) { typedef uint32_t K; __VA_ARGS__; } \
+    else { typedef uint64_t K; __VA_ARGS__; }             \
+  } while (0)
+
+void drop_indices(Relation& R) {
+  for (int i = 0; i < kMaxArity; ++i) R.idx[i] = Index();
+}
+
+void drop_current(Relation& R) {
+  R.cur_keys.reset(); R.cur_tags.reset();
+  R.cur_owned = false;
+  R.n = R.n_facts;
+  R.soa_valid = false;
+  for (int i = 0; i < kMaxArity; ++i) R.cols[i].reset();
+  drop_indices(R);
+}
+
+void set_current(Relation& R, KeyTags&& kt) {
+  R.cur_keys = std::move(kt.keys);
+  R.cur_tags = std::move(kt.tags);
+  R.cur_owned = true;
+  R.n = kt.n;
+  R.soa_valid = false;
+  drop_indices(R);
+}
+
+// Column-major int32 view of the current contents.
+void ensure_soa(Ctx* c, Relation& R) {
+  if (R.soa_valid) return;
+  ColPtrsMut out{};
+  for (int i = 0; i < R.arity; ++i) {
+    R.cols[i] = DevBuf(c, (size_t)std::max(R.n, 1u) * 4);
+    out.c[i] = R.cols[i].as<int32_t>();
+  }
+  if (R.n) DISPATCH_K(R.key_bytes, XLOG_LAUNCH(c, (k_unpack<K>), grid_for(R.n, 256), 256, 0, (const K*)R.keys(), (int64_t)R.n, R.layout, out));
+  R.soa_valid = true;
+}
+
+// Repack the loaded facts under a wider layout (derived tuples need more bits than the facts).
+void relayout_facts(Ctx* c, Relation& R, const KeyLayout& L) {
+  if (same_layout(R.layout, L)) return;
+  const int nkb = L.total_bits <= 32 ? 4 : 8;
+  if (R.n_facts) {
+    ColPtrsMut tmp{}; ColPtrs tmpc{};
+    DevBuf cols[kMaxArity];
+    for (int i = 0; i < R.arity; ++i) { cols[i] = DevBuf(c, (size_t)R.n_facts * 4); tmp.c[i] = cols[i].as<int32_t>(); tmpc.c[i] = tmp.c[i]; }
+    DISPATCH_K(R.key_bytes, XLOG_LAUNCH(c, (k_unpack<K>), grid_for(R.n_facts, 256), 256, 0, R.fact_keys.as<K>(), (int64_t)R.n_facts, R.layout, tmp));
+    DevBuf nk(c, (size_t)R.n_facts * nkb);
+    DISPATCH_K(nkb, XLOG_LAUNCH(c, (k_pack<K>), grid_for(R.n_facts, 256), 256, 0, tmpc, R.fact_tags.as<float>(), (int64_t)R.n_facts, L,
+                                 0.f, nk.as<K>(), R.fact_tags.as<float>()));
+    XLOG_CUDA(cudaStreamSynchronize(c->stream));
+    R.fact_keys = std::move(nk);
+  }
+  R.layout = L;
+  R.key_bytes = nkb;
+  drop_current(R);
+}
+
+// ---- load ------------------------------------------------------------------------
+void load_relation(Ctx* c, Relation& R, const int32_t* const* cols, const float* tags, int64_t n, xlog_memspace space) {
+  if (n < 0 || n > (int64_t)1 << 31) fail(XLOG_ERR_CAPACITY_EXCEEDED, "row count must be in [0, 2^31]");
+  if (n > 0 && !cols) fail(XLOG_ERR_INVALID_ARGUMENT, "cols is NULL");
+  // drop everything the relation held
+  drop_current(R);
+  R.fact_keys.reset(); R.fact_tags.reset();
+  R.n_facts = R.n = 0;
+  for (int i = 0; i < kMaxArity; ++i) R.col_max[i] = 0;
+  R.layout = make_layout(R.arity, R.col_max);
+  R.key_bytes = 4;
+  c->idb_dirty = true;
+  if (n == 0) return;
+
+  // stage the input columns on the device
+  DevBuf stage[kMaxArity], stage_t;
+  ColPtrs in{};
+  const float* dtags = nullptr;
+  if (space == XLOG_MEM_HOST) {
+    for (int i = 0; i < R.arity; ++i) {
+      if (!cols[i]) fail(XLOG_ERR_INVALID_ARGUMENT, "column pointer is NULL");
+      stage[i] = DevBuf(c, (size_t)n * 4);
+      XLOG_CUDA(cudaMemcpyAsync(stage[i].p, cols[i], (size_t)n * 4, cudaMemcpyHostToDevice, c->stream));
+      in.c[i] = stage[i].as<int32_t>();
+    }
+    if (tags) {
+      stage_t = DevBuf(c, (size_t)n * 4);
+      XLOG_CUDA(cudaMemcpyAsync(stage_t.p, tags, (size_t)n * 4, cudaMemcpyHostToDevice, c->stream));
+      dtags = stage_t.as<float>();
+    }
+    c->h2d_bytes += (int64_t)n * 4 * (R.arity + (tags ? 1 : 0));
+  } else {
+    for (int i = 0; i < R.arity; ++i) { if (!cols[i]) fail(XLOG_ERR_INVALID_ARGUMENT, "column pointer is NULL"); in.c[i] = cols[i]; }
+    dtags = tags;
+  }
+
+  // validate, find the column maxima (they fix the key layout)
+  zero_ctrl(c, kSlotErr);
+  zero_ctrl(c, kSlotA, 4);
+  XLOG_LAUNCH(c, k_col_stats, grid_for(n, 256, kSMs * 8), 256, 0, in, dtags, n, R.arity, R.sr,
+              reinterpret_cast<int32_t*>(c->d_ctrl + kSlotA), ctrl_u32(c, kSlotErr));
+  sync_ctrl(c);
+  const int32_t* mx = reinterpret_cast<const int32_t*>(c->h_ctrl + kSlotA);
+  for (int i = 0; i < R.arity; ++i) R.col_max[i] = mx[i];
+  zero_ctrl(c, kSlotA, 4);
+  R.layout = make_layout(R.arity, R.col_max);
+  if (R.layout.total_bits > 64) fail(XLOG_ERR_CAPACITY_EXCEEDED, "packed key of relation '" + R.name + "' needs more than 64 bits");
+  R.key_bytes = R.layout.total_bits <= 32 ? 4 : 8;
+
+  // pack -> sort -> combine duplicates
+  DISPATCH_K(R.key_bytes, {
+    DevBuf k0(c, (size_t)n * sizeof(K)), t0(c, (size_t)n * 4), k1(c, (size_t)n * sizeof(K)), t1(c, (size_t)n * 4);
+    XLOG_LAUNCH(c, (k_pack<K>), grid_for(n, 256), 256, 0, in, dtags, n, R.layout, one_of(R.sr), k0.as<K>(), t0.as<float>());
+    for (int i = 0; i < kMaxArity; ++i) stage[i].reset();
+    stage_t.reset();
+    KeyTags kt = sort_reduce<K>(c, R.sr, k0, t0, k1, t1, (uint64_t)n, R.layout.total_bits, false);
+    R.fact_keys = std::move(kt.keys);
+    R.fact_tags = std::move(kt.tags);
+    R.n_facts = R.n = kt.n;
+  });
+  if (c->flags & XLOG_FLAG_CHECK_INVARIANTS) {
+    DISPATCH_K(R.key_bytes, XLOG_LAUNCH(c, (k_check_sorted<K>), grid_for(R.n, 256), 256, 0, R.fact_keys.as<K>(), (int64_t)R.n, ctrl_u32(c, kSlotErr)));
+    sync_ctrl(c);
+  }
+}
+
+// ---- rules -----------------------------------------------------------------------
+bool is_plain_var(const xlog_arg& a) { return a.kind == XLOG_ARG_VAR && a.mul == 1 && a.add == 0; }
+
+JoinShape join_shape(Ctx* c, const xlog_plan& p, int outer) {
+  JoinShape s;
+  s.outer = outer; s.inner = 1 - outer;
+  const xlog_atom& A = p.atoms[s.outer];
+  const xlog_atom& B = p.atoms[s.inner];
+  const int ka = c->rels[A.rel]->arity, kb = c->rels[B.rel]->arity;
+  bool bound[XLOG_MAX_VARS] = {false};
+  for (int i = 0; i < ka; ++i) if (A.args[i].kind == XLOG_ARG_VAR) bound[A.args[i].var] = true;
+  int probe = -1;
+  for (int i = 0; i < kb && probe < 0; ++i)
+    if (B.args[i].kind == XLOG_ARG_VAR && bound[B.args[i].var]) probe = i;
+  if (probe < 0) return s;                       // cross product: not supported
+  bool seen[XLOG_MAX_VARS] = {false};
+  for (int i = 0; i < kb; ++i) {
+    if (i == probe) continue;
+    const xlog_arg& a = B.args[i];
+    // every other inner column must introduce a fresh variable (filters on the inner side are not supported)
+    if (a.kind != XLOG_ARG_VAR || a.mul != 1 || bound[a.var] || seen[a.var]) return s;
+    seen[a.var] = true;
+  }
+  s.probe_col = probe;
+  s.probe_var = B.args[probe].var; s.probe_mul = B.args[probe].mul; s.probe_add = B.args[probe].add;
+  s.ok = true;
+  return s;
+}
+
+void add_rule(Ctx* c, const xlog_plan* p, xlog_rule* out) {
+  if (!p || !out) fail(XLOG_ERR_INVALID_ARGUMENT, "plan or out is NULL");
+  if (p->struct_size != sizeof(xlog_plan)) fail(XLOG_ERR_INVALID_ARGUMENT, "xlog_plan.struct_size mismatch");
+  Relation& H = rel_of(c, p->head_rel);
+  if (p->n_atoms < 1 || p->n_atoms > XLOG_MAX_ATOMS) fail(XLOG_ERR_INVALID_ARGUMENT, "n_atoms must be 1..3");
+  if (p->n_head_cols < 1 || p->n_head_cols + (p->emit_count_column ? 1 : 0) != H.arity)
+    fail(XLOG_ERR_INVALID_ARGUMENT, "head columns do not match the head relation's arity");
+  bool bound[XLOG_MAX_VARS] = {false};
+  for (int j = 0; j < p->n_atoms; ++j) {
+    Relation& R = rel_of(c, p->atoms[j].rel);
+    if ((R.sr == XLOG_SR_SUMPROD) != (H.sr == XLOG_SR_SUMPROD))
+      fail(XLOG_ERR_INVALID_ARGUMENT, "body relation '" + R.name + "' does not share the head's otimes");
+    for (int i = 0; i < R.arity; ++i) {
+      const xlog_arg& a = p->atoms[j].args[i];
+      if (a.kind == XLOG_ARG_VAR) {
+        if (a.var < 0 || a.var >= XLOG_MAX_VARS || a.mul <= 0) fail(XLOG_ERR_INVALID_ARGUMENT, "bad variable pattern");
+        bound[a.var] = true;
+      } else if (a.kind != XLOG_ARG_CONST) fail(XLOG_ERR_INVALID_ARGUMENT, "bad argument kind");
+    }
+  }
+  for (int h = 0; h < p->n_head_cols; ++h)
+    for (int v = 0; v < XLOG_MAX_VARS; ++v)
+      if (p->head[h].coef[v] != 0 && !bound[v]) fail(XLOG_ERR_INVALID_ARGUMENT, "head uses a variable no body atom binds");
+  RuleC r;
+  r.plan = *p;
+  if (p->n_atoms == 1) r.kind = 1;
+  else if (p->n_atoms == 2) {
+    r.kind = 2;
+    r.shape[0] = join_shape(c, *p, 0);
+    r.shape[1] = join_shape(c, *p, 1);
+    if (!r.shape[0].ok && !r.shape[1].ok)
+      fail(XLOG_ERR_UNSUPPORTED, "two-atom rule must join on one variable with the looked-up side's other columns plain fresh variables");
+  } else {
+    // directed triangle  h(x) :- e(x,y), e(y,z), e(z,x)
+    const xlog_atom* a = p->atoms;
+    bool ok = a[0].rel == a[1].rel && a[1].rel == a[2].rel && c->rels[a[0].rel]->arity == 2;
+    for (int j = 0; j < 3 && ok; ++j) ok = is_plain_var(a[j].args[0]) && is_plain_var(a[j].args[1]);
+    if (ok) {
+      const int x = a[0].args[0].var, y = a[0].args[1].var, z = a[1].args[1].var;
+      ok = x != y && y != z && x != z && a[1].args[0].var == y && a[2].args[0].var == z && a[2].args[1].var == x;
+      ok = ok && p->n_head_cols == 1 && p->head[0].c0 == 0;
+      for (int v = 0; v < XLOG_MAX_VARS && ok; ++v) ok = p->head[0].coef[v] == (v == x ? 1 : 0);
+    }
+    if (!ok) fail(XLOG_ERR_UNSUPPORTED, "three-atom rules are supported only as the directed triangle h(x) :- e(x,y), e(y,z), e(z,x)");
+    r.kind = 3;
+  }
+  c->rules.push_back(r);
+  H.is_head = true;
+  c->idb_dirty = true;
+  *out = (xlog_rule)c->rules.size() - 1;
+}
+
+// ---- indices ---------------------------------------------------------------------
+// Sorted access path on column `col` of R's current contents: offsets over that column plus the
+// remaining columns and tags in (col, others...) order.  Column 0 reuses the store itself.
+Index& ensure_index(Ctx* c, Relation& R, int col) {
+  Index& ix = R.idx[col];
+  if (ix.valid) return ix;
+  ensure_soa(c, R);
+  ix = Index();
+  ix.domain = (int64_t)R.col_max[col] + 1;
+  ix.n_other = R.arity - 1;
+  const int32_t* lead = nullptr;
+  if (col == 0 || R.n == 0) {
+    lead = R.cols[col].as<int32_t>();
+    for (int i = 1; i < R.arity; ++i) { ix.other_src[i - 1] = i; ix.other[i - 1] = R.cols[i].as<int32_t>(); }
+    if (col != 0) { int k = 0; for (int i = 0; i < R.arity; ++i) if (i != col) { ix.other_src[k] = i; ix.other[k] = R.cols[i].as<int32_t>(); ++k; } }
+    ix.tags = R.tags();
+  } else {
+    // permuted copy sorted by (col, remaining columns in order)
+    int perm[kMaxArity] = {0, 1, 2, 3};
+    perm[0] = col;
+    { int k = 1; for (int i = 0; i < R.arity; ++i) if (i != col) perm[k++] = i; }
+    int32_t pmax[kMaxArity] = {0, 0, 0, 0};
+    for (int i = 0; i < R.arity; ++i) pmax[i] = R.col_max[perm[i]];
+    const KeyLayout PL = make_layout(R.arity, pmax);
+    const int kb = PL.total_bits <= 32 ? 4 : 8;
+    ColPtrs in{};
+    for (int i = 0; i < R.arity; ++i) in.c[i] = R.cols[perm[i]].as<int32_t>();
+    DevBuf lead_buf(c, (size_t)R.n * 4);
+    for (int i = 1; i < R.arity; ++i) { ix.own_cols[i - 1] = DevBuf(c, (size_t)R.n * 4); ix.other_src[i - 1] = perm[i]; }
+    ix.own_tags = DevBuf(c, (size_t)R.n * 4);
+    DISPATCH_K(kb, {
+      DevBuf k0(c, (size_t)R.n * sizeof(K)), t0(c, (size_t)R.n * 4), k1(c, (size_t)R.n * sizeof(K)), t1(c, (size_t)R.n * 4);
+      XLOG_LAUNCH(c, (k_pack<K>), grid_for(R.n, 256), 256, 0, in, (const float*)R.tags(), (int64_t)R.n, PL, 0.f, k0.as<K>(), t0.as<float>());
+      K* ka = k0.as<K>(); K* kbuf = k1.as<K>();
+      float* ta = t0.as<float>(); float* tb = t1.as<float>();
+      sort_pairs<K>(c, ka, ta, kbuf, tb, R.n, PL.total_bits);
+      ColPtrsMut out{};
+      out.c[0] = lead_buf.as<int32_t>();
+      for (int i = 1; i < R.arity; ++i) out.c[i] = ix.own_cols[i - 1].as<int32_t>();
+      XLOG_LAUNCH(c, (k_unpack<K>), grid_for(R.n, 256), 256, 0, (const K*)ka, (int64_t)R.n, PL, out);
+      XLOG_CUDA(cudaMemcpyAsync(ix.own_tags.p, ta, (size_t)R.n * 4, cudaMemcpyDeviceToDevice, c->stream));
+      XLOG_CUDA(cudaStreamSynchronize(c->stream));
+    });
+    for (int i = 1; i < R.arity; ++i) ix.other[i - 1] = ix.own_cols[i - 1].as<int32_t>();
+    ix.tags = ix.own_tags.as<float>();
+    ix.off = DevBuf(c, ((size_t)ix.domain + 1) * 4);
+    XLOG_LAUNCH(c, k_build_offsets, grid_for(ix.domain + 1, 256), 256, 0, (const int32_t*)lead_buf.as<int32_t>(), R.n, ix.domain, ix.off.as<uint32_t>());
+    XLOG_CUDA(cudaStreamSynchronize(c->stream));
+    ix.valid = true;
+    return ix;
+  }
+  ix.off = DevBuf(c, ((size_t)ix.domain + 1) * 4);
+  XLOG_LAUNCH(c, k_build_offsets, grid_for(ix.domain + 1, 256), 256, 0, lead, R.n, ix.domain, ix.off.as<uint32_t>());
+  ix.valid = true;
+  return ix;
+}
+
+// ---- one round of rule evaluation --------------------------------------------------
+struct Source {                          // a packed (keys, tags) list standing for one atom's relation
+  const void* keys; const float* tags; uint32_t n; KeyLayout layout; int key_bytes;
+};
+Source full_source(const Relation& R) { return Source{R.keys(), R.tags(), R.n, R.layout, R.key_bytes}; }
+
+struct Variant {
+  const RuleC* rule;
+  int outer_atom;                        // the scanned atom (delta position for delta variants)
+  Source outer;
+};
+
+struct Counted {                         // a variant after count + scan
+  JoinSpec spec;
+  Source outer;
+  DevBuf deg, first, start, sums;
+  uint64_t total = 0;
+  int slot = 0;
+};
+
+JoinSpec make_spec(Ctx* c, const Variant& v, const Relation& H) {
+  const xlog_plan& p = v.rule->plan;
+  JoinSpec S{};
+  S.outer = v.outer.layout;
+  const xlog_atom& A = p.atoms[v.outer_atom];
+  for (int i = 0; i < c->rels[A.rel]->arity; ++i) S.outer_args[i] = ArgSpec{A.args[i].kind, A.args[i].var, A.args[i].mul, A.args[i].add};
+  S.has_inner = 0;
+  if (v.rule->kind == 2) {
+    const JoinShape& sh = v.rule->shape[v.outer_atom];
+    if (!sh.ok) fail(XLOG_ERR_UNSUPPORTED, "this rule cannot be evaluated with the required atom as the scanned side");
+    const xlog_atom& B = p.atoms[sh.inner];
+    Relation& RB = *c->rels[B.rel];
+    Index& ix = ensure_index(c, RB, sh.probe_col);
+    S.has_inner = 1;
+    S.probe_var = sh.probe_var; S.probe_mul = sh.probe_mul; S.probe_add = sh.probe_add;
+    S.inner_domain = ix.domain;
+    S.inner_off = ix.off.as<uint32_t>();
+    S.inner_free = ix.n_other;
+    for (int i = 0; i < ix.n_other; ++i) {
+      S.inner_col[i] = ix.other[i];
+      S.inner_var[i] = B.args[ix.other_src[i]].var;
+      S.inner_add[i] = B.args[ix.other_src[i]].add;
+    }
+    S.inner_tag = ix.tags;
+  }
+  S.head = H.layout;
+  if (p.emit_count_column) {             // candidates are keyed by the declared head columns only
+    int32_t mx[kMaxArity] = {0, 0, 0, 0};
+    for (int i = 0; i < p.n_head_cols; ++i) mx[i] = H.col_max[i];
+    S.head = make_layout(p.n_head_cols, mx);
+  }
+  for (int i = 0; i < p.n_head_cols; ++i) {
+    S.head_c0[i] = p.head[i].c0;
+    for (int k = 0; k < kMaxVars; ++k) S.head_coef[i][k] = p.head[i].coef[k];
+  }
+  S.times = H.sr == XLOG_SR_SUMPROD ? 1 : 0;
+  return S;
+}
+
+constexpr int kSlotTotals = 16;          // uint64 candidate totals of the variants of a round
+
+// Evaluate the variants, all deriving head relation H: join, project, sort, reduce by key.
+// `extra` (optional) is appended to the candidates before the sort (loaded facts of H in a
+// non-recursive stratum).  Returns the sorted unique candidates.
+KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Source* extra, const KeyLayout& cand_layout,
+                 bool want_head_pos) {
+  const int ckb = cand_layout.total_bits <= 32 ? 4 : 8;
+  std::vector<Counted> counted;
+  counted.reserve(variants.size());
+  if (variants.size() > (size_t)(kCtrlSlots - kSlotTotals)) fail(XLOG_ERR_UNSUPPORTED, "too many rule variants for one head");
+  // count + scan for every variant, then one control read for all totals
+  for (Variant& v : variants) {
+    if (v.outer.n == 0) continue;
+    counted.emplace_back();
+    Counted& q = counted.back();
+    q.spec = make_spec(c, v, H);
+    q.outer = v.outer;
+    q.slot = kSlotTotals + (int)counted.size() - 1;
+    const uint32_t n = v.outer.n;
+    const unsigned tiles = (n + kScanTile - 1) / kScanTile;
+    q.deg = DevBuf(c, (size_t)n * 4); q.first = DevBuf(c, (size_t)n * 4);
+    q.start = DevBuf(c, (size_t)n * 8); q.sums = DevBuf(c, (size_t)tiles * 8);
+    DISPATCH_K(v.outer.key_bytes, XLOG_LAUNCH(c, (k_join_count<K>), (n + 255) / 256, 256, 0, q.spec, (const K*)v.outer.keys, n,
+                                               q.deg.as<uint32_t>(), q.first.as<uint32_t>()));
+    XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)q.deg.as<uint32_t>(), (int64_t)n, q.sums.as<uint64_t>());
+    XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, q.sums.as<uint64_t>(), (int64_t)tiles, (uint64_t*)(c->d_ctrl + q.slot));
+    XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)q.deg.as<uint32_t>(), (int64_t)n,
+                (const uint64_t*)q.sums.as<uint64_t>(), q.start.as<uint64_t>());
+  }
+  uint64_t total = extra ? extra->n : 0;
+  if (!counted.empty()) {
+    sync_ctrl(c);
+    for (Counted& q : counted) { q.total = c->h_ctrl[q.slot]; total += q.total; q.deg.reset(); q.sums.reset(); }
+  }
+  c->r_candidates += (int64_t)total;
+  KeyTags result;
+  if (total == 0) return result;
+
+  // batch capacity: bounded by the configured chunk size and by what the arena can hold
+  const size_t per = (size_t)(ckb + 4) * 2;                                  // two buffers per candidate (sort ping-pong)
+  uint64_t cap = total;
+  if (c->chunk_bytes) cap = std::min<uint64_t>(cap, std::max<uint64_t>(1, c->chunk_bytes / per));
+  cap = std::min<uint64_t>(cap, (uint64_t)1 << 31);
+  {
+    const uint64_t fit = c->arena.largest_free() / (per + 1) ;                // leave room for sort scratch
+    if (fit < cap) cap = std::max<uint64_t>(std::min<uint64_t>(fit, cap), 1);
+  }
+  if (want_head_pos && cap < total) fail(XLOG_ERR_RESOURCE_EXHAUSTED, "a counted aggregate must fit one candidate batch");
+
+  size_t vi = 0; uint64_t vpos = 0; bool extra_done = extra == nullptr || extra->n == 0;
+  while (vi < counted.size() || !extra_done) {
+    DevBuf k0(c, cap * ckb), t0(c, cap * 4), k1(c, cap * ckb), t1(c, cap * 4);
+    uint64_t fill = 0;
+    while (fill < cap && vi < counted.size()) {
+      Counted& q = counted[vi];
+      const uint64_t take = std::min<uint64_t>(cap - fill, q.total - vpos);
+      if (take) {
+        const unsigned blocks = (unsigned)((take + kExpTile - 1) / kExpTile);
+        if (q.outer.key_bytes == 4 && ckb == 4)
+          XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint32_t>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.tags, q.outer.n,
+                      (const uint64_t*)q.start.as<uint64_t>(), (const uint32_t*)q.first.as<uint32_t>(), vpos, vpos + take, k0.as<uint32_t>() + fill, t0.as<float>() + fill, ctrl_u32(c, kSlotErr));
+        else if (q.outer.key_bytes == 4)
+          XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint64_t>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.tags, q.outer.n,
+                      (const uint64_t*)q.start.as<uint64_t>(), (const uint32_t*)q.first.as<uint32_t>(), vpos, vpos + take, k0.as<uint64_t>() + fill, t0.as<float>() + fill, ctrl_u32(c, kSlotErr));
+        else if (ckb == 4)
+          XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint32_t>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.tags, q.outer.n,
+                      (const uint64_t*)q.start.as<uint64_t>(), (const uint32_t*)q.first.as<uint32_t>(), vpos, vpos + take, k0.as<uint32_t>() + fill, t0.as<float>() + fill, ctrl_u32(c, kSlotErr));
+        else
+          XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint64_t>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.tags, q.outer.n,
+                      (const uint64_t*)q.start.as<uint64_t>(), (const uint32_t*)q.first.as<uint32_t>(), vpos, vpos + take, k0.as<uint64_t>() + fill, t0.as<float>() + fill, ctrl_u32(c, kSlotErr));
+        fill += take; vpos += take;
+      }
+      if (vpos == q.total) { q.start.reset(); q.first.reset(); ++vi; vpos = 0; }
+    }
+    if (!extra_done && vi == counted.size() && cap - fill >= extra->n) {
+      XLOG_CUDA(cudaMemcpyAsync((char*)k0.p + fill * ckb, extra->keys, (size_t)extra->n * ckb, cudaMemcpyDeviceToDevice, c->stream));
+      XLOG_CUDA(cudaMemcpyAsync(t0.as<float>() + fill, extra->tags, (size_t)extra->n * 4, cudaMemcpyDeviceToDevice, c->stream));
+      fill += extra->n;
+      extra_done = true;
+    } else if (!extra_done && vi == counted.size() && fill == 0) {
+      fail(XLOG_ERR_RESOURCE_EXHAUSTED, "candidate batch too small for the relation's loaded facts");
+    }
+    KeyTags part;
+    DISPATCH_K(ckb, part = sort_reduce<K>(c, H.sr, k0, t0, k1, t1, fill, cand_layout.total_bits, want_head_pos));
+    if (result.n == 0) result = std::move(part);
+    else {
+      // a later batch: union with oplus into the running result
+      MergeResult m;
+      DISPATCH_K(ckb, m = merge<K>(c, H.sr, part.keys.as<K>(), part.tags.as<float>(), part.n, result.keys.as<K>(), result.tags.as<float>(),
+                                    result.n, false, false));
+      XLOG_CUDA(cudaStreamSynchronize(c->stream));
+      result = std::move(m.full);
+    }
+  }
+  c->r_unique += result.n;
+  return result;
+}
+
+// ---- strata ------------------------------------------------------------------------
+std::vector<std::vector<int>> components(Ctx* c) {
+  const int n = (int)c->rels.size();
+  std::vector<std::set<int>> dep(n);
+  for (const RuleC& r : c->rules) for (int j = 0; j < r.plan.n_atoms; ++j) dep[r.plan.head_rel].insert(r.plan.atoms[j].rel);
+  std::vector<int> idx(n, -1), low(n, 0), stack; std::vector<char> on(n, 0);
+  std::vector<std::vector<int>> out; int counter = 0;
+  std::function<void(int)> visit = [&](int v) {
+    idx[v] = low[v] = counter++; stack.push_back(v); on[v] = 1;
+    for (int w : dep[v]) {
+      if (idx[w] < 0) { visit(w); low[v] = std::min(low[v], low[w]); }
+      else if (on[w]) low[v] = std::min(low[v], idx[w]);
+    }
+    if (low[v] == idx[v]) {
+      std::vector<int> comp;
+      for (;;) { int w = stack.back(); stack.pop_back(); on[w] = 0; comp.push_back(w); if (w == v) break; }
+      std::sort(comp.begin(), comp.end());
+      out.push_back(comp);                 // emitted after everything it depends on
+    }
+  };
+  for (int v = 0; v < n; ++v) if (idx[v] < 0) visit(v);
+  return out;
+}
+
+// Upper bounds of every column of every relation (loaded maxima pushed through the rules),
+// which fix the packed-key layouts before any kernel runs.
+void propagate_bounds(Ctx* c) {
+  const int n = (int)c->rels.size();
+  std::vector<std::array<int64_t, kMaxArity>> ub(n);
+  for (int r = 0; r < n; ++r) for (int i = 0; i < kMaxArity; ++i) ub[r][i] = c->rels[r]->n_facts ? c->rels[r]->col_max[i] : 0;
+  for (int round = 0; round < n + 3; ++round) {
+    bool changed = false;
+    for (const RuleC& rc : c->rules) {
+      const xlog_plan& p = rc.plan;
+      int64_t vub[XLOG_MAX_VARS];
+      for (int v = 0; v < XLOG_MAX_VARS; ++v) vub[v] = INT32_MAX;
+      for (int j = 0; j < p.n_atoms; ++j) {
+        const Relation& R = *c->rels[p.atoms[j].rel];
+        for (int i = 0; i < R.arity; ++i) {
+          const xlog_arg& a = p.atoms[j].args[i];
+          if (a.kind != XLOG_ARG_VAR) continue;
+          const int64_t b = (ub[p.atoms[j].rel][i] - a.add) / a.mul;
+          vub[a.var] = std::min(vub[a.var], std::max<int64_t>(b, 0));
+        }
+      }
+      for (int h = 0; h < p.n_head_cols; ++h) {
+        int64_t b = p.head[h].c0;
+        for (int v = 0; v < XLOG_MAX_VARS; ++v) if (p.head[h].coef[v] > 0) b += (int64_t)p.head[h].coef[v] * vub[v];
+        b = std::min<int64_t>(std::max<int64_t>(b, 0), INT32_MAX);
+        if (round >= n + 1 && b > ub[p.head_rel][h]) b = INT32_MAX;      // still growing: recursive arithmetic
+        if (b > ub[p.head_rel][h]) { ub[p.head_rel][h] = b; changed = true; }
+      }
+    }
+    if (!changed) break;
+  }
+  for (int r = 0; r < n; ++r) {
+    Relation& R = *c->rels[r];
+    if (!R.is_head) continue;
+    int32_t mx[kMaxArity] = {0, 0, 0, 0};
+    for (int i = 0; i < R.arity; ++i) mx[i] = (int32_t)ub[r][i];
+    // a trailing count column is sized when its values are known
+    const KeyLayout L = make_layout(R.arity, mx);
+    if (L.total_bits > 64) fail(XLOG_ERR_CAPACITY_EXCEEDED, "packed key of relation '" + R.name + "' needs more than 64 bits");
+    for (int i = 0; i < R.arity; ++i) R.col_max[i] = mx[i];
+    relayout_facts(c, R, L);
+  }
+}
+
+void reset_idb(Ctx* c) {
+  for (Relation* R : c->rels) if (R->is_head) drop_current(*R);
+  c->poisoned = false;
+  c->evaluated = false;
+}
+
+bool in_set(const std::vector<int>& comp, int r) { return std::binary_search(comp.begin(), comp.end(), r); }
+
+// Turn groups keyed by the declared head columns into rows of the counted head relation:
+// (declared columns..., group size), tag unchanged.  `counts` has one entry per group.
+void append_counts(Ctx* c, Relation& H, KeyTags& u, const KeyLayout& cl, const uint32_t* counts, uint32_t max_count) {
+  if (max_count > (uint32_t)INT32_MAX) fail(XLOG_ERR_CAPACITY_EXCEEDED, "count exceeds INT32_MAX");
+  const int nd = cl.arity;
+  H.col_max[nd] = (int32_t)max_count;
+  const KeyLayout L = make_layout(H.arity, H.col_max);
+  if (L.total_bits > 64) fail(XLOG_ERR_CAPACITY_EXCEEDED, "packed key of relation '" + H.name + "' needs more than 64 bits");
+  const int kb_in = cl.total_bits <= 32 ? 4 : 8, kb_out = L.total_bits <= 32 ? 4 : 8;
+  const int cbits = L.shift[nd - 1];               // bits of the count column = shift of the column before it
+  KeyTags out;
+  out.n = u.n;
+  out.keys = DevBuf(c, (size_t)std::max(u.n, 1u) * kb_out);
+  out.tags = std::move(u.tags);
+  if (u.n) {
+    const unsigned g = grid_for(u.n, 256);
+    if (kb_in == 4 && kb_out == 4) XLOG_LAUNCH(c, (k_append_count<uint32_t, uint32_t>), g, 256, 0, u.keys.as<uint32_t>(), counts, u.n, cbits, out.keys.as<uint32_t>());
+    else if (kb_in == 4) XLOG_LAUNCH(c, (k_append_count<uint32_t, uint64_t>), g, 256, 0, u.keys.as<uint32_t>(), counts, u.n, cbits, out.keys.as<uint64_t>());
+    else XLOG_LAUNCH(c, (k_append_count<uint64_t, uint64_t>), g, 256, 0, u.keys.as<uint64_t>(), counts, u.n, cbits, out.keys.as<uint64_t>());
+    XLOG_CUDA(cudaStreamSynchronize(c->stream));
+  }
+  H.layout = L;
+  H.key_bytes = kb_out;
+  set_current(H, std::move(out));
+}
+
+void append_count_column(Ctx* c, Relation& H, KeyTags& u, const KeyLayout& cl) {
+  DevBuf counts(c, (size_t)std::max(u.n, 1u) * 4);
+  zero_ctrl(c, kSlotD);
+  if (u.n) XLOG_LAUNCH(c, k_group_sizes, grid_for(u.n, 256), 256, 0, (const uint32_t*)u.head_pos.as<uint32_t>(), u.n, counts.as<uint32_t>(), ctrl_u32(c, kSlotD));
+  sync_ctrl(c);
+  append_counts(c, H, u, cl, counts.as<uint32_t>(), (uint32_t)c->h_ctrl[kSlotD]);
+}
+
+void triangle_aggregate(Ctx* c, Relation& H, const RuleC& r) { (void)c; (void)H; (void)r; fail(XLOG_ERR_UNSUPPORTED, "triangle rule: not built yet"); }
+void rule_backward(Ctx* c, const RuleC& r, const float* g, float* const* grads) { (void)c; (void)r; (void)g; (void)grads; fail(XLOG_ERR_UNSUPPORTED, "backward: not built yet"); }
+
+// Non-recursive stratum:  I(P) = facts(P) oplus (oplus over rules of T_r), each rule evaluated once.
+void stratum_once(Ctx* c, int head, const std::vector<const RuleC*>& rs) {
+  Relation& H = *c->rels[head];
+  const bool counted = rs[0]->plan.emit_count_column != 0;
+  for (const RuleC* r : rs) if ((r->plan.emit_count_column != 0) != counted) fail(XLOG_ERR_UNSUPPORTED, "rules of one head disagree on emit_count_column");
+  if (counted && H.n_facts) fail(XLOG_ERR_UNSUPPORTED, "a counted head relation cannot also hold loaded facts");
+  if (counted && rs.size() > 1) fail(XLOG_ERR_UNSUPPORTED, "a counted head relation takes exactly one rule");
+  ++c->r_iterations;
+  if (rs.size() == 1 && rs[0]->kind == 3) { triangle_aggregate(c, H, *rs[0]); return; }
+  std::vector<Variant> vs;
+  for (const RuleC* r : rs) {
+    if (r->kind == 3) fail(XLOG_ERR_UNSUPPORTED, "a triangle rule must be the only rule of its head");
+    int outer = 0;
+    if (r->kind == 2 && !r->shape[0].ok) outer = 1;
+    vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
+  }
+  KeyLayout cl = H.layout;
+  if (counted) { int32_t mx[kMaxArity] = {0, 0, 0, 0}; for (int i = 0; i < rs[0]->plan.n_head_cols; ++i) mx[i] = H.col_max[i]; cl = make_layout(rs[0]->plan.n_head_cols, mx); }
+  Source facts{H.fact_keys.p, H.fact_tags.as<float>(), H.n_facts, H.layout, H.key_bytes};
+  KeyTags u = evaluate(c, H, vs, H.n_facts ? &facts : nullptr, cl, counted);
+  if (counted) append_count_column(c, H, u, cl);
+  else set_current(H, std::move(u));
+  c->r_new += (int64_t)H.n - H.n_facts;
+}
+
+// Recursive component: Algorithm 1 with tag improvement.
+void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<const RuleC*>& rs) {
+  for (int p : comp) if (c->rels[p]->sr != XLOG_SR_MAXPLUS && c->rels[p]->sr != XLOG_SR_MINPLUS)
+    fail(XLOG_ERR_UNSUPPORTED, "relation '" + c->rels[p]->name + "': only max/min tags may be aggregated inside a recursive component");
+  for (const RuleC* r : rs) {
+    if (r->plan.emit_count_column) fail(XLOG_ERR_UNSUPPORTED, "count inside a recursive component");
+    if (r->kind == 3) fail(XLOG_ERR_UNSUPPORTED, "triangle rule inside a recursive component");
+  }
+  std::vector<KeyTags> delta(c->rels.size());
+  for (int64_t round = 0;; ++round) {
+    if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
+    ++c->r_iterations;
+    // evaluate every head against the same state, then absorb
+    std::vector<std::pair<int, KeyTags>> produced;
+    for (int h : comp) {
+      Relation& H = *c->rels[h];
+      std::vector<Variant> vs;
+      for (const RuleC* r : rs) {
+        if (r->plan.head_rel != h) continue;
+        if (round == 0) {                                   // seed: every atom reads the full relation
+          int outer = 0;
+          if (r->kind == 2) {
+            const bool in0 = in_set(comp, r->plan.atoms[0].rel), in1 = in_set(comp, r->plan.atoms[1].rel);
+            if (in0 && in1) fail(XLOG_ERR_UNSUPPORTED, "rules with two recursive atoms are not supported");
+            outer = in1 ? 1 : 0;                            // scan the recursive side, look up the stable side
+            if (!r->shape[outer].ok) { if (!in0 && !in1 && r->shape[1 - outer].ok) outer = 1 - outer; else fail(XLOG_ERR_UNSUPPORTED, "no index path for this rule"); }
+          }
+          vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
+        } else {
+          for (int j = 0; j < r->plan.n_atoms; ++j) {
+            const int ar = r->plan.atoms[j].rel;
+            if (!in_set(comp, ar)) continue;
+            if (r->kind == 2 && in_set(comp, r->plan.atoms[1 - j].rel)) fail(XLOG_ERR_UNSUPPORTED, "rules with two recursive atoms are not supported");
+            const KeyTags& d = delta[ar];
+            if (d.n == 0) continue;
+            const Relation& RA = *c->rels[ar];
+            vs.push_back(Variant{r, j, Source{d.keys.p, d.tags.as<float>(), d.n, RA.layout, RA.key_bytes}});
+          }
+        }
+      }
+      if (vs.empty()) continue;
+      produced.emplace_back(h, evaluate(c, H, vs, nullptr, H.layout, false));
+    }
+    for (int p : comp) delta[p] = KeyTags();
+    uint64_t changed = 0;
+    for (auto& pr : produced) {
+      Relation& H = *c->rels[pr.first];
+      KeyTags& u = pr.second;
+      if (u.n == 0) continue;
+      if (!H.cur_owned && H.n_facts) {
+        // first derivation into a relation that holds facts: work on a private copy
+        KeyTags copy; copy.n = H.n_facts;
+        copy.keys = DevBuf(c, (size_t)H.n_facts * H.key_bytes); copy.tags = DevBuf(c, (size_t)H.n_facts * 4);
+        XLOG_CUDA(cudaMemcpyAsync(copy.keys.p, H.fact_keys.p, (size_t)H.n_facts * H.key_bytes, cudaMemcpyDeviceToDevice, c->stream));
+        XLOG_CUDA(cudaMemcpyAsync(copy.tags.p, H.fact_tags.p, (size_t)H.n_facts * 4, cudaMemcpyDeviceToDevice, c->stream));
+        set_current(H, std::move(copy));
+      }
+      MergeResult m;
+      DISPATCH_K(H.key_bytes, m = merge<K>(c, H.sr, u.keys.as<K>(), u.tags.as<float>(), u.n, (const K*)H.keys(), H.tags(), H.n, true, H.cur_owned));
+      XLOG_CUDA(cudaStreamSynchronize(c->stream));
+      if (!m.in_place) set_current(H, std::move(m.full));
+      c->r_new += m.n_new; c->r_improved += m.n_improved;
+      changed += (uint64_t)m.n_new + m.n_improved;
+      delta[pr.first] = std::move(m.delta);
+      if (c->flags & XLOG_FLAG_CHECK_INVARIANTS) {
+        DISPATCH_K(H.key_bytes, XLOG_LAUNCH(c, (k_check_sorted<K>), grid_for(H.n, 256), 256, 0, (const K*)H.keys(), (int64_t)H.n, ctrl_u32(c, kSlotErr)));
+        sync_ctrl(c);
+      }
+    }
+    if (changed == 0) break;
+  }
+}
+
+void run_fixpoint(Ctx* c) {
+  if (c->idb_dirty) { reset_idb(c); c->idb_dirty = false; }
+  if (c->poisoned) fail(XLOG_ERR_INVALID_STATE, "derived relations are poisoned by an earlier failure; call xlog_ctx_reset_idb");
+  c->poisoned = true;                      // cleared on success
+  zero_ctrl(c, kSlotErr);
+  propagate_bounds(c);
+  for (const std::vector<int>& comp : components(c)) {
+    std::vector<const RuleC*> rs;
+    for (const RuleC& r : c->rules) if (in_set(comp, r.plan.head_rel)) rs.push_back(&r);
+    if (rs.empty()) continue;
+    ++c->r_strata;
+    bool recursive = comp.size() > 1;
+    for (const RuleC* r : rs) for (int j = 0; j < r->plan.n_atoms; ++j) if (in_set(comp, r->plan.atoms[j].rel)) recursive = true;
+    if (!recursive) stratum_once(c, comp[0], rs); else stratum_recursive(c, comp, rs);
+  }
+  for (Relation* R : c->rels) if (R->is_head) ensure_soa(c, *R);
+  sync_ctrl(c);
+  c->poisoned = false;
+  c->evaluated = true;
+}
+
+}  // namespace
+
+// =====================================================================================
+extern "C" {
+
+xlog_status xlog_ctx_create(const xlog_config* cfg, xlog_ctx** out) {
+  if (!cfg || !out || cfg->struct_size != sizeof(xlog_config) || !cfg->arena || cfg->arena_bytes < (1u << 16)) return XLOG_ERR_INVALID_ARGUMENT;
+  xlog_ctx* c = new (std::nothrow) xlog_ctx();
+  if (!c) return XLOG_ERR_INTERNAL;
+  c->device = cfg->device;
+  c->stream = (cudaStream_t)cfg->stream;
+  c->max_iter = cfg->max_iterations > 0 ? cfg->max_iterations : (int64_t)1 << 20;
+  c->chunk_bytes = cfg->candidate_chunk_bytes;
+  c->flags = cfg->flags;
+  c->arena.init(cfg->arena, cfg->arena_bytes);
+  xlog_status st = guarded(c, [&] {
+    c->d_ctrl = reinterpret_cast<uint64_t*>(c->arena.alloc(kCtrlSlots * sizeof(uint64_t)));
+    if (!c->d_ctrl) fail(XLOG_ERR_RESOURCE_EXHAUSTED, "arena too small");
+    XLOG_CUDA(cudaHostAlloc(&c->h_ctrl, kCtrlSlots * sizeof(uint64_t), cudaHostAllocDefault));
+    XLOG_CUDA(cudaMemsetAsync(c->d_ctrl, 0, kCtrlSlots * sizeof(uint64_t), c->stream));
+    XLOG_CUDA(cudaEventCreate(&c->ev0));
+    XLOG_CUDA(cudaEventCreate(&c->ev1));
+    XLOG_CUDA(cudaFuncSetAttribute(k_sort_scatter<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_scatter_smem<uint32_t>()));
+    XLOG_CUDA(cudaFuncSetAttribute(k_sort_scatter<uint64_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_scatter_smem<uint64_t>()));
+    XLOG_CUDA(cudaStreamSynchronize(c->stream));
+  });
+  if (st != XLOG_OK) { if (c->h_ctrl) cudaFreeHost(c->h_ctrl); delete c; return st; }
+  *out = c;
+  return XLOG_OK;
+}
+
+xlog_status xlog_ctx_destroy(xlog_ctx* c) {
+  if (!c) return XLOG_ERR_INVALID_ARGUMENT;
+  cudaSetDevice(c->device);
+  cudaStreamSynchronize(c->stream);
+  for (Relation* R : c->rels) delete R;
+  if (c->h_ctrl) cudaFreeHost(c->h_ctrl);
+  if (c->ev0) cudaEventDestroy(c->ev0);
+  if (c->ev1) cudaEventDestroy(c->ev1);
+  delete c;
+  return XLOG_OK;
+}
+
+const char* xlog_last_error(const xlog_ctx* c) { return c ? c->err.c_str() : "null context"; }
+
+xlog_status xlog_relation_create(xlog_ctx* c, int32_t arity, xlog_semiring sr, const char* name, xlog_rel* out) {
+  return guarded(c, [&] {
+    if (!out || arity < 1 || arity > XLOG_MAX_ARITY || (int)sr < 0 || (int)sr > 3) fail(XLOG_ERR_INVALID_ARGUMENT, "bad arity or semiring");
+    Relation* R = new Relation();
+    R->arity = arity; R->sr = (int)sr; R->name = name ? name : "";
+    R->layout = make_layout(arity, R->col_max);
+    c->rels.push_back(R);
+    *out = (xlog_rel)c->rels.size() - 1;
+  });
+}
+
+xlog_status xlog_relation_load(xlog_ctx* c, xlog_rel rel, const int32_t* const* cols, const float* tags, int64_t n, xlog_memspace space) {
+  return guarded(c, [&] {
+    Relation& R = rel_of(c, rel);
+    try { load_relation(c, R, cols, tags, n, space); }
+    catch (...) {                          // a rejected load leaves the relation empty
+      drop_current(R); R.fact_keys.reset(); R.fact_tags.reset(); R.n = R.n_facts = 0;
+      for (int i = 0; i < kMaxArity; ++i) R.col_max[i] = 0;
+      R.layout = make_layout(R.arity, R.col_max); R.key_bytes = 4;
+      throw;
+    }
+  });
+}
+
+xlog_status xlog_relation_size(xlog_ctx* c, xlog_rel rel, int64_t* n) {
+  return guarded(c, [&] {
+    Relation& R = rel_of(c, rel);
+    if (!n) fail(XLOG_ERR_INVALID_ARGUMENT, "n is NULL");
+    if (R.is_head && c->poisoned) fail(XLOG_ERR_INVALID_STATE, "derived relations are poisoned");
+    if (R.is_head && c->idb_dirty) { reset_idb(c); c->idb_dirty = false; }
+    *n = R.n;
+  });
+}
+
+xlog_status xlog_relation_view(xlog_ctx* c, xlog_rel rel, const int32_t** cols, const float** tags, int64_t* n) {
+  return guarded(c, [&] {
+    Relation& R = rel_of(c, rel);
+    if (R.is_head && c->poisoned) fail(XLOG_ERR_INVALID_STATE, "derived relations are poisoned");
+    if (R.is_head && c->idb_dirty) { reset_idb(c); c->idb_dirty = false; }
+    ensure_soa(c, R);
+    XLOG_CUDA(cudaStreamSynchronize(c->stream));
+    if (cols) for (int i = 0; i < R.arity; ++i) cols[i] = R.cols[i].as<int32_t>();
+    if (tags) *tags = R.tags();
+    if (n) *n = R.n;
+  });
+}
+
+xlog_status xlog_relation_read(xlog_ctx* c, xlog_rel rel, int32_t* const* cols_out, float* tags_out, int64_t capacity, int64_t* n_out,
+                               xlog_memspace space) {
+  return guarded(c, [&] {
+    Relation& R = rel_of(c, rel);
+    if (R.is_head && c->poisoned) fail(XLOG_ERR_INVALID_STATE, "derived relations are poisoned");
+    if (R.is_head && c->idb_dirty) { reset_idb(c); c->idb_dirty = false; }
+    if ((int64_t)R.n > capacity) { if (n_out) *n_out = R.n; fail(XLOG_ERR_BUFFER_TOO_SMALL, "capacity smaller than the relation"); }
+    ensure_soa(c, R);
+    const cudaMemcpyKind kind = space == XLOG_MEM_HOST ? cudaMemcpyDeviceToHost : cudaMemcpyDeviceToDevice;
+    if (R.n) {
+      if (cols_out) for (int i = 0; i < R.arity; ++i) if (cols_out[i]) XLOG_CUDA(cudaMemcpyAsync(cols_out[i], R.cols[i].p, (size_t)R.n * 4, kind, c->stream));
+      if (tags_out) XLOG_CUDA(cudaMemcpyAsync(tags_out, R.tags(), (size_t)R.n * 4, kind, c->stream));
+    }
+    XLOG_CUDA(cudaStreamSynchronize(c->stream));
+    if (space == XLOG_MEM_HOST) c->d2h_bytes += (int64_t)R.n * 4 * (R.arity + 1);
+    if (n_out) *n_out = R.n;
+  });
+}
+
+xlog_status xlog_rule_add(xlog_ctx* c, const xlog_plan* plan, xlog_rule* out) {
+  return guarded(c, [&] { add_rule(c, plan, out); });
+}
+
+xlog_status xlog_ctx_reset_idb(xlog_ctx* c) {
+  return guarded(c, [&] { XLOG_CUDA(cudaStreamSynchronize(c->stream)); reset_idb(c); c->idb_dirty = false; });
+}
+
+xlog_status xlog_fixpoint(xlog_ctx* c, xlog_receipt* receipt) {
+  if (!c) return XLOG_ERR_INVALID_ARGUMENT;
+  if (receipt && receipt->struct_size != sizeof(xlog_receipt)) return XLOG_ERR_INVALID_ARGUMENT;
+  const int64_t l0 = c->launches, d0 = c->d2h_bytes, h0 = c->h2d_bytes;
+  c->r_candidates = c->r_unique = c->r_new = c->r_improved = c->r_iterations = c->r_strata = 0;
+  c->arena.reset_peak();
+  cudaSetDevice(c->device);
+  cudaEventRecord(c->ev0, c->stream);
+  xlog_status st = guarded(c, [&] { run_fixpoint(c); });
+  cudaEventRecord(c->ev1, c->stream);
+  cudaEventSynchronize(c->ev1);
+  if (st != XLOG_OK) {
+    // leave no work in flight and no error flag behind; the derived relations stay poisoned
+    cudaStreamSynchronize(c->stream);
+    cudaMemsetAsync(c->d_ctrl, 0, kCtrlSlots * sizeof(uint64_t), c->stream);
+    cudaStreamSynchronize(c->stream);
+  }
+  if (receipt) {
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, c->ev0, c->ev1);
+    receipt->status = st;
+    receipt->strata = c->r_strata;
+    receipt->iterations = c->r_iterations;
+    int64_t derived = 0;
+    if (st == XLOG_OK) for (Relation* R : c->rels) if (R->is_head) derived += (int64_t)R->n - R->n_facts;
+    receipt->derived_tuples = derived;
+    receipt->candidates = c->r_candidates;
+    receipt->unique_candidates = c->r_unique;
+    receipt->new_tuples = c->r_new;
+    receipt->improved_tags = c->r_improved;
+    receipt->h2d_bytes = c->h2d_bytes - h0;
+    receipt->d2h_bytes = c->d2h_bytes - d0;
+    receipt->kernel_launches = c->launches - l0;
+    receipt->peak_arena_bytes = (int64_t)c->arena.peak();
+    receipt->device_ms = ms;
+  }
+  return st;
+}
+
+xlog_status xlog_rule_backward(xlog_ctx* c, xlog_rule rule, const float* grad_head, float* const* grad_atoms) {
+  return guarded(c, [&] {
+    if (rule < 0 || rule >= (int)c->rules.size()) fail(XLOG_ERR_INVALID_ARGUMENT, "bad rule handle");
+    if (!grad_head || !grad_atoms) fail(XLOG_ERR_INVALID_ARGUMENT, "NULL gradient pointer");
+    if (c->poisoned || !c->evaluated || c->idb_dirty) fail(XLOG_ERR_INVALID_STATE, "xlog_rule_backward needs a successful xlog_fixpoint first");
+    rule_backward(c, c->rules[rule], grad_head, grad_atoms);
+  });
+}
+
+}  // extern "C"

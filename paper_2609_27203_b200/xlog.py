@@ -1,0 +1,293 @@
+"""Thin ctypes binding over ``libxlog.so`` (the C ABI declared in ``include/xlog.h``).
+
+Argument marshalling only: every step of the fixpoint runs in the CUDA library.  PyTorch
+supplies device memory (the arena and any device-resident inputs) and the stream.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libxlog.so")
+
+MAX_ARITY, MAX_ATOMS, MAX_VARS = 4, 3, 8
+SEMIRING = {"maxplus": 0, "minplus": 1, "logsumexp": 2, "sumprod": 3}
+STATUS = ["OK", "INVALID_ARGUMENT", "INVALID_VALUE", "UNSUPPORTED", "RESOURCE_EXHAUSTED", "CAPACITY_EXCEEDED",
+          "CONVERGENCE_FAILURE", "BUFFER_TOO_SMALL", "INVALID_STATE", "CUDA", "INTERNAL"]
+MEM_HOST, MEM_DEVICE = 0, 1
+FLAG_CHECK_INVARIANTS = 1
+
+EXPORTS = ["xlog_ctx_create", "xlog_ctx_destroy", "xlog_last_error", "xlog_relation_create", "xlog_relation_load",
+           "xlog_relation_size", "xlog_relation_read", "xlog_relation_view", "xlog_rule_add", "xlog_fixpoint",
+           "xlog_ctx_reset_idb", "xlog_rule_backward"]
+
+
+class XlogError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        self.code = code
+        self.status = STATUS[code] if 0 <= code < len(STATUS) else str(code)
+        super().__init__(f"{self.status}: {msg}")
+
+
+class Config(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("device", C.c_int32), ("stream", C.c_void_p), ("arena", C.c_void_p),
+                ("arena_bytes", C.c_uint64), ("max_iterations", C.c_int64), ("candidate_chunk_bytes", C.c_uint64),
+                ("flags", C.c_uint32)]
+
+
+class Arg(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("var", C.c_int32), ("mul", C.c_int32), ("add", C.c_int32)]
+
+
+class AtomS(C.Structure):
+    _fields_ = [("rel", C.c_int32), ("args", Arg * MAX_ARITY)]
+
+
+class Expr(C.Structure):
+    _fields_ = [("c0", C.c_int64), ("coef", C.c_int32 * MAX_VARS)]
+
+
+class Plan(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("head_rel", C.c_int32), ("n_head_cols", C.c_int32),
+                ("head", Expr * MAX_ARITY), ("n_atoms", C.c_int32), ("atoms", AtomS * MAX_ATOMS),
+                ("emit_count_column", C.c_int32)]
+
+
+class Receipt(C.Structure):
+    _fields_ = [("struct_size", C.c_uint32), ("status", C.c_int32), ("strata", C.c_int64), ("iterations", C.c_int64),
+                ("derived_tuples", C.c_int64), ("candidates", C.c_int64), ("unique_candidates", C.c_int64),
+                ("new_tuples", C.c_int64), ("improved_tags", C.c_int64), ("h2d_bytes", C.c_int64),
+                ("d2h_bytes", C.c_int64), ("kernel_launches", C.c_int64), ("peak_arena_bytes", C.c_int64),
+                ("device_ms", C.c_double)]
+
+    def as_dict(self) -> Dict[str, object]:
+        return {k: getattr(self, k) for k, _ in self._fields_ if k != "struct_size"}
+
+
+_lib = None
+
+
+def lib():
+    """Load the CUDA library; its absence is an error (there is no fallback path)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2609_27203_b200.build`")
+        L = C.CDLL(_LIB_PATH)
+        vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+        L.xlog_ctx_create.argtypes = [C.POINTER(Config), C.POINTER(vp)]
+        L.xlog_ctx_destroy.argtypes = [vp]
+        L.xlog_last_error.argtypes = [vp]
+        L.xlog_last_error.restype = C.c_char_p
+        L.xlog_relation_create.argtypes = [vp, i32, i32, C.c_char_p, C.POINTER(i32)]
+        L.xlog_relation_load.argtypes = [vp, i32, C.POINTER(vp), vp, i64, i32]
+        L.xlog_relation_size.argtypes = [vp, i32, C.POINTER(i64)]
+        L.xlog_relation_read.argtypes = [vp, i32, C.POINTER(vp), vp, i64, C.POINTER(i64), i32]
+        L.xlog_relation_view.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(i64)]
+        L.xlog_rule_add.argtypes = [vp, C.POINTER(Plan), C.POINTER(i32)]
+        L.xlog_fixpoint.argtypes = [vp, C.POINTER(Receipt)]
+        L.xlog_ctx_reset_idb.argtypes = [vp]
+        L.xlog_rule_backward.argtypes = [vp, i32, vp, C.POINTER(vp)]
+        for name in EXPORTS:
+            if name != "xlog_last_error":
+                getattr(L, name).restype = C.c_int
+        _lib = L
+    return _lib
+
+
+class Context:
+    """One engine context over a caller-owned device arena (a torch uint8 CUDA tensor)."""
+
+    def __init__(self, arena_bytes: int = 1 << 30, device: int = 0, max_iterations: int = 0,
+                 candidate_chunk_bytes: int = 0, flags: int = 0, stream=None):
+        import torch
+        if not torch.cuda.is_available():
+            raise RuntimeError("paper_2609_27203_b200 needs a CUDA device; there is no CPU path")
+        self._L = lib()
+        self._torch = torch
+        self.device = device
+        torch.cuda.set_device(device)
+        self._arena = torch.empty(arena_bytes, dtype=torch.uint8, device=f"cuda:{device}")
+        self._stream = stream if stream is not None else torch.cuda.current_stream(device)
+        cfg = Config(C.sizeof(Config), device, self._stream.cuda_stream, self._arena.data_ptr(), arena_bytes,
+                     max_iterations, candidate_chunk_bytes, flags)
+        h = C.c_void_p()
+        st = self._L.xlog_ctx_create(C.byref(cfg), C.byref(h))
+        if st:
+            raise XlogError(st, "xlog_ctx_create failed")
+        self._h = h
+        self._arity: List[int] = []
+        self._rule_atoms: List[List[int]] = []
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._L.xlog_ctx_destroy(self._h)
+            self._h = None
+            self._arena = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, st: int):
+        if st:
+            raise XlogError(st, (self._L.xlog_last_error(self._h) or b"").decode())
+
+    # ---- relations ----
+    def relation(self, arity: int, semiring: str, name: str = "") -> int:
+        out = C.c_int32()
+        self._check(self._L.xlog_relation_create(self._h, arity, SEMIRING[semiring], name.encode(), C.byref(out)))
+        self._arity.append(arity)
+        return out.value
+
+    def load(self, rel: int, cols: Sequence, tags=None):
+        """cols/tags: numpy arrays (host) or torch CUDA tensors (device), int32 / float32."""
+        torch = self._torch
+        k = self._arity[rel]
+        assert len(cols) == k
+        on_device = isinstance(cols[0], torch.Tensor)
+        keep = []
+        ptrs = (C.c_void_p * k)()
+        if on_device:
+            for i, c in enumerate(cols):
+                c = c.to(torch.int32).contiguous()
+                keep.append(c)
+                ptrs[i] = c.data_ptr()
+            n = int(cols[0].numel())
+            tp = None
+            if tags is not None:
+                t = tags.to(torch.float32).contiguous()
+                keep.append(t)
+                tp = t.data_ptr()
+        else:
+            for i, c in enumerate(cols):
+                c = np.ascontiguousarray(c, np.int32)
+                keep.append(c)
+                ptrs[i] = c.ctypes.data
+            n = len(keep[0])
+            tp = None
+            if tags is not None:
+                t = np.ascontiguousarray(tags, np.float32)
+                keep.append(t)
+                tp = t.ctypes.data
+        self._check(self._L.xlog_relation_load(self._h, rel, ptrs, tp, n, MEM_DEVICE if on_device else MEM_HOST))
+
+    def size(self, rel: int) -> int:
+        n = C.c_int64()
+        self._check(self._L.xlog_relation_size(self._h, rel, C.byref(n)))
+        return n.value
+
+    def read(self, rel: int):
+        """Host copy: ([col arrays], tags) in ascending lexicographic order."""
+        n, k = self.size(rel), self._arity[rel]
+        cols = [np.zeros(n, np.int32) for _ in range(k)]
+        tags = np.zeros(n, np.float32)
+        ptrs = (C.c_void_p * k)(*[c.ctypes.data for c in cols])
+        got = C.c_int64()
+        self._check(self._L.xlog_relation_read(self._h, rel, ptrs, tags.ctypes.data, n, C.byref(got), MEM_HOST))
+        assert got.value == n
+        return cols, tags
+
+    def read_device(self, rel: int):
+        torch = self._torch
+        n, k = self.size(rel), self._arity[rel]
+        cols = [torch.empty(n, dtype=torch.int32, device=f"cuda:{self.device}") for _ in range(k)]
+        tags = torch.empty(n, dtype=torch.float32, device=f"cuda:{self.device}")
+        ptrs = (C.c_void_p * k)(*[c.data_ptr() for c in cols])
+        got = C.c_int64()
+        self._check(self._L.xlog_relation_read(self._h, rel, ptrs, tags.data_ptr(), n, C.byref(got), MEM_DEVICE))
+        return cols, tags
+
+    def view(self, rel: int):
+        """Borrowed device pointers (ints) to the stored columns and tags, and the row count."""
+        k = self._arity[rel]
+        ptrs = (C.c_void_p * k)()
+        tp = C.c_void_p()
+        n = C.c_int64()
+        self._check(self._L.xlog_relation_view(self._h, rel, ptrs, C.byref(tp), C.byref(n)))
+        return [int(p or 0) for p in ptrs], int(tp.value or 0), n.value
+
+    # ---- rules ----
+    def rule(self, head: int, head_exprs, atoms, emit_count: bool = False) -> int:
+        """head_exprs: [(c0, {var: coef})]; atoms: [(rel, [("c", value) | ("v", var, mul, add)])]."""
+        p = Plan()
+        p.struct_size = C.sizeof(Plan)
+        p.head_rel = head
+        p.n_head_cols = len(head_exprs)
+        for i, (c0, coef) in enumerate(head_exprs):
+            p.head[i].c0 = c0
+            for v, kf in dict(coef).items():
+                p.head[i].coef[v] = kf
+        p.n_atoms = len(atoms)
+        for j, (rel, al) in enumerate(atoms):
+            p.atoms[j].rel = rel
+            for c, a in enumerate(al):
+                if a[0] == "c":
+                    p.atoms[j].args[c] = Arg(0, 0, 1, a[1])
+                else:
+                    p.atoms[j].args[c] = Arg(1, a[1], a[2], a[3])
+        p.emit_count_column = int(emit_count)
+        out = C.c_int32()
+        self._check(self._L.xlog_rule_add(self._h, C.byref(p), C.byref(out)))
+        self._rule_atoms.append([rel for rel, _ in atoms])
+        return out.value
+
+    # ---- evaluation ----
+    def fixpoint(self) -> Dict[str, object]:
+        r = Receipt()
+        r.struct_size = C.sizeof(Receipt)
+        st = self._L.xlog_fixpoint(self._h, C.byref(r))
+        self.last_receipt = r.as_dict()
+        self._check(st)
+        return self.last_receipt
+
+    def reset_idb(self):
+        self._check(self._L.xlog_ctx_reset_idb(self._h))
+
+    def backward(self, rule: int, grad_head, same_buffer_for_same_relation: bool = True):
+        """grad_head: torch CUDA float32 tensor over head rows.  Returns one torch tensor per atom
+        (atoms naming the same relation share one tensor, which then holds the sum)."""
+        torch = self._torch
+        g = grad_head.to(torch.float32).contiguous()
+        rels = self._rule_atoms[rule]
+        bufs: Dict[int, object] = {}
+        outs = []
+        for j, r in enumerate(rels):
+            key = r if same_buffer_for_same_relation else (r, j)
+            if key not in bufs:
+                bufs[key] = torch.empty(self.size(r), dtype=torch.float32, device=f"cuda:{self.device}")
+            outs.append(bufs[key])
+        ptrs = (C.c_void_p * len(outs))(*[o.data_ptr() for o in outs])
+        self._check(self._L.xlog_rule_backward(self._h, rule, g.data_ptr(), ptrs))
+        return outs
+
+
+def load_program(program, ctx: Optional[Context] = None, device_inputs: bool = False, **ctx_kw):
+    """Instantiate a ``workloads.Program`` on a context.  Returns (ctx, relation ids, rule ids)."""
+    if ctx is None:
+        ctx = Context(**ctx_kw)
+    ids = {name: ctx.relation(ar, sr, name) for name, (ar, sr) in program.relations.items()}
+    for name, (cols, tags) in program.facts.items():
+        if device_inputs:
+            import torch
+            dev = f"cuda:{ctx.device}"
+            cols = [torch.from_numpy(np.ascontiguousarray(c, np.int32)).to(dev) for c in cols]
+            tags = None if tags is None else torch.from_numpy(np.ascontiguousarray(tags, np.float32)).to(dev)
+        ctx.load(ids[name], cols, tags)
+    rule_ids = []
+    for r in program.rules:
+        he = [(e.c0, dict(e.coef)) for e in r.head_exprs]
+        atoms = []
+        for a in r.atoms:
+            al = []
+            for g in a.args:
+                al.append(("c", g.value) if hasattr(g, "value") else ("v", g.var, g.mul, g.add))
+            atoms.append((ids[a.rel], al))
+        rule_ids.append(ctx.rule(ids[r.head], he, atoms, r.emit_count))
+    return ctx, ids, rule_ids

@@ -1,0 +1,245 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element.
+
+Tolerances (from the benchmark spec): tuple sets bit-exact; max-plus / min-plus tags 1e-5
+relative (expected and reported: bit-equal); logsumexp tags 1e-4 absolute; counts exact.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_27203_b200 import synth, workloads as W
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+MINMAX_REL = 1e-5
+LSE_ABS = 1e-4
+
+
+def gpu_run(program, **kw):
+    from paper_2609_27203_b200 import xlog
+    kw.setdefault("arena_bytes", 1 << 28)
+    kw.setdefault("flags", xlog.FLAG_CHECK_INVARIANTS)
+    ctx, ids, rules = xlog.load_program(program, **kw)
+    receipt = ctx.fixpoint()
+    return ctx, ids, rules, receipt
+
+
+def oracle_run(program, mode="seminaive"):
+    o, ids, rules = oracle.load_program(program)
+    stats = o.run(mode)
+    return o, ids, rules, stats
+
+
+def check_program(program, rel_tol=MINMAX_REL, abs_tol=0.0, expect_bit_equal=True, mode="seminaive", **kw):
+    ctx, gids, _, receipt = gpu_run(program, **kw)
+    o, oids, _, stats = oracle_run(program, mode)
+    for name in program.outputs:
+        rep = H.compare_relations(ctx.read(gids[name]), o.read(oids[name]), rel_tol=rel_tol, abs_tol=abs_tol,
+                                  what=f"{program.name}:{name}")
+        if expect_bit_equal:
+            assert rep["bit_unequal"] == 0, rep
+    assert receipt["derived_tuples"] == stats["derived_tuples"]
+    ctx.close()
+    return receipt, stats
+
+
+# ---- relation store: load / read ---------------------------------------------------------
+
+@pytest.mark.parametrize("n,arity,sr", [(1, 1, "maxplus"), (7, 2, "minplus"), (5000, 2, "maxplus"),
+                                        (100_003, 2, "minplus"), (30_000, 3, "logsumexp"), (20_000, 1, "sumprod")])
+def test_load_sorts_and_combines_duplicates(n, arity, sr):
+    from paper_2609_27203_b200 import xlog
+    hi = [50, 300, 7, 5][:arity] if n > 10 else [3, 3, 3, 3][:arity]        # small domains force duplicates
+    cols = [synth.randint(9, 20 + c, 0, n, hi[c]).astype(np.int32) for c in range(arity)]
+    tags = (synth.normal(9, 30, n)).astype(np.float32)
+    if sr == "sumprod":
+        tags = np.abs(tags) + 0.5
+    ctx = xlog.Context(arena_bytes=1 << 27, flags=xlog.FLAG_CHECK_INVARIANTS)
+    r = ctx.relation(arity, sr)
+    ctx.load(r, cols, tags)
+    o = oracle.Oracle()
+    ro = o.relation(arity, sr)
+    o.load(ro, cols, tags)
+    tol = dict(rel_tol=0, abs_tol=0) if sr in ("maxplus", "minplus") else dict(rel_tol=1e-5, abs_tol=LSE_ABS)
+    rep = H.compare_relations(ctx.read(r), o.read(ro), what="load", **tol)
+    if sr in ("maxplus", "minplus"):
+        assert rep["bit_unequal"] == 0
+    # device-resident input gives the same relation
+    import torch
+    ctx.load(r, [torch.from_numpy(c).cuda() for c in cols], torch.from_numpy(tags).cuda())
+    H.compare_relations(ctx.read(r), o.read(ro), what="load(device)", **tol)
+    dc, dt = ctx.read_device(r)
+    assert np.array_equal(dt.cpu().numpy(), ctx.read(r)[1])
+    ctx.close()
+
+
+def test_empty_and_single_relations():
+    from paper_2609_27203_b200 import xlog
+    ctx = xlog.Context(arena_bytes=1 << 24)
+    r = ctx.relation(2, "maxplus")
+    assert ctx.size(r) == 0
+    ctx.load(r, [np.zeros(0, np.int32), np.zeros(0, np.int32)], np.zeros(0, np.float32))
+    assert ctx.size(r) == 0 and len(ctx.read(r)[1]) == 0
+    ctx.load(r, [np.array([5], np.int32), np.array([9], np.int32)], None)
+    cols, tags = ctx.read(r)
+    assert cols[0].tolist() == [5] and cols[1].tolist() == [9] and tags.tolist() == [0.0]
+    ctx.close()
+
+
+def test_wide_keys_use_64_bit_packing():
+    # two 31-bit columns: 62 key bits
+    from paper_2609_27203_b200 import xlog
+    n = 20_000
+    a = synth.randint(3, 1, 0, n, (1 << 31) - 1).astype(np.int32)
+    b = synth.randint(3, 2, 0, n, (1 << 31) - 1).astype(np.int32)
+    a[:100] = a[100:200]                                 # some equal leading columns
+    t = synth.normal(3, 3, n).astype(np.float32)
+    ctx = xlog.Context(arena_bytes=1 << 26, flags=xlog.FLAG_CHECK_INVARIANTS)
+    r = ctx.relation(2, "maxplus")
+    ctx.load(r, [a, b], t)
+    o = oracle.Oracle()
+    ro = o.relation(2, "maxplus")
+    o.load(ro, [a, b], t)
+    assert H.compare_relations(ctx.read(r), o.read(ro))["bit_unequal"] == 0
+    ctx.close()
+
+
+# ---- golden cases ------------------------------------------------------------------------
+
+def test_golden_listing1_chain():
+    g = H.read_golden("listing1_chain_maxplus.txt")
+    e, c = g["edges"], g["closure"]
+    ctx, ids, _, rc = gpu_run(W.closure_program(e[:, 0], e[:, 1], e[:, 2]))
+    rep = H.compare_relations(ctx.read(ids["path"]), ([c[:, 0], c[:, 1]], c[:, 2]))
+    assert rep["bit_unequal"] == 0 and rc["derived_tuples"] == 6
+    ctx.close()
+
+
+def test_golden_diamond_and_cycle():
+    g = H.read_golden("diamond_sssp_minplus.txt")
+    e, d = g["edges"], g["dist"]
+    ctx, ids, _, rc = gpu_run(W.sssp_program(e[:, 0], e[:, 1], e[:, 2], 0))
+    assert H.compare_relations(ctx.read(ids["dist"]), ([d[:, 0]], d[:, 1]))["bit_unequal"] == 0
+    assert rc["improved_tags"] == 2 and rc["new_tuples"] == 3
+    ctx.close()
+    g = H.read_golden("cycle3_maxplus.txt")
+    e, c = g["edges"], g["closure"]
+    ctx, ids, _, _ = gpu_run(W.closure_program(e[:, 0], e[:, 1], e[:, 2]))
+    assert H.compare_relations(ctx.read(ids["path"]), ([c[:, 0], c[:, 1]], c[:, 2]))["bit_unequal"] == 0
+    ctx.close()
+
+
+# ---- recursive workloads -----------------------------------------------------------------
+
+@pytest.mark.parametrize("n,m", [(4, 5), (50, 120), (200, 800), (1000, 4000)])
+def test_closure_maxplus_ladder(n, m):
+    check_program(W.config1(n, m))
+
+
+def test_closure_adversarial_shapes():
+    # chain (maximal iteration count), star (one hub), one group holding every candidate
+    n = 300
+    check_program(W.closure_program(np.arange(n - 1), np.arange(1, n), synth.log_prob_tags(n - 1, 3)))
+    hub_out = W.closure_program(np.zeros(n - 1, np.int32), np.arange(1, n), synth.log_prob_tags(n - 1, 4))
+    check_program(hub_out)
+    src = np.concatenate([np.zeros(n - 1, np.int32), np.arange(1, n)])
+    dst = np.concatenate([np.arange(1, n), np.full(n - 1, n, np.int32)])      # 0 -> i -> n: n-1 candidates for (0, n)
+    check_program(W.closure_program(src, dst, synth.log_prob_tags(len(src), 5)))
+    # complete DAG with +1 weights under max-plus: j-i-1 successive improvements of one tuple
+    s, d = np.triu_indices(40, 1)
+    check_program(W.closure_program(s, d, np.ones(len(s), np.float32)))
+    # zero-improvement cycle
+    check_program(W.closure_program(np.arange(9), (np.arange(9) + 1) % 9, np.zeros(9, np.float32)))
+
+
+@pytest.mark.parametrize("scale", [8, 12, 16])
+def test_sssp_minplus_ladder(scale):
+    check_program(W.config2(scale=scale))
+
+
+@pytest.mark.parametrize("scale,ns", [(8, 4), (12, 64), (15, 64)])
+def test_multi_source_reach_ladder(scale, ns):
+    check_program(W.config5(scale=scale, n_sources=ns))
+
+
+def test_right_linear_rule_uses_a_transposed_index():
+    # path(x,z) :- edge(x,y), path(y,z): the delta sits on the second atom, edge is looked up by its second column
+    s, d = synth.uniform_digraph(120, 400, 21)
+    t = synth.log_prob_tags(400, 21)
+    prog = W.closure_program(s, d, t)
+    prog.rules[1] = W.Rule("path", (W.V(0), W.V(2)), (W.Atom("edge", (W.Var(0), W.Var(1))), W.Atom("path", (W.Var(1), W.Var(2)))))
+    # fl(w + t) == fl(t + w): still expected bit-equal for two-term products, but sums are folded from
+    # the other end of the path, so compare with tolerance only
+    check_program(prog, expect_bit_equal=False)
+
+
+def test_chunked_candidates_match_single_batch():
+    p = W.config1(300, 1500)
+    a, _ = check_program(p)
+    b, _ = check_program(p, candidate_chunk_bytes=64 << 10)
+    assert a["derived_tuples"] == b["derived_tuples"] and a["candidates"] == b["candidates"]
+    check_program(W.config2(scale=12), candidate_chunk_bytes=32 << 10)
+
+
+def test_fixpoint_idempotent_and_reset():
+    p = W.config1(200, 700)
+    ctx, ids, _, r1 = gpu_run(p)
+    first = ctx.read(ids["path"])
+    r2 = ctx.fixpoint()
+    assert r2["new_tuples"] == 0 and r2["improved_tags"] == 0
+    assert H.compare_relations(ctx.read(ids["path"]), first)["bit_unequal"] == 0
+    ctx.reset_idb()
+    assert ctx.size(ids["path"]) == 0
+    r3 = ctx.fixpoint()
+    assert r3["derived_tuples"] == r1["derived_tuples"]
+    assert H.compare_relations(ctx.read(ids["path"]), first)["bit_unequal"] == 0
+    ctx.close()
+
+
+def test_typed_failures_leave_the_context_usable():
+    from paper_2609_27203_b200 import xlog
+    chain = W.closure_program(np.arange(30), np.arange(1, 31), -np.ones(30, np.float32))
+    ctx, ids, _ = xlog.load_program(chain, arena_bytes=1 << 26, max_iterations=5)
+    with pytest.raises(xlog.XlogError) as e:
+        ctx.fixpoint()
+    assert e.value.status == "CONVERGENCE_FAILURE"
+    with pytest.raises(xlog.XlogError) as e:       # partial counters do not turn it into a result
+        ctx.read(ids["path"])
+    assert e.value.status == "INVALID_STATE"
+    ctx.reset_idb()
+    assert ctx.size(ids["path"]) == 0
+    ctx.close()
+    # arena too small for the closure
+    big = W.config1(400, 3000)
+    ctx, ids, _ = xlog.load_program(big, arena_bytes=1 << 19)
+    with pytest.raises(xlog.XlogError) as e:
+        ctx.fixpoint()
+    assert e.value.status == "RESOURCE_EXHAUSTED"
+    ctx.close()
+    # NaN tag, semiring zero, negative key
+    ctx = xlog.Context(arena_bytes=1 << 24)
+    r = ctx.relation(1, "minplus")
+    for cols, tags in [([np.array([1], np.int32)], np.array([np.nan], np.float32)),
+                       ([np.array([1], np.int32)], np.array([np.inf], np.float32)),
+                       ([np.array([-4], np.int32)], None)]:
+        with pytest.raises(xlog.XlogError) as e:
+            ctx.load(r, cols, tags)
+        assert e.value.status == "INVALID_VALUE"
+    ctx.load(r, [np.array([2], np.int32)], None)
+    assert ctx.size(r) == 1
+    # non-idempotent oplus in a recursive component
+    ctx2, _, _ = xlog.load_program(W.closure_program([0, 1], [1, 2], None, W.LOGSUMEXP), arena_bytes=1 << 24)
+    with pytest.raises(xlog.XlogError) as e:
+        ctx2.fixpoint()
+    assert e.value.status == "UNSUPPORTED"
+    # head arithmetic leaving [0, 2^31)
+    prog = W.Program("ovf", {"a": (1, W.MAXPLUS), "b": (1, W.MAXPLUS)},
+                     [W.Rule("b", (W.Affine(-5, ((0, 1),)),), (W.Atom("a", (W.Var(0),)),))],
+                     {"a": ([np.array([1, 9], np.int32)], None)})
+    ctx3, _, _ = xlog.load_program(prog, arena_bytes=1 << 24)
+    with pytest.raises(xlog.XlogError) as e:
+        ctx3.fixpoint()
+    assert e.value.status == "CAPACITY_EXCEEDED"
+    for c in (ctx, ctx2, ctx3):
+        c.close()
