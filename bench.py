@@ -1,0 +1,325 @@
+#!/usr/bin/env python
+"""Benchmark: derived tuples per second to fixpoint on one B200 (per GPU: independent replicas).
+
+A step is one whole fixpoint (all rounds of join / project / sort / reduce / diff-merge) over a
+seeded synthetic workload whose facts are already loaded and indexed on the device.  The default
+workload is the single-source min-plus shortest-path program on an R-MAT scale-20 graph.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload sssp|closure|reach|triangles|digits]
+  python bench.py --impl reference ...      # times the CPU oracle on the host cores instead
+
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "derived tuples/sec to fixpoint"
+UNIT = "tuples/s"
+
+# DRAM bytes per algorithmic byte of each kernel, from the ncu captures summarised under profiles/
+# (dram__bytes_read.sum + dram__bytes_write.sum over the launch's algorithmic bytes).  Used only to
+# scale a captured launch to the bench's launch size; None = not captured.
+NCU_TRAFFIC_RATIO = {}
+
+
+def make_program(name: str, scale: int | None):
+    from paper_2609_27203_b200 import workloads as W
+    if name == "sssp":
+        return W.config2(scale=scale or 20), 4 << 30
+    if name == "closure":
+        return W.config1(), 1 << 28
+    if name == "reach":
+        s = scale or 22
+        return W.config5(scale=s), (56 << 30) if s >= 21 else (8 << 30)
+    if name == "triangles":
+        return W.config3(scale=scale or 18), 2 << 30
+    if name == "digits":
+        return W.config4(), 1 << 30
+    raise SystemExit(f"unknown workload {name}")
+
+
+class ClockSampler:
+    """nvidia-smi clocks / throttle reasons sampled every 100 ms while a region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc, self.path = index, None, None
+
+    def __enter__(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.index)], stdout=open(self.path, "w"),
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+        return self
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        if not self.path or not os.path.exists(self.path):
+            return None
+        sm, mx, reasons = [], [], set()
+        for line in open(self.path):
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        os.unlink(self.path)
+        if not sm:
+            return None
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": max(mx), "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def measured_peak_gbs():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def reduce_max(values, world, backend_device=None):
+    """Element-wise max over ranks of a list of floats (torch.distributed when world > 1)."""
+    if world == 1:
+        return list(values)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(values, dtype=torch.float64, device=backend_device or "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t.cpu()]
+
+
+def run_oracle_once(program, mode="seminaive"):
+    import oracle
+    o, ids, _ = oracle.load_program(program)
+    t0 = time.perf_counter()
+    stats = o.run(mode)
+    return time.perf_counter() - t0, stats, o
+
+
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2609_27203_b200 import xlog
+
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    program, arena = make_program(args.workload, args.scale)
+
+    # facts resident in HBM before any timed region
+    ctx, ids, rules = xlog.load_program(program, device=local_rank, arena_bytes=arena, device_inputs=True)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)          # > 126 MB L2
+
+    def step(c):
+        c.reset_idb()
+        flush.fill_(1)                                                       # evict L2 between iterations
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        r = c.fixpoint()
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1), r
+
+    for _ in range(args.warmup):
+        step(ctx)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    times, launches, receipt = [], 0, None
+    with ClockSampler(local_rank) as clk:
+        for _ in range(args.steps):
+            ms, receipt = step(ctx)
+            times.append(ms)
+            launches += receipt["kernel_launches"]
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    total_ms = reduce_max([sum(times)], world, dev)[0]
+    ms_per_step = total_ms / args.steps
+    derived = receipt["derived_tuples"]
+    value = derived * world / (ms_per_step / 1e3)
+
+    # per-kernel timing: the same steps again with CUDA events around every launch
+    ctx.close()
+    pctx, pids, _ = xlog.load_program(program, device=local_rank, arena_bytes=arena, device_inputs=True,
+                                      flags=xlog.FLAG_PROFILE)
+    step(pctx)
+    pctx.profile_reset()
+    for _ in range(args.steps):
+        step(pctx)
+    prof = pctx.profile()
+    pctx.close()
+    ktot = sum(v["ms"] for v in prof.values()) or 1.0
+    dom = max((k for k in prof if prof[k]["bytes"] > 0), key=lambda k: prof[k]["ms"])
+    d = prof[dom]
+    peak, peak_src = measured_peak_gbs()
+    achieved = d["bytes"] / (d["ms"] / 1e3) / 1e9 if d["ms"] > 0 else 0.0
+    ratio = NCU_TRAFFIC_RATIO.get(dom)
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "peak_source": peak_src,
+                "traffic": None if ratio is None else ratio * d["bytes"] / d["launches"],
+                "algorithmic_bytes_per_launch": d["bytes"] / d["launches"], "launches_per_step": d["launches"] / args.steps,
+                "avg_launch_us": 1e3 * d["ms"] / d["launches"], "share_of_kernel_time": d["ms"] / ktot,
+                "kernels": {k: {"launches_per_step": v["launches"] / args.steps, "ms_per_step": v["ms"] / args.steps,
+                                "GBps": (v["bytes"] / (v["ms"] / 1e3) / 1e9) if v["ms"] > 0 and v["bytes"] else None}
+                            for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])},
+                "how": "second pass of the same steps with XLOG_FLAG_PROFILE (CUDA events around every launch on the ctx stream)"}
+
+    # end to end through the C ABI with HOST buffers: load (H2D + sort + index), fixpoint, read back (D2H)
+    pinned = {}
+    h2d = 0
+    for name, (cols, tags) in program.facts.items():
+        pc = [torch.from_numpy(np.ascontiguousarray(c, np.int32)).pin_memory() for c in cols]
+        pt = None if tags is None else torch.from_numpy(np.ascontiguousarray(tags, np.float32)).pin_memory()
+        pinned[name] = (pc, pt)
+        h2d += sum(c.numel() * 4 for c in pc) + (0 if pt is None else pt.numel() * 4)
+    empty = type(program)(program.name, program.relations, program.rules, {}, program.outputs)
+    ectx, eids, _ = xlog.load_program(empty, device=local_rank, arena_bytes=arena)
+
+    def e2e_step():
+        t0 = time.perf_counter()
+        for name, (pc, pt) in pinned.items():
+            ectx.load(eids[name], [c.numpy() for c in pc], None if pt is None else pt.numpy())
+        r = ectx.fixpoint()
+        d2h = 0
+        for name in program.outputs:
+            cols, tags = ectx.read(eids[name])
+            d2h += (len(cols) + 1) * 4 * len(tags)
+        torch.cuda.synchronize()
+        return (time.perf_counter() - t0) * 1e3, r, d2h
+
+    for _ in range(min(args.warmup, 2)):
+        e2e_step()
+    if world > 1:
+        dist.barrier()
+    e_times, d2h = [], 0
+    for _ in range(max(1, min(args.steps, 5))):
+        ms, r, d2h = e2e_step()
+        e_times.append(ms)
+    e_ms = reduce_max([sum(e_times) / len(e_times)], world, dev)[0]
+    ectx.close()
+    e2e = {"value": derived * world / (e_ms / 1e3), "unit": UNIT, "ms_per_step": e_ms, "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "how": "xlog_relation_load from pinned host + xlog_fixpoint + xlog_relation_read to host, wall clock"}
+
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+           "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32 keys / f32 tags",
+           "data": "synthetic", "impl": "ours",
+           "config": {"workload": program.name, "program": args.workload, **{k: v for k, v in program.info.items()},
+                      "derived_tuples": derived, "rounds": receipt["iterations"], "candidates": receipt["candidates"],
+                      "unique_candidates": receipt["unique_candidates"], "l2": "flushed between steps (256 MB fill)",
+                      "parallelism": "replicas only" if world > 1 else "1 gpu", "facts": "resident and indexed before timing"},
+           "clocks": clk.summary(), "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
+           "step_ms_min_med_max": [min(times), statistics.median(times), max(times)]}
+
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        # the oracle as it stands, on this machine's host cores, on a bounded sample of the same workload
+        sample, _ = make_program(args.workload, args.cpu_scale) if args.workload in ("sssp", "reach", "triangles") and args.cpu_scale else (program, 0)
+        sec, stats, _o = run_oracle_once(sample)
+        out["cpu_baseline"] = {"value": stats["derived_tuples"] / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
+                               "seconds": sec, "host_cores_available": os.cpu_count(),
+                               "sample": f"{sample.name}: one semi-naive fixpoint of the std::map oracle, single thread, facts pre-loaded"}
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+
+
+# ------------------------------------------------------------------------------------------------
+def run_reference(args):
+    """The oracle on the host cores, same metric; each step is one fixpoint of a bounded sample."""
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    est20 = {"sssp": 16.0, "reach": 600.0, "closure": 3.0, "triangles": 200.0, "digits": 10.0}[args.workload]
+    scale = args.scale
+    if args.workload in ("sssp", "reach", "triangles") and scale is None:
+        full = {"sssp": 20, "reach": 22, "triangles": 18}[args.workload]
+        scale = full
+        while scale > 8 and (args.steps + args.warmup) * est20 * 2.0 ** (scale - full) > 150.0:
+            scale -= 1
+    program, _ = make_program(args.workload, scale)
+    import oracle
+    o, ids, _ = oracle.load_program(program)
+    times, stats = [], None
+    for i in range(args.warmup + args.steps):
+        o.reset()
+        t0 = time.perf_counter()
+        stats = o.run("seminaive")
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            times.append(dt * 1e3)
+    ms = sum(times) / len(times)
+    value = stats["derived_tuples"] / (ms / 1e3)
+    sample = f"{program.name}: semi-naive fixpoint of the std::map oracle, single thread, facts pre-loaded"
+    print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+                      "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                      "dtype": "int32 keys / f32 tags", "data": "synthetic", "impl": "reference",
+                      "config": {"workload": program.name, "program": args.workload, **program.info,
+                                 "derived_tuples": stats["derived_tuples"]},
+                      "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+                      "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="sssp", choices=["sssp", "closure", "reach", "triangles", "digits"])
+    ap.add_argument("--scale", type=int, default=None, help="R-MAT scale override (smaller cases for profiling)")
+    ap.add_argument("--cpu-scale", type=int, default=None, help="R-MAT scale of the cpu_baseline sample (default: the workload's)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 0)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        if args.warmup < 3:
+            print("note: fewer than 3 warm-up steps requested", file=sys.stderr)
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

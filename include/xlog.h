@@ -73,6 +73,7 @@ typedef struct {
 } xlog_config;
 
 #define XLOG_FLAG_CHECK_INVARIANTS 1u  /* after every load/merge verify keys strictly increase (slow, for tests) */
+#define XLOG_FLAG_PROFILE          2u  /* CUDA events around every kernel launch; read with xlog_profile_read */
 
 /* ---- context --------------------------------------------------------------- */
 xlog_status xlog_ctx_create(const xlog_config* cfg, xlog_ctx** out);
@@ -173,6 +174,22 @@ xlog_status xlog_ctx_reset_idb(xlog_ctx* ctx);
  *   SUMPROD:    grad_j[row] += g[h] * prod_{i != j} tag_i
  * Passing the same pointer for two atoms of one relation yields the sum. */
 xlog_status xlog_rule_backward(xlog_ctx* ctx, xlog_rule rule, const float* grad_head, float* const* grad_atoms);
+
+/* ---- per-kernel statistics (Section "Semi-naive evaluation on GPU": the profiler records
+ * per-operator timing and row counts) ------------------------------------------------
+ * With XLOG_FLAG_PROFILE every kernel launch is bracketed by CUDA events on the context's
+ * stream.  xlog_profile_read waits for the stream, then writes one entry per kernel
+ * (accumulated since creation or the last reset): launches, summed device time, and the
+ * algorithmic bytes the launch sites declared (0 for helper kernels).  out may be NULL to
+ * query the count; at most `capacity` entries are written. */
+typedef struct {
+  char    name[48];
+  int64_t launches;
+  double  device_ms;
+  int64_t algorithmic_bytes;
+} xlog_kernel_stat;
+xlog_status xlog_profile_read(xlog_ctx* ctx, xlog_kernel_stat* out, int32_t capacity, int32_t* n_out);
+xlog_status xlog_profile_reset(xlog_ctx* ctx);
 
 #ifdef __cplusplus
 }

@@ -8,6 +8,7 @@
 #include <cstdio>
 #include <cstring>
 #include <functional>
+#include <map>
 #include <set>
 #include <string>
 #include <vector>
@@ -123,6 +124,14 @@ struct Ctx {
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   // receipt counters of the running fixpoint
   int64_t r_candidates = 0, r_unique = 0, r_new = 0, r_improved = 0, r_iterations = 0, r_strata = 0;
+  // optional per-kernel timing (XLOG_FLAG_PROFILE): CUDA events around every launch
+  struct ProfEntry { std::string name; int64_t launches = 0; double ms = 0; int64_t bytes = 0; };
+  struct ProfPending { int entry; cudaEvent_t a, b; };
+  std::vector<ProfEntry> prof;
+  std::map<std::string, int> prof_index;
+  std::vector<ProfPending> prof_pending;
+  std::vector<cudaEvent_t> ev_pool;
+  int64_t note_bytes = 0;                 // algorithmic bytes of the next launch (consumed by the launch macro)
 };
 
 inline DevBuf::DevBuf(Ctx* ctx, size_t n) : c(ctx), bytes(n) {
@@ -139,13 +148,49 @@ inline void DevBuf::reset() {
   p = nullptr; bytes = 0;
 }
 
+inline cudaEvent_t prof_event(Ctx* c) {
+  if (!c->ev_pool.empty()) { cudaEvent_t e = c->ev_pool.back(); c->ev_pool.pop_back(); return e; }
+  cudaEvent_t e = nullptr;
+  if (cudaEventCreate(&e) != cudaSuccess) fail(XLOG_ERR_CUDA, "cudaEventCreate");
+  return e;
+}
+inline void prof_begin(Ctx* c, const char* what) {
+  std::string name(what);
+  if (!name.empty() && name[0] == '(') name = name.substr(1);
+  name = name.substr(0, name.find_first_of("<)"));
+  auto it = c->prof_index.find(name);
+  if (it == c->prof_index.end()) {
+    it = c->prof_index.emplace(name, (int)c->prof.size()).first;
+    c->prof.push_back(Ctx::ProfEntry{name, 0, 0.0, 0});
+  }
+  Ctx::ProfPending p{it->second, prof_event(c), prof_event(c)};
+  cudaEventRecord(p.a, c->stream);
+  c->prof_pending.push_back(p);
+}
+// Fold finished launches into the table; call only when the stream is known to be idle.
+inline void prof_collect(Ctx* c) {
+  for (Ctx::ProfPending& p : c->prof_pending) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, p.a, p.b) == cudaSuccess) c->prof[p.entry].ms += ms;
+    c->ev_pool.push_back(p.a); c->ev_pool.push_back(p.b);
+  }
+  c->prof_pending.clear();
+}
 inline void check_launch(Ctx* c, const char* what) {
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) fail(XLOG_ERR_CUDA, std::string(what) + ": " + cudaGetErrorString(e));
   ++c->launches;
+  if (c->flags & XLOG_FLAG_PROFILE) {
+    Ctx::ProfPending& p = c->prof_pending.back();
+    cudaEventRecord(p.b, c->stream);
+    c->prof[p.entry].launches += 1;
+    c->prof[p.entry].bytes += c->note_bytes;
+  }
+  c->note_bytes = 0;
 }
 #define XLOG_LAUNCH(ctx, kern, grid, block, smem, ...)                   \
   do {                                                                   \
+    if ((ctx)->flags & XLOG_FLAG_PROFILE) prof_begin((ctx), #kern);      \
     kern<<<(grid), (block), (smem), (ctx)->stream>>>(__VA_ARGS__);       \
     check_launch((ctx), #kern);                                          \
   } while (0)
@@ -159,6 +204,7 @@ inline unsigned grid_for(uint64_t n, int block, int cap = kSMs * 16) {
 inline void sync_ctrl(Ctx* c) {
   XLOG_CUDA(cudaMemcpyAsync(c->h_ctrl, c->d_ctrl, kCtrlSlots * sizeof(uint64_t), cudaMemcpyDeviceToHost, c->stream));
   XLOG_CUDA(cudaStreamSynchronize(c->stream));
+  if (!c->prof_pending.empty()) prof_collect(c);
   c->d2h_bytes += kCtrlSlots * sizeof(uint64_t);
   const uint32_t e = (uint32_t)c->h_ctrl[kSlotErr];
   if (e) {
@@ -220,9 +266,11 @@ inline void sort_pairs(Ctx* c, K*& keys, float*& tags, K*& keys_alt, float*& tag
     const int nb = std::min(p.bits_per_pass, nbits - shift);
     if (nb <= 0) break;
     const int nbins = 1 << nb;
+    c->note_bytes = (int64_t)n * sizeof(K);
     XLOG_LAUNCH(c, (k_sort_hist<K>), (p.ntiles + kHistGroup - 1) / kHistGroup, kSortBlock, 0, keys, (uint32_t)n, shift, nbins,
                 p.ntiles, hist.as<uint32_t>());
     scan_exclusive_u32_inplace<uint32_t>(c, hist.as<uint32_t>(), (uint64_t)nbins * p.ntiles, spine.as<uint32_t>());
+    c->note_bytes = (int64_t)n * 2 * (sizeof(K) + 4);
     XLOG_LAUNCH(c, (k_sort_scatter<K>), p.ntiles, kSortBlock, sort_scatter_smem<K>(), keys,
                 reinterpret_cast<const uint32_t*>(tags), keys_alt, reinterpret_cast<uint32_t*>(tags_alt), (uint32_t)n, shift,
                 nbins, p.ntiles, hist.as<uint32_t>());
@@ -252,12 +300,14 @@ inline uint32_t reduce_by_key_t(Ctx* c, const K* keys, const float* tags, uint32
   typedef typename Op::A A;
   const unsigned tiles = (n + kRbkTile - 1) / kRbkTile;
   DevBuf heads(c, (size_t)tiles * 4), tails(c, (size_t)tiles * sizeof(A)), carry(c, (size_t)tiles * sizeof(A));
+  c->note_bytes = (int64_t)n * (sizeof(K) + 4);
   XLOG_LAUNCH(c, (k_rbk_tiles<K, Op>), tiles, kRbkBlock, 0, keys, tags, n, heads.as<uint32_t>(), tails.as<A>());
   XLOG_LAUNCH(c, (k_rbk_spine<Op>), 1, 1024, 0, heads.as<uint32_t>(), tails.as<A>(), carry.as<A>(), tiles, ctrl_u32(c, kSlotA));
   sync_ctrl(c);
   const uint32_t u = (uint32_t)c->h_ctrl[kSlotA];
   uint32_t* hp = nullptr;
   if (head_pos) { *head_pos = DevBuf(c, ((size_t)u + 1) * 4); hp = head_pos->as<uint32_t>(); }
+  c->note_bytes = ((int64_t)n + u) * (sizeof(K) + 4);
   XLOG_LAUNCH(c, (k_rbk_emit<K, Op>), tiles, kRbkBlock, 0, keys, tags, n, heads.as<uint32_t>(), carry.as<A>(), out_keys, out_tags, hp);
   if (hp) XLOG_CUDA(cudaMemcpyAsync(hp + u, &n, 4, cudaMemcpyHostToDevice, c->stream));
   XLOG_CUDA(cudaStreamSynchronize(c->stream));           // scratch is released on return
@@ -314,6 +364,7 @@ inline MergeResult merge_t(Ctx* c, const K* A, const float* TA, uint32_t na, con
   if (tiles == 0) return r;
   DevBuf a_start(c, ((size_t)tiles + 1) * 4), nf(c, (size_t)tiles * 4), nd(c, (size_t)tiles * 4);
   XLOG_LAUNCH(c, (k_merge_partition<K>), (tiles + 1 + 255) / 256, 256, 0, A, na, B, nb, tiles, a_start.as<uint32_t>());
+  c->note_bytes = (int64_t)total * (sizeof(K) + 4);
   XLOG_LAUNCH(c, (k_merge<K, Op, false>), tiles, kMrgBlock, 0, A, TA, na, B, TB, nb, a_start.as<uint32_t>(), nf.as<uint32_t>(),
               nd.as<uint32_t>(), (K*)nullptr, (float*)nullptr, (K*)nullptr, (float*)nullptr, 0);
   XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, nf.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotB));
@@ -333,6 +384,7 @@ inline MergeResult merge_t(Ctx* c, const K* A, const float* TA, uint32_t na, con
   r.delta.n = tot_d;
   r.delta.keys = DevBuf(c, (size_t)std::max(tot_d, 1u) * sizeof(K));
   r.delta.tags = DevBuf(c, (size_t)std::max(tot_d, 1u) * 4);
+  c->note_bytes = ((int64_t)total + (r.in_place ? 0 : tot_f) + tot_d) * (sizeof(K) + 4);
   XLOG_LAUNCH(c, (k_merge<K, Op, true>), tiles, kMrgBlock, 0, A, TA, na, B, TB, nb, a_start.as<uint32_t>(), nf.as<uint32_t>(),
               nd.as<uint32_t>(), r.full.keys.as<K>(), r.full.tags.as<float>(), r.delta.keys.as<K>(), r.delta.tags.as<float>(),
               r.in_place ? 1 : 0);

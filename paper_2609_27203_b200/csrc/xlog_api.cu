@@ -415,6 +415,8 @@ KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Sour
       const uint64_t take = std::min<uint64_t>(cap - fill, q.total - vpos);
       if (take) {
         const unsigned blocks = (unsigned)((take + kExpTile - 1) / kExpTile);
+        // per candidate: key + tag written, one inner column + inner tag read (outer rows amortise over the degree)
+        c->note_bytes = (int64_t)take * (ckb + 4 + (q.spec.has_inner ? 4 * (q.spec.inner_free + 1) : 0));
         if (q.outer.key_bytes == 4 && ckb == 4)
           XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint32_t>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.tags, q.outer.n,
                       (const uint64_t*)q.start.as<uint64_t>(), (const uint32_t*)q.first.as<uint32_t>(), vpos, vpos + take, k0.as<uint32_t>() + fill, t0.as<float>() + fill, ctrl_u32(c, kSlotErr));
@@ -726,6 +728,8 @@ xlog_status xlog_ctx_destroy(xlog_ctx* c) {
   if (c->h_ctrl) cudaFreeHost(c->h_ctrl);
   if (c->ev0) cudaEventDestroy(c->ev0);
   if (c->ev1) cudaEventDestroy(c->ev1);
+  for (auto& p : c->prof_pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
+  for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   delete c;
   return XLOG_OK;
 }
@@ -843,6 +847,30 @@ xlog_status xlog_fixpoint(xlog_ctx* c, xlog_receipt* receipt) {
     receipt->device_ms = ms;
   }
   return st;
+}
+
+xlog_status xlog_profile_read(xlog_ctx* c, xlog_kernel_stat* out, int32_t capacity, int32_t* n_out) {
+  return guarded(c, [&] {
+    XLOG_CUDA(cudaStreamSynchronize(c->stream));
+    prof_collect(c);
+    if (n_out) *n_out = (int32_t)c->prof.size();
+    if (!out) return;
+    for (int i = 0; i < (int)c->prof.size() && i < capacity; ++i) {
+      memset(&out[i], 0, sizeof(out[i]));
+      strncpy(out[i].name, c->prof[i].name.c_str(), sizeof(out[i].name) - 1);
+      out[i].launches = c->prof[i].launches;
+      out[i].device_ms = c->prof[i].ms;
+      out[i].algorithmic_bytes = c->prof[i].bytes;
+    }
+  });
+}
+
+xlog_status xlog_profile_reset(xlog_ctx* c) {
+  return guarded(c, [&] {
+    XLOG_CUDA(cudaStreamSynchronize(c->stream));
+    prof_collect(c);
+    c->prof.clear(); c->prof_index.clear();
+  });
 }
 
 xlog_status xlog_rule_backward(xlog_ctx* c, xlog_rule rule, const float* grad_head, float* const* grad_atoms) {

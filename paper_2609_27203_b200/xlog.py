@@ -20,10 +20,11 @@ STATUS = ["OK", "INVALID_ARGUMENT", "INVALID_VALUE", "UNSUPPORTED", "RESOURCE_EX
           "CONVERGENCE_FAILURE", "BUFFER_TOO_SMALL", "INVALID_STATE", "CUDA", "INTERNAL"]
 MEM_HOST, MEM_DEVICE = 0, 1
 FLAG_CHECK_INVARIANTS = 1
+FLAG_PROFILE = 2
 
 EXPORTS = ["xlog_ctx_create", "xlog_ctx_destroy", "xlog_last_error", "xlog_relation_create", "xlog_relation_load",
            "xlog_relation_size", "xlog_relation_read", "xlog_relation_view", "xlog_rule_add", "xlog_fixpoint",
-           "xlog_ctx_reset_idb", "xlog_rule_backward"]
+           "xlog_ctx_reset_idb", "xlog_rule_backward", "xlog_profile_read", "xlog_profile_reset"]
 
 
 class XlogError(RuntimeError):
@@ -68,6 +69,11 @@ class Receipt(C.Structure):
         return {k: getattr(self, k) for k, _ in self._fields_ if k != "struct_size"}
 
 
+class KernelStat(C.Structure):
+    _fields_ = [("name", C.c_char * 48), ("launches", C.c_int64), ("device_ms", C.c_double),
+                ("algorithmic_bytes", C.c_int64)]
+
+
 _lib = None
 
 
@@ -92,6 +98,8 @@ def lib():
         L.xlog_fixpoint.argtypes = [vp, C.POINTER(Receipt)]
         L.xlog_ctx_reset_idb.argtypes = [vp]
         L.xlog_rule_backward.argtypes = [vp, i32, vp, C.POINTER(vp)]
+        L.xlog_profile_read.argtypes = [vp, C.POINTER(KernelStat), i32, C.POINTER(i32)]
+        L.xlog_profile_reset.argtypes = [vp]
         for name in EXPORTS:
             if name != "xlog_last_error":
                 getattr(L, name).restype = C.c_int
@@ -246,6 +254,18 @@ class Context:
         self.last_receipt = r.as_dict()
         self._check(st)
         return self.last_receipt
+
+    def profile(self) -> Dict[str, Dict[str, float]]:
+        """Per-kernel launches / device ms / algorithmic bytes (needs FLAG_PROFILE)."""
+        n = C.c_int32()
+        self._check(self._L.xlog_profile_read(self._h, None, 0, C.byref(n)))
+        buf = (KernelStat * max(n.value, 1))()
+        self._check(self._L.xlog_profile_read(self._h, buf, n.value, C.byref(n)))
+        return {buf[i].name.decode(): dict(launches=buf[i].launches, ms=buf[i].device_ms, bytes=buf[i].algorithmic_bytes)
+                for i in range(n.value)}
+
+    def profile_reset(self):
+        self._check(self._L.xlog_profile_reset(self._h))
 
     def reset_idb(self):
         self._check(self._L.xlog_ctx_reset_idb(self._h))
