@@ -13,7 +13,7 @@ namespace xlog {
 struct ColPtrs { const int32_t* c[kMaxArity]; };
 struct ColPtrsMut { int32_t* c[kMaxArity]; };
 
-__global__ void __launch_bounds__(256) k_col_stats(ColPtrs cols, const float* __restrict__ tags, int64_t n, int arity, int sr,
+static __global__ void __launch_bounds__(256) k_col_stats(ColPtrs cols, const float* __restrict__ tags, int64_t n, int arity, int sr,
                                                    int32_t* __restrict__ col_max /*[arity]*/, uint32_t* __restrict__ err) {
   int32_t mx[kMaxArity] = {0, 0, 0, 0};
   uint32_t e = 0;
@@ -69,14 +69,14 @@ __global__ void __launch_bounds__(256) k_unpack(const K* __restrict__ keys, int6
 }
 
 // Permuted copy used to build an index on a non-leading column: out column j = in column perm[j].
-__global__ void __launch_bounds__(256) k_permute_cols(ColPtrs in, ColPtrsMut out, int64_t n, int arity, int p0, int p1, int p2, int p3) {
+static __global__ void __launch_bounds__(256) k_permute_cols(ColPtrs in, ColPtrsMut out, int64_t n, int arity, int p0, int p1, int p2, int p3) {
   const int perm[kMaxArity] = {p0, p1, p2, p3};
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
     for (int c = 0; c < arity; ++c) out.c[c][i] = in.c[perm[c]][i];
 }
 
 // off[v] = first row whose leading column is >= v, for v in [0, domain]  (off[domain] = n).
-__global__ void __launch_bounds__(256) k_build_offsets(const int32_t* __restrict__ lead, uint32_t n, int64_t domain,
+static __global__ void __launch_bounds__(256) k_build_offsets(const int32_t* __restrict__ lead, uint32_t n, int64_t domain,
                                                        uint32_t* __restrict__ off) {
   for (int64_t v = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; v <= domain; v += (int64_t)gridDim.x * blockDim.x) {
     uint32_t lo = 0, hi = n;
@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(256) k_check_sorted(const K* __restrict__ keys
 // count aggregate: group sizes from group-head positions, and the trailing count column
 // (paper Listing 7: count is a head column)
 // ---------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256) k_group_sizes(const uint32_t* __restrict__ head_pos, uint32_t u, uint32_t* __restrict__ counts,
+static __global__ void __launch_bounds__(256) k_group_sizes(const uint32_t* __restrict__ head_pos, uint32_t u, uint32_t* __restrict__ counts,
                                                      uint32_t* __restrict__ max_count) {
   uint32_t m = 0;
   for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < u; i += gridDim.x * blockDim.x) {
