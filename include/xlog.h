@@ -191,6 +191,33 @@ typedef struct {
 xlog_status xlog_profile_read(xlog_ctx* ctx, xlog_kernel_stat* out, int32_t capacity, int32_t* n_out);
 xlog_status xlog_profile_reset(xlog_ctx* ctx);
 
+/* ---- reduce-by-key that allocates nothing --------------------------------------------
+ * (The paper has no counterpart for this entry point.)
+ *
+ * For callers that cannot allocate device memory at call time: a serving loop whose memory
+ * was all handed out at start-up, a process whose device pool belongs to another component,
+ * or a stream that must not see the implicit synchronisation an allocation can cause.  It
+ * needs no context and no arena: the scratch of the segmented reduction lives in a fixed
+ * device array inside the library (about 164 KB, held by every GPU that loads the library
+ * until the process exits), which bounds the input at XLOG_STATIC_REDUCE_MAX_ROWS rows.
+ *
+ * Input: n rows with keys ascending (equal keys adjacent, keys >= 0) and their tags, both
+ * DEVICE pointers.  Output: one row per distinct key with the oplus of its tags under `sr`
+ * (same arithmetic as the engine's group-by), written to out_keys / out_tags (DEVICE, room
+ * for n rows; may not overlap the inputs); *n_out (HOST) receives the number of groups.
+ * errbuf (HOST, optional) receives a message on failure.
+ *
+ * Returns CAPACITY_EXCEEDED, touching nothing, when n > XLOG_STATIC_REDUCE_MAX_ROWS.
+ * Calls no cudaMalloc / cudaFree or other allocating routine.  Runs on `stream` of the
+ * CURRENT device and waits for it before returning.  The first call on each device also
+ * looks up the array's device address (once per device); make that first call before
+ * starting any stream capture.  All calls on a device share the one array, which keeps
+ * whatever the last call left there: each call overwrites every slot before reading it, but
+ * two calls whose kernels overlap on the GPU (different streams or threads) race. */
+#define XLOG_STATIC_REDUCE_MAX_ROWS (1 << 24)
+xlog_status xlog_reduce_by_key_static(void* stream, xlog_semiring sr, const int32_t* keys, const float* tags, int64_t n,
+                                      int32_t* out_keys, float* out_tags, int64_t* n_out, char* errbuf, size_t errbuf_len);
+
 #ifdef __cplusplus
 }
 #endif

@@ -24,7 +24,8 @@ FLAG_PROFILE = 2
 
 EXPORTS = ["xlog_ctx_create", "xlog_ctx_destroy", "xlog_last_error", "xlog_relation_create", "xlog_relation_load",
            "xlog_relation_size", "xlog_relation_read", "xlog_relation_view", "xlog_rule_add", "xlog_fixpoint",
-           "xlog_ctx_reset_idb", "xlog_rule_backward", "xlog_profile_read", "xlog_profile_reset"]
+           "xlog_ctx_reset_idb", "xlog_rule_backward", "xlog_profile_read", "xlog_profile_reset",
+           "xlog_reduce_by_key_static"]
 
 
 class XlogError(RuntimeError):
@@ -100,6 +101,7 @@ def lib():
         L.xlog_rule_backward.argtypes = [vp, i32, vp, C.POINTER(vp)]
         L.xlog_profile_read.argtypes = [vp, C.POINTER(KernelStat), i32, C.POINTER(i32)]
         L.xlog_profile_reset.argtypes = [vp]
+        L.xlog_reduce_by_key_static.argtypes = [vp, i32, vp, vp, i64, vp, vp, C.POINTER(i64), C.c_char_p, C.c_size_t]
         for name in EXPORTS:
             if name != "xlog_last_error":
                 getattr(L, name).restype = C.c_int
@@ -286,6 +288,25 @@ class Context:
         ptrs = (C.c_void_p * len(outs))(*[o.data_ptr() for o in outs])
         self._check(self._L.xlog_rule_backward(self._h, rule, g.data_ptr(), ptrs))
         return outs
+
+
+STATIC_REDUCE_MAX_ROWS = 1 << 24
+
+
+def reduce_by_key_static(semiring: str, keys, tags, out_keys, out_tags, stream=None) -> int:
+    """Reduce-by-key for callers that must not allocate device memory during the call (no context,
+    no arena: the library's own fixed scratch array is used).  keys (int32, ascending) / tags
+    (float32) and the two output tensors are torch CUDA tensors the caller already owns; returns the
+    number of groups written.  At most STATIC_REDUCE_MAX_ROWS rows."""
+    import torch
+    s = stream if stream is not None else torch.cuda.current_stream()
+    n_out = C.c_int64()
+    err = C.create_string_buffer(256)
+    st = lib().xlog_reduce_by_key_static(s.cuda_stream, SEMIRING[semiring], keys.data_ptr(), tags.data_ptr(), keys.numel(),
+                                         out_keys.data_ptr(), out_tags.data_ptr(), C.byref(n_out), err, len(err))
+    if st:
+        raise XlogError(st, err.value.decode())
+    return n_out.value
 
 
 def load_program(program, ctx: Optional[Context] = None, device_inputs: bool = False, **ctx_kw):
