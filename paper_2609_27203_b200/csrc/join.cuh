@@ -94,14 +94,28 @@ constexpr int kExpItems = 8;
 constexpr int kExpTile = kExpBlock * kExpItems;       // candidates per block
 constexpr int kExpRows = 2048;                        // outer-row starts staged in shared memory
 
+// Backward pass of a logsumexp / sum rule: instead of writing the candidate, look its head row up
+// and scatter the gradient to the two body rows (Section "End-to-end training": exact gradients
+// of a query value with respect to the weighted facts).
+struct BwdArgs {
+  const void* head_keys;        // stored head relation: packed keys (KH), ascending
+  const float* head_tags;       // its tags (the forward result)
+  uint32_t n_head;
+  int count_bits;               // a counted head stores (declared columns, count): compare keys >> count_bits
+  const float* grad_head;       // upstream gradient per head row
+  float* grad_outer;            // per row of the scanned atom's relation
+  float* grad_inner;            // per row of the looked-up atom's relation (NULL for one-atom rules)
+  int lse;                      // 1: logsumexp weights, 0: sum-product
+};
+
 // Block b writes candidates [out_lo + b*kExpTile, ...).  `start` is the exclusive scan of
 // `deg` (global candidate index of each outer row's first match).
-template <typename KO, typename KH>
+template <typename KO, typename KH, bool BWD>
 __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, const float* __restrict__ otags,
                                                            uint32_t n_outer, const uint64_t* __restrict__ start,
                                                            const uint32_t* __restrict__ first, uint64_t out_lo, uint64_t out_hi,
                                                            KH* __restrict__ ckeys, float* __restrict__ ctags,
-                                                           uint32_t* __restrict__ err) {
+                                                           uint32_t* __restrict__ err, BwdArgs bw) {
   __shared__ uint64_t sstart[kExpRows + 1];
   __shared__ uint32_t srow[2];
   const uint64_t t_lo = out_lo + (uint64_t)blockIdx.x * kExpTile;
@@ -138,8 +152,11 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
     int64_t var[kMaxVars];
     bind_outer<KO>(S, okeys[row], var);
     float tag = otags[row];
+    const float otag = tag;
+    float itag = S.times ? 1.f : 0.f;
+    uint32_t ir = 0;
     if (S.has_inner) {
-      const uint32_t ir = first[row] + j;
+      ir = first[row] + j;
 #pragma unroll
       for (int c = 0; c < kMaxArity - 1; ++c)
         if (c < S.inner_free) {
@@ -148,6 +165,7 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
           for (int v = 0; v < kMaxVars; ++v) if (v == S.inner_var[c]) var[v] = val;
         }
       const float it = S.inner_tag[ir];
+      itag = it;
       tag = S.times ? tag * it : tag + it;
     }
     KH key = 0;
@@ -160,8 +178,27 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
         if (h < 0 || h > (int64_t)S.head.mask[c]) { e |= kErrHeadRange; h = 0; }
         key |= (KH)(uint32_t)h << S.head.shift[c];
       }
-    ckeys[p - out_lo] = key;
-    ctags[p - out_lo] = tag;
+    if (!BWD) {
+      ckeys[p - out_lo] = key;
+      ctags[p - out_lo] = tag;
+    } else {
+      // head row of this binding: lower bound of the key among the stored head keys
+      const KH* hk = reinterpret_cast<const KH*>(bw.head_keys);
+      const KH want = key;
+      uint32_t a = 0, b = bw.n_head;
+      while (a < b) { const uint32_t mid = a + ((b - a) >> 1); if ((hk[mid] >> bw.count_bits) < want) a = mid + 1; else b = mid; }
+      if (a < bw.n_head && (hk[a] >> bw.count_bits) == want) {
+        const float g = bw.grad_head[a];
+        if (bw.lse) {
+          const float w = g * expf(tag - bw.head_tags[a]);
+          atomicAdd(&bw.grad_outer[row], w);
+          if (bw.grad_inner) atomicAdd(&bw.grad_inner[ir], w);
+        } else {
+          atomicAdd(&bw.grad_outer[row], g * itag);
+          if (bw.grad_inner) atomicAdd(&bw.grad_inner[ir], g * otag);
+        }
+      } else e |= kErrInternal;
+    }
   }
   if (e) atomicOr(err, e);
 }

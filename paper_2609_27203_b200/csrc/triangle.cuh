@@ -1,3 +1,114 @@
-// Fused triangle intersect-and-aggregate kernels (filled in below).
+// Fused directed-triangle aggregate  h(x, count) :- e(x,y), e(y,z), e(z,x)  (paper: "Worst-case-
+// optimal joins" and the fused triangle counting of "Head-to-head comparisons": triangles are
+// counted and their tags combined without ever materialising the tri relation).
+//
+// For every edge (x,y) the sorted out-list of y is intersected with the sorted in-list of x; each
+// common z contributes (w_xy otimes w_yz) otimes w_zx to x's group.  One warp per edge walks the
+// shorter list and binary-searches the longer one; per-edge partial aggregates are then combined
+// per x in a fixed order (edges of x are contiguous in the store), so results are reproducible.
 #pragma once
-#include "engine.cuh"
+#include "common.cuh"
+
+namespace xlog {
+
+struct TriGraph {
+  uint32_t n_edges;
+  const int32_t* src;            // column 0 of the store (ascending)
+  const int32_t* dst;            // column 1
+  const float* w;                // tags in stored order
+  int64_t out_domain, in_domain;
+  const uint32_t* out_off;       // offsets over src: out-list of v is dst[out_off[v] .. out_off[v+1])
+  const uint32_t* in_off;        // offsets over dst of the transposed copy
+  const int32_t* in_src;         // transposed copy: sources of the edges into v, ascending
+  const float* in_w;             // and their tags
+};
+
+template <typename Op>
+__global__ void __launch_bounds__(256) k_tri_edges(TriGraph G, int times, uint32_t* __restrict__ edge_cnt,
+                                                   typename Op::A* __restrict__ edge_acc) {
+  typedef typename Op::A A;
+  const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+  const unsigned lane = lane_id();
+  for (uint32_t e = warp; e < G.n_edges; e += nwarps) {
+    const int32_t x = G.src[e], y = G.dst[e];
+    const float wxy = G.w[e];
+    uint32_t a0 = 0, a1 = 0, b0 = 0, b1 = 0;
+    if (y < G.out_domain) { a0 = G.out_off[y]; a1 = G.out_off[y + 1]; }      // out(y): candidates z with e(y,z)
+    if (x < G.in_domain) { b0 = G.in_off[x]; b1 = G.in_off[x + 1]; }         // in(x):  candidates z with e(z,x)
+    const uint32_t la = a1 - a0, lb = b1 - b0;
+    uint32_t cnt = 0;
+    A acc = Op::identity();
+    if (la && lb) {
+      const bool walk_a = la <= lb;
+      const int32_t* wl = walk_a ? G.dst + a0 : G.in_src + b0;                // walked list
+      const int32_t* sl = walk_a ? G.in_src + b0 : G.dst + a0;                // searched list
+      const uint32_t nw = walk_a ? la : lb, ns = walk_a ? lb : la;
+      for (uint32_t i = lane; i < nw; i += 32) {
+        const int32_t z = wl[i];
+        uint32_t lo = 0, hi = ns;
+        while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (sl[mid] < z) lo = mid + 1; else hi = mid; }
+        if (lo < ns && sl[lo] == z) {
+          const float wyz = walk_a ? G.w[a0 + i] : G.w[a0 + lo];
+          const float wzx = walk_a ? G.in_w[b0 + lo] : G.in_w[b0 + i];
+          const float t = times ? (wxy * wyz) * wzx : (wxy + wyz) + wzx;
+          acc = Op::combine(acc, Op::lift(t));
+          ++cnt;
+        }
+      }
+    }
+#pragma unroll
+    for (int d = 16; d; d >>= 1) {
+      cnt += __shfl_down_sync(0xffffffffu, cnt, d);
+      const A o = shfl_down(acc, d);
+      acc = Op::combine(acc, o);
+    }
+    if (lane == 0) { edge_cnt[e] = cnt; edge_acc[e] = acc; }
+  }
+}
+
+// One warp per x: combine the partials of its edges (contiguous), write count, tag and a presence flag.
+template <typename Op>
+__global__ void __launch_bounds__(256) k_tri_groups(const uint32_t* __restrict__ out_off, int64_t domain,
+                                                    const uint32_t* __restrict__ edge_cnt, const typename Op::A* __restrict__ edge_acc,
+                                                    uint32_t* __restrict__ grp_cnt, float* __restrict__ grp_tag,
+                                                    uint32_t* __restrict__ flag, uint32_t* __restrict__ max_cnt,
+                                                    uint32_t* __restrict__ err) {
+  typedef typename Op::A A;
+  const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+  const unsigned lane = lane_id();
+  for (int64_t x = warp; x < domain; x += nwarps) {
+    const uint32_t e0 = out_off[x], e1 = out_off[x + 1];
+    uint64_t cnt = 0;
+    A acc = Op::identity();
+    for (uint32_t e = e0 + lane; e < e1; e += 32) {
+      cnt += edge_cnt[e];
+      acc = Op::combine(acc, edge_acc[e]);
+    }
+#pragma unroll
+    for (int d = 16; d; d >>= 1) {
+      cnt += __shfl_down_sync(0xffffffffu, cnt, d);
+      const A o = shfl_down(acc, d);
+      acc = Op::combine(acc, o);
+    }
+    if (lane == 0) {
+      if (cnt > 0x7fffffffull) { atomicOr(err, kErrCountOverflow); cnt = 0x7fffffffull; }
+      grp_cnt[x] = (uint32_t)cnt;
+      grp_tag[x] = cnt ? Op::lower(acc) : 0.f;
+      flag[x] = cnt ? 1u : 0u;
+      if (cnt) atomicMax(max_cnt, (uint32_t)cnt);
+    }
+  }
+}
+
+// Keep the x that have at least one triangle: pos = exclusive scan of flag.
+template <typename K>
+__global__ void __launch_bounds__(256) k_tri_compact(const uint32_t* __restrict__ flag, const uint32_t* __restrict__ pos, int64_t domain,
+                                                     const uint32_t* __restrict__ grp_cnt, const float* __restrict__ grp_tag,
+                                                     K* __restrict__ keys, uint32_t* __restrict__ counts, float* __restrict__ tags) {
+  for (int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; x < domain; x += (int64_t)gridDim.x * blockDim.x)
+    if (flag[x]) { const uint32_t p = pos[x]; keys[p] = (K)x; counts[p] = grp_cnt[x]; tags[p] = grp_tag[x]; }
+}
+
+}  // namespace xlog

@@ -1,7 +1,6 @@
 // C ABI of the engine (see include/xlog.h) and the host-side fixpoint driver.
 #include "engine.cuh"
 #include "triangle.cuh"
-#include "backward.cuh"
 
 using namespace xlog;
 
@@ -356,6 +355,40 @@ JoinSpec make_spec(Ctx* c, const Variant& v, const Relation& H) {
   return S;
 }
 
+// count -> scan for one variant; the grand total lands in control slot `slot` (read after sync_ctrl)
+void count_variant(Ctx* c, const Variant& v, const Relation& H, Counted& q, int slot) {
+  q.spec = make_spec(c, v, H);
+  q.outer = v.outer;
+  q.slot = slot;
+  const uint32_t n = v.outer.n;
+  const unsigned tiles = (n + kScanTile - 1) / kScanTile;
+  q.deg = DevBuf(c, (size_t)n * 4); q.first = DevBuf(c, (size_t)n * 4);
+  q.start = DevBuf(c, (size_t)n * 8); q.sums = DevBuf(c, (size_t)tiles * 8);
+  DISPATCH_K(v.outer.key_bytes, XLOG_LAUNCH(c, (k_join_count<K>), (n + 255) / 256, 256, 0, q.spec, (const K*)v.outer.keys, n,
+                                             q.deg.as<uint32_t>(), q.first.as<uint32_t>()));
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)q.deg.as<uint32_t>(), (int64_t)n, q.sums.as<uint64_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, q.sums.as<uint64_t>(), (int64_t)tiles, (uint64_t*)(c->d_ctrl + q.slot));
+  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)q.deg.as<uint32_t>(), (int64_t)n,
+              (const uint64_t*)q.sums.as<uint64_t>(), q.start.as<uint64_t>());
+}
+
+// materialise candidates [lo, hi) of a counted variant into (ckeys, ctags), or (bw != NULL) run the backward scatter
+template <bool BWD>
+void launch_expand(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, void* ckeys, float* ctags, const BwdArgs& bw) {
+  const unsigned blocks = (unsigned)((hi - lo + kExpTile - 1) / kExpTile);
+  const uint64_t* st = q.start.as<uint64_t>();
+  const uint32_t* fi = q.first.as<uint32_t>();
+  uint32_t* err = ctrl_u32(c, kSlotErr);
+  if (q.outer.key_bytes == 4 && ckb == 4)
+    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint32_t, BWD>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.tags, q.outer.n, st, fi, lo, hi, (uint32_t*)ckeys, ctags, err, bw);
+  else if (q.outer.key_bytes == 4)
+    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint64_t, BWD>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.tags, q.outer.n, st, fi, lo, hi, (uint64_t*)ckeys, ctags, err, bw);
+  else if (ckb == 4)
+    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint32_t, BWD>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.tags, q.outer.n, st, fi, lo, hi, (uint32_t*)ckeys, ctags, err, bw);
+  else
+    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint64_t, BWD>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.tags, q.outer.n, st, fi, lo, hi, (uint64_t*)ckeys, ctags, err, bw);
+}
+
 constexpr int kSlotTotals = 16;          // uint64 candidate totals of the variants of a round
 
 // Evaluate the variants, all deriving head relation H: join, project, sort, reduce by key.
@@ -372,19 +405,7 @@ KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Sour
     if (v.outer.n == 0) continue;
     counted.emplace_back();
     Counted& q = counted.back();
-    q.spec = make_spec(c, v, H);
-    q.outer = v.outer;
-    q.slot = kSlotTotals + (int)counted.size() - 1;
-    const uint32_t n = v.outer.n;
-    const unsigned tiles = (n + kScanTile - 1) / kScanTile;
-    q.deg = DevBuf(c, (size_t)n * 4); q.first = DevBuf(c, (size_t)n * 4);
-    q.start = DevBuf(c, (size_t)n * 8); q.sums = DevBuf(c, (size_t)tiles * 8);
-    DISPATCH_K(v.outer.key_bytes, XLOG_LAUNCH(c, (k_join_count<K>), (n + 255) / 256, 256, 0, q.spec, (const K*)v.outer.keys, n,
-                                               q.deg.as<uint32_t>(), q.first.as<uint32_t>()));
-    XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)q.deg.as<uint32_t>(), (int64_t)n, q.sums.as<uint64_t>());
-    XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, q.sums.as<uint64_t>(), (int64_t)tiles, (uint64_t*)(c->d_ctrl + q.slot));
-    XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)q.deg.as<uint32_t>(), (int64_t)n,
-                (const uint64_t*)q.sums.as<uint64_t>(), q.start.as<uint64_t>());
+    count_variant(c, v, H, q, kSlotTotals + (int)counted.size() - 1);
   }
   uint64_t total = extra ? extra->n : 0;
   if (!counted.empty()) {
@@ -414,21 +435,9 @@ KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Sour
       Counted& q = counted[vi];
       const uint64_t take = std::min<uint64_t>(cap - fill, q.total - vpos);
       if (take) {
-        const unsigned blocks = (unsigned)((take + kExpTile - 1) / kExpTile);
         // per candidate: key + tag written, one inner column + inner tag read (outer rows amortise over the degree)
         c->note_bytes = (int64_t)take * (ckb + 4 + (q.spec.has_inner ? 4 * (q.spec.inner_free + 1) : 0));
-        if (q.outer.key_bytes == 4 && ckb == 4)
-          XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint32_t>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.tags, q.outer.n,
-                      (const uint64_t*)q.start.as<uint64_t>(), (const uint32_t*)q.first.as<uint32_t>(), vpos, vpos + take, k0.as<uint32_t>() + fill, t0.as<float>() + fill, ctrl_u32(c, kSlotErr));
-        else if (q.outer.key_bytes == 4)
-          XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint64_t>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.tags, q.outer.n,
-                      (const uint64_t*)q.start.as<uint64_t>(), (const uint32_t*)q.first.as<uint32_t>(), vpos, vpos + take, k0.as<uint64_t>() + fill, t0.as<float>() + fill, ctrl_u32(c, kSlotErr));
-        else if (ckb == 4)
-          XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint32_t>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.tags, q.outer.n,
-                      (const uint64_t*)q.start.as<uint64_t>(), (const uint32_t*)q.first.as<uint32_t>(), vpos, vpos + take, k0.as<uint32_t>() + fill, t0.as<float>() + fill, ctrl_u32(c, kSlotErr));
-        else
-          XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint64_t>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.tags, q.outer.n,
-                      (const uint64_t*)q.start.as<uint64_t>(), (const uint32_t*)q.first.as<uint32_t>(), vpos, vpos + take, k0.as<uint64_t>() + fill, t0.as<float>() + fill, ctrl_u32(c, kSlotErr));
+        launch_expand<false>(c, q, vpos, vpos + take, ckb, (char*)k0.p + fill * ckb, t0.as<float>() + fill, BwdArgs{});
         fill += take; vpos += take;
       }
       if (vpos == q.total) { q.start.reset(); q.first.reset(); ++vi; vpos = 0; }
@@ -567,8 +576,102 @@ void append_count_column(Ctx* c, Relation& H, KeyTags& u, const KeyLayout& cl) {
   append_counts(c, H, u, cl, counts.as<uint32_t>(), (uint32_t)c->h_ctrl[kSlotD]);
 }
 
-void triangle_aggregate(Ctx* c, Relation& H, const RuleC& r) { (void)c; (void)H; (void)r; fail(XLOG_ERR_UNSUPPORTED, "triangle rule: not built yet"); }
-void rule_backward(Ctx* c, const RuleC& r, const float* g, float* const* grads) { (void)c; (void)r; (void)g; (void)grads; fail(XLOG_ERR_UNSUPPORTED, "backward: not built yet"); }
+// h(x[, count]) :- e(x,y), e(y,z), e(z,x): per-edge sorted-list intersection, then per-x combination.
+template <typename Op>
+void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
+  typedef typename Op::A A;
+  Relation& E = *c->rels[r.plan.atoms[0].rel];
+  const bool counted = r.plan.emit_count_column != 0;
+  int32_t mx[kMaxArity] = {H.col_max[0], 0, 0, 0};
+  const KeyLayout cl = make_layout(1, mx);
+  if (E.n == 0) { KeyTags empty; set_current(H, std::move(empty)); return; }
+  Index& out_ix = ensure_index(c, E, 0);
+  Index& in_ix = ensure_index(c, E, 1);
+  TriGraph G{};
+  G.n_edges = E.n;
+  G.src = E.cols[0].as<int32_t>(); G.dst = E.cols[1].as<int32_t>(); G.w = E.tags();
+  G.out_domain = out_ix.domain; G.in_domain = in_ix.domain;
+  G.out_off = out_ix.off.as<uint32_t>(); G.in_off = in_ix.off.as<uint32_t>();
+  G.in_src = in_ix.other[0]; G.in_w = in_ix.tags;
+  const int64_t domain = out_ix.domain;
+  DevBuf ecnt(c, (size_t)E.n * 4), eacc(c, (size_t)E.n * sizeof(A));
+  DevBuf gcnt(c, (size_t)domain * 4), gtag(c, (size_t)domain * 4), flag(c, (size_t)domain * 4);
+  const unsigned scan_tiles = (unsigned)((domain + kScanTile - 1) / kScanTile);
+  DevBuf spine(c, ((size_t)scan_tiles + 1) * 4);
+  zero_ctrl(c, kSlotA, 4);
+  XLOG_LAUNCH(c, (k_tri_edges<Op>), kSMs * 8, 256, 0, G, H.sr == XLOG_SR_SUMPROD ? 1 : 0, ecnt.as<uint32_t>(), eacc.as<A>());
+  XLOG_LAUNCH(c, (k_tri_groups<Op>), grid_for((uint64_t)domain * 32, 256, kSMs * 8), 256, 0, G.out_off, domain, (const uint32_t*)ecnt.as<uint32_t>(),
+              (const A*)eacc.as<A>(), gcnt.as<uint32_t>(), gtag.as<float>(), flag.as<uint32_t>(), ctrl_u32(c, kSlotD), ctrl_u32(c, kSlotErr));
+  // positions of the surviving x: exclusive scan of the flags (kept in a second buffer)
+  DevBuf pos(c, (size_t)domain * 4);
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), scan_tiles, kScanBlock, 0, (const uint32_t*)flag.as<uint32_t>(), domain, spine.as<uint32_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, spine.as<uint32_t>(), (int64_t)scan_tiles, ctrl_u32(c, kSlotA));
+  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), scan_tiles, kScanBlock, 0, (const uint32_t*)flag.as<uint32_t>(), domain,
+              (const uint32_t*)spine.as<uint32_t>(), pos.as<uint32_t>());
+  sync_ctrl(c);
+  const uint32_t u = (uint32_t)c->h_ctrl[kSlotA], max_count = (uint32_t)c->h_ctrl[kSlotD];
+  c->r_candidates += 0; c->r_unique += u;
+  KeyTags kt;
+  kt.n = u;
+  const int kb = cl.total_bits <= 32 ? 4 : 8;
+  kt.keys = DevBuf(c, (size_t)std::max(u, 1u) * kb);
+  kt.tags = DevBuf(c, (size_t)std::max(u, 1u) * 4);
+  DevBuf counts(c, (size_t)std::max(u, 1u) * 4);
+  DISPATCH_K(kb, XLOG_LAUNCH(c, (k_tri_compact<K>), grid_for(domain, 256), 256, 0, (const uint32_t*)flag.as<uint32_t>(), (const uint32_t*)pos.as<uint32_t>(), domain,
+                              (const uint32_t*)gcnt.as<uint32_t>(), (const float*)gtag.as<float>(), kt.keys.as<K>(), counts.as<uint32_t>(), kt.tags.as<float>()));
+  XLOG_CUDA(cudaStreamSynchronize(c->stream));
+  if (counted) append_counts(c, H, kt, cl, counts.as<uint32_t>(), max_count);
+  else set_current(H, std::move(kt));
+}
+
+void triangle_aggregate(Ctx* c, Relation& H, const RuleC& r) {
+  if (c->rels[r.plan.atoms[0].rel]->is_head && r.plan.atoms[0].rel == r.plan.head_rel) fail(XLOG_ERR_UNSUPPORTED, "recursive triangle rule");
+  switch (H.sr) {
+    case XLOG_SR_MAXPLUS: triangle_aggregate_t<OpMax>(c, H, r); break;
+    case XLOG_SR_MINPLUS: triangle_aggregate_t<OpMin>(c, H, r); break;
+    case XLOG_SR_LOGSUMEXP: triangle_aggregate_t<OpLse>(c, H, r); break;
+    default: triangle_aggregate_t<OpSum>(c, H, r); break;
+  }
+}
+
+// Gradient of a non-recursive logsumexp / sum rule with respect to its body tags: enumerate the
+// bindings again (count -> scan -> tiled walk) and scatter g[h] * weight to the body rows.
+void rule_backward(Ctx* c, const RuleC& r, const float* g, float* const* grads) {
+  Relation& H = *c->rels[r.plan.head_rel];
+  if (H.sr != XLOG_SR_LOGSUMEXP && H.sr != XLOG_SR_SUMPROD) fail(XLOG_ERR_UNSUPPORTED, "backward is defined for logsumexp and sum heads only");
+  if (r.kind == 3) fail(XLOG_ERR_UNSUPPORTED, "backward of the triangle aggregate is not built");
+  for (int j = 0; j < r.plan.n_atoms; ++j) {
+    if (!grads[j]) fail(XLOG_ERR_INVALID_ARGUMENT, "NULL gradient buffer");
+    if (r.plan.atoms[j].rel == r.plan.head_rel) fail(XLOG_ERR_UNSUPPORTED, "backward of a recursive rule");
+  }
+  int outer = 0;
+  if (r.kind == 2 && !r.shape[0].ok) outer = 1;
+  if (r.kind == 2 && r.shape[outer].probe_col != 0) fail(XLOG_ERR_UNSUPPORTED, "backward needs the looked-up atom probed on its first column");
+  // zero-fill each distinct buffer once
+  for (int j = 0; j < r.plan.n_atoms; ++j) {
+    bool seen = false;
+    for (int i = 0; i < j; ++i) seen = seen || grads[i] == grads[j];
+    if (!seen) XLOG_CUDA(cudaMemsetAsync(grads[j], 0, (size_t)c->rels[r.plan.atoms[j].rel]->n * 4, c->stream));
+  }
+  Relation& RA = *c->rels[r.plan.atoms[outer].rel];
+  if (RA.n == 0 || H.n == 0) { XLOG_CUDA(cudaStreamSynchronize(c->stream)); return; }
+  Variant v{&r, outer, full_source(RA)};
+  Counted q;
+  count_variant(c, v, H, q, kSlotTotals);
+  sync_ctrl(c);
+  q.total = c->h_ctrl[q.slot];
+  const int ckb = q.spec.head.total_bits <= 32 ? 4 : 8;
+  if (ckb != H.key_bytes) fail(XLOG_ERR_UNSUPPORTED, "backward: head key width differs from the declared-column key width");
+  BwdArgs bw{};
+  bw.head_keys = H.keys(); bw.head_tags = H.tags(); bw.n_head = H.n;
+  bw.count_bits = r.plan.emit_count_column ? H.layout.shift[r.plan.n_head_cols - 1] : 0;
+  bw.grad_head = g;
+  bw.grad_outer = grads[outer];
+  bw.grad_inner = r.kind == 2 ? grads[1 - outer] : nullptr;
+  bw.lse = H.sr == XLOG_SR_LOGSUMEXP ? 1 : 0;
+  if (q.total) launch_expand<true>(c, q, 0, q.total, ckb, nullptr, nullptr, bw);
+  sync_ctrl(c);
+}
 
 // Non-recursive stratum:  I(P) = facts(P) oplus (oplus over rules of T_r), each rule evaluated once.
 void stratum_once(Ctx* c, int head, const std::vector<const RuleC*>& rs) {

@@ -1,0 +1,164 @@
+"""Parity of the non-recursive aggregate rules (count, logsumexp, sum) and of the logsumexp-rule
+gradient with the CPU oracle.  Tolerances: counts and tuple sets exact; logsumexp tags 1e-4 absolute;
+gradients |d| <= 1e-5 + 1e-4 |ref| (fp32 exp and accumulation over at most 19 terms per row)."""
+import math
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2609_27203_b200 import synth, workloads as W
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+LSE_ABS = 1e-4
+
+
+def both(program, **kw):
+    from paper_2609_27203_b200 import xlog
+    kw.setdefault("arena_bytes", 1 << 28)
+    kw.setdefault("flags", xlog.FLAG_CHECK_INVARIANTS)
+    ctx, gids, grules = xlog.load_program(program, **kw)
+    receipt = ctx.fixpoint()
+    o, oids, orules = oracle.load_program(program)
+    o.run("naive")
+    return ctx, gids, grules, o, oids, orules, receipt
+
+
+def test_golden_listing7_degree_and_k3_triangle():
+    g = H.read_golden("listing7_degree_count.txt")
+    prog = W.Program("degree", {"edge": (2, W.SUMPROD), "degree": (2, W.SUMPROD)},
+                     [W.Rule("degree", (W.V(0),), (W.Atom("edge", (W.Var(0), W.Var(1))),), emit_count=True)],
+                     {"edge": ([g["edges"][:, 0].astype(np.int32), g["edges"][:, 1].astype(np.int32)], None)}, ("degree",))
+    ctx, gids, _, o, oids, _, _ = both(prog)
+    cols, tags = ctx.read(gids["degree"])
+    assert cols[0].tolist() == [1, 2] and cols[1].tolist() == [3, 1] and tags.tolist() == [3.0, 1.0]
+    ctx.close()
+    g = H.read_golden("k3_triangle_lse.txt")
+    e, t = g["edges"], g["tri_agg"]
+    ctx, gids, _, o, oids, _, _ = both(W.triangle_program(e[:, 0], e[:, 1], e[:, 2]))
+    cols, tags = ctx.read(gids["tri_agg"])
+    assert cols[0].tolist() == [0, 1, 2] and cols[1].tolist() == [2, 2, 2]
+    assert np.allclose(tags, t[:, 2], atol=2e-6)
+    ctx.close()
+
+
+@pytest.mark.parametrize("scale", [6, 10, 13])
+def test_triangle_aggregate_ladder(scale):
+    prog = W.config3(scale=scale)
+    ctx, gids, _, o, oids, _, _ = both(prog)
+    rep = H.compare_relations(ctx.read(gids["tri_agg"]), o.read(oids["tri_agg"]), abs_tol=LSE_ABS, what=prog.name)
+    assert rep["rows"] > 0
+    assert int(ctx.read(gids["tri_agg"])[0][1].sum()) % 3 == 0
+    ctx.close()
+
+
+def test_triangle_degenerate_graphs():
+    # no triangle at all; one 3-cycle (single-term groups pass through bit-exactly); complete digraph; a hub
+    for s, d, w in [([0, 1], [1, 2], [0.5, 0.25]),
+                    ([0, 1, 2], [1, 2, 0], [0.1, 0.2, 0.7])]:
+        prog = W.triangle_program(s, d, np.asarray(w, np.float32))
+        ctx, gids, _, o, oids, _, _ = both(prog)
+        rep = H.compare_relations(ctx.read(gids["tri_agg"]), o.read(oids["tri_agg"]), abs_tol=0, what="tiny")
+        assert rep["bit_unequal"] == 0
+        ctx.close()
+    n = 40
+    s, d = np.nonzero(~np.eye(n, dtype=bool))
+    ctx, gids, _, o, oids, _, _ = both(W.triangle_program(s, d, np.zeros(len(s), np.float32)))
+    cols, tags = ctx.read(gids["tri_agg"])
+    assert cols[1].tolist() == [(n - 1) * (n - 2)] * n
+    assert np.allclose(tags, math.log((n - 1) * (n - 2)), atol=1e-5)     # all-zero weights: LSE == ln(count)
+    ctx.close()
+    # hub: node 0 linked both ways with everyone, plus a ring among the others -> one group holds most terms
+    m = 3000
+    others = np.arange(1, m)
+    s = np.concatenate([np.zeros(m - 1, np.int64), others, others])
+    d = np.concatenate([others, np.zeros(m - 1, np.int64), np.roll(others, -1)])
+    w = synth.normal(8, 1, len(s)).astype(np.float32)
+    ctx, gids, _, o, oids, _, _ = both(W.triangle_program(s, d, w))
+    H.compare_relations(ctx.read(gids["tri_agg"]), o.read(oids["tri_agg"]), abs_tol=LSE_ABS, what="hub")
+    ctx.close()
+
+
+@pytest.mark.parametrize("B", [1, 16, 1024])
+def test_digit_sum_forward_and_backward(B):
+    import torch
+    prog = W.config4(n_pairs=B)
+    ctx, gids, grules, o, oids, orules, receipt = both(prog)
+    got = ctx.read(gids["sum"])
+    want = o.read(oids["sum"])
+    H.compare_relations(got, want, abs_tol=LSE_ABS, what=prog.name)
+    assert len(got[1]) == 19 * B and receipt["candidates"] == 100 * B
+    g = synth.head_gradient(19 * B, 77)
+    og = o.backward(orules[0], g)
+    ref = (og[0].astype(np.float64) + og[1].astype(np.float64))
+    gg = ctx.backward(grules[0], torch.from_numpy(g).cuda())
+    assert gg[0].data_ptr() == gg[1].data_ptr()                           # both atoms read `digit`: one buffer, the sum
+    out = gg[0].cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(out - ref) <= 1e-5 + 1e-4 * np.abs(ref))
+    # separate buffers per atom give the two parts
+    parts = ctx.backward(grules[0], torch.from_numpy(g).cuda(), same_buffer_for_same_relation=False)
+    for j in range(2):
+        r = og[j].astype(np.float64)
+        assert np.all(np.abs(parts[j].cpu().numpy() - r) <= 1e-5 + 1e-4 * np.abs(r))
+    # one-hot upstream gradient: the weights of one head row's bindings sum to one
+    e = np.zeros(19 * B, np.float32)
+    e[min(9, 19 * B - 1)] = 1.0
+    parts = ctx.backward(grules[0], torch.from_numpy(e).cuda(), same_buffer_for_same_relation=False)
+    assert abs(float(parts[0].sum().item()) - 1.0) < 1e-5 and abs(float(parts[1].sum().item()) - 1.0) < 1e-5
+    ctx.close()
+
+
+def test_uniform_digits_golden():
+    import torch
+    g = H.read_golden("uniform_digits_lse.txt")
+    B = 5
+    lt = np.full((2 * B, 10), -math.log(10.0), np.float32)
+    from paper_2609_27203_b200 import xlog
+    ctx, ids, rules = xlog.load_program(W.digits_program(lt), arena_bytes=1 << 26)
+    ctx.fixpoint()
+    cols, tags = ctx.read(ids["sum"])
+    for s_, v in g["out"]:
+        for s2 in (int(s_), 18 - int(s_)):
+            assert np.all(np.abs(tags[cols[1] == s2] - v) < 5e-6)
+    grad = ctx.backward(rules[0], torch.ones(len(tags), device="cuda"))[0].cpu().numpy().reshape(2 * B, 10)
+    for a, v in g["grad"]:
+        assert np.all(np.abs(grad[:, int(a)] - v) < 1e-5)
+    ctx.close()
+
+
+def test_sum_semiring_two_step_walk_counts_and_facts_of_a_derived_relation():
+    s, d = synth.uniform_digraph(60, 400, 3)
+    prog = W.Program("p2", {"e": (2, W.SUMPROD), "p2": (2, W.SUMPROD)},
+                     [W.Rule("p2", (W.V(0), W.V(2)), (W.Atom("e", (W.Var(0), W.Var(1))), W.Atom("e", (W.Var(1), W.Var(2)))))],
+                     {"e": ([s, d], None)}, ("p2",))
+    ctx, gids, _, o, oids, _, _ = both(prog)
+    rep = H.compare_relations(ctx.read(gids["p2"]), o.read(oids["p2"]), what="p2")
+    assert rep["bit_unequal"] == 0
+    ctx.close()
+    prog = W.Program("mix", {"a": (1, W.LOGSUMEXP), "q": (1, W.LOGSUMEXP)},
+                     [W.Rule("q", (W.V(0),), (W.Atom("a", (W.Var(0),)),))],
+                     {"a": ([np.array([1, 2], np.int32)], np.array([0.0, -1.0], np.float32)),
+                      "q": ([np.array([2, 5], np.int32)], np.array([-1.0, -3.0], np.float32))}, ("q",))
+    ctx, gids, _, o, oids, _, _ = both(prog)
+    H.compare_relations(ctx.read(gids["q"]), o.read(oids["q"]), abs_tol=1e-6, what="mix")
+    ctx.fixpoint()                                   # recomputed, not accumulated twice
+    H.compare_relations(ctx.read(gids["q"]), o.read(oids["q"]), abs_tol=1e-6, what="mix again")
+    ctx.close()
+
+
+def test_backward_requires_a_forward_and_a_supported_head():
+    import torch
+    from paper_2609_27203_b200 import xlog
+    prog = W.config4(n_pairs=2)
+    ctx, ids, rules = xlog.load_program(prog, arena_bytes=1 << 26)
+    with pytest.raises(xlog.XlogError) as e:
+        ctx.backward(rules[0], torch.ones(38, device="cuda"))
+    assert e.value.status == "INVALID_STATE"
+    ctx.close()
+    ctx, ids, rules = xlog.load_program(W.config1(20, 40), arena_bytes=1 << 26)
+    ctx.fixpoint()
+    with pytest.raises(xlog.XlogError) as e:
+        ctx.backward(rules[0], torch.ones(ctx.size(ids["path"]), device="cuda"))
+    assert e.value.status == "UNSUPPORTED"
+    ctx.close()
