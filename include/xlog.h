@@ -175,6 +175,13 @@ xlog_status xlog_ctx_reset_idb(xlog_ctx* ctx);
  * Passing the same pointer for two atoms of one relation yields the sum. */
 xlog_status xlog_rule_backward(xlog_ctx* ctx, xlog_rule rule, const float* grad_head, float* const* grad_atoms);
 
+/* ---- the sort on its own (paper kernel table: `sort`) ---------------------------------
+ * Stable ascending sort of n (key, 4-byte payload) pairs by the low key_bits bits of the key.
+ * keys / payload: DEVICE, sorted in place; key_bytes is 4 or 8; n < 2^30.  Scratch (a second
+ * buffer pair and the pass bookkeeping) comes from the context's arena: RESOURCE_EXHAUSTED if
+ * it does not fit.  Used by load, by index builds and once per round by the fixpoint. */
+xlog_status xlog_sort_pairs(xlog_ctx* ctx, void* keys, void* payload, int64_t n, int32_t key_bytes, int32_t key_bits);
+
 /* ---- per-kernel statistics (Section "Semi-naive evaluation on GPU": the profiler records
  * per-operator timing and row counts) ------------------------------------------------
  * With XLOG_FLAG_PROFILE every kernel launch is bracketed by CUDA events on the context's

@@ -29,6 +29,19 @@ struct KeyLayout {
   int total_bits;
 };
 
+// Optional order-preserving dictionaries: a column whose values come from a small set stores the
+// rank of the value in the sorted set instead of the value (dense ids, as the paper's symbol table
+// makes strings dense: Section "Reversible symbols").  n[c] == 0: column c holds plain values.
+struct DictSet {
+  const int32_t* v[kMaxArity];
+  uint32_t n[kMaxArity];
+};
+__device__ __forceinline__ uint32_t dict_rank(const int32_t* v, uint32_t n, int64_t value) {   // lower bound
+  uint32_t lo = 0, hi = n;
+  while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if ((int64_t)v[mid] < value) lo = mid + 1; else hi = mid; }
+  return lo;
+}
+
 template <typename K>
 __host__ __device__ __forceinline__ K pack_key(const KeyLayout& L, const int32_t* cols) {
   K k = 0;

@@ -16,6 +16,7 @@
 #include "../../include/xlog.h"
 #include "arena.h"
 #include "common.cuh"
+#include "dense_reduce.cuh"
 #include "join.cuh"
 #include "relops.cuh"
 #include "scan.cuh"
@@ -77,7 +78,11 @@ struct Relation {
   // loaded facts: packed keys sorted ascending, unique
   KeyLayout layout{};
   int key_bytes = 4;
-  int32_t col_max[kMaxArity] = {0, 0, 0, 0};
+  int32_t col_max[kMaxArity] = {0, 0, 0, 0};      // bound of what is stored (the code when the column has a dictionary)
+  int32_t fact_max[kMaxArity] = {0, 0, 0, 0};     // column maxima of the loaded facts
+  int32_t val_max[kMaxArity] = {0, 0, 0, 0};      // bound of the column's values
+  DevBuf dict[kMaxArity];                         // sorted distinct values of a dictionary-encoded column
+  uint32_t dict_n[kMaxArity] = {0, 0, 0, 0};
   DevBuf fact_keys, fact_tags;
   uint32_t n_facts = 0;
   // current contents; alias the facts until something is derived
@@ -90,6 +95,11 @@ struct Relation {
   Index idx[kMaxArity];
   bool is_head = false;
 
+  DictSet dicts() const {
+    DictSet d{};
+    for (int i = 0; i < kMaxArity; ++i) { d.v[i] = dict[i].as<int32_t>(); d.n[i] = dict_n[i]; }
+    return d;
+  }
   const void* keys() const { return cur_owned ? cur_keys.p : fact_keys.p; }
   float* tags() const { return reinterpret_cast<float*>(cur_owned ? cur_tags.p : fact_tags.p); }
 };
@@ -256,24 +266,40 @@ inline void scan_exclusive_u32_inplace(Ctx* c, uint32_t* v, uint64_t n, uint32_t
 // Sort n (key, tag) pairs on key bits [0, nbits).  On return keys/tags point at the sorted data
 // (either the original buffers or the alternates).
 template <typename K>
-inline void sort_pairs(Ctx* c, K*& keys, float*& tags, K*& keys_alt, float*& tags_alt, uint64_t n, int nbits) {
+inline void sort_pairs(Ctx* c, K*& keys, float*& tags, K*& keys_alt, float*& tags_alt, uint64_t n, int nbits, int low_bit = 0) {
   if (n <= 1) return;
-  const SortPlan p = make_sort_plan<K>(n, nbits);
-  if (p.passes == 0) return;
-  DevBuf hist(c, p.hist_entries * 4), spine(c, (p.scan_tiles + 1) * 4);
-  for (int pass = 0; pass < p.passes; ++pass) {
-    const int shift = pass * p.bits_per_pass;
-    const int nb = std::min(p.bits_per_pass, nbits - shift);
-    if (nb <= 0) break;
-    const int nbins = 1 << nb;
-    c->note_bytes = (int64_t)n * sizeof(K);
-    XLOG_LAUNCH(c, (k_sort_hist<K>), (p.ntiles + kHistGroup - 1) / kHistGroup, kSortBlock, 0, keys, (uint32_t)n, shift, nbins,
-                p.ntiles, hist.as<uint32_t>());
-    scan_exclusive_u32_inplace<uint32_t>(c, hist.as<uint32_t>(), (uint64_t)nbins * p.ntiles, spine.as<uint32_t>());
+  if (n > kSortMaxN) fail(XLOG_ERR_CAPACITY_EXCEEDED, "a single sort is limited to 2^30 - 1 rows");
+  const SortPasses P = make_sort_passes(low_bit, nbits);
+  if (P.passes == 0) return;
+  const uint32_t ntiles = (uint32_t)((n + sort_tile<K>() - 1) / sort_tile<K>());
+  // scratch: digit histograms of every pass, one ticket per pass, the look-back status words (reused by every pass)
+  const size_t head_words = (size_t)kSortMaxPasses * kSortMaxBins + kSortMaxPasses;
+  DevBuf scratch(c, (head_words + (size_t)ntiles * kSortMaxBins) * 4);
+  uint32_t* hist = scratch.as<uint32_t>();
+  uint32_t* tickets = hist + kSortMaxPasses * kSortMaxBins;
+  uint32_t* status = hist + head_words;
+  XLOG_CUDA(cudaMemsetAsync(hist, 0, head_words * 4, c->stream));
+  c->note_bytes = (int64_t)n * sizeof(K);
+  XLOG_LAUNCH(c, (k_sort_digit_hist<K>), grid_for(n, 256 * 8, kSMs * 8), 256, 0, keys, (uint32_t)n, P, hist);
+  XLOG_LAUNCH(c, k_sort_digit_bases, 1, 256, 0, hist, P.passes);
+  for (int pass = 0; pass < P.passes; ++pass) {
+    XLOG_CUDA(cudaMemsetAsync(status, 0, (size_t)ntiles * kSortMaxBins * 4, c->stream));
     c->note_bytes = (int64_t)n * 2 * (sizeof(K) + 4);
-    XLOG_LAUNCH(c, (k_sort_scatter<K>), p.ntiles, kSortBlock, sort_scatter_smem<K>(), keys,
-                reinterpret_cast<const uint32_t*>(tags), keys_alt, reinterpret_cast<uint32_t*>(tags_alt), (uint32_t)n, shift,
-                nbins, p.ntiles, hist.as<uint32_t>());
+#define XLOG_SORT_PASS(B)                                                                                                          \
+  XLOG_LAUNCH(c, (k_sort_pass<K, B>), ntiles, kSortBlock, sort_pass_smem<K>(), keys, reinterpret_cast<const uint32_t*>(tags), keys_alt, \
+              reinterpret_cast<uint32_t*>(tags_alt), (uint32_t)n, P.shift[pass], hist + pass * kSortMaxBins, status, tickets + pass,  \
+              ctrl_u32(c, kSlotErr))
+    switch (P.bits[pass]) {
+      case 1: XLOG_SORT_PASS(1); break;
+      case 2: XLOG_SORT_PASS(2); break;
+      case 3: XLOG_SORT_PASS(3); break;
+      case 4: XLOG_SORT_PASS(4); break;
+      case 5: XLOG_SORT_PASS(5); break;
+      case 6: XLOG_SORT_PASS(6); break;
+      case 7: XLOG_SORT_PASS(7); break;
+      default: XLOG_SORT_PASS(8); break;
+    }
+#undef XLOG_SORT_PASS
     std::swap(keys, keys_alt);
     std::swap(tags, tags_alt);
   }
@@ -324,10 +350,64 @@ inline uint32_t reduce_by_key(Ctx* c, int sr, const K* keys, const float* tags, 
   }
 }
 
+// max/min reduce-by-key that sorts only the high key bits and reduces each group of equal high
+// bits in a shared-memory table (dense_reduce.cuh).  Worth it when groups are well filled.
+inline bool dense_reduce_applies(int sr, uint64_t n, int nbits, bool want_head_pos) {
+  if (want_head_pos || (sr != XLOG_SR_MAXPLUS && sr != XLOG_SR_MINPLUS)) return false;
+  const int H = nbits > kDenseBits ? nbits - kDenseBits : 0;
+  if (H > kDenseMaxGroupBits) return false;
+  return n >= (1u << 18) && n >= ((uint64_t)32 << H);
+}
+
+template <typename K, typename Op>
+inline KeyTags sort_dense_reduce(Ctx* c, DevBuf& k0, DevBuf& t0, DevBuf& k1, DevBuf& t1, uint64_t n, int nbits) {
+  KeyTags out;
+  K* ka = k0.as<K>(); K* kb = k1.as<K>();
+  float* ta = t0.as<float>(); float* tb = t1.as<float>();
+  const int L = std::min(nbits, kDenseBits), H = nbits - L;
+  const uint32_t G = 1u << H;
+  sort_pairs<K>(c, ka, ta, kb, tb, n, nbits, L);                       // high bits only
+  uint32_t part = (uint32_t)std::min<uint64_t>(std::max<uint64_t>(n / (kSMs * 8), 8192), 131072);
+  part = (part + 1023) / 1024 * 1024;
+  const uint32_t spill_cap = std::min<uint32_t>((uint32_t)(n / part) + 1, G), max_items = (uint32_t)(n / part) + G + 1;
+  DevBuf gstart(c, ((size_t)G + 1) * 4), part_base(c, ((size_t)G + 1) * 4), spill(c, (size_t)G * 4), done(c, (size_t)G * 4),
+      ucount(c, ((size_t)G + 1) * 4), spill_tab(c, (size_t)spill_cap * kDenseSlots * 4);
+  XLOG_CUDA(cudaMemsetAsync(ucount.p, 0, ((size_t)G + 1) * 4, c->stream));
+  XLOG_LAUNCH(c, (k_group_bounds<K>), grid_for((uint64_t)G + 1, 256), 256, 0, (const K*)ka, (uint32_t)n, L, G, gstart.as<uint32_t>());
+  XLOG_LAUNCH(c, k_group_plan, 1, 1024, 0, (const uint32_t*)gstart.as<uint32_t>(), G, part, part_base.as<uint32_t>(), spill.as<uint32_t>(),
+              done.as<uint32_t>(), ctrl_u32(c, kSlotB));
+  XLOG_LAUNCH(c, k_fill_i32, grid_for((uint64_t)spill_cap * kDenseSlots, 256 * 8), 256, 0, spill_tab.as<int32_t>(),
+              (uint64_t)spill_cap * kDenseSlots, DenseOp<Op>::empty);
+  c->note_bytes = (int64_t)n * (sizeof(K) + 4);
+  XLOG_LAUNCH(c, (k_dense_reduce<K, Op>), max_items, kDenseBlock, 0, (const K*)ka, (const float*)ta, L, G, part,
+              (const uint32_t*)gstart.as<uint32_t>(), (const uint32_t*)part_base.as<uint32_t>(), (const uint32_t*)spill.as<uint32_t>(), spill_cap,
+              spill_tab.as<int32_t>(), done.as<uint32_t>(), kb, tb, ucount.as<uint32_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, ucount.as<uint32_t>(), (int64_t)G + 1, ctrl_u32(c, kSlotA));
+  sync_ctrl(c);
+  out.n = (uint32_t)c->h_ctrl[kSlotA];
+  const bool sorted_in_0 = (void*)ka == k0.p;
+  (sorted_in_0 ? k0 : k1).reset();
+  (sorted_in_0 ? t0 : t1).reset();
+  spill_tab.reset();
+  out.keys = DevBuf(c, (size_t)std::max(out.n, 1u) * sizeof(K));
+  out.tags = DevBuf(c, (size_t)std::max(out.n, 1u) * 4);
+  if (out.n) {
+    c->note_bytes = (int64_t)out.n * 2 * (sizeof(K) + 4);
+    XLOG_LAUNCH(c, (k_dense_compact<K>), grid_for((uint64_t)G * 32, 256), 256, 0, (const K*)kb, (const float*)tb, (const uint32_t*)gstart.as<uint32_t>(),
+                (const uint32_t*)ucount.as<uint32_t>(), G, out.keys.as<K>(), out.tags.as<float>());
+    XLOG_CUDA(cudaStreamSynchronize(c->stream));
+  }
+  k0.reset(); t0.reset(); k1.reset(); t1.reset();
+  return out;
+}
+
 // Sort + reduce the first n pairs of (k0,t0) using (k1,t1) as the second half of the double
 // buffer; releases both and returns the groups in exact-size buffers.
 template <typename K>
 inline KeyTags sort_reduce(Ctx* c, int sr, DevBuf& k0, DevBuf& t0, DevBuf& k1, DevBuf& t1, uint64_t n, int nbits, bool want_head_pos) {
+  if (dense_reduce_applies(sr, n, nbits, want_head_pos))
+    return sr == XLOG_SR_MAXPLUS ? sort_dense_reduce<K, OpMax>(c, k0, t0, k1, t1, n, nbits)
+                                 : sort_dense_reduce<K, OpMin>(c, k0, t0, k1, t1, n, nbits);
   KeyTags out;
   K* ka = k0.as<K>(); K* kb = k1.as<K>();
   float* ta = t0.as<float>(); float* tb = t1.as<float>();

@@ -17,6 +17,9 @@ struct JoinSpec {
   // outer side: packed keys + tags
   KeyLayout outer;
   ArgSpec outer_args[kMaxArity];
+  DictSet outer_dict;                                         // dictionaries of the outer relation's columns
+  int outer_decode[kMaxArity];                                // 1: turn the stored code into the value when binding
+
   // inner side (absent for one-atom rules): offsets over the probed column, the other columns, tags
   int has_inner;
   int probe_var, probe_mul, probe_add;                        // probed value = probe_mul * var + probe_add
@@ -29,6 +32,9 @@ struct JoinSpec {
   const float* inner_tag;
   // head
   KeyLayout head;
+  DictSet head_dict;                                          // dictionaries of the head relation's columns
+  int head_encode[kMaxArity];                                 // 1: the head expression yields a value that must be ranked;
+                                                              // 0 with a dictionary: the variable already carries the code
   int64_t head_c0[kMaxArity];
   int32_t head_coef[kMaxArity][kMaxVars];
   int times;                                                  // otimes: 0 = add, 1 = multiply
@@ -45,7 +51,8 @@ __device__ __forceinline__ bool bind_outer(const JoinSpec& S, KO key, int64_t* v
 #pragma unroll
   for (int c = 0; c < kMaxArity; ++c) {
     if (c < S.outer.arity) {
-      const int64_t val = key_col<KO>(S.outer, key, c);
+      int64_t val = key_col<KO>(S.outer, key, c);
+      if (S.outer_decode[c]) val = S.outer_dict.v[c][min((uint32_t)val, S.outer_dict.n[c] - 1)];
       const ArgSpec a = S.outer_args[c];
       if (a.kind == 0) ok = ok && val == a.add;
       else {
@@ -175,6 +182,10 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
         int64_t h = S.head_c0[c];
 #pragma unroll
         for (int v = 0; v < kMaxVars; ++v) h += (int64_t)S.head_coef[c][v] * var[v];
+        if (S.head_encode[c]) {
+          const uint32_t r = dict_rank(S.head_dict.v[c], S.head_dict.n[c], h);
+          if (r >= S.head_dict.n[c] || (int64_t)S.head_dict.v[c][r] != h) { e |= kErrInternal; h = 0; } else h = r;
+        }
         if (h < 0 || h > (int64_t)S.head.mask[c]) { e |= kErrHeadRange; h = 0; }
         key |= (KH)(uint32_t)h << S.head.shift[c];
       }

@@ -45,12 +45,15 @@ static __global__ void __launch_bounds__(256) k_col_stats(ColPtrs cols, const fl
 }
 
 template <typename K>
-__global__ void __launch_bounds__(256) k_pack(ColPtrs cols, const float* __restrict__ tags, int64_t n, KeyLayout L, float one,
+__global__ void __launch_bounds__(256) k_pack(ColPtrs cols, const float* __restrict__ tags, int64_t n, KeyLayout L, DictSet D, float one,
                                               K* __restrict__ keys, float* __restrict__ tag_out) {
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     int32_t v[kMaxArity];
 #pragma unroll
-    for (int c = 0; c < kMaxArity; ++c) v[c] = c < L.arity ? cols.c[c][i] : 0;
+    for (int c = 0; c < kMaxArity; ++c) {
+      v[c] = c < L.arity ? cols.c[c][i] : 0;
+      if (c < L.arity && D.n[c]) v[c] = (int32_t)dict_rank(D.v[c], D.n[c], v[c]);
+    }
     keys[i] = pack_key<K>(L, v);
     float t = tags ? tags[i] : one;
     if (t == 0.f) t = 0.f;                         // -0.0 -> +0.0
@@ -59,12 +62,15 @@ __global__ void __launch_bounds__(256) k_pack(ColPtrs cols, const float* __restr
 }
 
 template <typename K>
-__global__ void __launch_bounds__(256) k_unpack(const K* __restrict__ keys, int64_t n, KeyLayout L, ColPtrsMut cols) {
+__global__ void __launch_bounds__(256) k_unpack(const K* __restrict__ keys, int64_t n, KeyLayout L, DictSet D, ColPtrsMut cols) {
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
     const K k = keys[i];
 #pragma unroll
     for (int c = 0; c < kMaxArity; ++c)
-      if (c < L.arity) cols.c[c][i] = key_col<K>(L, k, c);
+      if (c < L.arity) {
+        const int32_t code = key_col<K>(L, k, c);
+        cols.c[c][i] = D.n[c] ? D.v[c][min((uint32_t)code, D.n[c] - 1)] : code;
+      }
   }
 }
 

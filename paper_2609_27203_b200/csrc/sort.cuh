@@ -3,98 +3,164 @@
 // digits and 8 passes per 32-bit key; here digits are up to 8 bits and only the bits the
 // key layout actually uses are sorted, e.g. 28 bits -> 4 passes of 7 bits).
 //
-// Per pass:  k_sort_hist   per-tile digit counts            (reads keys)
-//            scan          exclusive scan, digit-major      (tiny)
-//            k_sort_scatter rank inside the tile with warp match, order the tile in shared
-//                          memory, write each digit's run contiguously (reads+writes pairs)
-// No block waits on another block, so there is no spin loop anywhere in the sort.
+// One read of the keys builds the digit histograms of every pass (k_sort_digit_hist); each pass
+// is then a single kernel (k_sort_pass) that ranks a tile with warp match, orders it in shared
+// memory, and learns where its digit runs start from the tiles before it by decoupled look-back
+// over a per-tile status word (count + 2 flag bits).  Tiles take their index from an atomic
+// ticket, so a tile only ever waits for tiles that are already running; every wait is bounded
+// and a timeout raises the error flag and skips the tile's writes instead of hanging.
 #pragma once
 #include "common.cuh"
 #include "scan.cuh"
 
 namespace xlog {
 
-constexpr int kSortBlock = 512;
+#ifndef XLOG_SORT_BLOCK
+#define XLOG_SORT_BLOCK 256
+#endif
+#ifndef XLOG_SORT_ITEMS
+#define XLOG_SORT_ITEMS 16
+#endif
+#ifndef XLOG_SORT_MINB
+#define XLOG_SORT_MINB 4
+#endif
+constexpr int kSortBlock = XLOG_SORT_BLOCK;
 constexpr int kSortWarps = kSortBlock / 32;
 constexpr int kSortMaxBins = 256;
-constexpr int kHistGroup = 8;            // tiles per histogram block: 8 counters = one 32-byte sector per digit
+constexpr int kSortMaxPasses = 8;
+constexpr uint32_t kSortMaxN = (1u << 30) - 1;       // status words keep 30 bits of count
+constexpr uint32_t kFlagLocal = 1u << 30, kFlagGlobal = 2u << 30, kCountMask = (1u << 30) - 1;
+constexpr uint32_t kSpinLimit = 1u << 22;            // polls of one status word before giving up
 
-template <typename K> struct SortCfg { static constexpr int items = sizeof(K) == 4 ? 16 : 12; };
+template <typename K> struct SortCfg { static constexpr int items = XLOG_SORT_ITEMS; };
 template <typename K> constexpr int sort_tile() { return kSortBlock * SortCfg<K>::items; }
 
-// hist[d * ntiles + tile] = number of keys of `tile` whose digit is d
+struct SortPasses {
+  int passes;
+  int shift[kSortMaxPasses];
+  int bits[kSortMaxPasses];
+};
+
+// passes covering key bits [lo, hi), least significant first
+inline SortPasses make_sort_passes(int lo, int hi) {
+  SortPasses p{};
+  const int nbits = hi > lo ? hi - lo : 0;
+  p.passes = (nbits + 7) / 8;
+  int done = 0;
+  for (int i = 0; i < p.passes; ++i) {
+    const int b = (nbits - done + (p.passes - i) - 1) / (p.passes - i);     // spread the bits evenly
+    p.shift[i] = lo + done; p.bits[i] = b; done += b;
+  }
+  return p;
+}
+
+__device__ __forceinline__ uint32_t ld_volatile_u32(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.volatile.global.u32 %0, [%1];" : "=r"(v) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_volatile_u32(uint32_t* p, uint32_t v) {
+  asm volatile("st.volatile.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// hist[pass * 256 + d] += number of keys whose digit of `pass` is d.  Persistent grid.
 template <typename K>
-__global__ void __launch_bounds__(kSortBlock) k_sort_hist(const K* __restrict__ keys, uint32_t n, int shift, int nbins,
-                                                          uint32_t ntiles, uint32_t* __restrict__ hist) {
-  constexpr int TILE = kSortBlock * SortCfg<K>::items;
-  __shared__ uint32_t cnt[kHistGroup][kSortMaxBins];
-  for (int i = threadIdx.x; i < kHistGroup * kSortMaxBins; i += kSortBlock) (&cnt[0][0])[i] = 0;
+__global__ void __launch_bounds__(256) k_sort_digit_hist(const K* __restrict__ keys, uint32_t n, SortPasses P,
+                                                         uint32_t* __restrict__ hist) {
+  __shared__ uint32_t sh[kSortMaxPasses * kSortMaxBins];
+  for (int i = threadIdx.x; i < P.passes * kSortMaxBins; i += blockDim.x) sh[i] = 0;
   __syncthreads();
-  const uint32_t mask = (uint32_t)nbins - 1u;
-  const uint32_t tile0 = blockIdx.x * kHistGroup;
-  for (int g = 0; g < kHistGroup; ++g) {
-    const uint32_t tile = tile0 + g;
-    if (tile >= ntiles) break;
-    const uint64_t base = (uint64_t)tile * TILE;
-#pragma unroll 4
-    for (int i = 0; i < SortCfg<K>::items; ++i) {
-      const uint64_t p = base + (uint64_t)i * kSortBlock + threadIdx.x;
-      const bool ok = p < n;
-      const uint32_t d = ok ? (uint32_t)(keys[p] >> shift) & mask : 0xffffffffu;
-      const unsigned peers = __match_any_sync(0xffffffffu, d);
-      if (ok && (peers & lanemask_lt()) == 0) atomicAdd(&cnt[g][d], (uint32_t)__popc(peers));
+  // each block takes chunks of 256*8 keys; a thread issues its 8 loads before it touches any of them
+  constexpr int U = 8;
+  const uint64_t chunk = (uint64_t)blockDim.x * U;
+  for (uint64_t c0 = (uint64_t)blockIdx.x * chunk; c0 < n; c0 += (uint64_t)gridDim.x * chunk) {
+    K k[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const uint64_t i = c0 + (uint64_t)u * blockDim.x + threadIdx.x;
+      k[u] = i < n ? keys[i] : K(0);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const bool ok = c0 + (uint64_t)u * blockDim.x + threadIdx.x < n;
+#pragma unroll
+      for (int p = 0; p < kSortMaxPasses; ++p) {
+        if (p < P.passes) {
+          // lanes sharing the digit of the first active lane are counted with one ballot (covers the
+          // skewed case: a hot key, or a high digit that is constant across the tile); the others
+          // add individually (few conflicts when digits are spread out)
+          const uint32_t d = ok ? (uint32_t)(k[u] >> P.shift[p]) & ((1u << P.bits[p]) - 1u) : 0xffffffffu;
+          const unsigned act = __ballot_sync(0xffffffffu, ok);
+          if (act) {
+            const int first = __ffs(act) - 1;
+            const uint32_t d0 = __shfl_sync(0xffffffffu, d, first);
+            const unsigned same = __ballot_sync(0xffffffffu, ok && d == d0);
+            if ((int)lane_id() == first) atomicAdd(&sh[p * kSortMaxBins + d0], (uint32_t)__popc(same));
+            else if (ok && d != d0) atomicAdd(&sh[p * kSortMaxBins + d], 1u);
+          }
+        }
+      }
     }
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < nbins * kHistGroup; i += kSortBlock) {
-    const int d = i / kHistGroup, g = i % kHistGroup;
-    if (tile0 + g < ntiles) hist[(uint64_t)d * ntiles + tile0 + g] = cnt[g][d];
+  for (int i = threadIdx.x; i < P.passes * kSortMaxBins; i += blockDim.x)
+    if (sh[i]) atomicAdd(&hist[i], sh[i]);
+}
+
+// In place: hist[pass*256 + d] becomes the number of keys with a smaller digit in that pass.
+static __global__ void __launch_bounds__(256) k_sort_digit_bases(uint32_t* __restrict__ hist, int passes) {
+  __shared__ uint32_t sh[256 / 32 + 1];
+  for (int p = 0; p < passes; ++p) {
+    const uint32_t v = hist[p * kSortMaxBins + threadIdx.x];
+    uint32_t total;
+    const uint32_t e = block_scan_excl<256, uint32_t>(v, sh, total);
+    hist[p * kSortMaxBins + threadIdx.x] = e;
   }
 }
 
-// offs = exclusive scan of hist (digit-major), i.e. offs[d*ntiles+tile] is where this tile's
-// run of digit d starts in the output.
-template <typename K>
-__global__ void __launch_bounds__(kSortBlock) k_sort_scatter(const K* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
-                                                             K* __restrict__ keys_out, uint32_t* __restrict__ vals_out, uint32_t n,
-                                                             int shift, int nbins, uint32_t ntiles,
-                                                             const uint32_t* __restrict__ offs) {
+// One pass.  status[tile*256 + d]: 0 = not ready, kFlagLocal|count = this tile's count of digit d,
+// kFlagGlobal|count = count summed over tiles 0..tile.  ticket: one counter per pass, starts at 0.
+// Lanes of the warp whose digit equals this lane's: one ballot per digit bit (the hardware
+// match instruction is an order of magnitude slower than BITS ballots on this part).
+template <int BITS>
+__device__ __forceinline__ unsigned match_digit(uint32_t d) {
+  unsigned peers = 0xffffffffu;
+#pragma unroll
+  for (int b = 0; b < BITS; ++b) {
+    const bool bit = (d >> b) & 1u;
+    const unsigned m = __ballot_sync(0xffffffffu, bit);
+    peers &= bit ? m : ~m;
+  }
+  return peers;
+}
+
+// Body of one tile; FULL = the tile has no padding (all bounds tests fold away).
+template <typename K, int BITS, bool FULL>
+__device__ __forceinline__ void sort_tile_body(const K* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
+                                               K* __restrict__ keys_out, uint32_t* __restrict__ vals_out, const uint64_t base,
+                                               const uint32_t valid, const uint32_t tile, const int shift,
+                                               const uint32_t* __restrict__ digit_base, uint32_t* __restrict__ status,
+                                               uint32_t* __restrict__ err, K* skeys, uint32_t* svals, uint32_t* whist,
+                                               uint32_t* lbase, uint32_t* goff, uint32_t* scan_sh) {
   constexpr int ITEMS = SortCfg<K>::items;
   constexpr int TILE = kSortBlock * ITEMS;
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  K* skeys = reinterpret_cast<K*>(smem_raw);                                   // TILE keys
-  uint32_t* svals = reinterpret_cast<uint32_t*>(smem_raw + sizeof(K) * TILE);  // TILE payloads
-  uint32_t* whist = svals + TILE;                                              // [kSortWarps][256]
-  uint32_t* lbase = whist + kSortWarps * kSortMaxBins;                         // [256] tile-local start of each digit
-  uint32_t* goff = lbase + kSortMaxBins;                                       // [256] global start minus local start
-  uint32_t* scan_sh = goff + kSortMaxBins;                                     // block scan scratch
-
-  const uint32_t tile = blockIdx.x;
-  const uint64_t base = (uint64_t)tile * TILE;
-  const uint32_t valid = (uint32_t)min((uint64_t)TILE, (uint64_t)n - base);
-  const uint32_t mask = (uint32_t)nbins - 1u;
+  constexpr int nbins = 1 << BITS;
+  constexpr uint32_t mask = (uint32_t)nbins - 1u;
   const unsigned w = warp_id(), l = lane_id();
-
-  for (int i = threadIdx.x; i < kSortWarps * kSortMaxBins; i += kSortBlock) whist[i] = 0;
-  __syncthreads();
 
   // warp-striped load: item r of lane l sits at tile position w*32*ITEMS + r*32 + l
   K key[ITEMS];
-  uint32_t val[ITEMS];
   uint32_t rank[ITEMS];
-  const uint32_t wbase = w * 32 * ITEMS;
+  const uint32_t wbase = w * 32 * ITEMS + l;
+  const K* kin = keys_in + base + wbase;
 #pragma unroll
-  for (int r = 0; r < ITEMS; ++r) {
-    const uint32_t p = wbase + r * 32 + l;
-    if (p < valid) { key[r] = keys_in[base + p]; val[r] = vals_in[base + p]; }
-    else { key[r] = ~K(0); val[r] = 0; }
-  }
+  for (int r = 0; r < ITEMS; ++r) key[r] = (FULL || wbase + r * 32 < valid) ? kin[r * 32] : ~K(0);
   uint32_t* myhist = whist + w * kSortMaxBins;
 #pragma unroll
   for (int r = 0; r < ITEMS; ++r) {
-    const uint32_t p = wbase + r * 32 + l;
-    const uint32_t d = p < valid ? (uint32_t)(key[r] >> shift) & mask : mask;   // padding ranks last in the last bin
-    const unsigned peers = __match_any_sync(0xffffffffu, d);
+    // padding carries all-ones keys: it ranks last in the last bin
+    const uint32_t d = (uint32_t)(key[r] >> shift) & mask;
+    const unsigned peers = match_digit<BITS>(d);
     const int leader = __ffs(peers) - 1;
     uint32_t before = 0;
     if ((int)l == leader) { before = myhist[d]; myhist[d] = before + __popc(peers); }
@@ -104,7 +170,7 @@ __global__ void __launch_bounds__(kSortBlock) k_sort_scatter(const K* __restrict
   }
   __syncthreads();
 
-  // per digit: exclusive prefix over warps (in place) and the tile total
+  // per digit: exclusive prefix over warps (in place) and the tile total; publish the tile's counts
   uint32_t total_d = 0;
   if ((int)threadIdx.x < nbins) {
     const int d = threadIdx.x;
@@ -116,28 +182,59 @@ __global__ void __launch_bounds__(kSortBlock) k_sort_scatter(const K* __restrict
       run += c;
     }
     total_d = run;
+    if (!FULL && d == nbins - 1) total_d -= (uint32_t)TILE - valid;             // padding is not data
+    st_volatile_u32(&status[(uint64_t)tile * kSortMaxBins + d], (tile == 0 ? kFlagGlobal : kFlagLocal) | total_d);
   }
   uint32_t tile_total;
   const uint32_t lb = block_scan_excl<kSortBlock, uint32_t>(total_d, scan_sh, tile_total);
-  if ((int)threadIdx.x < nbins) {
-    lbase[threadIdx.x] = lb;
-    goff[threadIdx.x] = offs[(uint64_t)threadIdx.x * ntiles + tile] - lb;
-  }
+  if ((int)threadIdx.x < nbins) lbase[threadIdx.x] = lb;
   __syncthreads();
 
-  // order the tile in shared memory
+  // order the tile's keys in shared memory; remember each item's slot for its payload
 #pragma unroll
   for (int r = 0; r < ITEMS; ++r) {
-    const uint32_t p = wbase + r * 32 + l;
-    const uint32_t d = p < valid ? (uint32_t)(key[r] >> shift) & mask : mask;
-    const uint32_t pos = lbase[d] + myhist[d] + rank[r];
-    skeys[pos] = key[r];
-    svals[pos] = val[r];
+    const uint32_t d = (uint32_t)(key[r] >> shift) & mask;
+    rank[r] += lbase[d] + myhist[d];
+    if (FULL || rank[r] < valid) skeys[rank[r]] = key[r];
+  }
+  // payloads: same slots
+  const uint32_t* vin = vals_in + base + wbase;
+#pragma unroll
+  for (int r = 0; r < ITEMS; ++r)
+    if (FULL || wbase + r * 32 < valid) svals[rank[r]] = vin[r * 32];
+
+  // decoupled look-back: keys with digit d in all earlier tiles
+  if ((int)threadIdx.x < nbins) {
+    const int d = threadIdx.x;
+    uint32_t excl = 0;
+    bool timeout = false;
+    if (tile > 0) {
+      int64_t look = (int64_t)tile - 1;
+      uint32_t spins = 0;
+      while (true) {
+        const uint32_t s = ld_volatile_u32(&status[(uint64_t)look * kSortMaxBins + d]);
+        const uint32_t flag = s & ~kCountMask;
+        if (flag == 0) {
+          if (++spins > kSpinLimit) { timeout = true; break; }
+          __nanosleep(64);
+          continue;
+        }
+        excl += s & kCountMask;
+        if (flag == kFlagGlobal || look == 0) break;
+        --look;
+        spins = 0;
+      }
+      st_volatile_u32(&status[(uint64_t)tile * kSortMaxBins + d], kFlagGlobal | ((excl + total_d) & kCountMask));
+    }
+    if (timeout) { atomicOr(err, kErrInternal); scan_sh[kSortBlock / 32 + 2] = 1u; }
+    goff[d] = digit_base[d] + excl - lb;
   }
   __syncthreads();
+  if (scan_sh[kSortBlock / 32 + 2]) return;             // a wait ran out: the error flag is set, write nothing
 
   // each digit's run is contiguous in shared memory and in the output
-  for (uint32_t i = threadIdx.x; i < valid; i += kSortBlock) {
+#pragma unroll 4
+  for (uint32_t i = threadIdx.x; i < (FULL ? (uint32_t)TILE : valid); i += kSortBlock) {
     const K k = skeys[i];
     const uint32_t d = (uint32_t)(k >> shift) & mask;
     const uint32_t g = goff[d] + i;
@@ -146,28 +243,41 @@ __global__ void __launch_bounds__(kSortBlock) k_sort_scatter(const K* __restrict
   }
 }
 
-template <typename K>
-constexpr size_t sort_scatter_smem() {
-  return (sizeof(K) + 4) * (size_t)sort_tile<K>() + 4 * (size_t)(kSortWarps * kSortMaxBins + 2 * kSortMaxBins + kSortBlock / 32 + 1);
+// One pass.  status[tile*256 + d]: 0 = not ready, kFlagLocal|count = this tile's count of digit d,
+// kFlagGlobal|count = count summed over tiles 0..tile.  ticket: one counter per pass, starts at 0.
+template <typename K, int BITS>
+__global__ void __launch_bounds__(kSortBlock, sizeof(K) == 4 ? XLOG_SORT_MINB : XLOG_SORT_MINB / 2) k_sort_pass(const K* __restrict__ keys_in, const uint32_t* __restrict__ vals_in,
+                                                          K* __restrict__ keys_out, uint32_t* __restrict__ vals_out, uint32_t n,
+                                                          int shift, const uint32_t* __restrict__ digit_base,
+                                                          uint32_t* __restrict__ status, uint32_t* __restrict__ ticket,
+                                                          uint32_t* __restrict__ err) {
+  constexpr int ITEMS = SortCfg<K>::items;
+  constexpr int TILE = kSortBlock * ITEMS;
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  K* skeys = reinterpret_cast<K*>(smem_raw);                                   // TILE keys
+  uint32_t* svals = reinterpret_cast<uint32_t*>(smem_raw + sizeof(K) * TILE);  // TILE payloads
+  uint32_t* whist = svals + TILE;                                              // [kSortWarps][256]
+  uint32_t* lbase = whist + kSortWarps * kSortMaxBins;                         // [256] tile-local start of each digit
+  uint32_t* goff = lbase + kSortMaxBins;                                       // [256] global start minus local start
+  uint32_t* scan_sh = goff + kSortMaxBins;                                     // block scan scratch + ticket + abort flag
+
+  if (threadIdx.x == 0) { scan_sh[kSortBlock / 32 + 1] = atomicAdd(ticket, 1u); scan_sh[kSortBlock / 32 + 2] = 0u; }
+  for (int i = threadIdx.x; i < kSortWarps * (1 << BITS); i += kSortBlock) whist[(i >> BITS) * kSortMaxBins + (i & ((1 << BITS) - 1))] = 0;
+  __syncthreads();
+  const uint32_t tile = scan_sh[kSortBlock / 32 + 1];
+  const uint64_t base = (uint64_t)tile * TILE;
+  const uint32_t valid = (uint32_t)min((uint64_t)TILE, (uint64_t)n - base);
+  if (valid == (uint32_t)TILE)
+    sort_tile_body<K, BITS, true>(keys_in, vals_in, keys_out, vals_out, base, valid, tile, shift, digit_base, status, err, skeys, svals,
+                                  whist, lbase, goff, scan_sh);
+  else
+    sort_tile_body<K, BITS, false>(keys_in, vals_in, keys_out, vals_out, base, valid, tile, shift, digit_base, status, err, skeys, svals,
+                                   whist, lbase, goff, scan_sh);
 }
 
-struct SortPlan {
-  int passes;
-  int bits_per_pass;
-  uint32_t ntiles;
-  size_t hist_entries;       // uint32 entries of scratch for the histogram matrix (reused every pass)
-  size_t scan_tiles;         // uint32 entries of scratch for the scan spine
-};
-
 template <typename K>
-inline SortPlan make_sort_plan(uint64_t n, int nbits) {
-  SortPlan p;
-  p.passes = (nbits + 7) / 8;
-  p.bits_per_pass = p.passes ? (nbits + p.passes - 1) / p.passes : 0;
-  p.ntiles = (uint32_t)((n + sort_tile<K>() - 1) / sort_tile<K>());
-  p.hist_entries = (size_t)kSortMaxBins * p.ntiles;
-  p.scan_tiles = (p.hist_entries + kScanTile - 1) / kScanTile;
-  return p;
+constexpr size_t sort_pass_smem() {
+  return (sizeof(K) + 4) * (size_t)sort_tile<K>() + 4 * (size_t)(kSortWarps * kSortMaxBins + 2 * kSortMaxBins + kSortBlock / 32 + 4);
 }
 
 }  // namespace xlog

@@ -25,6 +25,18 @@ xlog_status guarded(xlog_ctx* c, F&& f) {
   }
 }
 
+// the sort pass needs more than 48 KB of dynamic shared memory and the largest carve-out
+template <typename K, int B>
+void set_sort_attributes_b() {
+  XLOG_CUDA(cudaFuncSetAttribute(k_sort_pass<K, B>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_pass_smem<K>()));
+  XLOG_CUDA(cudaFuncSetAttribute(k_sort_pass<K, B>, cudaFuncAttributePreferredSharedMemoryCarveout, 100));
+}
+template <typename K>
+void set_sort_attributes() {
+  set_sort_attributes_b<K, 1>(); set_sort_attributes_b<K, 2>(); set_sort_attributes_b<K, 3>(); set_sort_attributes_b<K, 4>();
+  set_sort_attributes_b<K, 5>(); set_sort_attributes_b<K, 6>(); set_sort_attributes_b<K, 7>(); set_sort_attributes_b<K, 8>();
+}
+
 Relation& rel_of(Ctx* c, xlog_rel r) {
   if (r < 0 || r >= (int)c->rels.size()) fail(XLOG_ERR_INVALID_ARGUMENT, "bad relation handle");
   return *c->rels[r];
@@ -68,7 +80,7 @@ void ensure_soa(Ctx* c, Relation& R) {
     R.cols[i] = DevBuf(c, (size_t)std::max(R.n, 1u) * 4);
     out.c[i] = R.cols[i].as<int32_t>();
   }
-  if (R.n) DISPATCH_K(R.key_bytes, XLOG_LAUNCH(c, (k_unpack<K>), grid_for(R.n, 256), 256, 0, (const K*)R.keys(), (int64_t)R.n, R.layout, out));
+  if (R.n) DISPATCH_K(R.key_bytes, XLOG_LAUNCH(c, (k_unpack<K>), grid_for(R.n, 256), 256, 0, (const K*)R.keys(), (int64_t)R.n, R.layout, R.dicts(), out));
   R.soa_valid = true;
 }
 
@@ -80,10 +92,10 @@ void relayout_facts(Ctx* c, Relation& R, const KeyLayout& L) {
     ColPtrsMut tmp{}; ColPtrs tmpc{};
     DevBuf cols[kMaxArity];
     for (int i = 0; i < R.arity; ++i) { cols[i] = DevBuf(c, (size_t)R.n_facts * 4); tmp.c[i] = cols[i].as<int32_t>(); tmpc.c[i] = tmp.c[i]; }
-    DISPATCH_K(R.key_bytes, XLOG_LAUNCH(c, (k_unpack<K>), grid_for(R.n_facts, 256), 256, 0, R.fact_keys.as<K>(), (int64_t)R.n_facts, R.layout, tmp));
+    DISPATCH_K(R.key_bytes, XLOG_LAUNCH(c, (k_unpack<K>), grid_for(R.n_facts, 256), 256, 0, R.fact_keys.as<K>(), (int64_t)R.n_facts, R.layout, DictSet{}, tmp));
     DevBuf nk(c, (size_t)R.n_facts * nkb);
     DISPATCH_K(nkb, XLOG_LAUNCH(c, (k_pack<K>), grid_for(R.n_facts, 256), 256, 0, tmpc, R.fact_tags.as<float>(), (int64_t)R.n_facts, L,
-                                 0.f, nk.as<K>(), R.fact_tags.as<float>()));
+                                 DictSet{}, 0.f, nk.as<K>(), R.fact_tags.as<float>()));
     XLOG_CUDA(cudaStreamSynchronize(c->stream));
     R.fact_keys = std::move(nk);
   }
@@ -94,13 +106,13 @@ void relayout_facts(Ctx* c, Relation& R, const KeyLayout& L) {
 
 // ---- load ------------------------------------------------------------------------
 void load_relation(Ctx* c, Relation& R, const int32_t* const* cols, const float* tags, int64_t n, xlog_memspace space) {
-  if (n < 0 || n > (int64_t)1 << 31) fail(XLOG_ERR_CAPACITY_EXCEEDED, "row count must be in [0, 2^31]");
+  if (n < 0 || n > (int64_t)kSortMaxN) fail(XLOG_ERR_CAPACITY_EXCEEDED, "row count must be in [0, 2^30)");
   if (n > 0 && !cols) fail(XLOG_ERR_INVALID_ARGUMENT, "cols is NULL");
   // drop everything the relation held
   drop_current(R);
   R.fact_keys.reset(); R.fact_tags.reset();
   R.n_facts = R.n = 0;
-  for (int i = 0; i < kMaxArity; ++i) R.col_max[i] = 0;
+  for (int i = 0; i < kMaxArity; ++i) { R.col_max[i] = R.fact_max[i] = R.val_max[i] = 0; R.dict[i].reset(); R.dict_n[i] = 0; }
   R.layout = make_layout(R.arity, R.col_max);
   R.key_bytes = 4;
   c->idb_dirty = true;
@@ -135,7 +147,7 @@ void load_relation(Ctx* c, Relation& R, const int32_t* const* cols, const float*
               reinterpret_cast<int32_t*>(c->d_ctrl + kSlotA), ctrl_u32(c, kSlotErr));
   sync_ctrl(c);
   const int32_t* mx = reinterpret_cast<const int32_t*>(c->h_ctrl + kSlotA);
-  for (int i = 0; i < R.arity; ++i) R.col_max[i] = mx[i];
+  for (int i = 0; i < R.arity; ++i) R.col_max[i] = R.fact_max[i] = R.val_max[i] = mx[i];
   zero_ctrl(c, kSlotA, 4);
   R.layout = make_layout(R.arity, R.col_max);
   if (R.layout.total_bits > 64) fail(XLOG_ERR_CAPACITY_EXCEEDED, "packed key of relation '" + R.name + "' needs more than 64 bits");
@@ -144,7 +156,7 @@ void load_relation(Ctx* c, Relation& R, const int32_t* const* cols, const float*
   // pack -> sort -> combine duplicates
   DISPATCH_K(R.key_bytes, {
     DevBuf k0(c, (size_t)n * sizeof(K)), t0(c, (size_t)n * 4), k1(c, (size_t)n * sizeof(K)), t1(c, (size_t)n * 4);
-    XLOG_LAUNCH(c, (k_pack<K>), grid_for(n, 256), 256, 0, in, dtags, n, R.layout, one_of(R.sr), k0.as<K>(), t0.as<float>());
+    XLOG_LAUNCH(c, (k_pack<K>), grid_for(n, 256), 256, 0, in, dtags, n, R.layout, DictSet{}, one_of(R.sr), k0.as<K>(), t0.as<float>());
     for (int i = 0; i < kMaxArity; ++i) stage[i].reset();
     stage_t.reset();
     KeyTags kt = sort_reduce<K>(c, R.sr, k0, t0, k1, t1, (uint64_t)n, R.layout.total_bits, false);
@@ -247,7 +259,7 @@ Index& ensure_index(Ctx* c, Relation& R, int col) {
   if (ix.valid) return ix;
   ensure_soa(c, R);
   ix = Index();
-  ix.domain = (int64_t)R.col_max[col] + 1;
+  ix.domain = (int64_t)R.val_max[col] + 1;
   ix.n_other = R.arity - 1;
   const int32_t* lead = nullptr;
   if (col == 0 || R.n == 0) {
@@ -261,7 +273,7 @@ Index& ensure_index(Ctx* c, Relation& R, int col) {
     perm[0] = col;
     { int k = 1; for (int i = 0; i < R.arity; ++i) if (i != col) perm[k++] = i; }
     int32_t pmax[kMaxArity] = {0, 0, 0, 0};
-    for (int i = 0; i < R.arity; ++i) pmax[i] = R.col_max[perm[i]];
+    for (int i = 0; i < R.arity; ++i) pmax[i] = R.val_max[perm[i]];
     const KeyLayout PL = make_layout(R.arity, pmax);
     const int kb = PL.total_bits <= 32 ? 4 : 8;
     ColPtrs in{};
@@ -271,14 +283,14 @@ Index& ensure_index(Ctx* c, Relation& R, int col) {
     ix.own_tags = DevBuf(c, (size_t)R.n * 4);
     DISPATCH_K(kb, {
       DevBuf k0(c, (size_t)R.n * sizeof(K)), t0(c, (size_t)R.n * 4), k1(c, (size_t)R.n * sizeof(K)), t1(c, (size_t)R.n * 4);
-      XLOG_LAUNCH(c, (k_pack<K>), grid_for(R.n, 256), 256, 0, in, (const float*)R.tags(), (int64_t)R.n, PL, 0.f, k0.as<K>(), t0.as<float>());
+      XLOG_LAUNCH(c, (k_pack<K>), grid_for(R.n, 256), 256, 0, in, (const float*)R.tags(), (int64_t)R.n, PL, DictSet{}, 0.f, k0.as<K>(), t0.as<float>());
       K* ka = k0.as<K>(); K* kbuf = k1.as<K>();
       float* ta = t0.as<float>(); float* tb = t1.as<float>();
       sort_pairs<K>(c, ka, ta, kbuf, tb, R.n, PL.total_bits);
       ColPtrsMut out{};
       out.c[0] = lead_buf.as<int32_t>();
       for (int i = 1; i < R.arity; ++i) out.c[i] = ix.own_cols[i - 1].as<int32_t>();
-      XLOG_LAUNCH(c, (k_unpack<K>), grid_for(R.n, 256), 256, 0, (const K*)ka, (int64_t)R.n, PL, out);
+      XLOG_LAUNCH(c, (k_unpack<K>), grid_for(R.n, 256), 256, 0, (const K*)ka, (int64_t)R.n, PL, DictSet{}, out);
       XLOG_CUDA(cudaMemcpyAsync(ix.own_tags.p, ta, (size_t)R.n * 4, cudaMemcpyDeviceToDevice, c->stream));
       XLOG_CUDA(cudaStreamSynchronize(c->stream));
     });
@@ -340,6 +352,29 @@ JoinSpec make_spec(Ctx* c, const Variant& v, const Relation& H) {
       S.inner_add[i] = B.args[ix.other_src[i]].add;
     }
     S.inner_tag = ix.tags;
+  }
+  // dictionaries: the outer relation's codes are turned into values when a variable is bound, and head
+  // values are ranked into codes, unless a variable only carries a column of the head relation
+  // itself through unchanged (then the code is passed along untouched)
+  const Relation& RA = *c->rels[A.rel];
+  S.outer_dict = RA.dicts();
+  S.head_dict = H.dicts();
+  for (int i = 0; i < kMaxArity; ++i) { S.outer_decode[i] = i < RA.arity && RA.dict_n[i] ? 1 : 0; S.head_encode[i] = i < p.n_head_cols && H.dict_n[i] ? 1 : 0; }
+  for (int i = 0; i < RA.arity; ++i) {
+    if (!RA.dict_n[i] || !is_plain_var(A.args[i])) continue;
+    const int v = A.args[i].var;
+    int uses = 0;
+    for (int j = 0; j < p.n_atoms; ++j)
+      for (int k = 0; k < c->rels[p.atoms[j].rel]->arity; ++k)
+        if (p.atoms[j].args[k].kind == XLOG_ARG_VAR && p.atoms[j].args[k].var == v) ++uses;
+    bool pass = uses == 1 && A.rel == p.head_rel;
+    for (int h = 0; h < p.n_head_cols && pass; ++h) {
+      if (p.head[h].coef[v] == 0) continue;
+      bool identity = h == i && p.head[h].c0 == 0 && p.head[h].coef[v] == 1;
+      for (int k = 0; k < kMaxVars; ++k) if (k != v && p.head[h].coef[k] != 0) identity = false;
+      pass = identity;
+    }
+    if (pass) { S.outer_decode[i] = 0; S.head_encode[i] = 0; }
   }
   S.head = H.layout;
   if (p.emit_count_column) {             // candidates are keyed by the declared head columns only
@@ -420,10 +455,13 @@ KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Sour
   const size_t per = (size_t)(ckb + 4) * 2;                                  // two buffers per candidate (sort ping-pong)
   uint64_t cap = total;
   if (c->chunk_bytes) cap = std::min<uint64_t>(cap, std::max<uint64_t>(1, c->chunk_bytes / per));
-  cap = std::min<uint64_t>(cap, (uint64_t)1 << 31);
+  cap = std::min<uint64_t>(cap, (uint64_t)kSortMaxN);
   {
-    const uint64_t fit = c->arena.largest_free() / (per + 1) ;                // leave room for sort scratch
-    if (fit < cap) cap = std::max<uint64_t>(std::min<uint64_t>(fit, cap), 1);
+    // besides the two candidate buffers a batch needs sort status words (1/4 B per row), the reduce's
+    // spill tables (up to 2 B per row) and a few MB of per-group arrays
+    const size_t free_bytes = c->arena.largest_free();
+    const uint64_t fit = free_bytes > (6u << 20) ? (free_bytes - (6u << 20)) / (per + 3) : 1;
+    if (fit < cap) cap = std::max<uint64_t>(fit, 1);
   }
   if (want_head_pos && cap < total) fail(XLOG_ERR_RESOURCE_EXHAUSTED, "a counted aggregate must fit one candidate batch");
 
@@ -490,12 +528,25 @@ std::vector<std::vector<int>> components(Ctx* c) {
   return out;
 }
 
-// Upper bounds of every column of every relation (loaded maxima pushed through the rules),
-// which fix the packed-key layouts before any kernel runs.
+// Sorted distinct values of column `col` of (non-derived) relation S: the dictionary of a head column fed by it.
+DevBuf distinct_values(Ctx* c, Relation& S, int col, uint32_t* n_out) {
+  ensure_soa(c, S);
+  const uint32_t n = S.n;
+  DevBuf k0(c, (size_t)n * 4), t0(c, (size_t)n * 4), k1(c, (size_t)n * 4), t1(c, (size_t)n * 4);
+  XLOG_CUDA(cudaMemcpyAsync(k0.p, S.cols[col].p, (size_t)n * 4, cudaMemcpyDeviceToDevice, c->stream));
+  XLOG_CUDA(cudaMemsetAsync(t0.p, 0, (size_t)n * 4, c->stream));
+  KeyTags u = sort_reduce<uint32_t>(c, XLOG_SR_MAXPLUS, k0, t0, k1, t1, n, bit_length(S.val_max[col]), false);
+  *n_out = u.n;
+  return std::move(u.keys);
+}
+
+// Upper bounds of every column of every relation (loaded maxima pushed through the rules), which fix
+// the packed-key layouts before any kernel runs; and dictionaries for head columns that only ever
+// carry values of one small stored column (e.g. reach(s, .) with s drawn from 64 sources).
 void propagate_bounds(Ctx* c) {
   const int n = (int)c->rels.size();
   std::vector<std::array<int64_t, kMaxArity>> ub(n);
-  for (int r = 0; r < n; ++r) for (int i = 0; i < kMaxArity; ++i) ub[r][i] = c->rels[r]->n_facts ? c->rels[r]->col_max[i] : 0;
+  for (int r = 0; r < n; ++r) for (int i = 0; i < kMaxArity; ++i) ub[r][i] = c->rels[r]->n_facts ? c->rels[r]->fact_max[i] : 0;
   for (int round = 0; round < n + 3; ++round) {
     bool changed = false;
     for (const RuleC& rc : c->rules) {
@@ -525,8 +576,45 @@ void propagate_bounds(Ctx* c) {
     Relation& R = *c->rels[r];
     if (!R.is_head) continue;
     int32_t mx[kMaxArity] = {0, 0, 0, 0};
-    for (int i = 0; i < R.arity; ++i) mx[i] = (int32_t)ub[r][i];
-    // a trailing count column is sized when its values are known
+    for (int i = 0; i < R.arity; ++i) { mx[i] = (int32_t)ub[r][i]; R.val_max[i] = mx[i]; R.dict[i].reset(); R.dict_n[i] = 0; }
+    // dictionary candidates: every rule writes the column as a bare variable that is bound either by the
+    // same column of this relation (carried along) or by a column of a stored, non-derived relation
+    bool plain_rules = R.n_facts == 0;
+    for (const RuleC& rc : c->rules) if (rc.plan.head_rel == r && (rc.kind == 3 || rc.plan.emit_count_column)) plain_rules = false;
+    for (int col = 0; col < R.arity && plain_rules; ++col) {
+      int src_rel = -1, src_col = -1;
+      bool ok = true;
+      for (const RuleC& rc : c->rules) {
+        const xlog_plan& p = rc.plan;
+        if (p.head_rel != r) continue;
+        int v = -1;
+        bool identity = p.head[col].c0 == 0;
+        for (int k = 0; k < XLOG_MAX_VARS; ++k) if (p.head[col].coef[k] != 0) { if (v >= 0 || p.head[col].coef[k] != 1) identity = false; v = k; }
+        if (!identity || v < 0) { ok = false; break; }
+        // where the variable comes from: a carry of this very column, else the smallest stored relation binding it plainly
+        bool carried = false;
+        int best_rel = -1, best_col = -1;
+        for (int j = 0; j < p.n_atoms; ++j)
+          for (int k = 0; k < c->rels[p.atoms[j].rel]->arity; ++k) {
+            const xlog_arg& g = p.atoms[j].args[k];
+            if (g.kind != XLOG_ARG_VAR || g.var != v || g.mul != 1 || g.add != 0) continue;
+            if (p.atoms[j].rel == r && k == col) carried = true;
+            else if (!c->rels[p.atoms[j].rel]->is_head && (best_rel < 0 || c->rels[p.atoms[j].rel]->n < c->rels[best_rel]->n)) { best_rel = p.atoms[j].rel; best_col = k; }
+          }
+        if (carried && best_rel < 0) continue;                         // pure carry: adds no values
+        if (best_rel < 0) { ok = false; break; }
+        if (src_rel >= 0 && (src_rel != best_rel || src_col != best_col)) { ok = false; break; }   // one source column only
+        src_rel = best_rel; src_col = best_col;
+      }
+      if (!ok || src_rel < 0) continue;
+      Relation& S = *c->rels[src_rel];
+      // worth it only if the codes are clearly narrower than the values
+      if (S.n == 0 || S.n > (1u << 16) || bit_length((int64_t)S.n - 1) + 2 > bit_length(mx[col])) continue;
+      uint32_t dn = 0;
+      R.dict[col] = distinct_values(c, S, src_col, &dn);
+      R.dict_n[col] = dn;
+      mx[col] = (int32_t)dn - 1;
+    }
     const KeyLayout L = make_layout(R.arity, mx);
     if (L.total_bits > 64) fail(XLOG_ERR_CAPACITY_EXCEEDED, "packed key of relation '" + R.name + "' needs more than 64 bits");
     for (int i = 0; i < R.arity; ++i) R.col_max[i] = mx[i];
@@ -814,8 +902,8 @@ xlog_status xlog_ctx_create(const xlog_config* cfg, xlog_ctx** out) {
     XLOG_CUDA(cudaMemsetAsync(c->d_ctrl, 0, kCtrlSlots * sizeof(uint64_t), c->stream));
     XLOG_CUDA(cudaEventCreate(&c->ev0));
     XLOG_CUDA(cudaEventCreate(&c->ev1));
-    XLOG_CUDA(cudaFuncSetAttribute(k_sort_scatter<uint32_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_scatter_smem<uint32_t>()));
-    XLOG_CUDA(cudaFuncSetAttribute(k_sort_scatter<uint64_t>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sort_scatter_smem<uint64_t>()));
+    set_sort_attributes<uint32_t>();
+    set_sort_attributes<uint64_t>();
     XLOG_CUDA(cudaStreamSynchronize(c->stream));
   });
   if (st != XLOG_OK) { if (c->h_ctrl) cudaFreeHost(c->h_ctrl); delete c; return st; }
@@ -950,6 +1038,25 @@ xlog_status xlog_fixpoint(xlog_ctx* c, xlog_receipt* receipt) {
     receipt->device_ms = ms;
   }
   return st;
+}
+
+xlog_status xlog_sort_pairs(xlog_ctx* c, void* keys, void* payload, int64_t n, int32_t key_bytes, int32_t key_bits) {
+  return guarded(c, [&] {
+    if (n < 0 || (n > 0 && (!keys || !payload)) || (key_bytes != 4 && key_bytes != 8) || key_bits < 0 || key_bits > key_bytes * 8)
+      fail(XLOG_ERR_INVALID_ARGUMENT, "xlog_sort_pairs: bad argument");
+    if (n <= 1) return;
+    DevBuf k1(c, (size_t)n * key_bytes), t1(c, (size_t)n * 4);
+    DISPATCH_K(key_bytes, {
+      K* ka = (K*)keys; K* kb = k1.as<K>();
+      float* ta = (float*)payload; float* tb = t1.as<float>();
+      sort_pairs<K>(c, ka, ta, kb, tb, (uint64_t)n, key_bits);
+      if ((void*)ka != keys) {
+        XLOG_CUDA(cudaMemcpyAsync(keys, ka, (size_t)n * key_bytes, cudaMemcpyDeviceToDevice, c->stream));
+        XLOG_CUDA(cudaMemcpyAsync(payload, ta, (size_t)n * 4, cudaMemcpyDeviceToDevice, c->stream));
+      }
+    });
+    sync_ctrl(c);
+  });
 }
 
 xlog_status xlog_profile_read(xlog_ctx* c, xlog_kernel_stat* out, int32_t capacity, int32_t* n_out) {

@@ -25,7 +25,7 @@ FLAG_PROFILE = 2
 EXPORTS = ["xlog_ctx_create", "xlog_ctx_destroy", "xlog_last_error", "xlog_relation_create", "xlog_relation_load",
            "xlog_relation_size", "xlog_relation_read", "xlog_relation_view", "xlog_rule_add", "xlog_fixpoint",
            "xlog_ctx_reset_idb", "xlog_rule_backward", "xlog_profile_read", "xlog_profile_reset",
-           "xlog_reduce_by_key_static"]
+           "xlog_reduce_by_key_static", "xlog_sort_pairs"]
 
 
 class XlogError(RuntimeError):
@@ -101,6 +101,7 @@ def lib():
         L.xlog_rule_backward.argtypes = [vp, i32, vp, C.POINTER(vp)]
         L.xlog_profile_read.argtypes = [vp, C.POINTER(KernelStat), i32, C.POINTER(i32)]
         L.xlog_profile_reset.argtypes = [vp]
+        L.xlog_sort_pairs.argtypes = [vp, vp, vp, i64, i32, i32]
         L.xlog_reduce_by_key_static.argtypes = [vp, i32, vp, vp, i64, vp, vp, C.POINTER(i64), C.c_char_p, C.c_size_t]
         for name in EXPORTS:
             if name != "xlog_last_error":
@@ -268,6 +269,12 @@ class Context:
 
     def profile_reset(self):
         self._check(self._L.xlog_profile_reset(self._h))
+
+    def sort_pairs(self, keys, payload, key_bits: int):
+        """In-place stable sort of torch CUDA tensors: keys int32/int64 (non-negative), payload 4-byte."""
+        assert keys.is_contiguous() and payload.is_contiguous() and payload.element_size() == 4
+        self._check(self._L.xlog_sort_pairs(self._h, keys.data_ptr(), payload.data_ptr(), keys.numel(),
+                                            keys.element_size(), key_bits))
 
     def reset_idb(self):
         self._check(self._L.xlog_ctx_reset_idb(self._h))

@@ -47,10 +47,15 @@ def check_program(program, rel_tol=MINMAX_REL, abs_tol=0.0, expect_bit_equal=Tru
 # ---- relation store: load / read ---------------------------------------------------------
 
 @pytest.mark.parametrize("n,arity,sr", [(1, 1, "maxplus"), (7, 2, "minplus"), (5000, 2, "maxplus"),
-                                        (100_003, 2, "minplus"), (30_000, 3, "logsumexp"), (20_000, 1, "sumprod")])
+                                        (100_003, 2, "minplus"), (30_000, 3, "logsumexp"), (20_000, 1, "sumprod"),
+                                        # big enough for the high-bit sort + shared-memory table reduction, with groups
+                                        # so large that they are split and merged through the spill tables
+                                        (2_000_003, 1, "minplus"), (3_000_000, 2, "maxplus"), (1_500_000, 3, "minplus")])
 def test_load_sorts_and_combines_duplicates(n, arity, sr):
     from paper_2609_27203_b200 import xlog
     hi = [50, 300, 7, 5][:arity] if n > 10 else [3, 3, 3, 3][:arity]        # small domains force duplicates
+    if n > 1_000_000 and arity == 1:
+        hi = [5000]
     cols = [synth.randint(9, 20 + c, 0, n, hi[c]).astype(np.int32) for c in range(arity)]
     tags = (synth.normal(9, 30, n)).astype(np.float32)
     if sr == "sumprod":
@@ -158,7 +163,7 @@ def test_sssp_minplus_ladder(scale):
     check_program(W.config2(scale=scale))
 
 
-@pytest.mark.parametrize("scale,ns", [(8, 4), (12, 64), (15, 64)])
+@pytest.mark.parametrize("scale,ns", [(8, 4), (12, 64), (12, 300), (15, 64)])
 def test_multi_source_reach_ladder(scale, ns):
     check_program(W.config5(scale=scale, n_sources=ns))
 
