@@ -38,6 +38,10 @@ struct JoinSpec {
   int64_t head_c0[kMaxArity];
   int32_t head_coef[kMaxArity][kMaxVars];
   int times;                                                  // otimes: 0 = add, 1 = multiply
+  // fast shape: head key = row part + sum_j inner_col[j] * inner_mult[j]
+  int fast;
+  int32_t head_coef_outer[kMaxArity][kMaxVars];               // head_coef restricted to variables the outer atom binds
+  uint64_t inner_mult[kMaxArity - 1];
 };
 
 // Decode an outer row into variable values; false if a constant / repeated variable /
@@ -71,14 +75,20 @@ __device__ __forceinline__ bool bind_outer(const JoinSpec& S, KO key, int64_t* v
   return ok;
 }
 
-// One thread per outer row: degree (number of inner matches) and the first matching inner row.
+// One thread per outer row: degree (number of inner matches) and a 16-byte row record
+// {first matching inner row, outer tag, row part of the head key}.  In the fast shape the head key
+// is linear in the inner columns, key = rowkey + sum_j inner_col_j * inner_mult[j], so everything that
+// depends on the outer row alone (constants, outer variables, dictionary ranks, range checks) is done
+// here once per row instead of once per candidate.
 template <typename KO>
-__global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
-                                                    uint32_t* __restrict__ deg, uint32_t* __restrict__ first) {
+__global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __restrict__ okeys, const float* __restrict__ otags,
+                                                    uint32_t n_outer, uint32_t* __restrict__ deg, uint4* __restrict__ rowinfo,
+                                                    uint32_t* __restrict__ err) {
   const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n_outer) return;
   int64_t var[kMaxVars];
   uint32_t d = 0, lo = 0;
+  uint64_t rowkey = 0;
   if (bind_outer<KO>(S, okeys[i], var)) {
     if (!S.has_inner) d = 1;
     else {
@@ -91,15 +101,32 @@ __global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __rest
         d = S.inner_off[pv + 1] - lo;
       }
     }
+    if (S.fast && d) {
+      uint32_t e = 0;
+#pragma unroll
+      for (int c = 0; c < kMaxArity; ++c)
+        if (c < S.head.arity) {
+          int64_t h = S.head_c0[c];
+#pragma unroll
+          for (int v = 0; v < kMaxVars; ++v) h += (int64_t)S.head_coef_outer[c][v] * var[v];
+          if (S.head_encode[c]) {
+            const uint32_t r = dict_rank(S.head_dict.v[c], S.head_dict.n[c], h);
+            if (r >= S.head_dict.n[c] || (int64_t)S.head_dict.v[c][r] != h) { e |= kErrInternal; h = 0; } else h = r;
+          }
+          if (h < 0 || h > (int64_t)S.head.mask[c]) { e |= kErrHeadRange; h = 0; }
+          rowkey |= (uint64_t)h << S.head.shift[c];
+        }
+      if (e) atomicOr(err, e);
+    }
   }
   deg[i] = d;
-  first[i] = lo;
+  rowinfo[i] = make_uint4(lo, __float_as_uint(otags[i]), (uint32_t)rowkey, (uint32_t)(rowkey >> 32));
 }
 
 constexpr int kExpBlock = 256;
 constexpr int kExpItems = 8;
 constexpr int kExpTile = kExpBlock * kExpItems;       // candidates per block
-constexpr int kExpRows = 2048;                        // outer-row starts staged in shared memory
+constexpr int kExpRows = 2048;                        // outer rows staged in shared memory per tile
 
 // Backward pass of a logsumexp / sum rule: instead of writing the candidate, look its head row up
 // and scatter the gradient to the two body rows (Section "End-to-end training": exact gradients
@@ -115,15 +142,19 @@ struct BwdArgs {
   int lse;                      // 1: logsumexp weights, 0: sum-product
 };
 
-// Block b writes candidates [out_lo + b*kExpTile, ...).  `start` is the exclusive scan of
-// `deg` (global candidate index of each outer row's first match).
-template <typename KO, typename KH, bool BWD>
-__global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, const float* __restrict__ otags,
-                                                           uint32_t n_outer, const uint64_t* __restrict__ start,
-                                                           const uint32_t* __restrict__ first, uint64_t out_lo, uint64_t out_hi,
-                                                           KH* __restrict__ ckeys, float* __restrict__ ctags,
-                                                           uint32_t* __restrict__ err, BwdArgs bw) {
-  __shared__ uint64_t sstart[kExpRows + 1];
+enum { kExpFast = 0, kExpGeneric = 1, kExpBackward = 2 };
+
+// Block b produces candidates [out_lo + b*kExpTile, ...).  `start` is the exclusive scan of `deg`
+// (global candidate index of each outer row's first match).  The outer rows covering the tile are
+// staged in shared memory (their starts relative to the tile and their row records), so the per-
+// candidate work is a short binary search in shared memory plus the coalesced inner reads.
+template <typename KO, typename KH, int MODE>
+__global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
+                                                           const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo,
+                                                           uint64_t out_lo, uint64_t out_hi, KH* __restrict__ ckeys,
+                                                           float* __restrict__ ctags, uint32_t* __restrict__ err, BwdArgs bw) {
+  __shared__ uint32_t sstart[kExpRows];
+  __shared__ uint4 sinfo[kExpRows];
   __shared__ uint32_t srow[2];
   const uint64_t t_lo = out_lo + (uint64_t)blockIdx.x * kExpTile;
   const uint64_t t_hi = min(t_lo + kExpTile, out_hi);
@@ -142,28 +173,53 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
   const uint32_t r_lo = srow[0], r_hi = srow[1];
   const uint32_t nrows = r_hi - r_lo + 1;
   const bool staged = nrows <= kExpRows;
-  if (staged) for (uint32_t i = threadIdx.x; i < nrows; i += kExpBlock) sstart[i] = start[r_lo + i];
+  if (staged)
+    for (uint32_t i = threadIdx.x; i < nrows; i += kExpBlock) {
+      const uint64_t st = start[r_lo + i];
+      sstart[i] = st <= t_lo ? 0u : (uint32_t)(st - t_lo);      // only the first row can start before the tile
+      sinfo[i] = rowinfo[r_lo + i];
+    }
   __syncthreads();
+  const uint64_t first_start = start[r_lo];
 
   uint32_t e = 0;
-  for (uint64_t p = t_lo + threadIdx.x; p < t_hi; p += kExpBlock) {
+  for (uint32_t q = threadIdx.x; q < (uint32_t)(t_hi - t_lo); q += kExpBlock) {
+    const uint64_t p = t_lo + q;
     // row = last row in [r_lo, r_hi] with start <= p   (rows of degree 0 share a start and are skipped)
     uint32_t lo = 0, hi = nrows;
+    uint32_t row, j;
+    uint4 info;
     if (staged) {
-      while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (sstart[mid] <= p) lo = mid + 1; else hi = mid; }
+      while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (sstart[mid] <= q) lo = mid + 1; else hi = mid; }
+      row = r_lo + lo - 1;
+      j = lo == 1 ? (uint32_t)(p - first_start) : q - sstart[lo - 1];
+      info = sinfo[lo - 1];
     } else {
       while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (start[r_lo + mid] <= p) lo = mid + 1; else hi = mid; }
+      row = r_lo + lo - 1;
+      j = (uint32_t)(p - start[row]);
+      info = rowinfo[row];
     }
-    const uint32_t row = r_lo + lo - 1;
-    const uint32_t j = (uint32_t)(p - (staged ? sstart[lo - 1] : start[row]));
+    const uint32_t ir = info.x + j;
+    const float otag = __uint_as_float(info.y);
+    float itag = S.times ? 1.f : 0.f;
+    float tag = otag;
+    if (S.has_inner) {
+      itag = S.inner_tag[ir];
+      tag = S.times ? otag * itag : otag + itag;
+    }
+    if (MODE == kExpFast) {
+      KH key = (KH)(((uint64_t)info.w << 32) | info.z);
+#pragma unroll
+      for (int c = 0; c < kMaxArity - 1; ++c)
+        if (c < S.inner_free) key += (KH)(uint32_t)S.inner_col[c][ir] * (KH)S.inner_mult[c];
+      ckeys[q + (t_lo - out_lo)] = key;
+      ctags[q + (t_lo - out_lo)] = tag;
+      continue;
+    }
     int64_t var[kMaxVars];
     bind_outer<KO>(S, okeys[row], var);
-    float tag = otags[row];
-    const float otag = tag;
-    float itag = S.times ? 1.f : 0.f;
-    uint32_t ir = 0;
     if (S.has_inner) {
-      ir = first[row] + j;
 #pragma unroll
       for (int c = 0; c < kMaxArity - 1; ++c)
         if (c < S.inner_free) {
@@ -171,9 +227,6 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
 #pragma unroll
           for (int v = 0; v < kMaxVars; ++v) if (v == S.inner_var[c]) var[v] = val;
         }
-      const float it = S.inner_tag[ir];
-      itag = it;
-      tag = S.times ? tag * it : tag + it;
     }
     KH key = 0;
 #pragma unroll
@@ -189,7 +242,7 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
         if (h < 0 || h > (int64_t)S.head.mask[c]) { e |= kErrHeadRange; h = 0; }
         key |= (KH)(uint32_t)h << S.head.shift[c];
       }
-    if (!BWD) {
+    if (MODE != kExpBackward) {
       ckeys[p - out_lo] = key;
       ctags[p - out_lo] = tag;
     } else {

@@ -323,7 +323,7 @@ struct Variant {
 struct Counted {                         // a variant after count + scan
   JoinSpec spec;
   Source outer;
-  DevBuf deg, first, start, sums;
+  DevBuf deg, rowinfo, start, sums;
   uint64_t total = 0;
   int slot = 0;
 };
@@ -387,6 +387,32 @@ JoinSpec make_spec(Ctx* c, const Variant& v, const Relation& H) {
     for (int k = 0; k < kMaxVars; ++k) S.head_coef[i][k] = p.head[i].coef[k];
   }
   S.times = H.sr == XLOG_SR_SUMPROD ? 1 : 0;
+  // Fast shape: the head key is the row part plus non-negative multiples of the looked-up atom's other
+  // columns.  Needs: those columns bind bare variables; their head coefficients are >= 0; any head column
+  // they feed has a non-negative row part (c0 >= 0, outer coefficients >= 0, outer variables >= 0) and no dictionary.
+  bool outer_bound[kMaxVars] = {false};
+  for (int i = 0; i < c->rels[A.rel]->arity; ++i) if (A.args[i].kind == XLOG_ARG_VAR) outer_bound[A.args[i].var] = true;
+  bool outer_nonneg = true;
+  for (int i = 0; i < c->rels[A.rel]->arity; ++i) if (A.args[i].kind == XLOG_ARG_VAR && A.args[i].add > 0) outer_nonneg = false;
+  bool fast = true;
+  for (int h = 0; h < p.n_head_cols; ++h)
+    for (int k = 0; k < kMaxVars; ++k) S.head_coef_outer[h][k] = outer_bound[k] ? p.head[h].coef[k] : 0;
+  for (int j = 0; j < kMaxArity - 1; ++j) S.inner_mult[j] = 0;
+  if (S.has_inner) {
+    for (int j = 0; j < S.inner_free && fast; ++j) {
+      if (S.inner_add[j] != 0) fast = false;
+      uint64_t mult = 0;
+      for (int h = 0; h < p.n_head_cols && fast; ++h) {
+        const int cf = p.head[h].coef[S.inner_var[j]];
+        if (cf == 0) continue;
+        if (cf < 0 || S.head_encode[h] || H.dict_n[h] || p.head[h].c0 < 0 || !outer_nonneg) { fast = false; break; }
+        for (int k = 0; k < kMaxVars; ++k) if (outer_bound[k] && p.head[h].coef[k] < 0) fast = false;
+        mult += (uint64_t)cf << S.head.shift[h];
+      }
+      S.inner_mult[j] = mult;
+    }
+  }
+  S.fast = fast ? 1 : 0;
   return S;
 }
 
@@ -397,31 +423,37 @@ void count_variant(Ctx* c, const Variant& v, const Relation& H, Counted& q, int 
   q.slot = slot;
   const uint32_t n = v.outer.n;
   const unsigned tiles = (n + kScanTile - 1) / kScanTile;
-  q.deg = DevBuf(c, (size_t)n * 4); q.first = DevBuf(c, (size_t)n * 4);
+  q.deg = DevBuf(c, (size_t)n * 4); q.rowinfo = DevBuf(c, (size_t)n * 16);
   q.start = DevBuf(c, (size_t)n * 8); q.sums = DevBuf(c, (size_t)tiles * 8);
-  DISPATCH_K(v.outer.key_bytes, XLOG_LAUNCH(c, (k_join_count<K>), (n + 255) / 256, 256, 0, q.spec, (const K*)v.outer.keys, n,
-                                             q.deg.as<uint32_t>(), q.first.as<uint32_t>()));
+  DISPATCH_K(v.outer.key_bytes, XLOG_LAUNCH(c, (k_join_count<K>), (n + 255) / 256, 256, 0, q.spec, (const K*)v.outer.keys, v.outer.tags, n,
+                                             q.deg.as<uint32_t>(), q.rowinfo.as<uint4>(), ctrl_u32(c, kSlotErr)));
   XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)q.deg.as<uint32_t>(), (int64_t)n, q.sums.as<uint64_t>());
   XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, q.sums.as<uint64_t>(), (int64_t)tiles, (uint64_t*)(c->d_ctrl + q.slot));
   XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)q.deg.as<uint32_t>(), (int64_t)n,
               (const uint64_t*)q.sums.as<uint64_t>(), q.start.as<uint64_t>());
 }
 
-// materialise candidates [lo, hi) of a counted variant into (ckeys, ctags), or (bw != NULL) run the backward scatter
-template <bool BWD>
-void launch_expand(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, void* ckeys, float* ctags, const BwdArgs& bw) {
+// materialise candidates [lo, hi) of a counted variant into (ckeys, ctags), or (MODE == kExpBackward) run the backward scatter
+template <int MODE>
+void launch_expand_mode(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, void* ckeys, float* ctags, const BwdArgs& bw) {
   const unsigned blocks = (unsigned)((hi - lo + kExpTile - 1) / kExpTile);
   const uint64_t* st = q.start.as<uint64_t>();
-  const uint32_t* fi = q.first.as<uint32_t>();
+  const uint4* ri = q.rowinfo.as<uint4>();
   uint32_t* err = ctrl_u32(c, kSlotErr);
   if (q.outer.key_bytes == 4 && ckb == 4)
-    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint32_t, BWD>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.tags, q.outer.n, st, fi, lo, hi, (uint32_t*)ckeys, ctags, err, bw);
+    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint32_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.n, st, ri, lo, hi, (uint32_t*)ckeys, ctags, err, bw);
   else if (q.outer.key_bytes == 4)
-    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint64_t, BWD>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.tags, q.outer.n, st, fi, lo, hi, (uint64_t*)ckeys, ctags, err, bw);
+    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint64_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.n, st, ri, lo, hi, (uint64_t*)ckeys, ctags, err, bw);
   else if (ckb == 4)
-    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint32_t, BWD>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.tags, q.outer.n, st, fi, lo, hi, (uint32_t*)ckeys, ctags, err, bw);
+    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint32_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.n, st, ri, lo, hi, (uint32_t*)ckeys, ctags, err, bw);
   else
-    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint64_t, BWD>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.tags, q.outer.n, st, fi, lo, hi, (uint64_t*)ckeys, ctags, err, bw);
+    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint64_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.n, st, ri, lo, hi, (uint64_t*)ckeys, ctags, err, bw);
+}
+template <bool BWD>
+void launch_expand(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, void* ckeys, float* ctags, const BwdArgs& bw) {
+  if (BWD) launch_expand_mode<kExpBackward>(c, q, lo, hi, ckb, ckeys, ctags, bw);
+  else if (q.spec.fast) launch_expand_mode<kExpFast>(c, q, lo, hi, ckb, ckeys, ctags, bw);
+  else launch_expand_mode<kExpGeneric>(c, q, lo, hi, ckb, ckeys, ctags, bw);
 }
 
 constexpr int kSlotTotals = 16;          // uint64 candidate totals of the variants of a round
@@ -478,7 +510,7 @@ KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Sour
         launch_expand<false>(c, q, vpos, vpos + take, ckb, (char*)k0.p + fill * ckb, t0.as<float>() + fill, BwdArgs{});
         fill += take; vpos += take;
       }
-      if (vpos == q.total) { q.start.reset(); q.first.reset(); ++vi; vpos = 0; }
+      if (vpos == q.total) { q.start.reset(); q.rowinfo.reset(); ++vi; vpos = 0; }
     }
     if (!extra_done && vi == counted.size() && cap - fill >= extra->n) {
       XLOG_CUDA(cudaMemcpyAsync((char*)k0.p + fill * ckb, extra->keys, (size_t)extra->n * ckb, cudaMemcpyDeviceToDevice, c->stream));
