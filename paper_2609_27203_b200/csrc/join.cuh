@@ -155,6 +155,8 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
                                                            float* __restrict__ ctags, uint32_t* __restrict__ err, BwdArgs bw) {
   __shared__ uint32_t sstart[kExpRows];
   __shared__ uint4 sinfo[kExpRows];
+  __shared__ uint16_t srowidx[kExpTile];             // staged row of every candidate position of the tile
+  __shared__ uint32_t swarp[kExpBlock / 32];
   __shared__ uint32_t srow[2];
   const uint64_t t_lo = out_lo + (uint64_t)blockIdx.x * kExpTile;
   const uint64_t t_hi = min(t_lo + kExpTile, out_hi);
@@ -169,32 +171,60 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
     }
     srow[threadIdx.x] = lo - 1;
   }
+#pragma unroll
+  for (int i = 0; i < kExpItems; ++i) srowidx[i * kExpBlock + threadIdx.x] = 0;
   __syncthreads();
   const uint32_t r_lo = srow[0], r_hi = srow[1];
   const uint32_t nrows = r_hi - r_lo + 1;
   const bool staged = nrows <= kExpRows;
-  if (staged)
+  const uint64_t first_start = start[r_lo];
+  if (staged) {
     for (uint32_t i = threadIdx.x; i < nrows; i += kExpBlock) {
       const uint64_t st = start[r_lo + i];
-      sstart[i] = st <= t_lo ? 0u : (uint32_t)(st - t_lo);      // only the first row can start before the tile
+      const uint32_t rel = st <= t_lo ? 0u : (uint32_t)(st - t_lo);    // only the first row can start before the tile
+      sstart[i] = rel;
       sinfo[i] = rowinfo[r_lo + i];
     }
+    __syncthreads();
+    // mark the position where each row with at least one match starts (rows without matches share a start with
+    // their successor and are skipped), then a running maximum turns the marks into "row of position q"
+    for (uint32_t i = threadIdx.x; i < nrows; i += kExpBlock) {
+      const uint32_t rel = sstart[i];
+      const uint32_t nxt = i + 1 < nrows ? sstart[i + 1] : (uint32_t)(t_hi - t_lo);
+      if (i > 0 && nxt > rel) srowidx[rel] = (uint16_t)i;
+    }
+    __syncthreads();
+    uint32_t loc[kExpItems];
+    uint32_t run = 0;
+#pragma unroll
+    for (int i = 0; i < kExpItems; ++i) { run = max(run, (uint32_t)srowidx[threadIdx.x * kExpItems + i]); loc[i] = run; }
+    uint32_t incl = run;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) { const uint32_t o = __shfl_up_sync(0xffffffffu, incl, d); if ((int)lane_id() >= d) incl = max(incl, o); }
+    if (lane_id() == 31) swarp[warp_id()] = incl;
+    __syncthreads();
+    uint32_t carry = 0;
+    for (int w = 0; w < (int)warp_id(); ++w) carry = max(carry, swarp[w]);
+    const uint32_t prev = __shfl_up_sync(0xffffffffu, incl, 1);
+    if (lane_id() > 0) carry = max(carry, prev);
+#pragma unroll
+    for (int i = 0; i < kExpItems; ++i) srowidx[threadIdx.x * kExpItems + i] = (uint16_t)max(loc[i], carry);
+  }
   __syncthreads();
-  const uint64_t first_start = start[r_lo];
 
   uint32_t e = 0;
   for (uint32_t q = threadIdx.x; q < (uint32_t)(t_hi - t_lo); q += kExpBlock) {
     const uint64_t p = t_lo + q;
-    // row = last row in [r_lo, r_hi] with start <= p   (rows of degree 0 share a start and are skipped)
-    uint32_t lo = 0, hi = nrows;
     uint32_t row, j;
     uint4 info;
     if (staged) {
-      while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (sstart[mid] <= q) lo = mid + 1; else hi = mid; }
-      row = r_lo + lo - 1;
-      j = lo == 1 ? (uint32_t)(p - first_start) : q - sstart[lo - 1];
-      info = sinfo[lo - 1];
+      const uint32_t li = srowidx[q];
+      row = r_lo + li;
+      j = li == 0 ? (uint32_t)(p - first_start) : q - sstart[li];
+      info = sinfo[li];
     } else {
+      // row = last row in [r_lo, r_hi] with start <= p   (rows of degree 0 share a start and are skipped)
+      uint32_t lo = 0, hi = nrows;
       while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (start[r_lo + mid] <= p) lo = mid + 1; else hi = mid; }
       row = r_lo + lo - 1;
       j = (uint32_t)(p - start[row]);

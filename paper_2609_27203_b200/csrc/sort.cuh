@@ -86,17 +86,16 @@ __global__ void __launch_bounds__(256) k_sort_digit_hist(const K* __restrict__ k
 #pragma unroll
       for (int p = 0; p < kSortMaxPasses; ++p) {
         if (p < P.passes) {
-          // lanes sharing the digit of the first active lane are counted with one ballot (covers the
-          // skewed case: a hot key, or a high digit that is constant across the tile); the others
-          // add individually (few conflicts when digits are spread out)
+          // one shared-memory add per RUN of equal digits across the lanes: keys usually arrive in
+          // runs (sorted adjacency lists, a constant high digit), and spread-out digits conflict little
           const uint32_t d = ok ? (uint32_t)(k[u] >> P.shift[p]) & ((1u << P.bits[p]) - 1u) : 0xffffffffu;
-          const unsigned act = __ballot_sync(0xffffffffu, ok);
-          if (act) {
-            const int first = __ffs(act) - 1;
-            const uint32_t d0 = __shfl_sync(0xffffffffu, d, first);
-            const unsigned same = __ballot_sync(0xffffffffu, ok && d == d0);
-            if ((int)lane_id() == first) atomicAdd(&sh[p * kSortMaxBins + d0], (uint32_t)__popc(same));
-            else if (ok && d != d0) atomicAdd(&sh[p * kSortMaxBins + d], 1u);
+          const uint32_t dp = __shfl_up_sync(0xffffffffu, d, 1);
+          const bool head = lane_id() == 0 || d != dp;
+          const unsigned heads = __ballot_sync(0xffffffffu, head);
+          if (head && ok) {
+            const unsigned later = lane_id() == 31 ? 0u : heads >> (lane_id() + 1);
+            const uint32_t len = later ? (uint32_t)__ffs(later) : 32u - lane_id();
+            atomicAdd(&sh[p * kSortMaxBins + d], len);
           }
         }
       }
