@@ -41,7 +41,9 @@ constexpr int kSlotErr = 0;
 
 struct Ctx;
 
-// Arena allocation with scope lifetime.
+// Arena allocation with scope lifetime.  Every kernel and copy of a context is issued on its one
+// stream, so a block may be released (and handed out again) while work that uses it is still queued:
+// whatever reuses the memory is queued later and therefore runs later.
 struct DevBuf {
   Ctx* c = nullptr;
   void* p = nullptr;
@@ -336,7 +338,6 @@ inline uint32_t reduce_by_key_t(Ctx* c, const K* keys, const float* tags, uint32
   c->note_bytes = ((int64_t)n + u) * (sizeof(K) + 4);
   XLOG_LAUNCH(c, (k_rbk_emit<K, Op>), tiles, kRbkBlock, 0, keys, tags, n, heads.as<uint32_t>(), carry.as<A>(), out_keys, out_tags, hp);
   if (hp) XLOG_CUDA(cudaMemcpyAsync(hp + u, &n, 4, cudaMemcpyHostToDevice, c->stream));
-  XLOG_CUDA(cudaStreamSynchronize(c->stream));           // scratch is released on return
   return u;
 }
 template <typename K>
@@ -395,7 +396,6 @@ inline KeyTags sort_dense_reduce(Ctx* c, DevBuf& k0, DevBuf& t0, DevBuf& k1, Dev
     c->note_bytes = (int64_t)out.n * 2 * (sizeof(K) + 4);
     XLOG_LAUNCH(c, (k_dense_compact<K>), grid_for((uint64_t)G * 32, 256), 256, 0, (const K*)kb, (const float*)tb, (const uint32_t*)gstart.as<uint32_t>(),
                 (const uint32_t*)ucount.as<uint32_t>(), G, out.keys.as<K>(), out.tags.as<float>());
-    XLOG_CUDA(cudaStreamSynchronize(c->stream));
   }
   k0.reset(); t0.reset(); k1.reset(); t1.reset();
   return out;
@@ -422,7 +422,6 @@ inline KeyTags sort_reduce(Ctx* c, int sr, DevBuf& k0, DevBuf& t0, DevBuf& k1, D
   if (out.n) {
     XLOG_CUDA(cudaMemcpyAsync(out.keys.p, kb, (size_t)out.n * sizeof(K), cudaMemcpyDeviceToDevice, c->stream));
     XLOG_CUDA(cudaMemcpyAsync(out.tags.p, tb, (size_t)out.n * 4, cudaMemcpyDeviceToDevice, c->stream));
-    XLOG_CUDA(cudaStreamSynchronize(c->stream));
   }
   k0.reset(); t0.reset(); k1.reset(); t1.reset();
   return out;

@@ -144,6 +144,29 @@ struct BwdArgs {
 
 enum { kExpFast = 0, kExpGeneric = 1, kExpBackward = 2 };
 
+// One thread per tile: the first and last outer row that contribute candidates to the tile
+// (r_lo = last row with start <= tile begin, r_hi = last row with start < tile end).  Done for all
+// tiles at once so that the dependent binary-search loads of one tile overlap with those of the others.
+static __global__ void __launch_bounds__(256) k_expand_partition(const uint64_t* __restrict__ start, uint32_t n_outer, uint64_t out_lo,
+                                                                 uint64_t out_hi, uint32_t ntiles, uint2* __restrict__ tile_rows) {
+  const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= ntiles) return;
+  const uint64_t t_lo = out_lo + (uint64_t)t * kExpTile;
+  const uint64_t t_hi = min(t_lo + kExpTile, out_hi);
+  uint32_t r[2];
+#pragma unroll
+  for (int k = 0; k < 2; ++k) {
+    const uint64_t target = k == 0 ? t_lo : t_hi - 1;
+    uint32_t lo = 0, hi = n_outer;                    // upper_bound(start, target) - 1
+    while (lo < hi) {
+      const uint32_t mid = lo + ((hi - lo) >> 1);
+      if (start[mid] <= target) lo = mid + 1; else hi = mid;
+    }
+    r[k] = lo - 1;
+  }
+  tile_rows[t] = make_uint2(r[0], r[1]);
+}
+
 // Block b produces candidates [out_lo + b*kExpTile, ...).  `start` is the exclusive scan of `deg`
 // (global candidate index of each outer row's first match).  The outer rows covering the tile are
 // staged in shared memory (their starts relative to the tile and their row records), so the per-
@@ -151,30 +174,20 @@ enum { kExpFast = 0, kExpGeneric = 1, kExpBackward = 2 };
 template <typename KO, typename KH, int MODE>
 __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
                                                            const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo,
-                                                           uint64_t out_lo, uint64_t out_hi, KH* __restrict__ ckeys,
+                                                           const uint2* __restrict__ tile_rows, uint64_t out_lo, uint64_t out_hi,
+                                                           KH* __restrict__ ckeys,
                                                            float* __restrict__ ctags, uint32_t* __restrict__ err, BwdArgs bw) {
   __shared__ uint32_t sstart[kExpRows];
   __shared__ uint4 sinfo[kExpRows];
   __shared__ uint16_t srowidx[kExpTile];             // staged row of every candidate position of the tile
   __shared__ uint32_t swarp[kExpBlock / 32];
-  __shared__ uint32_t srow[2];
   const uint64_t t_lo = out_lo + (uint64_t)blockIdx.x * kExpTile;
   const uint64_t t_hi = min(t_lo + kExpTile, out_hi);
   if (t_lo >= t_hi) return;
-  // outer rows covering this tile: r_lo = last row with start <= t_lo, r_hi = last row with start < t_hi
-  if (threadIdx.x < 2) {
-    const uint64_t target = threadIdx.x == 0 ? t_lo : t_hi - 1;
-    uint32_t lo = 0, hi = n_outer;                    // upper_bound(start, target) - 1
-    while (lo < hi) {
-      const uint32_t mid = lo + ((hi - lo) >> 1);
-      if (start[mid] <= target) lo = mid + 1; else hi = mid;
-    }
-    srow[threadIdx.x] = lo - 1;
-  }
+  const uint2 tr = tile_rows[blockIdx.x];
 #pragma unroll
   for (int i = 0; i < kExpItems; ++i) srowidx[i * kExpBlock + threadIdx.x] = 0;
-  __syncthreads();
-  const uint32_t r_lo = srow[0], r_hi = srow[1];
+  const uint32_t r_lo = tr.x, r_hi = tr.y;
   const uint32_t nrows = r_hi - r_lo + 1;
   const bool staged = nrows <= kExpRows;
   const uint64_t first_start = start[r_lo];

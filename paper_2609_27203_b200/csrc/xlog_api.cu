@@ -96,7 +96,6 @@ void relayout_facts(Ctx* c, Relation& R, const KeyLayout& L) {
     DevBuf nk(c, (size_t)R.n_facts * nkb);
     DISPATCH_K(nkb, XLOG_LAUNCH(c, (k_pack<K>), grid_for(R.n_facts, 256), 256, 0, tmpc, R.fact_tags.as<float>(), (int64_t)R.n_facts, L,
                                  DictSet{}, 0.f, nk.as<K>(), R.fact_tags.as<float>()));
-    XLOG_CUDA(cudaStreamSynchronize(c->stream));
     R.fact_keys = std::move(nk);
   }
   R.layout = L;
@@ -292,13 +291,11 @@ Index& ensure_index(Ctx* c, Relation& R, int col) {
       for (int i = 1; i < R.arity; ++i) out.c[i] = ix.own_cols[i - 1].as<int32_t>();
       XLOG_LAUNCH(c, (k_unpack<K>), grid_for(R.n, 256), 256, 0, (const K*)ka, (int64_t)R.n, PL, DictSet{}, out);
       XLOG_CUDA(cudaMemcpyAsync(ix.own_tags.p, ta, (size_t)R.n * 4, cudaMemcpyDeviceToDevice, c->stream));
-      XLOG_CUDA(cudaStreamSynchronize(c->stream));
     });
     for (int i = 1; i < R.arity; ++i) ix.other[i - 1] = ix.own_cols[i - 1].as<int32_t>();
     ix.tags = ix.own_tags.as<float>();
     ix.off = DevBuf(c, ((size_t)ix.domain + 1) * 4);
     XLOG_LAUNCH(c, k_build_offsets, grid_for(ix.domain + 1, 256), 256, 0, (const int32_t*)lead_buf.as<int32_t>(), R.n, ix.domain, ix.off.as<uint32_t>());
-    XLOG_CUDA(cudaStreamSynchronize(c->stream));
     ix.valid = true;
     return ix;
   }
@@ -440,14 +437,22 @@ void launch_expand_mode(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, v
   const uint64_t* st = q.start.as<uint64_t>();
   const uint4* ri = q.rowinfo.as<uint4>();
   uint32_t* err = ctrl_u32(c, kSlotErr);
+  // all work is issued on one stream, so a scratch block may be released as soon as its last kernel is queued:
+  // whatever reuses the memory runs later in stream order
+  DevBuf tile_rows(c, (size_t)blocks * 8);
+  const int64_t bytes = c->note_bytes;
+  c->note_bytes = 0;
+  XLOG_LAUNCH(c, k_expand_partition, (blocks + 255) / 256, 256, 0, st, q.outer.n, lo, hi, blocks, tile_rows.as<uint2>());
+  const uint2* tr = tile_rows.as<uint2>();
+  c->note_bytes = bytes;
   if (q.outer.key_bytes == 4 && ckb == 4)
-    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint32_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.n, st, ri, lo, hi, (uint32_t*)ckeys, ctags, err, bw);
+    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint32_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.n, st, ri, tr, lo, hi, (uint32_t*)ckeys, ctags, err, bw);
   else if (q.outer.key_bytes == 4)
-    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint64_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.n, st, ri, lo, hi, (uint64_t*)ckeys, ctags, err, bw);
+    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint64_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.n, st, ri, tr, lo, hi, (uint64_t*)ckeys, ctags, err, bw);
   else if (ckb == 4)
-    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint32_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.n, st, ri, lo, hi, (uint32_t*)ckeys, ctags, err, bw);
+    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint32_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.n, st, ri, tr, lo, hi, (uint32_t*)ckeys, ctags, err, bw);
   else
-    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint64_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.n, st, ri, lo, hi, (uint64_t*)ckeys, ctags, err, bw);
+    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint64_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.n, st, ri, tr, lo, hi, (uint64_t*)ckeys, ctags, err, bw);
 }
 template <bool BWD>
 void launch_expand(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, void* ckeys, float* ctags, const BwdArgs& bw) {
@@ -528,7 +533,6 @@ KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Sour
       MergeResult m;
       DISPATCH_K(ckb, m = merge<K>(c, H.sr, part.keys.as<K>(), part.tags.as<float>(), part.n, result.keys.as<K>(), result.tags.as<float>(),
                                     result.n, false, false));
-      XLOG_CUDA(cudaStreamSynchronize(c->stream));
       result = std::move(m.full);
     }
   }
@@ -681,7 +685,6 @@ void append_counts(Ctx* c, Relation& H, KeyTags& u, const KeyLayout& cl, const u
     if (kb_in == 4 && kb_out == 4) XLOG_LAUNCH(c, (k_append_count<uint32_t, uint32_t>), g, 256, 0, u.keys.as<uint32_t>(), counts, u.n, cbits, out.keys.as<uint32_t>());
     else if (kb_in == 4) XLOG_LAUNCH(c, (k_append_count<uint32_t, uint64_t>), g, 256, 0, u.keys.as<uint32_t>(), counts, u.n, cbits, out.keys.as<uint64_t>());
     else XLOG_LAUNCH(c, (k_append_count<uint64_t, uint64_t>), g, 256, 0, u.keys.as<uint64_t>(), counts, u.n, cbits, out.keys.as<uint64_t>());
-    XLOG_CUDA(cudaStreamSynchronize(c->stream));
   }
   H.layout = L;
   H.key_bytes = kb_out;
@@ -739,7 +742,6 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
   DevBuf counts(c, (size_t)std::max(u, 1u) * 4);
   DISPATCH_K(kb, XLOG_LAUNCH(c, (k_tri_compact<K>), grid_for(domain, 256), 256, 0, (const uint32_t*)flag.as<uint32_t>(), (const uint32_t*)pos.as<uint32_t>(), domain,
                               (const uint32_t*)gcnt.as<uint32_t>(), (const float*)gtag.as<float>(), kt.keys.as<K>(), counts.as<uint32_t>(), kt.tags.as<float>()));
-  XLOG_CUDA(cudaStreamSynchronize(c->stream));
   if (counted) append_counts(c, H, kt, cl, counts.as<uint32_t>(), max_count);
   else set_current(H, std::move(kt));
 }
@@ -877,7 +879,6 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
       }
       MergeResult m;
       DISPATCH_K(H.key_bytes, m = merge<K>(c, H.sr, u.keys.as<K>(), u.tags.as<float>(), u.n, (const K*)H.keys(), H.tags(), H.n, true, H.cur_owned));
-      XLOG_CUDA(cudaStreamSynchronize(c->stream));
       if (!m.in_place) set_current(H, std::move(m.full));
       c->r_new += m.n_new; c->r_improved += m.n_improved;
       changed += (uint64_t)m.n_new + m.n_improved;
