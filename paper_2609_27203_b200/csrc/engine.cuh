@@ -274,18 +274,19 @@ inline void sort_pairs(Ctx* c, K*& keys, float*& tags, K*& keys_alt, float*& tag
   const SortPasses P = make_sort_passes(low_bit, nbits);
   if (P.passes == 0) return;
   const uint32_t ntiles = (uint32_t)((n + sort_tile<K>() - 1) / sort_tile<K>());
-  // scratch: digit histograms of every pass, one ticket per pass, the look-back status words (reused by every pass)
-  const size_t head_words = (size_t)kSortMaxPasses * kSortMaxBins + kSortMaxPasses;
-  DevBuf scratch(c, (head_words + (size_t)ntiles * kSortMaxBins) * 4);
+  // scratch: digit histograms of every pass, one ticket per pass, a block counter, then the look-back status words of
+  // every pass; zeroed by one memset
+  const size_t head_words = (size_t)kSortMaxPasses * kSortMaxBins + kSortMaxPasses + 8;
+  const size_t pass_words = (size_t)ntiles * kSortMaxBins;
+  DevBuf scratch(c, (head_words + pass_words * P.passes) * 4);
   uint32_t* hist = scratch.as<uint32_t>();
   uint32_t* tickets = hist + kSortMaxPasses * kSortMaxBins;
-  uint32_t* status = hist + head_words;
-  XLOG_CUDA(cudaMemsetAsync(hist, 0, head_words * 4, c->stream));
+  uint32_t* done = tickets + kSortMaxPasses;
+  XLOG_CUDA(cudaMemsetAsync(hist, 0, (head_words + pass_words * P.passes) * 4, c->stream));
   c->note_bytes = (int64_t)n * sizeof(K);
-  XLOG_LAUNCH(c, (k_sort_digit_hist<K>), grid_for(n, 256 * 8, kSMs * 8), 256, 0, keys, (uint32_t)n, P, hist);
-  XLOG_LAUNCH(c, k_sort_digit_bases, 1, 256, 0, hist, P.passes);
+  XLOG_LAUNCH(c, (k_sort_digit_hist<K>), grid_for(n, 256 * 8, kSMs * 8), 256, 0, keys, (uint32_t)n, P, hist, done);
   for (int pass = 0; pass < P.passes; ++pass) {
-    XLOG_CUDA(cudaMemsetAsync(status, 0, (size_t)ntiles * kSortMaxBins * 4, c->stream));
+    uint32_t* status = hist + head_words + pass_words * pass;
     c->note_bytes = (int64_t)n * 2 * (sizeof(K) + 4);
 #define XLOG_SORT_PASS(B)                                                                                                          \
   XLOG_LAUNCH(c, (k_sort_pass<K, B>), ntiles, kSortBlock, sort_pass_smem<K>(), keys, reinterpret_cast<const uint32_t*>(tags), keys_alt, \
@@ -316,15 +317,14 @@ struct KeyTags {
 
 constexpr int kSlotA = 8, kSlotB = 9, kSlotC = 10, kSlotD = 11;
 
-// Reduce-by-key of a sorted list into caller-provided buffers of capacity n (typically the idle
-// half of the sort's double buffer, so nothing is allocated while the candidates are alive).
-// One control read returns the number of groups.  head_pos (optional, filled when
-// want_head_pos) gets the row index of each group's first row plus a sentinel n, so that a
-// group's size is head_pos[u+1] - head_pos[u].
+// Reduce-by-key of a sorted list.  One control read returns the number of groups; the idle buffers
+// `free_a` / `free_b` (the other half of the sort's double buffer) are released at that point, so the
+// result can be allocated at its exact size without raising the peak.  head_pos (optional) gets the row
+// index of each group's first row plus a sentinel n, so that a group's size is head_pos[u+1] - head_pos[u].
 template <typename K, typename Op>
-inline uint32_t reduce_by_key_t(Ctx* c, const K* keys, const float* tags, uint32_t n, K* out_keys, float* out_tags,
-                                DevBuf* head_pos) {
-  if (n == 0) return 0;
+inline KeyTags reduce_by_key_t(Ctx* c, const K* keys, const float* tags, uint32_t n, DevBuf* free_a, DevBuf* free_b, bool want_head_pos) {
+  KeyTags out;
+  if (n == 0) { if (free_a) free_a->reset(); if (free_b) free_b->reset(); return out; }
   typedef typename Op::A A;
   const unsigned tiles = (n + kRbkTile - 1) / kRbkTile;
   DevBuf heads(c, (size_t)tiles * 4), tails(c, (size_t)tiles * sizeof(A)), carry(c, (size_t)tiles * sizeof(A));
@@ -333,21 +333,27 @@ inline uint32_t reduce_by_key_t(Ctx* c, const K* keys, const float* tags, uint32
   XLOG_LAUNCH(c, (k_rbk_spine<Op>), 1, 1024, 0, heads.as<uint32_t>(), tails.as<A>(), carry.as<A>(), tiles, ctrl_u32(c, kSlotA));
   sync_ctrl(c);
   const uint32_t u = (uint32_t)c->h_ctrl[kSlotA];
+  if (free_a) free_a->reset();
+  if (free_b) free_b->reset();
+  out.n = u;
+  out.keys = DevBuf(c, (size_t)std::max(u, 1u) * sizeof(K));
+  out.tags = DevBuf(c, (size_t)std::max(u, 1u) * 4);
   uint32_t* hp = nullptr;
-  if (head_pos) { *head_pos = DevBuf(c, ((size_t)u + 1) * 4); hp = head_pos->as<uint32_t>(); }
+  if (want_head_pos) { out.head_pos = DevBuf(c, ((size_t)u + 1) * 4); hp = out.head_pos.as<uint32_t>(); }
   c->note_bytes = ((int64_t)n + u) * (sizeof(K) + 4);
-  XLOG_LAUNCH(c, (k_rbk_emit<K, Op>), tiles, kRbkBlock, 0, keys, tags, n, heads.as<uint32_t>(), carry.as<A>(), out_keys, out_tags, hp);
+  XLOG_LAUNCH(c, (k_rbk_emit<K, Op>), tiles, kRbkBlock, 0, keys, tags, n, heads.as<uint32_t>(), carry.as<A>(), out.keys.as<K>(),
+              out.tags.as<float>(), hp);
   if (hp) XLOG_CUDA(cudaMemcpyAsync(hp + u, &n, 4, cudaMemcpyHostToDevice, c->stream));
-  return u;
+  return out;
 }
 template <typename K>
-inline uint32_t reduce_by_key(Ctx* c, int sr, const K* keys, const float* tags, uint32_t n, K* out_keys, float* out_tags,
-                              DevBuf* head_pos = nullptr) {
+inline KeyTags reduce_by_key(Ctx* c, int sr, const K* keys, const float* tags, uint32_t n, DevBuf* free_a, DevBuf* free_b,
+                             bool want_head_pos = false) {
   switch (sr) {
-    case XLOG_SR_MAXPLUS: return reduce_by_key_t<K, OpMax>(c, keys, tags, n, out_keys, out_tags, head_pos);
-    case XLOG_SR_MINPLUS: return reduce_by_key_t<K, OpMin>(c, keys, tags, n, out_keys, out_tags, head_pos);
-    case XLOG_SR_LOGSUMEXP: return reduce_by_key_t<K, OpLse>(c, keys, tags, n, out_keys, out_tags, head_pos);
-    default: return reduce_by_key_t<K, OpSum>(c, keys, tags, n, out_keys, out_tags, head_pos);
+    case XLOG_SR_MAXPLUS: return reduce_by_key_t<K, OpMax>(c, keys, tags, n, free_a, free_b, want_head_pos);
+    case XLOG_SR_MINPLUS: return reduce_by_key_t<K, OpMin>(c, keys, tags, n, free_a, free_b, want_head_pos);
+    case XLOG_SR_LOGSUMEXP: return reduce_by_key_t<K, OpLse>(c, keys, tags, n, free_a, free_b, want_head_pos);
+    default: return reduce_by_key_t<K, OpSum>(c, keys, tags, n, free_a, free_b, want_head_pos);
   }
 }
 
@@ -408,21 +414,11 @@ inline KeyTags sort_reduce(Ctx* c, int sr, DevBuf& k0, DevBuf& t0, DevBuf& k1, D
   if (dense_reduce_applies(sr, n, nbits, want_head_pos))
     return sr == XLOG_SR_MAXPLUS ? sort_dense_reduce<K, OpMax>(c, k0, t0, k1, t1, n, nbits)
                                  : sort_dense_reduce<K, OpMin>(c, k0, t0, k1, t1, n, nbits);
-  KeyTags out;
   K* ka = k0.as<K>(); K* kb = k1.as<K>();
   float* ta = t0.as<float>(); float* tb = t1.as<float>();
   sort_pairs<K>(c, ka, ta, kb, tb, n, nbits);
-  out.n = reduce_by_key<K>(c, sr, ka, ta, (uint32_t)n, kb, tb, want_head_pos ? &out.head_pos : nullptr);
-  // the sorted input is no longer needed: free it, then move the groups into exact-size storage
   const bool sorted_in_0 = (void*)ka == k0.p;
-  (sorted_in_0 ? k0 : k1).reset();
-  (sorted_in_0 ? t0 : t1).reset();
-  out.keys = DevBuf(c, (size_t)std::max(out.n, 1u) * sizeof(K));
-  out.tags = DevBuf(c, (size_t)std::max(out.n, 1u) * 4);
-  if (out.n) {
-    XLOG_CUDA(cudaMemcpyAsync(out.keys.p, kb, (size_t)out.n * sizeof(K), cudaMemcpyDeviceToDevice, c->stream));
-    XLOG_CUDA(cudaMemcpyAsync(out.tags.p, tb, (size_t)out.n * 4, cudaMemcpyDeviceToDevice, c->stream));
-  }
+  KeyTags out = reduce_by_key<K>(c, sr, ka, ta, (uint32_t)n, sorted_in_0 ? &k1 : &k0, sorted_in_0 ? &t1 : &t0, want_head_pos);
   k0.reset(); t0.reset(); k1.reset(); t1.reset();
   return out;
 }
@@ -446,8 +442,7 @@ inline MergeResult merge_t(Ctx* c, const K* A, const float* TA, uint32_t na, con
   c->note_bytes = (int64_t)total * (sizeof(K) + 4);
   XLOG_LAUNCH(c, (k_merge<K, Op, false>), tiles, kMrgBlock, 0, A, TA, na, B, TB, nb, a_start.as<uint32_t>(), nf.as<uint32_t>(),
               nd.as<uint32_t>(), (K*)nullptr, (float*)nullptr, (K*)nullptr, (float*)nullptr, 0);
-  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, nf.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotB));
-  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, nd.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotC));
+  XLOG_LAUNCH(c, (k_scan_spine2<uint32_t>), 1, 1024, 0, nf.as<uint32_t>(), nd.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotB), ctrl_u32(c, kSlotC));
   sync_ctrl(c);
   const uint32_t tot_f = (uint32_t)c->h_ctrl[kSlotB], tot_d = (uint32_t)c->h_ctrl[kSlotC];
   r.n_new = tot_f - nb;

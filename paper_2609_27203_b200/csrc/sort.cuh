@@ -64,10 +64,14 @@ __device__ __forceinline__ void st_volatile_u32(uint32_t* p, uint32_t v) {
 }
 
 // hist[pass * 256 + d] += number of keys whose digit of `pass` is d.  Persistent grid.
+// The block that finishes last turns every pass's counts into exclusive bases in place
+// (hist[pass*256 + d] = number of keys with a smaller digit in that pass).  `done` starts at 0.
 template <typename K>
 __global__ void __launch_bounds__(256) k_sort_digit_hist(const K* __restrict__ keys, uint32_t n, SortPasses P,
-                                                         uint32_t* __restrict__ hist) {
+                                                         uint32_t* __restrict__ hist, uint32_t* __restrict__ done) {
   __shared__ uint32_t sh[kSortMaxPasses * kSortMaxBins];
+  __shared__ uint32_t s_last;
+  __shared__ uint32_t scan_sh[256 / 32 + 1];
   for (int i = threadIdx.x; i < P.passes * kSortMaxBins; i += blockDim.x) sh[i] = 0;
   __syncthreads();
   // each block takes chunks of 256*8 keys; a thread issues its 8 loads before it touches any of them
@@ -104,15 +108,16 @@ __global__ void __launch_bounds__(256) k_sort_digit_hist(const K* __restrict__ k
   __syncthreads();
   for (int i = threadIdx.x; i < P.passes * kSortMaxBins; i += blockDim.x)
     if (sh[i]) atomicAdd(&hist[i], sh[i]);
-}
-
-// In place: hist[pass*256 + d] becomes the number of keys with a smaller digit in that pass.
-static __global__ void __launch_bounds__(256) k_sort_digit_bases(uint32_t* __restrict__ hist, int passes) {
-  __shared__ uint32_t sh[256 / 32 + 1];
-  for (int p = 0; p < passes; ++p) {
-    const uint32_t v = hist[p * kSortMaxBins + threadIdx.x];
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(done, 1u) == gridDim.x - 1 ? 1u : 0u;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  for (int p = 0; p < P.passes; ++p) {
+    const uint32_t v = __ldcg(&hist[p * kSortMaxBins + threadIdx.x]);
     uint32_t total;
-    const uint32_t e = block_scan_excl<256, uint32_t>(v, sh, total);
+    const uint32_t e = block_scan_excl<256, uint32_t>(v, scan_sh, total);
     hist[p * kSortMaxBins + threadIdx.x] = e;
   }
 }
