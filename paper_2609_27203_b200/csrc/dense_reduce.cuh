@@ -156,16 +156,19 @@ __global__ void __launch_bounds__(kDenseBlock) k_dense_reduce(const K* __restric
   if (threadIdx.x == 0) ucount[g] = total;
 }
 
-// One warp per group: copy its reduced rows from the group's offset to the dense position upos[g].
+// One thread per output row: find its group in upos (exclusive scan of the per-group row counts) and
+// copy the row from the group's offset to its final, dense position.
 template <typename K>
 __global__ void __launch_bounds__(256) k_dense_compact(const K* __restrict__ in_keys, const float* __restrict__ in_tags,
                                                        const uint32_t* __restrict__ gstart, const uint32_t* __restrict__ upos,
-                                                       uint32_t G, K* __restrict__ out_keys, float* __restrict__ out_tags) {
-  const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
-  for (uint32_t g = warp; g < G; g += nwarps) {
-    const uint32_t src = gstart[g], dst = upos[g], cnt = upos[g + 1] - dst;
-    for (uint32_t i = lane_id(); i < cnt; i += 32) { out_keys[dst + i] = in_keys[src + i]; out_tags[dst + i] = in_tags[src + i]; }
+                                                       uint32_t G, uint32_t u, K* __restrict__ out_keys, float* __restrict__ out_tags) {
+  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < u; i += gridDim.x * blockDim.x) {
+    uint32_t lo = 0, hi = G;                           // last group with upos[g] <= i
+    while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (upos[mid] <= i) lo = mid + 1; else hi = mid; }
+    const uint32_t g = lo - 1;
+    const uint32_t src = gstart[g] + (i - upos[g]);
+    out_keys[i] = in_keys[src];
+    out_tags[i] = in_tags[src];
   }
 }
 

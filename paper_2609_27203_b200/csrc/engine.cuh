@@ -400,8 +400,8 @@ inline KeyTags sort_dense_reduce(Ctx* c, DevBuf& k0, DevBuf& t0, DevBuf& k1, Dev
   out.tags = DevBuf(c, (size_t)std::max(out.n, 1u) * 4);
   if (out.n) {
     c->note_bytes = (int64_t)out.n * 2 * (sizeof(K) + 4);
-    XLOG_LAUNCH(c, (k_dense_compact<K>), grid_for((uint64_t)G * 32, 256), 256, 0, (const K*)kb, (const float*)tb, (const uint32_t*)gstart.as<uint32_t>(),
-                (const uint32_t*)ucount.as<uint32_t>(), G, out.keys.as<K>(), out.tags.as<float>());
+    XLOG_LAUNCH(c, (k_dense_compact<K>), grid_for(out.n, 256), 256, 0, (const K*)kb, (const float*)tb, (const uint32_t*)gstart.as<uint32_t>(),
+                (const uint32_t*)ucount.as<uint32_t>(), G, out.n, out.keys.as<K>(), out.tags.as<float>());
   }
   k0.reset(); t0.reset(); k1.reset(); t1.reset();
   return out;

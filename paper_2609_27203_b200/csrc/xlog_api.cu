@@ -727,6 +727,7 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
   const unsigned scan_tiles = (unsigned)((domain + kScanTile - 1) / kScanTile);
   DevBuf spine(c, ((size_t)scan_tiles + 1) * 4);
   zero_ctrl(c, kSlotA, 4);
+  c->note_bytes = (int64_t)E.n * 12 * 3;      // each edge is read as (x,y), inside an out-list and inside an in-list; partials are small
   XLOG_LAUNCH(c, (k_tri_edges<Op>), kSMs * 8, 256, 0, G, H.sr == XLOG_SR_SUMPROD ? 1 : 0, ecnt.as<uint32_t>(), eacc.as<A>());
   XLOG_LAUNCH(c, (k_tri_groups<Op>), grid_for((uint64_t)domain * 32, 256, kSMs * 8), 256, 0, G.out_off, domain, (const uint32_t*)ecnt.as<uint32_t>(),
               (const A*)eacc.as<A>(), gcnt.as<uint32_t>(), gtag.as<float>(), flag.as<uint32_t>(), ctrl_u32(c, kSlotD), ctrl_u32(c, kSlotErr));
