@@ -161,7 +161,9 @@ __global__ void __launch_bounds__(kDenseBlock) k_dense_reduce(const K* __restric
 template <typename K>
 __global__ void __launch_bounds__(256) k_dense_compact(const K* __restrict__ in_keys, const float* __restrict__ in_tags,
                                                        const uint32_t* __restrict__ gstart, const uint32_t* __restrict__ upos,
-                                                       uint32_t G, uint32_t u, K* __restrict__ out_keys, float* __restrict__ out_tags) {
+                                                       uint32_t G, const uint32_t* __restrict__ u_ptr, K* __restrict__ out_keys,
+                                                       float* __restrict__ out_tags) {
+  const uint32_t u = *u_ptr;
   for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < u; i += gridDim.x * blockDim.x) {
     uint32_t lo = 0, hi = G;                           // last group with upos[g] <= i
     while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (upos[mid] <= i) lo = mid + 1; else hi = mid; }

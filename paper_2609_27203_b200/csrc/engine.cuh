@@ -311,9 +311,11 @@ inline void sort_pairs(Ctx* c, K*& keys, float*& tags, K*& keys_alt, float*& tag
 // Sorted unique (key, tag) list in arena buffers of exact size.
 struct KeyTags {
   DevBuf keys, tags;
-  uint32_t n = 0;
+  uint32_t n = 0;                       // row count; an upper bound (the buffers' capacity) while n_slot >= 0
+  int n_slot = -1;                      // >= 0: the exact count is still on the device, in this control slot
   DevBuf head_pos;                      // optional: row index of each group head in the reduced input (+ sentinel n)
 };
+constexpr size_t kDeferBytes = 32u << 20;   // results up to this size are allocated at their upper bound to skip a control read
 
 constexpr int kSlotA = 8, kSlotB = 9, kSlotC = 10, kSlotD = 11;
 
@@ -322,7 +324,8 @@ constexpr int kSlotA = 8, kSlotB = 9, kSlotC = 10, kSlotD = 11;
 // result can be allocated at its exact size without raising the peak.  head_pos (optional) gets the row
 // index of each group's first row plus a sentinel n, so that a group's size is head_pos[u+1] - head_pos[u].
 template <typename K, typename Op>
-inline KeyTags reduce_by_key_t(Ctx* c, const K* keys, const float* tags, uint32_t n, DevBuf* free_a, DevBuf* free_b, bool want_head_pos) {
+inline KeyTags reduce_by_key_t(Ctx* c, const K* keys, const float* tags, uint32_t n, DevBuf* free_a, DevBuf* free_b, bool want_head_pos,
+                               int defer_slot) {
   KeyTags out;
   if (n == 0) { if (free_a) free_a->reset(); if (free_b) free_b->reset(); return out; }
   typedef typename Op::A A;
@@ -330,6 +333,19 @@ inline KeyTags reduce_by_key_t(Ctx* c, const K* keys, const float* tags, uint32_
   DevBuf heads(c, (size_t)tiles * 4), tails(c, (size_t)tiles * sizeof(A)), carry(c, (size_t)tiles * sizeof(A));
   c->note_bytes = (int64_t)n * (sizeof(K) + 4);
   XLOG_LAUNCH(c, (k_rbk_tiles<K, Op>), tiles, kRbkBlock, 0, keys, tags, n, heads.as<uint32_t>(), tails.as<A>());
+  if (defer_slot >= 0 && !want_head_pos && (size_t)n * (sizeof(K) + 4) <= kDeferBytes) {
+    // small result: write it into buffers of the upper-bound size n and leave the exact count on the device
+    XLOG_LAUNCH(c, (k_rbk_spine<Op>), 1, 1024, 0, heads.as<uint32_t>(), tails.as<A>(), carry.as<A>(), tiles, ctrl_u32(c, defer_slot));
+    if (free_a) free_a->reset();
+    if (free_b) free_b->reset();
+    out.n = n; out.n_slot = defer_slot;
+    out.keys = DevBuf(c, (size_t)n * sizeof(K));
+    out.tags = DevBuf(c, (size_t)n * 4);
+    c->note_bytes = (int64_t)n * 2 * (sizeof(K) + 4);
+    XLOG_LAUNCH(c, (k_rbk_emit<K, Op>), tiles, kRbkBlock, 0, keys, tags, n, heads.as<uint32_t>(), carry.as<A>(), out.keys.as<K>(),
+                out.tags.as<float>(), (uint32_t*)nullptr);
+    return out;
+  }
   XLOG_LAUNCH(c, (k_rbk_spine<Op>), 1, 1024, 0, heads.as<uint32_t>(), tails.as<A>(), carry.as<A>(), tiles, ctrl_u32(c, kSlotA));
   sync_ctrl(c);
   const uint32_t u = (uint32_t)c->h_ctrl[kSlotA];
@@ -348,12 +364,12 @@ inline KeyTags reduce_by_key_t(Ctx* c, const K* keys, const float* tags, uint32_
 }
 template <typename K>
 inline KeyTags reduce_by_key(Ctx* c, int sr, const K* keys, const float* tags, uint32_t n, DevBuf* free_a, DevBuf* free_b,
-                             bool want_head_pos = false) {
+                             bool want_head_pos = false, int defer_slot = -1) {
   switch (sr) {
-    case XLOG_SR_MAXPLUS: return reduce_by_key_t<K, OpMax>(c, keys, tags, n, free_a, free_b, want_head_pos);
-    case XLOG_SR_MINPLUS: return reduce_by_key_t<K, OpMin>(c, keys, tags, n, free_a, free_b, want_head_pos);
-    case XLOG_SR_LOGSUMEXP: return reduce_by_key_t<K, OpLse>(c, keys, tags, n, free_a, free_b, want_head_pos);
-    default: return reduce_by_key_t<K, OpSum>(c, keys, tags, n, free_a, free_b, want_head_pos);
+    case XLOG_SR_MAXPLUS: return reduce_by_key_t<K, OpMax>(c, keys, tags, n, free_a, free_b, want_head_pos, defer_slot);
+    case XLOG_SR_MINPLUS: return reduce_by_key_t<K, OpMin>(c, keys, tags, n, free_a, free_b, want_head_pos, defer_slot);
+    case XLOG_SR_LOGSUMEXP: return reduce_by_key_t<K, OpLse>(c, keys, tags, n, free_a, free_b, want_head_pos, defer_slot);
+    default: return reduce_by_key_t<K, OpSum>(c, keys, tags, n, free_a, free_b, want_head_pos, defer_slot);
   }
 }
 
@@ -367,7 +383,7 @@ inline bool dense_reduce_applies(int sr, uint64_t n, int nbits, bool want_head_p
 }
 
 template <typename K, typename Op>
-inline KeyTags sort_dense_reduce(Ctx* c, DevBuf& k0, DevBuf& t0, DevBuf& k1, DevBuf& t1, uint64_t n, int nbits) {
+inline KeyTags sort_dense_reduce(Ctx* c, DevBuf& k0, DevBuf& t0, DevBuf& k1, DevBuf& t1, uint64_t n, int nbits, int defer_slot) {
   KeyTags out;
   K* ka = k0.as<K>(); K* kb = k1.as<K>();
   float* ta = t0.as<float>(); float* tb = t1.as<float>();
@@ -389,10 +405,25 @@ inline KeyTags sort_dense_reduce(Ctx* c, DevBuf& k0, DevBuf& t0, DevBuf& k1, Dev
   XLOG_LAUNCH(c, (k_dense_reduce<K, Op>), max_items, kDenseBlock, 0, (const K*)ka, (const float*)ta, L, G, part,
               (const uint32_t*)gstart.as<uint32_t>(), (const uint32_t*)part_base.as<uint32_t>(), (const uint32_t*)spill.as<uint32_t>(), spill_cap,
               spill_tab.as<int32_t>(), done.as<uint32_t>(), kb, tb, ucount.as<uint32_t>());
+  const bool sorted_in_0 = (void*)ka == k0.p;
+  const uint64_t ucap = std::min<uint64_t>(n, nbits >= 32 ? n : ((uint64_t)1 << nbits));
+  if (defer_slot >= 0 && ucap * (sizeof(K) + 4) <= kDeferBytes) {
+    // small result: compact into buffers of the upper-bound size and leave the exact count on the device
+    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, ucount.as<uint32_t>(), (int64_t)G + 1, ctrl_u32(c, defer_slot));
+    (sorted_in_0 ? k0 : k1).reset();
+    (sorted_in_0 ? t0 : t1).reset();
+    spill_tab.reset();
+    out.n = (uint32_t)ucap; out.n_slot = defer_slot;
+    out.keys = DevBuf(c, (size_t)ucap * sizeof(K));
+    out.tags = DevBuf(c, (size_t)ucap * 4);
+    XLOG_LAUNCH(c, (k_dense_compact<K>), grid_for(ucap, 256), 256, 0, (const K*)kb, (const float*)tb, (const uint32_t*)gstart.as<uint32_t>(),
+                (const uint32_t*)ucount.as<uint32_t>(), G, (const uint32_t*)ctrl_u32(c, defer_slot), out.keys.as<K>(), out.tags.as<float>());
+    k0.reset(); t0.reset(); k1.reset(); t1.reset();
+    return out;
+  }
   XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, ucount.as<uint32_t>(), (int64_t)G + 1, ctrl_u32(c, kSlotA));
   sync_ctrl(c);
   out.n = (uint32_t)c->h_ctrl[kSlotA];
-  const bool sorted_in_0 = (void*)ka == k0.p;
   (sorted_in_0 ? k0 : k1).reset();
   (sorted_in_0 ? t0 : t1).reset();
   spill_tab.reset();
@@ -401,7 +432,7 @@ inline KeyTags sort_dense_reduce(Ctx* c, DevBuf& k0, DevBuf& t0, DevBuf& k1, Dev
   if (out.n) {
     c->note_bytes = (int64_t)out.n * 2 * (sizeof(K) + 4);
     XLOG_LAUNCH(c, (k_dense_compact<K>), grid_for(out.n, 256), 256, 0, (const K*)kb, (const float*)tb, (const uint32_t*)gstart.as<uint32_t>(),
-                (const uint32_t*)ucount.as<uint32_t>(), G, out.n, out.keys.as<K>(), out.tags.as<float>());
+                (const uint32_t*)ucount.as<uint32_t>(), G, (const uint32_t*)ctrl_u32(c, kSlotA), out.keys.as<K>(), out.tags.as<float>());
   }
   k0.reset(); t0.reset(); k1.reset(); t1.reset();
   return out;
@@ -410,15 +441,16 @@ inline KeyTags sort_dense_reduce(Ctx* c, DevBuf& k0, DevBuf& t0, DevBuf& k1, Dev
 // Sort + reduce the first n pairs of (k0,t0) using (k1,t1) as the second half of the double
 // buffer; releases both and returns the groups in exact-size buffers.
 template <typename K>
-inline KeyTags sort_reduce(Ctx* c, int sr, DevBuf& k0, DevBuf& t0, DevBuf& k1, DevBuf& t1, uint64_t n, int nbits, bool want_head_pos) {
+inline KeyTags sort_reduce(Ctx* c, int sr, DevBuf& k0, DevBuf& t0, DevBuf& k1, DevBuf& t1, uint64_t n, int nbits, bool want_head_pos,
+                           int defer_slot = -1) {
   if (dense_reduce_applies(sr, n, nbits, want_head_pos))
-    return sr == XLOG_SR_MAXPLUS ? sort_dense_reduce<K, OpMax>(c, k0, t0, k1, t1, n, nbits)
-                                 : sort_dense_reduce<K, OpMin>(c, k0, t0, k1, t1, n, nbits);
+    return sr == XLOG_SR_MAXPLUS ? sort_dense_reduce<K, OpMax>(c, k0, t0, k1, t1, n, nbits, defer_slot)
+                                 : sort_dense_reduce<K, OpMin>(c, k0, t0, k1, t1, n, nbits, defer_slot);
   K* ka = k0.as<K>(); K* kb = k1.as<K>();
   float* ta = t0.as<float>(); float* tb = t1.as<float>();
   sort_pairs<K>(c, ka, ta, kb, tb, n, nbits);
   const bool sorted_in_0 = (void*)ka == k0.p;
-  KeyTags out = reduce_by_key<K>(c, sr, ka, ta, (uint32_t)n, sorted_in_0 ? &k1 : &k0, sorted_in_0 ? &t1 : &t0, want_head_pos);
+  KeyTags out = reduce_by_key<K>(c, sr, ka, ta, (uint32_t)n, sorted_in_0 ? &k1 : &k0, sorted_in_0 ? &t1 : &t0, want_head_pos, defer_slot);
   k0.reset(); t0.reset(); k1.reset(); t1.reset();
   return out;
 }
@@ -429,19 +461,56 @@ struct MergeResult {
   KeyTags full, delta;
   uint32_t n_new = 0, n_improved = 0;
   bool in_place = false;
+  int slot = -1;                        // >= 0: totals are still on the device (slot: merged rows, slot + 1: delta rows)
+  uint32_t nb = 0;
+  bool allow_in_place = false;
 };
+
+// Read the totals of a deferred merge from the (already synchronised) control block and settle sizes.
+inline void finish_merge(Ctx* c, MergeResult& r) {
+  if (r.slot < 0) return;
+  const uint32_t tot_f = (uint32_t)c->h_ctrl[r.slot], tot_d = (uint32_t)c->h_ctrl[r.slot + 1];
+  r.n_new = tot_f - r.nb;
+  r.n_improved = tot_d - r.n_new;
+  r.in_place = r.allow_in_place && r.n_new == 0;
+  if (r.in_place) { r.full.keys.reset(); r.full.tags.reset(); r.full.n = 0; } else r.full.n = tot_f;
+  r.delta.n = tot_d;
+  r.full.n_slot = r.delta.n_slot = -1;
+  r.slot = -1;
+}
+
+// na_slot >= 0: A's exact row count is still on the device (na is then its upper bound).
+// defer_slot >= 0: if the upper-bound outputs are small, allocate them at once and skip the control read between the
+// count pass and the emit pass; finish_merge() settles the sizes after the caller's next control read.
 template <typename K, typename Op>
-inline MergeResult merge_t(Ctx* c, const K* A, const float* TA, uint32_t na, const K* B, float* TB, uint32_t nb, bool want_delta,
-                           bool allow_in_place) {
+inline MergeResult merge_t(Ctx* c, const K* A, const float* TA, uint32_t na, int na_slot, const K* B, float* TB, uint32_t nb,
+                           bool want_delta, bool allow_in_place, int defer_slot) {
   MergeResult r;
   const uint64_t total = (uint64_t)na + nb;
   const unsigned tiles = (unsigned)((total + kMrgTile - 1) / kMrgTile);
   if (tiles == 0) return r;
+  const uint32_t* na_ptr = na_slot >= 0 ? ctrl_u32(c, na_slot) : nullptr;
   DevBuf a_start(c, ((size_t)tiles + 1) * 4), nf(c, (size_t)tiles * 4), nd(c, (size_t)tiles * 4);
-  XLOG_LAUNCH(c, (k_merge_partition<K>), (tiles + 1 + 255) / 256, 256, 0, A, na, B, nb, tiles, a_start.as<uint32_t>());
+  XLOG_LAUNCH(c, (k_merge_partition<K>), (tiles + 1 + 255) / 256, 256, 0, A, na, na_ptr, B, nb, tiles, a_start.as<uint32_t>());
   c->note_bytes = (int64_t)total * (sizeof(K) + 4);
-  XLOG_LAUNCH(c, (k_merge<K, Op, false>), tiles, kMrgBlock, 0, A, TA, na, B, TB, nb, a_start.as<uint32_t>(), nf.as<uint32_t>(),
-              nd.as<uint32_t>(), (K*)nullptr, (float*)nullptr, (K*)nullptr, (float*)nullptr, 0);
+  XLOG_LAUNCH(c, (k_merge<K, Op, false>), tiles, kMrgBlock, 0, A, TA, na, na_ptr, B, TB, nb, a_start.as<uint32_t>(), nf.as<uint32_t>(),
+              nd.as<uint32_t>(), (K*)nullptr, (float*)nullptr, (K*)nullptr, (float*)nullptr, 0, (const uint32_t*)nullptr);
+  const bool defer = defer_slot >= 0 && want_delta && total * (sizeof(K) + 4) <= 2 * kDeferBytes;
+  if (defer) {
+    XLOG_LAUNCH(c, (k_scan_spine2<uint32_t>), 1, 1024, 0, nf.as<uint32_t>(), nd.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, defer_slot),
+                ctrl_u32(c, defer_slot + 1));
+    r.slot = defer_slot; r.nb = nb; r.allow_in_place = allow_in_place;
+    r.full.n = (uint32_t)total; r.delta.n = std::max(na, 1u);
+    r.full.keys = DevBuf(c, (size_t)total * sizeof(K));
+    r.full.tags = DevBuf(c, (size_t)total * 4);
+    r.delta.keys = DevBuf(c, (size_t)std::max(na, 1u) * sizeof(K));
+    r.delta.tags = DevBuf(c, (size_t)std::max(na, 1u) * 4);
+    c->note_bytes = (int64_t)total * 2 * (sizeof(K) + 4);
+    XLOG_LAUNCH(c, (k_merge<K, Op, true>), tiles, kMrgBlock, 0, A, TA, na, na_ptr, B, TB, nb, a_start.as<uint32_t>(), nf.as<uint32_t>(),
+                nd.as<uint32_t>(), r.full.keys.as<K>(), r.full.tags.as<float>(), r.delta.keys.as<K>(), r.delta.tags.as<float>(),
+                allow_in_place ? -1 : 0, (const uint32_t*)ctrl_u32(c, defer_slot));
+    return r;
+  }
   XLOG_LAUNCH(c, (k_scan_spine2<uint32_t>), 1, 1024, 0, nf.as<uint32_t>(), nd.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotB), ctrl_u32(c, kSlotC));
   sync_ctrl(c);
   const uint32_t tot_f = (uint32_t)c->h_ctrl[kSlotB], tot_d = (uint32_t)c->h_ctrl[kSlotC];
@@ -459,20 +528,20 @@ inline MergeResult merge_t(Ctx* c, const K* A, const float* TA, uint32_t na, con
   r.delta.keys = DevBuf(c, (size_t)std::max(tot_d, 1u) * sizeof(K));
   r.delta.tags = DevBuf(c, (size_t)std::max(tot_d, 1u) * 4);
   c->note_bytes = ((int64_t)total + (r.in_place ? 0 : tot_f) + tot_d) * (sizeof(K) + 4);
-  XLOG_LAUNCH(c, (k_merge<K, Op, true>), tiles, kMrgBlock, 0, A, TA, na, B, TB, nb, a_start.as<uint32_t>(), nf.as<uint32_t>(),
+  XLOG_LAUNCH(c, (k_merge<K, Op, true>), tiles, kMrgBlock, 0, A, TA, na, na_ptr, B, TB, nb, a_start.as<uint32_t>(), nf.as<uint32_t>(),
               nd.as<uint32_t>(), r.full.keys.as<K>(), r.full.tags.as<float>(), r.delta.keys.as<K>(), r.delta.tags.as<float>(),
-              r.in_place ? 1 : 0);
+              r.in_place ? 1 : 0, (const uint32_t*)nullptr);
   if (!want_delta) { r.delta.keys.reset(); r.delta.tags.reset(); r.delta.n = 0; }
   return r;
 }
 template <typename K>
-inline MergeResult merge(Ctx* c, int sr, const K* A, const float* TA, uint32_t na, const K* B, float* TB, uint32_t nb,
-                         bool want_delta, bool allow_in_place) {
+inline MergeResult merge(Ctx* c, int sr, const K* A, const float* TA, uint32_t na, int na_slot, const K* B, float* TB, uint32_t nb,
+                         bool want_delta, bool allow_in_place, int defer_slot = -1) {
   switch (sr) {
-    case XLOG_SR_MAXPLUS: return merge_t<K, OpMax>(c, A, TA, na, B, TB, nb, want_delta, allow_in_place);
-    case XLOG_SR_MINPLUS: return merge_t<K, OpMin>(c, A, TA, na, B, TB, nb, want_delta, allow_in_place);
-    case XLOG_SR_LOGSUMEXP: return merge_t<K, OpLse>(c, A, TA, na, B, TB, nb, want_delta, false);
-    default: return merge_t<K, OpSum>(c, A, TA, na, B, TB, nb, want_delta, false);
+    case XLOG_SR_MAXPLUS: return merge_t<K, OpMax>(c, A, TA, na, na_slot, B, TB, nb, want_delta, allow_in_place, defer_slot);
+    case XLOG_SR_MINPLUS: return merge_t<K, OpMin>(c, A, TA, na, na_slot, B, TB, nb, want_delta, allow_in_place, defer_slot);
+    case XLOG_SR_LOGSUMEXP: return merge_t<K, OpLse>(c, A, TA, na, na_slot, B, TB, nb, want_delta, false, defer_slot);
+    default: return merge_t<K, OpSum>(c, A, TA, na, na_slot, B, TB, nb, want_delta, false, defer_slot);
   }
 }
 

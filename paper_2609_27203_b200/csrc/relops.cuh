@@ -323,10 +323,12 @@ constexpr int kMrgItems = 8;
 constexpr int kMrgTile = kMrgBlock * kMrgItems;
 
 template <typename K>
-__global__ void __launch_bounds__(256) k_merge_partition(const K* __restrict__ A, uint32_t na, const K* __restrict__ B, uint32_t nb,
-                                                         uint32_t ntiles, uint32_t* __restrict__ a_start /*[ntiles+1]*/) {
+__global__ void __launch_bounds__(256) k_merge_partition(const K* __restrict__ A, uint32_t na, const uint32_t* __restrict__ na_ptr,
+                                                         const K* __restrict__ B, uint32_t nb, uint32_t ntiles,
+                                                         uint32_t* __restrict__ a_start /*[ntiles+1]*/) {
   const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t > ntiles) return;
+  if (na_ptr) na = min(na, *na_ptr);                   // the exact row count may still live on the device only
   const uint64_t diag = min((uint64_t)t * kMrgTile, (uint64_t)na + nb);
   uint32_t lo = diag > nb ? (uint32_t)(diag - nb) : 0u;
   uint32_t hi = (uint32_t)min((uint64_t)na, diag);
@@ -341,10 +343,14 @@ struct MergeCounts { uint32_t* tile_nf; uint32_t* tile_nd; };
 
 template <typename K, typename Op, bool EMIT>
 __global__ void __launch_bounds__(kMrgBlock) k_merge(const K* __restrict__ A, const float* __restrict__ TA, uint32_t na,
-                                                     const K* __restrict__ B, float* __restrict__ TB, uint32_t nb,
-                                                     const uint32_t* __restrict__ a_start, uint32_t* __restrict__ tile_nf,
-                                                     uint32_t* __restrict__ tile_nd, K* __restrict__ FK, float* __restrict__ FT,
-                                                     K* __restrict__ DK, float* __restrict__ DT, int inplace) {
+                                                     const uint32_t* __restrict__ na_ptr, const K* __restrict__ B,
+                                                     float* __restrict__ TB, uint32_t nb, const uint32_t* __restrict__ a_start,
+                                                     uint32_t* __restrict__ tile_nf, uint32_t* __restrict__ tile_nd,
+                                                     K* __restrict__ FK, float* __restrict__ FT, K* __restrict__ DK,
+                                                     float* __restrict__ DT, int inplace, const uint32_t* __restrict__ total_f) {
+  if (na_ptr) na = min(na, *na_ptr);
+  // inplace < 0: decide here from the merged row count (no new key <=> full' would have exactly nb rows)
+  if (EMIT && inplace < 0) inplace = *total_f == nb ? 1 : 0;
   __shared__ K sk[kMrgTile + 2];
   __shared__ float st[kMrgTile];
   __shared__ uint32_t shc[kMrgBlock / 32 + 1];
@@ -352,6 +358,10 @@ __global__ void __launch_bounds__(kMrgBlock) k_merge(const K* __restrict__ A, co
   __shared__ float peek_t;
   const uint32_t t = blockIdx.x;
   const uint64_t d0 = (uint64_t)t * kMrgTile;
+  if (d0 >= (uint64_t)na + nb) {                        // tile beyond the data (grid sized from an upper bound)
+    if (!EMIT && threadIdx.x == 0) { tile_nf[t] = 0; tile_nd[t] = 0; }
+    return;
+  }
   const uint64_t d1 = min(d0 + kMrgTile, (uint64_t)na + nb);
   const uint32_t a0 = a_start[t], a1 = a_start[t + 1];
   const uint32_t b0 = (uint32_t)(d0 - a0), b1 = (uint32_t)(d1 - a1);

@@ -471,12 +471,14 @@ constexpr int kSlotTotals = 16;          // uint64 candidate totals of the varia
 // Evaluate the variants, all deriving head relation H: join, project, sort, reduce by key.
 // `extra` (optional) is appended to the candidates before the sort (loaded facts of H in a
 // non-recursive stratum).  Returns the sorted unique candidates.
+// defer_slot >= 0: a small single-batch result may come back with its exact row count still on the device
+// (KeyTags::n_slot), saving a control read; the caller settles it after its next sync_ctrl.
 KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Source* extra, const KeyLayout& cand_layout,
-                 bool want_head_pos) {
+                 bool want_head_pos, int defer_slot = -1) {
   const int ckb = cand_layout.total_bits <= 32 ? 4 : 8;
   std::vector<Counted> counted;
   counted.reserve(variants.size());
-  if (variants.size() > (size_t)(kCtrlSlots - kSlotTotals)) fail(XLOG_ERR_UNSUPPORTED, "too many rule variants for one head");
+  if (variants.size() > 16) fail(XLOG_ERR_UNSUPPORTED, "too many rule variants for one head");
   // count + scan for every variant, then one control read for all totals
   for (Variant& v : variants) {
     if (v.outer.n == 0) continue;
@@ -531,17 +533,17 @@ KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Sour
       fail(XLOG_ERR_RESOURCE_EXHAUSTED, "candidate batch too small for the relation's loaded facts");
     }
     KeyTags part;
-    DISPATCH_K(ckb, part = sort_reduce<K>(c, H.sr, k0, t0, k1, t1, fill, cand_layout.total_bits, want_head_pos));
+    DISPATCH_K(ckb, part = sort_reduce<K>(c, H.sr, k0, t0, k1, t1, fill, cand_layout.total_bits, want_head_pos, cap >= total ? defer_slot : -1));
     if (result.n == 0) result = std::move(part);
     else {
       // a later batch: union with oplus into the running result
       MergeResult m;
-      DISPATCH_K(ckb, m = merge<K>(c, H.sr, part.keys.as<K>(), part.tags.as<float>(), part.n, result.keys.as<K>(), result.tags.as<float>(),
+      DISPATCH_K(ckb, m = merge<K>(c, H.sr, part.keys.as<K>(), part.tags.as<float>(), part.n, -1, result.keys.as<K>(), result.tags.as<float>(),
                                     result.n, false, false));
       result = std::move(m.full);
     }
   }
-  c->r_unique += result.n;
+  if (result.n_slot < 0) c->r_unique += result.n;     // a deferred count is added by the caller once it is known
   return result;
 }
 
@@ -867,13 +869,17 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
         }
       }
       if (vs.empty()) continue;
-      produced.emplace_back(h, evaluate(c, H, vs, nullptr, H.layout, false));
+      const int slot = produced.size() < 8 ? 32 + 4 * (int)produced.size() : -1;
+      produced.emplace_back(h, evaluate(c, H, vs, nullptr, H.layout, false, slot));
     }
     for (int p : comp) delta[p] = KeyTags();
-    uint64_t changed = 0;
-    for (auto& pr : produced) {
-      Relation& H = *c->rels[pr.first];
-      KeyTags& u = pr.second;
+    // merge every head's candidates into its full relation; small merges leave their totals on the device and all of
+    // them are settled by one control read
+    std::vector<MergeResult> merged(produced.size());
+    bool need_read = false;
+    for (size_t i = 0; i < produced.size(); ++i) {
+      Relation& H = *c->rels[produced[i].first];
+      KeyTags& u = produced[i].second;
       if (u.n == 0) continue;
       if (!H.cur_owned && H.n_facts) {
         // first derivation into a relation that holds facts: work on a private copy
@@ -883,12 +889,24 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
         XLOG_CUDA(cudaMemcpyAsync(copy.tags.p, H.fact_tags.p, (size_t)H.n_facts * 4, cudaMemcpyDeviceToDevice, c->stream));
         set_current(H, std::move(copy));
       }
-      MergeResult m;
-      DISPATCH_K(H.key_bytes, m = merge<K>(c, H.sr, u.keys.as<K>(), u.tags.as<float>(), u.n, (const K*)H.keys(), H.tags(), H.n, true, H.cur_owned));
+      const int slot = i < 8 ? 32 + 4 * (int)i + 1 : -1;
+      DISPATCH_K(H.key_bytes, merged[i] = merge<K>(c, H.sr, u.keys.as<K>(), u.tags.as<float>(), u.n, u.n_slot, (const K*)H.keys(), H.tags(), H.n,
+                                                    true, H.cur_owned, slot));
+      if (merged[i].slot >= 0) need_read = true;
+    }
+    if (need_read) sync_ctrl(c);
+    uint64_t changed = 0;
+    for (size_t i = 0; i < produced.size(); ++i) {
+      Relation& H = *c->rels[produced[i].first];
+      KeyTags& u = produced[i].second;
+      if (u.n == 0) continue;
+      if (u.n_slot >= 0) c->r_unique += (int64_t)(uint32_t)c->h_ctrl[u.n_slot];
+      MergeResult& m = merged[i];
+      finish_merge(c, m);
       if (!m.in_place) set_current(H, std::move(m.full));
       c->r_new += m.n_new; c->r_improved += m.n_improved;
       changed += (uint64_t)m.n_new + m.n_improved;
-      delta[pr.first] = std::move(m.delta);
+      delta[produced[i].first] = std::move(m.delta);
       if (c->flags & XLOG_FLAG_CHECK_INVARIANTS) {
         DISPATCH_K(H.key_bytes, XLOG_LAUNCH(c, (k_check_sorted<K>), grid_for(H.n, 256), 256, 0, (const K*)H.keys(), (int64_t)H.n, ctrl_u32(c, kSlotErr)));
         sync_ctrl(c);
