@@ -119,7 +119,10 @@ xlog_status xlog_relation_view(xlog_ctx* ctx, xlog_rel rel, const int32_t** cols
  * the 3-atom directed triangle  h(x..) :- e(x,y), e(y,z), e(z,x)  evaluated as a
  * fused intersect-and-aggregate (Section "Worst-case-optimal joins").  Anything
  * else: UNSUPPORTED.  Which atoms are recursive is derived from the strongly
- * connected components of the relation dependency graph. */
+ * connected components of the relation dependency graph; a rule may have one or two
+ * recursive atoms (p(x,z) :- p(x,y), p(y,z) is evaluated with one delta variant per
+ * occurrence, Section "Semi-naive evaluation on GPU"), and a component may hold
+ * several mutually recursive relations. */
 typedef enum { XLOG_ARG_CONST = 0, XLOG_ARG_VAR = 1 } xlog_arg_kind;
 typedef struct { int32_t kind; int32_t var; int32_t mul; int32_t add; /* CONST: add is the value */ } xlog_arg;
 typedef struct { xlog_rel rel; xlog_arg args[XLOG_MAX_ARITY]; } xlog_atom;

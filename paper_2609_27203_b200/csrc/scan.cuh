@@ -65,21 +65,22 @@ template <typename Tin, typename Tout>
 __global__ void __launch_bounds__(1024) k_scan_block(const Tin* __restrict__ in, int64_t n, Tout* __restrict__ out,
                                                      Tout* __restrict__ total_out) {
   __shared__ Tout sh[1024 / 32 + 1];
+  constexpr int PER = 16;
   Tout carry = 0;
-  for (int64_t base = 0; base < n; base += 1024 * 4) {
-    Tout x[4];
+  for (int64_t base = 0; base < n; base += 1024 * PER) {
+    Tout x[PER];
     Tout s = 0;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int64_t p = base + (int64_t)threadIdx.x * 4 + i;
+    for (int i = 0; i < PER; ++i) {
+      const int64_t p = base + (int64_t)threadIdx.x * PER + i;
       x[i] = p < n ? (Tout)in[p] : Tout(0);
       s += x[i];
     }
     Tout total;
     Tout run = carry + block_scan_excl<1024, Tout>(s, sh, total);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const int64_t p = base + (int64_t)threadIdx.x * 4 + i;
+    for (int i = 0; i < PER; ++i) {
+      const int64_t p = base + (int64_t)threadIdx.x * PER + i;
       if (p < n) out[p] = run;
       run += x[i];
     }

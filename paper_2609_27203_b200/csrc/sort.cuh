@@ -10,6 +10,8 @@
 // ticket, so a tile only ever waits for tiles that are already running; every wait is bounded
 // and a timeout raises the error flag and skips the tile's writes instead of hanging.
 #pragma once
+#include <string.h>
+
 #include "common.cuh"
 #include "scan.cuh"
 
@@ -74,34 +76,42 @@ __global__ void __launch_bounds__(256) k_sort_digit_hist(const K* __restrict__ k
   __shared__ uint32_t scan_sh[256 / 32 + 1];
   for (int i = threadIdx.x; i < P.passes * kSortMaxBins; i += blockDim.x) sh[i] = 0;
   __syncthreads();
-  // each block takes chunks of 256*8 keys; a thread issues its 8 loads before it touches any of them
+  // Each thread takes 8 CONSECUTIVE keys (vector loads when the array is 16-byte aligned) and, per pass,
+  // adds one count per run of equal digits among them: keys usually arrive in runs (sorted adjacency lists,
+  // a constant high digit), and for spread-out digits this is still only one shared-memory add per key.
   constexpr int U = 8;
   const uint64_t chunk = (uint64_t)blockDim.x * U;
+  const bool vec = (reinterpret_cast<uintptr_t>(keys) & 15u) == 0;
   for (uint64_t c0 = (uint64_t)blockIdx.x * chunk; c0 < n; c0 += (uint64_t)gridDim.x * chunk) {
+    const uint64_t i0 = c0 + (uint64_t)threadIdx.x * U;
     K k[U];
+    int cnt = 0;
+    if (i0 + U <= n && vec) {
+      const uint4* src = reinterpret_cast<const uint4*>(keys + i0);
+      uint4 v[U * sizeof(K) / 16];
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const uint64_t i = c0 + (uint64_t)u * blockDim.x + threadIdx.x;
-      k[u] = i < n ? keys[i] : K(0);
+      for (int j = 0; j < (int)(U * sizeof(K) / 16); ++j) v[j] = src[j];
+      memcpy(k, v, sizeof(k));
+      cnt = U;
+    } else {
+#pragma unroll
+      for (int u = 0; u < U; ++u) if (i0 + u < n) { k[u] = keys[i0 + u]; cnt = u + 1; }
     }
+    if (cnt == 0) continue;
 #pragma unroll
-    for (int u = 0; u < U; ++u) {
-      const bool ok = c0 + (uint64_t)u * blockDim.x + threadIdx.x < n;
+    for (int p = 0; p < kSortMaxPasses; ++p) {
+      if (p < P.passes) {
+        const uint32_t m = (1u << P.bits[p]) - 1u;
+        uint32_t run_d = (uint32_t)(k[0] >> P.shift[p]) & m, run_n = 1;
 #pragma unroll
-      for (int p = 0; p < kSortMaxPasses; ++p) {
-        if (p < P.passes) {
-          // one shared-memory add per RUN of equal digits across the lanes: keys usually arrive in
-          // runs (sorted adjacency lists, a constant high digit), and spread-out digits conflict little
-          const uint32_t d = ok ? (uint32_t)(k[u] >> P.shift[p]) & ((1u << P.bits[p]) - 1u) : 0xffffffffu;
-          const uint32_t dp = __shfl_up_sync(0xffffffffu, d, 1);
-          const bool head = lane_id() == 0 || d != dp;
-          const unsigned heads = __ballot_sync(0xffffffffu, head);
-          if (head && ok) {
-            const unsigned later = lane_id() == 31 ? 0u : heads >> (lane_id() + 1);
-            const uint32_t len = later ? (uint32_t)__ffs(later) : 32u - lane_id();
-            atomicAdd(&sh[p * kSortMaxBins + d], len);
+        for (int u = 1; u < U; ++u) {
+          if (u < cnt) {
+            const uint32_t d = (uint32_t)(k[u] >> P.shift[p]) & m;
+            if (d != run_d) { atomicAdd(&sh[p * kSortMaxBins + run_d], run_n); run_d = d; run_n = 0; }
+            ++run_n;
           }
         }
+        atomicAdd(&sh[p * kSortMaxBins + run_d], run_n);
       }
     }
   }

@@ -424,7 +424,7 @@ void count_variant(Ctx* c, const Variant& v, const Relation& H, Counted& q, int 
   q.start = DevBuf(c, (size_t)n * 8); q.sums = DevBuf(c, (size_t)tiles * 8);
   DISPATCH_K(v.outer.key_bytes, XLOG_LAUNCH(c, (k_join_count<K>), (n + 255) / 256, 256, 0, q.spec, (const K*)v.outer.keys, v.outer.tags, n,
                                              q.deg.as<uint32_t>(), q.rowinfo.as<uint4>(), ctrl_u32(c, kSlotErr)));
-  if (n <= (1u << 17)) {
+  if (n <= (1u << 16)) {
     XLOG_LAUNCH(c, (k_scan_block<uint32_t, uint64_t>), 1, 1024, 0, (const uint32_t*)q.deg.as<uint32_t>(), (int64_t)n, q.start.as<uint64_t>(),
                 (uint64_t*)(c->d_ctrl + q.slot));
     return;
@@ -851,16 +851,16 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
           int outer = 0;
           if (r->kind == 2) {
             const bool in0 = in_set(comp, r->plan.atoms[0].rel), in1 = in_set(comp, r->plan.atoms[1].rel);
-            if (in0 && in1) fail(XLOG_ERR_UNSUPPORTED, "rules with two recursive atoms are not supported");
-            outer = in1 ? 1 : 0;                            // scan the recursive side, look up the stable side
-            if (!r->shape[outer].ok) { if (!in0 && !in1 && r->shape[1 - outer].ok) outer = 1 - outer; else fail(XLOG_ERR_UNSUPPORTED, "no index path for this rule"); }
+            // scan the recursive side and look up the stable side; with two recursive atoms (non-linear rule)
+            // the looked-up side is the full relation, indexed afresh in every round it changed
+            outer = in1 && !in0 ? 1 : 0;
+            if (!r->shape[outer].ok) { if (in0 == in1 && r->shape[1 - outer].ok) outer = 1 - outer; else fail(XLOG_ERR_UNSUPPORTED, "no index path for this rule"); }
           }
           vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
         } else {
           for (int j = 0; j < r->plan.n_atoms; ++j) {
             const int ar = r->plan.atoms[j].rel;
             if (!in_set(comp, ar)) continue;
-            if (r->kind == 2 && in_set(comp, r->plan.atoms[1 - j].rel)) fail(XLOG_ERR_UNSUPPORTED, "rules with two recursive atoms are not supported");
             const KeyTags& d = delta[ar];
             if (d.n == 0) continue;
             const Relation& RA = *c->rels[ar];
@@ -904,6 +904,7 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
       MergeResult& m = merged[i];
       finish_merge(c, m);
       if (!m.in_place) set_current(H, std::move(m.full));
+      else if (m.n_improved) drop_indices(H);           // tags changed in place: permuted index copies are stale
       c->r_new += m.n_new; c->r_improved += m.n_improved;
       changed += (uint64_t)m.n_new + m.n_improved;
       delta[produced[i].first] = std::move(m.delta);

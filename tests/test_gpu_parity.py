@@ -179,6 +179,36 @@ def test_right_linear_rule_uses_a_transposed_index():
     check_program(prog, expect_bit_equal=False)
 
 
+def test_non_linear_and_mutual_recursion():
+    # p(x,z) :- p(x,y), p(y,z): two recursive atoms, so each round joins delta with the full relation on both sides
+    # (the looked-up side is indexed afresh, once by its first and once by its second column)
+    s, d = synth.uniform_digraph(150, 500, 31)
+    t = synth.log_prob_tags(500, 31)
+    edge = ([s, d], t)
+    nl = W.Program("nonlinear", {"e": (2, W.MAXPLUS), "p": (2, W.MAXPLUS)},
+                   [W.Rule("p", (W.V(0), W.V(1)), (W.Atom("e", (W.Var(0), W.Var(1))),)),
+                    W.Rule("p", (W.V(0), W.V(2)), (W.Atom("p", (W.Var(0), W.Var(1))), W.Atom("p", (W.Var(1), W.Var(2)))))],
+                   {"e": edge}, ("p",))
+    r_nl, _ = check_program(nl)
+    # same relation as the linear closure (tuple set; tags may differ in the last place: other association of the sums)
+    from paper_2609_27203_b200 import xlog
+    c1, i1, _ = xlog.load_program(nl, arena_bytes=1 << 27)
+    c1.fixpoint()
+    c2, i2, _ = xlog.load_program(W.closure_program(s, d, t), arena_bytes=1 << 27)
+    c2.fixpoint()
+    H.compare_relations(c1.read(i1["p"]), c2.read(i2["path"]), rel_tol=1e-5, what="non-linear vs linear closure")
+    assert r_nl["iterations"] < c2.last_receipt["iterations"]          # path doubling needs fewer rounds
+    c1.close(); c2.close()
+    # odd / even length walks: two heads in one recursive component
+    w = (1 + 9 * synth.uniform01(31, 9, 0, 500)).astype(np.float32)
+    mut = W.Program("odd_even", {"e": (2, W.MINPLUS), "odd": (2, W.MINPLUS), "even": (2, W.MINPLUS)},
+                    [W.Rule("odd", (W.V(0), W.V(1)), (W.Atom("e", (W.Var(0), W.Var(1))),)),
+                     W.Rule("even", (W.V(0), W.V(2)), (W.Atom("odd", (W.Var(0), W.Var(1))), W.Atom("e", (W.Var(1), W.Var(2))))),
+                     W.Rule("odd", (W.V(0), W.V(2)), (W.Atom("even", (W.Var(0), W.Var(1))), W.Atom("e", (W.Var(1), W.Var(2)))))],
+                    {"e": ([s, d], w)}, ("odd", "even"))
+    check_program(mut)
+
+
 def test_chunked_candidates_match_single_batch():
     p = W.config1(300, 1500)
     a, _ = check_program(p)
