@@ -116,8 +116,10 @@ xlog_status xlog_relation_view(xlog_ctx* ctx, xlog_rel rel, const int32_t** cols
  * Listing 7), so the head relation's arity is n_head_cols + 1.
  * Supported shapes: 1 atom; 2 atoms joined on one variable, the second side looked
  * up through a sorted index on that column, its other columns plain variables;
- * the 3-atom directed triangle  h(x..) :- e(x,y), e(y,z), e(z,x)  evaluated as a
- * fused intersect-and-aggregate (Section "Worst-case-optimal joins").  Anything
+ * the 3-atom directed triangle over one binary relation, either aggregated per x,
+ * h(x[, count]) :- e(x,y), e(y,z), e(z,x)  (fused intersect-and-aggregate, nothing
+ * materialised), or materialised,  h(x,y,z) :- e(x,y), e(y,z), e(z,x)  (count ->
+ * scan -> write, rows born sorted; Section "Worst-case-optimal joins").  Anything
  * else: UNSUPPORTED.  Which atoms are recursive is derived from the strongly
  * connected components of the relation dependency graph; a rule may have one or two
  * recursive atoms (p(x,z) :- p(x,y), p(y,z) is evaluated with one delta variant per

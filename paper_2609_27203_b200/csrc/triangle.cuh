@@ -102,6 +102,55 @@ __global__ void __launch_bounds__(256) k_tri_groups(const uint32_t* __restrict__
   }
 }
 
+// Materialising variant  tri(x,y,z) :- e(x,y), e(y,z), e(z,x)  (paper: "Worst-case-optimal joins": count ->
+// device prefix scan -> materialise over flat sorted-column storage).  edge_off = exclusive scan of the
+// per-edge match counts.  One warp per edge walks the shorter list in order, 32 entries at a time; a
+// ballot ranks the hits, so an edge's rows come out in increasing z and the whole output is already
+// sorted by (x,y,z) and duplicate-free: no sort, no reduce.
+template <typename K>
+__global__ void __launch_bounds__(256) k_tri_materialise(TriGraph G, int times, const uint64_t* __restrict__ edge_off, KeyLayout L,
+                                                         K* __restrict__ out_keys, float* __restrict__ out_tags) {
+  const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+  const unsigned lane = lane_id();
+  for (uint32_t e = warp; e < G.n_edges; e += nwarps) {
+    const int32_t x = G.src[e], y = G.dst[e];
+    const float wxy = G.w[e];
+    uint32_t a0 = 0, a1 = 0, b0 = 0, b1 = 0;
+    if (y < G.out_domain) { a0 = G.out_off[y]; a1 = G.out_off[y + 1]; }
+    if (x < G.in_domain) { b0 = G.in_off[x]; b1 = G.in_off[x + 1]; }
+    const uint32_t la = a1 - a0, lb = b1 - b0;
+    if (!la || !lb) continue;
+    const bool walk_a = la <= lb;
+    const int32_t* wl = walk_a ? G.dst + a0 : G.in_src + b0;
+    const int32_t* sl = walk_a ? G.in_src + b0 : G.dst + a0;
+    const uint32_t nw = walk_a ? la : lb, ns = walk_a ? lb : la;
+    uint64_t pos = edge_off[e];
+    const K xy = ((K)(uint32_t)x << L.shift[0]) | ((K)(uint32_t)y << L.shift[1]);
+    for (uint32_t i0 = 0; i0 < nw; i0 += 32) {
+      const uint32_t i = i0 + lane;
+      bool hit = false;
+      int32_t z = 0;
+      uint32_t lo = 0;
+      if (i < nw) {
+        z = wl[i];
+        uint32_t hi = ns;
+        while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (sl[mid] < z) lo = mid + 1; else hi = mid; }
+        hit = lo < ns && sl[lo] == z;
+      }
+      const unsigned m = __ballot_sync(0xffffffffu, hit);
+      if (hit) {
+        const float wyz = walk_a ? G.w[a0 + i] : G.w[a0 + lo];
+        const float wzx = walk_a ? G.in_w[b0 + lo] : G.in_w[b0 + i];
+        const uint64_t o = pos + __popc(m & lanemask_lt());
+        out_keys[o] = xy | ((K)(uint32_t)z << L.shift[2]);
+        out_tags[o] = times ? (wxy * wyz) * wzx : (wxy + wyz) + wzx;
+      }
+      pos += __popc(m);
+    }
+  }
+}
+
 // Keep the x that have at least one triangle: pos = exclusive scan of flag.
 template <typename K>
 __global__ void __launch_bounds__(256) k_tri_compact(const uint32_t* __restrict__ flag, const uint32_t* __restrict__ pos, int64_t domain,

@@ -238,11 +238,17 @@ void add_rule(Ctx* c, const xlog_plan* p, xlog_rule* out) {
     if (ok) {
       const int x = a[0].args[0].var, y = a[0].args[1].var, z = a[1].args[1].var;
       ok = x != y && y != z && x != z && a[1].args[0].var == y && a[2].args[0].var == z && a[2].args[1].var == x;
-      ok = ok && p->n_head_cols == 1 && p->head[0].c0 == 0;
-      for (int v = 0; v < XLOG_MAX_VARS && ok; ++v) ok = p->head[0].coef[v] == (v == x ? 1 : 0);
+      const int hv[3] = {x, y, z};
+      bool agg = ok && p->n_head_cols == 1, mat = ok && p->n_head_cols == 3 && !p->emit_count_column;
+      for (int h = 0; h < p->n_head_cols && h < 3; ++h) {
+        bool id = p->head[h].c0 == 0;
+        for (int v = 0; v < XLOG_MAX_VARS; ++v) id = id && p->head[h].coef[v] == (v == hv[h] ? 1 : 0);
+        agg = agg && id; mat = mat && id;
+      }
+      ok = agg || mat;
+      r.kind = mat ? 4 : 3;
     }
-    if (!ok) fail(XLOG_ERR_UNSUPPORTED, "three-atom rules are supported only as the directed triangle h(x) :- e(x,y), e(y,z), e(z,x)");
-    r.kind = 3;
+    if (!ok) fail(XLOG_ERR_UNSUPPORTED, "three-atom rules are supported only as the directed triangle h(x) or h(x,y,z) :- e(x,y), e(y,z), e(z,x)");
   }
   c->rules.push_back(r);
   H.is_head = true;
@@ -623,7 +629,7 @@ void propagate_bounds(Ctx* c) {
     // dictionary candidates: every rule writes the column as a bare variable that is bound either by the
     // same column of this relation (carried along) or by a column of a stored, non-derived relation
     bool plain_rules = R.n_facts == 0;
-    for (const RuleC& rc : c->rules) if (rc.plan.head_rel == r && (rc.kind == 3 || rc.plan.emit_count_column)) plain_rules = false;
+    for (const RuleC& rc : c->rules) if (rc.plan.head_rel == r && (rc.kind >= 3 || rc.plan.emit_count_column)) plain_rules = false;
     for (int col = 0; col < R.arity && plain_rules; ++col) {
       int src_rel = -1, src_col = -1;
       bool ok = true;
@@ -754,6 +760,43 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
   else set_current(H, std::move(kt));
 }
 
+// tri(x,y,z) :- e(x,y), e(y,z), e(z,x): count per edge -> scan -> materialise; the result is born sorted.
+void triangle_materialise(Ctx* c, Relation& H, const RuleC& r) {
+  Relation& E = *c->rels[r.plan.atoms[0].rel];
+  if (H.n_facts) fail(XLOG_ERR_UNSUPPORTED, "a materialised triangle relation cannot also hold loaded facts");
+  if (E.n == 0) { KeyTags empty; set_current(H, std::move(empty)); return; }
+  Index& out_ix = ensure_index(c, E, 0);
+  Index& in_ix = ensure_index(c, E, 1);
+  TriGraph G{};
+  G.n_edges = E.n;
+  G.src = E.cols[0].as<int32_t>(); G.dst = E.cols[1].as<int32_t>(); G.w = E.tags();
+  G.out_domain = out_ix.domain; G.in_domain = in_ix.domain;
+  G.out_off = out_ix.off.as<uint32_t>(); G.in_off = in_ix.off.as<uint32_t>();
+  G.in_src = in_ix.other[0]; G.in_w = in_ix.tags;
+  const int times = H.sr == XLOG_SR_SUMPROD ? 1 : 0;
+  DevBuf ecnt(c, (size_t)E.n * 4), eacc(c, (size_t)E.n * 4), eoff(c, (size_t)E.n * 8);
+  const unsigned tiles = (E.n + kScanTile - 1) / kScanTile;
+  DevBuf sums(c, (size_t)tiles * 8);
+  c->note_bytes = (int64_t)E.n * 12 * 3;
+  XLOG_LAUNCH(c, (k_tri_edges<OpMax>), kSMs * 8, 256, 0, G, times, ecnt.as<uint32_t>(), eacc.as<float>());
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)ecnt.as<uint32_t>(), (int64_t)E.n, sums.as<uint64_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, sums.as<uint64_t>(), (int64_t)tiles, (uint64_t*)(c->d_ctrl + kSlotTotals));
+  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)ecnt.as<uint32_t>(), (int64_t)E.n,
+              (const uint64_t*)sums.as<uint64_t>(), eoff.as<uint64_t>());
+  sync_ctrl(c);                                            // the one small metadata read that sizes the output
+  const uint64_t total = c->h_ctrl[kSlotTotals];
+  if (total > kSortMaxN) fail(XLOG_ERR_CAPACITY_EXCEEDED, "materialised triangle relation exceeds 2^30 - 1 rows");
+  c->r_candidates += (int64_t)total; c->r_unique += (int64_t)total;
+  KeyTags kt;
+  kt.n = (uint32_t)total;
+  kt.keys = DevBuf(c, (size_t)std::max<uint64_t>(total, 1) * H.key_bytes);
+  kt.tags = DevBuf(c, (size_t)std::max<uint64_t>(total, 1) * 4);
+  c->note_bytes = (int64_t)total * (H.key_bytes + 4);
+  DISPATCH_K(H.key_bytes, XLOG_LAUNCH(c, (k_tri_materialise<K>), kSMs * 8, 256, 0, G, times, (const uint64_t*)eoff.as<uint64_t>(), H.layout,
+                                       kt.keys.as<K>(), kt.tags.as<float>()));
+  set_current(H, std::move(kt));
+}
+
 void triangle_aggregate(Ctx* c, Relation& H, const RuleC& r) {
   if (c->rels[r.plan.atoms[0].rel]->is_head && r.plan.atoms[0].rel == r.plan.head_rel) fail(XLOG_ERR_UNSUPPORTED, "recursive triangle rule");
   switch (H.sr) {
@@ -769,7 +812,7 @@ void triangle_aggregate(Ctx* c, Relation& H, const RuleC& r) {
 void rule_backward(Ctx* c, const RuleC& r, const float* g, float* const* grads) {
   Relation& H = *c->rels[r.plan.head_rel];
   if (H.sr != XLOG_SR_LOGSUMEXP && H.sr != XLOG_SR_SUMPROD) fail(XLOG_ERR_UNSUPPORTED, "backward is defined for logsumexp and sum heads only");
-  if (r.kind == 3) fail(XLOG_ERR_UNSUPPORTED, "backward of the triangle aggregate is not built");
+  if (r.kind >= 3) fail(XLOG_ERR_UNSUPPORTED, "backward of the triangle rules is not built");
   for (int j = 0; j < r.plan.n_atoms; ++j) {
     if (!grads[j]) fail(XLOG_ERR_INVALID_ARGUMENT, "NULL gradient buffer");
     if (r.plan.atoms[j].rel == r.plan.head_rel) fail(XLOG_ERR_UNSUPPORTED, "backward of a recursive rule");
@@ -812,9 +855,10 @@ void stratum_once(Ctx* c, int head, const std::vector<const RuleC*>& rs) {
   if (counted && rs.size() > 1) fail(XLOG_ERR_UNSUPPORTED, "a counted head relation takes exactly one rule");
   ++c->r_iterations;
   if (rs.size() == 1 && rs[0]->kind == 3) { triangle_aggregate(c, H, *rs[0]); return; }
+  if (rs.size() == 1 && rs[0]->kind == 4) { triangle_materialise(c, H, *rs[0]); c->r_new += H.n; return; }
   std::vector<Variant> vs;
   for (const RuleC* r : rs) {
-    if (r->kind == 3) fail(XLOG_ERR_UNSUPPORTED, "a triangle rule must be the only rule of its head");
+    if (r->kind >= 3) fail(XLOG_ERR_UNSUPPORTED, "a triangle rule must be the only rule of its head");
     int outer = 0;
     if (r->kind == 2 && !r->shape[0].ok) outer = 1;
     vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
@@ -834,7 +878,7 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
     fail(XLOG_ERR_UNSUPPORTED, "relation '" + c->rels[p]->name + "': only max/min tags may be aggregated inside a recursive component");
   for (const RuleC* r : rs) {
     if (r->plan.emit_count_column) fail(XLOG_ERR_UNSUPPORTED, "count inside a recursive component");
-    if (r->kind == 3) fail(XLOG_ERR_UNSUPPORTED, "triangle rule inside a recursive component");
+    if (r->kind >= 3) fail(XLOG_ERR_UNSUPPORTED, "triangle rule inside a recursive component");
   }
   std::vector<KeyTags> delta(c->rels.size());
   for (int64_t round = 0;; ++round) {

@@ -124,6 +124,19 @@ def triangle_program(src, dst, w, name="triangles") -> Program:
     )
 
 
+def triangle_rows_program(src, dst, w, semiring=MAXPLUS, name="triangle_rows") -> Program:
+    """tri(x,y,z) :- e(x,y), e(y,z), e(z,x): the materialised three-way cyclic join; tag = (w_xy + w_yz) + w_zx."""
+    return Program(
+        name=name,
+        relations={"e": (2, semiring), "tri": (3, semiring)},
+        rules=[Rule("tri", (V(0), V(1), V(2)),
+                    (Atom("e", (Var(0), Var(1))), Atom("e", (Var(1), Var(2))), Atom("e", (Var(2), Var(0)))))],
+        facts={"e": ([np.ascontiguousarray(src, np.int32), np.ascontiguousarray(dst, np.int32)],
+                     np.ascontiguousarray(w, np.float32))},
+        outputs=("tri",),
+    )
+
+
 def digits_program(log_tags: np.ndarray, name="digits") -> Program:
     """sum(p, a+b) :- digit(2p, a), digit(2p+1, b), logsumexp per (p, a+b).
 
