@@ -37,15 +37,33 @@ template <> struct DenseOp<OpMax> {
   __device__ __forceinline__ static void upd(int32_t* p, int32_t v) { atomicMax(p, v); }
 };
 
-// gstart[g] = first row with (key >> L) >= g, for g in [0, G]
+// How the rows are grouped.  A key is (top | mid | low): `low` = L table bits, `mid` = M bits that were radix
+// sorted, `top` = T bits by which the candidate stream was already ordered when it was produced (leading head
+// columns carried over from the leading columns of the sorted outer relation).  A stable sort on the mid bits
+// alone leaves the rows ordered by (mid, top), so the group number is  g = mid << T | top  and increases along
+// the array; with T = 0 this is simply key >> L.
+struct GroupShape { int L, M, T; };
 template <typename K>
-__global__ void __launch_bounds__(256) k_group_bounds(const K* __restrict__ keys, uint32_t n, int L, uint32_t G,
+__device__ __forceinline__ uint32_t group_of(const GroupShape& S, K key) {
+  const uint32_t mid = (uint32_t)(key >> S.L) & ((1u << S.M) - 1u);
+  const uint32_t top = S.T ? (uint32_t)(key >> (S.L + S.M)) : 0u;
+  return (mid << S.T) | top;
+}
+template <typename K>
+__device__ __forceinline__ K group_key(const GroupShape& S, uint32_t g, uint32_t slot) {
+  const uint32_t top = g & ((1u << S.T) - 1u), mid = g >> S.T;
+  return ((K)top << (S.L + S.M)) | ((K)mid << S.L) | (K)slot;
+}
+
+// gstart[g] = first row whose group number is >= g, for g in [0, G]
+template <typename K>
+__global__ void __launch_bounds__(256) k_group_bounds(const K* __restrict__ keys, uint32_t n, GroupShape S, uint32_t G,
                                                       uint32_t* __restrict__ gstart) {
   for (uint32_t g = blockIdx.x * blockDim.x + threadIdx.x; g <= G; g += gridDim.x * blockDim.x) {
     uint32_t lo = 0, hi = n;
     while (lo < hi) {
       const uint32_t mid = lo + ((hi - lo) >> 1);
-      if ((uint64_t)(keys[mid] >> L) < (uint64_t)g) lo = mid + 1; else hi = mid;
+      if (group_of<K>(S, keys[mid]) < g) lo = mid + 1; else hi = mid;
     }
     gstart[g] = lo;
   }
@@ -76,7 +94,7 @@ static __global__ void __launch_bounds__(256) k_fill_i32(int32_t* __restrict__ p
 }
 
 template <typename K, typename Op>
-__global__ void __launch_bounds__(kDenseBlock) k_dense_reduce(const K* __restrict__ keys, const float* __restrict__ tags, int L,
+__global__ void __launch_bounds__(kDenseBlock) k_dense_reduce(const K* __restrict__ keys, const float* __restrict__ tags, GroupShape S,
                                                                uint32_t G, uint32_t part, const uint32_t* __restrict__ gstart,
                                                                const uint32_t* __restrict__ part_base, const uint32_t* __restrict__ spill,
                                                                uint32_t n_spill_tables, int32_t* __restrict__ spill_tab,
@@ -100,7 +118,7 @@ __global__ void __launch_bounds__(kDenseBlock) k_dense_reduce(const K* __restric
   const uint32_t nparts = part_base[g + 1] - part_base[g];
   const uint32_t r0 = g0 + (item - part_base[g]) * part;
   const uint32_t r1 = min(r0 + part, g1);
-  const uint32_t mask = (1u << L) - 1u;
+  const uint32_t mask = (1u << S.L) - 1u;
   // reduce this piece into the table; 4 independent loads per thread in flight
   for (uint32_t i = r0 + threadIdx.x; i < r1; i += 4 * kDenseBlock) {
     K k[4]; float t[4];
@@ -148,7 +166,7 @@ __global__ void __launch_bounds__(kDenseBlock) k_dense_reduce(const K* __restric
   for (int i = 0; i < kDensePer; ++i) {
     const int32_t v = tbl[s0 + i];
     if (v != DenseOp<Op>::empty) {
-      out_keys[pos] = ((K)g << L) | (K)(s0 + i);
+      out_keys[pos] = group_key<K>(S, g, (uint32_t)(s0 + i));
       out_tags[pos] = ord2f(v);
       ++pos;
     }

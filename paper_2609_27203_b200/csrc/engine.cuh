@@ -382,27 +382,40 @@ inline bool dense_reduce_applies(int sr, uint64_t n, int nbits, bool want_head_p
   return n >= (1u << 18) && n >= ((uint64_t)32 << H);
 }
 
+// presorted_top: the input is already ordered by its top `presorted_top` key bits (see GroupShape), so those
+// bits need no sorting; what is left of the group bits is sorted, and the reduced rows are put back into key
+// order by a sort on the top bits (the reduced rows are few).
 template <typename K, typename Op>
-inline KeyTags sort_dense_reduce(Ctx* c, DevBuf& k0, DevBuf& t0, DevBuf& k1, DevBuf& t1, uint64_t n, int nbits, int defer_slot) {
+inline KeyTags sort_dense_reduce(Ctx* c, DevBuf& k0, DevBuf& t0, DevBuf& k1, DevBuf& t1, uint64_t n, int nbits, int defer_slot,
+                                 int presorted_top) {
   KeyTags out;
   K* ka = k0.as<K>(); K* kb = k1.as<K>();
   float* ta = t0.as<float>(); float* tb = t1.as<float>();
   const int L = std::min(nbits, kDenseBits), H = nbits - L;
   const uint32_t G = 1u << H;
-  sort_pairs<K>(c, ka, ta, kb, tb, n, nbits, L);                       // high bits only
+  GroupShape GS{L, H, 0};
+  if (presorted_top >= H) {
+    // every group bit is already in order: no radix pass at all (M = H, T = 0 describes plain key order)
+  } else if (presorted_top > 0) {
+    GS.T = presorted_top; GS.M = H - presorted_top;
+    sort_pairs<K>(c, ka, ta, kb, tb, n, nbits - presorted_top, L);     // middle bits only; rows end up ordered by (mid, top)
+    defer_slot = -1;                                                   // the reorder below needs the exact row count
+  } else {
+    sort_pairs<K>(c, ka, ta, kb, tb, n, nbits, L);                     // all group bits
+  }
   uint32_t part = (uint32_t)std::min<uint64_t>(std::max<uint64_t>(n / (kSMs * 8), 8192), 131072);
   part = (part + 1023) / 1024 * 1024;
   const uint32_t spill_cap = std::min<uint32_t>((uint32_t)(n / part) + 1, G), max_items = (uint32_t)(n / part) + G + 1;
   DevBuf gstart(c, ((size_t)G + 1) * 4), part_base(c, ((size_t)G + 1) * 4), spill(c, (size_t)G * 4), done(c, (size_t)G * 4),
       ucount(c, ((size_t)G + 1) * 4), spill_tab(c, (size_t)spill_cap * kDenseSlots * 4);
   XLOG_CUDA(cudaMemsetAsync(ucount.p, 0, ((size_t)G + 1) * 4, c->stream));
-  XLOG_LAUNCH(c, (k_group_bounds<K>), grid_for((uint64_t)G + 1, 256), 256, 0, (const K*)ka, (uint32_t)n, L, G, gstart.as<uint32_t>());
+  XLOG_LAUNCH(c, (k_group_bounds<K>), grid_for((uint64_t)G + 1, 256), 256, 0, (const K*)ka, (uint32_t)n, GS, G, gstart.as<uint32_t>());
   XLOG_LAUNCH(c, k_group_plan, 1, 1024, 0, (const uint32_t*)gstart.as<uint32_t>(), G, part, part_base.as<uint32_t>(), spill.as<uint32_t>(),
               done.as<uint32_t>(), ctrl_u32(c, kSlotB));
   XLOG_LAUNCH(c, k_fill_i32, grid_for((uint64_t)spill_cap * kDenseSlots, 256 * 8), 256, 0, spill_tab.as<int32_t>(),
               (uint64_t)spill_cap * kDenseSlots, DenseOp<Op>::empty);
   c->note_bytes = (int64_t)n * (sizeof(K) + 4);
-  XLOG_LAUNCH(c, (k_dense_reduce<K, Op>), max_items, kDenseBlock, 0, (const K*)ka, (const float*)ta, L, G, part,
+  XLOG_LAUNCH(c, (k_dense_reduce<K, Op>), max_items, kDenseBlock, 0, (const K*)ka, (const float*)ta, GS, G, part,
               (const uint32_t*)gstart.as<uint32_t>(), (const uint32_t*)part_base.as<uint32_t>(), (const uint32_t*)spill.as<uint32_t>(), spill_cap,
               spill_tab.as<int32_t>(), done.as<uint32_t>(), kb, tb, ucount.as<uint32_t>());
   const bool sorted_in_0 = (void*)ka == k0.p;
@@ -435,6 +448,14 @@ inline KeyTags sort_dense_reduce(Ctx* c, DevBuf& k0, DevBuf& t0, DevBuf& k1, Dev
                 (const uint32_t*)ucount.as<uint32_t>(), G, (const uint32_t*)ctrl_u32(c, kSlotA), out.keys.as<K>(), out.tags.as<float>());
   }
   k0.reset(); t0.reset(); k1.reset(); t1.reset();
+  if (GS.T && out.n > 1) {
+    // rows are ordered by (mid, top, low): a stable sort on the top bits restores key order (top, mid, low)
+    DevBuf ak(c, (size_t)out.n * sizeof(K)), at(c, (size_t)out.n * 4);
+    K* pk = out.keys.as<K>(); K* qk = ak.as<K>();
+    float* pt = out.tags.as<float>(); float* qt = at.as<float>();
+    sort_pairs<K>(c, pk, pt, qk, qt, out.n, nbits, nbits - GS.T);
+    if ((void*)pk != out.keys.p) { std::swap(out.keys, ak); std::swap(out.tags, at); }
+  }
   return out;
 }
 
@@ -442,10 +463,10 @@ inline KeyTags sort_dense_reduce(Ctx* c, DevBuf& k0, DevBuf& t0, DevBuf& k1, Dev
 // buffer; releases both and returns the groups in exact-size buffers.
 template <typename K>
 inline KeyTags sort_reduce(Ctx* c, int sr, DevBuf& k0, DevBuf& t0, DevBuf& k1, DevBuf& t1, uint64_t n, int nbits, bool want_head_pos,
-                           int defer_slot = -1) {
+                           int defer_slot = -1, int presorted_top = 0) {
   if (dense_reduce_applies(sr, n, nbits, want_head_pos))
-    return sr == XLOG_SR_MAXPLUS ? sort_dense_reduce<K, OpMax>(c, k0, t0, k1, t1, n, nbits, defer_slot)
-                                 : sort_dense_reduce<K, OpMin>(c, k0, t0, k1, t1, n, nbits, defer_slot);
+    return sr == XLOG_SR_MAXPLUS ? sort_dense_reduce<K, OpMax>(c, k0, t0, k1, t1, n, nbits, defer_slot, presorted_top)
+                                 : sort_dense_reduce<K, OpMin>(c, k0, t0, k1, t1, n, nbits, defer_slot, presorted_top);
   K* ka = k0.as<K>(); K* kb = k1.as<K>();
   float* ta = t0.as<float>(); float* tb = t1.as<float>();
   sort_pairs<K>(c, ka, ta, kb, tb, n, nbits);

@@ -327,6 +327,7 @@ struct Counted {                         // a variant after count + scan
   JoinSpec spec;
   Source outer;
   DevBuf deg, rowinfo, start, sums;
+  int presorted_top = 0;                 // the candidates come out ordered by this many leading key bits
   uint64_t total = 0;
   int slot = 0;
 };
@@ -424,6 +425,23 @@ void count_variant(Ctx* c, const Variant& v, const Relation& H, Counted& q, int 
   q.spec = make_spec(c, v, H);
   q.outer = v.outer;
   q.slot = slot;
+  {
+    // Leading head columns that are the leading columns of the scanned atom, in the same order, are carried over
+    // unchanged; the scanned relation is sorted by them (dictionary codes keep the order of the values), so the
+    // candidate stream is already ordered by those key bits.
+    const xlog_plan& p = v.rule->plan;
+    const xlog_atom& A = p.atoms[v.outer_atom];
+    const int ka = c->rels[A.rel]->arity;
+    int k = 0;
+    for (; k < p.n_head_cols && k < ka; ++k) {
+      if (!is_plain_var(A.args[k])) break;
+      const int var = A.args[k].var;
+      bool id = p.head[k].c0 == 0;
+      for (int w = 0; w < kMaxVars; ++w) id = id && p.head[k].coef[w] == (w == var ? 1 : 0);
+      if (!id) break;
+    }
+    q.presorted_top = k ? q.spec.head.total_bits - q.spec.head.shift[k - 1] : 0;
+  }
   const uint32_t n = v.outer.n;
   const unsigned tiles = (n + kScanTile - 1) / kScanTile;
   q.deg = DevBuf(c, (size_t)n * 4); q.rowinfo = DevBuf(c, (size_t)n * 16);
@@ -514,6 +532,8 @@ KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Sour
     if (fit < cap) cap = std::max<uint64_t>(fit, 1);
   }
   if (want_head_pos && cap < total) fail(XLOG_ERR_RESOURCE_EXHAUSTED, "a counted aggregate must fit one candidate batch");
+  // one variant and nothing appended: every batch is a contiguous slice of one ordered stream
+  const int presorted_top = counted.size() == 1 && (extra == nullptr || extra->n == 0) ? counted[0].presorted_top : 0;
 
   size_t vi = 0; uint64_t vpos = 0; bool extra_done = extra == nullptr || extra->n == 0;
   while (vi < counted.size() || !extra_done) {
@@ -539,7 +559,8 @@ KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Sour
       fail(XLOG_ERR_RESOURCE_EXHAUSTED, "candidate batch too small for the relation's loaded facts");
     }
     KeyTags part;
-    DISPATCH_K(ckb, part = sort_reduce<K>(c, H.sr, k0, t0, k1, t1, fill, cand_layout.total_bits, want_head_pos, cap >= total ? defer_slot : -1));
+    DISPATCH_K(ckb, part = sort_reduce<K>(c, H.sr, k0, t0, k1, t1, fill, cand_layout.total_bits, want_head_pos, cap >= total ? defer_slot : -1,
+                                          presorted_top));
     if (result.n == 0) result = std::move(part);
     else {
       // a later batch: union with oplus into the running result
