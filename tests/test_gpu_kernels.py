@@ -21,7 +21,9 @@ def _keys(n, bits, seed, skew):
 @pytest.mark.parametrize("n,bits,kb,skew", [
     (1, 8, 4, "uniform"), (2, 1, 4, "uniform"), (4097, 7, 4, "uniform"), (100_003, 20, 4, "uniform"),
     (1_000_000, 28, 4, "hot"), (3_000_017, 28, 4, "top"), (500_000, 32, 4, "uniform"),
-    (250_000, 38, 8, "uniform"), (1_200_007, 62, 8, "hot"), (70_000, 9, 8, "top"), (65_536, 0, 4, "uniform")])
+    (250_000, 38, 8, "uniform"), (1_200_007, 62, 8, "hot"), (70_000, 9, 8, "top"), (65_536, 0, 4, "uniform"),
+    # a thousand tiles and more
+    (4_200_011, 30, 4, "hot"), (5_000_000, 19, 4, "uniform"), (4_500_003, 10, 4, "top"), (4_300_000, 47, 8, "uniform")])
 def test_sort_pairs_is_a_stable_sort_on_the_low_bits(n, bits, kb, skew):
     import torch
     from paper_2609_27203_b200 import xlog
