@@ -256,15 +256,6 @@ inline bool same_layout(const KeyLayout& a, const KeyLayout& b) {
 // typed building blocks
 // ---------------------------------------------------------------------------------
 
-template <typename T>
-inline void scan_exclusive_u32_inplace(Ctx* c, uint32_t* v, uint64_t n, uint32_t* spine /* >= tiles entries */) {
-  if (n == 0) return;
-  const unsigned tiles = (unsigned)((n + kScanTile - 1) / kScanTile);
-  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), tiles, kScanBlock, 0, v, (int64_t)n, spine);
-  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, spine, (int64_t)tiles, (uint32_t*)nullptr);
-  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), tiles, kScanBlock, 0, v, (int64_t)n, spine, v);
-}
-
 // Sort n (key, tag) pairs on key bits [0, nbits).  On return keys/tags point at the sorted data
 // (either the original buffers or the alternates).
 template <typename K>

@@ -74,13 +74,6 @@ __global__ void __launch_bounds__(256) k_unpack(const K* __restrict__ keys, int6
   }
 }
 
-// Permuted copy used to build an index on a non-leading column: out column j = in column perm[j].
-static __global__ void __launch_bounds__(256) k_permute_cols(ColPtrs in, ColPtrsMut out, int64_t n, int arity, int p0, int p1, int p2, int p3) {
-  const int perm[kMaxArity] = {p0, p1, p2, p3};
-  for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
-    for (int c = 0; c < arity; ++c) out.c[c][i] = in.c[perm[c]][i];
-}
-
 // off[v] = first row whose leading column is >= v, for v in [0, domain]  (off[domain] = n).
 static __global__ void __launch_bounds__(256) k_build_offsets(const int32_t* __restrict__ lead, uint32_t n, int64_t domain,
                                                        uint32_t* __restrict__ off) {

@@ -215,6 +215,11 @@ def test_chunked_candidates_match_single_batch():
     b, _ = check_program(p, candidate_chunk_bytes=64 << 10)
     assert a["derived_tuples"] == b["derived_tuples"] and a["candidates"] == b["candidates"]
     check_program(W.config2(scale=12), candidate_chunk_bytes=32 << 10)
+    # batches large enough for the high-bit sort + table reduce, several per round, with a dictionary column
+    # and a stream that is already ordered by its leading key bits
+    c, _ = check_program(W.config5(scale=14, n_sources=32), candidate_chunk_bytes=6 << 20)
+    d, _ = check_program(W.config5(scale=14, n_sources=32))
+    assert c["derived_tuples"] == d["derived_tuples"] and c["candidates"] == d["candidates"]
 
 
 def test_fixpoint_idempotent_and_reset():
