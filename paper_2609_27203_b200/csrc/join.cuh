@@ -225,6 +225,40 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
   }
   __syncthreads();
 
+  if (MODE == kExpFast && staged) {
+    // lean loop of the common case: everything per row is in shared memory, everything per candidate is one
+    // (or a few) coalesced inner reads, one multiply-add and two coalesced writes; all indices are 32-bit
+    const uint32_t ntile = (uint32_t)(t_hi - t_lo);
+    const uint32_t j0 = (uint32_t)(t_lo - first_start);              // candidates of the first row that precede the tile
+    KH* __restrict__ kout = ckeys + (t_lo - out_lo);
+    float* __restrict__ tout = ctags + (t_lo - out_lo);
+    const float* __restrict__ itg = S.inner_tag;
+    const int32_t* __restrict__ ic0 = S.inner_col[0];
+    const KH m0 = (KH)S.inner_mult[0];
+    const int nin = S.has_inner ? S.inner_free : -1;                 // -1: one-atom rule
+    const bool times = S.times != 0;
+#pragma unroll
+    for (int k = 0; k < kExpItems; ++k) {
+      const uint32_t q = threadIdx.x + k * kExpBlock;
+      if (q < ntile) {
+        const uint32_t li = srowidx[q];
+        const uint4 info = sinfo[li];
+        const uint32_t ir = info.x + (li ? q - sstart[li] : q + j0);
+        KH key = (KH)(((uint64_t)info.w << 32) | info.z);
+        float tag = __uint_as_float(info.y);
+        if (nin >= 0) {
+          const float it = itg[ir];
+          tag = times ? tag * it : tag + it;
+          if (nin >= 1) key += (KH)(uint32_t)ic0[ir] * m0;
+          for (int c = 1; c < nin; ++c) key += (KH)(uint32_t)S.inner_col[c][ir] * (KH)S.inner_mult[c];
+        }
+        kout[q] = key;
+        tout[q] = tag;
+      }
+    }
+    return;
+  }
+
   uint32_t e = 0;
   for (uint32_t q = threadIdx.x; q < (uint32_t)(t_hi - t_lo); q += kExpBlock) {
     const uint64_t p = t_lo + q;
