@@ -47,7 +47,7 @@ def _load():
         L.orc_destroy.argtypes = [C.c_void_p]
         L.orc_relation.argtypes = [C.c_void_p, C.c_int, C.c_int]
         L.orc_load.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int64]
-        L.orc_rule.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int]
+        L.orc_rule.argtypes = [C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
         L.orc_reset.argtypes = [C.c_void_p]
         L.orc_run.argtypes = [C.c_void_p, C.c_int, C.c_int64, C.c_void_p]
         L.orc_delta_trace.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
@@ -91,8 +91,9 @@ class Oracle:
         if st:
             raise OracleError(st)
 
-    def rule(self, head: int, head_exprs, atoms, emit_count: bool = False) -> int:
-        """head_exprs: [(c0, {var: coef})]; atoms: [(rel, [("c", value) | ("v", var, mul, add)])]."""
+    def rule(self, head: int, head_exprs, atoms, emit_count: bool = False, negated=()) -> int:
+        """head_exprs: [(c0, {var: coef})]; atoms: [(rel, [("c", value) | ("v", var, mul, add)])];
+        negated: indices of atoms under negation as failure."""
         he = np.zeros((len(head_exprs), 1 + MAXV), np.int64)
         for i, (c0, coef) in enumerate(head_exprs):
             he[i, 0] = c0
@@ -106,8 +107,11 @@ class Oracle:
                     args[j, c] = (0, 0, 1, a[1])
                 else:
                     args[j, c] = (1, a[1], a[2], a[3])
+        neg = np.zeros(len(atoms), np.int32)
+        for j in negated:
+            neg[j] = 1
         r = self._L.orc_rule(self._h, head, len(head_exprs), he.ctypes.data, len(atoms),
-                             rel_ids.ctypes.data, args.ctypes.data, int(emit_count))
+                             rel_ids.ctypes.data, args.ctypes.data, int(emit_count), neg.ctypes.data)
         if r < 0:
             raise ValueError("bad rule")
         self._rule_atoms.append([int(x) for x in rel_ids])
@@ -167,5 +171,5 @@ def load_program(program) -> "tuple[Oracle, Dict[str, int], List[int]]":
                 else:
                     al.append(("v", g.var, g.mul, g.add))
             atoms.append((ids[a.rel], al))
-        rule_ids.append(o.rule(ids[r.head], he, atoms, r.emit_count))
+        rule_ids.append(o.rule(ids[r.head], he, atoms, r.emit_count, [j for j, a in enumerate(r.atoms) if a.negated]))
     return o, ids, rule_ids

@@ -20,6 +20,10 @@
 //     rejects aggregation inside a recursive component) iterates
 //     I_{k+1} = I_k oplus T(I_k) on a snapshot until nothing changes
 //     (Algorithm 1's "until all Delta empty", naive form);
+//   * a negated atom (stratified negation-as-failure over a relation of a lower stratum: paper sections
+//     "Aggregations and constraints" and "Completeness over finite domains", Listing 7's constraint
+//     `:- edge(X,_), not degree(X,_)`) holds for a binding iff no stored row matches it; variables that occur
+//     nowhere else act as wildcards; it contributes the semiring one to the tag;
 //   * otimes is evaluated in fp32 for MAXPLUS/MINPLUS (which makes tags
 //     bit-comparable) and in fp64 with one final rounding for LOGSUMEXP/SUMPROD;
 //     logsumexp of a group is  m + log(sum exp(v - m)), m = max v, in fp64.
@@ -56,7 +60,7 @@ typedef std::array<int32_t, MAXA> Key;        // unused columns stay 0
 typedef std::map<Key, float> Table;
 
 struct Arg  { int kind; int var; int64_t mul, add, c; };          // kind 0: constant c; 1: column == mul*var+add
-struct Atom { int rel; std::vector<Arg> args; };
+struct Atom { int rel; std::vector<Arg> args; bool neg = false; };
 struct Expr { int64_t c0; int64_t coef[MAXV]; };
 struct Rule { int head; std::vector<Atom> atoms; std::vector<Expr> head_cols; bool emit_count; };
 struct Rel  { int arity; int sr; Table facts; Table rows; };
@@ -98,6 +102,21 @@ struct Engine {
       if (j == (int)r.atoms.size()) { b.tf = tf; b.td = td; cb(b); return; }
       const Atom& a = r.atoms[j];
       const int k = rels[a.rel].arity;
+      if (a.neg) {
+        // negation as failure: does any stored row agree with every column that is fixed by now?
+        bool exists = false;
+        for (const auto& rowkv : *src[j]) {
+          bool m = true;
+          for (int c = 0; c < k && m; ++c) {
+            const Arg& g = a.args[c];
+            if (g.kind == 0) m = rowkv.first[c] == g.c;
+            else if (bound[g.var]) m = g.mul * b.var[g.var] + g.add == rowkv.first[c];
+          }
+          if (m) { exists = true; break; }
+        }
+        if (!exists) { b.row[j] = nullptr; level(j + 1, tf, td); }
+        return;
+      }
       // leading columns whose value is already determined
       Key lo{}; int pre = 0;
       for (; pre < k; ++pre) {
@@ -211,7 +230,7 @@ struct Engine {
       for (const Rule& r : rules) if (in.count(r.head)) rs.push_back(&r);
       if (rs.empty()) { for (int p : comp) rels[p].rows = rels[p].facts; continue; }   // loaded facts only
       bool recursive = comp.size() > 1;
-      for (const Rule* r : rs) for (const Atom& a : r->atoms) if (in.count(a.rel)) recursive = true;
+      for (const Rule* r : rs) for (const Atom& a : r->atoms) if (in.count(a.rel)) { recursive = true; if (a.neg) return status = ST_UNSUPPORTED; }
       if (!recursive) stratum_once(comp[0], rs);
       else {
         for (int p : comp) if (rels[p].sr != SR_MAXPLUS && rels[p].sr != SR_MINPLUS) return status = ST_UNSUPPORTED;
@@ -303,7 +322,7 @@ struct Engine {
       std::map<int, AccTable> acc;
       for (const Rule* r : rs)
         for (size_t i = 0; i < r->atoms.size(); ++i) {
-          if (!in.count(r->atoms[i].rel)) continue;
+          if (!in.count(r->atoms[i].rel) || r->atoms[i].neg) continue;
           auto s = full_sources(*r);
           s[i] = &delta[r->atoms[i].rel];
           contribute(*r, s.data(), acc[r->head]);
@@ -339,9 +358,10 @@ struct Engine {
       Key k; if (!head_key(r, b, k)) return;
       const int64_t h = head_index.at(k);
       for (size_t j = 0; j < r.atoms.size(); ++j) {
+        if (r.atoms[j].neg) continue;                      // a negated atom carries no tag
         double w;
         if (H.sr == SR_LOGSUMEXP) w = std::exp(b.td - out[h]);
-        else { w = 1.0; for (size_t i = 0; i < r.atoms.size(); ++i) if (i != j) w *= (double)b.row[i]->second; }
+        else { w = 1.0; for (size_t i = 0; i < r.atoms.size(); ++i) if (i != j && !r.atoms[i].neg) w *= (double)b.row[i]->second; }
         acc[j][row_index[j].at(b.row[j]->first)] += (double)g[h] * w;
       }
     });
@@ -396,7 +416,7 @@ int orc_load(void* e, int rel, const int32_t* rows, const float* tags, int64_t n
 // atom_args: per atom, per column, 4 values (kind, var, mul, add-or-constant), MAXA columns reserved per atom.
 // head_exprs: per head column, 1 + MAXV values (c0, coef[0..MAXV-1]).
 int orc_rule(void* e, int head, int n_head_cols, const int64_t* head_exprs, int n_atoms,
-             const int32_t* atom_rel, const int64_t* atom_args, int emit_count) {
+             const int32_t* atom_rel, const int64_t* atom_args, int emit_count, const int32_t* atom_neg) {
   Engine* E = (Engine*)e; Rule r; r.head = head; r.emit_count = emit_count != 0;
   if (n_atoms < 1 || n_atoms > 3) return -1;
   for (int c = 0; c < n_head_cols; ++c) {
@@ -406,7 +426,8 @@ int orc_rule(void* e, int head, int n_head_cols, const int64_t* head_exprs, int 
   }
   if ((int)r.head_cols.size() + (r.emit_count ? 1 : 0) != E->rels[head].arity) return -1;
   for (int j = 0; j < n_atoms; ++j) {
-    Atom a; a.rel = atom_rel[j];
+    Atom a; a.rel = atom_rel[j]; a.neg = atom_neg && atom_neg[j];
+    if (a.neg && j == 0) return -1;                        // the first atom binds the variables
     for (int c = 0; c < E->rels[a.rel].arity; ++c) {
       const int64_t* p = atom_args + (j * MAXA + c) * 4;
       Arg g; g.kind = (int)p[0]; g.var = (int)p[1]; g.mul = p[2]; g.add = p[3]; g.c = p[3];

@@ -44,6 +44,7 @@ def V(v: int) -> Affine:
 class Atom:
     rel: str
     args: Tuple[object, ...]
+    negated: bool = False          # negation as failure over a relation of a lower stratum
 
 
 @dataclass(frozen=True)

@@ -228,3 +228,56 @@ def test_facts_of_a_derived_relation_are_one_more_contribution():
     assert np.allclose(tags, [0.0, -1.0 + math.log(2.0), -3.0], atol=1e-6)
     o.run("naive")                                  # evaluating again recomputes the same relation
     assert np.allclose(o.read(ids["q"])[1], tags, atol=0)
+
+
+# ---- stratified negation ------------------------------------------------------------------
+
+def test_negation_is_set_difference_and_wildcards_mean_exists():
+    a = np.array([1, 2, 3, 5, 8, 13], np.int32)
+    b = np.array([2, 3, 4, 13, 21], np.int32)
+    prog = W.Program("diff", {"a": (1, W.MINPLUS), "b": (1, W.MINPLUS), "only_a": (1, W.MINPLUS)},
+                     [W.Rule("only_a", (W.V(0),), (W.Atom("a", (W.Var(0),)), W.Atom("b", (W.Var(0),), negated=True)))],
+                     {"a": ([a], np.arange(6, dtype=np.float32)), "b": ([b], None)}, ("only_a",))
+    o, ids, _ = run(prog)
+    cols, tags = o.read(ids["only_a"])
+    keep = np.setdiff1d(a, b)
+    assert cols[0].tolist() == keep.tolist()
+    assert tags.tolist() == [float(np.flatnonzero(a == v)[0]) for v in keep]      # the negated atom adds nothing to the tag
+    # paper Listing 7: the constraint  :- edge(X,_), not degree(X,_)  has no violation
+    g = H.read_golden("listing7_degree_count.txt")
+    e0, e1 = g["edges"][:, 0].astype(np.int32), g["edges"][:, 1].astype(np.int32)
+    prog = W.Program("l7", {"edge": (2, W.SUMPROD), "degree": (2, W.SUMPROD), "viol": (1, W.SUMPROD)},
+                     [W.Rule("degree", (W.V(0),), (W.Atom("edge", (W.Var(0), W.Var(1))),), emit_count=True),
+                      W.Rule("viol", (W.V(0),), (W.Atom("edge", (W.Var(0), W.Var(1))), W.Atom("degree", (W.Var(0), W.Var(2)), negated=True)))],
+                     {"edge": ([e0, e1], None)}, ("viol",))
+    o, ids, _ = run(prog)
+    assert o.size(ids["viol"]) == 0
+    # and with a node that has an in-edge only, `sink(y) :- edge(x,y), not edge(y,_)` lists the sinks
+    prog = W.Program("sinks", {"edge": (2, W.MAXPLUS), "sink": (1, W.MAXPLUS)},
+                     [W.Rule("sink", (W.V(1),), (W.Atom("edge", (W.Var(0), W.Var(1))), W.Atom("edge", (W.Var(1), W.Var(2)), negated=True)))],
+                     {"edge": ([e0, e1], None)}, ("sink",))
+    o, ids, _ = run(prog)
+    assert o.read(ids["sink"])[0][0].tolist() == sorted(set(e1.tolist()) - set(e0.tolist()))
+
+
+def test_negation_over_a_recursive_lower_stratum():
+    # unreached(x) :- node(x), not dist(x): everything the BFS from node 0 does not reach
+    s, d = synth.uniform_digraph(80, 110, 17)
+    w = np.ones(len(s), np.float32)
+    prog = W.sssp_program(s, d, w, 0)
+    prog.relations["node"] = (1, W.MINPLUS)
+    prog.relations["unreached"] = (1, W.MINPLUS)
+    prog.facts["node"] = ([np.arange(80, dtype=np.int32)], None)
+    prog.rules.append(W.Rule("unreached", (W.V(0),), (W.Atom("node", (W.Var(0),)), W.Atom("dist", (W.Var(0),), negated=True))))
+    for mode in ("naive", "seminaive"):
+        o, ids, _ = run(prog, mode)
+        reached = {0} | {y for (x, y) in H.reachable_pairs(80, s, d) if x == 0}
+        assert o.read(ids["unreached"])[0][0].tolist() == sorted(set(range(80)) - reached)
+    # negation through recursion is not stratified
+    bad = W.Program("bad", {"e": (1, W.MINPLUS), "p": (1, W.MINPLUS)},
+                    [W.Rule("p", (W.V(0),), (W.Atom("e", (W.Var(0),)), W.Atom("p", (W.Var(0),), negated=True)))],
+                    {"e": ([np.array([1], np.int32)], None)})
+    o, ids, _ = oracle.load_program(bad)
+    with pytest.raises(oracle.OracleError) as e:
+        o.run("naive")
+    assert e.value.status == "UNSUPPORTED"
