@@ -120,6 +120,12 @@ xlog_status xlog_relation_view(xlog_ctx* ctx, xlog_rel rel, const int32_t** cols
  * h(x[, count]) :- e(x,y), e(y,z), e(z,x)  (fused intersect-and-aggregate, nothing
  * materialised), or materialised,  h(x,y,z) :- e(x,y), e(y,z), e(z,x)  (count ->
  * scan -> write, rows born sorted; Section "Worst-case-optimal joins").  Anything
+ * Negation (Sections "Aggregations and constraints", "Completeness over finite domains":
+ * explicit stratified negation-as-failure): a rule of one positive atom followed by one
+ * negated atom,  h(..) :- a(..), not b(..).  The negated atom holds iff no row of b matches;
+ * its first column, or its first two, must be fixed by constants / variables of the positive
+ * atom, the remaining columns must be variables that occur nowhere else (wildcards); it adds
+ * nothing to the tag; b must belong to a lower stratum.  Anything
  * else: UNSUPPORTED.  Which atoms are recursive is derived from the strongly
  * connected components of the relation dependency graph; a rule may have one or two
  * recursive atoms (p(x,z) :- p(x,y), p(y,z) is evaluated with one delta variant per
@@ -127,7 +133,7 @@ xlog_status xlog_relation_view(xlog_ctx* ctx, xlog_rel rel, const int32_t** cols
  * several mutually recursive relations. */
 typedef enum { XLOG_ARG_CONST = 0, XLOG_ARG_VAR = 1 } xlog_arg_kind;
 typedef struct { int32_t kind; int32_t var; int32_t mul; int32_t add; /* CONST: add is the value */ } xlog_arg;
-typedef struct { xlog_rel rel; xlog_arg args[XLOG_MAX_ARITY]; } xlog_atom;
+typedef struct { xlog_rel rel; xlog_arg args[XLOG_MAX_ARITY]; int32_t negated; /* 1: negation as failure, see below */ } xlog_atom;
 typedef struct { int64_t c0; int32_t coef[XLOG_MAX_VARS]; } xlog_expr;
 typedef struct {
   uint32_t  struct_size;           /* sizeof(xlog_plan) */

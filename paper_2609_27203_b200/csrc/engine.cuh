@@ -115,7 +115,8 @@ struct JoinShape {                      // how a two-atom rule is evaluated with
 
 struct RuleC {
   xlog_plan plan;
-  int kind = 0;                         // 1: one atom, 2: two-atom join, 3: directed triangle
+  int kind = 0;                         // 1: one atom, 2: two-atom join, 3/4: directed triangle (aggregate / rows), 5: atom + negated atom
+  int neg_prefix = 0;                   // kind 5: how many leading columns of the negated atom are fixed
   JoinShape shape[2];                   // indexed by the outer atom
 };
 
@@ -144,6 +145,7 @@ struct Ctx {
   std::vector<ProfPending> prof_pending;
   std::vector<cudaEvent_t> ev_pool;
   int64_t note_bytes = 0;                 // algorithmic bytes of the next launch (consumed by the launch macro)
+  std::vector<char> stratum_done;         // per relation: its stratum has been evaluated in the running fixpoint
 };
 
 inline DevBuf::DevBuf(Ctx* ctx, size_t n) : c(ctx), bytes(n) {

@@ -38,6 +38,13 @@ struct JoinSpec {
   int64_t head_c0[kMaxArity];
   int32_t head_coef[kMaxArity][kMaxVars];
   int times;                                                  // otimes: 0 = add, 1 = multiply
+  // negated second atom (negation as failure): a row of the scanned atom survives iff the other relation has no row
+  // whose first neg_prefix (1 or 2) columns equal the given constants / variables
+  int neg_prefix;                                             // 0: no negated atom
+  ArgSpec neg_args[2];
+  int64_t neg_domain;
+  const uint32_t* neg_off;                                    // offsets over the negated relation's first column
+  const int32_t* neg_col1;                                    // its second column (sorted inside each first-column run)
   // fast shape: head key = row part + sum_j inner_col[j] * inner_mult[j]
   int fast;
   int32_t head_coef_outer[kMaxArity][kMaxVars];               // head_coef restricted to variables the outer atom binds
@@ -90,7 +97,27 @@ __global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __rest
   uint32_t d = 0, lo = 0;
   uint64_t rowkey = 0;
   if (bind_outer<KO>(S, okeys[i], var)) {
-    if (!S.has_inner) d = 1;
+    if (S.neg_prefix) {
+      int64_t val[2] = {0, 0};
+#pragma unroll
+      for (int k = 0; k < 2; ++k) {
+        const ArgSpec a = S.neg_args[k];
+        int64_t x = 0;
+#pragma unroll
+        for (int v = 0; v < kMaxVars; ++v) if (v == a.var) x = var[v];
+        val[k] = a.kind == 0 ? (int64_t)a.add : x * a.mul + a.add;
+      }
+      bool exists = false;
+      if (val[0] >= 0 && val[0] < S.neg_domain) {
+        uint32_t a0 = S.neg_off[val[0]], a1 = S.neg_off[val[0] + 1];
+        if (S.neg_prefix == 1) exists = a1 > a0;
+        else {
+          while (a0 < a1) { const uint32_t mid = a0 + ((a1 - a0) >> 1); if ((int64_t)S.neg_col1[mid] < val[1]) a0 = mid + 1; else a1 = mid; }
+          exists = a0 < S.neg_off[val[0] + 1] && (int64_t)S.neg_col1[a0] == val[1];
+        }
+      }
+      d = exists ? 0 : 1;
+    } else if (!S.has_inner) d = 1;
     else {
       int64_t pv = 0;
 #pragma unroll

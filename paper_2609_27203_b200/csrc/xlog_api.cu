@@ -223,8 +223,32 @@ void add_rule(Ctx* c, const xlog_plan* p, xlog_rule* out) {
       if (p->head[h].coef[v] != 0 && !bound[v]) fail(XLOG_ERR_INVALID_ARGUMENT, "head uses a variable no body atom binds");
   RuleC r;
   r.plan = *p;
+  for (int j = 0; j < p->n_atoms; ++j)
+    if (p->atoms[j].negated && !(p->n_atoms == 2 && j == 1)) fail(XLOG_ERR_UNSUPPORTED, "negation is supported as  h :- a(..), not b(..)  only");
   if (p->n_atoms == 1) r.kind = 1;
-  else if (p->n_atoms == 2) {
+  else if (p->n_atoms == 2 && p->atoms[1].negated) {
+    // the negated atom: a fixed prefix of one or two columns, then wildcards
+    const xlog_atom& A = p->atoms[0];
+    const xlog_atom& B = p->atoms[1];
+    bool in_a[XLOG_MAX_VARS] = {false};
+    for (int i = 0; i < c->rels[A.rel]->arity; ++i) if (A.args[i].kind == XLOG_ARG_VAR) in_a[A.args[i].var] = true;
+    const int kb = c->rels[B.rel]->arity;
+    int prefix = 0;
+    for (; prefix < kb && prefix < 2; ++prefix) {
+      const xlog_arg& g = B.args[prefix];
+      if (!(g.kind == XLOG_ARG_CONST || in_a[g.var])) break;
+    }
+    bool ok = prefix >= 1;
+    for (int i = prefix; i < kb && ok; ++i) {
+      const xlog_arg& g = B.args[i];
+      ok = g.kind == XLOG_ARG_VAR && !in_a[g.var];
+      for (int k = 0; k < kb && ok; ++k) if (k != i && B.args[k].kind == XLOG_ARG_VAR && B.args[k].var == g.var) ok = false;
+      for (int hcol = 0; hcol < p->n_head_cols && ok; ++hcol) if (p->head[hcol].coef[g.var] != 0) ok = false;
+    }
+    if (!ok) fail(XLOG_ERR_UNSUPPORTED, "negated atom: its first one or two columns must be fixed by the positive atom, the rest wildcards");
+    r.kind = 5;
+    r.neg_prefix = prefix;
+  } else if (p->n_atoms == 2) {
     r.kind = 2;
     r.shape[0] = join_shape(c, *p, 0);
     r.shape[1] = join_shape(c, *p, 1);
@@ -339,6 +363,18 @@ JoinSpec make_spec(Ctx* c, const Variant& v, const Relation& H) {
   const xlog_atom& A = p.atoms[v.outer_atom];
   for (int i = 0; i < c->rels[A.rel]->arity; ++i) S.outer_args[i] = ArgSpec{A.args[i].kind, A.args[i].var, A.args[i].mul, A.args[i].add};
   S.has_inner = 0;
+  S.neg_prefix = 0;
+  if (v.rule->kind == 5) {
+    const xlog_atom& B = p.atoms[1];
+    Relation& RB = *c->rels[B.rel];
+    if (RB.is_head && !c->stratum_done[B.rel]) fail(XLOG_ERR_UNSUPPORTED, "negation must be stratified: '" + RB.name + "' is not complete yet");
+    Index& ix = ensure_index(c, RB, 0);
+    S.neg_prefix = v.rule->neg_prefix;
+    for (int k = 0; k < S.neg_prefix; ++k) S.neg_args[k] = ArgSpec{B.args[k].kind, B.args[k].var, B.args[k].mul, B.args[k].add};
+    S.neg_domain = ix.domain;
+    S.neg_off = ix.off.as<uint32_t>();
+    S.neg_col1 = RB.arity > 1 ? ix.other[0] : nullptr;
+  }
   if (v.rule->kind == 2) {
     const JoinShape& sh = v.rule->shape[v.outer_atom];
     if (!sh.ok) fail(XLOG_ERR_UNSUPPORTED, "this rule cannot be evaluated with the required atom as the scanned side");
@@ -625,6 +661,7 @@ void propagate_bounds(Ctx* c) {
       for (int v = 0; v < XLOG_MAX_VARS; ++v) vub[v] = INT32_MAX;
       for (int j = 0; j < p.n_atoms; ++j) {
         const Relation& R = *c->rels[p.atoms[j].rel];
+        if (p.atoms[j].negated) continue;                  // binds nothing
         for (int i = 0; i < R.arity; ++i) {
           const xlog_arg& a = p.atoms[j].args[i];
           if (a.kind != XLOG_ARG_VAR) continue;
@@ -667,7 +704,7 @@ void propagate_bounds(Ctx* c) {
         for (int j = 0; j < p.n_atoms; ++j)
           for (int k = 0; k < c->rels[p.atoms[j].rel]->arity; ++k) {
             const xlog_arg& g = p.atoms[j].args[k];
-            if (g.kind != XLOG_ARG_VAR || g.var != v || g.mul != 1 || g.add != 0) continue;
+            if (p.atoms[j].negated || g.kind != XLOG_ARG_VAR || g.var != v || g.mul != 1 || g.add != 0) continue;
             if (p.atoms[j].rel == r && k == col) carried = true;
             else if (!c->rels[p.atoms[j].rel]->is_head && (best_rel < 0 || c->rels[p.atoms[j].rel]->n < c->rels[best_rel]->n)) { best_rel = p.atoms[j].rel; best_col = k; }
           }
@@ -833,7 +870,7 @@ void triangle_aggregate(Ctx* c, Relation& H, const RuleC& r) {
 void rule_backward(Ctx* c, const RuleC& r, const float* g, float* const* grads) {
   Relation& H = *c->rels[r.plan.head_rel];
   if (H.sr != XLOG_SR_LOGSUMEXP && H.sr != XLOG_SR_SUMPROD) fail(XLOG_ERR_UNSUPPORTED, "backward is defined for logsumexp and sum heads only");
-  if (r.kind >= 3) fail(XLOG_ERR_UNSUPPORTED, "backward of the triangle rules is not built");
+  if (r.kind == 3 || r.kind == 4) fail(XLOG_ERR_UNSUPPORTED, "backward of the triangle rules is not built");
   for (int j = 0; j < r.plan.n_atoms; ++j) {
     if (!grads[j]) fail(XLOG_ERR_INVALID_ARGUMENT, "NULL gradient buffer");
     if (r.plan.atoms[j].rel == r.plan.head_rel) fail(XLOG_ERR_UNSUPPORTED, "backward of a recursive rule");
@@ -861,7 +898,7 @@ void rule_backward(Ctx* c, const RuleC& r, const float* g, float* const* grads) 
   bw.count_bits = r.plan.emit_count_column ? H.layout.shift[r.plan.n_head_cols - 1] : 0;
   bw.grad_head = g;
   bw.grad_outer = grads[outer];
-  bw.grad_inner = r.kind == 2 ? grads[1 - outer] : nullptr;
+  bw.grad_inner = r.kind == 2 ? grads[1 - outer] : nullptr;     // a negated atom (kind 5) carries no tag: its buffer stays zero
   bw.lse = H.sr == XLOG_SR_LOGSUMEXP ? 1 : 0;
   if (q.total) launch_expand<true>(c, q, 0, q.total, ckb, nullptr, nullptr, bw);
   sync_ctrl(c);
@@ -879,7 +916,7 @@ void stratum_once(Ctx* c, int head, const std::vector<const RuleC*>& rs) {
   if (rs.size() == 1 && rs[0]->kind == 4) { triangle_materialise(c, H, *rs[0]); c->r_new += H.n; return; }
   std::vector<Variant> vs;
   for (const RuleC* r : rs) {
-    if (r->kind >= 3) fail(XLOG_ERR_UNSUPPORTED, "a triangle rule must be the only rule of its head");
+    if (r->kind == 3 || r->kind == 4) fail(XLOG_ERR_UNSUPPORTED, "a triangle rule must be the only rule of its head");
     int outer = 0;
     if (r->kind == 2 && !r->shape[0].ok) outer = 1;
     vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
@@ -899,7 +936,7 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
     fail(XLOG_ERR_UNSUPPORTED, "relation '" + c->rels[p]->name + "': only max/min tags may be aggregated inside a recursive component");
   for (const RuleC* r : rs) {
     if (r->plan.emit_count_column) fail(XLOG_ERR_UNSUPPORTED, "count inside a recursive component");
-    if (r->kind >= 3) fail(XLOG_ERR_UNSUPPORTED, "triangle rule inside a recursive component");
+    if (r->kind == 3 || r->kind == 4) fail(XLOG_ERR_UNSUPPORTED, "triangle rule inside a recursive component");
   }
   std::vector<KeyTags> delta(c->rels.size());
   for (int64_t round = 0;; ++round) {
@@ -925,7 +962,7 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
         } else {
           for (int j = 0; j < r->plan.n_atoms; ++j) {
             const int ar = r->plan.atoms[j].rel;
-            if (!in_set(comp, ar)) continue;
+            if (!in_set(comp, ar) || r->plan.atoms[j].negated) continue;
             const KeyTags& d = delta[ar];
             if (d.n == 0) continue;
             const Relation& RA = *c->rels[ar];
@@ -984,6 +1021,7 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
 
 void run_fixpoint(Ctx* c) {
   if (c->idb_dirty) { reset_idb(c); c->idb_dirty = false; }
+  c->stratum_done.assign(c->rels.size(), 0);
   if (c->poisoned) fail(XLOG_ERR_INVALID_STATE, "derived relations are poisoned by an earlier failure; call xlog_ctx_reset_idb");
   c->poisoned = true;                      // cleared on success
   zero_ctrl(c, kSlotErr);
@@ -995,7 +1033,10 @@ void run_fixpoint(Ctx* c) {
     ++c->r_strata;
     bool recursive = comp.size() > 1;
     for (const RuleC* r : rs) for (int j = 0; j < r->plan.n_atoms; ++j) if (in_set(comp, r->plan.atoms[j].rel)) recursive = true;
+    for (const RuleC* r : rs)
+      if (r->kind == 5 && in_set(comp, r->plan.atoms[1].rel)) fail(XLOG_ERR_UNSUPPORTED, "negation must be stratified: the negated relation depends on the rule's head");
     if (!recursive) stratum_once(c, comp[0], rs); else stratum_recursive(c, comp, rs);
+    for (int p : comp) c->stratum_done[p] = 1;
   }
   for (Relation* R : c->rels) if (R->is_head) ensure_soa(c, *R);
   sync_ctrl(c);

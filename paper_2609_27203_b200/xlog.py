@@ -46,7 +46,7 @@ class Arg(C.Structure):
 
 
 class AtomS(C.Structure):
-    _fields_ = [("rel", C.c_int32), ("args", Arg * MAX_ARITY)]
+    _fields_ = [("rel", C.c_int32), ("args", Arg * MAX_ARITY), ("negated", C.c_int32)]
 
 
 class Expr(C.Structure):
@@ -225,8 +225,9 @@ class Context:
         return [int(p or 0) for p in ptrs], int(tp.value or 0), n.value
 
     # ---- rules ----
-    def rule(self, head: int, head_exprs, atoms, emit_count: bool = False) -> int:
-        """head_exprs: [(c0, {var: coef})]; atoms: [(rel, [("c", value) | ("v", var, mul, add)])]."""
+    def rule(self, head: int, head_exprs, atoms, emit_count: bool = False, negated=()) -> int:
+        """head_exprs: [(c0, {var: coef})]; atoms: [(rel, [("c", value) | ("v", var, mul, add)])];
+        negated: indices of atoms under negation as failure."""
         p = Plan()
         p.struct_size = C.sizeof(Plan)
         p.head_rel = head
@@ -243,6 +244,8 @@ class Context:
                     p.atoms[j].args[c] = Arg(0, 0, 1, a[1])
                 else:
                     p.atoms[j].args[c] = Arg(1, a[1], a[2], a[3])
+        for j in negated:
+            p.atoms[j].negated = 1
         p.emit_count_column = int(emit_count)
         out = C.c_int32()
         self._check(self._L.xlog_rule_add(self._h, C.byref(p), C.byref(out)))
@@ -337,5 +340,5 @@ def load_program(program, ctx: Optional[Context] = None, device_inputs: bool = F
             for g in a.args:
                 al.append(("c", g.value) if hasattr(g, "value") else ("v", g.var, g.mul, g.add))
             atoms.append((ids[a.rel], al))
-        rule_ids.append(ctx.rule(ids[r.head], he, atoms, r.emit_count))
+        rule_ids.append(ctx.rule(ids[r.head], he, atoms, r.emit_count, [j for j, a in enumerate(r.atoms) if a.negated]))
     return ctx, ids, rule_ids

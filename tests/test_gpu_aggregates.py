@@ -181,3 +181,48 @@ def test_backward_requires_a_forward_and_a_supported_head():
         ctx.backward(rules[0], torch.ones(ctx.size(ids["path"]), device="cuda"))
     assert e.value.status == "UNSUPPORTED"
     ctx.close()
+
+
+def test_stratified_negation_matches_oracle():
+    # set difference with tags kept; wildcard in the negated atom; two fixed columns; negation over a recursive lower stratum
+    a = np.sort(synth.randint(5, 1, 0, 3000, 5000).astype(np.int32))
+    b = np.sort(synth.randint(5, 2, 0, 3000, 5000).astype(np.int32))
+    prog = W.Program("diff", {"a": (1, W.MINPLUS), "b": (1, W.MINPLUS), "only_a": (1, W.MINPLUS)},
+                     [W.Rule("only_a", (W.V(0),), (W.Atom("a", (W.Var(0),)), W.Atom("b", (W.Var(0),), negated=True)))],
+                     {"a": ([a], synth.normal(5, 3, 3000).astype(np.float32)), "b": ([b], None)}, ("only_a",))
+    ctx, gids, _, o, oids, _, _ = both(prog)
+    rep = H.compare_relations(ctx.read(gids["only_a"]), o.read(oids["only_a"]), what="only_a")
+    assert rep["bit_unequal"] == 0 and set(ctx.read(gids["only_a"])[0][0].tolist()) == set(a.tolist()) - set(b.tolist())
+    ctx.close()
+    s, d = synth.uniform_digraph(300, 900, 23)
+    w = synth.log_prob_tags(900, 23)
+    prog = W.Program("neg2", {"edge": (2, W.MAXPLUS), "sink": (1, W.MAXPLUS), "oneway": (2, W.MAXPLUS)},
+                     [W.Rule("sink", (W.V(1),), (W.Atom("edge", (W.Var(0), W.Var(1))), W.Atom("edge", (W.Var(1), W.Var(2)), negated=True))),
+                      W.Rule("oneway", (W.V(0), W.V(1)), (W.Atom("edge", (W.Var(0), W.Var(1))), W.Atom("edge", (W.Var(1), W.Var(0)), negated=True)))],
+                     {"edge": ([s, d], w)}, ("sink", "oneway"))
+    ctx, gids, _, o, oids, _, _ = both(prog)
+    for name in ("sink", "oneway"):
+        assert H.compare_relations(ctx.read(gids[name]), o.read(oids[name]), what=name)["bit_unequal"] == 0
+    ctx.close()
+    prog = W.config2(scale=10)
+    n = 1 << 10
+    prog.relations["node"] = (1, W.MINPLUS)
+    prog.relations["unreached"] = (1, W.MINPLUS)
+    prog.facts["node"] = ([np.arange(n, dtype=np.int32)], None)
+    prog.rules.append(W.Rule("unreached", (W.V(0),), (W.Atom("node", (W.Var(0),)), W.Atom("dist", (W.Var(0),), negated=True))))
+    prog.outputs = ("dist", "unreached")
+    ctx, gids, _, o, oids, _, _ = both(prog)
+    for name in prog.outputs:
+        assert H.compare_relations(ctx.read(gids[name]), o.read(oids[name]), what=name)["bit_unequal"] == 0
+    assert ctx.size(gids["dist"]) + ctx.size(gids["unreached"]) == n
+    ctx.close()
+    # negation through recursion is rejected
+    from paper_2609_27203_b200 import xlog
+    bad = W.Program("bad", {"e": (1, W.MINPLUS), "p": (1, W.MINPLUS)},
+                    [W.Rule("p", (W.V(0),), (W.Atom("e", (W.Var(0),)), W.Atom("p", (W.Var(0),), negated=True)))],
+                    {"e": ([np.array([1], np.int32)], None)})
+    c2, _, _ = xlog.load_program(bad, arena_bytes=1 << 24)
+    with pytest.raises(xlog.XlogError) as e:
+        c2.fixpoint()
+    assert e.value.status == "UNSUPPORTED"
+    c2.close()
