@@ -74,6 +74,7 @@ typedef struct {
 
 #define XLOG_FLAG_CHECK_INVARIANTS 1u  /* after every load/merge verify keys strictly increase (slow, for tests) */
 #define XLOG_FLAG_PROFILE          2u  /* CUDA events around every kernel launch; read with xlog_profile_read */
+#define XLOG_FLAG_NO_TAG_MIRROR    4u  /* evaluate every recursive component by sort -> reduce-by-key -> merge, never through a tag mirror */
 
 /* ---- context --------------------------------------------------------------- */
 xlog_status xlog_ctx_create(const xlog_config* cfg, xlog_ctx** out);
@@ -157,7 +158,8 @@ typedef struct {
   int64_t  iterations;             /* join rounds over all components, seed rounds included */
   int64_t  derived_tuples;         /* sum over rule heads of rows - loaded facts */
   int64_t  candidates;             /* join outputs before aggregation */
-  int64_t  unique_candidates;      /* after reduce-by-key */
+  int64_t  unique_candidates;      /* after reduce-by-key; -1 if a component was evaluated through a tag mirror,
+                                      which never forms the list of distinct candidate keys */
   int64_t  new_tuples;
   int64_t  improved_tags;
   int64_t  h2d_bytes, d2h_bytes;   /* control traffic of this call (counters only) */

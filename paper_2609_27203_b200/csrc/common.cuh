@@ -155,4 +155,8 @@ __device__ __forceinline__ T block_scan_excl(T v, T* sh, T& total) {
   return r;
 }
 
+// order-preserving map float -> int32 (so integer atomicMin/atomicMax implement the float ones)
+__device__ __forceinline__ int32_t f2ord(float f) { const int32_t i = __float_as_int(f); return i ^ ((i >> 31) & 0x7fffffff); }
+__device__ __forceinline__ float ord2f(int32_t i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
+
 }  // namespace xlog

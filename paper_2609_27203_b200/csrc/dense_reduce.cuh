@@ -23,10 +23,6 @@ constexpr int kDenseBlock = 256;
 constexpr int kDensePer = kDenseSlots / kDenseBlock;   // table slots owned by one thread at emit time
 constexpr int kDenseMaxGroupBits = 16;
 
-// order-preserving map float -> int32 (so integer atomicMin/atomicMax implement the float ones)
-__device__ __forceinline__ int32_t f2ord(float f) { const int32_t i = __float_as_int(f); return i ^ ((i >> 31) & 0x7fffffff); }
-__device__ __forceinline__ float ord2f(int32_t i) { return __int_as_float(i ^ ((i >> 31) & 0x7fffffff)); }
-
 template <typename Op> struct DenseOp;
 template <> struct DenseOp<OpMin> {
   static constexpr int32_t empty = 0x7fffffff;

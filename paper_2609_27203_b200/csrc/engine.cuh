@@ -145,6 +145,7 @@ struct Ctx {
   std::vector<ProfPending> prof_pending;
   std::vector<cudaEvent_t> ev_pool;
   int64_t note_bytes = 0;                 // algorithmic bytes of the next launch (consumed by the launch macro)
+  bool unique_untracked = false;          // a stratum went through the tag mirror, which does not count distinct candidate keys
   std::vector<char> stratum_done;         // per relation: its stratum has been evaluated in the running fixpoint
 };
 

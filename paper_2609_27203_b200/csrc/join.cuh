@@ -171,6 +171,38 @@ struct BwdArgs {
 
 enum { kExpFast = 0, kExpGeneric = 1, kExpBackward = 2 };
 
+// Where a candidate goes.  kSinkWrite: into the candidate arrays (to be sorted and reduced).  kSinkMin / kSinkMax:
+// straight into the head relation's tag mirror, a table with one order-mapped tag per possible head key
+// (max / min are idempotent and order-independent, so "oplus into the slot" is one atomic and needs no sort).
+// A candidate that improves its slot sets the key's bit in `changed`; the thread that replaces the empty marker
+// counts a new tuple.  The slot is read first because most candidates of a fixpoint round do not improve anything.
+enum { kSinkWrite = 0, kSinkMin = 1, kSinkMax = 2 };
+struct MirrorArgs {
+  int32_t* table;               // 2^key_bits order-mapped tags; kMirrorEmptyMin / kMirrorEmptyMax where no tuple is
+  uint32_t* changed;            // one bit per key
+  unsigned long long* n_new;    // running count of keys that left the empty state
+  uint32_t key_max;             // last valid key; anything above raises the head-range error instead of being stored
+  uint32_t* err;
+};
+constexpr int32_t kMirrorEmptyMin = 0x7fffffff;
+constexpr int32_t kMirrorEmptyMax = (int32_t)0x80000000;
+
+template <int SINK>
+__device__ __forceinline__ void mirror_commit(const MirrorArgs& m, uint32_t key, int32_t v, uint32_t& n_new) {
+  const int32_t old = SINK == kSinkMin ? atomicMin(m.table + key, v) : atomicMax(m.table + key, v);
+  if (SINK == kSinkMin ? v < old : v > old) {
+    atomicOr(m.changed + (key >> 5), 1u << (key & 31));
+    if (old == (SINK == kSinkMin ? kMirrorEmptyMin : kMirrorEmptyMax)) ++n_new;
+  }
+}
+template <int SINK>
+__device__ __forceinline__ void mirror_apply(const MirrorArgs& m, uint32_t key, float tag, uint32_t& n_new) {
+  const int32_t v = f2ord(tag);
+  if (key > m.key_max) { atomicOr(m.err, kErrHeadRange); return; }
+  const int32_t cur = __ldcg(m.table + key);
+  if (SINK == kSinkMin ? v < cur : v > cur) mirror_commit<SINK>(m, key, v, n_new);
+}
+
 // One thread per tile: the first and last outer row that contribute candidates to the tile
 // (r_lo = last row with start <= tile begin, r_hi = last row with start < tile end).  Done for all
 // tiles at once so that the dependent binary-search loads of one tile overlap with those of the others.
@@ -198,12 +230,12 @@ static __global__ void __launch_bounds__(256) k_expand_partition(const uint64_t*
 // (global candidate index of each outer row's first match).  The outer rows covering the tile are
 // staged in shared memory (their starts relative to the tile and their row records), so the per-
 // candidate work is a short binary search in shared memory plus the coalesced inner reads.
-template <typename KO, typename KH, int MODE>
+template <typename KO, typename KH, int MODE, int SINK = kSinkWrite>
 __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
                                                            const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo,
                                                            const uint2* __restrict__ tile_rows, uint64_t out_lo, uint64_t out_hi,
                                                            KH* __restrict__ ckeys,
-                                                           float* __restrict__ ctags, uint32_t* __restrict__ err, BwdArgs bw) {
+                                                           float* __restrict__ ctags, uint32_t* __restrict__ err, BwdArgs bw, MirrorArgs mr) {
   __shared__ uint32_t sstart[kExpRows];
   __shared__ uint4 sinfo[kExpRows];
   __shared__ uint16_t srowidx[kExpTile];             // staged row of every candidate position of the tile
@@ -264,29 +296,62 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
     const KH m0 = (KH)S.inner_mult[0];
     const int nin = S.has_inner ? S.inner_free : -1;                 // -1: one-atom rule
     const bool times = S.times != 0;
+    uint32_t n_new = 0;
+    // three sweeps over the thread's items, so that the loads of one kind are all in flight together: (1) row record
+    // from shared memory, inner tag and columns from global memory; (2) for the mirror, the current slot values;
+    // (3) the stores, or the atomics of the few candidates that improve their slot
+    KH key[kExpItems];
+    float tag[kExpItems];
 #pragma unroll
     for (int k = 0; k < kExpItems; ++k) {
       const uint32_t q = threadIdx.x + k * kExpBlock;
+      key[k] = 0; tag[k] = 0.f;
       if (q < ntile) {
         const uint32_t li = srowidx[q];
         const uint4 info = sinfo[li];
         const uint32_t ir = info.x + (li ? q - sstart[li] : q + j0);
-        KH key = (KH)(((uint64_t)info.w << 32) | info.z);
-        float tag = __uint_as_float(info.y);
+        key[k] = (KH)(((uint64_t)info.w << 32) | info.z);
+        tag[k] = __uint_as_float(info.y);
         if (nin >= 0) {
           const float it = itg[ir];
-          tag = times ? tag * it : tag + it;
-          if (nin >= 1) key += (KH)(uint32_t)ic0[ir] * m0;
-          for (int c = 1; c < nin; ++c) key += (KH)(uint32_t)S.inner_col[c][ir] * (KH)S.inner_mult[c];
+          tag[k] = times ? tag[k] * it : tag[k] + it;
+          if (nin >= 1) key[k] += (KH)(uint32_t)ic0[ir] * m0;
+          for (int c = 1; c < nin; ++c) key[k] += (KH)(uint32_t)S.inner_col[c][ir] * (KH)S.inner_mult[c];
         }
-        kout[q] = key;
-        tout[q] = tag;
       }
+    }
+    if (SINK == kSinkWrite) {
+#pragma unroll
+      for (int k = 0; k < kExpItems; ++k) {
+        const uint32_t q = threadIdx.x + k * kExpBlock;
+        if (q < ntile) { kout[q] = key[k]; tout[q] = tag[k]; }
+      }
+    } else {
+      int32_t cur[kExpItems];
+#pragma unroll
+      for (int k = 0; k < kExpItems; ++k) {
+        const uint32_t q = threadIdx.x + k * kExpBlock;
+        cur[k] = SINK == kSinkMin ? (int32_t)0x80000000 : 0x7fffffff;        // nothing improves on this
+        if (q < ntile) {
+          if ((uint32_t)key[k] > mr.key_max) atomicOr(mr.err, kErrHeadRange);
+          else cur[k] = __ldcg(mr.table + (uint32_t)key[k]);
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < kExpItems; ++k) {
+        const int32_t v = f2ord(tag[k]);
+        if (SINK == kSinkMin ? v < cur[k] : v > cur[k]) mirror_commit<SINK>(mr, (uint32_t)key[k], v, n_new);
+      }
+    }
+    if (SINK != kSinkWrite) {
+      n_new = __reduce_add_sync(0xffffffffu, n_new);
+      if (lane_id() == 0 && n_new) atomicAdd(mr.n_new, (unsigned long long)n_new);
     }
     return;
   }
 
   uint32_t e = 0;
+  uint32_t n_new = 0;
   for (uint32_t q = threadIdx.x; q < (uint32_t)(t_hi - t_lo); q += kExpBlock) {
     const uint64_t p = t_lo + q;
     uint32_t row, j;
@@ -317,8 +382,8 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
 #pragma unroll
       for (int c = 0; c < kMaxArity - 1; ++c)
         if (c < S.inner_free) key += (KH)(uint32_t)S.inner_col[c][ir] * (KH)S.inner_mult[c];
-      ckeys[q + (t_lo - out_lo)] = key;
-      ctags[q + (t_lo - out_lo)] = tag;
+      if (SINK == kSinkWrite) { ckeys[q + (t_lo - out_lo)] = key; ctags[q + (t_lo - out_lo)] = tag; }
+      else mirror_apply<SINK>(mr, (uint32_t)key, tag, n_new);
       continue;
     }
     int64_t var[kMaxVars];
@@ -347,8 +412,8 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
         key |= (KH)(uint32_t)h << S.head.shift[c];
       }
     if (MODE != kExpBackward) {
-      ckeys[p - out_lo] = key;
-      ctags[p - out_lo] = tag;
+      if (SINK == kSinkWrite) { ckeys[p - out_lo] = key; ctags[p - out_lo] = tag; }
+      else if (!e) mirror_apply<SINK>(mr, (uint32_t)key, tag, n_new);
     } else {
       // head row of this binding: lower bound of the key among the stored head keys
       const KH* hk = reinterpret_cast<const KH*>(bw.head_keys);
@@ -369,6 +434,7 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
     }
   }
   if (e) atomicOr(err, e);
+  if (SINK != kSinkWrite && n_new) atomicAdd(mr.n_new, (unsigned long long)n_new);
 }
 
 }  // namespace xlog

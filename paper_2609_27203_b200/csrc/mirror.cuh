@@ -1,0 +1,117 @@
+// Tag mirror of a max/min head relation: a direct-addressed table with one order-mapped tag per
+// possible packed key, used by the fixpoint of a linear recursive rule set in place of
+// sort -> reduce-by-key -> diff/merge (Algorithm 1 lines 6-9).  The join kernel applies every
+// candidate to its slot with one atomic max/min; the keys whose slot improved in a round are
+// flagged in a bitmap, and compacting that bitmap in key order yields the next delta, already
+// sorted and free of duplicates.  After the last round the table itself is compacted into the
+// relation's sorted (key, tag) arrays.  max and min are exact and order-independent, so the
+// relation is bit-identical to the one the sorting path derives.
+//
+//   k_mirror_scatter        loaded facts -> table
+//   k_mirror_changed_count  set bits per 32768-key tile of the changed bitmap
+//   k_mirror_changed_emit   bitmap -> delta (keys ascending, tags read from the table); clears the bitmap
+//   k_mirror_full_count     occupied slots per 4096-slot tile
+//   k_mirror_full_emit      table -> relation
+#pragma once
+#include "common.cuh"
+
+namespace xlog {
+
+constexpr int kMirBlock = 256;
+constexpr int kMirWordsPerTile = kMirBlock * 4;        // bitmap words per tile (one uint4 per thread)
+constexpr int kMirSlotsPerTile = kMirBlock * 16;       // table slots per tile (four int4 per thread)
+
+template <typename K>
+__global__ void __launch_bounds__(256) k_mirror_scatter(const K* __restrict__ keys, const float* __restrict__ tags, uint32_t n,
+                                                        int32_t* __restrict__ table) {
+  const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) table[keys[i]] = f2ord(tags[i]);
+}
+
+// nquads = number of uint4 groups of the bitmap (its length is padded to a multiple of four words)
+static __global__ void __launch_bounds__(kMirBlock) k_mirror_changed_count(const uint4* __restrict__ bitmap, uint32_t nquads,
+                                                                           uint32_t* __restrict__ tile_sums) {
+  __shared__ uint32_t sh[kMirBlock / 32 + 1];
+  const uint32_t q = blockIdx.x * kMirBlock + threadIdx.x;
+  uint32_t s = 0;
+  if (q < nquads) { const uint4 w = bitmap[q]; s = __popc(w.x) + __popc(w.y) + __popc(w.z) + __popc(w.w); }
+  uint32_t total;
+  block_scan_excl<kMirBlock, uint32_t>(s, sh, total);
+  if (threadIdx.x == 0) tile_sums[blockIdx.x] = total;
+}
+
+template <typename K>
+__global__ void __launch_bounds__(kMirBlock) k_mirror_changed_emit(uint4* __restrict__ bitmap, uint32_t nquads,
+                                                                   const uint32_t* __restrict__ tile_base, const int32_t* __restrict__ table,
+                                                                   K* __restrict__ keys, float* __restrict__ tags) {
+  __shared__ uint32_t sh[kMirBlock / 32 + 1];
+  const uint32_t q = blockIdx.x * kMirBlock + threadIdx.x;
+  uint4 w = make_uint4(0, 0, 0, 0);
+  if (q < nquads) w = bitmap[q];
+  const uint32_t s = __popc(w.x) + __popc(w.y) + __popc(w.z) + __popc(w.w);
+  uint32_t total;
+  uint32_t pos = tile_base[blockIdx.x] + block_scan_excl<kMirBlock, uint32_t>(s, sh, total);
+  if (s == 0) return;
+  uint32_t word[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+  for (int j = 0; j < 4; ++j) {
+    uint32_t bits = word[j];
+    const uint32_t base = (q * 4 + j) << 5;
+    while (bits) {
+      const int b = __ffs(bits) - 1;
+      bits &= bits - 1;
+      const uint32_t key = base + b;
+      keys[pos] = (K)key;
+      tags[pos] = ord2f(__ldcg(table + key));
+      ++pos;
+    }
+  }
+  bitmap[q] = make_uint4(0, 0, 0, 0);
+}
+
+// Slots are read in a striped arrangement (coalesced int4 loads); the output order is the slot order, so the four
+// stripes of a tile are scanned one after the other.
+static __global__ void __launch_bounds__(kMirBlock) k_mirror_full_count(const int4* __restrict__ table4, uint64_t nquads, int32_t empty,
+                                                                        uint32_t* __restrict__ tile_sums) {
+  __shared__ uint32_t sh[kMirBlock / 32 + 1];
+  uint32_t s = 0;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint64_t q = ((uint64_t)blockIdx.x * 4 + i) * kMirBlock + threadIdx.x;
+    if (q < nquads) {
+      const int4 v = table4[q];
+      s += (v.x != empty) + (v.y != empty) + (v.z != empty) + (v.w != empty);
+    }
+  }
+  uint32_t total;
+  block_scan_excl<kMirBlock, uint32_t>(s, sh, total);
+  if (threadIdx.x == 0) tile_sums[blockIdx.x] = total;
+}
+
+template <typename K>
+__global__ void __launch_bounds__(kMirBlock) k_mirror_full_emit(const int4* __restrict__ table4, uint64_t nquads, int32_t empty,
+                                                                const uint32_t* __restrict__ tile_base, K* __restrict__ keys,
+                                                                float* __restrict__ tags) {
+  __shared__ uint32_t sh[kMirBlock / 32 + 1];
+  uint32_t run = tile_base[blockIdx.x];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const uint64_t q = ((uint64_t)blockIdx.x * 4 + i) * kMirBlock + threadIdx.x;
+    int4 v = make_int4(empty, empty, empty, empty);
+    if (q < nquads) v = table4[q];
+    const uint32_t s = (v.x != empty) + (v.y != empty) + (v.z != empty) + (v.w != empty);
+    uint32_t total;
+    uint32_t pos = run + block_scan_excl<kMirBlock, uint32_t>(s, sh, total);
+    run += total;
+    const int32_t e[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j)
+      if (e[j] != empty) {
+        keys[pos] = (K)(q * 4 + j);
+        tags[pos] = ord2f(e[j]);
+        ++pos;
+      }
+  }
+}
+
+}  // namespace xlog

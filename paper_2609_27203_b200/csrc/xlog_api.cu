@@ -1,5 +1,6 @@
 // C ABI of the engine (see include/xlog.h) and the host-side fixpoint driver.
 #include "engine.cuh"
+#include "mirror.cuh"
 #include "triangle.cuh"
 
 using namespace xlog;
@@ -495,9 +496,10 @@ void count_variant(Ctx* c, const Variant& v, const Relation& H, Counted& q, int 
               (const uint64_t*)q.sums.as<uint64_t>(), q.start.as<uint64_t>());
 }
 
-// materialise candidates [lo, hi) of a counted variant into (ckeys, ctags), or (MODE == kExpBackward) run the backward scatter
-template <int MODE>
-void launch_expand_mode(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, void* ckeys, float* ctags, const BwdArgs& bw) {
+// materialise candidates [lo, hi) of a counted variant into (ckeys, ctags), or (MODE == kExpBackward) run the backward
+// scatter, or (SINK != kSinkWrite) apply them to the head relation's tag mirror
+template <int MODE, int SINK>
+void launch_expand_mode(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, void* ckeys, float* ctags, const BwdArgs& bw, const MirrorArgs& mr) {
   const unsigned blocks = (unsigned)((hi - lo + kExpTile - 1) / kExpTile);
   const uint64_t* st = q.start.as<uint64_t>();
   const uint4* ri = q.rowinfo.as<uint4>();
@@ -511,19 +513,33 @@ void launch_expand_mode(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, v
   const uint2* tr = tile_rows.as<uint2>();
   c->note_bytes = bytes;
   if (q.outer.key_bytes == 4 && ckb == 4)
-    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint32_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.n, st, ri, tr, lo, hi, (uint32_t*)ckeys, ctags, err, bw);
-  else if (q.outer.key_bytes == 4)
-    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint64_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.n, st, ri, tr, lo, hi, (uint64_t*)ckeys, ctags, err, bw);
+    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint32_t, MODE, SINK>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.n, st, ri, tr, lo, hi, (uint32_t*)ckeys, ctags, err, bw, mr);
   else if (ckb == 4)
-    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint32_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.n, st, ri, tr, lo, hi, (uint32_t*)ckeys, ctags, err, bw);
+    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint32_t, MODE, SINK>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.n, st, ri, tr, lo, hi, (uint32_t*)ckeys, ctags, err, bw, mr);
+  else if (SINK != kSinkWrite)
+    fail(XLOG_ERR_INTERNAL, "tag mirror with wide keys");
+  else if (q.outer.key_bytes == 4)
+    XLOG_LAUNCH(c, (k_join_expand<uint32_t, uint64_t, MODE, kSinkWrite>), blocks, kExpBlock, 0, q.spec, (const uint32_t*)q.outer.keys, q.outer.n, st, ri, tr, lo, hi, (uint64_t*)ckeys, ctags, err, bw, mr);
   else
-    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint64_t, MODE>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.n, st, ri, tr, lo, hi, (uint64_t*)ckeys, ctags, err, bw);
+    XLOG_LAUNCH(c, (k_join_expand<uint64_t, uint64_t, MODE, kSinkWrite>), blocks, kExpBlock, 0, q.spec, (const uint64_t*)q.outer.keys, q.outer.n, st, ri, tr, lo, hi, (uint64_t*)ckeys, ctags, err, bw, mr);
 }
 template <bool BWD>
 void launch_expand(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, void* ckeys, float* ctags, const BwdArgs& bw) {
-  if (BWD) launch_expand_mode<kExpBackward>(c, q, lo, hi, ckb, ckeys, ctags, bw);
-  else if (q.spec.fast) launch_expand_mode<kExpFast>(c, q, lo, hi, ckb, ckeys, ctags, bw);
-  else launch_expand_mode<kExpGeneric>(c, q, lo, hi, ckb, ckeys, ctags, bw);
+  const MirrorArgs none{};
+  if (BWD) launch_expand_mode<kExpBackward, kSinkWrite>(c, q, lo, hi, ckb, ckeys, ctags, bw, none);
+  else if (q.spec.fast) launch_expand_mode<kExpFast, kSinkWrite>(c, q, lo, hi, ckb, ckeys, ctags, bw, none);
+  else launch_expand_mode<kExpGeneric, kSinkWrite>(c, q, lo, hi, ckb, ckeys, ctags, bw, none);
+}
+// every candidate of a counted variant goes straight into the tag mirror
+void launch_expand_mirror(Ctx* c, Counted& q, bool is_max, const MirrorArgs& mr) {
+  const BwdArgs bw{};
+  if (q.spec.fast) {
+    if (is_max) launch_expand_mode<kExpFast, kSinkMax>(c, q, 0, q.total, 4, nullptr, nullptr, bw, mr);
+    else launch_expand_mode<kExpFast, kSinkMin>(c, q, 0, q.total, 4, nullptr, nullptr, bw, mr);
+  } else {
+    if (is_max) launch_expand_mode<kExpGeneric, kSinkMax>(c, q, 0, q.total, 4, nullptr, nullptr, bw, mr);
+    else launch_expand_mode<kExpGeneric, kSinkMin>(c, q, 0, q.total, 4, nullptr, nullptr, bw, mr);
+  }
 }
 
 constexpr int kSlotTotals = 16;          // uint64 candidate totals of the variants of a round
@@ -930,6 +946,148 @@ void stratum_once(Ctx* c, int head, const std::vector<const RuleC*>& rs) {
   c->r_new += (int64_t)H.n - H.n_facts;
 }
 
+// Which atom a rule scans in the seed round (every atom reads its full relation): the recursive side if exactly one atom
+// is recursive, else whichever side has an index path.
+int seed_outer(const std::vector<int>& comp, const RuleC* r) {
+  int outer = 0;
+  if (r->kind == 2) {
+    const bool in0 = in_set(comp, r->plan.atoms[0].rel), in1 = in_set(comp, r->plan.atoms[1].rel);
+    // scan the recursive side and look up the stable side; with two recursive atoms (non-linear rule)
+    // the looked-up side is the full relation, indexed afresh in every round it changed
+    outer = in1 && !in0 ? 1 : 0;
+    if (!r->shape[outer].ok) { if (in0 == in1 && r->shape[1 - outer].ok) outer = 1 - outer; else fail(XLOG_ERR_UNSUPPORTED, "no index path for this rule"); }
+  }
+  return outer;
+}
+
+constexpr int kSlotMirNew = 12, kSlotMirChanged = 13;
+constexpr int kMirrorMaxBits = 30;
+
+// The tag mirror serves a component of one max/min relation whose rules are all linear (at most one atom over the
+// relation itself, and that atom is the scanned side): then the relation is only ever read through its delta, and
+// its sorted form is needed again only after the last round.
+bool mirror_applies(Ctx* c, const std::vector<int>& comp, const std::vector<const RuleC*>& rs) {
+  if ((c->flags & XLOG_FLAG_NO_TAG_MIRROR) || comp.size() != 1) return false;
+  const Relation& H = *c->rels[comp[0]];
+  if (H.sr != XLOG_SR_MAXPLUS && H.sr != XLOG_SR_MINPLUS) return false;
+  if (H.layout.total_bits > kMirrorMaxBits || H.key_bytes != 4) return false;
+  for (const RuleC* r : rs) {
+    if (r->plan.emit_count_column || r->kind == 3 || r->kind == 4) return false;
+    int in = 0, pos = 0;
+    for (int j = 0; j < r->plan.n_atoms; ++j)
+      if (r->plan.atoms[j].rel == comp[0]) { if (r->plan.atoms[j].negated) return false; ++in; pos = j; }
+    if (in > 1) return false;
+    if (in == 1 && r->kind == 2 && !r->shape[pos].ok) return false;
+    if (in == 1 && r->kind != 2 && pos != 0) return false;
+    if (in == 0 && r->kind == 2 && !r->shape[0].ok && !r->shape[1].ok) return false;
+  }
+  const uint64_t need = ((uint64_t)4 << H.layout.total_bits) + ((uint64_t)1 << H.layout.total_bits) / 8 + (1u << 20);
+  return need <= c->arena.largest_free() / 2;
+}
+
+// Algorithm 1 over a tag mirror (mirror.cuh): per round  count -> scan -> join straight into the table -> compact the
+// changed bitmap into the next delta.  No candidate is ever written to memory.
+void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs) {
+  Relation& H = *c->rels[h];
+  const std::vector<int> comp{h};
+  const uint64_t dom = (uint64_t)1 << H.layout.total_bits;
+  const bool is_max = H.sr == XLOG_SR_MAXPLUS;
+  const int32_t empty = is_max ? kMirrorEmptyMax : kMirrorEmptyMin;
+  const uint64_t slots = std::max<uint64_t>(dom, 4);
+  const uint32_t bm_quads = (uint32_t)((std::max<uint64_t>(dom / 32, 1) + 3) / 4);
+  DevBuf table(c, slots * 4), bitmap(c, (size_t)bm_quads * 16);
+  XLOG_LAUNCH(c, k_fill_i32, grid_for(slots, 256 * 8), 256, 0, table.as<int32_t>(), slots, empty);
+  XLOG_CUDA(cudaMemsetAsync(bitmap.p, 0, (size_t)bm_quads * 16, c->stream));
+  // what the relation holds now (its loaded facts, or the result of an earlier fixpoint) is the starting state
+  const uint32_t n_start = H.n;
+  if (n_start)
+    XLOG_LAUNCH(c, (k_mirror_scatter<uint32_t>), grid_for(n_start, 256, 1 << 30), 256, 0, (const uint32_t*)H.keys(), (const float*)H.tags(), n_start,
+                table.as<int32_t>());
+  zero_ctrl(c, kSlotMirNew, 2);
+  const MirrorArgs mr{table.as<int32_t>(), bitmap.as<uint32_t>(), (unsigned long long*)(c->d_ctrl + kSlotMirNew), (uint32_t)(dom - 1),
+                      ctrl_u32(c, kSlotErr)};
+  const unsigned ch_tiles = (bm_quads + kMirBlock - 1) / kMirBlock;
+  DevBuf ch_sums(c, (size_t)ch_tiles * 4);
+  c->unique_untracked = true;
+  KeyTags delta;
+  uint64_t total_new = 0;
+  for (int64_t round = 0;; ++round) {
+    if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
+    ++c->r_iterations;
+    std::vector<Variant> vs;
+    for (const RuleC* r : rs) {
+      if (round == 0) {
+        const int outer = seed_outer(comp, r);
+        vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
+      } else {
+        for (int j = 0; j < r->plan.n_atoms; ++j)
+          if (r->plan.atoms[j].rel == h && delta.n) vs.push_back(Variant{r, j, Source{delta.keys.p, delta.tags.as<float>(), delta.n, H.layout, H.key_bytes}});
+      }
+    }
+    if (vs.size() > 16) fail(XLOG_ERR_UNSUPPORTED, "too many rule variants for one head");
+    std::vector<Counted> counted;
+    counted.reserve(vs.size());
+    for (Variant& v : vs) {
+      if (v.outer.n == 0) continue;
+      counted.emplace_back();
+      count_variant(c, v, H, counted.back(), kSlotTotals + (int)counted.size() - 1);
+    }
+    uint64_t total = 0;
+    if (!counted.empty()) {
+      sync_ctrl(c);
+      for (Counted& q : counted) { q.total = c->h_ctrl[q.slot]; total += q.total; q.deg.reset(); q.sums.reset(); }
+    }
+    c->r_candidates += (int64_t)total;
+    for (Counted& q : counted) {
+      if (q.total) {
+        // per candidate: the looked-up atom's other columns and tag are read, and the key's slot is read (and now and then written)
+        c->note_bytes = (int64_t)q.total * (4 + (q.spec.has_inner ? 4 * (q.spec.inner_free + 1) : 0));
+        launch_expand_mirror(c, q, is_max, mr);
+      }
+      q.start.reset(); q.rowinfo.reset();
+    }
+    delta = KeyTags();
+    if (total == 0) break;
+    XLOG_LAUNCH(c, k_mirror_changed_count, ch_tiles, kMirBlock, 0, (const uint4*)bitmap.as<uint4>(), bm_quads, ch_sums.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, ch_sums.as<uint32_t>(), (int64_t)ch_tiles, ctrl_u32(c, kSlotMirChanged));
+    sync_ctrl(c);
+    const uint32_t changed = (uint32_t)c->h_ctrl[kSlotMirChanged];
+    const uint64_t n_new = c->h_ctrl[kSlotMirNew] - total_new;
+    total_new += n_new;
+    c->r_new += (int64_t)n_new; c->r_improved += (int64_t)changed - (int64_t)n_new;
+    if (changed == 0) break;
+    delta.n = changed;
+    delta.keys = DevBuf(c, (size_t)changed * 4);
+    delta.tags = DevBuf(c, (size_t)changed * 4);
+    c->note_bytes = (int64_t)bm_quads * 16 + (int64_t)changed * 12;
+    XLOG_LAUNCH(c, (k_mirror_changed_emit<uint32_t>), ch_tiles, kMirBlock, 0, bitmap.as<uint4>(), bm_quads, (const uint32_t*)ch_sums.as<uint32_t>(),
+                (const int32_t*)table.as<int32_t>(), delta.keys.as<uint32_t>(), delta.tags.as<float>());
+  }
+  // the relation in sorted form: every occupied slot, in slot order
+  const uint64_t n_out = (uint64_t)n_start + total_new;
+  KeyTags full;
+  full.n = (uint32_t)n_out;
+  full.keys = DevBuf(c, (size_t)std::max<uint64_t>(n_out, 1) * 4);
+  full.tags = DevBuf(c, (size_t)std::max<uint64_t>(n_out, 1) * 4);
+  if (n_out) {
+    const uint64_t nquads = slots / 4;
+    const unsigned tiles = (unsigned)((slots + kMirSlotsPerTile - 1) / kMirSlotsPerTile);
+    DevBuf sums(c, (size_t)tiles * 4);
+    c->note_bytes = (int64_t)slots * 4;
+    XLOG_LAUNCH(c, k_mirror_full_count, tiles, kMirBlock, 0, (const int4*)table.as<int4>(), nquads, empty, sums.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, sums.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotA));
+    c->note_bytes = (int64_t)slots * 4 + (int64_t)n_out * 8;
+    XLOG_LAUNCH(c, (k_mirror_full_emit<uint32_t>), tiles, kMirBlock, 0, (const int4*)table.as<int4>(), nquads, empty, (const uint32_t*)sums.as<uint32_t>(),
+                full.keys.as<uint32_t>(), full.tags.as<float>());
+  }
+  set_current(H, std::move(full));
+  if (c->flags & XLOG_FLAG_CHECK_INVARIANTS) {
+    XLOG_LAUNCH(c, (k_check_sorted<uint32_t>), grid_for(H.n, 256), 256, 0, (const uint32_t*)H.keys(), (int64_t)H.n, ctrl_u32(c, kSlotErr));
+    sync_ctrl(c);
+    if ((uint64_t)(uint32_t)c->h_ctrl[kSlotA] != n_out) fail(XLOG_ERR_INTERNAL, "tag mirror: occupied slots disagree with the tuple count");
+  }
+}
+
 // Recursive component: Algorithm 1 with tag improvement.
 void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<const RuleC*>& rs) {
   for (int p : comp) if (c->rels[p]->sr != XLOG_SR_MAXPLUS && c->rels[p]->sr != XLOG_SR_MINPLUS)
@@ -938,6 +1096,7 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
     if (r->plan.emit_count_column) fail(XLOG_ERR_UNSUPPORTED, "count inside a recursive component");
     if (r->kind == 3 || r->kind == 4) fail(XLOG_ERR_UNSUPPORTED, "triangle rule inside a recursive component");
   }
+  if (mirror_applies(c, comp, rs)) { stratum_recursive_mirror(c, comp[0], rs); return; }
   std::vector<KeyTags> delta(c->rels.size());
   for (int64_t round = 0;; ++round) {
     if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
@@ -950,14 +1109,7 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
       for (const RuleC* r : rs) {
         if (r->plan.head_rel != h) continue;
         if (round == 0) {                                   // seed: every atom reads the full relation
-          int outer = 0;
-          if (r->kind == 2) {
-            const bool in0 = in_set(comp, r->plan.atoms[0].rel), in1 = in_set(comp, r->plan.atoms[1].rel);
-            // scan the recursive side and look up the stable side; with two recursive atoms (non-linear rule)
-            // the looked-up side is the full relation, indexed afresh in every round it changed
-            outer = in1 && !in0 ? 1 : 0;
-            if (!r->shape[outer].ok) { if (in0 == in1 && r->shape[1 - outer].ok) outer = 1 - outer; else fail(XLOG_ERR_UNSUPPORTED, "no index path for this rule"); }
-          }
+          const int outer = seed_outer(comp, r);
           vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
         } else {
           for (int j = 0; j < r->plan.n_atoms; ++j) {
@@ -1170,6 +1322,7 @@ xlog_status xlog_fixpoint(xlog_ctx* c, xlog_receipt* receipt) {
   if (receipt && receipt->struct_size != sizeof(xlog_receipt)) return XLOG_ERR_INVALID_ARGUMENT;
   const int64_t l0 = c->launches, d0 = c->d2h_bytes, h0 = c->h2d_bytes;
   c->r_candidates = c->r_unique = c->r_new = c->r_improved = c->r_iterations = c->r_strata = 0;
+  c->unique_untracked = false;
   c->arena.reset_peak();
   cudaSetDevice(c->device);
   cudaEventRecord(c->ev0, c->stream);
@@ -1192,7 +1345,7 @@ xlog_status xlog_fixpoint(xlog_ctx* c, xlog_receipt* receipt) {
     if (st == XLOG_OK) for (Relation* R : c->rels) if (R->is_head) derived += (int64_t)R->n - R->n_facts;
     receipt->derived_tuples = derived;
     receipt->candidates = c->r_candidates;
-    receipt->unique_candidates = c->r_unique;
+    receipt->unique_candidates = c->unique_untracked ? -1 : c->r_unique;
     receipt->new_tuples = c->r_new;
     receipt->improved_tags = c->r_improved;
     receipt->h2d_bytes = c->h2d_bytes - h0;

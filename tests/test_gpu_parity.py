@@ -32,16 +32,30 @@ def oracle_run(program, mode="seminaive"):
 
 
 def check_program(program, rel_tol=MINMAX_REL, abs_tol=0.0, expect_bit_equal=True, mode="seminaive", **kw):
-    ctx, gids, _, receipt = gpu_run(program, **kw)
+    """Both evaluation paths of the CUDA engine against the oracle: the default one (a linear max/min recursion goes
+    through the tag mirror) and the one that always sorts, reduces by key and merges.  The two must agree with each
+    other bit for bit, relation and counters alike."""
+    from paper_2609_27203_b200 import xlog
     o, oids, _, stats = oracle_run(program, mode)
+    receipts, results = [], []
+    for extra in (0, xlog.FLAG_NO_TAG_MIRROR):
+        ctx, gids, _, receipt = gpu_run(program, **dict(kw, flags=kw.get("flags", xlog.FLAG_CHECK_INVARIANTS) | extra))
+        got = {}
+        for name in program.outputs:
+            got[name] = ctx.read(gids[name])
+            rep = H.compare_relations(got[name], o.read(oids[name]), rel_tol=rel_tol, abs_tol=abs_tol,
+                                      what=f"{program.name}:{name}")
+            if expect_bit_equal:
+                assert rep["bit_unequal"] == 0, rep
+        assert receipt["derived_tuples"] == stats["derived_tuples"]
+        ctx.close()
+        receipts.append(receipt); results.append(got)
     for name in program.outputs:
-        rep = H.compare_relations(ctx.read(gids[name]), o.read(oids[name]), rel_tol=rel_tol, abs_tol=abs_tol,
-                                  what=f"{program.name}:{name}")
-        if expect_bit_equal:
-            assert rep["bit_unequal"] == 0, rep
-    assert receipt["derived_tuples"] == stats["derived_tuples"]
-    ctx.close()
-    return receipt, stats
+        assert H.compare_relations(results[0][name], results[1][name], what="mirror vs sorted path")["bit_unequal"] == 0
+    for k in ("iterations", "candidates", "new_tuples", "improved_tags", "derived_tuples", "strata"):
+        assert receipts[0][k] == receipts[1][k], (k, receipts[0][k], receipts[1][k])
+    assert receipts[1]["unique_candidates"] >= 0
+    return receipts[0], stats
 
 
 # ---- relation store: load / read ---------------------------------------------------------
