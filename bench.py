@@ -36,7 +36,7 @@ UNIT = "tuples/s"
 NCU_TRAFFIC_RATIO = {"k_sort_pass": 0.99, "k_join_expand": 0.92, "k_dense_reduce": 1.04, "k_merge": 1.0}
 
 
-def make_program(name: str, scale: int | None):
+def make_program(name: str, scale: int | None, sources: int | None = None):
     from paper_2609_27203_b200 import workloads as W
     if name == "sssp":
         return W.config2(scale=scale or 20), 4 << 30
@@ -44,7 +44,8 @@ def make_program(name: str, scale: int | None):
         return W.config1(), 1 << 28
     if name == "reach":
         s = scale or 22
-        return W.config5(scale=s), (56 << 30) if s >= 21 else (8 << 30)
+        ns = sources or 64
+        return W.config5(scale=s, n_sources=ns), (56 << 30) if s >= 21 and ns > 16 else (8 << 30)
     if name == "triangles":
         return W.config3(scale=scale or 18), 2 << 30
     if name == "digits":
@@ -189,10 +190,11 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
-    program, arena = make_program(args.workload, args.scale)
+    program, arena = make_program(args.workload, args.scale, args.sources)
 
     # facts resident in HBM before any timed region
-    ctx, ids, rules = xlog.load_program(program, device=local_rank, arena_bytes=arena, device_inputs=True)
+    base_flags = xlog.FLAG_NO_TAG_MIRROR if args.no_tag_mirror else 0
+    ctx, ids, rules = xlog.load_program(program, device=local_rank, arena_bytes=arena, device_inputs=True, flags=base_flags)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)          # > 126 MB L2
 
     def step(c):
@@ -227,7 +229,7 @@ def run_ours(args):
     # per-kernel timing: the same steps again with CUDA events around every launch
     ctx.close()
     pctx, pids, _ = xlog.load_program(program, device=local_rank, arena_bytes=arena, device_inputs=True,
-                                      flags=xlog.FLAG_PROFILE)
+                                      flags=xlog.FLAG_PROFILE | base_flags)
     step(pctx)
     pctx.profile_reset()
     for _ in range(args.steps):
@@ -262,7 +264,7 @@ def run_ours(args):
         pinned[name] = (pc, pt)
         h2d += sum(c.numel() * 4 for c in pc) + (0 if pt is None else pt.numel() * 4)
     empty = type(program)(program.name, program.relations, program.rules, {}, program.outputs)
-    ectx, eids, _ = xlog.load_program(empty, device=local_rank, arena_bytes=arena)
+    ectx, eids, _ = xlog.load_program(empty, device=local_rank, arena_bytes=arena, flags=base_flags)
 
     def e2e_step():
         t0 = time.perf_counter()
@@ -359,6 +361,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="sssp", choices=["sssp", "closure", "reach", "triangles", "digits"])
     ap.add_argument("--scale", type=int, default=None, help="R-MAT scale override (smaller cases for profiling)")
+    ap.add_argument("--sources", type=int, default=None, help="reach: number of sources (fewer for a small profiling case)")
+    ap.add_argument("--no-tag-mirror", action="store_true", help="evaluate recursion by sort -> reduce-by-key -> merge only")
     ap.add_argument("--cpu-scale", type=int, default=None, help="R-MAT scale of the cpu_baseline sample (default: the workload's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

@@ -74,6 +74,8 @@ typedef struct {
 
 #define XLOG_FLAG_CHECK_INVARIANTS 1u  /* after every load/merge verify keys strictly increase (slow, for tests) */
 #define XLOG_FLAG_PROFILE          2u  /* CUDA events around every kernel launch; read with xlog_profile_read */
+#define XLOG_FLAG_NO_RESIDENT_LOOP 8u  /* the host drives every round of a tag-mirror fixpoint (one control read per round) */
+#define XLOG_FLAG_NO_GRAPH        16u  /* resident rounds are launched one by one instead of as one graph with a WHILE node */
 #define XLOG_FLAG_NO_TAG_MIRROR    4u  /* evaluate every recursive component by sort -> reduce-by-key -> merge, never through a tag mirror */
 
 /* ---- context --------------------------------------------------------------- */

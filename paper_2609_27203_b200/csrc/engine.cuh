@@ -9,6 +9,7 @@
 #include <cstring>
 #include <functional>
 #include <map>
+#include <memory>
 #include <set>
 #include <string>
 #include <vector>
@@ -36,7 +37,8 @@ struct Fail {
     if (e__ != cudaSuccess) fail(XLOG_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e__)); \
   } while (0)
 
-constexpr int kCtrlSlots = 64;          // uint64 control words mirrored to pinned host memory
+constexpr int kCtrlSlots = 96;          // uint64 control words mirrored to pinned host memory
+constexpr int kSlotResState = 64;       // the resident loop's state block (resident.cuh) lives in the control words from here on
 constexpr int kSlotErr = 0;
 
 struct Ctx;
@@ -120,9 +122,27 @@ struct RuleC {
   JoinShape shape[2];                   // indexed by the outer atom
 };
 
+// Everything the resident rounds of one head relation need, kept across fixpoint calls so that the instantiated
+// graph (which holds the buffers' addresses) can be launched again: the tag mirror, the delta and the join scratch
+// at their fixed capacities.
+struct Resident {
+  uint64_t slots = 0;
+  uint32_t max_tiles = 0;
+  DevBuf table, bitmap, ch_sums, dkeys, dtags, deg, rowinfo, start, sums, tile_rows;
+  cudaGraph_t graph = nullptr;
+  cudaGraphExec_t exec = nullptr;
+  std::vector<char> sig;                  // every kernel argument of the captured body, byte for byte
+  int64_t body_launches = 0;
+  ~Resident() {
+    if (exec) cudaGraphExecDestroy(exec);
+    if (graph) cudaGraphDestroy(graph);
+  }
+};
+
 struct Ctx {
   int device = 0;
   cudaStream_t stream = nullptr;
+  cudaStream_t capture_stream = nullptr;  // only ever records graph bodies
   Arena arena;
   int64_t max_iter = 1 << 20;
   size_t chunk_bytes = 0;
@@ -145,6 +165,7 @@ struct Ctx {
   std::vector<ProfPending> prof_pending;
   std::vector<cudaEvent_t> ev_pool;
   int64_t note_bytes = 0;                 // algorithmic bytes of the next launch (consumed by the launch macro)
+  std::map<int, std::unique_ptr<Resident>> resident;   // by head relation
   bool unique_untracked = false;          // a stratum went through the tag mirror, which does not count distinct candidate keys
   std::vector<char> stratum_done;         // per relation: its stratum has been evaluated in the running fixpoint
 };

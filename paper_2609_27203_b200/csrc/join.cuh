@@ -88,11 +88,8 @@ __device__ __forceinline__ bool bind_outer(const JoinSpec& S, KO key, int64_t* v
 // depends on the outer row alone (constants, outer variables, dictionary ranks, range checks) is done
 // here once per row instead of once per candidate.
 template <typename KO>
-__global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __restrict__ okeys, const float* __restrict__ otags,
-                                                    uint32_t n_outer, uint32_t* __restrict__ deg, uint4* __restrict__ rowinfo,
-                                                    uint32_t* __restrict__ err) {
-  const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n_outer) return;
+__device__ __forceinline__ void join_count_row(const JoinSpec& S, const KO* __restrict__ okeys, const float* __restrict__ otags, uint32_t i,
+                                               uint32_t* __restrict__ deg, uint4* __restrict__ rowinfo, uint32_t* __restrict__ err) {
   int64_t var[kMaxVars];
   uint32_t d = 0, lo = 0;
   uint64_t rowkey = 0;
@@ -148,6 +145,14 @@ __global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __rest
   }
   deg[i] = d;
   rowinfo[i] = make_uint4(lo, __float_as_uint(otags[i]), (uint32_t)rowkey, (uint32_t)(rowkey >> 32));
+}
+
+template <typename KO>
+__global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __restrict__ okeys, const float* __restrict__ otags,
+                                                    uint32_t n_outer, uint32_t* __restrict__ deg, uint4* __restrict__ rowinfo,
+                                                    uint32_t* __restrict__ err) {
+  const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n_outer) join_count_row<KO>(S, okeys, otags, i, deg, rowinfo, err);
 }
 
 constexpr int kExpBlock = 256;
@@ -226,24 +231,24 @@ static __global__ void __launch_bounds__(256) k_expand_partition(const uint64_t*
   tile_rows[t] = make_uint2(r[0], r[1]);
 }
 
-// Block b produces candidates [out_lo + b*kExpTile, ...).  `start` is the exclusive scan of `deg`
-// (global candidate index of each outer row's first match).  The outer rows covering the tile are
-// staged in shared memory (their starts relative to the tile and their row records), so the per-
-// candidate work is a short binary search in shared memory plus the coalesced inner reads.
-template <typename KO, typename KH, int MODE, int SINK = kSinkWrite>
-__global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
-                                                           const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo,
-                                                           const uint2* __restrict__ tile_rows, uint64_t out_lo, uint64_t out_hi,
-                                                           KH* __restrict__ ckeys,
-                                                           float* __restrict__ ctags, uint32_t* __restrict__ err, BwdArgs bw, MirrorArgs mr) {
-  __shared__ uint32_t sstart[kExpRows];
-  __shared__ uint4 sinfo[kExpRows];
-  __shared__ uint16_t srowidx[kExpTile];             // staged row of every candidate position of the tile
-  __shared__ uint32_t swarp[kExpBlock / 32];
-  const uint64_t t_lo = out_lo + (uint64_t)blockIdx.x * kExpTile;
-  const uint64_t t_hi = min(t_lo + kExpTile, out_hi);
-  if (t_lo >= t_hi) return;
-  const uint2 tr = tile_rows[blockIdx.x];
+struct ExpSmem {
+  uint32_t sstart[kExpRows];
+  uint4 sinfo[kExpRows];
+  uint16_t srowidx[kExpTile];             // staged row of every candidate position of the tile
+  uint32_t swarp[kExpBlock / 32];
+};
+
+// Candidates [t_lo, t_hi) (one tile, at most kExpTile of them), covered by outer rows tr.x .. tr.y.  Called by all
+// threads of a block; error bits go to `e` and new-tuple counts to `n_new` (the caller flushes both).
+template <typename KO, typename KH, int MODE, int SINK>
+__device__ __forceinline__ void expand_tile(ExpSmem& sm, const JoinSpec& S, const KO* __restrict__ okeys, uint32_t n_outer,
+                                            const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo, const uint2 tr,
+                                            const uint64_t t_lo, const uint64_t t_hi, const uint64_t out_lo, KH* __restrict__ ckeys,
+                                            float* __restrict__ ctags, const BwdArgs& bw, const MirrorArgs& mr, uint32_t& e, uint32_t& n_new) {
+  uint32_t* sstart = sm.sstart;
+  uint4* sinfo = sm.sinfo;
+  uint16_t* srowidx = sm.srowidx;
+  uint32_t* swarp = sm.swarp;
 #pragma unroll
   for (int i = 0; i < kExpItems; ++i) srowidx[i * kExpBlock + threadIdx.x] = 0;
   const uint32_t r_lo = tr.x, r_hi = tr.y;
@@ -296,7 +301,6 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
     const KH m0 = (KH)S.inner_mult[0];
     const int nin = S.has_inner ? S.inner_free : -1;                 // -1: one-atom rule
     const bool times = S.times != 0;
-    uint32_t n_new = 0;
     // three sweeps over the thread's items, so that the loads of one kind are all in flight together: (1) row record
     // from shared memory, inner tag and columns from global memory; (2) for the mirror, the current slot values;
     // (3) the stores, or the atomics of the few candidates that improve their slot
@@ -343,15 +347,9 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
         if (SINK == kSinkMin ? v < cur[k] : v > cur[k]) mirror_commit<SINK>(mr, (uint32_t)key[k], v, n_new);
       }
     }
-    if (SINK != kSinkWrite) {
-      n_new = __reduce_add_sync(0xffffffffu, n_new);
-      if (lane_id() == 0 && n_new) atomicAdd(mr.n_new, (unsigned long long)n_new);
-    }
     return;
   }
 
-  uint32_t e = 0;
-  uint32_t n_new = 0;
   for (uint32_t q = threadIdx.x; q < (uint32_t)(t_hi - t_lo); q += kExpBlock) {
     const uint64_t p = t_lo + q;
     uint32_t row, j;
@@ -433,8 +431,29 @@ __global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO*
       } else e |= kErrInternal;
     }
   }
+}
+
+// Block b produces candidates [out_lo + b*kExpTile, ...).  `start` is the exclusive scan of `deg`
+// (global candidate index of each outer row's first match).  The outer rows covering the tile are
+// staged in shared memory (their starts relative to the tile and their row records), so the per-
+// candidate work is a short binary search in shared memory plus the coalesced inner reads.
+template <typename KO, typename KH, int MODE, int SINK = kSinkWrite>
+__global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
+                                                           const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo,
+                                                           const uint2* __restrict__ tile_rows, uint64_t out_lo, uint64_t out_hi,
+                                                           KH* __restrict__ ckeys,
+                                                           float* __restrict__ ctags, uint32_t* __restrict__ err, BwdArgs bw, MirrorArgs mr) {
+  __shared__ ExpSmem sm;
+  const uint64_t t_lo = out_lo + (uint64_t)blockIdx.x * kExpTile;
+  const uint64_t t_hi = min(t_lo + kExpTile, out_hi);
+  if (t_lo >= t_hi) return;
+  uint32_t e = 0, n_new = 0;
+  expand_tile<KO, KH, MODE, SINK>(sm, S, okeys, n_outer, start, rowinfo, tile_rows[blockIdx.x], t_lo, t_hi, out_lo, ckeys, ctags, bw, mr, e, n_new);
   if (e) atomicOr(err, e);
-  if (SINK != kSinkWrite && n_new) atomicAdd(mr.n_new, (unsigned long long)n_new);
+  if (SINK != kSinkWrite) {
+    n_new = __reduce_add_sync(0xffffffffu, n_new);
+    if (lane_id() == 0 && n_new) atomicAdd(mr.n_new, (unsigned long long)n_new);
+  }
 }
 
 }  // namespace xlog

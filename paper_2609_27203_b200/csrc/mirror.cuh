@@ -43,8 +43,10 @@ static __global__ void __launch_bounds__(kMirBlock) k_mirror_changed_count(const
 template <typename K>
 __global__ void __launch_bounds__(kMirBlock) k_mirror_changed_emit(uint4* __restrict__ bitmap, uint32_t nquads,
                                                                    const uint32_t* __restrict__ tile_base, const int32_t* __restrict__ table,
-                                                                   K* __restrict__ keys, float* __restrict__ tags) {
+                                                                   K* __restrict__ keys, float* __restrict__ tags,
+                                                                   const uint32_t* __restrict__ skip_if_nonzero) {
   __shared__ uint32_t sh[kMirBlock / 32 + 1];
+  if (skip_if_nonzero && *skip_if_nonzero) return;       // the round was abandoned: keep the bitmap and the old delta
   const uint32_t q = blockIdx.x * kMirBlock + threadIdx.x;
   uint4 w = make_uint4(0, 0, 0, 0);
   if (q < nquads) w = bitmap[q];

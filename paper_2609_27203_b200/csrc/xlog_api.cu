@@ -1,6 +1,7 @@
 // C ABI of the engine (see include/xlog.h) and the host-side fixpoint driver.
 #include "engine.cuh"
 #include "mirror.cuh"
+#include "resident.cuh"
 #include "triangle.cuh"
 
 using namespace xlog;
@@ -359,7 +360,8 @@ struct Counted {                         // a variant after count + scan
 
 JoinSpec make_spec(Ctx* c, const Variant& v, const Relation& H) {
   const xlog_plan& p = v.rule->plan;
-  JoinSpec S{};
+  JoinSpec S;
+  memset(&S, 0, sizeof S);                 // padding included: specs are compared byte for byte (graph reuse)
   S.outer = v.outer.layout;
   const xlog_atom& A = p.atoms[v.outer_atom];
   for (int i = 0; i < c->rels[A.rel]->arity; ++i) S.outer_args[i] = ArgSpec{A.args[i].kind, A.args[i].var, A.args[i].mul, A.args[i].add};
@@ -985,32 +987,180 @@ bool mirror_applies(Ctx* c, const std::vector<int>& comp, const std::vector<cons
   return need <= c->arena.largest_free() / 2;
 }
 
+// ---- resident rounds (resident.cuh) --------------------------------------------------------------------
+constexpr int kResidentMaxBits = 24;
+constexpr uint32_t kResidentMaxTiles = 1u << 20;
+
+ResState* res_state(Ctx* c) { return reinterpret_cast<ResState*>(c->d_ctrl + kSlotResState); }
+static_assert(sizeof(ResState) <= (kCtrlSlots - kSlotResState) * sizeof(uint64_t), "state block must fit the control words");
+
+// The persistent buffers of head relation h at their fixed capacities, or nullptr when the resident rounds do not
+// apply (domain too large for fixed-capacity buffers, not enough arena, or switched off).
+Resident* resident_for(Ctx* c, int h, int bits, uint64_t slots, uint32_t bm_quads, unsigned ch_tiles) {
+  if ((c->flags & XLOG_FLAG_NO_RESIDENT_LOOP) || bits > kResidentMaxBits) { c->resident.erase(h); return nullptr; }
+  uint32_t max_tiles = kResidentMaxTiles;
+  if (c->chunk_bytes) max_tiles = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(max_tiles, c->chunk_bytes / 16 / kExpTile));
+  auto it = c->resident.find(h);
+  if (it != c->resident.end() && it->second->slots == slots && it->second->max_tiles == max_tiles) return it->second.get();
+  c->resident.erase(h);
+  const uint64_t dom = (uint64_t)1 << bits;
+  const uint64_t need = slots * 4 + (uint64_t)bm_quads * 16 + dom * 36 + (uint64_t)max_tiles * 8 + (2u << 20);
+  if (need > c->arena.largest_free() / 3) return nullptr;
+  std::unique_ptr<Resident> R(new Resident());
+  R->slots = slots; R->max_tiles = max_tiles;
+  R->table = DevBuf(c, slots * 4);
+  R->bitmap = DevBuf(c, (size_t)bm_quads * 16);
+  R->ch_sums = DevBuf(c, (size_t)ch_tiles * 4);
+  R->dkeys = DevBuf(c, dom * 4); R->dtags = DevBuf(c, dom * 4);
+  R->deg = DevBuf(c, dom * 4); R->rowinfo = DevBuf(c, dom * 16); R->start = DevBuf(c, dom * 8);
+  R->sums = DevBuf(c, (dom / kScanTile + 1) * 8);
+  R->tile_rows = DevBuf(c, (size_t)max_tiles * 8);
+  Resident* out = R.get();
+  c->resident[h] = std::move(R);
+  return out;
+}
+
+template <typename T> void sig_add(std::vector<char>& sig, const T& v) {
+  const char* p = reinterpret_cast<const char*>(&v);
+  sig.insert(sig.end(), p, p + sizeof(T));
+}
+
+// One round's launches.  Nothing here allocates, copies or waits: the same calls are either captured into the WHILE
+// body or issued directly (host-driven rounds, used when launches are being timed one by one).
+void resident_body(Ctx* c, Resident& R, const std::vector<JoinSpec>& specs, bool is_max, const MirrorArgs& mr, uint32_t bm_quads, unsigned ch_tiles,
+                   cudaGraphConditionalHandle handle, int use_handle) {
+  ResState* st = res_state(c);
+  uint32_t* err = ctrl_u32(c, kSlotErr);
+  const uint32_t* dk = R.dkeys.as<uint32_t>();
+  for (const JoinSpec& S : specs) {
+    XLOG_LAUNCH(c, (k_res_count<uint32_t>), kSMs * 8, 256, 0, S, dk, (const float*)R.dtags.as<float>(), (const ResState*)st, R.deg.as<uint32_t>(),
+                R.rowinfo.as<uint4>(), err);
+    XLOG_LAUNCH(c, k_res_tile_sums, kSMs * 2, kScanBlock, 0, (const uint32_t*)R.deg.as<uint32_t>(), (const ResState*)st, R.sums.as<uint64_t>());
+    XLOG_LAUNCH(c, k_res_spine, 1, 1024, 0, R.sums.as<uint64_t>(), st);
+    XLOG_LAUNCH(c, k_res_apply, kSMs * 2, kScanBlock, 0, (const uint32_t*)R.deg.as<uint32_t>(), (const ResState*)st, (const uint64_t*)R.sums.as<uint64_t>(),
+                R.start.as<uint64_t>());
+    XLOG_LAUNCH(c, k_res_partition, kSMs, 256, 0, (const uint64_t*)R.start.as<uint64_t>(), (const ResState*)st, R.tile_rows.as<uint2>());
+#define XLOG_RES_EXPAND(MODE, SINK)                                                                                                         \
+  XLOG_LAUNCH(c, (k_res_expand<uint32_t, MODE, SINK>), kSMs * 4, kExpBlock, 0, S, dk, (const ResState*)st, (const uint64_t*)R.start.as<uint64_t>(), \
+              (const uint4*)R.rowinfo.as<uint4>(), (const uint2*)R.tile_rows.as<uint2>(), err, mr)
+    if (S.fast) { if (is_max) XLOG_RES_EXPAND(kExpFast, kSinkMax); else XLOG_RES_EXPAND(kExpFast, kSinkMin); }
+    else { if (is_max) XLOG_RES_EXPAND(kExpGeneric, kSinkMax); else XLOG_RES_EXPAND(kExpGeneric, kSinkMin); }
+#undef XLOG_RES_EXPAND
+  }
+  XLOG_LAUNCH(c, k_mirror_changed_count, ch_tiles, kMirBlock, 0, (const uint4*)R.bitmap.as<uint4>(), bm_quads, R.ch_sums.as<uint32_t>());
+  XLOG_LAUNCH(c, k_res_round_end, 1, 1024, 0, R.ch_sums.as<uint32_t>(), (uint32_t)ch_tiles, st, (const unsigned long long*)mr.n_new, handle, use_handle);
+  XLOG_LAUNCH(c, (k_mirror_changed_emit<uint32_t>), ch_tiles, kMirBlock, 0, R.bitmap.as<uint4>(), bm_quads, (const uint32_t*)R.ch_sums.as<uint32_t>(),
+              (const int32_t*)R.table.as<int32_t>(), R.dkeys.as<uint32_t>(), R.dtags.as<float>(), (const uint32_t*)&st->status);
+}
+
+// Run rounds on the device until the delta is empty, the round budget is used up or a round needs more tiles than
+// planned.  Returns the final state block (read once, after the loop).
+ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*>& rs, bool is_max, const MirrorArgs& mr, uint32_t bm_quads,
+                      unsigned ch_tiles, uint32_t n_delta, int64_t rounds_left, uint64_t new_seen) {
+  Relation& H = *c->rels[h];
+  std::vector<JoinSpec> specs;
+  for (const RuleC* r : rs)
+    for (int j = 0; j < r->plan.n_atoms; ++j)
+      if (r->plan.atoms[j].rel == h) {
+        const Variant v{r, j, Source{R.dkeys.p, R.dtags.as<float>(), n_delta, H.layout, H.key_bytes}};
+        specs.push_back(make_spec(c, v, H));              // builds the looked-up relation's index if it is missing
+      }
+  if (specs.size() > 16) fail(XLOG_ERR_UNSUPPORTED, "too many rule variants for one head");
+  const uint32_t budget = (uint32_t)std::min<int64_t>(rounds_left, 0x7fffffff);
+  XLOG_LAUNCH(c, k_res_init, 1, 32, 0, res_state(c), n_delta, budget, R.max_tiles, (unsigned long long)new_seen);
+  const int64_t l0 = c->launches;
+  const bool use_graph = !(c->flags & (XLOG_FLAG_PROFILE | XLOG_FLAG_NO_GRAPH));
+  ResState out{};
+  auto read_state = [&]() {
+    sync_ctrl(c);
+    memcpy(&out, c->h_ctrl + kSlotResState, sizeof out);
+  };
+  if (use_graph) {
+    std::vector<char> sig;
+    for (const JoinSpec& S : specs) sig_add(sig, S);
+    sig_add(sig, mr.table); sig_add(sig, mr.changed); sig_add(sig, mr.n_new); sig_add(sig, mr.key_max); sig_add(sig, mr.err);
+    sig_add(sig, is_max); sig_add(sig, bm_quads); sig_add(sig, ch_tiles); sig_add(sig, c->d_ctrl);
+    if (!R.exec || sig != R.sig) {
+      if (R.exec) { cudaGraphExecDestroy(R.exec); R.exec = nullptr; }
+      if (R.graph) { cudaGraphDestroy(R.graph); R.graph = nullptr; }
+      XLOG_CUDA(cudaGraphCreate(&R.graph, 0));
+      cudaGraphConditionalHandle handle;
+      XLOG_CUDA(cudaGraphConditionalHandleCreate(&handle, R.graph, 1, cudaGraphCondAssignDefault));
+      cudaGraphNodeParams np = {};
+      np.type = cudaGraphNodeTypeConditional;
+      np.conditional.handle = handle;
+      np.conditional.type = cudaGraphCondTypeWhile;
+      np.conditional.size = 1;
+      cudaGraphNode_t node;
+      XLOG_CUDA(cudaGraphAddNode(&node, R.graph, nullptr, 0, &np));
+      cudaGraph_t body = np.conditional.phGraph_out[0];
+      // the body is recorded on a stream of the context's own (the caller's stream may be the legacy default stream,
+      // which cannot capture); the instantiated graph is launched on the caller's stream like everything else
+      if (!c->capture_stream) XLOG_CUDA(cudaStreamCreateWithFlags(&c->capture_stream, cudaStreamNonBlocking));
+      XLOG_CUDA(cudaStreamBeginCaptureToGraph(c->capture_stream, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal));
+      cudaStream_t caller = c->stream;
+      c->stream = c->capture_stream;
+      const int64_t b0 = c->launches;
+      try {
+        resident_body(c, R, specs, is_max, mr, bm_quads, ch_tiles, handle, 1);
+      } catch (...) {
+        c->stream = caller;
+        cudaGraph_t dummy = nullptr;
+        cudaStreamEndCapture(c->capture_stream, &dummy);
+        throw;
+      }
+      c->stream = caller;
+      R.body_launches = c->launches - b0;
+      XLOG_CUDA(cudaStreamEndCapture(c->capture_stream, nullptr));
+      XLOG_CUDA(cudaGraphInstantiate(&R.exec, R.graph, 0));
+      R.sig = std::move(sig);
+    }
+    XLOG_CUDA(cudaGraphLaunch(R.exec, c->stream));
+    read_state();
+    c->launches = l0 + R.body_launches * (int64_t)out.rounds + (out.status == kResOverflow ? R.body_launches : 0);
+  } else {
+    for (;;) {
+      resident_body(c, R, specs, is_max, mr, bm_quads, ch_tiles, cudaGraphConditionalHandle{}, 0);
+      read_state();
+      if (out.status != kResOk || out.n_delta == 0) break;
+    }
+  }
+  return out;
+}
+
 // Algorithm 1 over a tag mirror (mirror.cuh): per round  count -> scan -> join straight into the table -> compact the
-// changed bitmap into the next delta.  No candidate is ever written to memory.
+// changed bitmap into the next delta.  No candidate is ever written to memory.  The seed round is driven by the host
+// (its rules scan whole relations of known size); the delta rounds run resident where the fixed-capacity buffers fit.
 void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs) {
   Relation& H = *c->rels[h];
   const std::vector<int> comp{h};
-  const uint64_t dom = (uint64_t)1 << H.layout.total_bits;
+  const int bits = H.layout.total_bits;
+  const uint64_t dom = (uint64_t)1 << bits;
   const bool is_max = H.sr == XLOG_SR_MAXPLUS;
   const int32_t empty = is_max ? kMirrorEmptyMax : kMirrorEmptyMin;
   const uint64_t slots = std::max<uint64_t>(dom, 4);
   const uint32_t bm_quads = (uint32_t)((std::max<uint64_t>(dom / 32, 1) + 3) / 4);
-  DevBuf table(c, slots * 4), bitmap(c, (size_t)bm_quads * 16);
-  XLOG_LAUNCH(c, k_fill_i32, grid_for(slots, 256 * 8), 256, 0, table.as<int32_t>(), slots, empty);
-  XLOG_CUDA(cudaMemsetAsync(bitmap.p, 0, (size_t)bm_quads * 16, c->stream));
+  const unsigned ch_tiles = (bm_quads + kMirBlock - 1) / kMirBlock;
+  Resident* R = resident_for(c, h, bits, slots, bm_quads, ch_tiles);
+  DevBuf table_own, bitmap_own, ch_sums_own;
+  if (!R) { table_own = DevBuf(c, slots * 4); bitmap_own = DevBuf(c, (size_t)bm_quads * 16); ch_sums_own = DevBuf(c, (size_t)ch_tiles * 4); }
+  int32_t* table = R ? R->table.as<int32_t>() : table_own.as<int32_t>();
+  uint4* bitmap = R ? R->bitmap.as<uint4>() : bitmap_own.as<uint4>();
+  uint32_t* ch_sums = R ? R->ch_sums.as<uint32_t>() : ch_sums_own.as<uint32_t>();
+  XLOG_LAUNCH(c, k_fill_i32, grid_for(slots, 256 * 8), 256, 0, table, slots, empty);
+  XLOG_CUDA(cudaMemsetAsync(bitmap, 0, (size_t)bm_quads * 16, c->stream));
   // what the relation holds now (its loaded facts, or the result of an earlier fixpoint) is the starting state
   const uint32_t n_start = H.n;
   if (n_start)
-    XLOG_LAUNCH(c, (k_mirror_scatter<uint32_t>), grid_for(n_start, 256, 1 << 30), 256, 0, (const uint32_t*)H.keys(), (const float*)H.tags(), n_start,
-                table.as<int32_t>());
+    XLOG_LAUNCH(c, (k_mirror_scatter<uint32_t>), grid_for(n_start, 256, 1 << 30), 256, 0, (const uint32_t*)H.keys(), (const float*)H.tags(), n_start, table);
   zero_ctrl(c, kSlotMirNew, 2);
-  const MirrorArgs mr{table.as<int32_t>(), bitmap.as<uint32_t>(), (unsigned long long*)(c->d_ctrl + kSlotMirNew), (uint32_t)(dom - 1),
+  const MirrorArgs mr{table, reinterpret_cast<uint32_t*>(bitmap), (unsigned long long*)(c->d_ctrl + kSlotMirNew), (uint32_t)(dom - 1),
                       ctrl_u32(c, kSlotErr)};
-  const unsigned ch_tiles = (bm_quads + kMirBlock - 1) / kMirBlock;
-  DevBuf ch_sums(c, (size_t)ch_tiles * 4);
   c->unique_untracked = true;
-  KeyTags delta;
+  KeyTags delta_own;                       // host-driven rounds without persistent buffers keep their delta here
+  const void* dk = nullptr; const float* dt = nullptr; uint32_t dn = 0;
   uint64_t total_new = 0;
+  bool resident_done = false;
   for (int64_t round = 0;; ++round) {
     if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
     ++c->r_iterations;
@@ -1021,7 +1171,7 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
         vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
       } else {
         for (int j = 0; j < r->plan.n_atoms; ++j)
-          if (r->plan.atoms[j].rel == h && delta.n) vs.push_back(Variant{r, j, Source{delta.keys.p, delta.tags.as<float>(), delta.n, H.layout, H.key_bytes}});
+          if (r->plan.atoms[j].rel == h && dn) vs.push_back(Variant{r, j, Source{dk, dt, dn, H.layout, H.key_bytes}});
       }
     }
     if (vs.size() > 16) fail(XLOG_ERR_UNSUPPORTED, "too many rule variants for one head");
@@ -1046,22 +1196,39 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
       }
       q.start.reset(); q.rowinfo.reset();
     }
-    delta = KeyTags();
     if (total == 0) break;
-    XLOG_LAUNCH(c, k_mirror_changed_count, ch_tiles, kMirBlock, 0, (const uint4*)bitmap.as<uint4>(), bm_quads, ch_sums.as<uint32_t>());
-    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, ch_sums.as<uint32_t>(), (int64_t)ch_tiles, ctrl_u32(c, kSlotMirChanged));
+    XLOG_LAUNCH(c, k_mirror_changed_count, ch_tiles, kMirBlock, 0, (const uint4*)bitmap, bm_quads, ch_sums);
+    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, ch_sums, (int64_t)ch_tiles, ctrl_u32(c, kSlotMirChanged));
     sync_ctrl(c);
     const uint32_t changed = (uint32_t)c->h_ctrl[kSlotMirChanged];
     const uint64_t n_new = c->h_ctrl[kSlotMirNew] - total_new;
     total_new += n_new;
     c->r_new += (int64_t)n_new; c->r_improved += (int64_t)changed - (int64_t)n_new;
     if (changed == 0) break;
-    delta.n = changed;
-    delta.keys = DevBuf(c, (size_t)changed * 4);
-    delta.tags = DevBuf(c, (size_t)changed * 4);
+    uint32_t* ek; float* et;
+    if (R) { ek = R->dkeys.as<uint32_t>(); et = R->dtags.as<float>(); }
+    else {
+      delta_own = KeyTags();
+      delta_own.keys = DevBuf(c, (size_t)changed * 4);
+      delta_own.tags = DevBuf(c, (size_t)changed * 4);
+      ek = delta_own.keys.as<uint32_t>(); et = delta_own.tags.as<float>();
+    }
     c->note_bytes = (int64_t)bm_quads * 16 + (int64_t)changed * 12;
-    XLOG_LAUNCH(c, (k_mirror_changed_emit<uint32_t>), ch_tiles, kMirBlock, 0, bitmap.as<uint4>(), bm_quads, (const uint32_t*)ch_sums.as<uint32_t>(),
-                (const int32_t*)table.as<int32_t>(), delta.keys.as<uint32_t>(), delta.tags.as<float>());
+    XLOG_LAUNCH(c, (k_mirror_changed_emit<uint32_t>), ch_tiles, kMirBlock, 0, bitmap, bm_quads, (const uint32_t*)ch_sums, (const int32_t*)table, ek, et,
+                (const uint32_t*)nullptr);
+    dk = ek; dt = et; dn = changed;
+    if (R && !resident_done) {
+      // hand the delta rounds to the device
+      const ResState s = run_resident(c, *R, h, rs, is_max, mr, bm_quads, ch_tiles, dn, c->max_iter - (round + 1), total_new);
+      resident_done = true;                  // after an overflow the host finishes the job
+      round += s.rounds;
+      c->r_iterations += s.rounds; c->r_candidates += (int64_t)s.candidates;
+      c->r_new += (int64_t)s.n_new; c->r_improved += (int64_t)s.n_improved;
+      total_new = s.new_seen;
+      dn = s.n_delta;
+      if (s.status == kResCap) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
+      if (s.status == kResOk) break;         // the delta ran empty
+    }
   }
   // the relation in sorted form: every occupied slot, in slot order
   const uint64_t n_out = (uint64_t)n_start + total_new;
@@ -1074,10 +1241,10 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
     const unsigned tiles = (unsigned)((slots + kMirSlotsPerTile - 1) / kMirSlotsPerTile);
     DevBuf sums(c, (size_t)tiles * 4);
     c->note_bytes = (int64_t)slots * 4;
-    XLOG_LAUNCH(c, k_mirror_full_count, tiles, kMirBlock, 0, (const int4*)table.as<int4>(), nquads, empty, sums.as<uint32_t>());
+    XLOG_LAUNCH(c, k_mirror_full_count, tiles, kMirBlock, 0, (const int4*)table, nquads, empty, sums.as<uint32_t>());
     XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, sums.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotA));
     c->note_bytes = (int64_t)slots * 4 + (int64_t)n_out * 8;
-    XLOG_LAUNCH(c, (k_mirror_full_emit<uint32_t>), tiles, kMirBlock, 0, (const int4*)table.as<int4>(), nquads, empty, (const uint32_t*)sums.as<uint32_t>(),
+    XLOG_LAUNCH(c, (k_mirror_full_emit<uint32_t>), tiles, kMirBlock, 0, (const int4*)table, nquads, empty, (const uint32_t*)sums.as<uint32_t>(),
                 full.keys.as<uint32_t>(), full.tags.as<float>());
   }
   set_current(H, std::move(full));
@@ -1235,6 +1402,8 @@ xlog_status xlog_ctx_destroy(xlog_ctx* c) {
   if (c->h_ctrl) cudaFreeHost(c->h_ctrl);
   if (c->ev0) cudaEventDestroy(c->ev0);
   if (c->ev1) cudaEventDestroy(c->ev1);
+  c->resident.clear();
+  if (c->capture_stream) cudaStreamDestroy(c->capture_stream);
   for (auto& p : c->prof_pending) { cudaEventDestroy(p.a); cudaEventDestroy(p.b); }
   for (cudaEvent_t e : c->ev_pool) cudaEventDestroy(e);
   delete c;

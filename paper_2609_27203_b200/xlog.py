@@ -22,6 +22,8 @@ MEM_HOST, MEM_DEVICE = 0, 1
 FLAG_CHECK_INVARIANTS = 1
 FLAG_PROFILE = 2
 FLAG_NO_TAG_MIRROR = 4
+FLAG_NO_RESIDENT_LOOP = 8
+FLAG_NO_GRAPH = 16
 
 EXPORTS = ["xlog_ctx_create", "xlog_ctx_destroy", "xlog_last_error", "xlog_relation_create", "xlog_relation_load",
            "xlog_relation_size", "xlog_relation_read", "xlog_relation_view", "xlog_rule_add", "xlog_fixpoint",

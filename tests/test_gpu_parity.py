@@ -38,7 +38,9 @@ def check_program(program, rel_tol=MINMAX_REL, abs_tol=0.0, expect_bit_equal=Tru
     from paper_2609_27203_b200 import xlog
     o, oids, _, stats = oracle_run(program, mode)
     receipts, results = [], []
-    for extra in (0, xlog.FLAG_NO_TAG_MIRROR):
+    # default (tag mirror, delta rounds resident in one graph) / the same rounds launched one by one / host-driven
+    # mirror rounds / the sorting path
+    for extra in (0, xlog.FLAG_NO_GRAPH, xlog.FLAG_NO_RESIDENT_LOOP, xlog.FLAG_NO_TAG_MIRROR):
         ctx, gids, _, receipt = gpu_run(program, **dict(kw, flags=kw.get("flags", xlog.FLAG_CHECK_INVARIANTS) | extra))
         got = {}
         for name in program.outputs:
@@ -50,11 +52,12 @@ def check_program(program, rel_tol=MINMAX_REL, abs_tol=0.0, expect_bit_equal=Tru
         assert receipt["derived_tuples"] == stats["derived_tuples"]
         ctx.close()
         receipts.append(receipt); results.append(got)
-    for name in program.outputs:
-        assert H.compare_relations(results[0][name], results[1][name], what="mirror vs sorted path")["bit_unequal"] == 0
-    for k in ("iterations", "candidates", "new_tuples", "improved_tags", "derived_tuples", "strata"):
-        assert receipts[0][k] == receipts[1][k], (k, receipts[0][k], receipts[1][k])
-    assert receipts[1]["unique_candidates"] >= 0
+    for i in range(1, len(results)):
+        for name in program.outputs:
+            assert H.compare_relations(results[0][name], results[i][name], what=f"path 0 vs path {i}")["bit_unequal"] == 0
+        for k in ("iterations", "candidates", "new_tuples", "improved_tags", "derived_tuples", "strata"):
+            assert receipts[0][k] == receipts[i][k], (i, k, receipts[0][k], receipts[i][k])
+    assert receipts[-1]["unique_candidates"] >= 0
     return receipts[0], stats
 
 
