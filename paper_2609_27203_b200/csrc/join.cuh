@@ -88,8 +88,8 @@ __device__ __forceinline__ bool bind_outer(const JoinSpec& S, KO key, int64_t* v
 // depends on the outer row alone (constants, outer variables, dictionary ranks, range checks) is done
 // here once per row instead of once per candidate.
 template <typename KO>
-__device__ __forceinline__ void join_count_row(const JoinSpec& S, const KO* __restrict__ okeys, const float* __restrict__ otags, uint32_t i,
-                                               uint32_t* __restrict__ deg, uint4* __restrict__ rowinfo, uint32_t* __restrict__ err) {
+__device__ __forceinline__ uint32_t join_count_row(const JoinSpec& S, const KO* __restrict__ okeys, const float* __restrict__ otags, uint32_t i,
+                                                   uint4* __restrict__ rowinfo, uint32_t* __restrict__ err) {
   int64_t var[kMaxVars];
   uint32_t d = 0, lo = 0;
   uint64_t rowkey = 0;
@@ -143,8 +143,8 @@ __device__ __forceinline__ void join_count_row(const JoinSpec& S, const KO* __re
       if (e) atomicOr(err, e);
     }
   }
-  deg[i] = d;
   rowinfo[i] = make_uint4(lo, __float_as_uint(otags[i]), (uint32_t)rowkey, (uint32_t)(rowkey >> 32));
+  return d;
 }
 
 template <typename KO>
@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __rest
                                                     uint32_t n_outer, uint32_t* __restrict__ deg, uint4* __restrict__ rowinfo,
                                                     uint32_t* __restrict__ err) {
   const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n_outer) join_count_row<KO>(S, okeys, otags, i, deg, rowinfo, err);
+  if (i < n_outer) deg[i] = join_count_row<KO>(S, okeys, otags, i, rowinfo, err);
 }
 
 constexpr int kExpBlock = 256;

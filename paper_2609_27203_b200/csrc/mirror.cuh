@@ -8,7 +8,7 @@
 // relation is bit-identical to the one the sorting path derives.
 //
 //   k_mirror_scatter        loaded facts -> table
-//   k_mirror_changed_count  set bits per 32768-key tile of the changed bitmap
+//   k_mirror_changed_count  set bits per tile of the changed bitmap
 //   k_mirror_changed_emit   bitmap -> delta (keys ascending, tags read from the table); clears the bitmap
 //   k_mirror_full_count     occupied slots per 4096-slot tile
 //   k_mirror_full_emit      table -> relation
@@ -18,7 +18,6 @@
 namespace xlog {
 
 constexpr int kMirBlock = 256;
-constexpr int kMirWordsPerTile = kMirBlock * 4;        // bitmap words per tile (one uint4 per thread)
 constexpr int kMirSlotsPerTile = kMirBlock * 16;       // table slots per tile (four int4 per thread)
 
 template <typename K>
@@ -28,47 +27,58 @@ __global__ void __launch_bounds__(256) k_mirror_scatter(const K* __restrict__ ke
   if (i < n) table[keys[i]] = f2ord(tags[i]);
 }
 
-// nquads = number of uint4 groups of the bitmap (its length is padded to a multiple of four words)
-static __global__ void __launch_bounds__(kMirBlock) k_mirror_changed_count(const uint4* __restrict__ bitmap, uint32_t nquads,
-                                                                           uint32_t* __restrict__ tile_sums) {
+// The changed bitmap is handled in tiles of SW * 256 words (SW "sweeps" of one word per thread).  Small domains take
+// SW = 1 so that there are enough tiles to occupy the GPU; large ones SW = 4 to keep the list of tile counts short.
+// nwords is the bitmap's (padded) length.
+template <int SW>
+__global__ void __launch_bounds__(kMirBlock) k_mirror_changed_count(const uint32_t* __restrict__ words, uint32_t nwords,
+                                                                    uint32_t* __restrict__ tile_sums) {
   __shared__ uint32_t sh[kMirBlock / 32 + 1];
-  const uint32_t q = blockIdx.x * kMirBlock + threadIdx.x;
   uint32_t s = 0;
-  if (q < nquads) { const uint4 w = bitmap[q]; s = __popc(w.x) + __popc(w.y) + __popc(w.z) + __popc(w.w); }
+#pragma unroll
+  for (int j = 0; j < SW; ++j) {
+    const uint32_t wi = (blockIdx.x * SW + j) * kMirBlock + threadIdx.x;
+    if (wi < nwords) s += __popc(words[wi]);
+  }
   uint32_t total;
   block_scan_excl<kMirBlock, uint32_t>(s, sh, total);
   if (threadIdx.x == 0) tile_sums[blockIdx.x] = total;
 }
 
-template <typename K>
-__global__ void __launch_bounds__(kMirBlock) k_mirror_changed_emit(uint4* __restrict__ bitmap, uint32_t nquads,
+// One block per tile.  In a sweep every thread expands the set bits of one word into a key list in shared memory
+// (at most 8192 keys); then the whole block turns the list into output rows, so the table reads are independent of
+// one another and the writes are coalesced however unevenly the bits are spread.
+template <typename K, int SW>
+__global__ void __launch_bounds__(kMirBlock) k_mirror_changed_emit(uint32_t* __restrict__ words, uint32_t nwords,
                                                                    const uint32_t* __restrict__ tile_base, const int32_t* __restrict__ table,
                                                                    K* __restrict__ keys, float* __restrict__ tags,
                                                                    const uint32_t* __restrict__ skip_if_nonzero) {
   __shared__ uint32_t sh[kMirBlock / 32 + 1];
+  __shared__ uint32_t list[kMirBlock * 32];
   if (skip_if_nonzero && *skip_if_nonzero) return;       // the round was abandoned: keep the bitmap and the old delta
-  const uint32_t q = blockIdx.x * kMirBlock + threadIdx.x;
-  uint4 w = make_uint4(0, 0, 0, 0);
-  if (q < nquads) w = bitmap[q];
-  const uint32_t s = __popc(w.x) + __popc(w.y) + __popc(w.z) + __popc(w.w);
-  uint32_t total;
-  uint32_t pos = tile_base[blockIdx.x] + block_scan_excl<kMirBlock, uint32_t>(s, sh, total);
-  if (s == 0) return;
-  uint32_t word[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    uint32_t bits = word[j];
-    const uint32_t base = (q * 4 + j) << 5;
+  uint32_t out = tile_base[blockIdx.x];
+#pragma unroll 1
+  for (int j = 0; j < SW; ++j) {
+    const uint32_t wi = (blockIdx.x * SW + j) * kMirBlock + threadIdx.x;
+    uint32_t bits = wi < nwords ? words[wi] : 0u;
+    uint32_t total;
+    uint32_t pos = block_scan_excl<kMirBlock, uint32_t>((uint32_t)__popc(bits), sh, total);
+    if (total == 0) continue;                            // uniform across the block
+    if (bits) words[wi] = 0u;
     while (bits) {
       const int b = __ffs(bits) - 1;
       bits &= bits - 1;
-      const uint32_t key = base + b;
-      keys[pos] = (K)key;
-      tags[pos] = ord2f(__ldcg(table + key));
-      ++pos;
+      list[pos++] = (wi << 5) + b;
     }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < total; i += kMirBlock) {
+      const uint32_t key = list[i];
+      keys[out + i] = (K)key;
+      tags[out + i] = ord2f(__ldcg(table + key));
+    }
+    out += total;
+    __syncthreads();
   }
-  bitmap[q] = make_uint4(0, 0, 0, 0);
 }
 
 // Slots are read in a striped arrangement (coalesced int4 loads); the output order is the slot order, so the four

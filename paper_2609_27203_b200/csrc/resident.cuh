@@ -3,8 +3,7 @@
 // host reads inside the loop).  One round over a tag mirror (mirror.cuh) is a fixed sequence of
 // launches whose sizes are read from a small state block in device memory:
 //
-//   per rule with a recursive atom:  k_res_count -> k_res_tile_sums -> k_res_spine -> k_res_apply
-//                                    -> k_res_partition -> k_res_expand
+//   per rule with a recursive atom:  k_res_count_scan -> k_res_expand
 //   then:                            k_mirror_changed_count -> k_res_round_end -> k_mirror_changed_emit
 //
 // Every kernel has a fixed grid and strides over however much work the state block announces, so the
@@ -19,7 +18,7 @@
 
 namespace xlog {
 
-enum { kResOk = 0, kResCap = 1, kResOverflow = 2 };
+enum { kResOk = 0, kResCap = 1, kResOverflow = 2, kResError = 3 };
 
 struct ResState {
   uint32_t n_delta;                  // rows of the current delta
@@ -36,103 +35,125 @@ struct ResState {
   unsigned long long n_improved;
 };
 
-static __global__ void k_res_init(ResState* st, uint32_t n_delta, uint32_t max_rounds, uint32_t max_tiles, unsigned long long new_seen) {
-  if (threadIdx.x == 0 && blockIdx.x == 0) {
+constexpr int kResMaxVariants = 16;
+constexpr int kResScanItems = 4;                       // rows per thread in the fused count + scan: short dependent chains
+constexpr int kResScanTile = kScanBlock * kResScanItems;
+constexpr uint64_t kScanFlagAgg = 1ull << 62, kScanFlagIncl = 2ull << 62, kScanValMask = (1ull << 62) - 1;
+constexpr uint32_t kResSpinLimit = 1u << 22;          // polls of one status word before giving up
+
+__device__ __forceinline__ unsigned long long ld_volatile_u64(const unsigned long long* p) { return *reinterpret_cast<const volatile unsigned long long*>(p); }
+__device__ __forceinline__ void st_volatile_u64(unsigned long long* p, unsigned long long v) { *reinterpret_cast<volatile unsigned long long*>(p) = v; }
+
+// Scratch that must be zero when a round starts: scan status words and tile tickets of every rule.
+struct ResScratch {
+  unsigned long long* scan_status;   // [kResMaxVariants][scan_tiles_cap]
+  uint32_t scan_tiles_cap;
+  uint32_t* tickets;                 // [kResMaxVariants]
+};
+
+static __global__ void __launch_bounds__(1024) k_res_init(ResState* st, ResScratch sc, uint32_t n_variants, uint32_t n_delta, uint32_t max_rounds,
+                                                          uint32_t max_tiles, unsigned long long new_seen) {
+  if (threadIdx.x == 0) {
     ResState s{};
     s.n_delta = n_delta; s.max_rounds = max_rounds; s.max_tiles = max_tiles; s.new_seen = new_seen;
     *st = s;
   }
+  // everything, not just what the first round will touch: an abandoned loop leaves its last round's words behind
+  for (size_t i = threadIdx.x; i < (size_t)n_variants * sc.scan_tiles_cap; i += blockDim.x) sc.scan_status[i] = 0;
+  for (uint32_t i = threadIdx.x; i < kResMaxVariants; i += blockDim.x) sc.tickets[i] = 0;
 }
 
+// Count, scan and partition of one rule in a single launch.  Blocks draw 1024-row tiles from a ticket counter (so a tile
+// only ever waits for tiles that running blocks already own).  For its tile a block computes every row's degree and
+// row record, reduces the degrees, resolves its exclusive prefix by looking back through the status words of the tiles
+// before it (aggregate first, inclusive prefix once known: a chained scan), writes the rows' start offsets, and - since
+// a row knows which candidate positions it covers - the first / last row of every expand tile whose boundary it covers.
+// The last tile publishes the candidate total and the expand tile count.  Waits are bounded: a status word that stays
+// empty for kResSpinLimit polls raises the internal-error flag and stops the resident loop.
 template <typename KO>
-__global__ void __launch_bounds__(256) k_res_count(JoinSpec S, const KO* __restrict__ okeys, const float* __restrict__ otags,
-                                                   const ResState* __restrict__ st, uint32_t* __restrict__ deg, uint4* __restrict__ rowinfo,
-                                                   uint32_t* __restrict__ err) {
-  const uint32_t n = st->status == kResOk ? st->n_delta : 0;
-  for (uint32_t i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x)
-    join_count_row<KO>(S, okeys, otags, i, deg, rowinfo, err);
-}
-
-static __global__ void __launch_bounds__(kScanBlock) k_res_tile_sums(const uint32_t* __restrict__ deg, const ResState* __restrict__ st,
-                                                                     uint64_t* __restrict__ tile_sums) {
+__global__ void __launch_bounds__(kScanBlock) k_res_count_scan(JoinSpec S, const KO* __restrict__ okeys, const float* __restrict__ otags,
+                                                               ResState* __restrict__ st, uint4* __restrict__ rowinfo, uint64_t* __restrict__ start,
+                                                               uint2* __restrict__ tile_rows, unsigned long long* __restrict__ status,
+                                                               uint32_t* __restrict__ ticket, uint32_t* __restrict__ err) {
   __shared__ uint64_t sh[kScanBlock / 32 + 1];
-  const uint32_t n = st->status == kResOk ? st->n_delta : 0;
-  const uint32_t tiles = (n + kScanTile - 1) / kScanTile;
-  for (uint32_t t = blockIdx.x; t < tiles; t += gridDim.x) {
-    const uint32_t base = t * kScanTile;
-    uint64_t s = 0;
-#pragma unroll
-    for (int i = 0; i < kScanItems; ++i) {
-      const uint32_t p = base + i * kScanBlock + threadIdx.x;
-      if (p < n) s += deg[p];
-    }
-    uint64_t total;
-    block_scan_excl<kScanBlock, uint64_t>(s, sh, total);
-    if (threadIdx.x == 0) tile_sums[t] = total;
-  }
-}
-
-// One block: exclusive scan of the tile sums in place; publishes the rule's candidate total and tile count.
-static __global__ void __launch_bounds__(1024) k_res_spine(uint64_t* __restrict__ tile_sums, ResState* __restrict__ st) {
-  __shared__ uint64_t sh[1024 / 32 + 1];
-  const uint32_t n = st->status == kResOk ? st->n_delta : 0;
-  const uint32_t tiles = (n + kScanTile - 1) / kScanTile;
-  uint64_t carry = 0;
-  for (uint32_t base = 0; base < tiles; base += 1024) {
-    const uint32_t p = base + threadIdx.x;
-    const uint64_t x = p < tiles ? tile_sums[p] : 0;
-    uint64_t total;
-    const uint64_t e = block_scan_excl<1024, uint64_t>(x, sh, total);
-    if (p < tiles) tile_sums[p] = carry + e;
-    carry += total;
-  }
-  if (threadIdx.x == 0) {
-    const uint64_t nt = (carry + kExpTile - 1) / kExpTile;
-    st->total = carry;
-    if (nt > st->max_tiles) { st->status = kResOverflow; st->ntiles = 0; }
-    else { st->ntiles = (uint32_t)nt; st->round_cand += carry; }
-  }
-}
-
-static __global__ void __launch_bounds__(kScanBlock) k_res_apply(const uint32_t* __restrict__ deg, const ResState* __restrict__ st,
-                                                                 const uint64_t* __restrict__ tile_base, uint64_t* __restrict__ start) {
-  __shared__ uint64_t sh[kScanBlock / 32 + 1];
-  const uint32_t n = st->status == kResOk ? st->n_delta : 0;
-  const uint32_t tiles = (n + kScanTile - 1) / kScanTile;
-  for (uint32_t t = blockIdx.x; t < tiles; t += gridDim.x) {
-    const uint32_t base = t * kScanTile + threadIdx.x * kScanItems;
-    uint64_t x[kScanItems];
-    uint64_t s = 0;
-#pragma unroll
-    for (int i = 0; i < kScanItems; ++i) { x[i] = base + i < n ? deg[base + i] : 0; s += x[i]; }
-    uint64_t total;
-    uint64_t run = block_scan_excl<kScanBlock, uint64_t>(s, sh, total) + tile_base[t];
-#pragma unroll
-    for (int i = 0; i < kScanItems; ++i) { if (base + i < n) start[base + i] = run; run += x[i]; }
-  }
-}
-
-// first and last outer row of every expand tile (see k_expand_partition)
-static __global__ void __launch_bounds__(256) k_res_partition(const uint64_t* __restrict__ start, const ResState* __restrict__ st,
-                                                              uint2* __restrict__ tile_rows) {
+  __shared__ uint32_t sdeg[kResScanTile];
+  __shared__ uint32_t s_tile;
+  __shared__ uint64_t s_excl;
   if (st->status != kResOk) return;
-  const uint32_t n = st->n_delta, ntiles = st->ntiles;
-  const uint64_t total = st->total;
-  for (uint32_t t = blockIdx.x * blockDim.x + threadIdx.x; t < ntiles; t += gridDim.x * blockDim.x) {
-    const uint64_t t_lo = (uint64_t)t * kExpTile;
-    const uint64_t t_hi = min(t_lo + kExpTile, total);
-    uint32_t r[2];
+  const uint32_t n = st->n_delta, max_tiles = st->max_tiles;
+  const uint32_t tiles = (n + kResScanTile - 1) / kResScanTile;
+  if (tiles == 0) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) { st->total = 0; st->ntiles = 0; }
+    return;
+  }
+  for (;;) {
+    if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
+    __syncthreads();
+    const uint32_t t = s_tile;
+    if (t >= tiles) break;
 #pragma unroll
-    for (int k = 0; k < 2; ++k) {
-      const uint64_t target = k == 0 ? t_lo : t_hi - 1;
-      uint32_t lo = 0, hi = n;
-      while (lo < hi) {
-        const uint32_t mid = lo + ((hi - lo) >> 1);
-        if (start[mid] <= target) lo = mid + 1; else hi = mid;
-      }
-      r[k] = lo - 1;
+    for (int i = 0; i < kResScanItems; ++i) {
+      const uint32_t row = t * kResScanTile + i * kScanBlock + threadIdx.x;
+      sdeg[i * kScanBlock + threadIdx.x] = row < n ? join_count_row<KO>(S, okeys, otags, row, rowinfo, err) : 0u;
     }
-    tile_rows[t] = make_uint2(r[0], r[1]);
+    __syncthreads();
+    uint32_t x[kResScanItems];
+    uint64_t s = 0;
+#pragma unroll
+    for (int i = 0; i < kResScanItems; ++i) { x[i] = sdeg[threadIdx.x * kResScanItems + i]; s += x[i]; }
+    uint64_t total;
+    const uint64_t in_tile = block_scan_excl<kScanBlock, uint64_t>(s, sh, total);
+    if (threadIdx.x == 0) {
+      uint64_t excl = 0;
+      bool timeout = false;
+      if (t > 0) {
+        st_volatile_u64(status + t, kScanFlagAgg | total);
+        uint32_t look = t - 1, spins = 0;
+        for (;;) {
+          const unsigned long long v = ld_volatile_u64(status + look);
+          const unsigned long long flag = v & ~kScanValMask;
+          if (flag == 0) {
+            if (++spins > kResSpinLimit) { timeout = true; break; }
+            __nanosleep(32);
+            continue;
+          }
+          excl += v & kScanValMask;
+          if (flag == kScanFlagIncl || look == 0) break;
+          --look;
+          spins = 0;
+        }
+      }
+      st_volatile_u64(status + t, kScanFlagIncl | (excl + total));
+      if (timeout) { atomicOr(err, kErrInternal); st->status = kResError; }
+      s_excl = excl;
+      if (t == tiles - 1 && !timeout) {
+        const uint64_t all = excl + total;
+        const uint64_t nt = (all + kExpTile - 1) / kExpTile;
+        st->total = all;
+        if (nt > max_tiles) { st->status = kResOverflow; st->ntiles = 0; }
+        else {
+          st->ntiles = (uint32_t)nt; st->round_cand += all;
+          if (nt) tile_rows[nt - 1].y = n - 1;           // rows after the last candidate have no matches: harmless to include
+        }
+      }
+    }
+    __syncthreads();
+    uint64_t run = s_excl + in_tile;
+#pragma unroll
+    for (int i = 0; i < kResScanItems; ++i) {
+      const uint32_t row = t * kResScanTile + threadIdx.x * kResScanItems + i;
+      if (row < n) {
+        start[row] = run;
+        if (x[i]) {
+          // expand tile u begins at position u * kExpTile and ends at (u + 1) * kExpTile - 1
+          const uint64_t end = run + x[i];                                       // one past the row's last position
+          for (uint64_t u = (run + kExpTile - 1) / kExpTile; u * kExpTile < end && u < max_tiles; ++u) tile_rows[u].x = row;
+          for (uint64_t u = (run + kExpTile) / kExpTile; u * kExpTile <= end && u <= max_tiles; ++u) tile_rows[u - 1].y = row;
+        }
+        run += x[i];
+      }
+    }
+    __syncthreads();
   }
 }
 
@@ -159,21 +180,29 @@ __global__ void __launch_bounds__(kExpBlock) k_res_expand(JoinSpec S, const KO* 
   if (lane_id() == 0 && n_new) atomicAdd(mr.n_new, (unsigned long long)n_new);
 }
 
-// One block, after k_mirror_changed_count: scan the per-tile counts of changed keys, close the round's books and decide
-// whether another round runs.  `handle` is the WHILE node's condition (ignored when use_handle == 0: the host drives).
-static __global__ void __launch_bounds__(1024) k_res_round_end(uint32_t* __restrict__ ch_sums, uint32_t ch_tiles, ResState* __restrict__ st,
-                                                               const unsigned long long* __restrict__ new_counter,
+// One block, after k_mirror_changed_count: scan the per-tile counts of changed keys into the emit kernel's offsets,
+// close the round's books, clear the scratch of the next round and decide whether it runs.  `handle` is the WHILE
+// node's condition (ignored when use_handle == 0: the host drives).
+static __global__ void __launch_bounds__(1024) k_res_round_end(ResScratch sc, uint32_t n_variants, uint32_t* __restrict__ ch_sums, uint32_t ch_tiles,
+                                                               ResState* __restrict__ st, const unsigned long long* __restrict__ new_counter,
                                                                cudaGraphConditionalHandle handle, int use_handle) {
   __shared__ uint32_t sh[1024 / 32 + 1];
   const bool live = st->status == kResOk;
+  const uint32_t n_old = st->n_delta;
   uint32_t carry = 0;
-  for (uint32_t base = 0; base < ch_tiles; base += 1024) {
-    const uint32_t p = base + threadIdx.x;
-    const uint32_t x = p < ch_tiles ? ch_sums[p] : 0;
-    uint32_t total;
-    const uint32_t e = block_scan_excl<1024, uint32_t>(x, sh, total);
-    if (p < ch_tiles) ch_sums[p] = carry + e;
-    carry += total;
+  if (live) {
+    for (uint32_t base = 0; base < ch_tiles; base += 1024) {
+      const uint32_t p = base + threadIdx.x;
+      const uint32_t x = p < ch_tiles ? ch_sums[p] : 0;
+      uint32_t total;
+      const uint32_t e = block_scan_excl<1024, uint32_t>(x, sh, total);
+      if (p < ch_tiles) ch_sums[p] = carry + e;
+      carry += total;
+    }
+    const uint32_t tiles = (n_old + kResScanTile - 1) / kResScanTile + 1;
+    for (uint32_t v = 0; v < n_variants; ++v)
+      for (uint32_t i = threadIdx.x; i < tiles && i < sc.scan_tiles_cap; i += blockDim.x) sc.scan_status[(size_t)v * sc.scan_tiles_cap + i] = 0;
+    for (uint32_t i = threadIdx.x; i < kResMaxVariants; i += blockDim.x) sc.tickets[i] = 0;
   }
   if (threadIdx.x == 0) {
     unsigned again = 0;

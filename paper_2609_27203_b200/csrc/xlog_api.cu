@@ -1004,7 +1004,7 @@ Resident* resident_for(Ctx* c, int h, int bits, uint64_t slots, uint32_t bm_quad
   if (it != c->resident.end() && it->second->slots == slots && it->second->max_tiles == max_tiles) return it->second.get();
   c->resident.erase(h);
   const uint64_t dom = (uint64_t)1 << bits;
-  const uint64_t need = slots * 4 + (uint64_t)bm_quads * 16 + dom * 36 + (uint64_t)max_tiles * 8 + (2u << 20);
+  const uint64_t need = slots * 4 + (uint64_t)bm_quads * 16 + dom * 32 + (uint64_t)max_tiles * 8 + (4u << 20);
   if (need > c->arena.largest_free() / 3) return nullptr;
   std::unique_ptr<Resident> R(new Resident());
   R->slots = slots; R->max_tiles = max_tiles;
@@ -1012,12 +1012,28 @@ Resident* resident_for(Ctx* c, int h, int bits, uint64_t slots, uint32_t bm_quad
   R->bitmap = DevBuf(c, (size_t)bm_quads * 16);
   R->ch_sums = DevBuf(c, (size_t)ch_tiles * 4);
   R->dkeys = DevBuf(c, dom * 4); R->dtags = DevBuf(c, dom * 4);
-  R->deg = DevBuf(c, dom * 4); R->rowinfo = DevBuf(c, dom * 16); R->start = DevBuf(c, dom * 8);
-  R->sums = DevBuf(c, (dom / kScanTile + 1) * 8);
+  R->rowinfo = DevBuf(c, dom * 16); R->start = DevBuf(c, dom * 8);
+  R->scan_tiles_cap = (uint32_t)(dom / kResScanTile + 2);
+  R->scan_status = DevBuf(c, (size_t)kResMaxVariants * R->scan_tiles_cap * 8);
+  R->tickets = DevBuf(c, kResMaxVariants * 4);
   R->tile_rows = DevBuf(c, (size_t)max_tiles * 8);
   Resident* out = R.get();
   c->resident[h] = std::move(R);
   return out;
+}
+
+// bitmap tiles: one sweep of 256 words per tile for domains up to 2^22 keys (so that small domains still give hundreds of
+// blocks), four sweeps above that
+int mirror_sweeps(uint32_t nwords) { return nwords <= (1u << 17) ? 1 : 4; }
+unsigned mirror_tiles(uint32_t nwords) { const uint32_t per = kMirBlock * mirror_sweeps(nwords); return (nwords + per - 1) / per; }
+void launch_changed_count(Ctx* c, const uint32_t* words, uint32_t nwords, unsigned tiles, uint32_t* sums) {
+  if (mirror_sweeps(nwords) == 1) XLOG_LAUNCH(c, (k_mirror_changed_count<1>), tiles, kMirBlock, 0, words, nwords, sums);
+  else XLOG_LAUNCH(c, (k_mirror_changed_count<4>), tiles, kMirBlock, 0, words, nwords, sums);
+}
+void launch_changed_emit(Ctx* c, uint32_t* words, uint32_t nwords, unsigned tiles, const uint32_t* base, const int32_t* table, uint32_t* keys,
+                         float* tags, const uint32_t* skip) {
+  if (mirror_sweeps(nwords) == 1) XLOG_LAUNCH(c, (k_mirror_changed_emit<uint32_t, 1>), tiles, kMirBlock, 0, words, nwords, base, table, keys, tags, skip);
+  else XLOG_LAUNCH(c, (k_mirror_changed_emit<uint32_t, 4>), tiles, kMirBlock, 0, words, nwords, base, table, keys, tags, skip);
 }
 
 template <typename T> void sig_add(std::vector<char>& sig, const T& v) {
@@ -1032,14 +1048,11 @@ void resident_body(Ctx* c, Resident& R, const std::vector<JoinSpec>& specs, bool
   ResState* st = res_state(c);
   uint32_t* err = ctrl_u32(c, kSlotErr);
   const uint32_t* dk = R.dkeys.as<uint32_t>();
-  for (const JoinSpec& S : specs) {
-    XLOG_LAUNCH(c, (k_res_count<uint32_t>), kSMs * 8, 256, 0, S, dk, (const float*)R.dtags.as<float>(), (const ResState*)st, R.deg.as<uint32_t>(),
-                R.rowinfo.as<uint4>(), err);
-    XLOG_LAUNCH(c, k_res_tile_sums, kSMs * 2, kScanBlock, 0, (const uint32_t*)R.deg.as<uint32_t>(), (const ResState*)st, R.sums.as<uint64_t>());
-    XLOG_LAUNCH(c, k_res_spine, 1, 1024, 0, R.sums.as<uint64_t>(), st);
-    XLOG_LAUNCH(c, k_res_apply, kSMs * 2, kScanBlock, 0, (const uint32_t*)R.deg.as<uint32_t>(), (const ResState*)st, (const uint64_t*)R.sums.as<uint64_t>(),
-                R.start.as<uint64_t>());
-    XLOG_LAUNCH(c, k_res_partition, kSMs, 256, 0, (const uint64_t*)R.start.as<uint64_t>(), (const ResState*)st, R.tile_rows.as<uint2>());
+  const ResScratch sc{R.scan_status.as<unsigned long long>(), R.scan_tiles_cap, R.tickets.as<uint32_t>()};
+  for (size_t v = 0; v < specs.size(); ++v) {
+    const JoinSpec& S = specs[v];
+    XLOG_LAUNCH(c, (k_res_count_scan<uint32_t>), kSMs * 4, kScanBlock, 0, S, dk, (const float*)R.dtags.as<float>(), st, R.rowinfo.as<uint4>(),
+                R.start.as<uint64_t>(), R.tile_rows.as<uint2>(), sc.scan_status + v * R.scan_tiles_cap, sc.tickets + v, err);
 #define XLOG_RES_EXPAND(MODE, SINK)                                                                                                         \
   XLOG_LAUNCH(c, (k_res_expand<uint32_t, MODE, SINK>), kSMs * 4, kExpBlock, 0, S, dk, (const ResState*)st, (const uint64_t*)R.start.as<uint64_t>(), \
               (const uint4*)R.rowinfo.as<uint4>(), (const uint2*)R.tile_rows.as<uint2>(), err, mr)
@@ -1047,15 +1060,16 @@ void resident_body(Ctx* c, Resident& R, const std::vector<JoinSpec>& specs, bool
     else { if (is_max) XLOG_RES_EXPAND(kExpGeneric, kSinkMax); else XLOG_RES_EXPAND(kExpGeneric, kSinkMin); }
 #undef XLOG_RES_EXPAND
   }
-  XLOG_LAUNCH(c, k_mirror_changed_count, ch_tiles, kMirBlock, 0, (const uint4*)R.bitmap.as<uint4>(), bm_quads, R.ch_sums.as<uint32_t>());
-  XLOG_LAUNCH(c, k_res_round_end, 1, 1024, 0, R.ch_sums.as<uint32_t>(), (uint32_t)ch_tiles, st, (const unsigned long long*)mr.n_new, handle, use_handle);
-  XLOG_LAUNCH(c, (k_mirror_changed_emit<uint32_t>), ch_tiles, kMirBlock, 0, R.bitmap.as<uint4>(), bm_quads, (const uint32_t*)R.ch_sums.as<uint32_t>(),
-              (const int32_t*)R.table.as<int32_t>(), R.dkeys.as<uint32_t>(), R.dtags.as<float>(), (const uint32_t*)&st->status);
+  launch_changed_count(c, R.bitmap.as<uint32_t>(), bm_quads * 4, ch_tiles, R.ch_sums.as<uint32_t>());
+  XLOG_LAUNCH(c, k_res_round_end, 1, 1024, 0, sc, (uint32_t)specs.size(), R.ch_sums.as<uint32_t>(), (uint32_t)ch_tiles, st,
+              (const unsigned long long*)mr.n_new, handle, use_handle);
+  launch_changed_emit(c, R.bitmap.as<uint32_t>(), bm_quads * 4, ch_tiles, R.ch_sums.as<uint32_t>(), R.table.as<int32_t>(), R.dkeys.as<uint32_t>(),
+                      R.dtags.as<float>(), (const uint32_t*)&st->status);
 }
 
 // Run rounds on the device until the delta is empty, the round budget is used up or a round needs more tiles than
 // planned.  Returns the final state block (read once, after the loop).
-ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*>& rs, bool is_max, const MirrorArgs& mr, uint32_t bm_quads,
+ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*>& rs, bool is_max, const MirrorArgs& mr_host, uint32_t bm_quads,
                       unsigned ch_tiles, uint32_t n_delta, int64_t rounds_left, uint64_t new_seen) {
   Relation& H = *c->rels[h];
   std::vector<JoinSpec> specs;
@@ -1067,7 +1081,9 @@ ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*
       }
   if (specs.size() > 16) fail(XLOG_ERR_UNSUPPORTED, "too many rule variants for one head");
   const uint32_t budget = (uint32_t)std::min<int64_t>(rounds_left, 0x7fffffff);
-  XLOG_LAUNCH(c, k_res_init, 1, 32, 0, res_state(c), n_delta, budget, R.max_tiles, (unsigned long long)new_seen);
+  const ResScratch sc{R.scan_status.as<unsigned long long>(), R.scan_tiles_cap, R.tickets.as<uint32_t>()};
+  XLOG_LAUNCH(c, k_res_init, 1, 1024, 0, res_state(c), sc, (uint32_t)specs.size(), n_delta, budget, R.max_tiles, (unsigned long long)new_seen);
+  const MirrorArgs& mr = mr_host;
   const int64_t l0 = c->launches;
   const bool use_graph = !(c->flags & (XLOG_FLAG_PROFILE | XLOG_FLAG_NO_GRAPH));
   ResState out{};
@@ -1140,7 +1156,7 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
   const int32_t empty = is_max ? kMirrorEmptyMax : kMirrorEmptyMin;
   const uint64_t slots = std::max<uint64_t>(dom, 4);
   const uint32_t bm_quads = (uint32_t)((std::max<uint64_t>(dom / 32, 1) + 3) / 4);
-  const unsigned ch_tiles = (bm_quads + kMirBlock - 1) / kMirBlock;
+  const unsigned ch_tiles = mirror_tiles(bm_quads * 4);
   Resident* R = resident_for(c, h, bits, slots, bm_quads, ch_tiles);
   DevBuf table_own, bitmap_own, ch_sums_own;
   if (!R) { table_own = DevBuf(c, slots * 4); bitmap_own = DevBuf(c, (size_t)bm_quads * 16); ch_sums_own = DevBuf(c, (size_t)ch_tiles * 4); }
@@ -1197,7 +1213,7 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
       q.start.reset(); q.rowinfo.reset();
     }
     if (total == 0) break;
-    XLOG_LAUNCH(c, k_mirror_changed_count, ch_tiles, kMirBlock, 0, (const uint4*)bitmap, bm_quads, ch_sums);
+    launch_changed_count(c, reinterpret_cast<const uint32_t*>(bitmap), bm_quads * 4, ch_tiles, ch_sums);
     XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, ch_sums, (int64_t)ch_tiles, ctrl_u32(c, kSlotMirChanged));
     sync_ctrl(c);
     const uint32_t changed = (uint32_t)c->h_ctrl[kSlotMirChanged];
@@ -1214,8 +1230,7 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
       ek = delta_own.keys.as<uint32_t>(); et = delta_own.tags.as<float>();
     }
     c->note_bytes = (int64_t)bm_quads * 16 + (int64_t)changed * 12;
-    XLOG_LAUNCH(c, (k_mirror_changed_emit<uint32_t>), ch_tiles, kMirBlock, 0, bitmap, bm_quads, (const uint32_t*)ch_sums, (const int32_t*)table, ek, et,
-                (const uint32_t*)nullptr);
+    launch_changed_emit(c, reinterpret_cast<uint32_t*>(bitmap), bm_quads * 4, ch_tiles, ch_sums, table, ek, et, nullptr);
     dk = ek; dt = et; dn = changed;
     if (R && !resident_done) {
       // hand the delta rounds to the device
