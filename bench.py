@@ -193,7 +193,7 @@ def run_ours(args):
     program, arena = make_program(args.workload, args.scale, args.sources)
 
     # facts resident in HBM before any timed region
-    base_flags = xlog.FLAG_NO_TAG_MIRROR if args.no_tag_mirror else 0
+    base_flags = (xlog.FLAG_NO_TAG_MIRROR if args.no_tag_mirror else 0) | (xlog.FLAG_NO_GRAPH if args.no_graph else 0)
     ctx, ids, rules = xlog.load_program(program, device=local_rank, arena_bytes=arena, device_inputs=True, flags=base_flags)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)          # > 126 MB L2
 
@@ -362,6 +362,7 @@ def main():
     ap.add_argument("--workload", default="sssp", choices=["sssp", "closure", "reach", "triangles", "digits"])
     ap.add_argument("--scale", type=int, default=None, help="R-MAT scale override (smaller cases for profiling)")
     ap.add_argument("--sources", type=int, default=None, help="reach: number of sources (fewer for a small profiling case)")
+    ap.add_argument("--no-graph", action="store_true", help="launch the resident rounds one by one (for per-launch profiling)")
     ap.add_argument("--no-tag-mirror", action="store_true", help="evaluate recursion by sort -> reduce-by-key -> merge only")
     ap.add_argument("--cpu-scale", type=int, default=None, help="R-MAT scale of the cpu_baseline sample (default: the workload's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")

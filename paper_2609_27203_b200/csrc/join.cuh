@@ -192,6 +192,12 @@ struct MirrorArgs {
 constexpr int32_t kMirrorEmptyMin = 0x7fffffff;
 constexpr int32_t kMirrorEmptyMax = (int32_t)0x80000000;
 
+// The pre-check may read a stale slot: slots only ever move towards the better value, so a stale value can only make a
+// candidate look better than it is, and the atomic that follows decides.
+#ifndef XLOG_TABLE_LOAD
+#define XLOG_TABLE_LOAD(p) __ldcg(p)
+#endif
+
 template <int SINK>
 __device__ __forceinline__ void mirror_commit(const MirrorArgs& m, uint32_t key, int32_t v, uint32_t& n_new) {
   const int32_t old = SINK == kSinkMin ? atomicMin(m.table + key, v) : atomicMax(m.table + key, v);
@@ -338,7 +344,7 @@ __device__ __forceinline__ void expand_tile(ExpSmem& sm, const JoinSpec& S, cons
         cur[k] = SINK == kSinkMin ? (int32_t)0x80000000 : 0x7fffffff;        // nothing improves on this
         if (q < ntile) {
           if ((uint32_t)key[k] > mr.key_max) atomicOr(mr.err, kErrHeadRange);
-          else cur[k] = __ldcg(mr.table + (uint32_t)key[k]);
+          else cur[k] = XLOG_TABLE_LOAD(mr.table + (uint32_t)key[k]);
         }
       }
 #pragma unroll

@@ -4,7 +4,7 @@
 // launches whose sizes are read from a small state block in device memory:
 //
 //   per rule with a recursive atom:  k_res_count_scan -> k_res_expand
-//   then:                            k_mirror_changed_count -> k_res_round_end -> k_mirror_changed_emit
+//   then:                            k_res_emit (next delta, round bookkeeping, loop condition)
 //
 // Every kernel has a fixed grid and strides over however much work the state block announces, so the
 // sequence can be captured once as the body of a CUDA-graph WHILE node; k_res_round_end decides whether
@@ -14,6 +14,7 @@
 
 #include "common.cuh"
 #include "join.cuh"
+#include "mirror.cuh"
 #include "scan.cuh"
 
 namespace xlog {
@@ -48,7 +49,7 @@ __device__ __forceinline__ void st_volatile_u64(unsigned long long* p, unsigned 
 struct ResScratch {
   unsigned long long* scan_status;   // [kResMaxVariants][scan_tiles_cap]
   uint32_t scan_tiles_cap;
-  uint32_t* tickets;                 // [kResMaxVariants]
+  uint32_t* tickets;                 // [kResMaxVariants], then the emit kernel's two counters
 };
 
 static __global__ void __launch_bounds__(1024) k_res_init(ResState* st, ResScratch sc, uint32_t n_variants, uint32_t n_delta, uint32_t max_rounds,
@@ -60,7 +61,7 @@ static __global__ void __launch_bounds__(1024) k_res_init(ResState* st, ResScrat
   }
   // everything, not just what the first round will touch: an abandoned loop leaves its last round's words behind
   for (size_t i = threadIdx.x; i < (size_t)n_variants * sc.scan_tiles_cap; i += blockDim.x) sc.scan_status[i] = 0;
-  for (uint32_t i = threadIdx.x; i < kResMaxVariants; i += blockDim.x) sc.tickets[i] = 0;
+  for (uint32_t i = threadIdx.x; i < kResMaxVariants + 2; i += blockDim.x) sc.tickets[i] = 0;       // tickets and the emit kernel's two counters
 }
 
 // Count, scan and partition of one rule in a single launch.  Blocks draw 1024-row tiles from a ticket counter (so a tile
@@ -103,37 +104,50 @@ __global__ void __launch_bounds__(kScanBlock) k_res_count_scan(JoinSpec S, const
     for (int i = 0; i < kResScanItems; ++i) { x[i] = sdeg[threadIdx.x * kResScanItems + i]; s += x[i]; }
     uint64_t total;
     const uint64_t in_tile = block_scan_excl<kScanBlock, uint64_t>(s, sh, total);
-    if (threadIdx.x == 0) {
+    if (warp_id() == 0) {
+      // look back 32 tiles at a time: lane l polls tile (base - l) until it holds at least an aggregate; the nearest
+      // inclusive prefix among them ends the walk
       uint64_t excl = 0;
       bool timeout = false;
       if (t > 0) {
-        st_volatile_u64(status + t, kScanFlagAgg | total);
-        uint32_t look = t - 1, spins = 0;
+        if (lane_id() == 0) st_volatile_u64(status + t, kScanFlagAgg | total);
+        int64_t base = (int64_t)t - 1;
         for (;;) {
-          const unsigned long long v = ld_volatile_u64(status + look);
-          const unsigned long long flag = v & ~kScanValMask;
-          if (flag == 0) {
-            if (++spins > kResSpinLimit) { timeout = true; break; }
-            __nanosleep(32);
-            continue;
+          const int64_t idx = base - (int64_t)lane_id();
+          unsigned long long v = kScanFlagIncl;                         // before tile 0: an inclusive prefix of zero
+          if (idx >= 0) {
+            uint32_t spins = 0;
+            for (;;) {
+              v = ld_volatile_u64(status + idx);
+              if (v & ~kScanValMask) break;
+              if (++spins > kResSpinLimit) { timeout = true; v = kScanFlagIncl; break; }
+              if (spins > 64) __nanosleep(32);
+            }
           }
-          excl += v & kScanValMask;
-          if (flag == kScanFlagIncl || look == 0) break;
-          --look;
-          spins = 0;
+          const unsigned incl = __ballot_sync(0xffffffffu, (v & ~kScanValMask) == kScanFlagIncl);
+          const int first = incl ? __ffs(incl) - 1 : 31;                // lanes 0 .. first contribute
+          unsigned long long part = (int)lane_id() <= first ? (v & kScanValMask) : 0ull;
+#pragma unroll
+          for (int d = 16; d > 0; d >>= 1) part += __shfl_xor_sync(0xffffffffu, part, d);
+          excl += part;
+          if (incl) break;
+          base -= 32;
         }
+        timeout = __any_sync(0xffffffffu, timeout);
       }
-      st_volatile_u64(status + t, kScanFlagIncl | (excl + total));
-      if (timeout) { atomicOr(err, kErrInternal); st->status = kResError; }
-      s_excl = excl;
-      if (t == tiles - 1 && !timeout) {
-        const uint64_t all = excl + total;
-        const uint64_t nt = (all + kExpTile - 1) / kExpTile;
-        st->total = all;
-        if (nt > max_tiles) { st->status = kResOverflow; st->ntiles = 0; }
-        else {
-          st->ntiles = (uint32_t)nt; st->round_cand += all;
-          if (nt) tile_rows[nt - 1].y = n - 1;           // rows after the last candidate have no matches: harmless to include
+      if (lane_id() == 0) {
+        st_volatile_u64(status + t, kScanFlagIncl | (excl + total));
+        if (timeout) { atomicOr(err, kErrInternal); st->status = kResError; }
+        s_excl = excl;
+        if (t == tiles - 1 && !timeout) {
+          const uint64_t all = excl + total;
+          const uint64_t nt = (all + kExpTile - 1) / kExpTile;
+          st->total = all;
+          if (nt > max_tiles) { st->status = kResOverflow; st->ntiles = 0; }
+          else {
+            st->ntiles = (uint32_t)nt; st->round_cand += all;
+            if (nt) tile_rows[nt - 1].y = n - 1;           // rows after the last candidate have no matches: harmless to include
+          }
         }
       }
     }
@@ -153,6 +167,7 @@ __global__ void __launch_bounds__(kScanBlock) k_res_count_scan(JoinSpec S, const
         run += x[i];
       }
     }
+    if (tiles <= gridDim.x) break;            // every block draws one ticket first, so all tiles are already taken
     __syncthreads();
   }
 }
@@ -180,30 +195,77 @@ __global__ void __launch_bounds__(kExpBlock) k_res_expand(JoinSpec S, const KO* 
   if (lane_id() == 0 && n_new) atomicAdd(mr.n_new, (unsigned long long)n_new);
 }
 
-// One block, after k_mirror_changed_count: scan the per-tile counts of changed keys into the emit kernel's offsets,
-// close the round's books, clear the scratch of the next round and decide whether it runs.  `handle` is the WHILE
-// node's condition (ignored when use_handle == 0: the host drives).
-static __global__ void __launch_bounds__(1024) k_res_round_end(ResScratch sc, uint32_t n_variants, uint32_t* __restrict__ ch_sums, uint32_t ch_tiles,
-                                                               ResState* __restrict__ st, const unsigned long long* __restrict__ new_counter,
-                                                               cudaGraphConditionalHandle handle, int use_handle) {
-  __shared__ uint32_t sh[1024 / 32 + 1];
-  const bool live = st->status == kResOk;
-  const uint32_t n_old = st->n_delta;
-  uint32_t carry = 0;
+// Last kernel of a round: compact the changed bitmap into the next delta and close the round.  Inside the resident
+// loop the delta need not be in key order (the join reads it row by row and max / min do not care about order), so a
+// block reserves room for its tile's keys with one atomic add instead of waiting for a prefix sum; row order in the
+// delta therefore varies from run to run, the relation derived does not.  The block that finishes last closes the
+// round's books, clears the scratch of the next round and decides whether it runs: `handle` is the WHILE node's
+// condition (ignored when use_handle == 0: the host drives).
+// ctr[0] = rows reserved so far, ctr[1] = blocks done; both are left at zero.
+template <int SW>
+__global__ void __launch_bounds__(kMirBlock) k_res_emit(uint32_t* __restrict__ words, uint32_t nwords, const int32_t* __restrict__ table,
+                                                        uint32_t* __restrict__ keys, float* __restrict__ tags, ResState* __restrict__ st,
+                                                        ResScratch sc, uint32_t n_variants, const unsigned long long* __restrict__ new_counter,
+                                                        uint32_t* __restrict__ ctr, cudaGraphConditionalHandle handle, int use_handle) {
+  __shared__ uint32_t sh[kMirBlock / 32 + 1];
+  __shared__ uint32_t list[kMirBlock * 32];
+  __shared__ uint32_t s_base, s_last;
+  const bool live = st->status == kResOk;                // an abandoned round keeps its bitmap and its delta
   if (live) {
-    for (uint32_t base = 0; base < ch_tiles; base += 1024) {
-      const uint32_t p = base + threadIdx.x;
-      const uint32_t x = p < ch_tiles ? ch_sums[p] : 0;
-      uint32_t total;
-      const uint32_t e = block_scan_excl<1024, uint32_t>(x, sh, total);
-      if (p < ch_tiles) ch_sums[p] = carry + e;
-      carry += total;
+    uint32_t w[SW];
+    uint32_t cnt = 0;
+#pragma unroll
+    for (int j = 0; j < SW; ++j) {
+      const uint32_t wi = (blockIdx.x * SW + j) * kMirBlock + threadIdx.x;
+      w[j] = wi < nwords ? words[wi] : 0u;
+      cnt += __popc(w[j]);
     }
-    const uint32_t tiles = (n_old + kResScanTile - 1) / kResScanTile + 1;
+    uint32_t tile_total;
+    block_scan_excl<kMirBlock, uint32_t>(cnt, sh, tile_total);
+    if (tile_total) {                                    // uniform across the block
+      if (threadIdx.x == 0) s_base = atomicAdd(&ctr[0], tile_total);
+      __syncthreads();
+      uint32_t out = s_base;
+#pragma unroll
+      for (int j = 0; j < SW; ++j) {
+        const uint32_t wi = (blockIdx.x * SW + j) * kMirBlock + threadIdx.x;
+        uint32_t bits = w[j];
+        uint32_t total;
+        uint32_t pos = block_scan_excl<kMirBlock, uint32_t>((uint32_t)__popc(bits), sh, total);
+        if (total == 0) continue;
+        if (bits) words[wi] = 0u;
+        while (bits) {
+          const int b = __ffs(bits) - 1;
+          bits &= bits - 1;
+          list[pos++] = (wi << 5) + b;
+        }
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < total; i += kMirBlock) {
+          const uint32_t key = list[i];
+          keys[out + i] = key;
+          tags[out + i] = ord2f(__ldcg(table + key));
+        }
+        out += total;
+        __syncthreads();
+      }
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    s_last = atomicAdd(&ctr[1], 1u) == gridDim.x - 1 ? 1u : 0u;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  const uint32_t changed = live ? *reinterpret_cast<volatile uint32_t*>(&ctr[0]) : 0u;
+  if (live) {
+    const uint32_t tiles = (st->n_delta + kResScanTile - 1) / kResScanTile + 1;
     for (uint32_t v = 0; v < n_variants; ++v)
       for (uint32_t i = threadIdx.x; i < tiles && i < sc.scan_tiles_cap; i += blockDim.x) sc.scan_status[(size_t)v * sc.scan_tiles_cap + i] = 0;
     for (uint32_t i = threadIdx.x; i < kResMaxVariants; i += blockDim.x) sc.tickets[i] = 0;
   }
+  __syncthreads();
   if (threadIdx.x == 0) {
     unsigned again = 0;
     if (live) {
@@ -211,15 +273,16 @@ static __global__ void __launch_bounds__(1024) k_res_round_end(ResScratch sc, ui
       const unsigned long long fresh = seen - st->new_seen;
       st->new_seen = seen;
       st->n_new += fresh;
-      st->n_improved += (unsigned long long)carry - fresh;
+      st->n_improved += (unsigned long long)changed - fresh;
       st->candidates += st->round_cand;
       st->round_cand = 0;
-      st->n_delta = carry;
+      st->n_delta = changed;
       st->rounds += 1;
-      if (carry > 0) {
+      if (changed > 0) {
         if (st->rounds >= st->max_rounds) st->status = kResCap; else again = 1;
       }
     }
+    ctr[0] = 0; ctr[1] = 0;
     if (use_handle) cudaGraphSetConditional(handle, again);
   }
 }

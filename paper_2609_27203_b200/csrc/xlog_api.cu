@@ -1015,7 +1015,7 @@ Resident* resident_for(Ctx* c, int h, int bits, uint64_t slots, uint32_t bm_quad
   R->rowinfo = DevBuf(c, dom * 16); R->start = DevBuf(c, dom * 8);
   R->scan_tiles_cap = (uint32_t)(dom / kResScanTile + 2);
   R->scan_status = DevBuf(c, (size_t)kResMaxVariants * R->scan_tiles_cap * 8);
-  R->tickets = DevBuf(c, kResMaxVariants * 4);
+  R->tickets = DevBuf(c, (kResMaxVariants + 2) * 4);
   R->tile_rows = DevBuf(c, (size_t)max_tiles * 8);
   Resident* out = R.get();
   c->resident[h] = std::move(R);
@@ -1060,11 +1060,12 @@ void resident_body(Ctx* c, Resident& R, const std::vector<JoinSpec>& specs, bool
     else { if (is_max) XLOG_RES_EXPAND(kExpGeneric, kSinkMax); else XLOG_RES_EXPAND(kExpGeneric, kSinkMin); }
 #undef XLOG_RES_EXPAND
   }
-  launch_changed_count(c, R.bitmap.as<uint32_t>(), bm_quads * 4, ch_tiles, R.ch_sums.as<uint32_t>());
-  XLOG_LAUNCH(c, k_res_round_end, 1, 1024, 0, sc, (uint32_t)specs.size(), R.ch_sums.as<uint32_t>(), (uint32_t)ch_tiles, st,
-              (const unsigned long long*)mr.n_new, handle, use_handle);
-  launch_changed_emit(c, R.bitmap.as<uint32_t>(), bm_quads * 4, ch_tiles, R.ch_sums.as<uint32_t>(), R.table.as<int32_t>(), R.dkeys.as<uint32_t>(),
-                      R.dtags.as<float>(), (const uint32_t*)&st->status);
+  uint32_t* ctr = sc.tickets + kResMaxVariants;
+#define XLOG_RES_EMIT(SW)                                                                                                                  \
+  XLOG_LAUNCH(c, (k_res_emit<SW>), ch_tiles, kMirBlock, 0, R.bitmap.as<uint32_t>(), bm_quads * 4, (const int32_t*)R.table.as<int32_t>(),   \
+              R.dkeys.as<uint32_t>(), R.dtags.as<float>(), st, sc, (uint32_t)specs.size(), (const unsigned long long*)mr.n_new, ctr, handle, use_handle)
+  if (mirror_sweeps(bm_quads * 4) == 1) XLOG_RES_EMIT(1); else XLOG_RES_EMIT(4);
+#undef XLOG_RES_EMIT
 }
 
 // Run rounds on the device until the delta is empty, the round budget is used up or a round needs more tiles than
