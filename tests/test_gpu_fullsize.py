@@ -16,11 +16,24 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def gpu_fixpoint(program, arena):
+def gpu_fixpoint(program, arena, flags=0):
     from paper_2609_27203_b200 import xlog
-    ctx, ids, rules = xlog.load_program(program, arena_bytes=arena, device_inputs=True)
+    ctx, ids, rules = xlog.load_program(program, arena_bytes=arena, device_inputs=True, flags=flags)
     receipt = ctx.fixpoint()
     return ctx, ids, rules, receipt
+
+
+def same_on_the_sorting_path(program, arena, name, cols, tags, receipt):
+    """The default path evaluates these recursions through the tag mirror; sort -> reduce-by-key -> merge must derive
+    the same relation bit for bit, with the same counters."""
+    from paper_2609_27203_b200 import xlog
+    ctx, ids, _, r2 = gpu_fixpoint(program, arena, xlog.FLAG_NO_TAG_MIRROR)
+    c2, t2 = ctx.read(ids[name])
+    ctx.close()
+    assert all(np.array_equal(a, b) for a, b in zip(cols, c2)) and np.array_equal(tags.view(np.int32), t2.view(np.int32))
+    for k in ("iterations", "candidates", "new_tuples", "improved_tags", "derived_tuples"):
+        assert receipt[k] == r2[k], k
+    assert receipt["unique_candidates"] == -1 and r2["unique_candidates"] > 0
 
 
 def test_config2_sssp_rmat20_full():
@@ -32,7 +45,9 @@ def test_config2_sssp_rmat20_full():
     assert rep["bit_unequal"] == 0 and receipt["derived_tuples"] == stats["derived_tuples"]
     again = ctx.fixpoint()                      # fixpoint idempotence at full size
     assert again["new_tuples"] == 0 and again["improved_tags"] == 0
+    cols, tags = ctx.read(ids["dist"])
     ctx.close()
+    same_on_the_sorting_path(prog, 4 << 30, "dist", cols, tags, receipt)
 
 
 def test_config4_digits_full_forward_and_backward():
@@ -119,3 +134,4 @@ def test_config5_reach_rmat22_full_one_source_by_oracle():
     for dead in srcs[deg[srcs] == 0][:5].tolist():
         assert int((rc[0] == dead).sum()) == 1
     ctx.close()
+    same_on_the_sorting_path(prog, 56 << 30, "reach", rc, rt, receipt)
