@@ -34,6 +34,9 @@ UNIT = "tuples/s"
 # (dram__bytes_read.sum + dram__bytes_write.sum over the launch's algorithmic bytes).  Used only to
 # scale a captured launch to the bench's launch size; None = not captured.
 NCU_TRAFFIC_RATIO = {"k_sort_pass": 0.99, "k_join_expand": 0.92, "k_dense_reduce": 1.04, "k_merge": 1.0}
+# the join kernels when they apply candidates to the tag mirror instead of writing them: the slot reads hit L2, so DRAM
+# sees the adjacency reads (8 of the 12 algorithmic bytes per candidate) plus row records
+NCU_TRAFFIC_RATIO_MIRROR = {"k_join_expand": 0.80, "k_res_expand": 0.80}
 
 
 def make_program(name: str, scale: int | None, sources: int | None = None):
@@ -242,6 +245,9 @@ def run_ours(args):
     peak, peak_src = measured_peak_gbs()
     achieved = d["bytes"] / (d["ms"] / 1e3) / 1e9 if d["ms"] > 0 else 0.0
     ratio = NCU_TRAFFIC_RATIO.get(dom)
+    mirror_kernel = dom == "k_res_expand" or (dom == "k_join_expand" and not args.no_tag_mirror and "k_sort_pass" not in prof)
+    if mirror_kernel:
+        ratio = NCU_TRAFFIC_RATIO_MIRROR.get(dom)
     bound = "hbm"
     if dom.startswith("k_tri"):
         bound = "alu"      # sorted-list intersections out of L2: not an HBM-bound kernel (kernels)
@@ -253,7 +259,14 @@ def run_ours(args):
                 "kernels": {k: {"launches_per_step": v["launches"] / args.steps, "ms_per_step": v["ms"] / args.steps,
                                 "GBps": (v["bytes"] / (v["ms"] / 1e3) / 1e9) if v["ms"] > 0 and v["bytes"] else None}
                             for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])},
-                "how": "second pass of the same steps with XLOG_FLAG_PROFILE (CUDA events around every launch on the ctx stream)"}
+                "how": "second pass of the same steps with XLOG_FLAG_PROFILE (CUDA events around every launch on the ctx stream; "
+                       "the resident rounds are then launched one by one instead of as one graph)"}
+    if mirror_kernel:
+        # one random 32-byte L2 sector per candidate (the key's slot in the tag mirror) on top of the streamed adjacency
+        # reads: the kernel is bound by how many such sector requests the SMs keep in flight, not by HBM
+        roofline["limiter"] = "L2 random sector access (one tag-mirror slot per candidate); HBM carries about 8 B per candidate"
+        per_cand = 12.0
+        roofline["candidates_per_s"] = achieved * 1e9 / per_cand
 
     # end to end through the C ABI with HOST buffers: load (H2D + sort + index), fixpoint, read back (D2H)
     pinned = {}

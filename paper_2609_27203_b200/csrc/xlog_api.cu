@@ -1136,9 +1136,17 @@ ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*
     read_state();
     c->launches = l0 + R.body_launches * (int64_t)out.rounds + (out.status == kResOverflow ? R.body_launches : 0);
   } else {
+    unsigned long long seen = 0;
     for (;;) {
       resident_body(c, R, specs, is_max, mr, bm_quads, ch_tiles, cudaGraphConditionalHandle{}, 0);
       read_state();
+      if (c->flags & XLOG_FLAG_PROFILE) {
+        // algorithmic bytes of the round's expand launches (per candidate: the looked-up columns and tag, and the slot)
+        auto it = c->prof_index.find("k_res_expand");
+        if (it != c->prof_index.end())
+          c->prof[it->second].bytes += (int64_t)(out.candidates - seen) * (4 + (specs[0].has_inner ? 4 * (specs[0].inner_free + 1) : 0));
+        seen = out.candidates;
+      }
       if (out.status != kResOk || out.n_delta == 0) break;
     }
   }
