@@ -74,9 +74,22 @@ typedef struct {
 
 #define XLOG_FLAG_CHECK_INVARIANTS 1u  /* after every load/merge verify keys strictly increase (slow, for tests) */
 #define XLOG_FLAG_PROFILE          2u  /* CUDA events around every kernel launch; read with xlog_profile_read */
+#define XLOG_FLAG_NO_TAG_MIRROR    4u  /* evaluate every recursive component by sort -> reduce-by-key -> merge */
 #define XLOG_FLAG_NO_RESIDENT_LOOP 8u  /* the host drives every round of a tag-mirror fixpoint (one control read per round) */
 #define XLOG_FLAG_NO_GRAPH        16u  /* resident rounds are launched one by one instead of as one graph with a WHILE node */
-#define XLOG_FLAG_NO_TAG_MIRROR    4u  /* evaluate every recursive component by sort -> reduce-by-key -> merge, never through a tag mirror */
+
+/* Evaluation routes of a recursive component (Algorithm 1).  All of them derive the same relation,
+ * bit for bit, and the same receipt counters (unique_candidates excepted, see xlog_receipt).
+ *  - Sorting route: join -> sort -> reduce-by-key -> merge-path difference, as in the paper's kernel table.
+ *  - Tag mirror (default where it applies: one MAXPLUS/MINPLUS head relation, every rule with at most one
+ *    atom over it and that atom scanned, packed key <= 30 bits, table fits the arena): the relation is a
+ *    direct-addressed table of one tag per possible key; candidates are applied with one atomic max/min.
+ *  - Resident rounds (tag mirror with <= 2^24 possible keys): the delta rounds run as one CUDA graph with a
+ *    conditional WHILE node and fixed-capacity buffers (Section "GPU-Native Symbolic Substrate": resident
+ *    conditional graph, no host reads inside the loop).  The buffers (about 36 bytes per possible key
+ *    plus 12 MB) and the instantiated graph stay allocated in the arena from the first such xlog_fixpoint
+ *    until the context is destroyed or the relation's key layout changes.  The first call also
+ *    creates a private stream that records the graph; nothing else ever runs on it. */
 
 /* ---- context --------------------------------------------------------------- */
 xlog_status xlog_ctx_create(const xlog_config* cfg, xlog_ctx** out);

@@ -155,10 +155,16 @@ __global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __rest
   if (i < n_outer) deg[i] = join_count_row<KO>(S, okeys, otags, i, rowinfo, err);
 }
 
+// Tile shape of the materialising kernel.  The tag-mirror sinks are bound by the latency of one random L2 sector per
+// candidate, so what counts is how many slot reads an SM keeps in flight: blocks per SM x items per thread, against the
+// registers (<= 36 for 7 blocks) and shared memory that takes.  Measured on the two large workloads (single-source
+// R-MAT 20 / 64-source R-MAT 22, ms per fixpoint): 8 items, 2048 rows, 4 blocks 0.75 / 51.2; 8, 1024, 6 blocks 0.71 / 42.2;
+// 8, 1024, 8 blocks (spills) 0.85 / 60.0; 4, 512, 8 blocks 0.65 / 46.3; 5, 640, 8 blocks 0.66 / 43.0; 6, 768, 7 blocks 0.68 / 41.4.
 constexpr int kExpBlock = 256;
-constexpr int kExpItems = 8;
+constexpr int kExpItems = 6;
 constexpr int kExpTile = kExpBlock * kExpItems;       // candidates per block
-constexpr int kExpRows = 2048;                        // outer rows staged in shared memory per tile
+constexpr int kExpRows = 768;                         // outer rows staged in shared memory per tile
+constexpr int kExpMirrorBlocksPerSM = 7;              // occupancy asked of the tag-mirror instantiations
 
 // Backward pass of a logsumexp / sum rule: instead of writing the candidate, look its head row up
 // and scatter the gradient to the two body rows (Section "End-to-end training": exact gradients
@@ -444,7 +450,7 @@ __device__ __forceinline__ void expand_tile(ExpSmem& sm, const JoinSpec& S, cons
 // staged in shared memory (their starts relative to the tile and their row records), so the per-
 // candidate work is a short binary search in shared memory plus the coalesced inner reads.
 template <typename KO, typename KH, int MODE, int SINK = kSinkWrite>
-__global__ void __launch_bounds__(kExpBlock) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
+__global__ void __launch_bounds__(kExpBlock, SINK == kSinkWrite ? 1 : kExpMirrorBlocksPerSM) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
                                                            const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo,
                                                            const uint2* __restrict__ tile_rows, uint64_t out_lo, uint64_t out_hi,
                                                            KH* __restrict__ ckeys,

@@ -174,7 +174,7 @@ __global__ void __launch_bounds__(kScanBlock) k_res_count_scan(JoinSpec S, const
 
 // persistent blocks: block b takes tiles b, b + gridDim.x, ...
 template <typename KO, int MODE, int SINK>
-__global__ void __launch_bounds__(kExpBlock) k_res_expand(JoinSpec S, const KO* __restrict__ okeys, const ResState* __restrict__ st,
+__global__ void __launch_bounds__(kExpBlock, kExpMirrorBlocksPerSM) k_res_expand(JoinSpec S, const KO* __restrict__ okeys, const ResState* __restrict__ st,
                                                           const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo,
                                                           const uint2* __restrict__ tile_rows, uint32_t* __restrict__ err, MirrorArgs mr) {
   __shared__ ExpSmem sm;
