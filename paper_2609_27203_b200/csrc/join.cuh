@@ -160,11 +160,15 @@ __global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __rest
 // registers (<= 36 for 7 blocks) and shared memory that takes.  Measured on the two large workloads (single-source
 // R-MAT 20 / 64-source R-MAT 22, ms per fixpoint): 8 items, 2048 rows, 4 blocks 0.75 / 51.2; 8, 1024, 6 blocks 0.71 / 42.2;
 // 8, 1024, 8 blocks (spills) 0.85 / 60.0; 4, 512, 8 blocks 0.65 / 46.3; 5, 640, 8 blocks 0.66 / 43.0; 6, 768, 7 blocks 0.68 / 41.4.
+// The kernel that writes candidates (streaming, HBM-bound) keeps the larger tile: 8 items, 2048 rows, 4 blocks per SM.
 constexpr int kExpBlock = 256;
-constexpr int kExpItems = 6;
-constexpr int kExpTile = kExpBlock * kExpItems;       // candidates per block
-constexpr int kExpRows = 768;                         // outer rows staged in shared memory per tile
 constexpr int kExpMirrorBlocksPerSM = 7;              // occupancy asked of the tag-mirror instantiations
+template <bool MIRROR> struct ExpShapeT {
+  static constexpr int items = MIRROR ? 6 : 8;        // candidates per thread
+  static constexpr int tile = kExpBlock * items;      // candidates per block
+  static constexpr int rows = MIRROR ? 768 : 2048;    // outer rows staged in shared memory per tile
+};
+constexpr int kExpTileWrite = ExpShapeT<false>::tile, kExpTileMirror = ExpShapeT<true>::tile;
 
 // Backward pass of a logsumexp / sum rule: instead of writing the candidate, look its head row up
 // and scatter the gradient to the two body rows (Section "End-to-end training": exact gradients
@@ -224,11 +228,11 @@ __device__ __forceinline__ void mirror_apply(const MirrorArgs& m, uint32_t key, 
 // (r_lo = last row with start <= tile begin, r_hi = last row with start < tile end).  Done for all
 // tiles at once so that the dependent binary-search loads of one tile overlap with those of the others.
 static __global__ void __launch_bounds__(256) k_expand_partition(const uint64_t* __restrict__ start, uint32_t n_outer, uint64_t out_lo,
-                                                                 uint64_t out_hi, uint32_t ntiles, uint2* __restrict__ tile_rows) {
+                                                                 uint64_t out_hi, uint32_t ntiles, uint32_t tile, uint2* __restrict__ tile_rows) {
   const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t >= ntiles) return;
-  const uint64_t t_lo = out_lo + (uint64_t)t * kExpTile;
-  const uint64_t t_hi = min(t_lo + kExpTile, out_hi);
+  const uint64_t t_lo = out_lo + (uint64_t)t * tile;
+  const uint64_t t_hi = min(t_lo + tile, out_hi);
   uint32_t r[2];
 #pragma unroll
   for (int k = 0; k < 2; ++k) {
@@ -243,20 +247,22 @@ static __global__ void __launch_bounds__(256) k_expand_partition(const uint64_t*
   tile_rows[t] = make_uint2(r[0], r[1]);
 }
 
-struct ExpSmem {
-  uint32_t sstart[kExpRows];
-  uint4 sinfo[kExpRows];
-  uint16_t srowidx[kExpTile];             // staged row of every candidate position of the tile
+template <typename SH> struct ExpSmem {
+  uint32_t sstart[SH::rows];
+  uint4 sinfo[SH::rows];
+  uint16_t srowidx[SH::tile];             // staged row of every candidate position of the tile
   uint32_t swarp[kExpBlock / 32];
 };
 
-// Candidates [t_lo, t_hi) (one tile, at most kExpTile of them), covered by outer rows tr.x .. tr.y.  Called by all
+// Candidates [t_lo, t_hi) (one tile, at most SH::tile of them), covered by outer rows tr.x .. tr.y.  Called by all
 // threads of a block; error bits go to `e` and new-tuple counts to `n_new` (the caller flushes both).
 template <typename KO, typename KH, int MODE, int SINK>
-__device__ __forceinline__ void expand_tile(ExpSmem& sm, const JoinSpec& S, const KO* __restrict__ okeys, uint32_t n_outer,
+__device__ __forceinline__ void expand_tile(ExpSmem<ExpShapeT<SINK != kSinkWrite>>& sm, const JoinSpec& S, const KO* __restrict__ okeys, uint32_t n_outer,
                                             const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo, const uint2 tr,
                                             const uint64_t t_lo, const uint64_t t_hi, const uint64_t out_lo, KH* __restrict__ ckeys,
                                             float* __restrict__ ctags, const BwdArgs& bw, const MirrorArgs& mr, uint32_t& e, uint32_t& n_new) {
+  typedef ExpShapeT<SINK != kSinkWrite> SH;
+  constexpr int kExpItems = SH::items, kExpTile = SH::tile, kExpRows = SH::rows;
   uint32_t* sstart = sm.sstart;
   uint4* sinfo = sm.sinfo;
   uint16_t* srowidx = sm.srowidx;
@@ -302,8 +308,7 @@ __device__ __forceinline__ void expand_tile(ExpSmem& sm, const JoinSpec& S, cons
   __syncthreads();
 
   if (MODE == kExpFast && staged) {
-    // lean loop of the common case: everything per row is in shared memory, everything per candidate is one
-    // (or a few) coalesced inner reads, one multiply-add and two coalesced writes; all indices are 32-bit
+    // lean loop of the common case: everything per row is in shared memory; all indices are 32-bit
     const uint32_t ntile = (uint32_t)(t_hi - t_lo);
     const uint32_t j0 = (uint32_t)(t_lo - first_start);              // candidates of the first row that precede the tile
     KH* __restrict__ kout = ckeys + (t_lo - out_lo);
@@ -313,9 +318,32 @@ __device__ __forceinline__ void expand_tile(ExpSmem& sm, const JoinSpec& S, cons
     const KH m0 = (KH)S.inner_mult[0];
     const int nin = S.has_inner ? S.inner_free : -1;                 // -1: one-atom rule
     const bool times = S.times != 0;
-    // three sweeps over the thread's items, so that the loads of one kind are all in flight together: (1) row record
-    // from shared memory, inner tag and columns from global memory; (2) for the mirror, the current slot values;
-    // (3) the stores, or the atomics of the few candidates that improve their slot
+    if (SINK == kSinkWrite) {
+      // everything per candidate is one (or a few) coalesced inner reads, one multiply-add and two coalesced writes
+#pragma unroll
+      for (int k = 0; k < kExpItems; ++k) {
+        const uint32_t q = threadIdx.x + k * kExpBlock;
+        if (q < ntile) {
+          const uint32_t li = srowidx[q];
+          const uint4 info = sinfo[li];
+          const uint32_t ir = info.x + (li ? q - sstart[li] : q + j0);
+          KH key = (KH)(((uint64_t)info.w << 32) | info.z);
+          float tag = __uint_as_float(info.y);
+          if (nin >= 0) {
+            const float it = itg[ir];
+            tag = times ? tag * it : tag + it;
+            if (nin >= 1) key += (KH)(uint32_t)ic0[ir] * m0;
+            for (int c = 1; c < nin; ++c) key += (KH)(uint32_t)S.inner_col[c][ir] * (KH)S.inner_mult[c];
+          }
+          kout[q] = key;
+          tout[q] = tag;
+        }
+      }
+      return;
+    }
+    // tag mirror: three sweeps over the thread's items, so that the loads of one kind are all in flight together:
+    // (1) row record from shared memory, inner tag and columns from global memory; (2) the current slot values;
+    // (3) the atomics of the few candidates that improve their slot
     KH key[kExpItems];
     float tag[kExpItems];
 #pragma unroll
@@ -336,28 +364,20 @@ __device__ __forceinline__ void expand_tile(ExpSmem& sm, const JoinSpec& S, cons
         }
       }
     }
-    if (SINK == kSinkWrite) {
+    int32_t cur[kExpItems];
 #pragma unroll
-      for (int k = 0; k < kExpItems; ++k) {
-        const uint32_t q = threadIdx.x + k * kExpBlock;
-        if (q < ntile) { kout[q] = key[k]; tout[q] = tag[k]; }
+    for (int k = 0; k < kExpItems; ++k) {
+      const uint32_t q = threadIdx.x + k * kExpBlock;
+      cur[k] = SINK == kSinkMin ? (int32_t)0x80000000 : 0x7fffffff;        // nothing improves on this
+      if (q < ntile) {
+        if ((uint32_t)key[k] > mr.key_max) atomicOr(mr.err, kErrHeadRange);
+        else cur[k] = XLOG_TABLE_LOAD(mr.table + (uint32_t)key[k]);
       }
-    } else {
-      int32_t cur[kExpItems];
+    }
 #pragma unroll
-      for (int k = 0; k < kExpItems; ++k) {
-        const uint32_t q = threadIdx.x + k * kExpBlock;
-        cur[k] = SINK == kSinkMin ? (int32_t)0x80000000 : 0x7fffffff;        // nothing improves on this
-        if (q < ntile) {
-          if ((uint32_t)key[k] > mr.key_max) atomicOr(mr.err, kErrHeadRange);
-          else cur[k] = XLOG_TABLE_LOAD(mr.table + (uint32_t)key[k]);
-        }
-      }
-#pragma unroll
-      for (int k = 0; k < kExpItems; ++k) {
-        const int32_t v = f2ord(tag[k]);
-        if (SINK == kSinkMin ? v < cur[k] : v > cur[k]) mirror_commit<SINK>(mr, (uint32_t)key[k], v, n_new);
-      }
+    for (int k = 0; k < kExpItems; ++k) {
+      const int32_t v = f2ord(tag[k]);
+      if (SINK == kSinkMin ? v < cur[k] : v > cur[k]) mirror_commit<SINK>(mr, (uint32_t)key[k], v, n_new);
     }
     return;
   }
@@ -445,19 +465,20 @@ __device__ __forceinline__ void expand_tile(ExpSmem& sm, const JoinSpec& S, cons
   }
 }
 
-// Block b produces candidates [out_lo + b*kExpTile, ...).  `start` is the exclusive scan of `deg`
+// Block b produces candidates [out_lo + b*tile, ...).  `start` is the exclusive scan of `deg`
 // (global candidate index of each outer row's first match).  The outer rows covering the tile are
 // staged in shared memory (their starts relative to the tile and their row records), so the per-
 // candidate work is a short binary search in shared memory plus the coalesced inner reads.
 template <typename KO, typename KH, int MODE, int SINK = kSinkWrite>
-__global__ void __launch_bounds__(kExpBlock, SINK == kSinkWrite ? 1 : kExpMirrorBlocksPerSM) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
+__global__ void __launch_bounds__(kExpBlock, SINK == kSinkWrite ? 5 : kExpMirrorBlocksPerSM) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
                                                            const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo,
                                                            const uint2* __restrict__ tile_rows, uint64_t out_lo, uint64_t out_hi,
                                                            KH* __restrict__ ckeys,
                                                            float* __restrict__ ctags, uint32_t* __restrict__ err, BwdArgs bw, MirrorArgs mr) {
-  __shared__ ExpSmem sm;
-  const uint64_t t_lo = out_lo + (uint64_t)blockIdx.x * kExpTile;
-  const uint64_t t_hi = min(t_lo + kExpTile, out_hi);
+  typedef ExpShapeT<SINK != kSinkWrite> SH;
+  __shared__ ExpSmem<SH> sm;
+  const uint64_t t_lo = out_lo + (uint64_t)blockIdx.x * SH::tile;
+  const uint64_t t_hi = min(t_lo + SH::tile, out_hi);
   if (t_lo >= t_hi) return;
   uint32_t e = 0, n_new = 0;
   expand_tile<KO, KH, MODE, SINK>(sm, S, okeys, n_outer, start, rowinfo, tile_rows[blockIdx.x], t_lo, t_hi, out_lo, ckeys, ctags, bw, mr, e, n_new);

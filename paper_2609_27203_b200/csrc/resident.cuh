@@ -141,7 +141,7 @@ __global__ void __launch_bounds__(kScanBlock) k_res_count_scan(JoinSpec S, const
         s_excl = excl;
         if (t == tiles - 1 && !timeout) {
           const uint64_t all = excl + total;
-          const uint64_t nt = (all + kExpTile - 1) / kExpTile;
+          const uint64_t nt = (all + kExpTileMirror - 1) / kExpTileMirror;
           st->total = all;
           if (nt > max_tiles) { st->status = kResOverflow; st->ntiles = 0; }
           else {
@@ -159,10 +159,10 @@ __global__ void __launch_bounds__(kScanBlock) k_res_count_scan(JoinSpec S, const
       if (row < n) {
         start[row] = run;
         if (x[i]) {
-          // expand tile u begins at position u * kExpTile and ends at (u + 1) * kExpTile - 1
+          // expand tile u begins at position u * kExpTileMirror and ends at (u + 1) * kExpTileMirror - 1
           const uint64_t end = run + x[i];                                       // one past the row's last position
-          for (uint64_t u = (run + kExpTile - 1) / kExpTile; u * kExpTile < end && u < max_tiles; ++u) tile_rows[u].x = row;
-          for (uint64_t u = (run + kExpTile) / kExpTile; u * kExpTile <= end && u <= max_tiles; ++u) tile_rows[u - 1].y = row;
+          for (uint64_t u = (run + kExpTileMirror - 1) / kExpTileMirror; u * kExpTileMirror < end && u < max_tiles; ++u) tile_rows[u].x = row;
+          for (uint64_t u = (run + kExpTileMirror) / kExpTileMirror; u * kExpTileMirror <= end && u <= max_tiles; ++u) tile_rows[u - 1].y = row;
         }
         run += x[i];
       }
@@ -177,15 +177,15 @@ template <typename KO, int MODE, int SINK>
 __global__ void __launch_bounds__(kExpBlock, kExpMirrorBlocksPerSM) k_res_expand(JoinSpec S, const KO* __restrict__ okeys, const ResState* __restrict__ st,
                                                           const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo,
                                                           const uint2* __restrict__ tile_rows, uint32_t* __restrict__ err, MirrorArgs mr) {
-  __shared__ ExpSmem sm;
+  __shared__ ExpSmem<ExpShapeT<true>> sm;
   if (st->status != kResOk) return;
   const uint32_t ntiles = st->ntiles, n = st->n_delta;
   const uint64_t total = st->total;
   const BwdArgs bw{};
   uint32_t e = 0, n_new = 0;
   for (uint32_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
-    const uint64_t t_lo = (uint64_t)t * kExpTile;
-    const uint64_t t_hi = min(t_lo + kExpTile, total);
+    const uint64_t t_lo = (uint64_t)t * kExpTileMirror;
+    const uint64_t t_hi = min(t_lo + kExpTileMirror, total);
     expand_tile<KO, uint32_t, MODE, SINK>(sm, S, okeys, n, start, rowinfo, tile_rows[t], t_lo, t_hi, 0, (uint32_t*)nullptr, (float*)nullptr, bw, mr, e,
                                           n_new);
     __syncthreads();

@@ -502,7 +502,8 @@ void count_variant(Ctx* c, const Variant& v, const Relation& H, Counted& q, int 
 // scatter, or (SINK != kSinkWrite) apply them to the head relation's tag mirror
 template <int MODE, int SINK>
 void launch_expand_mode(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, void* ckeys, float* ctags, const BwdArgs& bw, const MirrorArgs& mr) {
-  const unsigned blocks = (unsigned)((hi - lo + kExpTile - 1) / kExpTile);
+  constexpr uint32_t tile = SINK == kSinkWrite ? kExpTileWrite : kExpTileMirror;
+  const unsigned blocks = (unsigned)((hi - lo + tile - 1) / tile);
   const uint64_t* st = q.start.as<uint64_t>();
   const uint4* ri = q.rowinfo.as<uint4>();
   uint32_t* err = ctrl_u32(c, kSlotErr);
@@ -511,7 +512,7 @@ void launch_expand_mode(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, v
   DevBuf tile_rows(c, (size_t)blocks * 8);
   const int64_t bytes = c->note_bytes;
   c->note_bytes = 0;
-  XLOG_LAUNCH(c, k_expand_partition, (blocks + 255) / 256, 256, 0, st, q.outer.n, lo, hi, blocks, tile_rows.as<uint2>());
+  XLOG_LAUNCH(c, k_expand_partition, (blocks + 255) / 256, 256, 0, st, q.outer.n, lo, hi, blocks, tile, tile_rows.as<uint2>());
   const uint2* tr = tile_rows.as<uint2>();
   c->note_bytes = bytes;
   if (q.outer.key_bytes == 4 && ckb == 4)
@@ -999,7 +1000,7 @@ static_assert(sizeof(ResState) <= (kCtrlSlots - kSlotResState) * sizeof(uint64_t
 Resident* resident_for(Ctx* c, int h, int bits, uint64_t slots, uint32_t bm_quads, unsigned ch_tiles) {
   if ((c->flags & XLOG_FLAG_NO_RESIDENT_LOOP) || bits > kResidentMaxBits) { c->resident.erase(h); return nullptr; }
   uint32_t max_tiles = kResidentMaxTiles;
-  if (c->chunk_bytes) max_tiles = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(max_tiles, c->chunk_bytes / 16 / kExpTile));
+  if (c->chunk_bytes) max_tiles = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(max_tiles, c->chunk_bytes / 16 / kExpTileMirror));
   auto it = c->resident.find(h);
   if (it != c->resident.end() && it->second->slots == slots && it->second->max_tiles == max_tiles) return it->second.get();
   c->resident.erase(h);
