@@ -262,7 +262,7 @@ __device__ __forceinline__ void expand_tile(ExpSmem<ExpShapeT<SINK != kSinkWrite
                                             const uint64_t t_lo, const uint64_t t_hi, const uint64_t out_lo, KH* __restrict__ ckeys,
                                             float* __restrict__ ctags, const BwdArgs& bw, const MirrorArgs& mr, uint32_t& e, uint32_t& n_new) {
   typedef ExpShapeT<SINK != kSinkWrite> SH;
-  constexpr int kExpItems = SH::items, kExpTile = SH::tile, kExpRows = SH::rows;
+  constexpr int kExpItems = SH::items, kExpRows = SH::rows;
   uint32_t* sstart = sm.sstart;
   uint4* sinfo = sm.sinfo;
   uint16_t* srowidx = sm.srowidx;
@@ -339,8 +339,7 @@ __device__ __forceinline__ void expand_tile(ExpSmem<ExpShapeT<SINK != kSinkWrite
           tout[q] = tag;
         }
       }
-      return;
-    }
+    } else {
     // tag mirror: three sweeps over the thread's items, so that the loads of one kind are all in flight together:
     // (1) row record from shared memory, inner tag and columns from global memory; (2) the current slot values;
     // (3) the atomics of the few candidates that improve their slot
@@ -378,6 +377,7 @@ __device__ __forceinline__ void expand_tile(ExpSmem<ExpShapeT<SINK != kSinkWrite
     for (int k = 0; k < kExpItems; ++k) {
       const int32_t v = f2ord(tag[k]);
       if (SINK == kSinkMin ? v < cur[k] : v > cur[k]) mirror_commit<SINK>(mr, (uint32_t)key[k], v, n_new);
+    }
     }
     return;
   }

@@ -1186,20 +1186,8 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
   KeyTags delta_own;                       // host-driven rounds without persistent buffers keep their delta here
   const void* dk = nullptr; const float* dt = nullptr; uint32_t dn = 0;
   uint64_t total_new = 0;
-  bool resident_done = false;
-  for (int64_t round = 0;; ++round) {
-    if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
-    ++c->r_iterations;
-    std::vector<Variant> vs;
-    for (const RuleC* r : rs) {
-      if (round == 0) {
-        const int outer = seed_outer(comp, r);
-        vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
-      } else {
-        for (int j = 0; j < r->plan.n_atoms; ++j)
-          if (r->plan.atoms[j].rel == h && dn) vs.push_back(Variant{r, j, Source{dk, dt, dn, H.layout, H.key_bytes}});
-      }
-    }
+  // count -> scan -> one control read -> join into the table, for a list of rule variants; returns the candidate total
+  auto host_apply = [&](std::vector<Variant>& vs) -> uint64_t {
     if (vs.size() > 16) fail(XLOG_ERR_UNSUPPORTED, "too many rule variants for one head");
     std::vector<Counted> counted;
     counted.reserve(vs.size());
@@ -1222,7 +1210,55 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
       }
       q.start.reset(); q.rowinfo.reset();
     }
-    if (total == 0) break;
+    return total;
+  };
+  auto over_h = [&](const RuleC* r) {
+    for (int j = 0; j < r->plan.n_atoms; ++j) if (r->plan.atoms[j].rel == h) return true;
+    return false;
+  };
+
+  int64_t round = 0;
+  bool plain_rules_done = false;           // the rules without an atom over H have had their one evaluation
+  bool converged = false;
+  if (R) {
+    // Resident route.  Seed round, part one: rules without an atom over H are evaluated once, by the host (they scan whole
+    // relations of known size).  Part two and every later round run on the device: for the rules over H the seed round
+    // is a delta round whose delta is everything H holds now.
+    std::vector<Variant> plain;
+    for (const RuleC* r : rs)
+      if (!over_h(r)) { const int outer = seed_outer(comp, r); plain.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])}); }
+    host_apply(plain);
+    plain_rules_done = true;
+    if (n_start) {
+      XLOG_CUDA(cudaMemcpyAsync(R->dkeys.p, H.keys(), (size_t)n_start * 4, cudaMemcpyDeviceToDevice, c->stream));
+      XLOG_CUDA(cudaMemcpyAsync(R->dtags.p, H.tags(), (size_t)n_start * 4, cudaMemcpyDeviceToDevice, c->stream));
+    }
+    const ResState s = run_resident(c, *R, h, rs, is_max, mr, bm_quads, ch_tiles, n_start, c->max_iter, 0);
+    round = s.rounds;
+    c->r_iterations += s.rounds; c->r_candidates += (int64_t)s.candidates;
+    c->r_new += (int64_t)s.n_new; c->r_improved += (int64_t)s.n_improved;
+    total_new = s.new_seen;
+    dk = R->dkeys.p; dt = R->dtags.as<float>(); dn = s.n_delta;
+    if (s.status == kResCap) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
+    if (s.status == kResOk) converged = true;             // the delta ran empty
+    // kResOverflow: a round needs more expand tiles than planned; the host redoes that round and finishes the job
+  }
+  for (; !converged; ++round) {
+    if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
+    ++c->r_iterations;
+    std::vector<Variant> vs;
+    for (const RuleC* r : rs) {
+      if (round == 0) {
+        if (plain_rules_done && !over_h(r)) continue;
+        const int outer = seed_outer(comp, r);
+        vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
+      } else {
+        for (int j = 0; j < r->plan.n_atoms; ++j)
+          if (r->plan.atoms[j].rel == h && dn) vs.push_back(Variant{r, j, Source{dk, dt, dn, H.layout, H.key_bytes}});
+      }
+    }
+    const uint64_t total = host_apply(vs);
+    if (total == 0 && !(round == 0 && plain_rules_done)) break;
     launch_changed_count(c, reinterpret_cast<const uint32_t*>(bitmap), bm_quads * 4, ch_tiles, ch_sums);
     XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, ch_sums, (int64_t)ch_tiles, ctrl_u32(c, kSlotMirChanged));
     sync_ctrl(c);
@@ -1242,18 +1278,6 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
     c->note_bytes = (int64_t)bm_quads * 16 + (int64_t)changed * 12;
     launch_changed_emit(c, reinterpret_cast<uint32_t*>(bitmap), bm_quads * 4, ch_tiles, ch_sums, table, ek, et, nullptr);
     dk = ek; dt = et; dn = changed;
-    if (R && !resident_done) {
-      // hand the delta rounds to the device
-      const ResState s = run_resident(c, *R, h, rs, is_max, mr, bm_quads, ch_tiles, dn, c->max_iter - (round + 1), total_new);
-      resident_done = true;                  // after an overflow the host finishes the job
-      round += s.rounds;
-      c->r_iterations += s.rounds; c->r_candidates += (int64_t)s.candidates;
-      c->r_new += (int64_t)s.n_new; c->r_improved += (int64_t)s.n_improved;
-      total_new = s.new_seen;
-      dn = s.n_delta;
-      if (s.status == kResCap) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
-      if (s.status == kResOk) break;         // the delta ran empty
-    }
   }
   // the relation in sorted form: every occupied slot, in slot order
   const uint64_t n_out = (uint64_t)n_start + total_new;
