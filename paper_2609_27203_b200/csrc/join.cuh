@@ -45,6 +45,14 @@ struct JoinSpec {
   int64_t neg_domain;
   const uint32_t* neg_off;                                    // offsets over the negated relation's first column
   const int32_t* neg_col1;                                    // its second column (sorted inside each first-column run)
+  // simple shape (a fast shape whose scanned atom binds each column to a constant or to a distinct bare variable, without
+  // dictionaries, and whose head columns each take a constant plus at most one of those variables): the per-row work
+  // is a handful of shifts and masks on the packed key instead of the general binding / affine evaluation
+  int simple;
+  uint64_t s_const_mask, s_const_val;                         // (key & mask) == val: every constant column matches
+  int s_probe_shift; uint32_t s_probe_mask;                   // column that binds the probe variable
+  int s_src_shift[kMaxArity]; uint32_t s_src_mask[kMaxArity]; // per head column: the outer column it copies (mask 0: none)
+  uint32_t s_c0[kMaxArity];
   // fast shape: head key = row part + sum_j inner_col[j] * inner_mult[j]
   int fast;
   int32_t head_coef_outer[kMaxArity][kMaxVars];               // head_coef restricted to variables the outer atom binds
@@ -68,8 +76,9 @@ __device__ __forceinline__ bool bind_outer(const JoinSpec& S, KO key, int64_t* v
       if (a.kind == 0) ok = ok && val == a.add;
       else {
         const int64_t d = val - a.add;
-        const int64_t q = d / a.mul;
-        const bool divides = q * a.mul == d;
+        int64_t q = d;
+        bool divides = true;
+        if (a.mul != 1) { q = d / a.mul; divides = q * a.mul == d; }       // the 64-bit division is rare: keep it off the common path
 #pragma unroll
         for (int v = 0; v < kMaxVars; ++v)
           if (v == a.var) {
@@ -93,7 +102,31 @@ __device__ __forceinline__ uint32_t join_count_row(const JoinSpec& S, const KO* 
   int64_t var[kMaxVars];
   uint32_t d = 0, lo = 0;
   uint64_t rowkey = 0;
-  if (bind_outer<KO>(S, okeys[i], var)) {
+  if (S.simple) {
+    const uint64_t k = (uint64_t)okeys[i];
+    if ((k & S.s_const_mask) == S.s_const_val) {
+      d = 1;
+      if (S.has_inner) {
+        const int64_t pv = (int64_t)((uint32_t)(k >> S.s_probe_shift) & S.s_probe_mask) * S.probe_mul + S.probe_add;
+        d = 0;
+        if (pv >= 0 && pv < S.inner_domain) {
+          lo = S.inner_off[pv];
+          d = S.inner_off[pv + 1] - lo;
+        }
+      }
+      if (d) {
+        uint32_t e = 0;
+#pragma unroll
+        for (int c = 0; c < kMaxArity; ++c)
+          if (c < S.head.arity) {
+            uint64_t h = (uint64_t)S.s_c0[c] + ((uint32_t)(k >> S.s_src_shift[c]) & S.s_src_mask[c]);
+            if (h > (uint64_t)S.head.mask[c]) { e |= kErrHeadRange; h = 0; }
+            rowkey |= h << S.head.shift[c];
+          }
+        if (e) atomicOr(err, e);
+      }
+    }
+  } else if (bind_outer<KO>(S, okeys[i], var)) {
     if (S.neg_prefix) {
       int64_t val[2] = {0, 0};
 #pragma unroll

@@ -456,6 +456,38 @@ JoinSpec make_spec(Ctx* c, const Variant& v, const Relation& H) {
     }
   }
   S.fast = fast ? 1 : 0;
+  // simple shape: see JoinSpec
+  bool simple = fast && S.neg_prefix == 0;
+  int col_of_var[kMaxVars];
+  for (int k = 0; k < kMaxVars; ++k) col_of_var[k] = -1;
+  for (int i = 0; i < RA.arity && simple; ++i) {
+    if (S.outer_decode[i]) simple = false;
+    else if (A.args[i].kind == XLOG_ARG_VAR) {
+      if (!is_plain_var(A.args[i]) || col_of_var[A.args[i].var] >= 0) simple = false; else col_of_var[A.args[i].var] = i;
+    } else {
+      const int64_t cv = A.args[i].add;
+      if (cv < 0 || cv > (int64_t)S.outer.mask[i]) simple = false;          // can never match: leave it to the general path
+      else { S.s_const_mask |= (uint64_t)S.outer.mask[i] << S.outer.shift[i]; S.s_const_val |= (uint64_t)cv << S.outer.shift[i]; }
+    }
+  }
+  if (simple && S.has_inner) {
+    const int pc = col_of_var[S.probe_var];
+    if (pc < 0) simple = false; else { S.s_probe_shift = S.outer.shift[pc]; S.s_probe_mask = S.outer.mask[pc]; }
+  }
+  for (int hc = 0; hc < p.n_head_cols && simple; ++hc) {
+    int src = -1;
+    if (S.head_encode[hc] || p.head[hc].c0 < 0 || p.head[hc].c0 > 0x7fffffff) simple = false;
+    for (int k = 0; k < kMaxVars && simple; ++k) {
+      const int cf = S.head_coef_outer[hc][k];
+      if (cf == 0) continue;
+      if (cf != 1 || src >= 0 || col_of_var[k] < 0) simple = false; else src = col_of_var[k];
+    }
+    S.s_c0[hc] = (uint32_t)p.head[hc].c0;
+    S.s_src_shift[hc] = src >= 0 ? S.outer.shift[src] : 0;
+    S.s_src_mask[hc] = src >= 0 ? S.outer.mask[src] : 0u;
+  }
+  if (p.emit_count_column) simple = false;
+  S.simple = simple ? 1 : 0;
   return S;
 }
 
