@@ -13,18 +13,25 @@ namespace xlog {
 struct ColPtrs { const int32_t* c[kMaxArity]; };
 struct ColPtrsMut { int32_t* c[kMaxArity]; };
 
+// Validation, column maxima and an order test in one read of the input: *unordered is raised when some row is not
+// lexicographically greater than the row before it (rows that arrive strictly increasing need no sort and hold no duplicates).
 static __global__ void __launch_bounds__(256) k_col_stats(ColPtrs cols, const float* __restrict__ tags, int64_t n, int arity, int sr,
-                                                   int32_t* __restrict__ col_max /*[arity]*/, uint32_t* __restrict__ err) {
+                                                   int32_t* __restrict__ col_max /*[arity]*/, uint32_t* __restrict__ err,
+                                                   uint32_t* __restrict__ unordered) {
   int32_t mx[kMaxArity] = {0, 0, 0, 0};
   uint32_t e = 0;
+  bool out_of_order = false;
   for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+    int cmp = 0;                                        // sign of (row i - row i-1), decided by the first differing column
 #pragma unroll
     for (int c = 0; c < kMaxArity; ++c)
       if (c < arity) {
         const int32_t v = cols.c[c][i];
         if (v < 0) e |= kErrNegativeKey;
         mx[c] = max(mx[c], v);
+        if (i > 0 && cmp == 0) { const int32_t p = cols.c[c][i - 1]; cmp = v > p ? 1 : v < p ? -1 : 0; }
       }
+    if (i > 0 && cmp <= 0) out_of_order = true;
     if (tags) {
       const float t = tags[i];
       const bool zero = sr == 0 || sr == 2 ? t == -INFINITY : sr == 1 ? t == INFINITY : false;
@@ -42,6 +49,7 @@ static __global__ void __launch_bounds__(256) k_col_stats(ColPtrs cols, const fl
     for (int c = 0; c < arity; ++c) atomicMax(&col_max[c], mx[c]);
     if (e) atomicOr(err, e);
   }
+  if (__any_sync(0xffffffffu, out_of_order) && lane_id() == 0) atomicOr(unordered, 1u);
 }
 
 template <typename K>

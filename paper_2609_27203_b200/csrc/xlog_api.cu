@@ -145,8 +145,9 @@ void load_relation(Ctx* c, Relation& R, const int32_t* const* cols, const float*
   zero_ctrl(c, kSlotErr);
   zero_ctrl(c, kSlotA, 4);
   XLOG_LAUNCH(c, k_col_stats, grid_for(n, 256, kSMs * 8), 256, 0, in, dtags, n, R.arity, R.sr,
-              reinterpret_cast<int32_t*>(c->d_ctrl + kSlotA), ctrl_u32(c, kSlotErr));
+              reinterpret_cast<int32_t*>(c->d_ctrl + kSlotA), ctrl_u32(c, kSlotErr), ctrl_u32(c, kSlotC));
   sync_ctrl(c);
+  const bool in_order = (uint32_t)c->h_ctrl[kSlotC] == 0;     // rows arrived strictly increasing: nothing to sort or combine
   const int32_t* mx = reinterpret_cast<const int32_t*>(c->h_ctrl + kSlotA);
   for (int i = 0; i < R.arity; ++i) R.col_max[i] = R.fact_max[i] = R.val_max[i] = mx[i];
   zero_ctrl(c, kSlotA, 4);
@@ -155,7 +156,14 @@ void load_relation(Ctx* c, Relation& R, const int32_t* const* cols, const float*
   R.key_bytes = R.layout.total_bits <= 32 ? 4 : 8;
 
   // pack -> sort -> combine duplicates
-  DISPATCH_K(R.key_bytes, {
+  if (in_order) {
+    DISPATCH_K(R.key_bytes, {
+      R.fact_keys = DevBuf(c, (size_t)n * sizeof(K));
+      R.fact_tags = DevBuf(c, (size_t)n * 4);
+      XLOG_LAUNCH(c, (k_pack<K>), grid_for(n, 256), 256, 0, in, dtags, n, R.layout, DictSet{}, one_of(R.sr), R.fact_keys.as<K>(), R.fact_tags.as<float>());
+      R.n_facts = R.n = (uint32_t)n;
+    });
+  } else DISPATCH_K(R.key_bytes, {
     DevBuf k0(c, (size_t)n * sizeof(K)), t0(c, (size_t)n * 4), k1(c, (size_t)n * sizeof(K)), t1(c, (size_t)n * 4);
     XLOG_LAUNCH(c, (k_pack<K>), grid_for(n, 256), 256, 0, in, dtags, n, R.layout, DictSet{}, one_of(R.sr), k0.as<K>(), t0.as<float>());
     for (int i = 0; i < kMaxArity; ++i) stage[i].reset();

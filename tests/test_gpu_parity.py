@@ -96,6 +96,27 @@ def test_load_sorts_and_combines_duplicates(n, arity, sr):
     ctx.close()
 
 
+def test_rows_that_arrive_in_order_take_the_short_load_path():
+    # strictly increasing rows are stored as they come (no sort, no duplicate pass); one swapped pair or one repeated row
+    # must send the load down the sorting path again.  All three must match the oracle.
+    from paper_2609_27203_b200 import xlog
+    n = 200_000
+    a = np.sort(synth.randint(5, 1, 0, n, 5000)).astype(np.int32)
+    b = np.arange(n, dtype=np.int32)                     # makes every row distinct and the pairs increasing
+    t = synth.normal(5, 2, n).astype(np.float32)
+    swapped = (a.copy(), b.copy()); swapped[1][[1000, 1001]] = swapped[1][[1001, 1000]]
+    repeated = (a.copy(), b.copy()); repeated[0][777] = repeated[0][776]; repeated[1][777] = repeated[1][776]
+    for cols in [(a, b), swapped, repeated]:
+        ctx = xlog.Context(arena_bytes=1 << 27, flags=xlog.FLAG_CHECK_INVARIANTS)
+        r = ctx.relation(2, "minplus")
+        ctx.load(r, list(cols), t)
+        o = oracle.Oracle()
+        ro = o.relation(2, "minplus")
+        o.load(ro, list(cols), t)
+        assert H.compare_relations(ctx.read(r), o.read(ro), what="in-order load")["bit_unequal"] == 0
+        ctx.close()
+
+
 def test_empty_and_single_relations():
     from paper_2609_27203_b200 import xlog
     ctx = xlog.Context(arena_bytes=1 << 24)
