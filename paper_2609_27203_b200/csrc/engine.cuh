@@ -128,7 +128,7 @@ struct RuleC {
 struct Resident {
   uint64_t slots = 0;
   uint32_t max_tiles = 0;
-  DevBuf table, bitmap, ch_sums, ch_counts, dkeys, dtags, rowinfo, start, tile_rows, scan_status, tickets;
+  DevBuf table, bitmap, present, ch_sums, ch_counts, dkeys, dtags, rowinfo, start, tile_rows, scan_status, tickets;
   uint32_t scan_tiles_cap = 0;
   cudaGraph_t graph = nullptr;
   cudaGraphExec_t exec = nullptr;

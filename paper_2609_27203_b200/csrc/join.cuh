@@ -222,13 +222,16 @@ enum { kExpFast = 0, kExpGeneric = 1, kExpBackward = 2 };
 // Where a candidate goes.  kSinkWrite: into the candidate arrays (to be sorted and reduced).  kSinkMin / kSinkMax:
 // straight into the head relation's tag mirror, a table with one order-mapped tag per possible head key
 // (max / min are idempotent and order-independent, so "oplus into the slot" is one atomic and needs no sort).
-// A candidate that improves its slot sets the key's bit in `changed`; the thread that replaces the empty marker
-// counts a new tuple.  The slot is read first because most candidates of a fixpoint round do not improve anything.
+// A candidate that is better than what its slot holds issues the atomic and sets the key's bit in `changed`, both as
+// fire-and-forget reductions: no thread ever waits for an atomic's result.  (If another candidate lowers the slot
+// between the read and the atomic, the key has changed in this round all the same, so the bit is right either way.)
+// The slot is read first because most candidates of a fixpoint round do not improve anything.  Which of the changed
+// keys are new is settled when the bitmap is compacted, against a bitmap of the keys the relation already holds.
 enum { kSinkWrite = 0, kSinkMin = 1, kSinkMax = 2 };
 struct MirrorArgs {
   int32_t* table;               // 2^key_bits order-mapped tags; kMirrorEmptyMin / kMirrorEmptyMax where no tuple is
   uint32_t* changed;            // one bit per key
-  unsigned long long* n_new;    // running count of keys that left the empty state
+  unsigned long long* n_new;    // running count of keys that entered the relation (kept by the compaction kernels)
   uint32_t key_max;             // last valid key; anything above raises the head-range error instead of being stored
   uint32_t* err;
 };
@@ -242,19 +245,16 @@ constexpr int32_t kMirrorEmptyMax = (int32_t)0x80000000;
 #endif
 
 template <int SINK>
-__device__ __forceinline__ void mirror_commit(const MirrorArgs& m, uint32_t key, int32_t v, uint32_t& n_new) {
-  const int32_t old = SINK == kSinkMin ? atomicMin(m.table + key, v) : atomicMax(m.table + key, v);
-  if (SINK == kSinkMin ? v < old : v > old) {
-    atomicOr(m.changed + (key >> 5), 1u << (key & 31));
-    if (old == (SINK == kSinkMin ? kMirrorEmptyMin : kMirrorEmptyMax)) ++n_new;
-  }
+__device__ __forceinline__ void mirror_commit(const MirrorArgs& m, uint32_t key, int32_t v) {
+  if (SINK == kSinkMin) atomicMin(m.table + key, v); else atomicMax(m.table + key, v);
+  atomicOr(m.changed + (key >> 5), 1u << (key & 31));
 }
 template <int SINK>
-__device__ __forceinline__ void mirror_apply(const MirrorArgs& m, uint32_t key, float tag, uint32_t& n_new) {
+__device__ __forceinline__ void mirror_apply(const MirrorArgs& m, uint32_t key, float tag) {
   const int32_t v = f2ord(tag);
   if (key > m.key_max) { atomicOr(m.err, kErrHeadRange); return; }
   const int32_t cur = __ldcg(m.table + key);
-  if (SINK == kSinkMin ? v < cur : v > cur) mirror_commit<SINK>(m, key, v, n_new);
+  if (SINK == kSinkMin ? v < cur : v > cur) mirror_commit<SINK>(m, key, v);
 }
 
 // One thread per tile: the first and last outer row that contribute candidates to the tile
@@ -288,12 +288,12 @@ template <typename SH> struct ExpSmem {
 };
 
 // Candidates [t_lo, t_hi) (one tile, at most SH::tile of them), covered by outer rows tr.x .. tr.y.  Called by all
-// threads of a block; error bits go to `e` and new-tuple counts to `n_new` (the caller flushes both).
+// threads of a block; error bits go to `e` (the caller flushes them).
 template <typename KO, typename KH, int MODE, int SINK>
 __device__ __forceinline__ void expand_tile(ExpSmem<ExpShapeT<SINK != kSinkWrite>>& sm, const JoinSpec& S, const KO* __restrict__ okeys, uint32_t n_outer,
                                             const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo, const uint2 tr,
                                             const uint64_t t_lo, const uint64_t t_hi, const uint64_t out_lo, KH* __restrict__ ckeys,
-                                            float* __restrict__ ctags, const BwdArgs& bw, const MirrorArgs& mr, uint32_t& e, uint32_t& n_new) {
+                                            float* __restrict__ ctags, const BwdArgs& bw, const MirrorArgs& mr, uint32_t& e) {
   typedef ExpShapeT<SINK != kSinkWrite> SH;
   constexpr int kExpItems = SH::items, kExpRows = SH::rows;
   uint32_t* sstart = sm.sstart;
@@ -409,7 +409,7 @@ __device__ __forceinline__ void expand_tile(ExpSmem<ExpShapeT<SINK != kSinkWrite
 #pragma unroll
     for (int k = 0; k < kExpItems; ++k) {
       const int32_t v = f2ord(tag[k]);
-      if (SINK == kSinkMin ? v < cur[k] : v > cur[k]) mirror_commit<SINK>(mr, (uint32_t)key[k], v, n_new);
+      if (SINK == kSinkMin ? v < cur[k] : v > cur[k]) mirror_commit<SINK>(mr, (uint32_t)key[k], v);
     }
     }
     return;
@@ -446,7 +446,7 @@ __device__ __forceinline__ void expand_tile(ExpSmem<ExpShapeT<SINK != kSinkWrite
       for (int c = 0; c < kMaxArity - 1; ++c)
         if (c < S.inner_free) key += (KH)(uint32_t)S.inner_col[c][ir] * (KH)S.inner_mult[c];
       if (SINK == kSinkWrite) { ckeys[q + (t_lo - out_lo)] = key; ctags[q + (t_lo - out_lo)] = tag; }
-      else mirror_apply<SINK>(mr, (uint32_t)key, tag, n_new);
+      else mirror_apply<SINK>(mr, (uint32_t)key, tag);
       continue;
     }
     int64_t var[kMaxVars];
@@ -476,7 +476,7 @@ __device__ __forceinline__ void expand_tile(ExpSmem<ExpShapeT<SINK != kSinkWrite
       }
     if (MODE != kExpBackward) {
       if (SINK == kSinkWrite) { ckeys[p - out_lo] = key; ctags[p - out_lo] = tag; }
-      else if (!e) mirror_apply<SINK>(mr, (uint32_t)key, tag, n_new);
+      else if (!e) mirror_apply<SINK>(mr, (uint32_t)key, tag);
     } else {
       // head row of this binding: lower bound of the key among the stored head keys
       const KH* hk = reinterpret_cast<const KH*>(bw.head_keys);
@@ -513,13 +513,9 @@ __global__ void __launch_bounds__(kExpBlock, SINK == kSinkWrite ? 5 : kExpMirror
   const uint64_t t_lo = out_lo + (uint64_t)blockIdx.x * SH::tile;
   const uint64_t t_hi = min(t_lo + SH::tile, out_hi);
   if (t_lo >= t_hi) return;
-  uint32_t e = 0, n_new = 0;
-  expand_tile<KO, KH, MODE, SINK>(sm, S, okeys, n_outer, start, rowinfo, tile_rows[blockIdx.x], t_lo, t_hi, out_lo, ckeys, ctags, bw, mr, e, n_new);
+  uint32_t e = 0;
+  expand_tile<KO, KH, MODE, SINK>(sm, S, okeys, n_outer, start, rowinfo, tile_rows[blockIdx.x], t_lo, t_hi, out_lo, ckeys, ctags, bw, mr, e);
   if (e) atomicOr(err, e);
-  if (SINK != kSinkWrite) {
-    n_new = __reduce_add_sync(0xffffffffu, n_new);
-    if (lane_id() == 0 && n_new) atomicAdd(mr.n_new, (unsigned long long)n_new);
-  }
 }
 
 }  // namespace xlog

@@ -22,27 +22,42 @@ constexpr int kMirSlotsPerTile = kMirBlock * 16;       // table slots per tile (
 
 template <typename K>
 __global__ void __launch_bounds__(256) k_mirror_scatter(const K* __restrict__ keys, const float* __restrict__ tags, uint32_t n,
-                                                        int32_t* __restrict__ table) {
+                                                        int32_t* __restrict__ table, uint32_t* __restrict__ present) {
   const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) table[keys[i]] = f2ord(tags[i]);
+  if (i < n) {
+    const uint32_t key = (uint32_t)keys[i];
+    table[key] = f2ord(tags[i]);
+    atomicOr(present + (key >> 5), 1u << (key & 31));
+  }
 }
 
 // The changed bitmap is handled in tiles of SW * 256 words (SW "sweeps" of one word per thread).  Small domains take
 // SW = 1 so that there are enough tiles to occupy the GPU; large ones SW = 4 to keep the list of tile counts short.
 // nwords is the bitmap's (padded) length.
+// Also settles which changed keys are new: those whose bit in `present` (the keys the relation holds) was clear; the
+// bits are set here and the count of new keys is added to *new_total.
 template <int SW>
-__global__ void __launch_bounds__(kMirBlock) k_mirror_changed_count(const uint32_t* __restrict__ words, uint32_t nwords,
-                                                                    uint32_t* __restrict__ tile_sums) {
+__global__ void __launch_bounds__(kMirBlock) k_mirror_changed_count(const uint32_t* __restrict__ words, uint32_t* __restrict__ present,
+                                                                    uint32_t nwords, uint32_t* __restrict__ tile_sums,
+                                                                    unsigned long long* __restrict__ new_total) {
   __shared__ uint32_t sh[kMirBlock / 32 + 1];
-  uint32_t s = 0;
+  uint32_t s = 0, fresh = 0;
 #pragma unroll
   for (int j = 0; j < SW; ++j) {
     const uint32_t wi = (blockIdx.x * SW + j) * kMirBlock + threadIdx.x;
-    if (wi < nwords) s += __popc(words[wi]);
+    const uint32_t w = wi < nwords ? words[wi] : 0u;
+    s += __popc(w);
+    if (w) {
+      const uint32_t had = present[wi];
+      fresh += __popc(w & ~had);
+      if (w & ~had) present[wi] = had | w;
+    }
   }
   uint32_t total;
   block_scan_excl<kMirBlock, uint32_t>(s, sh, total);
   if (threadIdx.x == 0) tile_sums[blockIdx.x] = total;
+  fresh = __reduce_add_sync(0xffffffffu, fresh);
+  if (lane_id() == 0 && fresh) atomicAdd(new_total, (unsigned long long)fresh);
 }
 
 // One block per tile.  In a sweep every thread expands the set bits of one word into a key list in shared memory

@@ -182,17 +182,14 @@ __global__ void __launch_bounds__(kExpBlock, kExpMirrorBlocksPerSM) k_res_expand
   const uint32_t ntiles = st->ntiles, n = st->n_delta;
   const uint64_t total = st->total;
   const BwdArgs bw{};
-  uint32_t e = 0, n_new = 0;
+  uint32_t e = 0;
   for (uint32_t t = blockIdx.x; t < ntiles; t += gridDim.x) {
     const uint64_t t_lo = (uint64_t)t * kExpTileMirror;
     const uint64_t t_hi = min(t_lo + kExpTileMirror, total);
-    expand_tile<KO, uint32_t, MODE, SINK>(sm, S, okeys, n, start, rowinfo, tile_rows[t], t_lo, t_hi, 0, (uint32_t*)nullptr, (float*)nullptr, bw, mr, e,
-                                          n_new);
+    expand_tile<KO, uint32_t, MODE, SINK>(sm, S, okeys, n, start, rowinfo, tile_rows[t], t_lo, t_hi, 0, (uint32_t*)nullptr, (float*)nullptr, bw, mr, e);
     __syncthreads();
   }
   if (e) atomicOr(err, e);
-  n_new = __reduce_add_sync(0xffffffffu, n_new);
-  if (lane_id() == 0 && n_new) atomicAdd(mr.n_new, (unsigned long long)n_new);
 }
 
 // Last kernel of a round: compact the changed bitmap into the next delta and close the round.  Inside the resident
@@ -203,7 +200,8 @@ __global__ void __launch_bounds__(kExpBlock, kExpMirrorBlocksPerSM) k_res_expand
 // condition (ignored when use_handle == 0: the host drives).
 // ctr[0] = rows reserved so far, ctr[1] = blocks done; both are left at zero.
 template <int SW>
-__global__ void __launch_bounds__(kMirBlock) k_res_emit(uint32_t* __restrict__ words, uint32_t nwords, const int32_t* __restrict__ table,
+__global__ void __launch_bounds__(kMirBlock) k_res_emit(uint32_t* __restrict__ words, uint32_t* __restrict__ present, uint32_t nwords,
+                                                        unsigned long long* __restrict__ new_total, const int32_t* __restrict__ table,
                                                         uint32_t* __restrict__ keys, float* __restrict__ tags, ResState* __restrict__ st,
                                                         ResScratch sc, uint32_t n_variants, const unsigned long long* __restrict__ new_counter,
                                                         uint32_t* __restrict__ ctr, cudaGraphConditionalHandle handle, int use_handle) {
@@ -213,16 +211,23 @@ __global__ void __launch_bounds__(kMirBlock) k_res_emit(uint32_t* __restrict__ w
   const bool live = st->status == kResOk;                // an abandoned round keeps its bitmap and its delta
   if (live) {
     uint32_t w[SW];
-    uint32_t cnt = 0;
+    uint32_t cnt = 0, fresh = 0;
 #pragma unroll
     for (int j = 0; j < SW; ++j) {
       const uint32_t wi = (blockIdx.x * SW + j) * kMirBlock + threadIdx.x;
       w[j] = wi < nwords ? words[wi] : 0u;
       cnt += __popc(w[j]);
+      if (w[j]) {                                        // changed keys the relation did not hold yet are new tuples
+        const uint32_t had = present[wi];
+        fresh += __popc(w[j] & ~had);
+        if (w[j] & ~had) present[wi] = had | w[j];
+      }
     }
     uint32_t tile_total;
     block_scan_excl<kMirBlock, uint32_t>(cnt, sh, tile_total);
     if (tile_total) {                                    // uniform across the block
+      fresh = __reduce_add_sync(0xffffffffu, fresh);
+      if (lane_id() == 0 && fresh) atomicAdd(new_total, (unsigned long long)fresh);
       if (threadIdx.x == 0) s_base = atomicAdd(&ctr[0], tile_total);
       __syncthreads();
       uint32_t out = s_base;

@@ -1024,7 +1024,7 @@ bool mirror_applies(Ctx* c, const std::vector<int>& comp, const std::vector<cons
     if (in == 1 && r->kind != 2 && pos != 0) return false;
     if (in == 0 && r->kind == 2 && !r->shape[0].ok && !r->shape[1].ok) return false;
   }
-  const uint64_t need = ((uint64_t)4 << H.layout.total_bits) + ((uint64_t)1 << H.layout.total_bits) / 8 + (1u << 20);
+  const uint64_t need = ((uint64_t)4 << H.layout.total_bits) + ((uint64_t)1 << H.layout.total_bits) / 4 + (1u << 20);
   return need <= c->arena.largest_free() / 2;
 }
 
@@ -1045,12 +1045,13 @@ Resident* resident_for(Ctx* c, int h, int bits, uint64_t slots, uint32_t bm_quad
   if (it != c->resident.end() && it->second->slots == slots && it->second->max_tiles == max_tiles) return it->second.get();
   c->resident.erase(h);
   const uint64_t dom = (uint64_t)1 << bits;
-  const uint64_t need = slots * 4 + (uint64_t)bm_quads * 16 + dom * 32 + (uint64_t)max_tiles * 8 + (4u << 20);
+  const uint64_t need = slots * 4 + (uint64_t)bm_quads * 32 + dom * 32 + (uint64_t)max_tiles * 8 + (4u << 20);
   if (need > c->arena.largest_free() / 3) return nullptr;
   std::unique_ptr<Resident> R(new Resident());
   R->slots = slots; R->max_tiles = max_tiles;
   R->table = DevBuf(c, slots * 4);
   R->bitmap = DevBuf(c, (size_t)bm_quads * 16);
+  R->present = DevBuf(c, (size_t)bm_quads * 16);
   R->ch_sums = DevBuf(c, (size_t)ch_tiles * 4);
   R->dkeys = DevBuf(c, dom * 4); R->dtags = DevBuf(c, dom * 4);
   R->rowinfo = DevBuf(c, dom * 16); R->start = DevBuf(c, dom * 8);
@@ -1067,9 +1068,9 @@ Resident* resident_for(Ctx* c, int h, int bits, uint64_t slots, uint32_t bm_quad
 // blocks), four sweeps above that
 int mirror_sweeps(uint32_t nwords) { return nwords <= (1u << 17) ? 1 : 4; }
 unsigned mirror_tiles(uint32_t nwords) { const uint32_t per = kMirBlock * mirror_sweeps(nwords); return (nwords + per - 1) / per; }
-void launch_changed_count(Ctx* c, const uint32_t* words, uint32_t nwords, unsigned tiles, uint32_t* sums) {
-  if (mirror_sweeps(nwords) == 1) XLOG_LAUNCH(c, (k_mirror_changed_count<1>), tiles, kMirBlock, 0, words, nwords, sums);
-  else XLOG_LAUNCH(c, (k_mirror_changed_count<4>), tiles, kMirBlock, 0, words, nwords, sums);
+void launch_changed_count(Ctx* c, const uint32_t* words, uint32_t* present, uint32_t nwords, unsigned tiles, uint32_t* sums, unsigned long long* new_total) {
+  if (mirror_sweeps(nwords) == 1) XLOG_LAUNCH(c, (k_mirror_changed_count<1>), tiles, kMirBlock, 0, words, present, nwords, sums, new_total);
+  else XLOG_LAUNCH(c, (k_mirror_changed_count<4>), tiles, kMirBlock, 0, words, present, nwords, sums, new_total);
 }
 void launch_changed_emit(Ctx* c, uint32_t* words, uint32_t nwords, unsigned tiles, const uint32_t* base, const int32_t* table, uint32_t* keys,
                          float* tags, const uint32_t* skip) {
@@ -1103,7 +1104,8 @@ void resident_body(Ctx* c, Resident& R, const std::vector<JoinSpec>& specs, bool
   }
   uint32_t* ctr = sc.tickets + kResMaxVariants;
 #define XLOG_RES_EMIT(SW)                                                                                                                  \
-  XLOG_LAUNCH(c, (k_res_emit<SW>), ch_tiles, kMirBlock, 0, R.bitmap.as<uint32_t>(), bm_quads * 4, (const int32_t*)R.table.as<int32_t>(),   \
+  XLOG_LAUNCH(c, (k_res_emit<SW>), ch_tiles, kMirBlock, 0, R.bitmap.as<uint32_t>(), R.present.as<uint32_t>(), bm_quads * 4, mr.n_new,        \
+              (const int32_t*)R.table.as<int32_t>(),                                                                                        \
               R.dkeys.as<uint32_t>(), R.dtags.as<float>(), st, sc, (uint32_t)specs.size(), (const unsigned long long*)mr.n_new, ctr, handle, use_handle)
   if (mirror_sweeps(bm_quads * 4) == 1) XLOG_RES_EMIT(1); else XLOG_RES_EMIT(4);
 #undef XLOG_RES_EMIT
@@ -1136,7 +1138,7 @@ ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*
   if (use_graph) {
     std::vector<char> sig;
     for (const JoinSpec& S : specs) sig_add(sig, S);
-    sig_add(sig, mr.table); sig_add(sig, mr.changed); sig_add(sig, mr.n_new); sig_add(sig, mr.key_max); sig_add(sig, mr.err);
+    sig_add(sig, mr.table); sig_add(sig, mr.changed); sig_add(sig, mr.n_new); sig_add(sig, mr.key_max); sig_add(sig, mr.err); sig_add(sig, R.present.p);
     sig_add(sig, is_max); sig_add(sig, bm_quads); sig_add(sig, ch_tiles); sig_add(sig, c->d_ctrl);
     if (!R.exec || sig != R.sig) {
       if (R.exec) { cudaGraphExecDestroy(R.exec); R.exec = nullptr; }
@@ -1208,17 +1210,22 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
   const uint32_t bm_quads = (uint32_t)((std::max<uint64_t>(dom / 32, 1) + 3) / 4);
   const unsigned ch_tiles = mirror_tiles(bm_quads * 4);
   Resident* R = resident_for(c, h, bits, slots, bm_quads, ch_tiles);
-  DevBuf table_own, bitmap_own, ch_sums_own;
-  if (!R) { table_own = DevBuf(c, slots * 4); bitmap_own = DevBuf(c, (size_t)bm_quads * 16); ch_sums_own = DevBuf(c, (size_t)ch_tiles * 4); }
+  DevBuf table_own, bitmap_own, present_own, ch_sums_own;
+  if (!R) {
+    table_own = DevBuf(c, slots * 4); bitmap_own = DevBuf(c, (size_t)bm_quads * 16); present_own = DevBuf(c, (size_t)bm_quads * 16);
+    ch_sums_own = DevBuf(c, (size_t)ch_tiles * 4);
+  }
+  uint32_t* present = R ? R->present.as<uint32_t>() : present_own.as<uint32_t>();
   int32_t* table = R ? R->table.as<int32_t>() : table_own.as<int32_t>();
   uint4* bitmap = R ? R->bitmap.as<uint4>() : bitmap_own.as<uint4>();
   uint32_t* ch_sums = R ? R->ch_sums.as<uint32_t>() : ch_sums_own.as<uint32_t>();
   XLOG_LAUNCH(c, k_fill_i32, grid_for(slots, 256 * 8), 256, 0, table, slots, empty);
   XLOG_CUDA(cudaMemsetAsync(bitmap, 0, (size_t)bm_quads * 16, c->stream));
+  XLOG_CUDA(cudaMemsetAsync(present, 0, (size_t)bm_quads * 16, c->stream));
   // what the relation holds now (its loaded facts, or the result of an earlier fixpoint) is the starting state
   const uint32_t n_start = H.n;
   if (n_start)
-    XLOG_LAUNCH(c, (k_mirror_scatter<uint32_t>), grid_for(n_start, 256, 1 << 30), 256, 0, (const uint32_t*)H.keys(), (const float*)H.tags(), n_start, table);
+    XLOG_LAUNCH(c, (k_mirror_scatter<uint32_t>), grid_for(n_start, 256, 1 << 30), 256, 0, (const uint32_t*)H.keys(), (const float*)H.tags(), n_start, table, present);
   zero_ctrl(c, kSlotMirNew, 2);
   const MirrorArgs mr{table, reinterpret_cast<uint32_t*>(bitmap), (unsigned long long*)(c->d_ctrl + kSlotMirNew), (uint32_t)(dom - 1),
                       ctrl_u32(c, kSlotErr)};
@@ -1299,7 +1306,7 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
     }
     const uint64_t total = host_apply(vs);
     if (total == 0 && !(round == 0 && plain_rules_done)) break;
-    launch_changed_count(c, reinterpret_cast<const uint32_t*>(bitmap), bm_quads * 4, ch_tiles, ch_sums);
+    launch_changed_count(c, reinterpret_cast<const uint32_t*>(bitmap), present, bm_quads * 4, ch_tiles, ch_sums, mr.n_new);
     XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, ch_sums, (int64_t)ch_tiles, ctrl_u32(c, kSlotMirChanged));
     sync_ctrl(c);
     const uint32_t changed = (uint32_t)c->h_ctrl[kSlotMirChanged];
