@@ -189,17 +189,17 @@ __global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __rest
 }
 
 // Tile shape of the materialising kernel.  The tag-mirror sinks are bound by the latency of one random L2 sector per
-// candidate, so what counts is how many slot reads an SM keeps in flight: blocks per SM x items per thread, against the
-// registers (<= 36 for 7 blocks) and shared memory that takes.  Measured on the two large workloads (single-source
-// R-MAT 20 / 64-source R-MAT 22, ms per fixpoint): 8 items, 2048 rows, 4 blocks 0.75 / 51.2; 8, 1024, 6 blocks 0.71 / 42.2;
-// 8, 1024, 8 blocks (spills) 0.85 / 60.0; 4, 512, 8 blocks 0.65 / 46.3; 5, 640, 8 blocks 0.66 / 43.0; 6, 768, 7 blocks 0.68 / 41.4.
+// candidate, so what counts is how many slot reads an SM keeps in flight: resident warps first, items per thread second.
+// Measured on the two large workloads (single-source R-MAT 20 / 64-source R-MAT 22, ms per fixpoint; items, staged
+// rows, blocks per SM): 8, 1024, 5: 0.62 / 34.6; 8, 1024, 6: 0.63 / 32.7; 6, 768, 6: 0.60 / 31.5; 6, 768, 7: 0.61 / 29.3;
+// 4, 512, 8 (64 warps, no spills): 0.58 / 29.0.
 // The kernel that writes candidates (streaming, HBM-bound) keeps the larger tile: 8 items, 2048 rows, 4 blocks per SM.
 constexpr int kExpBlock = 256;
-constexpr int kExpMirrorBlocksPerSM = 7;              // occupancy asked of the tag-mirror instantiations
+constexpr int kExpMirrorBlocksPerSM = 8;              // occupancy asked of the tag-mirror instantiations
 template <bool MIRROR> struct ExpShapeT {
-  static constexpr int items = MIRROR ? 6 : 8;        // candidates per thread
+  static constexpr int items = MIRROR ? 4 : 8;        // candidates per thread
   static constexpr int tile = kExpBlock * items;      // candidates per block
-  static constexpr int rows = MIRROR ? 768 : 2048;    // outer rows staged in shared memory per tile
+  static constexpr int rows = MIRROR ? 512 : 2048;    // outer rows staged in shared memory per tile
 };
 constexpr int kExpTileWrite = ExpShapeT<false>::tile, kExpTileMirror = ExpShapeT<true>::tile;
 
