@@ -1180,10 +1180,15 @@ ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*
     c->launches = l0 + R.body_launches * (int64_t)out.rounds + (out.status == kResOverflow ? R.body_launches : 0);
   } else {
     unsigned long long seen = 0;
+    uint32_t rows = n_delta;
     for (;;) {
       resident_body(c, R, specs, is_max, mr, bm_quads, ch_tiles, cudaGraphConditionalHandle{}, 0);
       read_state();
       if (c->flags & XLOG_FLAG_PROFILE) {
+        // per delta row and rule: key and tag read, two offsets probed, 16-byte row record and 8-byte start offset written
+        auto cs = c->prof_index.find("k_res_count_scan");
+        if (cs != c->prof_index.end()) c->prof[cs->second].bytes += (int64_t)rows * 40 * (int64_t)specs.size();
+        rows = out.n_delta;
         // algorithmic bytes of the round's expand launches (per candidate: the looked-up columns and tag, and the slot)
         auto it = c->prof_index.find("k_res_expand");
         if (it != c->prof_index.end())
