@@ -200,8 +200,11 @@ class Context:
     def read(self, rel: int):
         """Host copy: ([col arrays], tags) in ascending lexicographic order."""
         n, k = self.size(rel), self._arity[rel]
-        cols = [np.zeros(n, np.int32) for _ in range(k)]
-        tags = np.zeros(n, np.float32)
+        # page-locked destinations (torch's caching host allocator hands freed blocks out again), so that the copy runs
+        # at PCIe speed instead of through the driver's staging buffer
+        torch = self._torch
+        cols = [torch.empty(n, dtype=torch.int32, pin_memory=True).numpy() for _ in range(k)]
+        tags = torch.empty(n, dtype=torch.float32, pin_memory=True).numpy()
         ptrs = (C.c_void_p * k)(*[c.ctypes.data for c in cols])
         got = C.c_int64()
         self._check(self._L.xlog_relation_read(self._h, rel, ptrs, tags.ctypes.data, n, C.byref(got), MEM_HOST))
