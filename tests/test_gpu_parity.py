@@ -260,6 +260,25 @@ def test_chunked_candidates_match_single_batch():
     assert c["derived_tuples"] == d["derived_tuples"] and c["candidates"] == d["candidates"]
 
 
+def test_resident_graph_is_reused_and_rebuilt_when_the_inputs_change():
+    # same context: repeated fixpoints launch the instantiated graph again; a reload that moves or resizes the edge
+    # relation (other index pointers, other domain) must rebuild it.  Every result is checked against the oracle.
+    from paper_2609_27203_b200 import xlog
+    ctx, ids, _ = xlog.load_program(W.config2(scale=10), arena_bytes=1 << 28, flags=xlog.FLAG_CHECK_INVARIANTS)
+    for scale in (10, 10, 12, 9, 12):
+        prog = W.config2(scale=scale)
+        (s, d), w = prog.facts["edge"]
+        ctx.load(ids["edge"], [s, d], w)
+        ctx.load(ids["dist"], [np.array([0], np.int32)], np.zeros(1, np.float32))
+        o, oids, _, stats = oracle_run(prog)
+        for _ in range(3):
+            ctx.reset_idb()
+            r = ctx.fixpoint()
+            assert H.compare_relations(ctx.read(ids["dist"]), o.read(oids["dist"]), what=f"sssp scale {scale}")["bit_unequal"] == 0
+            assert r["derived_tuples"] == stats["derived_tuples"]
+    ctx.close()
+
+
 def test_fixpoint_idempotent_and_reset():
     p = W.config1(200, 700)
     ctx, ids, _, r1 = gpu_run(p)
