@@ -1095,8 +1095,9 @@ void resident_body(Ctx* c, Resident& R, const std::vector<JoinSpec>& specs, bool
     const JoinSpec& S = specs[v];
     XLOG_LAUNCH(c, (k_res_count_scan<uint32_t>), kSMs * 4, kScanBlock, 0, S, dk, (const float*)R.dtags.as<float>(), st, R.rowinfo.as<uint4>(),
                 R.start.as<uint64_t>(), R.tile_rows.as<uint2>(), sc.scan_status + v * R.scan_tiles_cap, sc.tickets + v, err);
+// four waves of blocks: the hardware hands a new block to whichever SM finishes first, which evens out skewed tiles
 #define XLOG_RES_EXPAND(MODE, SINK)                                                                                                         \
-  XLOG_LAUNCH(c, (k_res_expand<uint32_t, MODE, SINK>), kSMs * kExpMirrorBlocksPerSM, kExpBlock, 0, S, dk, (const ResState*)st, (const uint64_t*)R.start.as<uint64_t>(), \
+  XLOG_LAUNCH(c, (k_res_expand<uint32_t, MODE, SINK>), kSMs * kExpMirrorBlocksPerSM * 4, kExpBlock, 0, S, dk, (const ResState*)st, (const uint64_t*)R.start.as<uint64_t>(), \
               (const uint4*)R.rowinfo.as<uint4>(), (const uint2*)R.tile_rows.as<uint2>(), err, mr)
     if (S.fast) { if (is_max) XLOG_RES_EXPAND(kExpFast, kSinkMax); else XLOG_RES_EXPAND(kExpFast, kSinkMin); }
     else { if (is_max) XLOG_RES_EXPAND(kExpGeneric, kSinkMax); else XLOG_RES_EXPAND(kExpGeneric, kSinkMin); }
