@@ -250,7 +250,7 @@ def run_ours(args):
         ratio = NCU_TRAFFIC_RATIO_MIRROR.get(dom)
     bound = "hbm"
     if dom.startswith("k_tri"):
-        bound = "alu"      # sorted-list intersections out of L2: not an HBM-bound kernel (kernels)
+        bound = "alu"      # sorted-list intersections served from L2: compare and branch work, not an HBM-bound kernel
     roofline = {"bound": bound, "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src,
                 "traffic": None if ratio is None else ratio * d["bytes"] / d["launches"],
