@@ -247,6 +247,19 @@ def test_non_linear_and_mutual_recursion():
     check_program(mut)
 
 
+def test_recursion_with_head_arithmetic_takes_the_general_join_path():
+    # down(x - 1) :- down(x), pos(x): a negative head constant rules out the linear-key shape, so every route goes through
+    # the general per-candidate evaluation (with the tag mirror as sink on the default routes)
+    n = 3000
+    pos = np.arange(1, n + 1, dtype=np.int32)
+    w = (1 + 9 * synth.uniform01(41, 1, 0, n)).astype(np.float32)
+    prog = W.Program("countdown", {"pos": (1, W.MINPLUS), "down": (1, W.MINPLUS)},
+                     [W.Rule("down", (W.Affine(-1, ((0, 1),)),), (W.Atom("down", (W.Var(0),)), W.Atom("pos", (W.Var(0),))))],
+                     {"pos": ([pos], w), "down": ([np.array([n, n - 7], np.int32)], np.array([0.0, 100.0], np.float32))}, ("down",))
+    r, _ = check_program(prog, max_iterations=n + 5)
+    assert r["iterations"] == n + 1 and r["derived_tuples"] == n - 1      # n - 7 is a loaded fact
+
+
 def test_chunked_candidates_match_single_batch():
     p = W.config1(300, 1500)
     a, _ = check_program(p)
