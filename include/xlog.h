@@ -76,6 +76,8 @@ typedef struct {
 #define XLOG_FLAG_PROFILE          2u  /* CUDA events around every kernel launch; read with xlog_profile_read */
 #define XLOG_FLAG_NO_TAG_MIRROR    4u  /* evaluate every recursive component by sort -> reduce-by-key -> merge */
 #define XLOG_FLAG_NO_RESIDENT_LOOP 8u  /* the host drives every round of a tag-mirror fixpoint (one control read per round) */
+#define XLOG_FLAG_FORCE_WCOJ      32u  /* materialised triangle joins: always the multiway (worst-case-optimal) plan */
+#define XLOG_FLAG_FORCE_CHAIN     64u  /* ... always the binary-join chain (fails with RESOURCE_EXHAUSTED if its intermediate does not fit) */
 #define XLOG_FLAG_NO_GRAPH        16u  /* resident rounds are launched one by one instead of as one graph with a WHILE node */
 
 /* Evaluation routes of a recursive component (Algorithm 1).  All of them derive the same relation,
@@ -132,10 +134,17 @@ xlog_status xlog_relation_view(xlog_ctx* ctx, xlog_rel rel, const int32_t** cols
  * Listing 7), so the head relation's arity is n_head_cols + 1.
  * Supported shapes: 1 atom; 2 atoms joined on one variable, the second side looked
  * up through a sorted index on that column, its other columns plain variables;
- * the 3-atom directed triangle over one binary relation, either aggregated per x,
+ * the 3-atom triangle join, either aggregated per x over one binary relation,
  * h(x[, count]) :- e(x,y), e(y,z), e(z,x)  (fused intersect-and-aggregate, nothing
- * materialised), or materialised,  h(x,y,z) :- e(x,y), e(y,z), e(z,x)  (count ->
- * scan -> write, rows born sorted; Section "Worst-case-optimal joins").  Anything
+ * materialised), or materialised over up to three binary relations,
+ * h(x,y,z) :- r(x,y), s(y,z), t(z,x)  (rows born sorted).  The materialised form has two
+ * plans (Sections "Worst-case-optimal joins", "WCOJ vs. the binary-join plan"): the
+ * multiway join (count -> scan -> write per row of r, intersecting s's out-list of y with
+ * t's in-list of x) and the binary-join chain (all two-paths of r and s, then a probe of
+ * t).  A skew test chooses per evaluation: the chain when the two-paths, counted exactly,
+ * number at most four per input row of the largest relation and fit the arena, the
+ * multiway join otherwise; XLOG_FLAG_FORCE_WCOJ / XLOG_FLAG_FORCE_CHAIN override it and
+ * xlog_receipt.triangle_plan reports the choice.  Both plans produce identical rows.
  * Negation (Sections "Aggregations and constraints", "Completeness over finite domains":
  * explicit stratified negation-as-failure): a rule of one positive atom followed by one
  * negated atom,  h(..) :- a(..), not b(..).  The negated atom holds iff no row of b matches;
@@ -181,7 +190,12 @@ typedef struct {
   int64_t  kernel_launches;
   int64_t  peak_arena_bytes;
   double   device_ms;              /* CUDA-event time of the whole call on the ctx stream */
+  int32_t  triangle_plan;          /* XLOG_PLAN_*: how the last materialised triangle join of this call was evaluated */
+  int32_t  reserved;
 } xlog_receipt;
+#define XLOG_PLAN_NONE  0
+#define XLOG_PLAN_WCOJ  1          /* multiway join: per row of the first atom, intersect two sorted lists */
+#define XLOG_PLAN_CHAIN 2          /* binary-join chain: materialise the two-paths, then probe the third atom */
 
 /* Evaluate all rules to the least fixpoint, strata in dependency order
  * (Algorithm 1; non-recursive components evaluate each rule once).  On failure

@@ -167,6 +167,7 @@ struct Ctx {
   std::vector<cudaEvent_t> ev_pool;
   int64_t note_bytes = 0;                 // algorithmic bytes of the next launch (consumed by the launch macro)
   std::map<int, std::unique_ptr<Resident>> resident;   // by head relation
+  int last_triangle_plan = 0;             // XLOG_PLAN_* of the last materialised triangle join
   bool unique_untracked = false;          // a stratum went through the tag mirror, which does not count distinct candidate keys
   std::vector<char> stratum_done;         // per relation: its stratum has been evaluated in the running fixpoint
 };

@@ -16,8 +16,12 @@ struct TriGraph {
   const int32_t* src;            // column 0 of the store (ascending)
   const int32_t* dst;            // column 1
   const float* w;                // tags in stored order
+  // second atom's relation (the same store when all three atoms name one relation): column 1 and tags, with
   int64_t out_domain, in_domain;
-  const uint32_t* out_off;       // offsets over src: out-list of v is dst[out_off[v] .. out_off[v+1])
+  const uint32_t* out_off;       // offsets over its column 0: out-list of v is s_dst[out_off[v] .. out_off[v+1])
+  const int32_t* s_dst;
+  const float* s_w;
+  // third atom's relation, transposed:
   const uint32_t* in_off;        // offsets over dst of the transposed copy
   const int32_t* in_src;         // transposed copy: sources of the edges into v, ascending
   const float* in_w;             // and their tags
@@ -41,15 +45,15 @@ __global__ void __launch_bounds__(256) k_tri_edges(TriGraph G, int times, uint32
     A acc = Op::identity();
     if (la && lb) {
       const bool walk_a = la <= lb;
-      const int32_t* wl = walk_a ? G.dst + a0 : G.in_src + b0;                // walked list
-      const int32_t* sl = walk_a ? G.in_src + b0 : G.dst + a0;                // searched list
+      const int32_t* wl = walk_a ? G.s_dst + a0 : G.in_src + b0;                // walked list
+      const int32_t* sl = walk_a ? G.in_src + b0 : G.s_dst + a0;                // searched list
       const uint32_t nw = walk_a ? la : lb, ns = walk_a ? lb : la;
       for (uint32_t i = lane; i < nw; i += 32) {
         const int32_t z = wl[i];
         uint32_t lo = 0, hi = ns;
         while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (sl[mid] < z) lo = mid + 1; else hi = mid; }
         if (lo < ns && sl[lo] == z) {
-          const float wyz = walk_a ? G.w[a0 + i] : G.w[a0 + lo];
+          const float wyz = walk_a ? G.s_w[a0 + i] : G.s_w[a0 + lo];
           const float wzx = walk_a ? G.in_w[b0 + lo] : G.in_w[b0 + i];
           const float t = times ? (wxy * wyz) * wzx : (wxy + wyz) + wzx;
           acc = Op::combine(acc, Op::lift(t));
@@ -122,8 +126,8 @@ __global__ void __launch_bounds__(256) k_tri_materialise(TriGraph G, int times, 
     const uint32_t la = a1 - a0, lb = b1 - b0;
     if (!la || !lb) continue;
     const bool walk_a = la <= lb;
-    const int32_t* wl = walk_a ? G.dst + a0 : G.in_src + b0;
-    const int32_t* sl = walk_a ? G.in_src + b0 : G.dst + a0;
+    const int32_t* wl = walk_a ? G.s_dst + a0 : G.in_src + b0;
+    const int32_t* sl = walk_a ? G.in_src + b0 : G.s_dst + a0;
     const uint32_t nw = walk_a ? la : lb, ns = walk_a ? lb : la;
     uint64_t pos = edge_off[e];
     const K xy = ((K)(uint32_t)x << L.shift[0]) | ((K)(uint32_t)y << L.shift[1]);
@@ -140,7 +144,7 @@ __global__ void __launch_bounds__(256) k_tri_materialise(TriGraph G, int times, 
       }
       const unsigned m = __ballot_sync(0xffffffffu, hit);
       if (hit) {
-        const float wyz = walk_a ? G.w[a0 + i] : G.w[a0 + lo];
+        const float wyz = walk_a ? G.s_w[a0 + i] : G.s_w[a0 + lo];
         const float wzx = walk_a ? G.in_w[b0 + lo] : G.in_w[b0 + i];
         const uint64_t o = pos + __popc(m & lanemask_lt());
         out_keys[o] = xy | ((K)(uint32_t)z << L.shift[2]);
@@ -158,6 +162,58 @@ __global__ void __launch_bounds__(256) k_tri_compact(const uint32_t* __restrict_
                                                      K* __restrict__ keys, uint32_t* __restrict__ counts, float* __restrict__ tags) {
   for (int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; x < domain; x += (int64_t)gridDim.x * blockDim.x)
     if (flag[x]) { const uint32_t p = pos[x]; keys[p] = (K)x; counts[p] = grp_cnt[x]; tags[p] = grp_tag[x]; }
+}
+
+// ---- the binary-join plan of the same query (paper: "WCOJ vs. the binary-join plan") -------------------------------
+// Step one materialises every two-path (x,y,z) of the first two atoms with the ordinary join kernels; step two, here,
+// keeps the two-paths that the third atom closes: one thread per two-path looks (z, x) up in the third relation's
+// store (offsets over its column 0, then a binary search in the run's sorted column 1).  count -> scan -> emit, in
+// input order, so the output is sorted by (x,y,z) like the worst-case-optimal path's.
+struct ChainProbe {
+  KeyLayout L;                   // layout of the two-path keys (x,y,z): wide enough for everything r and s hold
+  KeyLayout out;                 // layout of the head relation (its bounds take t into account as well)
+  int64_t t_domain;
+  const uint32_t* t_off;         // offsets over the third relation's column 0
+  const int32_t* t_col1;         // its column 1, ascending inside each run
+  const float* t_w;
+  int times;
+};
+
+template <typename K>
+__device__ __forceinline__ bool chain_lookup(const ChainProbe& P, K key, uint32_t& pos) {
+  const int32_t x = key_col<K>(P.L, key, 0), z = key_col<K>(P.L, key, 2);
+  if (z >= P.t_domain) return false;
+  uint32_t lo = P.t_off[z];
+  const uint32_t end = P.t_off[z + 1];
+  uint32_t hi = end;
+  while (lo < hi) { const uint32_t mid = lo + ((hi - lo) >> 1); if (P.t_col1[mid] < x) lo = mid + 1; else hi = mid; }
+  pos = lo;
+  return lo < end && P.t_col1[lo] == x;
+}
+
+template <typename K>
+__global__ void __launch_bounds__(256) k_chain_probe_count(ChainProbe P, const K* __restrict__ keys, uint64_t n, uint32_t* __restrict__ hit) {
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+    uint32_t pos;
+    hit[i] = chain_lookup<K>(P, keys[i], pos) ? 1u : 0u;
+  }
+}
+
+template <typename K, typename KH>
+__global__ void __launch_bounds__(256) k_chain_probe_emit(ChainProbe P, const K* __restrict__ keys, const float* __restrict__ tags, uint64_t n,
+                                                          const uint32_t* __restrict__ hit, const uint64_t* __restrict__ off,
+                                                          KH* __restrict__ out_keys, float* __restrict__ out_tags) {
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+    if (!hit[i]) continue;
+    uint32_t pos = 0;
+    chain_lookup<K>(P, keys[i], pos);
+    const float w = P.t_w[pos];
+    KH hk = 0;
+#pragma unroll
+    for (int col = 0; col < 3; ++col) hk |= (KH)(uint32_t)key_col<K>(P.L, keys[i], col) << P.out.shift[col];
+    out_keys[off[i]] = hk;
+    out_tags[off[i]] = P.times ? tags[i] * w : tags[i] + w;
+  }
 }
 
 }  // namespace xlog

@@ -267,13 +267,14 @@ void add_rule(Ctx* c, const xlog_plan* p, xlog_rule* out) {
   } else {
     // directed triangle  h(x) :- e(x,y), e(y,z), e(z,x)
     const xlog_atom* a = p->atoms;
-    bool ok = a[0].rel == a[1].rel && a[1].rel == a[2].rel && c->rels[a[0].rel]->arity == 2;
+    const bool one_rel = a[0].rel == a[1].rel && a[1].rel == a[2].rel;
+    bool ok = c->rels[a[0].rel]->arity == 2 && c->rels[a[1].rel]->arity == 2 && c->rels[a[2].rel]->arity == 2;
     for (int j = 0; j < 3 && ok; ++j) ok = is_plain_var(a[j].args[0]) && is_plain_var(a[j].args[1]);
     if (ok) {
       const int x = a[0].args[0].var, y = a[0].args[1].var, z = a[1].args[1].var;
       ok = x != y && y != z && x != z && a[1].args[0].var == y && a[2].args[0].var == z && a[2].args[1].var == x;
       const int hv[3] = {x, y, z};
-      bool agg = ok && p->n_head_cols == 1, mat = ok && p->n_head_cols == 3 && !p->emit_count_column;
+      bool agg = ok && one_rel && p->n_head_cols == 1, mat = ok && p->n_head_cols == 3 && !p->emit_count_column;
       for (int h = 0; h < p->n_head_cols && h < 3; ++h) {
         bool id = p->head[h].c0 == 0;
         for (int v = 0; v < XLOG_MAX_VARS; ++v) id = id && p->head[h].coef[v] == (v == hv[h] ? 1 : 0);
@@ -282,7 +283,7 @@ void add_rule(Ctx* c, const xlog_plan* p, xlog_rule* out) {
       ok = agg || mat;
       r.kind = mat ? 4 : 3;
     }
-    if (!ok) fail(XLOG_ERR_UNSUPPORTED, "three-atom rules are supported only as the directed triangle h(x) or h(x,y,z) :- e(x,y), e(y,z), e(z,x)");
+    if (!ok) fail(XLOG_ERR_UNSUPPORTED, "three-atom rules are supported only as the triangle join h(x,y,z) :- r(x,y), s(y,z), t(z,x) or its per-x aggregate h(x) over one relation");
   }
   c->rules.push_back(r);
   H.is_head = true;
@@ -846,6 +847,7 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
   G.out_domain = out_ix.domain; G.in_domain = in_ix.domain;
   G.out_off = out_ix.off.as<uint32_t>(); G.in_off = in_ix.off.as<uint32_t>();
   G.in_src = in_ix.other[0]; G.in_w = in_ix.tags;
+  G.s_dst = G.dst; G.s_w = G.w;
   const int64_t domain = out_ix.domain;
   DevBuf ecnt(c, (size_t)E.n * 4), eacc(c, (size_t)E.n * sizeof(A));
   DevBuf gcnt(c, (size_t)domain * 4), gtag(c, (size_t)domain * 4), flag(c, (size_t)domain * 4);
@@ -878,27 +880,120 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
 }
 
 // tri(x,y,z) :- e(x,y), e(y,z), e(z,x): count per edge -> scan -> materialise; the result is born sorted.
+// tri(x,y,z) :- r(x,y), s(y,z), t(z,x), materialised.  Two plans (paper: "Worst-case-optimal joins"):
+//  - multiway: for every r row intersect s's out-list of y with t's in-list of x (count -> scan -> write);
+//  - binary chain: materialise every two-path of r and s with the ordinary join, then keep those t closes.
+// A skew test picks one per evaluation: the chain when its intermediate (the two-paths, counted exactly by the join's
+// count step) stays within a small multiple of the inputs, the multiway join otherwise.
+constexpr uint64_t kChainMaxBlowup = 4;      // two-paths per input row up to which the chain is chosen
+
+void triangle_chain(Ctx* c, Relation& H, const Relation& H2, Counted& q, Relation& T) {
+  const int times = H.sr == XLOG_SR_SUMPROD ? 1 : 0;
+  const int ckb = H2.key_bytes;
+  const uint64_t n2 = q.total;
+  // step one: all two-paths (x,y,z) with tag w_xy otimes w_yz, in (x,y,z) order
+  DevBuf k0(c, std::max<uint64_t>(n2, 1) * ckb), t0(c, std::max<uint64_t>(n2, 1) * 4);
+  c->note_bytes = (int64_t)n2 * (ckb + 4 + 8);
+  launch_expand<false>(c, q, 0, n2, ckb, k0.p, t0.as<float>(), BwdArgs{});
+  q.start.reset(); q.rowinfo.reset();
+  // step two: probe t with (z, x)
+  Index& tix = ensure_index(c, T, 0);
+  ChainProbe P{};
+  P.L = H2.layout; P.out = H.layout;
+  P.t_domain = tix.domain; P.t_off = tix.off.as<uint32_t>(); P.t_col1 = tix.other[0]; P.t_w = tix.tags; P.times = times;
+  DevBuf hit(c, std::max<uint64_t>(n2, 1) * 4), off(c, std::max<uint64_t>(n2, 1) * 8);
+  const unsigned tiles = (unsigned)((n2 + kScanTile - 1) / kScanTile);
+  DevBuf sums(c, (size_t)std::max(tiles, 1u) * 8);
+  zero_ctrl(c, kSlotTotals);
+  c->note_bytes = (int64_t)n2 * (ckb + 4);
+  DISPATCH_K(ckb, XLOG_LAUNCH(c, (k_chain_probe_count<K>), grid_for(n2, 256), 256, 0, P, (const K*)k0.p, n2, hit.as<uint32_t>()));
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)hit.as<uint32_t>(), (int64_t)n2, sums.as<uint64_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, sums.as<uint64_t>(), (int64_t)tiles, (uint64_t*)(c->d_ctrl + kSlotTotals));
+  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)hit.as<uint32_t>(), (int64_t)n2,
+              (const uint64_t*)sums.as<uint64_t>(), off.as<uint64_t>());
+  sync_ctrl(c);
+  const uint64_t total = c->h_ctrl[kSlotTotals];
+  if (total > kSortMaxN) fail(XLOG_ERR_CAPACITY_EXCEEDED, "materialised triangle relation exceeds 2^30 - 1 rows");
+  c->r_unique += (int64_t)total;
+  KeyTags kt;
+  kt.n = (uint32_t)total;
+  kt.keys = DevBuf(c, (size_t)std::max<uint64_t>(total, 1) * H.key_bytes);
+  kt.tags = DevBuf(c, (size_t)std::max<uint64_t>(total, 1) * 4);
+  c->note_bytes = (int64_t)n2 * (ckb + 4 + 12) + (int64_t)total * (H.key_bytes + 4);
+#define XLOG_CHAIN_EMIT(K2, KH)                                                                                                     \
+  XLOG_LAUNCH(c, (k_chain_probe_emit<K2, KH>), grid_for(n2, 256), 256, 0, P, (const K2*)k0.p, (const float*)t0.as<float>(), n2,    \
+              (const uint32_t*)hit.as<uint32_t>(), (const uint64_t*)off.as<uint64_t>(), kt.keys.as<KH>(), kt.tags.as<float>())
+  if (n2) {
+    if (ckb == 4 && H.key_bytes == 4) XLOG_CHAIN_EMIT(uint32_t, uint32_t);
+    else if (ckb == 4) XLOG_CHAIN_EMIT(uint32_t, uint64_t);
+    else if (H.key_bytes == 4) XLOG_CHAIN_EMIT(uint64_t, uint32_t);
+    else XLOG_CHAIN_EMIT(uint64_t, uint64_t);
+  }
+#undef XLOG_CHAIN_EMIT
+  set_current(H, std::move(kt));
+}
+
 void triangle_materialise(Ctx* c, Relation& H, const RuleC& r) {
-  Relation& E = *c->rels[r.plan.atoms[0].rel];
+  Relation& R = *c->rels[r.plan.atoms[0].rel];
+  Relation& S = *c->rels[r.plan.atoms[1].rel];
+  Relation& T = *c->rels[r.plan.atoms[2].rel];
   if (H.n_facts) fail(XLOG_ERR_UNSUPPORTED, "a materialised triangle relation cannot also hold loaded facts");
-  if (E.n == 0) { KeyTags empty; set_current(H, std::move(empty)); return; }
-  Index& out_ix = ensure_index(c, E, 0);
-  Index& in_ix = ensure_index(c, E, 1);
+  if (R.n == 0 || S.n == 0 || T.n == 0) { KeyTags empty; set_current(H, std::move(empty)); c->last_triangle_plan = XLOG_PLAN_CHAIN; return; }
+  const int times = H.sr == XLOG_SR_SUMPROD ? 1 : 0;
+
+  // skew test: count the two-paths of r and s exactly (the chain's intermediate); this is the chain's own count step
+  bool chain = (c->flags & XLOG_FLAG_FORCE_CHAIN) != 0;
+  if (!(c->flags & (XLOG_FLAG_FORCE_CHAIN | XLOG_FLAG_FORCE_WCOJ)) || chain) {
+    RuleC two;                                           // tmp(x,y,z) :- r(x,y), s(y,z)
+    two.plan = r.plan;
+    two.plan.n_atoms = 2;
+    two.kind = 2;
+    two.shape[0] = join_shape(c, two.plan, 0);
+    if (!two.shape[0].ok) fail(XLOG_ERR_INTERNAL, "triangle chain: no join path");
+    Relation H2;                                         // the two-paths' own layout: bounds from r and s alone
+    H2.arity = 3; H2.sr = H.sr;
+    H2.col_max[0] = R.val_max[0] ? R.val_max[0] : R.col_max[0]; H2.col_max[1] = R.val_max[1] ? R.val_max[1] : R.col_max[1];
+    H2.col_max[2] = S.val_max[1] ? S.val_max[1] : S.col_max[1];
+    H2.layout = make_layout(3, H2.col_max);
+    H2.key_bytes = H2.layout.total_bits <= 32 ? 4 : 8;
+    Variant v{&two, 0, full_source(R)};
+    Counted q;
+    count_variant(c, v, H2, q, kSlotTotals);
+    sync_ctrl(c);
+    q.total = c->h_ctrl[kSlotTotals];
+    q.deg.reset(); q.sums.reset();
+    const uint64_t biggest = std::max<uint64_t>(R.n, std::max<uint64_t>(S.n, T.n));
+    const size_t need = (size_t)q.total * (H2.key_bytes + 4 + 12) + (16u << 20);
+    const bool fits = q.total <= kSortMaxN && need <= c->arena.largest_free() / 2;
+    if (!(c->flags & XLOG_FLAG_FORCE_CHAIN)) chain = fits && q.total <= kChainMaxBlowup * biggest;
+    else if (!fits) fail(XLOG_ERR_RESOURCE_EXHAUSTED, "triangle chain: the two-path intermediate does not fit the arena");
+    if (chain) {
+      c->r_candidates += (int64_t)q.total;
+      c->last_triangle_plan = XLOG_PLAN_CHAIN;
+      triangle_chain(c, H, H2, q, T);
+      return;
+    }
+  }
+  c->last_triangle_plan = XLOG_PLAN_WCOJ;
+  Index& out_ix = ensure_index(c, S, 0);
+  Index& in_ix = ensure_index(c, T, 1);
+  ensure_soa(c, R);
+  ensure_soa(c, S);
   TriGraph G{};
-  G.n_edges = E.n;
-  G.src = E.cols[0].as<int32_t>(); G.dst = E.cols[1].as<int32_t>(); G.w = E.tags();
+  G.n_edges = R.n;
+  G.src = R.cols[0].as<int32_t>(); G.dst = R.cols[1].as<int32_t>(); G.w = R.tags();
   G.out_domain = out_ix.domain; G.in_domain = in_ix.domain;
   G.out_off = out_ix.off.as<uint32_t>(); G.in_off = in_ix.off.as<uint32_t>();
+  G.s_dst = out_ix.other[0]; G.s_w = out_ix.tags;
   G.in_src = in_ix.other[0]; G.in_w = in_ix.tags;
-  const int times = H.sr == XLOG_SR_SUMPROD ? 1 : 0;
-  DevBuf ecnt(c, (size_t)E.n * 4), eacc(c, (size_t)E.n * 4), eoff(c, (size_t)E.n * 8);
-  const unsigned tiles = (E.n + kScanTile - 1) / kScanTile;
+  DevBuf ecnt(c, (size_t)R.n * 4), eacc(c, (size_t)R.n * 4), eoff(c, (size_t)R.n * 8);
+  const unsigned tiles = (R.n + kScanTile - 1) / kScanTile;
   DevBuf sums(c, (size_t)tiles * 8);
-  c->note_bytes = (int64_t)E.n * 12 * 3;
+  c->note_bytes = (int64_t)(R.n + S.n + T.n) * 12;
   XLOG_LAUNCH(c, (k_tri_edges<OpMax>), kSMs * 8, 256, 0, G, times, ecnt.as<uint32_t>(), eacc.as<float>());
-  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)ecnt.as<uint32_t>(), (int64_t)E.n, sums.as<uint64_t>());
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)ecnt.as<uint32_t>(), (int64_t)R.n, sums.as<uint64_t>());
   XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, sums.as<uint64_t>(), (int64_t)tiles, (uint64_t*)(c->d_ctrl + kSlotTotals));
-  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)ecnt.as<uint32_t>(), (int64_t)E.n,
+  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)ecnt.as<uint32_t>(), (int64_t)R.n,
               (const uint64_t*)sums.as<uint64_t>(), eoff.as<uint64_t>());
   sync_ctrl(c);                                            // the one small metadata read that sizes the output
   const uint64_t total = c->h_ctrl[kSlotTotals];
@@ -1594,6 +1689,7 @@ xlog_status xlog_fixpoint(xlog_ctx* c, xlog_receipt* receipt) {
   const int64_t l0 = c->launches, d0 = c->d2h_bytes, h0 = c->h2d_bytes;
   c->r_candidates = c->r_unique = c->r_new = c->r_improved = c->r_iterations = c->r_strata = 0;
   c->unique_untracked = false;
+  c->last_triangle_plan = XLOG_PLAN_NONE;
   c->arena.reset_peak();
   cudaSetDevice(c->device);
   cudaEventRecord(c->ev0, c->stream);
@@ -1624,6 +1720,8 @@ xlog_status xlog_fixpoint(xlog_ctx* c, xlog_receipt* receipt) {
     receipt->kernel_launches = c->launches - l0;
     receipt->peak_arena_bytes = (int64_t)c->arena.peak();
     receipt->device_ms = ms;
+    receipt->triangle_plan = c->last_triangle_plan;
+    receipt->reserved = 0;
   }
   return st;
 }

@@ -138,6 +138,32 @@ def triangle_rows_program(src, dst, w, semiring=MAXPLUS, name="triangle_rows") -
     )
 
 
+def triangle_join_program(r, s, t, semiring=MAXPLUS, name="triangle_join") -> Program:
+    """tri(x,y,z) :- r(x,y), s(y,z), t(z,x) over three relations, each given as (col0, col1, tags)."""
+    def rel(x):
+        return ([np.ascontiguousarray(x[0], np.int32), np.ascontiguousarray(x[1], np.int32)], np.ascontiguousarray(x[2], np.float32))
+    return Program(
+        name=name,
+        relations={"r": (2, semiring), "s": (2, semiring), "t": (2, semiring), "tri": (3, semiring)},
+        rules=[Rule("tri", (V(0), V(1), V(2)),
+                    (Atom("r", (Var(0), Var(1))), Atom("s", (Var(1), Var(2))), Atom("t", (Var(2), Var(0)))))],
+        facts={"r": rel(r), "s": rel(s), "t": rel(t)},
+        outputs=("tri",),
+    )
+
+
+def hot_domain_triangle(n_rows=65536, domain=406, seed=synth.SEED_BASE + 6) -> Program:
+    """Three relations of n_rows distinct uniform pairs over a small domain: every join variable is hot, so the two-paths
+    of any two relations far outnumber the triangles (65,536 rows over 406 values: about 10.6 M two-paths, 4.2 M triples)."""
+    rels = []
+    for k in range(3):
+        a, b = synth.uniform_digraph(domain, n_rows, seed + 17 * k)
+        rels.append((a, b, synth.log_prob_tags(n_rows, seed + 17 * k + 1)))
+    p = triangle_join_program(*rels, name=f"triangle_join_hot{domain}_n{n_rows}")
+    p.info.update(n_rows=n_rows, domain=domain)
+    return p
+
+
 def digits_program(log_tags: np.ndarray, name="digits") -> Program:
     """sum(p, a+b) :- digit(2p, a), digit(2p+1, b), logsumexp per (p, a+b).
 

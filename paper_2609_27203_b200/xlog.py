@@ -24,6 +24,9 @@ FLAG_PROFILE = 2
 FLAG_NO_TAG_MIRROR = 4
 FLAG_NO_RESIDENT_LOOP = 8
 FLAG_NO_GRAPH = 16
+FLAG_FORCE_WCOJ = 32
+FLAG_FORCE_CHAIN = 64
+PLAN_NONE, PLAN_WCOJ, PLAN_CHAIN = 0, 1, 2
 
 EXPORTS = ["xlog_ctx_create", "xlog_ctx_destroy", "xlog_last_error", "xlog_relation_create", "xlog_relation_load",
            "xlog_relation_size", "xlog_relation_read", "xlog_relation_view", "xlog_rule_add", "xlog_fixpoint",
@@ -67,7 +70,7 @@ class Receipt(C.Structure):
                 ("derived_tuples", C.c_int64), ("candidates", C.c_int64), ("unique_candidates", C.c_int64),
                 ("new_tuples", C.c_int64), ("improved_tags", C.c_int64), ("h2d_bytes", C.c_int64),
                 ("d2h_bytes", C.c_int64), ("kernel_launches", C.c_int64), ("peak_arena_bytes", C.c_int64),
-                ("device_ms", C.c_double)]
+                ("device_ms", C.c_double), ("triangle_plan", C.c_int32), ("reserved", C.c_int32)]
 
     def as_dict(self) -> Dict[str, object]:
         return {k: getattr(self, k) for k, _ in self._fields_ if k != "struct_size"}

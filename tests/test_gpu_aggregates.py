@@ -72,6 +72,83 @@ def test_materialised_triangles_match_oracle_and_the_fused_aggregate(scale):
     ctx2.close()
 
 
+def dense_count(prog, n):
+    """Triangles of r, s, t by a dense matrix product: sum over (x,y,z) of R[x,y] S[y,z] T[z,x]."""
+    M = []
+    for name in ("r", "s", "t"):
+        (a, b), _ = prog.facts[name]
+        m = np.zeros((n, n), np.float64)
+        m[a, b] = 1
+        M.append(m)
+    return int(round(((M[0] @ M[1]) * M[2].T).sum()))
+
+
+def test_triangle_join_over_three_relations_both_plans_match_the_oracle():
+    from paper_2609_27203_b200 import xlog
+    prog = W.hot_domain_triangle(n_rows=3000, domain=70)
+    o, oids, _ = oracle.load_program(prog)
+    o.run("naive")
+    want = o.read(oids["tri"])
+    assert len(want[1]) == dense_count(prog, 70) > 0
+    for flags, plan in [(xlog.FLAG_FORCE_WCOJ, xlog.PLAN_WCOJ), (xlog.FLAG_FORCE_CHAIN, xlog.PLAN_CHAIN), (0, xlog.PLAN_WCOJ)]:
+        ctx, gids, _ = xlog.load_program(prog, arena_bytes=1 << 28, flags=xlog.FLAG_CHECK_INVARIANTS | flags)
+        r = ctx.fixpoint()
+        assert r["triangle_plan"] == plan
+        rep = H.compare_relations(ctx.read(gids["tri"]), want, what=f"{prog.name} plan {plan}")
+        assert rep["bit_unequal"] == 0            # both plans fold (w_xy + w_yz) + w_zx in that order, like the oracle
+        ctx.close()
+    # columns whose maxima differ between the relations: rows of r that t can never close must not trip the key range
+    (ra, rb), rw = prog.facts["r"]
+    prog.facts["r"] = ([np.concatenate([ra, [900, 901]]).astype(np.int32), np.concatenate([rb, [5, 6]]).astype(np.int32)],
+                       np.concatenate([rw, [-0.1, -0.2]]).astype(np.float32))
+    o, oids, _ = oracle.load_program(prog)
+    o.run("naive")
+    for flags in (xlog.FLAG_FORCE_WCOJ, xlog.FLAG_FORCE_CHAIN):
+        ctx, gids, _ = xlog.load_program(prog, arena_bytes=1 << 28, flags=xlog.FLAG_CHECK_INVARIANTS | flags)
+        ctx.fixpoint()
+        assert H.compare_relations(ctx.read(gids["tri"]), o.read(oids["tri"]), what="ragged maxima")["bit_unequal"] == 0
+        ctx.close()
+
+
+def test_skew_test_picks_the_plan_and_both_plans_give_identical_rows_on_the_hot_domain_fixture():
+    # three relations of 65,536 rows over a hot domain: about 4.19 M triples out of 10.6 M two-paths
+    from paper_2609_27203_b200 import xlog
+    prog = W.hot_domain_triangle()
+    n_tri = dense_count(prog, prog.info["domain"])
+    assert 3_900_000 < n_tri < 4_500_000
+    got = {}
+    for flags in (0, xlog.FLAG_FORCE_WCOJ, xlog.FLAG_FORCE_CHAIN):
+        ctx, gids, _ = xlog.load_program(prog, arena_bytes=1 << 30, flags=flags)
+        r = ctx.fixpoint()
+        got[flags] = (ctx.read(gids["tri"]), r)
+        ctx.close()
+    assert got[0][1]["triangle_plan"] == xlog.PLAN_WCOJ                      # skewed: the intermediate is 160x the inputs
+    assert got[xlog.FLAG_FORCE_CHAIN][1]["candidates"] > 2 * n_tri           # the chain really materialised the two-paths
+    base_cols, base_tags = got[xlog.FLAG_FORCE_WCOJ][0]
+    assert len(base_tags) == n_tri
+    key = (base_cols[0].astype(np.int64) << 40) | (base_cols[1].astype(np.int64) << 20) | base_cols[2]
+    assert np.all(np.diff(key) > 0)
+    for flags in (0, xlog.FLAG_FORCE_CHAIN):
+        cols, tags = got[flags][0]
+        assert all(np.array_equal(a, b) for a, b in zip(cols, base_cols)) and np.array_equal(tags.view(np.int32), base_tags.view(np.int32))
+    # uniform and empty inputs take the binary-join chain
+    sparse = W.hot_domain_triangle(n_rows=65536, domain=60000)
+    ctx, gids, _ = xlog.load_program(sparse, arena_bytes=1 << 30)
+    r = ctx.fixpoint()
+    assert r["triangle_plan"] == xlog.PLAN_CHAIN
+    ctx2, g2, _ = xlog.load_program(sparse, arena_bytes=1 << 30, flags=xlog.FLAG_FORCE_WCOJ)
+    r2 = ctx2.fixpoint()
+    assert r2["derived_tuples"] == r["derived_tuples"]
+    a, b = ctx.read(gids["tri"]), ctx2.read(g2["tri"])
+    assert all(np.array_equal(x, y) for x, y in zip(a[0], b[0])) and np.array_equal(a[1].view(np.int32), b[1].view(np.int32))
+    ctx.close(); ctx2.close()
+    empty = W.triangle_join_program(*[(np.zeros(0, np.int32), np.zeros(0, np.int32), np.zeros(0, np.float32))] * 3)
+    ctx, gids, _ = xlog.load_program(empty, arena_bytes=1 << 24)
+    r = ctx.fixpoint()
+    assert r["triangle_plan"] == xlog.PLAN_CHAIN and r["derived_tuples"] == 0
+    ctx.close()
+
+
 def test_triangle_degenerate_graphs():
     # no triangle at all; one 3-cycle (single-term groups pass through bit-exactly); complete digraph; a hub
     for s, d, w in [([0, 1], [1, 2], [0.5, 0.25]),

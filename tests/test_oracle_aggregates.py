@@ -281,3 +281,33 @@ def test_negation_over_a_recursive_lower_stratum():
     with pytest.raises(oracle.OracleError) as e:
         o.run("naive")
     assert e.value.status == "UNSUPPORTED"
+
+
+def test_triangle_join_over_three_relations_against_brute_force_and_a_matrix_product():
+    # tri(x,y,z) :- r(x,y), s(y,z), t(z,x): the row set by three nested Python loops, the tag (w_xy + w_yz) + w_zx in
+    # fp32, and the row count by the dense product sum((R @ S) * T^T), on the hot-domain recipe at a small size
+    prog = W.hot_domain_triangle(n_rows=400, domain=24)
+    o, ids, _ = oracle.load_program(prog)
+    o.run("naive")
+    cols, tags = o.read(ids["tri"])
+    rel = {}
+    for name in ("r", "s", "t"):
+        (a, b), w = prog.facts[name]
+        rel[name] = {(int(x), int(y)): np.float32(v) for x, y, v in zip(a, b, w)}
+    want = {}
+    for (x, y), wxy in rel["r"].items():
+        for (y2, z), wyz in rel["s"].items():
+            if y2 == y and (z, x) in rel["t"]:
+                want[(x, y, z)] = np.float32(np.float32(wxy + wyz) + rel["t"][(z, x)])
+    got = {(int(a), int(b), int(c)): t for a, b, c, t in zip(cols[0], cols[1], cols[2], tags)}
+    assert got.keys() == want.keys() and len(want) > 20
+    assert all(got[k] == want[k] for k in want)
+    M = []
+    for name in ("r", "s", "t"):
+        m = np.zeros((24, 24))
+        for (x, y) in rel[name]:
+            m[x, y] = 1
+        M.append(m)
+    assert len(want) == int(round(((M[0] @ M[1]) * M[2].T).sum()))
+    # rows come back in ascending (x, y, z)
+    assert sorted(got.keys()) == list(zip(cols[0].tolist(), cols[1].tolist(), cols[2].tolist()))
