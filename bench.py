@@ -51,6 +51,10 @@ def make_program(name: str, scale: int | None, sources: int | None = None):
         return W.config5(scale=s, n_sources=ns), (56 << 30) if s >= 21 and ns > 16 else (8 << 30)
     if name == "triangles":
         return W.config3(scale=scale or 18), 2 << 30
+    if name == "wcoj":
+        # the triangle-join fixture of the paper's WCOJ ablation: three relations of 2^scale rows over a hot domain
+        s = scale or 16
+        return W.hot_domain_triangle(n_rows=1 << s, domain=406 if s == 16 else max(int(1.4 * 2 ** (s / 2)), 8)), 2 << 30
     if name == "digits":
         return W.config4(), 1 << 30
     raise SystemExit(f"unknown workload {name}")
@@ -197,6 +201,7 @@ def run_ours(args):
 
     # facts resident in HBM before any timed region
     base_flags = (xlog.FLAG_NO_TAG_MIRROR if args.no_tag_mirror else 0) | (xlog.FLAG_NO_GRAPH if args.no_graph else 0)
+    base_flags |= {"auto": 0, "wcoj": xlog.FLAG_FORCE_WCOJ, "chain": xlog.FLAG_FORCE_CHAIN}[args.triangle_plan]
     ctx, ids, rules = xlog.load_program(program, device=local_rank, arena_bytes=arena, device_inputs=True, flags=base_flags)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)          # > 126 MB L2
 
@@ -309,6 +314,7 @@ def run_ours(args):
            "data": "synthetic", "impl": "ours",
            "config": {"workload": program.name, "program": args.workload, **{k: v for k, v in program.info.items()},
                       "derived_tuples": derived, "rounds": receipt["iterations"], "candidates": receipt["candidates"],
+                      "triangle_plan": {0: None, 1: "wcoj", 2: "chain"}[receipt["triangle_plan"]],
                       "unique_candidates": receipt["unique_candidates"], "l2": "flushed between steps (256 MB fill)",
                       "parallelism": "replicas only" if world > 1 else "1 gpu", "facts": "resident and indexed before timing"},
            "clocks": clk.summary(), "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
@@ -317,7 +323,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         # the oracle as it stands, on this machine's host cores, on a bounded sample of the same workload
         # bounded sample (about 10-30 s of CPU work): the full workload where the oracle manages it, else a smaller R-MAT scale
-        cpu_scale = args.cpu_scale or {"triangles": 14, "reach": 16}.get(args.workload)
+        cpu_scale = args.cpu_scale or {"triangles": 14, "reach": 16, "wcoj": 13}.get(args.workload)
         sample, _ = make_program(args.workload, cpu_scale) if cpu_scale else (program, 0)
         sec, stats, _o = run_oracle_once(sample)
         out["cpu_baseline"] = {"value": stats["derived_tuples"] / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
@@ -336,10 +342,10 @@ def run_reference(args):
     rank, _, world = dist_env()
     if rank != 0:
         return
-    est20 = {"sssp": 16.0, "reach": 600.0, "closure": 3.0, "triangles": 200.0, "digits": 10.0}[args.workload]
+    est20 = {"sssp": 16.0, "reach": 600.0, "closure": 3.0, "triangles": 200.0, "digits": 10.0, "wcoj": 60.0}[args.workload]
     scale = args.scale
-    if args.workload in ("sssp", "reach", "triangles") and scale is None:
-        full = {"sssp": 20, "reach": 22, "triangles": 18}[args.workload]
+    if args.workload in ("sssp", "reach", "triangles", "wcoj") and scale is None:
+        full = {"sssp": 20, "reach": 22, "triangles": 18, "wcoj": 16}[args.workload]
         scale = full
         while scale > 8 and (args.steps + args.warmup) * est20 * 2.0 ** (scale - full) > 150.0:
             scale -= 1
@@ -372,9 +378,10 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="sssp", choices=["sssp", "closure", "reach", "triangles", "digits"])
+    ap.add_argument("--workload", default="sssp", choices=["sssp", "closure", "reach", "triangles", "digits", "wcoj"])
     ap.add_argument("--scale", type=int, default=None, help="R-MAT scale override (smaller cases for profiling)")
     ap.add_argument("--sources", type=int, default=None, help="reach: number of sources (fewer for a small profiling case)")
+    ap.add_argument("--triangle-plan", default="auto", choices=["auto", "wcoj", "chain"], help="wcoj workload: force a join plan")
     ap.add_argument("--no-graph", action="store_true", help="launch the resident rounds one by one (for per-launch profiling)")
     ap.add_argument("--no-tag-mirror", action="store_true", help="evaluate recursion by sort -> reduce-by-key -> merge only")
     ap.add_argument("--cpu-scale", type=int, default=None, help="R-MAT scale of the cpu_baseline sample (default: the workload's)")

@@ -528,7 +528,7 @@ void count_variant(Ctx* c, const Variant& v, const Relation& H, Counted& q, int 
   q.start = DevBuf(c, (size_t)n * 8); q.sums = DevBuf(c, (size_t)tiles * 8);
   DISPATCH_K(v.outer.key_bytes, XLOG_LAUNCH(c, (k_join_count<K>), (n + 255) / 256, 256, 0, q.spec, (const K*)v.outer.keys, v.outer.tags, n,
                                              q.deg.as<uint32_t>(), q.rowinfo.as<uint4>(), ctrl_u32(c, kSlotErr)));
-  if (n <= (1u << 16)) {
+  if (n <= (1u << 13)) {
     XLOG_LAUNCH(c, (k_scan_block<uint32_t, uint64_t>), 1, 1024, 0, (const uint32_t*)q.deg.as<uint32_t>(), (int64_t)n, q.start.as<uint64_t>(),
                 (uint64_t*)(c->d_ctrl + q.slot));
     return;
