@@ -389,9 +389,9 @@ __device__ __forceinline__ void expand_tile(ExpSmem<ExpShapeT<SINK != kSinkWrite
         key[k] = (KH)(((uint64_t)info.w << 32) | info.z);
         tag[k] = __uint_as_float(info.y);
         if (nin >= 0) {
-          const float it = itg[ir];
+          const float it = __ldcs(itg + ir);                 // streamed once: evict first, the slots should stay in L2
           tag[k] = times ? tag[k] * it : tag[k] + it;
-          if (nin >= 1) key[k] += (KH)(uint32_t)ic0[ir] * m0;
+          if (nin >= 1) key[k] += (KH)(uint32_t)__ldcs(ic0 + ir) * m0;
           for (int c = 1; c < nin; ++c) key[k] += (KH)(uint32_t)S.inner_col[c][ir] * (KH)S.inner_mult[c];
         }
       }
