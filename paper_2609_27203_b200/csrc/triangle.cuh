@@ -27,38 +27,72 @@ struct TriGraph {
   const float* in_w;             // and their tags
 };
 
+constexpr uint32_t kTriChunk = 1024;     // walked entries per work item (32 sweeps of a warp)
+
+// Work items of the aggregate: an edge whose shorter list has n entries is cut into ceil(n / kTriChunk) items, so that a
+// hub edge (tens of thousands of entries to walk) is shared by many warps instead of serialising one; an edge with an
+// empty list gets none.  items[e] for e < n_edges, items[n_edges] = 0 (so that the exclusive scan has n_edges + 1 entries).
+static __global__ void __launch_bounds__(256) k_tri_plan(TriGraph G, uint32_t* __restrict__ items) {
+  for (uint32_t e = blockIdx.x * blockDim.x + threadIdx.x; e <= G.n_edges; e += gridDim.x * blockDim.x) {
+    uint32_t n = 0;
+    if (e < G.n_edges) {
+      const int32_t x = G.src[e], y = G.dst[e];
+      uint32_t la = 0, lb = 0;
+      if (y < G.out_domain) la = G.out_off[y + 1] - G.out_off[y];
+      if (x < G.in_domain) lb = G.in_off[x + 1] - G.in_off[x];
+      n = (min(la, lb) + kTriChunk - 1) / kTriChunk;
+    }
+    items[e] = n;
+  }
+}
+
+// item -> edge, written by the edge (item_off = exclusive scan of items)
+static __global__ void __launch_bounds__(256) k_tri_item_edges(uint32_t n_edges, const uint32_t* __restrict__ item_off, uint32_t* __restrict__ item_edge) {
+  for (uint32_t e = blockIdx.x * blockDim.x + threadIdx.x; e < n_edges; e += gridDim.x * blockDim.x)
+    for (uint32_t it = item_off[e]; it < item_off[e + 1]; ++it) item_edge[it] = e;
+}
+
+// One warp per work item: partial count and aggregate of its slice of the walked list.
 template <typename Op>
-__global__ void __launch_bounds__(256) k_tri_edges(TriGraph G, int times, uint32_t* __restrict__ edge_cnt,
-                                                   typename Op::A* __restrict__ edge_acc) {
+__global__ void __launch_bounds__(256) k_tri_edges(TriGraph G, int times, uint32_t n_items, const uint32_t* __restrict__ item_off,
+                                                   const uint32_t* __restrict__ item_edge, uint32_t* __restrict__ item_cnt,
+                                                   typename Op::A* __restrict__ item_acc) {
   typedef typename Op::A A;
   const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
   const unsigned lane = lane_id();
-  for (uint32_t e = warp; e < G.n_edges; e += nwarps) {
+  for (uint32_t it = warp; it < n_items; it += nwarps) {
+    const uint32_t e = item_edge[it];
+    const uint32_t first = (it - item_off[e]) * kTriChunk;                     // this item's slice of the walked list
     const int32_t x = G.src[e], y = G.dst[e];
     const float wxy = G.w[e];
-    uint32_t a0 = 0, a1 = 0, b0 = 0, b1 = 0;
-    if (y < G.out_domain) { a0 = G.out_off[y]; a1 = G.out_off[y + 1]; }      // out(y): candidates z with e(y,z)
-    if (x < G.in_domain) { b0 = G.in_off[x]; b1 = G.in_off[x + 1]; }         // in(x):  candidates z with e(z,x)
+    const uint32_t a0 = G.out_off[y], a1 = G.out_off[y + 1];                   // out(y): candidates z with s(y,z)
+    const uint32_t b0 = G.in_off[x], b1 = G.in_off[x + 1];                     // in(x):  candidates z with t(z,x)
     const uint32_t la = a1 - a0, lb = b1 - b0;
     uint32_t cnt = 0;
     A acc = Op::identity();
-    if (la && lb) {
-      const bool walk_a = la <= lb;
-      const int32_t* wl = walk_a ? G.s_dst + a0 : G.in_src + b0;                // walked list
-      const int32_t* sl = walk_a ? G.in_src + b0 : G.s_dst + a0;                // searched list
-      const uint32_t nw = walk_a ? la : lb, ns = walk_a ? lb : la;
-      for (uint32_t i = lane; i < nw; i += 32) {
-        const int32_t z = wl[i];
-        uint32_t lo = 0, hi = ns;
+    const bool walk_a = la <= lb;
+    const int32_t* wl = walk_a ? G.s_dst + a0 : G.in_src + b0;                  // walked list
+    const int32_t* sl = walk_a ? G.in_src + b0 : G.s_dst + a0;                  // searched list
+    const uint32_t nw = walk_a ? la : lb, ns = walk_a ? lb : la;
+    const uint32_t last = min(first + kTriChunk, nw);
+    // the walked list ascends, so whatever the last lane found in one sweep bounds every search of the next sweep
+    uint32_t floor = 0;
+    for (uint32_t i0 = first; i0 < last; i0 += 32) {
+      const uint32_t i = i0 + lane;
+      uint32_t lo = floor, hi = ns;
+      int32_t z = 0;
+      if (i < last) {
+        z = wl[i];
         while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (sl[mid] < z) lo = mid + 1; else hi = mid; }
-        if (lo < ns && sl[lo] == z) {
-          const float wyz = walk_a ? G.s_w[a0 + i] : G.s_w[a0 + lo];
-          const float wzx = walk_a ? G.in_w[b0 + lo] : G.in_w[b0 + i];
-          const float t = times ? (wxy * wyz) * wzx : (wxy + wyz) + wzx;
-          acc = Op::combine(acc, Op::lift(t));
-          ++cnt;
-        }
+      }
+      floor = __shfl_sync(0xffffffffu, lo, 31);
+      if (i < last && lo < ns && sl[lo] == z) {
+        const float wyz = walk_a ? G.s_w[a0 + i] : G.s_w[a0 + lo];
+        const float wzx = walk_a ? G.in_w[b0 + lo] : G.in_w[b0 + i];
+        const float t = times ? (wxy * wyz) * wzx : (wxy + wyz) + wzx;
+        acc = Op::combine(acc, Op::lift(t));
+        ++cnt;
       }
     }
 #pragma unroll
@@ -67,13 +101,50 @@ __global__ void __launch_bounds__(256) k_tri_edges(TriGraph G, int times, uint32
       const A o = shfl_down(acc, d);
       acc = Op::combine(acc, o);
     }
-    if (lane == 0) { edge_cnt[e] = cnt; edge_acc[e] = acc; }
+    if (lane == 0) { item_cnt[it] = cnt; item_acc[it] = acc; }
   }
 }
 
-// One warp per x: combine the partials of its edges (contiguous), write count, tag and a presence flag.
+// Matches per edge (the count step of the materialising variant): one warp per edge.
+static __global__ void __launch_bounds__(256) k_tri_count_edges(TriGraph G, uint32_t* __restrict__ edge_cnt) {
+  const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+  const unsigned lane = lane_id();
+  for (uint32_t e = warp; e < G.n_edges; e += nwarps) {
+    const int32_t x = G.src[e], y = G.dst[e];
+    uint32_t a0 = 0, a1 = 0, b0 = 0, b1 = 0;
+    if (y < G.out_domain) { a0 = G.out_off[y]; a1 = G.out_off[y + 1]; }
+    if (x < G.in_domain) { b0 = G.in_off[x]; b1 = G.in_off[x + 1]; }
+    const uint32_t la = a1 - a0, lb = b1 - b0;
+    uint32_t cnt = 0;
+    if (la && lb) {
+      const bool walk_a = la <= lb;
+      const int32_t* wl = walk_a ? G.s_dst + a0 : G.in_src + b0;
+      const int32_t* sl = walk_a ? G.in_src + b0 : G.s_dst + a0;
+      const uint32_t nw = walk_a ? la : lb, ns = walk_a ? lb : la;
+      uint32_t floor = 0;
+      for (uint32_t i0 = 0; i0 < nw; i0 += 32) {
+        const uint32_t i = i0 + lane;
+        uint32_t lo = floor, hi = ns;
+        int32_t z = 0;
+        if (i < nw) {
+          z = wl[i];
+          while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (sl[mid] < z) lo = mid + 1; else hi = mid; }
+        }
+        floor = __shfl_sync(0xffffffffu, lo, 31);
+        if (i < nw && lo < ns && sl[lo] == z) ++cnt;
+      }
+    }
+#pragma unroll
+    for (int d = 16; d; d >>= 1) cnt += __shfl_down_sync(0xffffffffu, cnt, d);
+    if (lane == 0) edge_cnt[e] = cnt;
+  }
+}
+
+// One warp per x: combine the partials of the work items of its edges (contiguous, in edge and slice order), write count,
+// tag and a presence flag.
 template <typename Op>
-__global__ void __launch_bounds__(256) k_tri_groups(const uint32_t* __restrict__ out_off, int64_t domain,
+__global__ void __launch_bounds__(256) k_tri_groups(const uint32_t* __restrict__ out_off, int64_t domain, const uint32_t* __restrict__ item_off,
                                                     const uint32_t* __restrict__ edge_cnt, const typename Op::A* __restrict__ edge_acc,
                                                     uint32_t* __restrict__ grp_cnt, float* __restrict__ grp_tag,
                                                     uint32_t* __restrict__ flag, uint32_t* __restrict__ max_cnt,
@@ -83,7 +154,7 @@ __global__ void __launch_bounds__(256) k_tri_groups(const uint32_t* __restrict__
   const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
   const unsigned lane = lane_id();
   for (int64_t x = warp; x < domain; x += nwarps) {
-    const uint32_t e0 = out_off[x], e1 = out_off[x + 1];
+    const uint32_t e0 = item_off[out_off[x]], e1 = item_off[out_off[x + 1]];
     uint64_t cnt = 0;
     A acc = Op::identity();
     for (uint32_t e = e0 + lane; e < e1; e += 32) {
@@ -131,17 +202,19 @@ __global__ void __launch_bounds__(256) k_tri_materialise(TriGraph G, int times, 
     const uint32_t nw = walk_a ? la : lb, ns = walk_a ? lb : la;
     uint64_t pos = edge_off[e];
     const K xy = ((K)(uint32_t)x << L.shift[0]) | ((K)(uint32_t)y << L.shift[1]);
+    uint32_t floor = 0;                                   // see k_tri_edges
     for (uint32_t i0 = 0; i0 < nw; i0 += 32) {
       const uint32_t i = i0 + lane;
       bool hit = false;
       int32_t z = 0;
-      uint32_t lo = 0;
+      uint32_t lo = floor;
       if (i < nw) {
         z = wl[i];
         uint32_t hi = ns;
         while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if (sl[mid] < z) lo = mid + 1; else hi = mid; }
         hit = lo < ns && sl[lo] == z;
       }
+      floor = __shfl_sync(0xffffffffu, lo, 31);
       const unsigned m = __ballot_sync(0xffffffffu, hit);
       if (hit) {
         const float wyz = walk_a ? G.s_w[a0 + i] : G.s_w[a0 + lo];

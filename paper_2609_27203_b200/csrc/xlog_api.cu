@@ -849,15 +849,32 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
   G.in_src = in_ix.other[0]; G.in_w = in_ix.tags;
   G.s_dst = G.dst; G.s_w = G.w;
   const int64_t domain = out_ix.domain;
-  DevBuf ecnt(c, (size_t)E.n * 4), eacc(c, (size_t)E.n * sizeof(A));
+  // work items: edges cut into slices of the walked list (count -> scan -> one control read for the item total)
+  const uint32_t ne1 = E.n + 1;
+  DevBuf items(c, (size_t)ne1 * 4), item_off(c, (size_t)ne1 * 4);
+  const unsigned it_tiles = (ne1 + kScanTile - 1) / kScanTile;
+  DevBuf it_sums(c, (size_t)it_tiles * 4);
+  zero_ctrl(c, kSlotA, 4);
+  XLOG_LAUNCH(c, k_tri_plan, grid_for(ne1, 256), 256, 0, G, items.as<uint32_t>());
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), it_tiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ne1, it_sums.as<uint32_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, it_sums.as<uint32_t>(), (int64_t)it_tiles, ctrl_u32(c, kSlotB));
+  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), it_tiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ne1,
+              (const uint32_t*)it_sums.as<uint32_t>(), item_off.as<uint32_t>());
+  sync_ctrl(c);
+  const uint32_t n_items = (uint32_t)c->h_ctrl[kSlotB];
+  items.reset(); it_sums.reset();
+  DevBuf item_edge(c, (size_t)std::max(n_items, 1u) * 4), ecnt(c, (size_t)std::max(n_items, 1u) * 4), eacc(c, (size_t)std::max(n_items, 1u) * sizeof(A));
   DevBuf gcnt(c, (size_t)domain * 4), gtag(c, (size_t)domain * 4), flag(c, (size_t)domain * 4);
   const unsigned scan_tiles = (unsigned)((domain + kScanTile - 1) / kScanTile);
   DevBuf spine(c, ((size_t)scan_tiles + 1) * 4);
   zero_ctrl(c, kSlotA, 4);
+  XLOG_LAUNCH(c, k_tri_item_edges, grid_for(E.n, 256), 256, 0, E.n, (const uint32_t*)item_off.as<uint32_t>(), item_edge.as<uint32_t>());
   c->note_bytes = (int64_t)E.n * 12 * 3;      // each edge is read as (x,y), inside an out-list and inside an in-list; partials are small
-  XLOG_LAUNCH(c, (k_tri_edges<Op>), kSMs * 8, 256, 0, G, H.sr == XLOG_SR_SUMPROD ? 1 : 0, ecnt.as<uint32_t>(), eacc.as<A>());
-  XLOG_LAUNCH(c, (k_tri_groups<Op>), grid_for((uint64_t)domain * 32, 256, kSMs * 8), 256, 0, G.out_off, domain, (const uint32_t*)ecnt.as<uint32_t>(),
-              (const A*)eacc.as<A>(), gcnt.as<uint32_t>(), gtag.as<float>(), flag.as<uint32_t>(), ctrl_u32(c, kSlotD), ctrl_u32(c, kSlotErr));
+  XLOG_LAUNCH(c, (k_tri_edges<Op>), kSMs * 8, 256, 0, G, H.sr == XLOG_SR_SUMPROD ? 1 : 0, n_items, (const uint32_t*)item_off.as<uint32_t>(),
+              (const uint32_t*)item_edge.as<uint32_t>(), ecnt.as<uint32_t>(), eacc.as<A>());
+  XLOG_LAUNCH(c, (k_tri_groups<Op>), grid_for((uint64_t)domain * 32, 256, kSMs * 8), 256, 0, G.out_off, domain, (const uint32_t*)item_off.as<uint32_t>(),
+              (const uint32_t*)ecnt.as<uint32_t>(), (const A*)eacc.as<A>(), gcnt.as<uint32_t>(), gtag.as<float>(), flag.as<uint32_t>(), ctrl_u32(c, kSlotD),
+              ctrl_u32(c, kSlotErr));
   // positions of the surviving x: exclusive scan of the flags (kept in a second buffer)
   DevBuf pos(c, (size_t)domain * 4);
   XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), scan_tiles, kScanBlock, 0, (const uint32_t*)flag.as<uint32_t>(), domain, spine.as<uint32_t>());
@@ -986,11 +1003,11 @@ void triangle_materialise(Ctx* c, Relation& H, const RuleC& r) {
   G.out_off = out_ix.off.as<uint32_t>(); G.in_off = in_ix.off.as<uint32_t>();
   G.s_dst = out_ix.other[0]; G.s_w = out_ix.tags;
   G.in_src = in_ix.other[0]; G.in_w = in_ix.tags;
-  DevBuf ecnt(c, (size_t)R.n * 4), eacc(c, (size_t)R.n * 4), eoff(c, (size_t)R.n * 8);
+  DevBuf ecnt(c, (size_t)R.n * 4), eoff(c, (size_t)R.n * 8);
   const unsigned tiles = (R.n + kScanTile - 1) / kScanTile;
   DevBuf sums(c, (size_t)tiles * 8);
   c->note_bytes = (int64_t)(R.n + S.n + T.n) * 12;
-  XLOG_LAUNCH(c, (k_tri_edges<OpMax>), kSMs * 8, 256, 0, G, times, ecnt.as<uint32_t>(), eacc.as<float>());
+  XLOG_LAUNCH(c, k_tri_count_edges, kSMs * 8, 256, 0, G, ecnt.as<uint32_t>());
   XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)ecnt.as<uint32_t>(), (int64_t)R.n, sums.as<uint64_t>());
   XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, sums.as<uint64_t>(), (int64_t)tiles, (uint64_t*)(c->d_ctrl + kSlotTotals));
   XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)ecnt.as<uint32_t>(), (int64_t)R.n,
