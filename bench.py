@@ -254,8 +254,14 @@ def run_ours(args):
     if mirror_kernel:
         ratio = NCU_TRAFFIC_RATIO_MIRROR.get(dom)
     bound = "hbm"
+    alu = None
     if dom.startswith("k_tri"):
-        bound = "alu"      # sorted-list intersections served from L2: compare and branch work, not an HBM-bound kernel
+        bound = "alu"      # sorted-list intersections served from L1 / L2: compare and branch work, not an HBM-bound kernel
+        # unit of work: one probe (binary search of a walked entry in the other sorted list).  ncu: 6.5 warp instructions per probe at
+        # R-MAT scale 18, so the issue-rate ceiling is 148 SMs x 4 schedulers x 1.965e9 / 6.5 probes per second.
+        if dom == "k_tri_edges" and "n_edges" in program.info:
+            probes = (d["bytes"] - 12.0 * program.info["n_edges"] * d["launches"]) / 4.0
+            alu = {"achieved": probes / (d["ms"] / 1e3) / 1e9, "peak": 148 * 4 * 1.965 / 6.5, "unit": "Gprobe/s"}
     roofline = {"bound": bound, "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src,
                 "traffic": None if ratio is None else ratio * d["bytes"] / d["launches"],
@@ -266,6 +272,9 @@ def run_ours(args):
                             for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])},
                 "how": "second pass of the same steps with XLOG_FLAG_PROFILE (CUDA events around every launch on the ctx stream; "
                        "the resident rounds are then launched one by one instead of as one graph)"}
+    if alu:
+        roofline.update(achieved=alu["achieved"], peak=alu["peak"], unit=alu["unit"], frac=alu["achieved"] / alu["peak"], traffic=None,
+                        peak_source="derived: issue slots x clock / measured warp instructions per probe")
     if mirror_kernel:
         # one random 32-byte L2 sector per candidate (the key's slot in the tag mirror) on top of the streamed adjacency
         # reads: the kernel is bound by how many such sector requests the SMs keep in flight, not by HBM

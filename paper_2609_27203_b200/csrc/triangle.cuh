@@ -32,7 +32,9 @@ constexpr uint32_t kTriChunk = 1024;     // walked entries per work item (32 swe
 // Work items of the aggregate: an edge whose shorter list has n entries is cut into ceil(n / kTriChunk) items, so that a
 // hub edge (tens of thousands of entries to walk) is shared by many warps instead of serialising one; an edge with an
 // empty list gets none.  items[e] for e < n_edges, items[n_edges] = 0 (so that the exclusive scan has n_edges + 1 entries).
-static __global__ void __launch_bounds__(256) k_tri_plan(TriGraph G, uint32_t* __restrict__ items) {
+// *walked accumulates the total number of entries to walk (one sorted-list probe each).
+static __global__ void __launch_bounds__(256) k_tri_plan(TriGraph G, uint32_t* __restrict__ items, unsigned long long* __restrict__ walked) {
+  unsigned long long mine = 0;
   for (uint32_t e = blockIdx.x * blockDim.x + threadIdx.x; e <= G.n_edges; e += gridDim.x * blockDim.x) {
     uint32_t n = 0;
     if (e < G.n_edges) {
@@ -41,9 +43,13 @@ static __global__ void __launch_bounds__(256) k_tri_plan(TriGraph G, uint32_t* _
       if (y < G.out_domain) la = G.out_off[y + 1] - G.out_off[y];
       if (x < G.in_domain) lb = G.in_off[x + 1] - G.in_off[x];
       n = (min(la, lb) + kTriChunk - 1) / kTriChunk;
+      mine += min(la, lb);
     }
     items[e] = n;
   }
+#pragma unroll
+  for (int d = 16; d; d >>= 1) mine += __shfl_down_sync(0xffffffffu, mine, d);
+  if (lane_id() == 0 && mine) atomicAdd(walked, mine);
 }
 
 // item -> edge, written by the edge (item_off = exclusive scan of items)

@@ -855,13 +855,14 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
   const unsigned it_tiles = (ne1 + kScanTile - 1) / kScanTile;
   DevBuf it_sums(c, (size_t)it_tiles * 4);
   zero_ctrl(c, kSlotA, 4);
-  XLOG_LAUNCH(c, k_tri_plan, grid_for(ne1, 256), 256, 0, G, items.as<uint32_t>());
+  XLOG_LAUNCH(c, k_tri_plan, grid_for(ne1, 256), 256, 0, G, items.as<uint32_t>(), (unsigned long long*)(c->d_ctrl + kSlotC));
   XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), it_tiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ne1, it_sums.as<uint32_t>());
   XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, it_sums.as<uint32_t>(), (int64_t)it_tiles, ctrl_u32(c, kSlotB));
   XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), it_tiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ne1,
               (const uint32_t*)it_sums.as<uint32_t>(), item_off.as<uint32_t>());
   sync_ctrl(c);
   const uint32_t n_items = (uint32_t)c->h_ctrl[kSlotB];
+  const uint64_t walked = c->h_ctrl[kSlotC];               // sorted-list probes of the whole join
   items.reset(); it_sums.reset();
   DevBuf item_edge(c, (size_t)std::max(n_items, 1u) * 4), ecnt(c, (size_t)std::max(n_items, 1u) * 4), eacc(c, (size_t)std::max(n_items, 1u) * sizeof(A));
   DevBuf gcnt(c, (size_t)domain * 4), gtag(c, (size_t)domain * 4), flag(c, (size_t)domain * 4);
@@ -869,7 +870,9 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
   DevBuf spine(c, ((size_t)scan_tiles + 1) * 4);
   zero_ctrl(c, kSlotA, 4);
   XLOG_LAUNCH(c, k_tri_item_edges, grid_for(E.n, 256), 256, 0, E.n, (const uint32_t*)item_off.as<uint32_t>(), item_edge.as<uint32_t>());
-  c->note_bytes = (int64_t)E.n * 12 * 3;      // each edge is read as (x,y), inside an out-list and inside an in-list; partials are small
+  // declared work: one 4-byte entry per probe (the walked lists) plus the edge rows; the searches themselves hit L1 / L2
+  c->note_bytes = (int64_t)walked * 4 + (int64_t)E.n * 12;
+  c->r_candidates += (int64_t)walked;
   XLOG_LAUNCH(c, (k_tri_edges<Op>), kSMs * 8, 256, 0, G, H.sr == XLOG_SR_SUMPROD ? 1 : 0, n_items, (const uint32_t*)item_off.as<uint32_t>(),
               (const uint32_t*)item_edge.as<uint32_t>(), ecnt.as<uint32_t>(), eacc.as<A>());
   XLOG_LAUNCH(c, (k_tri_groups<Op>), grid_for((uint64_t)domain * 32, 256, kSMs * 8), 256, 0, G.out_off, domain, (const uint32_t*)item_off.as<uint32_t>(),
@@ -883,7 +886,7 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
               (const uint32_t*)spine.as<uint32_t>(), pos.as<uint32_t>());
   sync_ctrl(c);
   const uint32_t u = (uint32_t)c->h_ctrl[kSlotA], max_count = (uint32_t)c->h_ctrl[kSlotD];
-  c->r_candidates += 0; c->r_unique += u;
+  c->r_unique += u;
   KeyTags kt;
   kt.n = u;
   const int kb = cl.total_bits <= 32 ? 4 : 8;
