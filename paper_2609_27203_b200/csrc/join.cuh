@@ -193,13 +193,15 @@ __global__ void __launch_bounds__(256) k_join_count(JoinSpec S, const KO* __rest
 // Measured on the two large workloads (single-source R-MAT 20 / 64-source R-MAT 22, ms per fixpoint; items, staged
 // rows, blocks per SM): 8, 1024, 5: 0.62 / 34.6; 8, 1024, 6: 0.63 / 32.7; 6, 768, 6: 0.60 / 31.5; 6, 768, 7: 0.61 / 29.3;
 // 4, 512, 8 (64 warps, no spills): 0.58 / 29.0.
-// The kernel that writes candidates (streaming, HBM-bound) keeps the larger tile: 8 items, 2048 rows, 4 blocks per SM.
+// The kernel that writes candidates (streaming) keeps 8 items per thread; it, too, gains from residency: on the 64-source
+// workload 2048 staged rows at 5 blocks per SM ran at 2.9 TB/s of algorithmic traffic, 1024 rows at 8 blocks (32 registers) at 3.9 TB/s.
 constexpr int kExpBlock = 256;
-constexpr int kExpMirrorBlocksPerSM = 8;              // occupancy asked of the tag-mirror instantiations
+constexpr int kExpMirrorBlocksPerSM = 8;
+constexpr int kExpWriteBlocksPerSM = 8;               // and of the candidate-writing ones
 template <bool MIRROR> struct ExpShapeT {
   static constexpr int items = MIRROR ? 4 : 8;        // candidates per thread
   static constexpr int tile = kExpBlock * items;      // candidates per block
-  static constexpr int rows = MIRROR ? 512 : 2048;    // outer rows staged in shared memory per tile
+  static constexpr int rows = MIRROR ? 512 : 1024;    // outer rows staged in shared memory per tile
 };
 constexpr int kExpTileWrite = ExpShapeT<false>::tile, kExpTileMirror = ExpShapeT<true>::tile;
 
@@ -503,7 +505,7 @@ __device__ __forceinline__ void expand_tile(ExpSmem<ExpShapeT<SINK != kSinkWrite
 // staged in shared memory (their starts relative to the tile and their row records), so the per-
 // candidate work is a short binary search in shared memory plus the coalesced inner reads.
 template <typename KO, typename KH, int MODE, int SINK = kSinkWrite>
-__global__ void __launch_bounds__(kExpBlock, SINK == kSinkWrite ? 5 : kExpMirrorBlocksPerSM) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
+__global__ void __launch_bounds__(kExpBlock, SINK == kSinkWrite ? kExpWriteBlocksPerSM : kExpMirrorBlocksPerSM) k_join_expand(JoinSpec S, const KO* __restrict__ okeys, uint32_t n_outer,
                                                            const uint64_t* __restrict__ start, const uint4* __restrict__ rowinfo,
                                                            const uint2* __restrict__ tile_rows, uint64_t out_lo, uint64_t out_hi,
                                                            KH* __restrict__ ckeys,
