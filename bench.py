@@ -200,7 +200,7 @@ def run_ours(args):
     program, arena = make_program(args.workload, args.scale, args.sources)
 
     # facts resident in HBM before any timed region
-    base_flags = (xlog.FLAG_NO_TAG_MIRROR if args.no_tag_mirror else 0) | (xlog.FLAG_NO_GRAPH if args.no_graph else 0)
+    base_flags = (xlog.FLAG_NO_TAG_MIRROR if args.no_tag_mirror else 0) | (xlog.FLAG_NO_GRAPH if args.no_graph else 0) | (xlog.FLAG_NO_RESIDENT_LOOP if args.no_resident_loop else 0)
     base_flags |= {"auto": 0, "wcoj": xlog.FLAG_FORCE_WCOJ, "chain": xlog.FLAG_FORCE_CHAIN}[args.triangle_plan]
     ctx, ids, rules = xlog.load_program(program, device=local_rank, arena_bytes=arena, device_inputs=True, flags=base_flags)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)          # > 126 MB L2
@@ -391,6 +391,7 @@ def main():
     ap.add_argument("--scale", type=int, default=None, help="R-MAT scale override (smaller cases for profiling)")
     ap.add_argument("--sources", type=int, default=None, help="reach: number of sources (fewer for a small profiling case)")
     ap.add_argument("--triangle-plan", default="auto", choices=["auto", "wcoj", "chain"], help="wcoj workload: force a join plan")
+    ap.add_argument("--no-resident-loop", action="store_true", help="tag-mirror rounds driven by the host (one control read per round)")
     ap.add_argument("--no-graph", action="store_true", help="launch the resident rounds one by one (for per-launch profiling)")
     ap.add_argument("--no-tag-mirror", action="store_true", help="evaluate recursion by sort -> reduce-by-key -> merge only")
     ap.add_argument("--cpu-scale", type=int, default=None, help="R-MAT scale of the cpu_baseline sample (default: the workload's)")
