@@ -78,6 +78,7 @@ typedef struct {
 #define XLOG_FLAG_NO_RESIDENT_LOOP 8u  /* the host drives every round of a tag-mirror fixpoint (one control read per round) */
 #define XLOG_FLAG_FORCE_WCOJ      32u  /* materialised triangle joins: always the multiway (worst-case-optimal) plan */
 #define XLOG_FLAG_FORCE_CHAIN     64u  /* ... always the binary-join chain (fails with RESOURCE_EXHAUSTED if its intermediate does not fit) */
+#define XLOG_FLAG_NO_GROUPED_JOIN 128u  /* tag mirror: always the row-wise join, never the grouped one (see csrc/group_join.cuh) */
 #define XLOG_FLAG_NO_GRAPH        16u  /* resident rounds are launched one by one instead of as one graph with a WHILE node */
 
 /* Evaluation routes of a recursive component (Algorithm 1).  All of them derive the same relation,

@@ -20,12 +20,22 @@ namespace xlog {
 constexpr int kMirBlock = 256;
 constexpr int kMirSlotsPerTile = kMirBlock * 16;       // table slots per tile (four int4 per thread)
 
+// `from` / `to`: the relation's own key layout and the mirror's (the same columns, possibly with the order of
+// significance changed: see group_join.cuh)
+__device__ __forceinline__ uint32_t relayout_key(const KeyLayout& from, const KeyLayout& to, uint32_t key) {
+  uint32_t out = 0;
+#pragma unroll
+  for (int c = 0; c < kMaxArity; ++c)
+    if (c < from.arity) out |= (uint32_t)key_col<uint32_t>(from, key, c) << to.shift[c];
+  return out;
+}
+
 template <typename K>
 __global__ void __launch_bounds__(256) k_mirror_scatter(const K* __restrict__ keys, const float* __restrict__ tags, uint32_t n,
-                                                        int32_t* __restrict__ table, uint32_t* __restrict__ present) {
+                                                        KeyLayout from, KeyLayout to, int32_t* __restrict__ table, uint32_t* __restrict__ present) {
   const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) {
-    const uint32_t key = (uint32_t)keys[i];
+    const uint32_t key = relayout_key(from, to, (uint32_t)keys[i]);
     table[key] = f2ord(tags[i]);
     atomicOr(present + (key >> 5), 1u << (key & 31));
   }
@@ -117,8 +127,8 @@ static __global__ void __launch_bounds__(kMirBlock) k_mirror_full_count(const in
 
 template <typename K>
 __global__ void __launch_bounds__(kMirBlock) k_mirror_full_emit(const int4* __restrict__ table4, uint64_t nquads, int32_t empty,
-                                                                const uint32_t* __restrict__ tile_base, K* __restrict__ keys,
-                                                                float* __restrict__ tags) {
+                                                                const uint32_t* __restrict__ tile_base, KeyLayout from, KeyLayout to,
+                                                                K* __restrict__ keys, float* __restrict__ tags) {
   __shared__ uint32_t sh[kMirBlock / 32 + 1];
   uint32_t run = tile_base[blockIdx.x];
 #pragma unroll
@@ -134,7 +144,7 @@ __global__ void __launch_bounds__(kMirBlock) k_mirror_full_emit(const int4* __re
 #pragma unroll
     for (int j = 0; j < 4; ++j)
       if (e[j] != empty) {
-        keys[pos] = (K)(q * 4 + j);
+        keys[pos] = (K)relayout_key(from, to, (uint32_t)(q * 4 + j));      // slot index (mirror layout) -> the relation's key
         tags[pos] = ord2f(e[j]);
         ++pos;
       }

@@ -1,5 +1,6 @@
 // C ABI of the engine (see include/xlog.h) and the host-side fixpoint driver.
 #include "engine.cuh"
+#include "group_join.cuh"
 #include "mirror.cuh"
 #include "resident.cuh"
 #include "triangle.cuh"
@@ -367,7 +368,7 @@ struct Counted {                         // a variant after count + scan
   int slot = 0;
 };
 
-JoinSpec make_spec(Ctx* c, const Variant& v, const Relation& H) {
+JoinSpec make_spec(Ctx* c, const Variant& v, const Relation& H, const KeyLayout* head_layout = nullptr) {
   const xlog_plan& p = v.rule->plan;
   JoinSpec S;
   memset(&S, 0, sizeof S);                 // padding included: specs are compared byte for byte (graph reuse)
@@ -428,7 +429,7 @@ JoinSpec make_spec(Ctx* c, const Variant& v, const Relation& H) {
     }
     if (pass) { S.outer_decode[i] = 0; S.head_encode[i] = 0; }
   }
-  S.head = H.layout;
+  S.head = head_layout ? *head_layout : H.layout;      // a tag mirror may order the head's columns its own way
   if (p.emit_count_column) {             // candidates are keyed by the declared head columns only
     int32_t mx[kMaxArity] = {0, 0, 0, 0};
     for (int i = 0; i < p.n_head_cols; ++i) mx[i] = H.col_max[i];
@@ -501,8 +502,8 @@ JoinSpec make_spec(Ctx* c, const Variant& v, const Relation& H) {
 }
 
 // count -> scan for one variant; the grand total lands in control slot `slot` (read after sync_ctrl)
-void count_variant(Ctx* c, const Variant& v, const Relation& H, Counted& q, int slot) {
-  q.spec = make_spec(c, v, H);
+void count_variant(Ctx* c, const Variant& v, const Relation& H, Counted& q, int slot, const KeyLayout* head_layout = nullptr) {
+  q.spec = make_spec(c, v, H, head_layout);
   q.outer = v.outer;
   q.slot = slot;
   {
@@ -1317,6 +1318,123 @@ ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*
   return out;
 }
 
+// ---- grouped join (group_join.cuh) -----------------------------------------------------------------------
+// The shape  h(a, c) :- h(a, b), r(b, c)  for every rule over h (binary h; a and b bare variables; c the looked-up
+// relation's other column).
+bool grouped_shape(Ctx* c, int h, const std::vector<const RuleC*>& rs) {
+  const Relation& H = *c->rels[h];
+  if (H.arity != 2) return false;
+  bool any = false;
+  for (const RuleC* r : rs) {
+    int j = -1;
+    for (int k = 0; k < r->plan.n_atoms; ++k) if (r->plan.atoms[k].rel == h) j = k;
+    if (j < 0) continue;
+    if (r->kind != 2 || !r->shape[j].ok) return false;
+    const xlog_plan& p = r->plan;
+    const xlog_atom& A = p.atoms[j];
+    const xlog_atom& B = p.atoms[1 - j];
+    if (!is_plain_var(A.args[0]) || !is_plain_var(A.args[1]) || A.args[0].var == A.args[1].var) return false;
+    if (c->rels[B.rel]->arity != 2 || r->shape[j].probe_col != 0 || r->shape[j].probe_var != A.args[1].var || r->shape[j].probe_mul != 1 ||
+        r->shape[j].probe_add != 0 || !is_plain_var(B.args[1]))
+      return false;
+    const int hv[2] = {A.args[0].var, B.args[1].var};
+    for (int col = 0; col < 2; ++col) {
+      if (p.head[col].c0 != 0) return false;
+      for (int v = 0; v < XLOG_MAX_VARS; ++v) if (p.head[col].coef[v] != (v == hv[col] ? 1 : 0)) return false;
+    }
+    any = true;
+  }
+  return any;
+}
+
+constexpr int kSlotSeg = 14;               // segment totals (low word: all, high word: with matches), then the candidate total
+
+// One delta variant through the grouped join.  Returns the candidate total, or UINT64_MAX when the compiled rule turns
+// out not to have the linear-key form (the caller then takes the row-wise join).
+uint64_t grouped_apply(Ctx* c, const Variant& v, const Relation& H, const KeyLayout& M, int carried_bits, bool is_max, const MirrorArgs& mr) {
+  const JoinSpec S = make_spec(c, v, H, &M);
+  if (!S.fast || !S.has_inner || S.inner_free != 1 || v.outer.key_bytes != 4) return UINT64_MAX;
+  const uint32_t n = v.outer.n;
+  const unsigned tiles = (n + kScanTile - 1) / kScanTile;
+  DevBuf deg(c, (size_t)n * 4), rowinfo(c, (size_t)n * 16), flags(c, (size_t)n * 8), idx(c, (size_t)n * 8), sums(c, (size_t)tiles * 8);
+  XLOG_LAUNCH(c, (k_join_count<uint32_t>), (n + 255) / 256, 256, 0, S, (const uint32_t*)v.outer.keys, v.outer.tags, n, deg.as<uint32_t>(),
+              rowinfo.as<uint4>(), ctrl_u32(c, kSlotErr));
+  XLOG_LAUNCH(c, k_seg_flags, grid_for(n, 256), 256, 0, (const uint32_t*)v.outer.keys, (const uint32_t*)deg.as<uint32_t>(), n, carried_bits, flags.as<uint64_t>());
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint64_t, uint64_t>), tiles, kScanBlock, 0, (const uint64_t*)flags.as<uint64_t>(), (int64_t)n, sums.as<uint64_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, sums.as<uint64_t>(), (int64_t)tiles, (uint64_t*)(c->d_ctrl + kSlotSeg));
+  XLOG_LAUNCH(c, (k_scan_apply<uint64_t, uint64_t>), tiles, kScanBlock, 0, (const uint64_t*)flags.as<uint64_t>(), (int64_t)n,
+              (const uint64_t*)sums.as<uint64_t>(), idx.as<uint64_t>());
+  sync_ctrl(c);
+  const uint32_t n_all = (uint32_t)c->h_ctrl[kSlotSeg], n_seg = (uint32_t)(c->h_ctrl[kSlotSeg] >> 32);
+  if (n_seg == 0) return 0;
+  DevBuf first_all(c, ((size_t)n_all + 1) * 4), seg_first(c, (size_t)n_seg * 4), seg_rows(c, (size_t)n_seg * 4), seg_cand(c, (size_t)n_seg * 8),
+      seg_start(c, (size_t)n_seg * 8);
+  XLOG_LAUNCH(c, k_seg_first, grid_for((uint64_t)n + 1, 256), 256, 0, (const uint64_t*)flags.as<uint64_t>(), (const uint64_t*)idx.as<uint64_t>(), n, n_all,
+              first_all.as<uint32_t>());
+  XLOG_LAUNCH(c, k_seg_build, grid_for(n, 256), 256, 0, (const uint64_t*)flags.as<uint64_t>(), (const uint64_t*)idx.as<uint64_t>(), n,
+              (const uint32_t*)first_all.as<uint32_t>(), (const uint32_t*)deg.as<uint32_t>(), seg_first.as<uint32_t>(), seg_rows.as<uint32_t>(),
+              seg_cand.as<uint64_t>());
+  flags.reset(); idx.reset(); first_all.reset();
+  const unsigned stiles = (n_seg + kScanTile - 1) / kScanTile;
+  DevBuf ssums(c, (size_t)stiles * 8);
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint64_t, uint64_t>), stiles, kScanBlock, 0, (const uint64_t*)seg_cand.as<uint64_t>(), (int64_t)n_seg, ssums.as<uint64_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, ssums.as<uint64_t>(), (int64_t)stiles, (uint64_t*)(c->d_ctrl + kSlotSeg + 1));
+  XLOG_LAUNCH(c, (k_scan_apply<uint64_t, uint64_t>), stiles, kScanBlock, 0, (const uint64_t*)seg_cand.as<uint64_t>(), (int64_t)n_seg,
+              (const uint64_t*)ssums.as<uint64_t>(), seg_start.as<uint64_t>());
+  sync_ctrl(c);
+  const uint64_t total = c->h_ctrl[kSlotSeg + 1];
+  if (getenv("XLOG_DEBUG_SEG")) fprintf(stderr, "seg: rows %u segments %u with matches %u candidates %llu\n", n, n_all, n_seg, (unsigned long long)total);
+  if (total == 0) return 0;
+  c->note_bytes = (int64_t)total * 12;       // per candidate, as for the row-wise kernel, so that the figures are comparable
+  if (total / n_seg >= 128) {
+    // big segments: the segment-stationary kernel (a warp keeps the delta rows in its lanes and walks the neighbours)
+    const int64_t bytes = c->note_bytes;
+    c->note_bytes = 0;
+    const uint32_t ns1 = n_seg + 1;
+    const unsigned ittiles = (ns1 + kScanTile - 1) / kScanTile;
+    DevBuf items(c, (size_t)ns1 * 4), item_off(c, (size_t)ns1 * 4), itsums(c, (size_t)ittiles * 4);
+    XLOG_LAUNCH(c, k_seg_items, grid_for(ns1, 256), 256, 0, (const uint32_t*)seg_first.as<uint32_t>(), (const uint32_t*)seg_rows.as<uint32_t>(), n_seg,
+                (const uint32_t*)deg.as<uint32_t>(), items.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), ittiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ns1, itsums.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, itsums.as<uint32_t>(), (int64_t)ittiles, ctrl_u32(c, kSlotSeg + 2));
+    XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), ittiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ns1,
+                (const uint32_t*)itsums.as<uint32_t>(), item_off.as<uint32_t>());
+    sync_ctrl(c);
+    const uint32_t n_items = (uint32_t)c->h_ctrl[kSlotSeg + 2];
+    items.reset(); itsums.reset();
+    DevBuf item_seg(c, (size_t)std::max(n_items, 1u) * 4);
+    XLOG_LAUNCH(c, k_seg_item_fill, grid_for(n_seg, 256), 256, 0, n_seg, (const uint32_t*)item_off.as<uint32_t>(), item_seg.as<uint32_t>());
+    c->note_bytes = bytes;
+    const unsigned grid = (unsigned)std::min<uint64_t>(((uint64_t)n_items + 7) / 8, (uint64_t)kSMs * 8 * 16);
+    if (is_max)
+      XLOG_LAUNCH(c, (k_seg_expand<kSinkMax>), grid, 256, 0, S, n_items, (const uint32_t*)item_off.as<uint32_t>(), (const uint32_t*)item_seg.as<uint32_t>(),
+                  (const uint32_t*)seg_first.as<uint32_t>(), (const uint32_t*)seg_rows.as<uint32_t>(), (const uint32_t*)deg.as<uint32_t>(),
+                  (const uint4*)rowinfo.as<uint4>(), mr);
+    else
+      XLOG_LAUNCH(c, (k_seg_expand<kSinkMin>), grid, 256, 0, S, n_items, (const uint32_t*)item_off.as<uint32_t>(), (const uint32_t*)item_seg.as<uint32_t>(),
+                  (const uint32_t*)seg_first.as<uint32_t>(), (const uint32_t*)seg_rows.as<uint32_t>(), (const uint32_t*)deg.as<uint32_t>(),
+                  (const uint4*)rowinfo.as<uint4>(), mr);
+    return total;
+  }
+  const uint64_t nblocks = (total + kGrpTile - 1) / kGrpTile;
+  if (nblocks > 0x7fffffffull) fail(XLOG_ERR_CAPACITY_EXCEEDED, "a join round produces more than 2^41 candidates");
+  DevBuf tile_rows(c, (size_t)nblocks * 8);
+  {
+    const int64_t bytes = c->note_bytes;
+    c->note_bytes = 0;
+    XLOG_LAUNCH(c, k_expand_partition, (unsigned)((nblocks + 255) / 256), 256, 0, (const uint64_t*)seg_start.as<uint64_t>(), n_seg, (uint64_t)0, total,
+                (uint32_t)nblocks, (uint32_t)kGrpTile, tile_rows.as<uint2>());
+    c->note_bytes = bytes;
+  }
+  if (is_max)
+    XLOG_LAUNCH(c, (k_group_expand<kSinkMax>), (unsigned)nblocks, kExpBlock, 0, S, (const uint64_t*)seg_start.as<uint64_t>(), (const uint32_t*)seg_first.as<uint32_t>(),
+                (const uint32_t*)seg_rows.as<uint32_t>(), (const uint4*)rowinfo.as<uint4>(), (const uint2*)tile_rows.as<uint2>(), total, mr);
+  else
+    XLOG_LAUNCH(c, (k_group_expand<kSinkMin>), (unsigned)nblocks, kExpBlock, 0, S, (const uint64_t*)seg_start.as<uint64_t>(), (const uint32_t*)seg_first.as<uint32_t>(),
+                (const uint32_t*)seg_rows.as<uint32_t>(), (const uint4*)rowinfo.as<uint4>(), (const uint2*)tile_rows.as<uint2>(), total, mr);
+  return total;
+}
+
 // Algorithm 1 over a tag mirror (mirror.cuh): per round  count -> scan -> join straight into the table -> compact the
 // changed bitmap into the next delta.  No candidate is ever written to memory.  The seed round is driven by the host
 // (its rules scan whole relations of known size); the delta rounds run resident where the fixed-capacity buffers fit.
@@ -1331,6 +1449,16 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
   const uint32_t bm_quads = (uint32_t)((std::max<uint64_t>(dom / 32, 1) + 3) / 4);
   const unsigned ch_tiles = mirror_tiles(bm_quads * 4);
   Resident* R = resident_for(c, h, bits, slots, bm_quads, ch_tiles);
+  // the mirror's own column order: for the grouped join the probed column is the major part of the index (group_join.cuh)
+  KeyLayout M = H.layout;
+  const bool grouped = !R && !(c->flags & XLOG_FLAG_NO_GROUPED_JOIN) && grouped_shape(c, h, rs);
+  int carried_bits = 0;
+  if (grouped) {
+    carried_bits = bits - H.layout.shift[0];             // width of column 0
+    M.shift[0] = 0;
+    M.shift[1] = carried_bits;
+  }
+  const KeyLayout* ML = grouped ? &M : nullptr;
   DevBuf table_own, bitmap_own, present_own, ch_sums_own;
   if (!R) {
     table_own = DevBuf(c, slots * 4); bitmap_own = DevBuf(c, (size_t)bm_quads * 16); present_own = DevBuf(c, (size_t)bm_quads * 16);
@@ -1346,7 +1474,7 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
   // what the relation holds now (its loaded facts, or the result of an earlier fixpoint) is the starting state
   const uint32_t n_start = H.n;
   if (n_start)
-    XLOG_LAUNCH(c, (k_mirror_scatter<uint32_t>), grid_for(n_start, 256, 1 << 30), 256, 0, (const uint32_t*)H.keys(), (const float*)H.tags(), n_start, table, present);
+    XLOG_LAUNCH(c, (k_mirror_scatter<uint32_t>), grid_for(n_start, 256, 1 << 30), 256, 0, (const uint32_t*)H.keys(), (const float*)H.tags(), n_start, H.layout, M, table, present);
   zero_ctrl(c, kSlotMirNew, 2);
   const MirrorArgs mr{table, reinterpret_cast<uint32_t*>(bitmap), (unsigned long long*)(c->d_ctrl + kSlotMirNew), (uint32_t)(dom - 1),
                       ctrl_u32(c, kSlotErr)};
@@ -1359,17 +1487,22 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
     if (vs.size() > 16) fail(XLOG_ERR_UNSUPPORTED, "too many rule variants for one head");
     std::vector<Counted> counted;
     counted.reserve(vs.size());
+    uint64_t total = 0;
     for (Variant& v : vs) {
       if (v.outer.n == 0) continue;
+      if (grouped && v.outer.keys == dk && v.rule->plan.atoms[v.outer_atom].rel == h) {
+        // a delta variant of the grouped shape: the delta is ordered by the probed column
+        const uint64_t t = grouped_apply(c, v, H, M, carried_bits, is_max, mr);
+        if (t != UINT64_MAX) { total += t; c->r_candidates += (int64_t)t; continue; }
+      }
       counted.emplace_back();
-      count_variant(c, v, H, counted.back(), kSlotTotals + (int)counted.size() - 1);
+      count_variant(c, v, H, counted.back(), kSlotTotals + (int)counted.size() - 1, ML);
     }
-    uint64_t total = 0;
     if (!counted.empty()) {
       sync_ctrl(c);
       for (Counted& q : counted) { q.total = c->h_ctrl[q.slot]; total += q.total; q.deg.reset(); q.sums.reset(); }
     }
-    c->r_candidates += (int64_t)total;
+    for (Counted& q : counted) c->r_candidates += (int64_t)q.total;
     for (Counted& q : counted) {
       if (q.total) {
         // per candidate: the looked-up atom's other columns and tag are read, and the key's slot is read (and now and then written)
@@ -1422,7 +1555,7 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
         vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
       } else {
         for (int j = 0; j < r->plan.n_atoms; ++j)
-          if (r->plan.atoms[j].rel == h && dn) vs.push_back(Variant{r, j, Source{dk, dt, dn, H.layout, H.key_bytes}});
+          if (r->plan.atoms[j].rel == h && dn) vs.push_back(Variant{r, j, Source{dk, dt, dn, M, H.key_bytes}});
       }
     }
     const uint64_t total = host_apply(vs);
@@ -1461,8 +1594,17 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
     XLOG_LAUNCH(c, k_mirror_full_count, tiles, kMirBlock, 0, (const int4*)table, nquads, empty, sums.as<uint32_t>());
     XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, sums.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotA));
     c->note_bytes = (int64_t)slots * 4 + (int64_t)n_out * 8;
-    XLOG_LAUNCH(c, (k_mirror_full_emit<uint32_t>), tiles, kMirBlock, 0, (const int4*)table, nquads, empty, (const uint32_t*)sums.as<uint32_t>(),
+    XLOG_LAUNCH(c, (k_mirror_full_emit<uint32_t>), tiles, kMirBlock, 0, (const int4*)table, nquads, empty, (const uint32_t*)sums.as<uint32_t>(), M, H.layout,
                 full.keys.as<uint32_t>(), full.tags.as<float>());
+    if (grouped && n_out > 1) {
+      // rows came out in the mirror's order (probed column first): one sort puts them in the relation's key order
+      table_own.reset(); bitmap_own.reset(); present_own.reset();
+      DevBuf ak(c, (size_t)n_out * 4), at(c, (size_t)n_out * 4);
+      uint32_t* pk = full.keys.as<uint32_t>(); uint32_t* qk = ak.as<uint32_t>();
+      float* pt = full.tags.as<float>(); float* qt = at.as<float>();
+      sort_pairs<uint32_t>(c, pk, pt, qk, qt, n_out, bits);
+      if ((void*)pk != full.keys.p) { std::swap(full.keys, ak); std::swap(full.tags, at); }
+    }
   }
   set_current(H, std::move(full));
   if (c->flags & XLOG_FLAG_CHECK_INVARIANTS) {
