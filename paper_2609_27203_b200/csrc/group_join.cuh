@@ -177,7 +177,7 @@ static __global__ void __launch_bounds__(256) k_seg_item_fill(uint32_t n_seg, co
 }
 
 template <int SINK>
-__global__ void __launch_bounds__(256) k_seg_expand(JoinSpec S, uint32_t n_items, const uint32_t* __restrict__ item_off, const uint32_t* __restrict__ item_seg,
+__global__ void __launch_bounds__(256, 8) k_seg_expand(JoinSpec S, uint32_t n_items, const uint32_t* __restrict__ item_off, const uint32_t* __restrict__ item_seg,
                                                     const uint32_t* __restrict__ seg_first, const uint32_t* __restrict__ seg_rows,
                                                     const uint32_t* __restrict__ deg, const uint4* __restrict__ rowinfo, MirrorArgs mr) {
   const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -208,20 +208,31 @@ __global__ void __launch_bounds__(256) k_seg_expand(JoinSpec S, uint32_t n_items
         uint32_t zr = 0;
         float wr = 0.f;
         if (lane < nj) { zr = (uint32_t)__ldcs(ic0 + lo + jb + lane); wr = __ldcs(itg + lo + jb + lane); }
-#pragma unroll 4
-        for (uint32_t s = 0; s < nj; s += per) {
-          const uint32_t jj = s + jsub;
-          const uint32_t z = __shfl_sync(0xffffffffu, zr, jj & 31);
-          const float w = __shfl_sync(0xffffffffu, wr, jj & 31);
-          if (has_row && jj < nj) {
-            const uint32_t key = ckey + z * m0;
-            if (key > mr.key_max) e |= kErrHeadRange;
-            else {
-              const int32_t v = f2ord(otag + w);
-              const int32_t cur = XLOG_TABLE_LOAD(mr.table + key);
-              if (SINK == kSinkMin ? v < cur : v > cur) mirror_commit<SINK>(mr, key, v);
+        // four steps at a time: keys first, then the four slot reads together, then the reductions of those that improve
+        for (uint32_t s0 = 0; s0 < nj; s0 += 4 * per) {
+          uint32_t key[4];
+          int32_t v[4], cur[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const uint32_t jj = s0 + u * per + jsub;
+            const uint32_t z = __shfl_sync(0xffffffffu, zr, jj & 31);
+            const float w = __shfl_sync(0xffffffffu, wr, jj & 31);
+            key[u] = 0xffffffffu;                        // nothing to do
+            v[u] = 0;
+            if (has_row && jj < nj) {
+              key[u] = ckey + z * m0;
+              v[u] = f2ord(otag + w);
+              if (key[u] > mr.key_max) { e |= kErrHeadRange; key[u] = 0xffffffffu; }
             }
           }
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            cur[u] = SINK == kSinkMin ? (int32_t)0x80000000 : 0x7fffffff;
+            if (key[u] != 0xffffffffu) cur[u] = XLOG_TABLE_LOAD(mr.table + key[u]);
+          }
+#pragma unroll
+          for (int u = 0; u < 4; ++u)
+            if (SINK == kSinkMin ? v[u] < cur[u] : v[u] > cur[u]) mirror_commit<SINK>(mr, key[u], v[u]);
         }
       }
     }
