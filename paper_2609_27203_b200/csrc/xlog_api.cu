@@ -1347,7 +1347,7 @@ bool grouped_shape(Ctx* c, int h, const std::vector<const RuleC*>& rs) {
   return any;
 }
 
-constexpr int kSlotSeg = 14;               // segment totals (low word: all, high word: with matches), then the candidate total
+constexpr int kSlotSeg = 80;               // grouped join: segments, candidates, work items (three control words)
 
 // One delta variant through the grouped join.  Returns the candidate total, or UINT64_MAX when the compiled rule turns
 // out not to have the linear-key form (the caller then takes the row-wise join).
@@ -1356,82 +1356,46 @@ uint64_t grouped_apply(Ctx* c, const Variant& v, const Relation& H, const KeyLay
   if (!S.fast || !S.has_inner || S.inner_free != 1 || v.outer.key_bytes != 4) return UINT64_MAX;
   const uint32_t n = v.outer.n;
   const unsigned tiles = (n + kScanTile - 1) / kScanTile;
-  DevBuf deg(c, (size_t)n * 4), rowinfo(c, (size_t)n * 16), flags(c, (size_t)n * 8), idx(c, (size_t)n * 8), sums(c, (size_t)tiles * 8);
-  XLOG_LAUNCH(c, (k_join_count<uint32_t>), (n + 255) / 256, 256, 0, S, (const uint32_t*)v.outer.keys, v.outer.tags, n, deg.as<uint32_t>(),
-              rowinfo.as<uint4>(), ctrl_u32(c, kSlotErr));
-  XLOG_LAUNCH(c, k_seg_flags, grid_for(n, 256), 256, 0, (const uint32_t*)v.outer.keys, (const uint32_t*)deg.as<uint32_t>(), n, carried_bits, flags.as<uint64_t>());
-  XLOG_LAUNCH(c, (k_scan_tile_sums<uint64_t, uint64_t>), tiles, kScanBlock, 0, (const uint64_t*)flags.as<uint64_t>(), (int64_t)n, sums.as<uint64_t>());
-  XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, sums.as<uint64_t>(), (int64_t)tiles, (uint64_t*)(c->d_ctrl + kSlotSeg));
-  XLOG_LAUNCH(c, (k_scan_apply<uint64_t, uint64_t>), tiles, kScanBlock, 0, (const uint64_t*)flags.as<uint64_t>(), (int64_t)n,
-              (const uint64_t*)sums.as<uint64_t>(), idx.as<uint64_t>());
+  DevBuf deg(c, (size_t)n * 4), rowinfo(c, (size_t)n * 16), flags(c, (size_t)n * 4), idx(c, (size_t)n * 4), sums(c, (size_t)tiles * 4);
+  zero_ctrl(c, kSlotSeg, 3);
+  XLOG_LAUNCH(c, (k_join_count_flags<uint32_t>), grid_for(n, 256, kSMs * 32), 256, 0, S, (const uint32_t*)v.outer.keys, v.outer.tags, n, carried_bits, deg.as<uint32_t>(),
+              rowinfo.as<uint4>(), flags.as<uint32_t>(), (unsigned long long*)(c->d_ctrl + kSlotSeg + 1), ctrl_u32(c, kSlotErr));
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), tiles, kScanBlock, 0, (const uint32_t*)flags.as<uint32_t>(), (int64_t)n, sums.as<uint32_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, sums.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotSeg));
+  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), tiles, kScanBlock, 0, (const uint32_t*)flags.as<uint32_t>(), (int64_t)n,
+              (const uint32_t*)sums.as<uint32_t>(), idx.as<uint32_t>());
   sync_ctrl(c);
-  const uint32_t n_all = (uint32_t)c->h_ctrl[kSlotSeg], n_seg = (uint32_t)(c->h_ctrl[kSlotSeg] >> 32);
-  if (n_seg == 0) return 0;
-  DevBuf first_all(c, ((size_t)n_all + 1) * 4), seg_first(c, (size_t)n_seg * 4), seg_rows(c, (size_t)n_seg * 4), seg_cand(c, (size_t)n_seg * 8),
-      seg_start(c, (size_t)n_seg * 8);
-  XLOG_LAUNCH(c, k_seg_first, grid_for((uint64_t)n + 1, 256), 256, 0, (const uint64_t*)flags.as<uint64_t>(), (const uint64_t*)idx.as<uint64_t>(), n, n_all,
-              first_all.as<uint32_t>());
-  XLOG_LAUNCH(c, k_seg_build, grid_for(n, 256), 256, 0, (const uint64_t*)flags.as<uint64_t>(), (const uint64_t*)idx.as<uint64_t>(), n,
-              (const uint32_t*)first_all.as<uint32_t>(), (const uint32_t*)deg.as<uint32_t>(), seg_first.as<uint32_t>(), seg_rows.as<uint32_t>(),
-              seg_cand.as<uint64_t>());
-  flags.reset(); idx.reset(); first_all.reset();
-  const unsigned stiles = (n_seg + kScanTile - 1) / kScanTile;
-  DevBuf ssums(c, (size_t)stiles * 8);
-  XLOG_LAUNCH(c, (k_scan_tile_sums<uint64_t, uint64_t>), stiles, kScanBlock, 0, (const uint64_t*)seg_cand.as<uint64_t>(), (int64_t)n_seg, ssums.as<uint64_t>());
-  XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, ssums.as<uint64_t>(), (int64_t)stiles, (uint64_t*)(c->d_ctrl + kSlotSeg + 1));
-  XLOG_LAUNCH(c, (k_scan_apply<uint64_t, uint64_t>), stiles, kScanBlock, 0, (const uint64_t*)seg_cand.as<uint64_t>(), (int64_t)n_seg,
-              (const uint64_t*)ssums.as<uint64_t>(), seg_start.as<uint64_t>());
-  sync_ctrl(c);
+  const uint32_t n_seg = (uint32_t)c->h_ctrl[kSlotSeg];
   const uint64_t total = c->h_ctrl[kSlotSeg + 1];
-  if (getenv("XLOG_DEBUG_SEG")) fprintf(stderr, "seg: rows %u segments %u with matches %u candidates %llu\n", n, n_all, n_seg, (unsigned long long)total);
   if (total == 0) return 0;
-  c->note_bytes = (int64_t)total * 12;       // per candidate, as for the row-wise kernel, so that the figures are comparable
-  if (total / n_seg >= 128) {
-    // big segments: the segment-stationary kernel (a warp keeps the delta rows in its lanes and walks the neighbours)
-    const int64_t bytes = c->note_bytes;
-    c->note_bytes = 0;
-    const uint32_t ns1 = n_seg + 1;
-    const unsigned ittiles = (ns1 + kScanTile - 1) / kScanTile;
-    DevBuf items(c, (size_t)ns1 * 4), item_off(c, (size_t)ns1 * 4), itsums(c, (size_t)ittiles * 4);
-    XLOG_LAUNCH(c, k_seg_items, grid_for(ns1, 256), 256, 0, (const uint32_t*)seg_first.as<uint32_t>(), (const uint32_t*)seg_rows.as<uint32_t>(), n_seg,
-                (const uint32_t*)deg.as<uint32_t>(), items.as<uint32_t>());
-    XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), ittiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ns1, itsums.as<uint32_t>());
-    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, itsums.as<uint32_t>(), (int64_t)ittiles, ctrl_u32(c, kSlotSeg + 2));
-    XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), ittiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ns1,
-                (const uint32_t*)itsums.as<uint32_t>(), item_off.as<uint32_t>());
-    sync_ctrl(c);
-    const uint32_t n_items = (uint32_t)c->h_ctrl[kSlotSeg + 2];
-    items.reset(); itsums.reset();
-    DevBuf item_seg(c, (size_t)std::max(n_items, 1u) * 4);
-    XLOG_LAUNCH(c, k_seg_item_fill, grid_for(n_seg, 256), 256, 0, n_seg, (const uint32_t*)item_off.as<uint32_t>(), item_seg.as<uint32_t>());
-    c->note_bytes = bytes;
-    const unsigned grid = (unsigned)std::min<uint64_t>(((uint64_t)n_items + 7) / 8, (uint64_t)kSMs * 8 * 16);
-    if (is_max)
-      XLOG_LAUNCH(c, (k_seg_expand<kSinkMax>), grid, 256, 0, S, n_items, (const uint32_t*)item_off.as<uint32_t>(), (const uint32_t*)item_seg.as<uint32_t>(),
-                  (const uint32_t*)seg_first.as<uint32_t>(), (const uint32_t*)seg_rows.as<uint32_t>(), (const uint32_t*)deg.as<uint32_t>(),
-                  (const uint4*)rowinfo.as<uint4>(), mr);
-    else
-      XLOG_LAUNCH(c, (k_seg_expand<kSinkMin>), grid, 256, 0, S, n_items, (const uint32_t*)item_off.as<uint32_t>(), (const uint32_t*)item_seg.as<uint32_t>(),
-                  (const uint32_t*)seg_first.as<uint32_t>(), (const uint32_t*)seg_rows.as<uint32_t>(), (const uint32_t*)deg.as<uint32_t>(),
-                  (const uint4*)rowinfo.as<uint4>(), mr);
-    return total;
-  }
-  const uint64_t nblocks = (total + kGrpTile - 1) / kGrpTile;
-  if (nblocks > 0x7fffffffull) fail(XLOG_ERR_CAPACITY_EXCEEDED, "a join round produces more than 2^41 candidates");
-  DevBuf tile_rows(c, (size_t)nblocks * 8);
-  {
-    const int64_t bytes = c->note_bytes;
-    c->note_bytes = 0;
-    XLOG_LAUNCH(c, k_expand_partition, (unsigned)((nblocks + 255) / 256), 256, 0, (const uint64_t*)seg_start.as<uint64_t>(), n_seg, (uint64_t)0, total,
-                (uint32_t)nblocks, (uint32_t)kGrpTile, tile_rows.as<uint2>());
-    c->note_bytes = bytes;
-  }
+  if (total / n_seg < 128) return UINT64_MAX;            // small segments: the row-wise join does as well, with fewer passes
+  const uint32_t ns1 = n_seg + 1;
+  DevBuf seg_first(c, (size_t)ns1 * 4);
+  XLOG_LAUNCH(c, k_seg_first, grid_for((uint64_t)n + 1, 256), 256, 0, (const uint32_t*)flags.as<uint32_t>(), (const uint32_t*)idx.as<uint32_t>(), n, n_seg,
+              seg_first.as<uint32_t>());
+  flags.reset(); idx.reset(); sums.reset();
+  const unsigned ittiles = (ns1 + kScanTile - 1) / kScanTile;
+  DevBuf items(c, (size_t)ns1 * 4), item_off(c, (size_t)ns1 * 4), itsums(c, (size_t)ittiles * 4);
+  XLOG_LAUNCH(c, k_seg_items, grid_for(ns1, 256), 256, 0, (const uint32_t*)seg_first.as<uint32_t>(), n_seg, (const uint32_t*)deg.as<uint32_t>(), items.as<uint32_t>());
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), ittiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ns1, itsums.as<uint32_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, itsums.as<uint32_t>(), (int64_t)ittiles, ctrl_u32(c, kSlotSeg + 2));
+  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), ittiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ns1,
+              (const uint32_t*)itsums.as<uint32_t>(), item_off.as<uint32_t>());
+  sync_ctrl(c);
+  const uint32_t n_items = (uint32_t)c->h_ctrl[kSlotSeg + 2];
+  items.reset(); itsums.reset();
+  DevBuf item_seg(c, (size_t)std::max(n_items, 1u) * 4);
+  XLOG_LAUNCH(c, k_seg_item_fill, grid_for(n_seg, 256), 256, 0, n_seg, (const uint32_t*)item_off.as<uint32_t>(), item_seg.as<uint32_t>());
+  // per candidate: its slot; per segment and neighbour: the looked-up column and tag, shared by the segment's rows (declared
+  // per candidate here, as for the row-wise kernel, so that the two report comparable figures)
+  c->note_bytes = (int64_t)total * 12;
+  const unsigned grid = (unsigned)std::min<uint64_t>(((uint64_t)n_items + 7) / 8, (uint64_t)kSMs * 8 * 16);
   if (is_max)
-    XLOG_LAUNCH(c, (k_group_expand<kSinkMax>), (unsigned)nblocks, kExpBlock, 0, S, (const uint64_t*)seg_start.as<uint64_t>(), (const uint32_t*)seg_first.as<uint32_t>(),
-                (const uint32_t*)seg_rows.as<uint32_t>(), (const uint4*)rowinfo.as<uint4>(), (const uint2*)tile_rows.as<uint2>(), total, mr);
+    XLOG_LAUNCH(c, (k_seg_expand<kSinkMax>), grid, 256, 0, S, n_items, (const uint32_t*)item_off.as<uint32_t>(), (const uint32_t*)item_seg.as<uint32_t>(),
+                (const uint32_t*)seg_first.as<uint32_t>(), (const uint32_t*)deg.as<uint32_t>(), (const uint4*)rowinfo.as<uint4>(), mr);
   else
-    XLOG_LAUNCH(c, (k_group_expand<kSinkMin>), (unsigned)nblocks, kExpBlock, 0, S, (const uint64_t*)seg_start.as<uint64_t>(), (const uint32_t*)seg_first.as<uint32_t>(),
-                (const uint32_t*)seg_rows.as<uint32_t>(), (const uint4*)rowinfo.as<uint4>(), (const uint2*)tile_rows.as<uint2>(), total, mr);
+    XLOG_LAUNCH(c, (k_seg_expand<kSinkMin>), grid, 256, 0, S, n_items, (const uint32_t*)item_off.as<uint32_t>(), (const uint32_t*)item_seg.as<uint32_t>(),
+                (const uint32_t*)seg_first.as<uint32_t>(), (const uint32_t*)deg.as<uint32_t>(), (const uint4*)rowinfo.as<uint4>(), mr);
   return total;
 }
 
