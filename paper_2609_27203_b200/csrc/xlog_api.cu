@@ -1561,12 +1561,13 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
     XLOG_LAUNCH(c, (k_mirror_full_emit<uint32_t>), tiles, kMirBlock, 0, (const int4*)table, nquads, empty, (const uint32_t*)sums.as<uint32_t>(), M, H.layout,
                 full.keys.as<uint32_t>(), full.tags.as<float>());
     if (grouped && n_out > 1) {
-      // rows came out in the mirror's order (probed column first): one sort puts them in the relation's key order
+      // rows came out in the mirror's order, (column 1, column 0) ascending: a stable sort on column 0's bits alone puts
+      // them in the relation's key order
       table_own.reset(); bitmap_own.reset(); present_own.reset();
       DevBuf ak(c, (size_t)n_out * 4), at(c, (size_t)n_out * 4);
       uint32_t* pk = full.keys.as<uint32_t>(); uint32_t* qk = ak.as<uint32_t>();
       float* pt = full.tags.as<float>(); float* qt = at.as<float>();
-      sort_pairs<uint32_t>(c, pk, pt, qk, qt, n_out, bits);
+      sort_pairs<uint32_t>(c, pk, pt, qk, qt, n_out, bits, H.layout.shift[0]);
       if ((void*)pk != full.keys.p) { std::swap(full.keys, ak); std::swap(full.tags, at); }
     }
   }
