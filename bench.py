@@ -36,7 +36,10 @@ UNIT = "tuples/s"
 NCU_TRAFFIC_RATIO = {"k_sort_pass": 0.99, "k_join_expand": 0.92, "k_dense_reduce": 1.04, "k_merge": 1.0}
 # the join kernels when they apply candidates to the tag mirror instead of writing them: the slot reads hit L2, so DRAM
 # sees the adjacency reads (8 of the 12 algorithmic bytes per candidate) plus row records
-NCU_TRAFFIC_RATIO_MIRROR = {"k_join_expand": 0.80, "k_res_expand": 0.80}
+NCU_TRAFFIC_RATIO_MIRROR = {"k_join_expand": 0.80, "k_res_expand": 0.80,
+                            # grouped join (rows of one probed value share the neighbour reads and sit in one table line): 5.1 B of DRAM
+                            # traffic per candidate at 32 sources against 5.3 algorithmic (4 for the slot, 8 / rows-per-node for the neighbour)
+                            "k_seg_expand": 0.95}
 
 
 def make_program(name: str, scale: int | None, sources: int | None = None):
@@ -250,7 +253,7 @@ def run_ours(args):
     peak, peak_src = measured_peak_gbs()
     achieved = d["bytes"] / (d["ms"] / 1e3) / 1e9 if d["ms"] > 0 else 0.0
     ratio = NCU_TRAFFIC_RATIO.get(dom)
-    mirror_kernel = dom == "k_res_expand" or (dom == "k_join_expand" and not args.no_tag_mirror and "k_sort_pass" not in prof)
+    mirror_kernel = dom in ("k_res_expand", "k_seg_expand") or (dom == "k_join_expand" and not args.no_tag_mirror and "k_sort_pass" not in prof)
     if mirror_kernel:
         ratio = NCU_TRAFFIC_RATIO_MIRROR.get(dom)
     bound = "hbm"
@@ -278,9 +281,11 @@ def run_ours(args):
     if mirror_kernel:
         # one random 32-byte L2 sector per candidate (the key's slot in the tag mirror) on top of the streamed adjacency
         # reads: the kernel is bound by how many such sector requests the SMs keep in flight, not by HBM
-        roofline["limiter"] = "L2 random sector access (one tag-mirror slot per candidate); HBM carries about 8 B per candidate"
-        per_cand = 12.0
-        roofline["candidates_per_s"] = achieved * 1e9 / per_cand
+        roofline["limiter"] = ("instruction issue (79 % of the issue slots busy under ncu at 32 sources); the table, too large for L2, is read from HBM one line per (node, neighbour)"
+                               if dom == "k_seg_expand" else
+                               "L2 random sector access (one tag-mirror slot per candidate); HBM carries about 8 B per candidate")
+        if dom != "k_seg_expand":
+            roofline["candidates_per_s"] = achieved * 1e9 / 12.0
 
     # end to end through the C ABI with HOST buffers: load (H2D + sort + index), fixpoint, read back (D2H)
     pinned = {}

@@ -54,17 +54,23 @@ __host__ __device__ __forceinline__ uint32_t seg_slice(uint32_t rows) {
   return s < 32u ? 32u : (s & ~31u);
 }
 
+// *neighbours accumulates the looked-up rows read by the join (one run per segment, whatever its number of delta rows)
 static __global__ void __launch_bounds__(256) k_seg_items(const uint32_t* __restrict__ seg_first, uint32_t n_seg, const uint32_t* __restrict__ deg,
-                                                         uint32_t* __restrict__ items) {
+                                                         uint32_t* __restrict__ items, unsigned long long* __restrict__ neighbours) {
+  unsigned long long mine = 0;
   for (uint32_t g = blockIdx.x * blockDim.x + threadIdx.x; g <= n_seg; g += gridDim.x * blockDim.x) {
     uint32_t n = 0;
     if (g < n_seg) {
       const uint32_t f = seg_first[g];
       const uint32_t sl = seg_slice(seg_first[g + 1] - f), dg = deg[f];      // a segment without matches gets no item
       n = (dg + sl - 1) / sl;
+      mine += dg;
     }
     items[g] = n;                                        // items[n_seg] = 0: the scan then has n_seg + 1 entries
   }
+#pragma unroll
+  for (int s = 16; s; s >>= 1) mine += __shfl_down_sync(0xffffffffu, mine, s);
+  if (lane_id() == 0 && mine) atomicAdd(neighbours, mine);
 }
 static __global__ void __launch_bounds__(256) k_seg_item_fill(uint32_t n_seg, const uint32_t* __restrict__ item_off, uint32_t* __restrict__ item_seg) {
   for (uint32_t g = blockIdx.x * blockDim.x + threadIdx.x; g < n_seg; g += gridDim.x * blockDim.x)

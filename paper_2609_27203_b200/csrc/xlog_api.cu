@@ -1347,7 +1347,7 @@ bool grouped_shape(Ctx* c, int h, const std::vector<const RuleC*>& rs) {
   return any;
 }
 
-constexpr int kSlotSeg = 80;               // grouped join: segments, candidates, work items (three control words)
+constexpr int kSlotSeg = 80;               // grouped join: segments, candidates, work items, neighbour rows read
 
 // One delta variant through the grouped join.  Returns the candidate total, or UINT64_MAX when the compiled rule turns
 // out not to have the linear-key form (the caller then takes the row-wise join).
@@ -1357,7 +1357,7 @@ uint64_t grouped_apply(Ctx* c, const Variant& v, const Relation& H, const KeyLay
   const uint32_t n = v.outer.n;
   const unsigned tiles = (n + kScanTile - 1) / kScanTile;
   DevBuf deg(c, (size_t)n * 4), rowinfo(c, (size_t)n * 16), flags(c, (size_t)n * 4), idx(c, (size_t)n * 4), sums(c, (size_t)tiles * 4);
-  zero_ctrl(c, kSlotSeg, 3);
+  zero_ctrl(c, kSlotSeg, 4);
   XLOG_LAUNCH(c, (k_join_count_flags<uint32_t>), grid_for(n, 256, kSMs * 32), 256, 0, S, (const uint32_t*)v.outer.keys, v.outer.tags, n, carried_bits, deg.as<uint32_t>(),
               rowinfo.as<uint4>(), flags.as<uint32_t>(), (unsigned long long*)(c->d_ctrl + kSlotSeg + 1), ctrl_u32(c, kSlotErr));
   XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), tiles, kScanBlock, 0, (const uint32_t*)flags.as<uint32_t>(), (int64_t)n, sums.as<uint32_t>());
@@ -1376,7 +1376,8 @@ uint64_t grouped_apply(Ctx* c, const Variant& v, const Relation& H, const KeyLay
   flags.reset(); idx.reset(); sums.reset();
   const unsigned ittiles = (ns1 + kScanTile - 1) / kScanTile;
   DevBuf items(c, (size_t)ns1 * 4), item_off(c, (size_t)ns1 * 4), itsums(c, (size_t)ittiles * 4);
-  XLOG_LAUNCH(c, k_seg_items, grid_for(ns1, 256), 256, 0, (const uint32_t*)seg_first.as<uint32_t>(), n_seg, (const uint32_t*)deg.as<uint32_t>(), items.as<uint32_t>());
+  XLOG_LAUNCH(c, k_seg_items, grid_for(ns1, 256, kSMs * 16), 256, 0, (const uint32_t*)seg_first.as<uint32_t>(), n_seg, (const uint32_t*)deg.as<uint32_t>(), items.as<uint32_t>(),
+              (unsigned long long*)(c->d_ctrl + kSlotSeg + 3));
   XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), ittiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ns1, itsums.as<uint32_t>());
   XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, itsums.as<uint32_t>(), (int64_t)ittiles, ctrl_u32(c, kSlotSeg + 2));
   XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), ittiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ns1,
@@ -1386,9 +1387,9 @@ uint64_t grouped_apply(Ctx* c, const Variant& v, const Relation& H, const KeyLay
   items.reset(); itsums.reset();
   DevBuf item_seg(c, (size_t)std::max(n_items, 1u) * 4);
   XLOG_LAUNCH(c, k_seg_item_fill, grid_for(n_seg, 256), 256, 0, n_seg, (const uint32_t*)item_off.as<uint32_t>(), item_seg.as<uint32_t>());
-  // per candidate: its slot; per segment and neighbour: the looked-up column and tag, shared by the segment's rows (declared
-  // per candidate here, as for the row-wise kernel, so that the two report comparable figures)
-  c->note_bytes = (int64_t)total * 12;
+  // per candidate: its slot; per segment and neighbour: the looked-up column and tag, read once for all the segment's rows;
+  // per delta row: its count record
+  c->note_bytes = (int64_t)total * 4 + (int64_t)c->h_ctrl[kSlotSeg + 3] * 8 + (int64_t)n * 16;
   const unsigned grid = (unsigned)std::min<uint64_t>(((uint64_t)n_items + 7) / 8, (uint64_t)kSMs * 8 * 16);
   if (is_max)
     XLOG_LAUNCH(c, (k_seg_expand<kSinkMax>), grid, 256, 0, S, n_items, (const uint32_t*)item_off.as<uint32_t>(), (const uint32_t*)item_seg.as<uint32_t>(),
