@@ -87,6 +87,9 @@ typedef struct {
  *  - Tag mirror (default where it applies: one MAXPLUS/MINPLUS head relation, every rule with at most one
  *    atom over it and that atom scanned, packed key <= 30 bits, table fits the arena): the relation is a
  *    direct-addressed table of one tag per possible key; candidates are applied with one atomic max/min.
+ *    Above 2^24 possible keys a rule of the shape h(a, c) :- h(a, b), r(b, c) is joined "grouped": the mirror is
+ *    indexed with the probed column as the major part, the delta comes out grouped by b, and the delta rows of one b
+ *    share the read of r's run of b and a line of the table (XLOG_FLAG_NO_GROUPED_JOIN switches this off).
  *  - Resident rounds (tag mirror with <= 2^24 possible keys): the delta rounds run as one CUDA graph with a
  *    conditional WHILE node and fixed-capacity buffers (Section "GPU-Native Symbolic Substrate": resident
  *    conditional graph, no host reads inside the loop).  The buffers (about 36 bytes per possible key
