@@ -39,8 +39,10 @@ def check_program(program, rel_tol=MINMAX_REL, abs_tol=0.0, expect_bit_equal=Tru
     o, oids, _, stats = oracle_run(program, mode)
     receipts, results = [], []
     # default (tag mirror, delta rounds resident in one graph) / the same rounds launched one by one / host-driven
-    # mirror rounds / the sorting path
-    for extra in (0, xlog.FLAG_NO_GRAPH, xlog.FLAG_NO_RESIDENT_LOOP, xlog.FLAG_NO_TAG_MIRROR):
+    # mirror rounds (with the grouped join where the rule has that shape) / the same with the row-wise join only / the
+    # sorting path
+    for extra in (0, xlog.FLAG_NO_GRAPH, xlog.FLAG_NO_RESIDENT_LOOP, xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_GROUPED_JOIN,
+                  xlog.FLAG_NO_TAG_MIRROR):
         ctx, gids, _, receipt = gpu_run(program, **dict(kw, flags=kw.get("flags", xlog.FLAG_CHECK_INVARIANTS) | extra))
         got = {}
         for name in program.outputs:
