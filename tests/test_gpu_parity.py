@@ -262,6 +262,31 @@ def test_recursion_with_head_arithmetic_takes_the_general_join_path():
     assert r["iterations"] == n + 1 and r["derived_tuples"] == n - 1      # n - 7 is a loaded fact
 
 
+def test_routes_agree_at_sizes_beyond_the_oracle():
+    # mid-size cases where segments of the grouped join hold hundreds of delta rows (several passes of 32 lanes) and hub
+    # nodes have tens of thousands of neighbours: every engine route must derive the same relation, bit for bit, with the
+    # same counters.  (The oracle would need minutes here; the smaller ladders above pin the routes to it.)
+    from paper_2609_27203_b200 import xlog
+    hs = synth.randint(71, 1, 0, 40000, 20); hd = synth.randint(71, 2, 0, 40000, 5000)
+    s = np.concatenate([hs, hd[:20000]]); t = np.concatenate([hd, hs[:20000]])
+    key = np.unique(s[s != t].astype(np.int64) * 10000 + t[s != t])
+    s, t = (key // 10000).astype(np.int32), (key % 10000).astype(np.int32)
+    w = (1 + 9 * synth.uniform01(71, 3, 0, len(s))).astype(np.float32)
+    for prog in (W.closure_program(s, t, w, W.MINPLUS, name="hubs"), W.config5(scale=16, n_sources=300)):
+        base = None
+        for flags in (xlog.FLAG_NO_TAG_MIRROR, 0, xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_GROUPED_JOIN, xlog.FLAG_NO_RESIDENT_LOOP):
+            ctx, ids, _ = xlog.load_program(prog, arena_bytes=6 << 30, flags=flags)
+            r = ctx.fixpoint()
+            out = ctx.read(ids[prog.outputs[0]])
+            ctx.close()
+            if base is None:
+                base = (r, out)
+                continue
+            assert all(np.array_equal(a, b) for a, b in zip(base[1][0], out[0])) and np.array_equal(base[1][1].view(np.int32), out[1].view(np.int32))
+            for k in ("iterations", "candidates", "new_tuples", "improved_tags", "derived_tuples"):
+                assert base[0][k] == r[k], (prog.name, flags, k)
+
+
 def test_chunked_candidates_match_single_batch():
     p = W.config1(300, 1500)
     a, _ = check_program(p)
