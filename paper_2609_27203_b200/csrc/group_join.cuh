@@ -4,9 +4,9 @@
 // The mirror of such a relation is addressed with the probed column as the major part of the index and the
 // carried column as the minor part, so (1) the delta, which is the changed bitmap read in index order, comes out
 // grouped by b, and (2) the slots of (a_1, c), (a_2, c), ... lie next to each other.  A segment = the delta rows of one
-// b (k rows) joined with r's run of b (d rows) = k * d candidates, enumerated with the carried row as the fast index:
-// candidate p of the segment is (row p % k, neighbour p / k).  Consecutive lanes therefore read one neighbour (a
-// broadcast) and consecutive slots (a few sectors instead of one per candidate).
+// b (k rows) joined with r's run of b (d rows) = k * d candidates.  A warp keeps the k rows in its lanes and walks the
+// d neighbours: one read of r's run serves all k rows, and the lanes of a step touch consecutive slots (a few sectors
+// instead of one per candidate).
 //
 //   k_join_count_flags  the join's count step, plus where a delta row starts a new segment and the candidate total
 //   k_seg_first         first row of every segment
