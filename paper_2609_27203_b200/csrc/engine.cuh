@@ -40,6 +40,7 @@ struct Fail {
 constexpr int kCtrlSlots = 96;          // uint64 control words mirrored to pinned host memory
 constexpr int kSlotResState = 64;       // the resident loop's state block (resident.cuh) lives in the control words from here on
 constexpr int kSlotErr = 0;
+constexpr int64_t kProfLargeBytes = (int64_t)4000000 * 12;
 
 struct Ctx;
 
@@ -160,7 +161,7 @@ struct Ctx {
   int64_t r_candidates = 0, r_unique = 0, r_new = 0, r_improved = 0, r_iterations = 0, r_strata = 0;
   // optional per-kernel timing (XLOG_FLAG_PROFILE): CUDA events around every launch
   struct ProfEntry { std::string name; int64_t launches = 0; double ms = 0; int64_t bytes = 0; };
-  struct ProfPending { int entry; cudaEvent_t a, b; };
+  struct ProfPending { int entry; cudaEvent_t a, b; int big_entry; };      // big_entry >= 0: also counted under "<name> (large)"
   std::vector<ProfEntry> prof;
   std::map<std::string, int> prof_index;
   std::vector<ProfPending> prof_pending;
@@ -201,7 +202,20 @@ inline void prof_begin(Ctx* c, const char* what) {
     it = c->prof_index.emplace(name, (int)c->prof.size()).first;
     c->prof.push_back(Ctx::ProfEntry{name, 0, 0.0, 0});
   }
-  Ctx::ProfPending p{it->second, prof_event(c), prof_event(c)};
+  // launches that declare at least kProfLargeBytes (4 M candidates of 12 bytes) are also totalled on their own, so that the
+  // large rounds of a fixpoint can be told from the launch-bound small ones
+  int big = -1;
+  if (c->note_bytes >= kProfLargeBytes) {
+    const std::string bn = name + " (large)";
+    auto bt = c->prof_index.find(bn);
+    if (bt == c->prof_index.end()) {
+      bt = c->prof_index.emplace(bn, (int)c->prof.size()).first;
+      c->prof.push_back(Ctx::ProfEntry{bn, 0, 0.0, 0});
+    }
+    big = bt->second;
+    it = c->prof_index.find(name);                       // the emplace may have moved nothing, but look the entry up again to be safe
+  }
+  Ctx::ProfPending p{it->second, prof_event(c), prof_event(c), big};
   cudaEventRecord(p.a, c->stream);
   c->prof_pending.push_back(p);
 }
@@ -209,7 +223,10 @@ inline void prof_begin(Ctx* c, const char* what) {
 inline void prof_collect(Ctx* c) {
   for (Ctx::ProfPending& p : c->prof_pending) {
     float ms = 0.f;
-    if (cudaEventElapsedTime(&ms, p.a, p.b) == cudaSuccess) c->prof[p.entry].ms += ms;
+    if (cudaEventElapsedTime(&ms, p.a, p.b) == cudaSuccess) {
+      c->prof[p.entry].ms += ms;
+      if (p.big_entry >= 0) c->prof[p.big_entry].ms += ms;
+    }
     c->ev_pool.push_back(p.a); c->ev_pool.push_back(p.b);
   }
   c->prof_pending.clear();
@@ -223,6 +240,7 @@ inline void check_launch(Ctx* c, const char* what) {
     cudaEventRecord(p.b, c->stream);
     c->prof[p.entry].launches += 1;
     c->prof[p.entry].bytes += c->note_bytes;
+    if (p.big_entry >= 0) { c->prof[p.big_entry].launches += 1; c->prof[p.big_entry].bytes += c->note_bytes; }
   }
   c->note_bytes = 0;
 }

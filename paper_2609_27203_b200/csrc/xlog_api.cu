@@ -1298,6 +1298,12 @@ ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*
   } else {
     unsigned long long seen = 0;
     uint32_t rows = n_delta;
+    double expand_ms_seen = 0.0;
+    int64_t expand_launches_seen = 0;
+    {
+      auto it0 = c->prof_index.find("k_res_expand");
+      if (it0 != c->prof_index.end()) { expand_ms_seen = c->prof[it0->second].ms; expand_launches_seen = c->prof[it0->second].launches; }
+    }
     for (;;) {
       resident_body(c, R, specs, is_max, mr, bm_quads, ch_tiles, cudaGraphConditionalHandle{}, 0);
       read_state();
@@ -1308,8 +1314,23 @@ ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*
         rows = out.n_delta;
         // algorithmic bytes of the round's expand launches (per candidate: the looked-up columns and tag, and the slot)
         auto it = c->prof_index.find("k_res_expand");
-        if (it != c->prof_index.end())
-          c->prof[it->second].bytes += (int64_t)(out.candidates - seen) * (4 + (specs[0].has_inner ? 4 * (specs[0].inner_free + 1) : 0));
+        if (it != c->prof_index.end()) {
+          const int64_t bytes = (int64_t)(out.candidates - seen) * (4 + (specs[0].has_inner ? 4 * (specs[0].inner_free + 1) : 0));
+          Ctx::ProfEntry& pe = c->prof[it->second];
+          pe.bytes += bytes;
+          if (bytes >= kProfLargeBytes) {                // this round's launches, totalled on their own like any large launch
+            const double round_ms = pe.ms - expand_ms_seen;
+            const int64_t round_launches = pe.launches - expand_launches_seen;
+            auto bt = c->prof_index.find("k_res_expand (large)");
+            if (bt == c->prof_index.end()) {
+              bt = c->prof_index.emplace("k_res_expand (large)", (int)c->prof.size()).first;
+              c->prof.push_back(Ctx::ProfEntry{"k_res_expand (large)", 0, 0.0, 0});
+            }
+            Ctx::ProfEntry& be = c->prof[bt->second];
+            be.ms += round_ms; be.launches += round_launches; be.bytes += bytes;
+          }
+          expand_ms_seen = c->prof[it->second].ms; expand_launches_seen = c->prof[it->second].launches;
+        }
         seen = out.candidates;
       }
       if (out.status != kResOk || out.n_delta == 0) break;
