@@ -74,7 +74,7 @@ typedef std::map<Key, Acc> AccTable;
 
 struct Binding {                   // what the innermost loop level sees
   int64_t var[MAXV];
-  const Table::value_type* row[3];
+  const Table::value_type* row[4];
   float  tf;                       // fp32 left-to-right otimes
   double td;                       // fp64 left-to-right otimes
 };
@@ -418,7 +418,7 @@ int orc_load(void* e, int rel, const int32_t* rows, const float* tags, int64_t n
 int orc_rule(void* e, int head, int n_head_cols, const int64_t* head_exprs, int n_atoms,
              const int32_t* atom_rel, const int64_t* atom_args, int emit_count, const int32_t* atom_neg) {
   Engine* E = (Engine*)e; Rule r; r.head = head; r.emit_count = emit_count != 0;
-  if (n_atoms < 1 || n_atoms > 3) return -1;
+  if (n_atoms < 1 || n_atoms > 4) return -1;
   for (int c = 0; c < n_head_cols; ++c) {
     Expr x; x.c0 = head_exprs[c * (1 + MAXV)];
     for (int v = 0; v < MAXV; ++v) x.coef[v] = head_exprs[c * (1 + MAXV) + 1 + v];

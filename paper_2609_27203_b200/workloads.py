@@ -152,6 +152,20 @@ def triangle_join_program(r, s, t, semiring=MAXPLUS, name="triangle_join") -> Pr
     )
 
 
+def four_cycle_program(r, s, t, u, semiring=MAXPLUS, name="four_cycle") -> Program:
+    """c4(x,y,z,w) :- r(x,y), s(y,z), t(z,w), u(w,x) over four relations, each given as (col0, col1, tags)."""
+    def rel(x):
+        return ([np.ascontiguousarray(x[0], np.int32), np.ascontiguousarray(x[1], np.int32)], np.ascontiguousarray(x[2], np.float32))
+    return Program(
+        name=name,
+        relations={"r": (2, semiring), "s": (2, semiring), "t": (2, semiring), "u": (2, semiring), "c4": (4, semiring)},
+        rules=[Rule("c4", (V(0), V(1), V(2), V(3)),
+                    (Atom("r", (Var(0), Var(1))), Atom("s", (Var(1), Var(2))), Atom("t", (Var(2), Var(3))), Atom("u", (Var(3), Var(0)))))],
+        facts={"r": rel(r), "s": rel(s), "t": rel(t), "u": rel(u)},
+        outputs=("c4",),
+    )
+
+
 def hot_domain_triangle(n_rows=65536, domain=406, seed=synth.SEED_BASE + 6) -> Program:
     """Three relations of n_rows distinct uniform pairs over a small domain: every join variable is hot, so the two-paths
     of any two relations far outnumber the triangles (65,536 rows over 406 values: about 10.6 M two-paths, 4.2 M triples)."""

@@ -311,3 +311,73 @@ def test_triangle_join_over_three_relations_against_brute_force_and_a_matrix_pro
     assert len(want) == int(round(((M[0] @ M[1]) * M[2].T).sum()))
     # rows come back in ascending (x, y, z)
     assert sorted(got.keys()) == list(zip(cols[0].tolist(), cols[1].tolist(), cols[2].tolist()))
+
+
+def four_cycle_fixture(n_rows, domain, semiring, seed=synth.SEED_BASE + 7):
+    rels = []
+    for k in range(4):
+        a, b = synth.uniform_digraph(domain, n_rows, seed + 17 * k)
+        rels.append((a, b, synth.log_prob_tags(n_rows, seed + 17 * k + 1)))
+    return W.four_cycle_program(*rels, semiring=semiring, name=f"four_cycle_n{n_rows}_d{domain}")
+
+
+def test_four_cycle_join_against_brute_force_and_matrix_products():
+    # c4(x,y,z,w) :- r(x,y), s(y,z), t(z,w), u(w,x) (the four-cycle template of "Worst-case-optimal joins"): the row set by
+    # four nested Python loops, the tag ((w_xy + w_yz) + w_zw) + w_wx in fp32, the row count by trace(R S T U) of the
+    # 0/1 matrices and, under sum-product, the sum of all tags by the trace of the weighted product
+    d = 14
+    prog = four_cycle_fixture(90, d, W.MAXPLUS)
+    o, ids, _ = oracle.load_program(prog)
+    o.run("naive")
+    cols, tags = o.read(ids["c4"])
+    rel, adj = {}, {}
+    for name in ("r", "s", "t", "u"):
+        (a, b), w = prog.facts[name]
+        rel[name] = {(int(x), int(y)): np.float32(v) for x, y, v in zip(a, b, w)}
+        m = np.zeros((d, d))
+        for (x, y) in rel[name]:
+            m[x, y] = 1
+        adj[name] = m
+    want = {}
+    for (x, y), w1 in rel["r"].items():
+        for (y2, z), w2 in rel["s"].items():
+            if y2 != y:
+                continue
+            for (z2, w), w3 in rel["t"].items():
+                if z2 == z and (w, x) in rel["u"]:
+                    want[(x, y, z, w)] = np.float32(np.float32(np.float32(w1 + w2) + w3) + rel["u"][(w, x)])
+    got = {(int(a), int(b), int(c), int(e)): t for a, b, c, e, t in zip(*cols, tags)}
+    assert got.keys() == want.keys() and len(want) > 50
+    assert all(got[k] == want[k] for k in want)
+    assert len(want) == int(round(np.trace(adj["r"] @ adj["s"] @ adj["t"] @ adj["u"])))
+    assert sorted(got.keys()) == list(zip(*(c.tolist() for c in cols)))       # ascending (x, y, z, w)
+
+    sp = four_cycle_fixture(90, d, W.SUMPROD)
+    wm = {}
+    for name in ("r", "s", "t", "u"):
+        (a, b), _ = sp.facts[name]
+        wv = (0.5 + 0.1 * (np.arange(len(a)) % 7)).astype(np.float32)          # weights of order one
+        sp.facts[name] = ([a, b], wv)
+        m = np.zeros((d, d))
+        m[a, b] = wv.astype(np.float64)
+        wm[name] = m
+    o2, ids2, _ = oracle.load_program(sp)
+    o2.run("naive")
+    _, t2 = o2.read(ids2["c4"])
+    assert len(t2) == len(want)
+    assert abs(float(t2.astype(np.float64).sum()) - np.trace(wm["r"] @ wm["s"] @ wm["t"] @ wm["u"])) < 1e-4 * len(t2)
+
+
+def test_four_cycles_of_one_relation_are_the_closed_walks_of_length_four():
+    # over a single 0/1 relation the rows of c4 are the closed walks x -> y -> z -> w -> x: trace(A^4); on the directed
+    # ring of n nodes with both directions there are n * 6 of them (2 choices per step, returning after four steps)
+    n = 9
+    a = np.concatenate([np.arange(n), np.arange(n)]).astype(np.int32)
+    b = np.concatenate([(np.arange(n) + 1) % n, (np.arange(n) - 1) % n]).astype(np.int32)
+    e = (a, b, np.zeros(2 * n, np.float32))
+    o, ids, _ = oracle.load_program(W.four_cycle_program(e, e, e, e))
+    o.run("naive")
+    assert o.size(ids["c4"]) == 6 * n
+    A = np.zeros((n, n))
+    A[a, b] = 1
+    assert o.size(ids["c4"]) == int(round(np.trace(np.linalg.matrix_power(A, 4))))
