@@ -33,7 +33,7 @@ extern "C" {
 #endif
 
 #define XLOG_MAX_ARITY 4
-#define XLOG_MAX_ATOMS 3
+#define XLOG_MAX_ATOMS 4
 #define XLOG_MAX_VARS  8
 
 /* Typed outcomes (Section "GPU residency model": RESOURCE_EXHAUSTED for bytes,
@@ -149,6 +149,11 @@ xlog_status xlog_relation_view(xlog_ctx* ctx, xlog_rel rel, const int32_t** cols
  * number at most four per input row of the largest relation and fit the arena, the
  * multiway join otherwise; XLOG_FLAG_FORCE_WCOJ / XLOG_FLAG_FORCE_CHAIN override it and
  * xlog_receipt.triangle_plan reports the choice.  Both plans produce identical rows.
+ * The four-cycle join  h(x,y,z,w) :- r(x,y), s(y,z), t(z,w), u(w,x)  (same sections: coverage
+ * spans the triangle and 4-cycles) over up to four binary relations, head columns exactly
+ * (x,y,z,w): the two-paths of r and s, then per two-path the intersection of t's out-list of
+ * z with u's in-list of x, count -> scan -> write; rows come out sorted.  It must be the only
+ * rule of its head, outside recursion; RESOURCE_EXHAUSTED if the two-paths do not fit the arena.
  * Negation (Sections "Aggregations and constraints", "Completeness over finite domains":
  * explicit stratified negation-as-failure): a rule of one positive atom followed by one
  * negated atom,  h(..) :- a(..), not b(..).  The negated atom holds iff no row of b matches;

@@ -118,7 +118,7 @@ struct JoinShape {                      // how a two-atom rule is evaluated with
 
 struct RuleC {
   xlog_plan plan;
-  int kind = 0;                         // 1: one atom, 2: two-atom join, 3/4: directed triangle (aggregate / rows), 5: atom + negated atom
+  int kind = 0;                         // 1: one atom, 2: two-atom join, 3/4: directed triangle (aggregate / rows), 5: atom + negated atom, 6: four-cycle (rows)
   int neg_prefix = 0;                   // kind 5: how many leading columns of the negated atom are fixed
   JoinShape shape[2];                   // indexed by the outer atom
 };

@@ -4,6 +4,7 @@
 #include "mirror.cuh"
 #include "resident.cuh"
 #include "triangle.cuh"
+#include "cycle4.cuh"
 
 using namespace xlog;
 
@@ -213,7 +214,7 @@ void add_rule(Ctx* c, const xlog_plan* p, xlog_rule* out) {
   if (!p || !out) fail(XLOG_ERR_INVALID_ARGUMENT, "plan or out is NULL");
   if (p->struct_size != sizeof(xlog_plan)) fail(XLOG_ERR_INVALID_ARGUMENT, "xlog_plan.struct_size mismatch");
   Relation& H = rel_of(c, p->head_rel);
-  if (p->n_atoms < 1 || p->n_atoms > XLOG_MAX_ATOMS) fail(XLOG_ERR_INVALID_ARGUMENT, "n_atoms must be 1..3");
+  if (p->n_atoms < 1 || p->n_atoms > XLOG_MAX_ATOMS) fail(XLOG_ERR_INVALID_ARGUMENT, "n_atoms must be 1..4");
   if (p->n_head_cols < 1 || p->n_head_cols + (p->emit_count_column ? 1 : 0) != H.arity)
     fail(XLOG_ERR_INVALID_ARGUMENT, "head columns do not match the head relation's arity");
   bool bound[XLOG_MAX_VARS] = {false};
@@ -265,6 +266,22 @@ void add_rule(Ctx* c, const xlog_plan* p, xlog_rule* out) {
     r.shape[1] = join_shape(c, *p, 1);
     if (!r.shape[0].ok && !r.shape[1].ok)
       fail(XLOG_ERR_UNSUPPORTED, "two-atom rule must join on one variable with the looked-up side's other columns plain fresh variables");
+  } else if (p->n_atoms == 4) {
+    // four-cycle  h(x,y,z,w) :- r(x,y), s(y,z), t(z,w), u(w,x)
+    const xlog_atom* a = p->atoms;
+    bool ok = p->n_head_cols == 4 && !p->emit_count_column;
+    for (int j = 0; j < 4 && ok; ++j) ok = c->rels[a[j].rel]->arity == 2 && is_plain_var(a[j].args[0]) && is_plain_var(a[j].args[1]);
+    if (ok) {
+      const int hv[4] = {a[0].args[0].var, a[0].args[1].var, a[1].args[1].var, a[2].args[1].var};
+      for (int i = 0; i < 4 && ok; ++i) for (int k = i + 1; k < 4 && ok; ++k) ok = hv[i] != hv[k];
+      ok = ok && a[1].args[0].var == hv[1] && a[2].args[0].var == hv[2] && a[3].args[0].var == hv[3] && a[3].args[1].var == hv[0];
+      for (int h = 0; h < 4 && ok; ++h) {
+        ok = p->head[h].c0 == 0;
+        for (int v = 0; v < XLOG_MAX_VARS; ++v) ok = ok && p->head[h].coef[v] == (v == hv[h] ? 1 : 0);
+      }
+    }
+    if (!ok) fail(XLOG_ERR_UNSUPPORTED, "four-atom rules are supported only as the four-cycle join h(x,y,z,w) :- r(x,y), s(y,z), t(z,w), u(w,x)");
+    r.kind = 6;
   } else {
     // directed triangle  h(x) :- e(x,y), e(y,z), e(z,x)
     const xlog_atom* a = p->atoms;
@@ -1030,6 +1047,89 @@ void triangle_materialise(Ctx* c, Relation& H, const RuleC& r) {
   set_current(H, std::move(kt));
 }
 
+// c4(x,y,z,w) :- r(x,y), s(y,z), t(z,w), u(w,x): the two-paths of r and s through the ordinary join, then per two-path
+// the intersection of t's out-list of z with u's in-list of x (count -> scan -> write; see cycle4.cuh).
+void cycle4_materialise(Ctx* c, Relation& H, const RuleC& r) {
+  Relation& R = *c->rels[r.plan.atoms[0].rel];
+  Relation& S = *c->rels[r.plan.atoms[1].rel];
+  Relation& T = *c->rels[r.plan.atoms[2].rel];
+  Relation& U = *c->rels[r.plan.atoms[3].rel];
+  if (H.n_facts) fail(XLOG_ERR_UNSUPPORTED, "a materialised four-cycle relation cannot also hold loaded facts");
+  c->last_triangle_plan = XLOG_PLAN_WCOJ;
+  if (R.n == 0 || S.n == 0 || T.n == 0 || U.n == 0) { KeyTags empty; set_current(H, std::move(empty)); return; }
+  RuleC two;                                             // tmp(x,y,z) :- r(x,y), s(y,z)
+  two.plan = r.plan;
+  two.plan.n_atoms = 2;
+  two.plan.n_head_cols = 3;
+  two.kind = 2;
+  two.shape[0] = join_shape(c, two.plan, 0);
+  if (!two.shape[0].ok) fail(XLOG_ERR_INTERNAL, "four-cycle: no join path");
+  Relation H2;
+  H2.arity = 3; H2.sr = H.sr;
+  H2.col_max[0] = R.val_max[0] ? R.val_max[0] : R.col_max[0]; H2.col_max[1] = R.val_max[1] ? R.val_max[1] : R.col_max[1];
+  H2.col_max[2] = S.val_max[1] ? S.val_max[1] : S.col_max[1];
+  H2.layout = make_layout(3, H2.col_max);
+  H2.key_bytes = H2.layout.total_bits <= 32 ? 4 : 8;
+  Variant v{&two, 0, full_source(R)};
+  Counted q;
+  count_variant(c, v, H2, q, kSlotTotals);
+  sync_ctrl(c);
+  q.total = c->h_ctrl[kSlotTotals];
+  q.deg.reset(); q.sums.reset();
+  const uint64_t n2 = q.total;
+  const int ckb = H2.key_bytes;
+  const size_t need = (size_t)n2 * (ckb + 4 + 12) + (16u << 20);
+  if (n2 > kSortMaxN) fail(XLOG_ERR_CAPACITY_EXCEEDED, "four-cycle: more than 2^30 - 1 two-paths");
+  if (need > c->arena.largest_free() / 2) fail(XLOG_ERR_RESOURCE_EXHAUSTED, "four-cycle: the two-paths do not fit the arena");
+  c->r_candidates += (int64_t)n2;
+  if (n2 == 0) { KeyTags empty; set_current(H, std::move(empty)); return; }
+  DevBuf k0(c, n2 * ckb), t0(c, n2 * 4);
+  c->note_bytes = (int64_t)n2 * (ckb + 4 + 8);
+  launch_expand<false>(c, q, 0, n2, ckb, k0.p, t0.as<float>(), BwdArgs{});
+  q.start.reset(); q.rowinfo.reset();
+  Index& tix = ensure_index(c, T, 0);
+  Index& uix = ensure_index(c, U, 1);
+  Cycle4 P{};
+  P.L2 = H2.layout; P.L = H.layout;
+  P.t_domain = tix.domain; P.t_off = tix.off.as<uint32_t>(); P.t_w = tix.other[0]; P.t_tag = tix.tags;
+  P.u_domain = uix.domain; P.u_off = uix.off.as<uint32_t>(); P.u_w = uix.other[0]; P.u_tag = uix.tags;
+  P.times = H.sr == XLOG_SR_SUMPROD ? 1 : 0;
+  DevBuf cnt(c, n2 * 4), off(c, n2 * 8);
+  const unsigned tiles = (unsigned)((n2 + kScanTile - 1) / kScanTile);
+  DevBuf sums(c, (size_t)tiles * 8);
+  zero_ctrl(c, kSlotTotals);
+  const unsigned grid = (unsigned)std::min<uint64_t>((n2 + 255) / 256, (uint64_t)kSMs * 8);
+  KeyTags kt;
+#define XLOG_C4(K2, KH, EMIT, KEYS, TAGS)                                                                                          \
+  XLOG_LAUNCH(c, (k_cycle4<K2, KH, EMIT>), grid, 256, 0, P, (const K2*)k0.p, (const float*)t0.as<float>(), n2, cnt.as<uint32_t>(),  \
+              (const uint64_t*)off.as<uint64_t>(), (KH*)(KEYS), (float*)(TAGS))
+#define XLOG_C4_DISPATCH(EMIT, KEYS, TAGS)                                        \
+  do {                                                                            \
+    if (ckb == 4 && H.key_bytes == 4) XLOG_C4(uint32_t, uint32_t, EMIT, KEYS, TAGS); \
+    else if (ckb == 4) XLOG_C4(uint32_t, uint64_t, EMIT, KEYS, TAGS);             \
+    else if (H.key_bytes == 4) XLOG_C4(uint64_t, uint32_t, EMIT, KEYS, TAGS);     \
+    else XLOG_C4(uint64_t, uint64_t, EMIT, KEYS, TAGS);                           \
+  } while (0)
+  c->note_bytes = (int64_t)n2 * (ckb + 4) + (int64_t)(T.n + U.n) * 4;
+  XLOG_C4_DISPATCH(false, nullptr, nullptr);
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)cnt.as<uint32_t>(), (int64_t)n2, sums.as<uint64_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, sums.as<uint64_t>(), (int64_t)tiles, (uint64_t*)(c->d_ctrl + kSlotTotals));
+  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)cnt.as<uint32_t>(), (int64_t)n2,
+              (const uint64_t*)sums.as<uint64_t>(), off.as<uint64_t>());
+  sync_ctrl(c);                                            // the one small metadata read that sizes the output
+  const uint64_t total = c->h_ctrl[kSlotTotals];
+  if (total > kSortMaxN) fail(XLOG_ERR_CAPACITY_EXCEEDED, "materialised four-cycle relation exceeds 2^30 - 1 rows");
+  c->r_unique += (int64_t)total;
+  kt.n = (uint32_t)total;
+  kt.keys = DevBuf(c, (size_t)std::max<uint64_t>(total, 1) * H.key_bytes);
+  kt.tags = DevBuf(c, (size_t)std::max<uint64_t>(total, 1) * 4);
+  c->note_bytes = (int64_t)n2 * (ckb + 4 + 8) + (int64_t)(T.n + U.n) * 8 + (int64_t)total * (H.key_bytes + 4);
+  XLOG_C4_DISPATCH(true, kt.keys.p, kt.tags.p);
+#undef XLOG_C4_DISPATCH
+#undef XLOG_C4
+  set_current(H, std::move(kt));
+}
+
 void triangle_aggregate(Ctx* c, Relation& H, const RuleC& r) {
   if (c->rels[r.plan.atoms[0].rel]->is_head && r.plan.atoms[0].rel == r.plan.head_rel) fail(XLOG_ERR_UNSUPPORTED, "recursive triangle rule");
   switch (H.sr) {
@@ -1045,7 +1145,7 @@ void triangle_aggregate(Ctx* c, Relation& H, const RuleC& r) {
 void rule_backward(Ctx* c, const RuleC& r, const float* g, float* const* grads) {
   Relation& H = *c->rels[r.plan.head_rel];
   if (H.sr != XLOG_SR_LOGSUMEXP && H.sr != XLOG_SR_SUMPROD) fail(XLOG_ERR_UNSUPPORTED, "backward is defined for logsumexp and sum heads only");
-  if (r.kind == 3 || r.kind == 4) fail(XLOG_ERR_UNSUPPORTED, "backward of the triangle rules is not built");
+  if (r.kind == 3 || r.kind == 4 || r.kind == 6) fail(XLOG_ERR_UNSUPPORTED, "backward of the triangle and four-cycle rules is not built");
   for (int j = 0; j < r.plan.n_atoms; ++j) {
     if (!grads[j]) fail(XLOG_ERR_INVALID_ARGUMENT, "NULL gradient buffer");
     if (r.plan.atoms[j].rel == r.plan.head_rel) fail(XLOG_ERR_UNSUPPORTED, "backward of a recursive rule");
@@ -1089,9 +1189,10 @@ void stratum_once(Ctx* c, int head, const std::vector<const RuleC*>& rs) {
   ++c->r_iterations;
   if (rs.size() == 1 && rs[0]->kind == 3) { triangle_aggregate(c, H, *rs[0]); return; }
   if (rs.size() == 1 && rs[0]->kind == 4) { triangle_materialise(c, H, *rs[0]); c->r_new += H.n; return; }
+  if (rs.size() == 1 && rs[0]->kind == 6) { cycle4_materialise(c, H, *rs[0]); c->r_new += H.n; return; }
   std::vector<Variant> vs;
   for (const RuleC* r : rs) {
-    if (r->kind == 3 || r->kind == 4) fail(XLOG_ERR_UNSUPPORTED, "a triangle rule must be the only rule of its head");
+    if (r->kind == 3 || r->kind == 4 || r->kind == 6) fail(XLOG_ERR_UNSUPPORTED, "a triangle or four-cycle rule must be the only rule of its head");
     int outer = 0;
     if (r->kind == 2 && !r->shape[0].ok) outer = 1;
     vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
@@ -1131,7 +1232,7 @@ bool mirror_applies(Ctx* c, const std::vector<int>& comp, const std::vector<cons
   if (H.sr != XLOG_SR_MAXPLUS && H.sr != XLOG_SR_MINPLUS) return false;
   if (H.layout.total_bits > kMirrorMaxBits || H.key_bytes != 4) return false;
   for (const RuleC* r : rs) {
-    if (r->plan.emit_count_column || r->kind == 3 || r->kind == 4) return false;
+    if (r->plan.emit_count_column || r->kind == 3 || r->kind == 4 || r->kind == 6) return false;
     int in = 0, pos = 0;
     for (int j = 0; j < r->plan.n_atoms; ++j)
       if (r->plan.atoms[j].rel == comp[0]) { if (r->plan.atoms[j].negated) return false; ++in; pos = j; }
@@ -1607,7 +1708,7 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
     fail(XLOG_ERR_UNSUPPORTED, "relation '" + c->rels[p]->name + "': only max/min tags may be aggregated inside a recursive component");
   for (const RuleC* r : rs) {
     if (r->plan.emit_count_column) fail(XLOG_ERR_UNSUPPORTED, "count inside a recursive component");
-    if (r->kind == 3 || r->kind == 4) fail(XLOG_ERR_UNSUPPORTED, "triangle rule inside a recursive component");
+    if (r->kind == 3 || r->kind == 4 || r->kind == 6) fail(XLOG_ERR_UNSUPPORTED, "triangle or four-cycle rule inside a recursive component");
   }
   if (mirror_applies(c, comp, rs)) { stratum_recursive_mirror(c, comp[0], rs); return; }
   std::vector<KeyTags> delta(c->rels.size());

@@ -166,6 +166,17 @@ def four_cycle_program(r, s, t, u, semiring=MAXPLUS, name="four_cycle") -> Progr
     )
 
 
+def uniform_four_cycle(n_rows=3000, domain=120, semiring=MAXPLUS, seed=synth.SEED_BASE + 7) -> Program:
+    """Four relations of n_rows distinct uniform pairs over `domain` values (tags: log-probabilities)."""
+    rels = []
+    for k in range(4):
+        a, b = synth.uniform_digraph(domain, n_rows, seed + 17 * k)
+        rels.append((a, b, synth.log_prob_tags(n_rows, seed + 17 * k + 1)))
+    p = four_cycle_program(*rels, semiring=semiring, name=f"four_cycle_n{n_rows}_d{domain}")
+    p.info.update(n_rows=n_rows, domain=domain)
+    return p
+
+
 def hot_domain_triangle(n_rows=65536, domain=406, seed=synth.SEED_BASE + 6) -> Program:
     """Three relations of n_rows distinct uniform pairs over a small domain: every join variable is hot, so the two-paths
     of any two relations far outnumber the triangles (65,536 rows over 406 values: about 10.6 M two-paths, 4.2 M triples)."""

@@ -14,7 +14,7 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libxlog.so")
 
-MAX_ARITY, MAX_ATOMS, MAX_VARS = 4, 3, 8
+MAX_ARITY, MAX_ATOMS, MAX_VARS = 4, 4, 8
 SEMIRING = {"maxplus": 0, "minplus": 1, "logsumexp": 2, "sumprod": 3}
 STATUS = ["OK", "INVALID_ARGUMENT", "INVALID_VALUE", "UNSUPPORTED", "RESOURCE_EXHAUSTED", "CAPACITY_EXCEEDED",
           "CONVERGENCE_FAILURE", "BUFFER_TOO_SMALL", "INVALID_STATE", "CUDA", "INTERNAL"]

@@ -303,3 +303,57 @@ def test_stratified_negation_matches_oracle():
         c2.fixpoint()
     assert e.value.status == "UNSUPPORTED"
     c2.close()
+
+
+def check_four_cycle(prog, what, **kw):
+    from paper_2609_27203_b200 import xlog
+    ctx, gids, _, o, oids, _, receipt = both(prog, **kw)
+    got, want = ctx.read(gids["c4"]), o.read(oids["c4"])
+    rep = H.compare_relations(got, want, what=what)
+    assert rep["bit_unequal"] == 0                # ((w_xy (x) w_yz) (x) w_zw) (x) w_wx in fp32 on both sides
+    assert receipt["derived_tuples"] == len(want[1]) and receipt["triangle_plan"] == xlog.PLAN_WCOJ
+    ctx.close()
+    return len(want[1])
+
+
+def test_four_cycle_join_matches_the_oracle():
+    # dense small domain (every two-path has two long lists: the warp-cooperative walk), sparse (short lists: a thread
+    # per two-path), sum-product tags, and a skewed graph used four times (hub two-paths next to empty ones)
+    assert check_four_cycle(W.uniform_four_cycle(3000, 70), "dense") > 100000
+    assert check_four_cycle(W.uniform_four_cycle(20000, 2500), "sparse") > 0
+    sp = W.uniform_four_cycle(2500, 90, W.SUMPROD)
+    for name in ("r", "s", "t", "u"):
+        (a, b), _ = sp.facts[name]
+        sp.facts[name] = ([a, b], (0.5 + 0.125 * (np.arange(len(a)) % 9)).astype(np.float32))
+    assert check_four_cycle(sp, "sum-product") > 10000
+    s, d, _ = synth.rmat_graph(9, 6, synth.SEED_BASE + 71, "n01")
+    e = (s, d, synth.log_prob_tags(len(s), synth.SEED_BASE + 72))
+    assert check_four_cycle(W.four_cycle_program(e, e, e, e, name="four_cycle_rmat9"), "rmat") > 10000
+
+
+def test_four_cycle_edge_cases():
+    from paper_2609_27203_b200 import xlog
+    # a relation that closes nothing; an empty relation; 64-bit head keys (four 16-bit columns); ragged column maxima
+    e = (np.array([0, 1, 2, 3], np.int32), np.array([1, 2, 3, 0], np.int32), np.array([0.5, 0.25, 0.125, 1.0], np.float32))
+    assert check_four_cycle(W.four_cycle_program(e, e, e, e), "one ring") == 4
+    none = (np.array([7], np.int32), np.array([8], np.int32), np.array([0.0], np.float32))
+    assert check_four_cycle(W.four_cycle_program(e, e, e, none), "u closes nothing") == 0
+    empty = (np.zeros(0, np.int32), np.zeros(0, np.int32), np.zeros(0, np.float32))
+    assert check_four_cycle(W.four_cycle_program(e, e, empty, e), "empty t") == 0
+    wide = W.uniform_four_cycle(3000, 70)
+    for name in ("r", "s", "t", "u"):
+        (a, b), w = wide.facts[name]
+        wide.facts[name] = ([(a * 900 + 11).astype(np.int32), (b * 900 + 11).astype(np.int32)], w)
+    assert check_four_cycle(wide, "64-bit keys") > 100000
+    rag = W.uniform_four_cycle(3000, 70)
+    (a, b), w = rag.facts["r"]
+    rag.facts["r"] = ([np.concatenate([a, [900, 3]]).astype(np.int32), np.concatenate([b, [5, 901]]).astype(np.int32)],
+                      np.concatenate([w, [-0.1, -0.2]]).astype(np.float32))
+    assert check_four_cycle(rag, "ragged maxima") > 100000
+    # anything else with four atoms is refused
+    bad = W.uniform_four_cycle(10, 5)
+    bad.rules[0] = W.Rule("c4", (W.V(0), W.V(1), W.V(2), W.V(3)),
+                          (W.Atom("r", (W.Var(0), W.Var(1))), W.Atom("s", (W.Var(1), W.Var(2))), W.Atom("t", (W.Var(2), W.Var(3))), W.Atom("u", (W.Var(0), W.Var(3)))))
+    with pytest.raises(xlog.XlogError) as ei:
+        xlog.load_program(bad, arena_bytes=1 << 26)
+    assert ei.value.status == "UNSUPPORTED"

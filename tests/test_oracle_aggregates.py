@@ -313,12 +313,8 @@ def test_triangle_join_over_three_relations_against_brute_force_and_a_matrix_pro
     assert sorted(got.keys()) == list(zip(cols[0].tolist(), cols[1].tolist(), cols[2].tolist()))
 
 
-def four_cycle_fixture(n_rows, domain, semiring, seed=synth.SEED_BASE + 7):
-    rels = []
-    for k in range(4):
-        a, b = synth.uniform_digraph(domain, n_rows, seed + 17 * k)
-        rels.append((a, b, synth.log_prob_tags(n_rows, seed + 17 * k + 1)))
-    return W.four_cycle_program(*rels, semiring=semiring, name=f"four_cycle_n{n_rows}_d{domain}")
+def four_cycle_fixture(n_rows, domain, semiring):
+    return W.uniform_four_cycle(n_rows, domain, semiring)
 
 
 def test_four_cycle_join_against_brute_force_and_matrix_products():
