@@ -58,6 +58,10 @@ def make_program(name: str, scale: int | None, sources: int | None = None):
         # the triangle-join fixture of the paper's WCOJ ablation: three relations of 2^scale rows over a hot domain
         s = scale or 16
         return W.hot_domain_triangle(n_rows=1 << s, domain=406 if s == 16 else max(int(1.4 * 2 ** (s / 2)), 8)), 2 << 30
+    if name == "cycle4":
+        # four-cycle join over four relations of 2^scale uniform rows, one pair in sixteen present (2^24 four-cycles at scale 16)
+        s = scale or 16
+        return W.uniform_four_cycle(n_rows=1 << s, domain=int(4 * 2 ** (s / 2))), 4 << 30
     if name == "digits":
         return W.config4(), 1 << 30
     raise SystemExit(f"unknown workload {name}")
@@ -268,6 +272,21 @@ def run_ours(args):
         if dom == "k_tri_edges" and "n_edges" in program.info:
             probes = (d["bytes"] - 12.0 * program.info["n_edges"] * d["launches"]) / 4.0
             alu = {"achieved": probes / (d["ms"] / 1e3) / 1e9, "peak": 148 * 4 * 1.965 / 6.5, "unit": "Gprobe/s"}
+    if dom == "k_cycle4" and program.info.get("domain", 1 << 30) <= 4096:
+        bound = "alu"      # sorted-list intersections served from L1 / L2 (DRAM 1 % busy under ncu), as for the triangles
+        # unit of work: one probe = one walked entry of the shorter list, searched in the other list; both launches (count, write)
+        # walk every two-path's list.  ncu at scale 16: 2.26e9 warp instructions for 5.0e8 probes = 4.5 per probe.
+        nd = program.info["domain"]
+        adj = {}
+        for nm in ("r", "s", "t", "u"):
+            (ca, cb), _ = program.facts[nm]
+            m = np.zeros((nd, nd), np.float64)
+            m[ca, cb] = 1.0
+            adj[nm] = m
+        two_paths = adj["r"] @ adj["s"]                                            # [x, z]
+        walk = np.minimum(adj["t"].sum(axis=1)[None, :], adj["u"].sum(axis=0)[:, None])     # min(out_t(z), in_u(x))
+        probes = float((two_paths * walk).sum()) * d["launches"]
+        alu = {"achieved": probes / (d["ms"] / 1e3) / 1e9, "peak": 148 * 4 * 1.965 / 4.5, "unit": "Gprobe/s"}
     roofline = {"bound": bound, "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src,
                 "traffic": None if ratio is None else ratio * d["bytes"] / d["launches"],
@@ -346,7 +365,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         # the oracle as it stands, on this machine's host cores, on a bounded sample of the same workload
         # bounded sample (about 10-30 s of CPU work): the full workload where the oracle manages it, else a smaller R-MAT scale
-        cpu_scale = args.cpu_scale or {"triangles": 14, "reach": 16, "wcoj": 13}.get(args.workload)
+        cpu_scale = args.cpu_scale or {"triangles": 14, "reach": 16, "wcoj": 13, "cycle4": 15}.get(args.workload)
         sample, _ = make_program(args.workload, cpu_scale) if cpu_scale else (program, 0)
         sec, stats, _o = run_oracle_once(sample)
         out["cpu_baseline"] = {"value": stats["derived_tuples"] / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
@@ -365,10 +384,10 @@ def run_reference(args):
     rank, _, world = dist_env()
     if rank != 0:
         return
-    est20 = {"sssp": 16.0, "reach": 600.0, "closure": 3.0, "triangles": 200.0, "digits": 10.0, "wcoj": 60.0}[args.workload]
+    est20 = {"sssp": 16.0, "reach": 600.0, "closure": 3.0, "triangles": 200.0, "digits": 10.0, "wcoj": 60.0, "cycle4": 60.0}[args.workload]
     scale = args.scale
-    if args.workload in ("sssp", "reach", "triangles", "wcoj") and scale is None:
-        full = {"sssp": 20, "reach": 22, "triangles": 18, "wcoj": 16}[args.workload]
+    if args.workload in ("sssp", "reach", "triangles", "wcoj", "cycle4") and scale is None:
+        full = {"sssp": 20, "reach": 22, "triangles": 18, "wcoj": 16, "cycle4": 16}[args.workload]
         scale = full
         while scale > 8 and (args.steps + args.warmup) * est20 * 2.0 ** (scale - full) > 150.0:
             scale -= 1
@@ -401,7 +420,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="sssp", choices=["sssp", "closure", "reach", "triangles", "digits", "wcoj"])
+    ap.add_argument("--workload", default="sssp", choices=["sssp", "closure", "reach", "triangles", "digits", "wcoj", "cycle4"])
     ap.add_argument("--scale", type=int, default=None, help="R-MAT scale override (smaller cases for profiling)")
     ap.add_argument("--sources", type=int, default=None, help="reach: number of sources (fewer for a small profiling case)")
     ap.add_argument("--triangle-plan", default="auto", choices=["auto", "wcoj", "chain"], help="wcoj workload: force a join plan")
