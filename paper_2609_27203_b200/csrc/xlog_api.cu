@@ -563,6 +563,7 @@ template <int MODE, int SINK>
 void launch_expand_mode(Ctx* c, Counted& q, uint64_t lo, uint64_t hi, int ckb, void* ckeys, float* ctags, const BwdArgs& bw, const MirrorArgs& mr) {
   constexpr uint32_t tile = SINK == kSinkWrite ? kExpTileWrite : kExpTileMirror;
   const unsigned blocks = (unsigned)((hi - lo + tile - 1) / tile);
+  if (blocks == 0) return;                               // no candidates in the range
   const uint64_t* st = q.start.as<uint64_t>();
   const uint4* ri = q.rowinfo.as<uint4>();
   uint32_t* err = ctrl_u32(c, kSlotErr);
@@ -628,6 +629,9 @@ KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Sour
   if (!counted.empty()) {
     sync_ctrl(c);
     for (Counted& q : counted) { q.total = c->h_ctrl[q.slot]; total += q.total; q.deg.reset(); q.sums.reset(); }
+    // a variant without candidates takes no part in the batches below (left in, it would open one more, empty batch
+    // after the last full one)
+    counted.erase(std::remove_if(counted.begin(), counted.end(), [](const Counted& q) { return q.total == 0; }), counted.end());
   }
   c->r_candidates += (int64_t)total;
   KeyTags result;
@@ -678,6 +682,7 @@ KeyTags evaluate(Ctx* c, Relation& H, std::vector<Variant>& variants, const Sour
     if (result.n == 0) result = std::move(part);
     else {
       // a later batch: union with oplus into the running result
+      if (result.n_slot >= 0) fail(XLOG_ERR_INTERNAL, "evaluate: a deferred row count met a second candidate batch");
       MergeResult m;
       DISPATCH_K(ckb, m = merge<K>(c, H.sr, part.keys.as<K>(), part.tags.as<float>(), part.n, -1, result.keys.as<K>(), result.tags.as<float>(),
                                     result.n, false, false));
@@ -1008,6 +1013,7 @@ void triangle_materialise(Ctx* c, Relation& H, const RuleC& r) {
     if (chain) {
       c->r_candidates += (int64_t)q.total;
       c->last_triangle_plan = XLOG_PLAN_CHAIN;
+      if (q.total == 0) { KeyTags empty; set_current(H, std::move(empty)); return; }      // no two-path at all
       triangle_chain(c, H, H2, q, T);
       return;
     }
@@ -1698,7 +1704,7 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
   if (c->flags & XLOG_FLAG_CHECK_INVARIANTS) {
     XLOG_LAUNCH(c, (k_check_sorted<uint32_t>), grid_for(H.n, 256), 256, 0, (const uint32_t*)H.keys(), (int64_t)H.n, ctrl_u32(c, kSlotErr));
     sync_ctrl(c);
-    if ((uint64_t)(uint32_t)c->h_ctrl[kSlotA] != n_out) fail(XLOG_ERR_INTERNAL, "tag mirror: occupied slots disagree with the tuple count");
+    if (n_out && (uint64_t)(uint32_t)c->h_ctrl[kSlotA] != n_out) fail(XLOG_ERR_INTERNAL, "tag mirror: occupied slots disagree with the tuple count");
   }
 }
 
