@@ -92,7 +92,7 @@ def random_program(seed: int) -> W.Program:
                           (Atom("e", (Var(0), Var(1))), Atom("f", (Var(1), Var(2))), Atom("f", (Var(2), Var(3))), Atom("e", (Var(3), Var(0))))))
         outputs += ["tri", "c4"]
     # a non-recursive aggregate stratum on its own relations
-    agg = int(rng.integers(0, 3))
+    agg = int(rng.integers(0, 8))
     if agg == 0:
         rels["a"] = (2, W.LOGSUMEXP); rels["b"] = (2, W.LOGSUMEXP); rels["s"] = (2, W.LOGSUMEXP)
         facts["a"] = _edb(rng, dom, 2, int(rng.integers(1, 4 * dom)), W.LOGSUMEXP)
@@ -104,4 +104,47 @@ def random_program(seed: int) -> W.Program:
         facts["c"] = _edb(rng, dom, 2, int(rng.integers(1, 4 * dom)), W.SUMPROD)
         rules.append(Rule("deg", (V(0),), (Atom("c", (Var(0), Var(1))),), emit_count=True))
         outputs.append("deg")
+    elif agg == 2:      # two rules and loaded facts into one logsumexp head
+        rels["a"] = (2, W.LOGSUMEXP); rels["b"] = (2, W.LOGSUMEXP); rels["s"] = (2, W.LOGSUMEXP)
+        facts["a"] = _edb(rng, dom, 2, int(rng.integers(1, 4 * dom)), W.LOGSUMEXP)
+        facts["b"] = _edb(rng, dom, 2, int(rng.integers(1, 4 * dom)), W.LOGSUMEXP)
+        facts["s"] = _edb(rng, dom, 2, int(rng.integers(0, dom)), W.LOGSUMEXP)
+        rules.append(Rule("s", (V(0), V(2)), (Atom("a", (Var(0), Var(1))), Atom("b", (Var(1), Var(2))))))
+        rules.append(Rule("s", (V(1), V(0)), (Atom("a", (Var(0), Var(1))),)))
+        outputs.append("s")
+    elif agg == 3:      # affine patterns on both atoms and an affine head column (the digit-sum shape)
+        rels["d"] = (2, W.LOGSUMEXP); rels["t"] = (2, W.LOGSUMEXP)
+        n_img = 2 * int(rng.integers(1, 3 * dom))
+        k = int(rng.integers(2, 11))
+        img = np.repeat(np.arange(n_img, dtype=np.int32), k)
+        dig = np.tile(np.arange(k, dtype=np.int32), n_img)
+        keep = rng.random(len(img)) < 0.8
+        facts["d"] = ([img[keep], dig[keep]], rng.normal(0, 1, int(keep.sum())).astype(np.float32))
+        rules.append(Rule("t", (V(0), W.Affine(0, ((1, 1), (2, 1)))), (Atom("d", (Var(0, 2, 0), Var(1))), Atom("d", (Var(0, 2, 1), Var(2))))))
+        outputs.append("t")
+    elif agg == 4:      # a three-column relation: projected with a reduction, and looked up by its first column
+        rels["g"] = (3, sr); rels["proj"] = (2, sr); rels["wide"] = (3, sr)
+        facts["g"] = _edb(rng, dom, 3, int(rng.integers(1, 6 * dom)), sr)
+        rules.append(Rule("proj", (V(0), V(2)), (Atom("g", (Var(0), Var(1), Var(2))),)))
+        rules.append(Rule("wide", (V(0), V(2), V(3)), (Atom("f", (Var(0), Var(1))), Atom("g", (Var(1), Var(2), Var(3))))))
+        outputs += ["proj", "wide"]
+    elif agg == 5:      # two-step walk counts under sum-product, with a constant on the scanned atom in a second rule
+        rels["c"] = (2, W.SUMPROD); rels["walk"] = (2, W.SUMPROD); rels["from0"] = (1, W.SUMPROD)
+        facts["c"] = _edb(rng, dom, 2, int(rng.integers(1, 4 * dom)), W.SUMPROD)
+        rules.append(Rule("walk", (V(0), V(2)), (Atom("c", (Var(0), Var(1))), Atom("c", (Var(1), Var(2))))))
+        rules.append(Rule("from0", (V(1),), (Atom("c", (Const(int(rng.integers(0, dom))), Var(0))), Atom("c", (Var(0), Var(1))))))
+        outputs += ["walk", "from0"]
     return W.Program(f"random_{seed}_shape{shape}_agg{agg}", rels, rules, facts, tuple(outputs))
+
+
+def stretch(program: W.Program, stride: int, offset: int = 0) -> W.Program:
+    """The same program with every stored value v replaced by v * stride + offset (and constants likewise): wide columns,
+    64-bit packed keys.  Only for programs whose rules use plain variables and constants."""
+    facts = {}
+    for name, (cols, tags) in program.facts.items():
+        facts[name] = ([(c.astype(np.int64) * stride + offset).astype(np.int32) for c in cols], tags)
+    rules = []
+    for r in program.rules:
+        atoms = tuple(Atom(a.rel, tuple(Const(g.value * stride + offset) if isinstance(g, Const) else g for g in a.args), a.negated) for a in r.atoms)
+        rules.append(Rule(r.head, r.head_exprs, atoms, r.emit_count))
+    return W.Program(program.name + f"_x{stride}", dict(program.relations), rules, facts, program.outputs)
