@@ -199,7 +199,7 @@ typedef struct {
   int64_t  kernel_launches;
   int64_t  peak_arena_bytes;
   double   device_ms;              /* CUDA-event time of the whole call on the ctx stream */
-  int32_t  triangle_plan;          /* XLOG_PLAN_*: how the last materialised triangle join of this call was evaluated */
+  int32_t  triangle_plan;          /* XLOG_PLAN_*: how the last materialised triangle join of this call was evaluated (a four-cycle join reports WCOJ) */
   int32_t  reserved;
 } xlog_receipt;
 #define XLOG_PLAN_NONE  0
