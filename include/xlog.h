@@ -223,7 +223,8 @@ xlog_status xlog_ctx_reset_idb(xlog_ctx* ctx);
  * order; each distinct buffer is zero-filled first, then
  *   LOGSUMEXP:  grad_j[row] += g[h] * exp(sum_i tag_i - out[h])
  *   SUMPROD:    grad_j[row] += g[h] * prod_{i != j} tag_i
- * Passing the same pointer for two atoms of one relation yields the sum. */
+ * Passing the same pointer for two atoms of one relation yields the sum.  A pointer
+ * whose relation holds no rows may be NULL; otherwise NULL is INVALID_ARGUMENT. */
 xlog_status xlog_rule_backward(xlog_ctx* ctx, xlog_rule rule, const float* grad_head, float* const* grad_atoms);
 
 /* ---- the sort on its own (paper kernel table: `sort`) ---------------------------------

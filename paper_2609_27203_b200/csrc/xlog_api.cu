@@ -1153,7 +1153,7 @@ void rule_backward(Ctx* c, const RuleC& r, const float* g, float* const* grads) 
   if (H.sr != XLOG_SR_LOGSUMEXP && H.sr != XLOG_SR_SUMPROD) fail(XLOG_ERR_UNSUPPORTED, "backward is defined for logsumexp and sum heads only");
   if (r.kind == 3 || r.kind == 4 || r.kind == 6) fail(XLOG_ERR_UNSUPPORTED, "backward of the triangle and four-cycle rules is not built");
   for (int j = 0; j < r.plan.n_atoms; ++j) {
-    if (!grads[j]) fail(XLOG_ERR_INVALID_ARGUMENT, "NULL gradient buffer");
+    if (!grads[j] && c->rels[r.plan.atoms[j].rel]->n) fail(XLOG_ERR_INVALID_ARGUMENT, "NULL gradient buffer");
     if (r.plan.atoms[j].rel == r.plan.head_rel) fail(XLOG_ERR_UNSUPPORTED, "backward of a recursive rule");
   }
   int outer = 0;
@@ -1163,7 +1163,7 @@ void rule_backward(Ctx* c, const RuleC& r, const float* g, float* const* grads) 
   for (int j = 0; j < r.plan.n_atoms; ++j) {
     bool seen = false;
     for (int i = 0; i < j; ++i) seen = seen || grads[i] == grads[j];
-    if (!seen) XLOG_CUDA(cudaMemsetAsync(grads[j], 0, (size_t)c->rels[r.plan.atoms[j].rel]->n * 4, c->stream));
+    if (!seen && grads[j]) XLOG_CUDA(cudaMemsetAsync(grads[j], 0, (size_t)c->rels[r.plan.atoms[j].rel]->n * 4, c->stream));
   }
   Relation& RA = *c->rels[r.plan.atoms[outer].rel];
   if (RA.n == 0 || H.n == 0) { XLOG_CUDA(cudaStreamSynchronize(c->stream)); return; }
@@ -2028,7 +2028,8 @@ xlog_status xlog_profile_reset(xlog_ctx* c) {
 xlog_status xlog_rule_backward(xlog_ctx* c, xlog_rule rule, const float* grad_head, float* const* grad_atoms) {
   return guarded(c, [&] {
     if (rule < 0 || rule >= (int)c->rules.size()) fail(XLOG_ERR_INVALID_ARGUMENT, "bad rule handle");
-    if (!grad_head || !grad_atoms) fail(XLOG_ERR_INVALID_ARGUMENT, "NULL gradient pointer");
+    if (!grad_atoms) fail(XLOG_ERR_INVALID_ARGUMENT, "NULL gradient pointer");
+    if (!grad_head && c->rels[c->rules[rule].plan.head_rel]->n) fail(XLOG_ERR_INVALID_ARGUMENT, "NULL gradient pointer");   // an empty head has no gradient rows
     if (c->poisoned || !c->evaluated || c->idb_dirty) fail(XLOG_ERR_INVALID_STATE, "xlog_rule_backward needs a successful xlog_fixpoint first");
     rule_backward(c, c->rules[rule], grad_head, grad_atoms);
   });

@@ -20,9 +20,11 @@ def _edb(rng, dom, arity, n, sr):
     return cols, tags.astype(np.float32)
 
 
-def random_program(seed: int) -> W.Program:
+def random_program(seed: int, dom: int = 0) -> W.Program:
+    """dom = 0: the domain size is drawn from {5, 17, 60, 250}; otherwise it is `dom` (relations grow with it)."""
     rng = np.random.default_rng(seed)
-    dom = int(rng.choice([5, 17, 60, 250]))
+    drawn = int(rng.choice([5, 17, 60, 250]))
+    dom = dom or drawn
     sr = str(rng.choice([W.MAXPLUS, W.MINPLUS]))
     n_e = int(rng.integers(0, 5 * dom)) if rng.random() > 0.05 else 0
     n_f = int(rng.integers(1, 3 * dom))

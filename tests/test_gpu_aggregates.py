@@ -357,3 +357,19 @@ def test_four_cycle_edge_cases():
     with pytest.raises(xlog.XlogError) as ei:
         xlog.load_program(bad, arena_bytes=1 << 26)
     assert ei.value.status == "UNSUPPORTED"
+
+
+def test_backward_of_a_rule_whose_head_is_empty():
+    # a and b share no join value: the head is empty, its gradient has no rows (a NULL pointer is accepted), and both
+    # atom gradients come back zero
+    import torch
+    a = ([np.array([0, 1], np.int32), np.array([5, 6], np.int32)], np.array([0.1, 0.2], np.float32))
+    b = ([np.array([7, 8], np.int32), np.array([1, 2], np.int32)], np.array([0.3, 0.4], np.float32))
+    prog = W.Program("empty_head", {"a": (2, W.LOGSUMEXP), "b": (2, W.LOGSUMEXP), "s": (2, W.LOGSUMEXP)},
+                     [W.Rule("s", (W.V(0), W.V(2)), (W.Atom("a", (W.Var(0), W.Var(1))), W.Atom("b", (W.Var(1), W.Var(2)))))],
+                     {"a": a, "b": b}, ("s",))
+    ctx, gids, grules, o, oids, orules, _ = both(prog)
+    assert ctx.size(gids["s"]) == 0 == o.size(oids["s"])
+    parts = ctx.backward(grules[0], torch.zeros(0, device="cuda"), same_buffer_for_same_relation=False)
+    assert all(float(p.abs().sum().item()) == 0.0 and p.numel() == 2 for p in parts)
+    ctx.close()
