@@ -272,7 +272,7 @@ def run_ours(args):
         if dom == "k_tri_edges" and "n_edges" in program.info:
             probes = (d["bytes"] - 12.0 * program.info["n_edges"] * d["launches"]) / 4.0
             alu = {"achieved": probes / (d["ms"] / 1e3) / 1e9, "peak": 148 * 4 * 1.965 / 6.5, "unit": "Gprobe/s"}
-    if dom == "k_cycle4" and program.info.get("domain", 1 << 30) <= 4096:
+    if dom in ("k_cycle4", "k_cycle4_bitmap") and program.info.get("domain", 1 << 30) <= 4096:
         bound = "alu"      # sorted-list intersections served from L1 / L2 (DRAM 1 % busy under ncu), as for the triangles
         # unit of work: one probe = one walked entry of the shorter list, searched in the other list; both launches (count, write)
         # walk every two-path's list.  ncu at scale 16: 2.26e9 warp instructions for 5.0e8 probes = 4.5 per probe.
@@ -285,8 +285,13 @@ def run_ours(args):
             adj[nm] = m
         two_paths = adj["r"] @ adj["s"]                                            # [x, z]
         walk = np.minimum(adj["t"].sum(axis=1)[None, :], adj["u"].sum(axis=0)[:, None])     # min(out_t(z), in_u(x))
+        per_probe = 4.5
+        if dom == "k_cycle4_bitmap":
+            # the bitmap kernel always walks t's out-list of z; ncu at scale 16: 1.55e9 warp instructions for 5.37e8 probes = 2.9 per probe
+            walk = np.broadcast_to(adj["t"].sum(axis=1)[None, :], two_paths.shape)
+            per_probe = 2.9
         probes = float((two_paths * walk).sum()) * d["launches"]
-        alu = {"achieved": probes / (d["ms"] / 1e3) / 1e9, "peak": 148 * 4 * 1.965 / 4.5, "unit": "Gprobe/s"}
+        alu = {"achieved": probes / (d["ms"] / 1e3) / 1e9, "peak": 148 * 4 * 1.965 / per_probe, "unit": "Gprobe/s"}
     roofline = {"bound": bound, "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src,
                 "traffic": None if ratio is None else ratio * d["bytes"] / d["launches"],

@@ -125,4 +125,108 @@ __global__ void __launch_bounds__(256) k_cycle4(Cycle4 P, const K2* __restrict__
   }
 }
 
+// The same join with u's in-list of x marked in a shared-memory bitmap.  The two-paths are sorted by x, so a block takes a
+// chunk of them and works through its runs of equal x: mark the in-list (w values below kC4BmWords * 32), then a warp per
+// two-path tests the entries of t's out-list of z against the bitmap (one load and a bit test per probe); only a hit, in
+// the writing launch, is looked up in the in-list by binary search for its tag.  Then the marked words are cleared again.
+constexpr uint32_t kC4BmWords = 8192;    // 32 KB of shared memory: w < 2^18
+constexpr uint32_t kC4Chunk = 1024;      // two-paths per block step
+
+template <typename K2, typename K, bool EMIT>
+__global__ void __launch_bounds__(256) k_cycle4_bitmap(Cycle4 P, const K2* __restrict__ keys2, const float* __restrict__ tags2, uint64_t n,
+                                                       uint32_t* __restrict__ cnt, const uint64_t* __restrict__ off,
+                                                       K* __restrict__ out_keys, float* __restrict__ out_tags) {
+  __shared__ uint32_t bm[kC4BmWords];
+  __shared__ unsigned long long run_end_s;
+  const unsigned lane = lane_id(), wid = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
+  for (uint32_t i = threadIdx.x; i < kC4BmWords; i += blockDim.x) bm[i] = 0u;
+  __syncthreads();
+  const uint64_t nchunks = (n + kC4Chunk - 1) / kC4Chunk;
+  for (uint64_t ch = blockIdx.x; ch < nchunks; ch += gridDim.x) {
+    uint64_t cur = ch * kC4Chunk;
+    const uint64_t cend = min(n, cur + (uint64_t)kC4Chunk);
+    while (cur < cend) {
+      const int32_t x = key_col<K2>(P.L2, keys2[cur], 0);
+      if (threadIdx.x == 0) {                              // end of the run of x inside the chunk
+        uint64_t lo = cur + 1, hi = cend;
+        while (lo < hi) { const uint64_t mid = (lo + hi) >> 1; if (key_col<K2>(P.L2, keys2[mid], 0) <= x) lo = mid + 1; else hi = mid; }
+        run_end_s = lo;
+      }
+      uint32_t b0 = 0, b1 = 0;
+      if (x < P.u_domain) { b0 = P.u_off[x]; b1 = P.u_off[x + 1]; }
+      for (uint32_t j = b0 + threadIdx.x; j < b1; j += blockDim.x) { const uint32_t w = (uint32_t)P.u_w[j]; atomicOr(&bm[w >> 5], 1u << (w & 31)); }
+      __syncthreads();
+      const uint64_t rend = run_end_s;
+      if (b1 > b0) {
+        // 32 two-paths at a time: their keys and list bounds are read by one lane each, then the warp takes them in turn,
+        // two sweeps of t's out-list per step
+        for (uint64_t base = cur + (uint64_t)wid * 32; base < rend; base += (uint64_t)nwarp * 32) {
+          const uint64_t i = base + lane;
+          const bool valid = i < rend;
+          uint32_t a0 = 0, a1 = 0;
+          K prefix = 0;
+          float tag = 0.f;
+          uint64_t pos = 0;
+          if (valid) {
+            const K2 k2 = keys2[i];
+            const int32_t y = key_col<K2>(P.L2, k2, 1), z = key_col<K2>(P.L2, k2, 2);
+            if (z < P.t_domain) { a0 = P.t_off[z]; a1 = P.t_off[z + 1]; }
+            if (EMIT) {
+              prefix = ((K)(uint32_t)x << P.L.shift[0]) | ((K)(uint32_t)y << P.L.shift[1]) | ((K)(uint32_t)z << P.L.shift[2]);
+              tag = tags2[i];
+              pos = off[i];
+            }
+          }
+          uint32_t mine = 0;
+          unsigned todo = __ballot_sync(0xffffffffu, valid && a1 > a0);
+          while (todo) {
+            const int src = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const uint32_t A0 = __shfl_sync(0xffffffffu, a0, src), A1 = __shfl_sync(0xffffffffu, a1, src);
+            K pre = 0;
+            float tg = 0.f;
+            uint64_t o = 0;
+            if (EMIT) {
+              pre = (K)__shfl_sync(0xffffffffu, (unsigned long long)prefix, src);
+              tg = __shfl_sync(0xffffffffu, tag, src);
+              o = __shfl_sync(0xffffffffu, (unsigned long long)pos, src);
+            }
+            uint32_t total = 0;
+            for (uint32_t j0 = A0; j0 < A1; j0 += 64) {
+              const uint32_t j[2] = {j0 + lane, j0 + 32 + lane};
+              uint32_t w[2];
+              bool hit[2];
+#pragma unroll
+              for (int u = 0; u < 2; ++u) w[u] = j[u] < A1 ? (uint32_t)P.t_w[j[u]] : 0xffffffffu;
+#pragma unroll
+              for (int u = 0; u < 2; ++u) hit[u] = (w[u] >> 5) < kC4BmWords && ((bm[w[u] >> 5] >> (w[u] & 31)) & 1u);
+              const unsigned m0 = __ballot_sync(0xffffffffu, hit[0]), m1 = __ballot_sync(0xffffffffu, hit[1]);
+              if (EMIT) {
+#pragma unroll
+                for (int u = 0; u < 2; ++u)
+                  if (hit[u]) {
+                    uint32_t lo = b0, hi = b1;             // where w sits in the in-list: its tag
+                    while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if ((uint32_t)P.u_w[mid] < w[u]) lo = mid + 1; else hi = mid; }
+                    const uint64_t at = o + total + (u ? __popc(m0) : 0) + __popc((u ? m1 : m0) & lanemask_lt());
+                    out_keys[at] = pre | ((K)w[u] << P.L.shift[3]);
+                    out_tags[at] = P.times ? (tg * P.t_tag[j[u]]) * P.u_tag[lo] : (tg + P.t_tag[j[u]]) + P.u_tag[lo];
+                  }
+              }
+              total += __popc(m0) + __popc(m1);
+            }
+            if ((int)lane == src) mine = total;
+          }
+          if (!EMIT && valid) cnt[i] = mine;
+        }
+      } else if (!EMIT) {
+        for (uint64_t i = cur + threadIdx.x; i < rend; i += blockDim.x) cnt[i] = 0u;
+      }
+      __syncthreads();
+      for (uint32_t j = b0 + threadIdx.x; j < b1; j += blockDim.x) bm[(uint32_t)P.u_w[j] >> 5] = 0u;
+      __syncthreads();
+      cur = rend;
+    }
+  }
+}
+
 }  // namespace xlog

@@ -1106,9 +1106,20 @@ void cycle4_materialise(Ctx* c, Relation& H, const RuleC& r) {
   zero_ctrl(c, kSlotTotals);
   const unsigned grid = (unsigned)std::min<uint64_t>((n2 + 255) / 256, (uint64_t)kSMs * 8);
   KeyTags kt;
+  // long runs of equal x and small w values: the bitmap kernel (see cycle4.cuh)
+  const uint64_t w_max = (uint64_t)(U.val_max[0] ? U.val_max[0] : U.col_max[0]);
+  const uint64_t x_values = std::min<uint64_t>(R.n, (uint64_t)(R.val_max[0] ? R.val_max[0] : R.col_max[0]) + 1);
+  const bool bitmap = w_max < (uint64_t)kC4BmWords * 32 && n2 >= 16 * x_values;
+  const unsigned bgrid = (unsigned)std::min<uint64_t>((n2 + kC4Chunk - 1) / kC4Chunk, (uint64_t)kSMs * 6);
 #define XLOG_C4(K2, KH, EMIT, KEYS, TAGS)                                                                                          \
-  XLOG_LAUNCH(c, (k_cycle4<K2, KH, EMIT>), grid, 256, 0, P, (const K2*)k0.p, (const float*)t0.as<float>(), n2, cnt.as<uint32_t>(),  \
-              (const uint64_t*)off.as<uint64_t>(), (KH*)(KEYS), (float*)(TAGS))
+  do {                                                                                                                             \
+    if (bitmap)                                                                                                                    \
+      XLOG_LAUNCH(c, (k_cycle4_bitmap<K2, KH, EMIT>), bgrid, 256, 0, P, (const K2*)k0.p, (const float*)t0.as<float>(), n2,         \
+                  cnt.as<uint32_t>(), (const uint64_t*)off.as<uint64_t>(), (KH*)(KEYS), (float*)(TAGS));                           \
+    else                                                                                                                           \
+      XLOG_LAUNCH(c, (k_cycle4<K2, KH, EMIT>), grid, 256, 0, P, (const K2*)k0.p, (const float*)t0.as<float>(), n2,                 \
+                  cnt.as<uint32_t>(), (const uint64_t*)off.as<uint64_t>(), (KH*)(KEYS), (float*)(TAGS));                           \
+  } while (0)
 #define XLOG_C4_DISPATCH(EMIT, KEYS, TAGS)                                        \
   do {                                                                            \
     if (ckb == 4 && H.key_bytes == 4) XLOG_C4(uint32_t, uint32_t, EMIT, KEYS, TAGS); \
