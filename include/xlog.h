@@ -19,7 +19,8 @@
  *   - all device work is issued on the stream given at context creation and every
  *     entry point is stream-synchronous on return;
  *   - a context is not thread-safe; there is no process-wide state
- *     (Section "Crate architecture": no runtime singleton).
+ *     (Section "Crate architecture": no runtime singleton), except the per-device
+ *     scratch array of xlog_reduce_by_key_static (see there).
  *   - keys are int32 and must be >= 0 (dense ids, Section "Reversible symbols").
  */
 #ifndef XLOG_H
@@ -209,8 +210,8 @@ typedef struct {
 /* Evaluate all rules to the least fixpoint, strata in dependency order
  * (Algorithm 1; non-recursive components evaluate each rule once).  On failure
  * the derived relations are poisoned: every later call that needs them returns
- * INVALID_STATE until xlog_ctx_reset_idb ("partial counters do not turn it into
- * a result", Section "Current limitations").  receipt may be NULL. */
+ * INVALID_STATE until xlog_ctx_reset_idb (counters of a failed run are not a
+ * result: Section "Current limitations").  receipt may be NULL. */
 xlog_status xlog_fixpoint(xlog_ctx* ctx, xlog_receipt* receipt);
 
 /* Drop all derived tuples; loaded facts and their join indices stay. */
@@ -263,7 +264,8 @@ xlog_status xlog_profile_reset(xlog_ctx* ctx);
  * Input: n rows with keys ascending (equal keys adjacent, keys >= 0) and their tags, both
  * DEVICE pointers.  Output: one row per distinct key with the oplus of its tags under `sr`
  * (same arithmetic as the engine's group-by), written to out_keys / out_tags (DEVICE, room
- * for n rows; may not overlap the inputs); *n_out (HOST) receives the number of groups.
+ * for n rows; an output that overlaps an input or the other output is rejected with
+ * INVALID_ARGUMENT); *n_out (HOST) receives the number of groups.
  * errbuf (HOST, optional) receives a message on failure.
  *
  * Returns CAPACITY_EXCEEDED, touching nothing, when n > XLOG_STATIC_REDUCE_MAX_ROWS.

@@ -51,8 +51,9 @@ xlog_status scratch_for_current_device(unsigned char** out) {
   return XLOG_OK;
 }
 
+// The first CUDA error of the call, or cudaSuccess (the caller formats it: asking the runtime again would find it cleared).
 template <typename Op>
-xlog_status run(cudaStream_t s, unsigned char* scratch, const uint32_t* keys, const float* tags, uint32_t n, uint32_t* out_keys,
+cudaError_t run(cudaStream_t s, unsigned char* scratch, const uint32_t* keys, const float* tags, uint32_t n, uint32_t* out_keys,
                 float* out_tags, int64_t* n_out) {
   typedef typename Op::A A;
   static_assert(sizeof(A) <= 8, "accumulator must fit the 8-byte scratch slots");
@@ -66,12 +67,19 @@ xlog_status run(cudaStream_t s, unsigned char* scratch, const uint32_t* keys, co
   k_rbk_tiles<uint32_t, Op><<<tiles, kRbkBlock, 0, s>>>(keys, tags, n, heads, tails);
   k_rbk_spine<Op><<<1, 1024, 0, s>>>(heads, tails, carry, tiles, total);
   k_rbk_emit<uint32_t, Op><<<tiles, kRbkBlock, 0, s>>>(keys, tags, n, heads, carry, out_keys, out_tags, (uint32_t*)nullptr);
-  if (cudaGetLastError() != cudaSuccess) return XLOG_ERR_CUDA;
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
   uint32_t u = 0;
-  if (cudaMemcpyAsync(&u, total, sizeof(u), cudaMemcpyDeviceToHost, s) != cudaSuccess) return XLOG_ERR_CUDA;
-  if (cudaStreamSynchronize(s) != cudaSuccess) return XLOG_ERR_CUDA;
+  if ((e = cudaMemcpyAsync(&u, total, sizeof(u), cudaMemcpyDeviceToHost, s)) != cudaSuccess) return e;
+  if ((e = cudaStreamSynchronize(s)) != cudaSuccess) return e;
   *n_out = u;
-  return XLOG_OK;
+  return cudaSuccess;
+}
+
+// [a, a + na) and [b, b + nb) share a byte
+bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+  const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+  return a0 < b0 + nb && b0 < a0 + na;
 }
 
 }  // namespace
@@ -90,6 +98,15 @@ extern "C" xlog_status xlog_reduce_by_key_static(void* stream, xlog_semiring sr,
     return XLOG_ERR_CAPACITY_EXCEEDED;
   }
   if (n == 0) { *n_out = 0; return XLOG_OK; }
+  {
+    // the emit kernel writes group u while other blocks still read rows >= u: an output on top of an input is a race
+    const size_t bytes = (size_t)n * 4;
+    if (overlaps(out_keys, bytes, keys, bytes) || overlaps(out_keys, bytes, tags, bytes) || overlaps(out_tags, bytes, keys, bytes) ||
+        overlaps(out_tags, bytes, tags, bytes) || overlaps(out_keys, bytes, out_tags, bytes)) {
+      if (can_say) snprintf(errbuf, errbuf_len, "xlog_reduce_by_key_static: the outputs may overlap neither the inputs nor each other");
+      return XLOG_ERR_INVALID_ARGUMENT;
+    }
+  }
   unsigned char* scratch = nullptr;
   xlog_status st = scratch_for_current_device(&scratch);
   if (st != XLOG_OK) {
@@ -99,12 +116,14 @@ extern "C" xlog_status xlog_reduce_by_key_static(void* stream, xlog_semiring sr,
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const uint32_t* k = reinterpret_cast<const uint32_t*>(keys);       // keys are >= 0: same order as unsigned
   uint32_t* ok = reinterpret_cast<uint32_t*>(out_keys);
+  cudaError_t e;
   switch (sr) {
-    case XLOG_SR_MAXPLUS: st = run<OpMax>(s, scratch, k, tags, (uint32_t)n, ok, out_tags, n_out); break;
-    case XLOG_SR_MINPLUS: st = run<OpMin>(s, scratch, k, tags, (uint32_t)n, ok, out_tags, n_out); break;
-    case XLOG_SR_LOGSUMEXP: st = run<OpLse>(s, scratch, k, tags, (uint32_t)n, ok, out_tags, n_out); break;
-    default: st = run<OpSum>(s, scratch, k, tags, (uint32_t)n, ok, out_tags, n_out); break;
+    case XLOG_SR_MAXPLUS: e = run<OpMax>(s, scratch, k, tags, (uint32_t)n, ok, out_tags, n_out); break;
+    case XLOG_SR_MINPLUS: e = run<OpMin>(s, scratch, k, tags, (uint32_t)n, ok, out_tags, n_out); break;
+    case XLOG_SR_LOGSUMEXP: e = run<OpLse>(s, scratch, k, tags, (uint32_t)n, ok, out_tags, n_out); break;
+    default: e = run<OpSum>(s, scratch, k, tags, (uint32_t)n, ok, out_tags, n_out); break;
   }
-  if (st != XLOG_OK && can_say) snprintf(errbuf, errbuf_len, "xlog_reduce_by_key_static: CUDA error: %s", cudaGetErrorString(cudaGetLastError()));
-  return st;
+  if (e == cudaSuccess) return XLOG_OK;
+  if (can_say) snprintf(errbuf, errbuf_len, "xlog_reduce_by_key_static: CUDA error: %s", cudaGetErrorString(e));
+  return XLOG_ERR_CUDA;
 }

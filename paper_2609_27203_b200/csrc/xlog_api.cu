@@ -165,6 +165,8 @@ void load_relation(Ctx* c, Relation& R, const int32_t* const* cols, const float*
       XLOG_LAUNCH(c, (k_pack<K>), grid_for(n, 256), 256, 0, in, dtags, n, R.layout, DictSet{}, one_of(R.sr), R.fact_keys.as<K>(), R.fact_tags.as<float>());
       R.n_facts = R.n = (uint32_t)n;
     });
+    // the pack kernel reads the caller's columns: the load has copied them only once it has run
+    XLOG_CUDA(cudaStreamSynchronize(c->stream));
   } else DISPATCH_K(R.key_bytes, {
     DevBuf k0(c, (size_t)n * sizeof(K)), t0(c, (size_t)n * 4), k1(c, (size_t)n * sizeof(K)), t1(c, (size_t)n * 4);
     XLOG_LAUNCH(c, (k_pack<K>), grid_for(n, 256), 256, 0, in, dtags, n, R.layout, DictSet{}, one_of(R.sr), k0.as<K>(), t0.as<float>());

@@ -165,11 +165,13 @@ class Context:
         return out.value
 
     def load(self, rel: int, cols: Sequence, tags=None):
-        """cols/tags: numpy arrays (host) or torch CUDA tensors (device), int32 / float32."""
+        """cols/tags: numpy arrays (host) or torch CUDA tensors (device), int32 / float32, all of one length."""
         torch = self._torch
         k = self._arity[rel]
-        assert len(cols) == k
+        if len(cols) != k:
+            raise ValueError(f"relation of arity {k} loaded with {len(cols)} columns")
         on_device = isinstance(cols[0], torch.Tensor)
+        n = check_load_shapes(cols, tags, self.device if on_device else None)
         keep = []
         ptrs = (C.c_void_p * k)()
         if on_device:
@@ -177,18 +179,19 @@ class Context:
                 c = c.to(torch.int32).contiguous()
                 keep.append(c)
                 ptrs[i] = c.data_ptr()
-            n = int(cols[0].numel())
             tp = None
             if tags is not None:
                 t = tags.to(torch.float32).contiguous()
                 keep.append(t)
                 tp = t.data_ptr()
+            # the conversions above ran on torch's current stream: the library's stream must see their results
+            if keep and torch.cuda.current_stream(self.device).cuda_stream != self._stream.cuda_stream:
+                self._stream.wait_stream(torch.cuda.current_stream(self.device))
         else:
             for i, c in enumerate(cols):
                 c = np.ascontiguousarray(c, np.int32)
                 keep.append(c)
                 ptrs[i] = c.ctypes.data
-            n = len(keep[0])
             tp = None
             if tags is not None:
                 t = np.ascontiguousarray(tags, np.float32)
@@ -313,17 +316,76 @@ class Context:
 STATIC_REDUCE_MAX_ROWS = 1 << 24
 
 
+def check_load_shapes(cols, tags, device) -> int:
+    """Every column and the tags must have one length (and, for device inputs, live on `device`).  Returns that length."""
+    def length(x):
+        return int(x.numel()) if hasattr(x, "numel") else len(x)
+    n = length(cols[0])
+    for i, c in enumerate(cols):
+        if length(c) != n:
+            raise ValueError(f"column {i} has {length(c)} rows, column 0 has {n}")
+        if getattr(c, "ndim", 1) != 1:
+            raise ValueError(f"column {i} is not one-dimensional")
+        if device is not None and (not getattr(c, "is_cuda", False) or c.device.index != device):
+            raise ValueError(f"column {i} does not live on cuda:{device}")
+    if tags is not None:
+        if length(tags) != n:
+            raise ValueError(f"tags have {length(tags)} rows, the columns have {n}")
+        if device is not None and (not getattr(tags, "is_cuda", False) or tags.device.index != device):
+            raise ValueError(f"tags do not live on cuda:{device}")
+    return n
+
+
+def check_static_reduce_args(keys, tags, out_keys, out_tags) -> None:
+    """Everything the C entry point takes on trust: dtypes, contiguity, one device, lengths, room in the outputs and
+    outputs that do not overlap the inputs.  Raises ValueError before anything is launched."""
+    import torch
+    named = {"keys": (keys, torch.int32), "tags": (tags, torch.float32), "out_keys": (out_keys, torch.int32), "out_tags": (out_tags, torch.float32)}
+    for name, (t, dt) in named.items():
+        if not isinstance(t, torch.Tensor):
+            raise ValueError(f"{name} must be a torch tensor")
+        if t.dtype != dt:
+            raise ValueError(f"{name} must be {dt}, not {t.dtype}")
+        if not t.is_cuda:
+            raise ValueError(f"{name} must be a CUDA tensor")
+        if not t.is_contiguous():
+            raise ValueError(f"{name} must be contiguous")
+        if t.device != keys.device:
+            raise ValueError(f"{name} lives on {t.device}, keys on {keys.device}")
+    n = keys.numel()
+    if tags.numel() != n:
+        raise ValueError(f"tags have {tags.numel()} rows, keys have {n}")
+    if out_keys.numel() < n or out_tags.numel() < n:
+        raise ValueError(f"the outputs need room for {n} rows")
+
+    def span(t):
+        return t.data_ptr(), t.data_ptr() + t.numel() * t.element_size()
+    if n:
+        for o in (out_keys, out_tags):
+            for i in (keys, tags):
+                (a0, a1), (b0, b1) = span(o), span(i)
+                if a0 < b1 and b0 < a1:
+                    raise ValueError("an output overlaps an input")
+        (a0, a1), (b0, b1) = span(out_keys), span(out_tags)
+        if a0 < b1 and b0 < a1:
+            raise ValueError("the two outputs overlap")
+
+
 def reduce_by_key_static(semiring: str, keys, tags, out_keys, out_tags, stream=None) -> int:
     """Reduce-by-key for callers that must not allocate device memory during the call (no context,
     no arena: the library's own fixed scratch array is used).  keys (int32, ascending) / tags
-    (float32) and the two output tensors are torch CUDA tensors the caller already owns; returns the
+    (float32) and the two output tensors are torch CUDA tensors the caller already owns, all on one
+    device; the outputs have room for as many rows as the input and overlap nothing.  Returns the
     number of groups written.  At most STATIC_REDUCE_MAX_ROWS rows."""
     import torch
-    s = stream if stream is not None else torch.cuda.current_stream()
+    check_static_reduce_args(keys, tags, out_keys, out_tags)
     n_out = C.c_int64()
     err = C.create_string_buffer(256)
-    st = lib().xlog_reduce_by_key_static(s.cuda_stream, SEMIRING[semiring], keys.data_ptr(), tags.data_ptr(), keys.numel(),
-                                         out_keys.data_ptr(), out_tags.data_ptr(), C.byref(n_out), err, len(err))
+    # the C side resolves its scratch array and the stream on the CURRENT device: make that the tensors' device
+    with torch.cuda.device(keys.device):
+        s = stream if stream is not None else torch.cuda.current_stream(keys.device)
+        st = lib().xlog_reduce_by_key_static(s.cuda_stream, SEMIRING[semiring], keys.data_ptr(), tags.data_ptr(), keys.numel(),
+                                             out_keys.data_ptr(), out_tags.data_ptr(), C.byref(n_out), err, len(err))
     if st:
         raise XlogError(st, err.value.decode())
     return n_out.value

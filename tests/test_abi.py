@@ -47,3 +47,30 @@ def test_binding_refuses_to_run_without_a_gpu():
         pytest.skip("GPU present")
     with pytest.raises(RuntimeError):
         xlog.Context(arena_bytes=1 << 20)
+
+
+def test_binding_rejects_bad_shapes_before_any_launch():
+    # the checks the wrapper makes on its own, so that a short or mistyped buffer never reaches a kernel
+    import numpy as np
+    import pytest
+    import torch
+    from paper_2609_27203_b200 import xlog
+    a, b = np.zeros(5, np.int32), np.zeros(4, np.int32)
+    assert xlog.check_load_shapes([a, a], np.zeros(5, np.float32), None) == 5
+    with pytest.raises(ValueError, match="column 1 has 4 rows"):
+        xlog.check_load_shapes([a, b], None, None)
+    with pytest.raises(ValueError, match="tags have 3 rows"):
+        xlog.check_load_shapes([a, a], np.zeros(3, np.float32), None)
+    with pytest.raises(ValueError, match="one-dimensional"):
+        xlog.check_load_shapes([np.zeros((5, 2), np.int32)], None, None)
+    with pytest.raises(ValueError, match="does not live on cuda:0"):
+        xlog.check_load_shapes([torch.zeros(5, dtype=torch.int32)], None, 0)            # a host tensor passed as a device input
+    k, t = torch.zeros(8, dtype=torch.int32), torch.zeros(8, dtype=torch.float32)
+    with pytest.raises(ValueError, match="must be torch.int32"):
+        xlog.check_static_reduce_args(k.to(torch.int64), t, k, t)
+    with pytest.raises(ValueError, match="must be a torch tensor"):
+        xlog.check_static_reduce_args(np.zeros(8, np.int32), t, k, t)
+    with pytest.raises(ValueError, match="must be a CUDA tensor"):
+        xlog.check_static_reduce_args(k, t, k, t)
+    with pytest.raises(ValueError):
+        xlog.reduce_by_key_static("minplus", k, t, k, t)                                 # the public call makes the same checks first

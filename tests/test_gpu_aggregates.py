@@ -243,6 +243,39 @@ def test_sum_semiring_two_step_walk_counts_and_facts_of_a_derived_relation():
     ctx.close()
 
 
+@pytest.mark.parametrize("n,m", [(9, 30), (300, 6000)])
+def test_sumprod_backward_matches_the_oracle(n, m):
+    # p2(x,z) :- e(x,y), e(y,z) under (+, *):  d loss / d tag = g[h] * (the other atom's tag), summed over the bindings
+    import torch
+    s, d = synth.uniform_digraph(n, m, 51)
+    w = (0.5 + synth.uniform01(51, 3, 0, m)).astype(np.float32)
+    prog = W.Program("p2", {"e": (2, W.SUMPROD), "p2": (2, W.SUMPROD)},
+                     [W.Rule("p2", (W.V(0), W.V(2)), (W.Atom("e", (W.Var(0), W.Var(1))), W.Atom("e", (W.Var(1), W.Var(2)))))],
+                     {"e": ([s, d], w)}, ("p2",))
+    ctx, gids, grules, o, oids, orules, _ = both(prog)
+    rep = H.compare_relations(ctx.read(gids["p2"]), o.read(oids["p2"]), rel_tol=1e-5, abs_tol=1e-6, what="p2 tags")
+    g = synth.head_gradient(rep["rows"], 52)
+    og = o.backward(orules[0], g)
+    parts = ctx.backward(grules[0], torch.from_numpy(g).cuda(), same_buffer_for_same_relation=False)
+    for j in range(2):
+        ref = og[j].astype(np.float64)
+        assert np.all(np.abs(parts[j].cpu().numpy() - ref) <= 1e-5 + 1e-4 * np.abs(ref)), f"atom {j}"
+    both_atoms = ctx.backward(grules[0], torch.from_numpy(g).cuda())[0].cpu().numpy()
+    ref = og[0].astype(np.float64) + og[1].astype(np.float64)
+    assert np.all(np.abs(both_atoms - ref) <= 2e-5 + 1e-4 * np.abs(ref))
+    ctx.close()
+    # one-atom rule: deg(x) :- e(x,y); every row of e receives the upstream gradient of its group
+    prog = W.Program("deg", {"e": (2, W.SUMPROD), "deg": (1, W.SUMPROD)}, [W.Rule("deg", (W.V(0),), (W.Atom("e", (W.Var(0), W.Var(1))),))],
+                     {"e": ([s, d], w)}, ("deg",))
+    ctx, gids, grules, o, oids, orules, _ = both(prog)
+    xs = ctx.read(gids["deg"])[0][0]
+    g = synth.head_gradient(len(xs), 53)
+    got = ctx.backward(grules[0], torch.from_numpy(g).cuda())[0].cpu().numpy()
+    assert np.array_equal(got, o.backward(orules[0], g)[0])
+    assert np.array_equal(got, g[np.searchsorted(xs, np.sort(s))])
+    ctx.close()
+
+
 def test_backward_requires_a_forward_and_a_supported_head():
     import torch
     from paper_2609_27203_b200 import xlog

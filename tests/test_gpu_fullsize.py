@@ -2,8 +2,9 @@
 (device-resident inputs, the arena sizes of bench.make_program).
 
 Where the oracle finishes in well under a minute the whole relation is compared; otherwise
-sampled outputs the oracle can compute one by one are compared (one source of the multi-source
-program, a sample of x for the triangle aggregate) together with properties that hold at any size.
+sampled outputs the oracle can compute one by one are compared (four sources of the multi-source
+program, a sample of x for the triangle aggregate) together with properties that hold at any size
+and with numpy / scipy restatements that share nothing with either side.
 Tolerances as in test_gpu_parity.py / test_gpu_aggregates.py.
 """
 import numpy as np
@@ -79,41 +80,109 @@ def test_config4_digits_full_forward_and_backward():
     ctx.close()
 
 
+def _triangle_terms_of(x, off, d, w, n):
+    """Every term (w_xy + w_yz) + w_zx of x's triangles in float64, straight from the edge arrays (numpy only)."""
+    in_w = np.full(n, np.nan)
+    zs_in = np.flatnonzero(d == x)                       # edges (z, x): rows whose destination is x
+    src_of = np.searchsorted(off, zs_in, side="right") - 1
+    in_w[src_of] = w[zs_in]
+    terms = []
+    ys = d[off[x]:off[x + 1]]
+    wxy = w[off[x]:off[x + 1]].astype(np.float64)
+    step = 256
+    for a in range(0, len(ys), step):
+        yb = ys[a:a + step]
+        lens = (off[yb + 1] - off[yb]).astype(np.int64)
+        if lens.sum() == 0:
+            continue
+        idx = np.repeat(off[yb].astype(np.int64) - np.concatenate([[0], np.cumsum(lens)[:-1]]), lens) + np.arange(lens.sum())
+        z = d[idx]
+        hit = ~np.isnan(in_w[z])
+        t = (np.repeat(wxy[a:a + step], lens)[hit] + w[idx][hit].astype(np.float64)) + in_w[z[hit]]
+        terms.append(t)
+    return np.concatenate(terms) if terms else np.zeros(0)
+
+
 def test_config3_triangles_rmat18_full_sampled():
+    import scipy.sparse as sp
     prog = W.config3()
+    n = 1 << 18
     ctx, ids, _, receipt = gpu_fixpoint(prog, 2 << 30)
     cols, tags = ctx.read(ids["tri_agg"])
+    ctx.close()
     xs, counts = cols[0], cols[1].astype(np.int64)
     assert counts.sum() % 3 == 0 and np.all(counts > 0) and np.all(np.diff(xs) > 0)
-    # sampled x, each computed by the oracle alone with x fixed as a constant
-    (s, d), w = prog.facts["e"]
-    deg = np.bincount(s, minlength=1 << 18)
+    got = {int(x): (int(c), float(t)) for x, c, t in zip(xs, counts, tags)}
+    (s, d), w = prog.facts["e"]                          # sorted by (s, d)
+    deg = np.bincount(s, minlength=n)
+    off = np.concatenate([[0], np.cumsum(deg)])
+
+    # (1) the group with the most terms, against a float64 sum over its terms written out with numpy
+    big = int(xs[np.argmax(counts)])
+    terms = _triangle_terms_of(big, off, d, w, n)
+    assert len(terms) == got[big][0] > 1_000_000, f"count of the largest group x={big}"
+    m = terms.max()
+    assert abs(got[big][1] - (m + np.log(np.exp(terms - m).sum()))) < 1e-4, f"logsumexp of the largest group x={big}"
+
+    # (2) counts of every x with x % 64 == 0 (4,096 nodes, the hub among them) against a sparse matrix product:
+    #     count(x) = sum over y, z of A[x,y] A[y,z] A[z,x]; x without a triangle must be absent
+    A = sp.csr_matrix((np.ones(len(s), np.int64), (s, d)), shape=(n, n))
+    S = np.arange(0, n, 64)
+    ref = np.asarray((A[S] @ A).multiply(A[:, S].T.tocsr()).sum(axis=1)).ravel()
+    mine = np.zeros(n, np.int64)
+    mine[xs] = counts
+    assert np.array_equal(mine[S], ref)
+    assert int(ref.sum()) > 10_000_000
+
+    # (3) sampled x computed by the oracle alone with x fixed as a constant: twelve of moderate degree, and four from the
+    #     top decile by count (those whose two-paths number at most 3 M, so that the oracle's nested loops finish in seconds),
+    #     and the largest group once more, this time by the oracle
     cand = xs[(deg[xs] >= 2) & (deg[xs] <= 300)]
-    pick = cand[synth.randint(3, 7, 0, 12, len(cand))]
+    pick = cand[synth.randint(3, 7, 0, 12, len(cand))].tolist()
+    two_paths = np.asarray((A[xs] @ sp.csr_matrix(deg.reshape(-1, 1))).todense()).ravel()
+    top = xs[(counts >= np.quantile(counts, 0.9)) & (two_paths <= 3_000_000)]
+    assert len(top) >= 4
+    pick += top[synth.randint(3, 8, 0, 4, len(top))].tolist() + [big]
     o = oracle.Oracle()
     e = o.relation(2, W.LOGSUMEXP)
     o.load(e, [s, d], w)
     heads = []
-    for x in pick.tolist():
+    for x in pick:
         h = o.relation(2, W.LOGSUMEXP)
         o.rule(h, [(x, {})], [(e, [("c", x), ("v", 1, 1, 0)]), (e, [("v", 1, 1, 0), ("v", 2, 1, 0)]), (e, [("v", 2, 1, 0), ("c", x)])], True)
         heads.append(h)
     o.run("naive")
-    got = {int(x): (int(c), float(t)) for x, c, t in zip(xs, counts, tags)}
-    for x, h in zip(pick.tolist(), heads):
+    for x, h in zip(pick, heads):
         oc, ot = o.read(h)
         assert len(ot) == 1 and int(oc[0][0]) == x
         assert got[x][0] == int(oc[1][0]), f"count of x={x}"
         assert abs(got[x][1] - float(ot[0])) < 1e-4, f"logsumexp of x={x}"
-    # x without any triangle must be absent: check a sample against a direct numpy intersection count
-    ctx.close()
 
 
-def test_config5_reach_rmat22_full_one_source_by_oracle():
+def _oracle_reach_rows(edges, sources):
+    """reach(s, .) of the given sources by the oracle alone (its own instance: callers run several in threads)."""
+    (s, d), w = edges
+    o, oids, _ = oracle.load_program(W.reach_program(s, d, w, np.asarray(sources, np.int32)))
+    o.run("seminaive")
+    return o.read(oids["reach"])
+
+
+def test_config5_reach_rmat22_full_four_sources_by_oracle():
+    from concurrent.futures import ThreadPoolExecutor
     prog = W.config5()
-    ctx, ids, _, receipt = gpu_fixpoint(prog, 56 << 30)
     (s, d), w = prog.facts["edge"]
     srcs = prog.facts["src"][0][0]
+    deg = np.bincount(s, minlength=1 << 22)
+    live = srcs[deg[srcs] > 0]
+    # four live sources, the one with the most out-edges among them; two oracle instances run side by side (the C++ engine
+    # runs outside the interpreter lock), two sources each
+    by_deg = live[np.argsort(-deg[live], kind="stable")]
+    chosen = [int(by_deg[0]), int(live[0]) if int(live[0]) != int(by_deg[0]) else int(live[1])]
+    chosen += [int(x) for x in live[::-1] if int(x) not in chosen][:2]
+    pool = ThreadPoolExecutor(2)
+    jobs = [pool.submit(_oracle_reach_rows, prog.facts["edge"], chosen[0:2]), pool.submit(_oracle_reach_rows, prog.facts["edge"], chosen[2:4])]
+
+    ctx, ids, _, receipt = gpu_fixpoint(prog, 56 << 30)
     rc, rt = ctx.read(ids["reach"])
     assert receipt["derived_tuples"] == len(rt) and np.array_equal(np.unique(rc[0]), np.sort(srcs))
     # every source reaches itself at distance 0; keys ascending (s, z)
@@ -121,17 +190,15 @@ def test_config5_reach_rmat22_full_one_source_by_oracle():
     assert np.all(np.diff(key) > 0)
     self_rows = rc[0] == rc[1]
     assert self_rows.sum() == len(srcs) and np.all(rt[self_rows] == 0.0)
-    # one non-trivial source, end to end by the oracle's single-source program on the same graph
-    deg = np.bincount(s, minlength=1 << 22)
-    src0 = int(srcs[deg[srcs] > 0][0])
-    o, oids, _ = oracle.load_program(W.sssp_program(s, d, w, src0))
-    o.run("seminaive")
-    oc, ot = o.read(oids["dist"])
-    sel = rc[0] == src0
-    assert np.array_equal(rc[1][sel], oc[0])
-    assert np.array_equal(rt[sel].view(np.int32), ot.view(np.int32))
     # sources without out-edges reach only themselves
     for dead in srcs[deg[srcs] == 0][:5].tolist():
         assert int((rc[0] == dead).sum()) == 1
     ctx.close()
     same_on_the_sorting_path(prog, 56 << 30, "reach", rc, rt, receipt)
+    for job in jobs:
+        oc, ot = job.result()
+        sel = np.isin(rc[0], np.unique(oc[0]))
+        assert np.array_equal(rc[0][sel], oc[0]) and np.array_equal(rc[1][sel], oc[1])
+        assert np.array_equal(rt[sel].view(np.int32), ot.view(np.int32))
+        assert len(ot) > 2_000_000
+    pool.shutdown()
