@@ -1,13 +1,15 @@
 #!/usr/bin/env python
 """Benchmark: derived tuples per second to fixpoint on one B200 (per GPU: independent replicas).
 
-A step is one whole fixpoint (all rounds of join / project / sort / reduce / diff-merge) over a
-seeded synthetic workload whose facts are already loaded and indexed on the device.  The default
-workload is the single-source min-plus shortest-path program on an R-MAT scale-20 graph.
+A step is one whole fixpoint (all rounds of join / project / aggregate / dedup / merge) over a seeded synthetic
+workload whose facts are already loaded and indexed on the device.  The headline line is the largest single-GPU
+configuration, multi-source reachability on an R-MAT scale-22 graph with 64 sources (`reach_rmat22_s64`); the same
+run also measures the other four configurations and reports them under `configs`.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload sssp|closure|reach|triangles|digits]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload reach|sssp|closure|triangles|digits|...]
   python bench.py --impl reference ...      # times the CPU oracle on the host cores instead
 
+`--gpus N` without a torchrun environment starts N replica processes (one per device) itself.
 Prints ONE JSON line (rank 0).
 """
 from __future__ import annotations
@@ -15,6 +17,8 @@ from __future__ import annotations
 import argparse
 import json
 import os
+import re
+import socket
 import statistics
 import subprocess
 import sys
@@ -29,17 +33,23 @@ import numpy as np  # noqa: E402
 
 METRIC = "derived tuples/sec to fixpoint"
 UNIT = "tuples/s"
+HEADLINE = "reach"
+ALL_FIVE = ["closure", "sssp", "triangles", "digits", "reach"]           # configurations 1-5
 
-# DRAM bytes per algorithmic byte of each kernel, from the ncu captures summarised under profiles/
-# (dram__bytes_read.sum + dram__bytes_write.sum over the launch's algorithmic bytes).  Used only to
-# scale a captured launch to the bench's launch size; None = not captured.
-NCU_TRAFFIC_RATIO = {"k_sort_pass": 0.99, "k_join_expand": 0.92, "k_dense_reduce": 1.04, "k_merge": 1.0}
-# the join kernels when they apply candidates to the tag mirror instead of writing them: the slot reads hit L2, so DRAM
-# sees the adjacency reads (8 of the 12 algorithmic bytes per candidate) plus row records
-NCU_TRAFFIC_RATIO_MIRROR = {"k_join_expand": 0.80, "k_res_expand": 0.80,
-                            # grouped join (rows of one probed value share the neighbour reads and sit in one table line): 5.1 B of DRAM
-                            # traffic per candidate at 32 sources against 5.3 algorithmic (4 for the slot, 8 / rows-per-node for the neighbour)
-                            "k_seg_expand": 0.95}
+
+def traffic_ratios():
+    """DRAM bytes per algorithmic byte of each kernel, as measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum
+    over the launch's algorithmic bytes) and kept in the table of profiles/ncu_traffic_ratios.md together with the
+    commands that made them.  Used only to scale a captured launch to the bench's launch size.  {(kernel, route): ratio}"""
+    out = {}
+    path = os.path.join(ROOT, "profiles", "ncu_traffic_ratios.md")
+    if not os.path.exists(path):
+        return out
+    for line in open(path):
+        m = re.match(r"\|\s*(k_\w+)\s*\|\s*(\w+)\s*\|\s*([0-9.]+)\s*\|", line)
+        if m:
+            out[(m.group(1), m.group(2))] = float(m.group(3))
+    return out
 
 
 def make_program(name: str, scale: int | None, sources: int | None = None):
@@ -194,64 +204,11 @@ def run_oracle_once(program, mode="seminaive"):
 
 
 # ------------------------------------------------------------------------------------------------
-def run_ours(args):
-    import torch
-    import torch.distributed as dist
-    from paper_2609_27203_b200 import xlog
+MIRROR_JOIN_KERNELS = ("k_res_expand", "k_seg_expand", "k_bm_expand")
 
-    rank, local_rank, world = dist_env()
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
-    torch.cuda.set_device(local_rank)
-    dev = f"cuda:{local_rank}"
-    program, arena = make_program(args.workload, args.scale, args.sources)
 
-    # facts resident in HBM before any timed region
-    base_flags = (xlog.FLAG_NO_TAG_MIRROR if args.no_tag_mirror else 0) | (xlog.FLAG_NO_GRAPH if args.no_graph else 0) | (xlog.FLAG_NO_RESIDENT_LOOP if args.no_resident_loop else 0)
-    base_flags |= {"auto": 0, "wcoj": xlog.FLAG_FORCE_WCOJ, "chain": xlog.FLAG_FORCE_CHAIN}[args.triangle_plan]
-    ctx, ids, rules = xlog.load_program(program, device=local_rank, arena_bytes=arena, device_inputs=True, flags=base_flags)
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)          # > 126 MB L2
-
-    def step(c):
-        c.reset_idb()
-        flush.fill_(1)                                                       # evict L2 between iterations
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        r = c.fixpoint()
-        e1.record()
-        e1.synchronize()
-        return e0.elapsed_time(e1), r
-
-    for _ in range(args.warmup):
-        step(ctx)
-    if world > 1:
-        dist.barrier()
-    torch.cuda.synchronize()
-    times, launches, receipt = [], 0, None
-    with ClockSampler(local_rank) as clk:
-        for _ in range(args.steps):
-            ms, receipt = step(ctx)
-            times.append(ms)
-            launches += receipt["kernel_launches"]
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    total_ms = reduce_max([sum(times)], world, dev)[0]
-    ms_per_step = total_ms / args.steps
-    derived = receipt["derived_tuples"]
-    value = derived * world / (ms_per_step / 1e3)
-
-    # per-kernel timing: the same steps again with CUDA events around every launch
-    ctx.close()
-    pctx, pids, _ = xlog.load_program(program, device=local_rank, arena_bytes=arena, device_inputs=True,
-                                      flags=xlog.FLAG_PROFILE | base_flags)
-    step(pctx)
-    pctx.profile_reset()
-    for _ in range(args.steps):
-        step(pctx)
-    prof_all = pctx.profile()
-    pctx.close()
-    # "<kernel> (large)" entries repeat, for launches of at least 4 M candidates, what the kernel's own entry already holds
+def roofline_of(program, prof_all, steps, sorting_route):
+    """The roofline object of the kernel that takes most of the device time, from the per-kernel CUDA-event table."""
     prof_large = {k[:-len(" (large)")]: v for k, v in prof_all.items() if k.endswith(" (large)")}
     prof = {k: v for k, v in prof_all.items() if not k.endswith(" (large)")}
     ktot = sum(v["ms"] for v in prof.values()) or 1.0
@@ -259,10 +216,8 @@ def run_ours(args):
     d = prof[dom]
     peak, peak_src = measured_peak_gbs()
     achieved = d["bytes"] / (d["ms"] / 1e3) / 1e9 if d["ms"] > 0 else 0.0
-    ratio = NCU_TRAFFIC_RATIO.get(dom)
-    mirror_kernel = dom in ("k_res_expand", "k_seg_expand") or (dom == "k_join_expand" and not args.no_tag_mirror and "k_sort_pass" not in prof)
-    if mirror_kernel:
-        ratio = NCU_TRAFFIC_RATIO_MIRROR.get(dom)
+    mirror_kernel = dom in MIRROR_JOIN_KERNELS or (dom == "k_join_expand" and not sorting_route and "k_sort_pass" not in prof)
+    ratio = traffic_ratios().get((dom, "mirror" if mirror_kernel else "sorting"))
     bound = "hbm"
     alu = None
     if dom.startswith("k_tri"):
@@ -295,9 +250,9 @@ def run_ours(args):
     roofline = {"bound": bound, "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src,
                 "traffic": None if ratio is None else ratio * d["bytes"] / d["launches"],
-                "algorithmic_bytes_per_launch": d["bytes"] / d["launches"], "launches_per_step": d["launches"] / args.steps,
+                "algorithmic_bytes_per_launch": d["bytes"] / d["launches"], "launches_per_step": d["launches"] / steps,
                 "avg_launch_us": 1e3 * d["ms"] / d["launches"], "share_of_kernel_time": d["ms"] / ktot,
-                "kernels": {k: {"launches_per_step": v["launches"] / args.steps, "ms_per_step": v["ms"] / args.steps,
+                "kernels": {k: {"launches_per_step": v["launches"] / steps, "ms_per_step": v["ms"] / steps,
                                 "GBps": (v["bytes"] / (v["ms"] / 1e3) / 1e9) if v["ms"] > 0 and v["bytes"] else None}
                             for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])},
                 "how": "second pass of the same steps with XLOG_FLAG_PROFILE (CUDA events around every launch on the ctx stream; "
@@ -306,72 +261,164 @@ def run_ours(args):
     if big and big["ms"] > 0:
         # the same kernel over its launches of at least 4 M candidates only (small rounds are launch- and latency-bound)
         g = big["bytes"] / (big["ms"] / 1e3) / 1e9
-        roofline["large_launches"] = {"launches_per_step": big["launches"] / args.steps, "ms_per_step": big["ms"] / args.steps,
+        roofline["large_launches"] = {"launches_per_step": big["launches"] / steps, "ms_per_step": big["ms"] / steps,
                                       "achieved": g, "frac": g / peak, "what": "this kernel's launches of at least 48 MB algorithmic bytes (4 M candidates x 12 B) only"}
     if alu:
         roofline.update(achieved=alu["achieved"], peak=alu["peak"], unit=alu["unit"], frac=alu["achieved"] / alu["peak"], traffic=None,
                         peak_source="derived: issue slots x clock / measured warp instructions per probe")
     if mirror_kernel:
-        # one random 32-byte L2 sector per candidate (the key's slot in the tag mirror) on top of the streamed adjacency
-        # reads: the kernel is bound by how many such sector requests the SMs keep in flight, not by HBM
-        roofline["limiter"] = ("instruction issue (79 % of the issue slots busy under ncu at 32 sources); the table, too large for L2, is read from HBM one line per (node, neighbour)"
-                               if dom == "k_seg_expand" else
+        # the tag-mirror joins move few bytes per candidate by construction; what limits them is said here
+        roofline["limiter"] = ("instruction issue; the table, too large for L2, is read from HBM one 128-byte line per (changed unit of 32 keys, neighbour)"
+                               if dom in ("k_seg_expand", "k_bm_expand") else
                                "L2 random sector access (one tag-mirror slot per candidate); HBM carries about 8 B per candidate")
-        if dom != "k_seg_expand":
+        if dom not in ("k_seg_expand", "k_bm_expand"):
             roofline["candidates_per_s"] = achieved * 1e9 / 12.0
+    return roofline
+
+
+def measure(name, args, steps, warmup, local_rank, world, flush, with_e2e):
+    """Timed fixpoints of one workload on this rank's device: (summary dict, program).  Facts are resident and indexed
+    before the timed region; L2 is flushed between steps."""
+    import torch
+    import torch.distributed as dist
+    from paper_2609_27203_b200 import xlog
+    dev = f"cuda:{local_rank}"
+    headline = name == args.workload
+    program, arena = make_program(name, args.scale if headline else None, args.sources if headline else None)
+    base_flags = (xlog.FLAG_NO_TAG_MIRROR if args.no_tag_mirror else 0) | (xlog.FLAG_NO_GRAPH if args.no_graph else 0) | (xlog.FLAG_NO_RESIDENT_LOOP if args.no_resident_loop else 0)
+    base_flags |= (xlog.FLAG_NO_BITMAP_JOIN if args.no_bitmap_join else 0)
+    base_flags |= {"auto": 0, "wcoj": xlog.FLAG_FORCE_WCOJ, "chain": xlog.FLAG_FORCE_CHAIN}[args.triangle_plan]
+    ctx, ids, rules = xlog.load_program(program, device=local_rank, arena_bytes=arena, device_inputs=True, flags=base_flags)
+
+    def step(c):
+        c.reset_idb()
+        flush.fill_(1)                                                       # evict L2 between iterations
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        r = c.fixpoint()
+        e1.record()
+        e1.synchronize()
+        return e0.elapsed_time(e1), r
+
+    for _ in range(warmup):
+        step(ctx)
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    times, launches, receipt = [], 0, None
+    with ClockSampler(local_rank) as clk:
+        for _ in range(steps):
+            ms, receipt = step(ctx)
+            times.append(ms)
+            launches += receipt["kernel_launches"]
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    total_ms = reduce_max([sum(times)], world, dev)[0]
+    ms_per_step = total_ms / steps
+    derived = receipt["derived_tuples"]
+    out = {"program": program, "ms_per_step": ms_per_step, "value": derived * world / (ms_per_step / 1e3), "times": times,
+           "launches": launches, "receipt": receipt, "clocks": clk.summary(), "derived": derived}
+
+    # per-kernel timing: the same steps again with CUDA events around every launch
+    ctx.close()
+    pctx, pids, _ = xlog.load_program(program, device=local_rank, arena_bytes=arena, device_inputs=True,
+                                      flags=xlog.FLAG_PROFILE | base_flags)
+    step(pctx)
+    pctx.profile_reset()
+    for _ in range(steps):
+        step(pctx)
+    prof_all = pctx.profile()
+    pctx.close()
+    out["roofline"] = roofline_of(program, prof_all, steps, args.no_tag_mirror)
+    if not with_e2e:
+        return out
 
     # end to end through the C ABI with HOST buffers: load (H2D + sort + index), fixpoint, read back (D2H)
     pinned = {}
     h2d = 0
-    for name, (cols, tags) in program.facts.items():
+    for rname, (cols, tags) in program.facts.items():
         pc = [torch.from_numpy(np.ascontiguousarray(c, np.int32)).pin_memory() for c in cols]
         pt = None if tags is None else torch.from_numpy(np.ascontiguousarray(tags, np.float32)).pin_memory()
-        pinned[name] = (pc, pt)
+        pinned[rname] = (pc, pt)
         h2d += sum(c.numel() * 4 for c in pc) + (0 if pt is None else pt.numel() * 4)
     empty = type(program)(program.name, program.relations, program.rules, {}, program.outputs)
     ectx, eids, _ = xlog.load_program(empty, device=local_rank, arena_bytes=arena, flags=base_flags)
 
     def e2e_step():
         t0 = time.perf_counter()
-        for name, (pc, pt) in pinned.items():
-            ectx.load(eids[name], [c.numpy() for c in pc], None if pt is None else pt.numpy())
+        for rname, (pc, pt) in pinned.items():
+            ectx.load(eids[rname], [c.numpy() for c in pc], None if pt is None else pt.numpy())
         r = ectx.fixpoint()
         d2h = 0
-        for name in program.outputs:
-            cols, tags = ectx.read(eids[name])
+        for rname in program.outputs:
+            cols, tags = ectx.read(eids[rname])
             d2h += (len(cols) + 1) * 4 * len(tags)
         torch.cuda.synchronize()
         return (time.perf_counter() - t0) * 1e3, r, d2h
 
-    for _ in range(min(args.warmup, 2)):
+    for _ in range(min(warmup, 2)):
         e2e_step()
     if world > 1:
         dist.barrier()
     e_times, d2h = [], 0
-    for _ in range(max(1, min(args.steps, 5))):
+    for _ in range(max(1, min(steps, 5))):
         ms, r, d2h = e2e_step()
         e_times.append(ms)
     e_ms = reduce_max([sum(e_times) / len(e_times)], world, dev)[0]
     ectx.close()
-    e2e = {"value": derived * world / (e_ms / 1e3), "unit": UNIT, "ms_per_step": e_ms, "h2d_bytes_per_step": h2d,
-           "d2h_bytes_per_step": d2h, "how": "xlog_relation_load from pinned host + xlog_fixpoint + xlog_relation_read to host, wall clock"}
+    out["e2e"] = {"value": derived * world / (e_ms / 1e3), "unit": UNIT, "ms_per_step": e_ms, "h2d_bytes_per_step": h2d,
+                  "d2h_bytes_per_step": d2h, "how": "xlog_relation_load from pinned host + xlog_fixpoint + xlog_relation_read to host, wall clock"}
+    return out
 
-    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-           "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32 keys / f32 tags",
-           "data": "synthetic", "impl": "ours",
-           "config": {"workload": program.name, "program": args.workload, **{k: v for k, v in program.info.items()},
-                      "derived_tuples": derived, "rounds": receipt["iterations"], "candidates": receipt["candidates"],
-                      "triangle_plan": {0: None, 1: "wcoj", 2: "chain"}[receipt["triangle_plan"]],
-                      "unique_candidates": receipt["unique_candidates"], "l2": "flushed between steps (256 MB fill)",
-                      "parallelism": "replicas only" if world > 1 else "1 gpu", "facts": "resident and indexed before timing"},
-           "clocks": clk.summary(), "e2e": e2e, "gpu_launches": launches, "roofline": roofline,
-           "step_ms_min_med_max": [min(times), statistics.median(times), max(times)]}
+
+def config_of(args_workload, m, world):
+    program, receipt = m["program"], m["receipt"]
+    return {"workload": program.name, "program": args_workload, **{k: v for k, v in program.info.items()},
+            "derived_tuples": m["derived"], "rounds": receipt["iterations"], "candidates": receipt["candidates"],
+            "triangle_plan": {0: None, 1: "wcoj", 2: "chain"}[receipt["triangle_plan"]],
+            "unique_candidates": receipt["unique_candidates"], "l2": "flushed between steps (256 MB fill)",
+            "parallelism": "replicas only" if world > 1 else "1 gpu", "facts": "resident and indexed before timing"}
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local_rank}"))
+    torch.cuda.set_device(local_rank)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=f"cuda:{local_rank}")          # > 126 MB L2
+
+    m = measure(args.workload, args, args.steps, args.warmup, local_rank, world, flush, with_e2e=True)
+    out = {"metric": METRIC, "value": m["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+           "ms_per_step": m["ms_per_step"], "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int32 keys / f32 tags",
+           "data": "synthetic", "impl": "ours", "config": config_of(args.workload, m, world),
+           "clocks": m["clocks"], "e2e": m["e2e"], "gpu_launches": m["launches"], "roofline": m["roofline"],
+           "step_ms_min_med_max": [min(m["times"]), statistics.median(m["times"]), max(m["times"])]}
+
+    # the other configurations, each at its full size: a short run of the same protocol (no end-to-end leg)
+    if args.workload == HEADLINE and args.scale is None and args.sources is None and not args.no_other_configs:
+        others = {}
+        for name in ALL_FIVE:
+            if name == args.workload:
+                continue
+            o = measure(name, args, min(args.steps, 5), 3, local_rank, world, flush, with_e2e=False)
+            r = o["roofline"]
+            others[o["program"].name] = {"program": name, "ms_per_fixpoint": o["ms_per_step"], "tuples_per_s": o["value"],
+                                         "derived_tuples": o["derived"], "rounds": o["receipt"]["iterations"], "candidates": o["receipt"]["candidates"],
+                                         "launches_per_fixpoint": o["launches"] / min(args.steps, 5),
+                                         "dominant_kernel": r["kernel"], "bound": r["bound"], "achieved": r["achieved"], "unit": r["unit"],
+                                         "frac": r["frac"], "large_launches_frac": (r.get("large_launches") or {}).get("frac"),
+                                         "clocks": o["clocks"]}
+        out["configs"] = others
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         # the oracle as it stands, on this box's host cores, on a bounded sample of the same workload
-        # bounded sample (about 10-30 s of CPU work): the full workload where the oracle manages it, else a smaller R-MAT scale
+        # (about 10-30 s of CPU work): the full workload where the oracle manages it, else a smaller R-MAT scale
         cpu_scale = args.cpu_scale or {"triangles": 14, "reach": 16, "wcoj": 13, "cycle4": 15}.get(args.workload)
-        sample, _ = make_program(args.workload, cpu_scale) if cpu_scale else (program, 0)
+        sample, _ = make_program(args.workload, cpu_scale) if cpu_scale else (m["program"], 0)
         sec, stats, _o = run_oracle_once(sample)
         out["cpu_baseline"] = {"value": stats["derived_tuples"] / sec, "unit": UNIT, "cores": 1, "kind": "oracle",
                                "seconds": sec, "host_cores_available": os.cpu_count(),
@@ -384,23 +431,31 @@ def run_ours(args):
 
 
 # ------------------------------------------------------------------------------------------------
+FULL_SCALE = {"sssp": 20, "reach": 22, "triangles": 18, "wcoj": 16, "cycle4": 16}
+# seconds of one oracle fixpoint at the full size (host-core measurements of earlier runs; only used to size the sample)
+ORACLE_SECONDS_FULL = {"sssp": 12.0, "reach": 3400.0, "closure": 3.0, "triangles": 3200.0, "digits": 3.0, "wcoj": 60.0, "cycle4": 60.0}
+REFERENCE_BUDGET_S = 420.0
+
+
 def run_reference(args):
-    """The oracle on the host cores, same metric; each step is one fixpoint of a bounded sample."""
+    """The oracle on the host cores, same metric and workload name as the GPU arm.  Each step is one fixpoint of the
+    workload itself where (steps + warmup) of them fit the time budget, else of a smaller R-MAT scale of the same program
+    (the line then says so in `sample_of` / `config.sample`)."""
     rank, _, world = dist_env()
     if rank != 0:
         return
-    est20 = {"sssp": 16.0, "reach": 600.0, "closure": 3.0, "triangles": 200.0, "digits": 10.0, "wcoj": 60.0, "cycle4": 60.0}[args.workload]
+    n_runs = args.steps + args.warmup
     scale = args.scale
-    if args.workload in ("sssp", "reach", "triangles", "wcoj", "cycle4") and scale is None:
-        full = {"sssp": 20, "reach": 22, "triangles": 18, "wcoj": 16, "cycle4": 16}[args.workload]
-        scale = full
-        while scale > 8 and (args.steps + args.warmup) * est20 * 2.0 ** (scale - full) > 150.0:
+    full_name = make_name(args.workload, args.scale, args.sources)
+    if args.workload in FULL_SCALE and scale is None:
+        scale = FULL_SCALE[args.workload]
+        while scale > 8 and n_runs * ORACLE_SECONDS_FULL[args.workload] * 2.0 ** (scale - FULL_SCALE[args.workload]) > REFERENCE_BUDGET_S:
             scale -= 1
-    program, _ = make_program(args.workload, scale)
+    program, _ = make_program(args.workload, scale, args.sources)
     import oracle
     o, ids, _ = oracle.load_program(program)
     times, stats = [], None
-    for i in range(args.warmup + args.steps):
+    for i in range(n_runs):
         o.reset()
         t0 = time.perf_counter()
         stats = o.run("seminaive")
@@ -410,13 +465,42 @@ def run_reference(args):
     ms = sum(times) / len(times)
     value = stats["derived_tuples"] / (ms / 1e3)
     sample = f"{program.name}: semi-naive fixpoint of the std::map oracle, single thread, facts pre-loaded"
-    print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-                      "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-                      "dtype": "int32 keys / f32 tags", "data": "synthetic", "impl": "reference",
-                      "config": {"workload": program.name, "program": args.workload, **program.info,
-                                 "derived_tuples": stats["derived_tuples"]},
-                      "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
-                      "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int32 keys / f32 tags", "data": "synthetic", "impl": "reference",
+            "config": {"workload": full_name, "program": args.workload, "sample": program.name, **program.info,
+                       "derived_tuples": stats["derived_tuples"]},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    if program.name != full_name:
+        line["sample_of"] = (f"{full_name}: one oracle fixpoint at full size takes about {ORACLE_SECONDS_FULL[args.workload]:.0f} s on one host core, "
+                             f"so {n_runs} of them do not fit {REFERENCE_BUDGET_S:.0f} s; each step is the same program on {program.name}")
+    print(json.dumps(line))
+
+
+def make_name(workload, scale, sources):
+    """Name of the workload make_program would build, without generating it."""
+    if workload == "sssp":
+        return f"sssp_rmat{scale or 20}"
+    if workload == "reach":
+        return f"reach_rmat{scale or 22}_s{sources or 64}"
+    if workload == "triangles":
+        return f"triangles_rmat{scale or 18}"
+    if workload == "closure":
+        return "closure_n1000_m4000"
+    if workload == "digits":
+        return "digits_B65536"
+    return make_program(workload, scale, sources)[0].name
+
+
+def spawn_replicas(n):
+    """`--gpus N` outside a torchrun environment: start N ranks of this script (one per device) on this node."""
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
 
 
 def main():
@@ -425,17 +509,21 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="sssp", choices=["sssp", "closure", "reach", "triangles", "digits", "wcoj", "cycle4"])
+    ap.add_argument("--workload", default=HEADLINE, choices=["sssp", "closure", "reach", "triangles", "digits", "wcoj", "cycle4"])
     ap.add_argument("--scale", type=int, default=None, help="R-MAT scale override (smaller cases for profiling)")
     ap.add_argument("--sources", type=int, default=None, help="reach: number of sources (fewer for a small profiling case)")
     ap.add_argument("--triangle-plan", default="auto", choices=["auto", "wcoj", "chain"], help="wcoj workload: force a join plan")
     ap.add_argument("--no-resident-loop", action="store_true", help="tag-mirror rounds driven by the host (one control read per round)")
     ap.add_argument("--no-graph", action="store_true", help="launch the resident rounds one by one (for per-launch profiling)")
     ap.add_argument("--no-tag-mirror", action="store_true", help="evaluate recursion by sort -> reduce-by-key -> merge only")
+    ap.add_argument("--no-bitmap-join", action="store_true", help="grouped join from a delta row list instead of the changed bitmap")
+    ap.add_argument("--no-other-configs", action="store_true", help="headline workload only (skip the `configs` object)")
     ap.add_argument("--cpu-scale", type=int, default=None, help="R-MAT scale of the cpu_baseline sample (default: the workload's)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 0)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(spawn_replicas(args.gpus))
     if args.impl == "reference":
         run_reference(args)
     else:

@@ -80,6 +80,7 @@ typedef struct {
 #define XLOG_FLAG_FORCE_WCOJ      32u  /* materialised triangle joins: always the multiway (worst-case-optimal) plan */
 #define XLOG_FLAG_FORCE_CHAIN     64u  /* ... always the binary-join chain (fails with RESOURCE_EXHAUSTED if its intermediate does not fit) */
 #define XLOG_FLAG_NO_GROUPED_JOIN 128u  /* tag mirror: always the row-wise join, never the grouped one (see csrc/group_join.cuh) */
+#define XLOG_FLAG_NO_BITMAP_JOIN  256u  /* tag mirror, grouped join: always from a delta row list, never straight from the changed bitmap (see csrc/bitmap_join.cuh) */
 #define XLOG_FLAG_NO_GRAPH        16u  /* resident rounds are launched one by one instead of as one graph with a WHILE node */
 
 /* Evaluation routes of a recursive component (Algorithm 1).  All of them derive the same relation,
@@ -90,7 +91,10 @@ typedef struct {
  *    direct-addressed table of one tag per possible key; candidates are applied with one atomic max/min.
  *    Above 2^24 possible keys a rule of the shape h(a, c) :- h(a, b), r(b, c) is joined "grouped": the mirror is
  *    indexed with the probed column as the major part, the delta comes out grouped by b, and the delta rows of one b
- *    share the read of r's run of b and a line of the table (XLOG_FLAG_NO_GROUPED_JOIN switches this off).
+ *    share the read of r's run of b and a line of the table (XLOG_FLAG_NO_GROUPED_JOIN switches this off).  With at
+ *    least 32 possible values of a and one such rule, the rounds are driven by the changed bitmap itself: one kernel
+ *    turns the bitmap into work items (no delta row list is written), one joins (XLOG_FLAG_NO_BITMAP_JOIN switches
+ *    this off); it takes a second table of the mirror's size for the tags as they stood at the start of the round.
  *  - Resident rounds (tag mirror with <= 2^24 possible keys): the delta rounds run as one CUDA graph with a
  *    conditional WHILE node and fixed-capacity buffers (Section "GPU-Native Symbolic Substrate": resident
  *    conditional graph, no host reads inside the loop).  The buffers (about 36 bytes per possible key

@@ -1,5 +1,6 @@
 // C ABI of the engine (see include/xlog.h) and the host-side fixpoint driver.
 #include "engine.cuh"
+#include "bitmap_join.cuh"
 #include "group_join.cuh"
 #include "mirror.cuh"
 #include "resident.cuh"
@@ -1541,6 +1542,48 @@ uint64_t grouped_apply(Ctx* c, const Variant& v, const Relation& H, const KeyLay
   return total;
 }
 
+constexpr int kSlotBm = 84;                // bitmap-driven grouped join: the kBmTotals counters of k_bm_plan
+static_assert(kSlotBm + kBmTotals <= kCtrlSlots, "control block too small");
+
+// What the bitmap-driven grouped join (bitmap_join.cuh) needs beyond the mirror itself; valid == false: not applicable.
+struct BitmapJoin {
+  bool valid = false;
+  JoinSpec spec;
+  DevBuf snap, items;
+  int carried_bits = 0;
+};
+
+// Applicable when exactly one rule has an atom over h (so a round is one join), that rule has the grouped shape with the
+// linear-key form, a unit of 32 carried values fits one value of the probed column, and the snapshot table and the item
+// list (sized for every unit changing in one round) fit the arena.
+void bitmap_join_setup(Ctx* c, int h, const std::vector<const RuleC*>& rs, const KeyLayout& M, int carried_bits, uint64_t slots, BitmapJoin& bj) {
+  if ((c->flags & XLOG_FLAG_NO_BITMAP_JOIN) || carried_bits < 5) return;
+  Relation& H = *c->rels[h];
+  if (H.dict_n[1]) return;
+  const RuleC* rule = nullptr; int pos = -1, n_over = 0;
+  for (const RuleC* r : rs)
+    for (int j = 0; j < r->plan.n_atoms; ++j)
+      if (r->plan.atoms[j].rel == h) { ++n_over; rule = r; pos = j; }
+  if (n_over != 1) return;
+  const Variant v{rule, pos, Source{nullptr, nullptr, 0, M, H.key_bytes}};
+  const JoinSpec S = make_spec(c, v, H, &M);               // builds the looked-up relation's index if it is missing
+  if (!S.fast || !S.has_inner || S.inner_free != 1 || S.outer_decode[0] || S.outer_decode[1] || S.head_encode[0] || S.head_encode[1] ||
+      S.inner_mult[0] != ((uint64_t)1 << carried_bits))
+    return;
+  const Relation& RB = *c->rels[rule->plan.atoms[1 - pos].rel];
+  const uint64_t units_per_value = (uint64_t)1 << (carried_bits - 5);
+  const uint64_t values = std::min<uint64_t>((uint64_t)S.inner_domain, slots >> carried_bits);
+  const uint64_t max_items = ((uint64_t)RB.n / kBmSlice + values + 1) * units_per_value;
+  if (max_items >= ((uint64_t)1 << 32)) return;
+  const uint64_t need = slots * 4 + max_items * 16 + (1u << 20);
+  if (need > c->arena.largest_free() / 2) return;
+  bj.snap = DevBuf(c, slots * 4);
+  bj.items = DevBuf(c, max_items * 16);
+  bj.spec = S;
+  bj.carried_bits = carried_bits;
+  bj.valid = true;
+}
+
 // Algorithm 1 over a tag mirror (mirror.cuh): per round  count -> scan -> join straight into the table -> compact the
 // changed bitmap into the next delta.  No candidate is ever written to memory.  The seed round is driven by the host
 // (its rules scan whole relations of known size); the delta rounds run resident where the fixed-capacity buffers fit.
@@ -1570,6 +1613,8 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
     table_own = DevBuf(c, slots * 4); bitmap_own = DevBuf(c, (size_t)bm_quads * 16); present_own = DevBuf(c, (size_t)bm_quads * 16);
     ch_sums_own = DevBuf(c, (size_t)ch_tiles * 4);
   }
+  BitmapJoin bj;
+  if (grouped) bitmap_join_setup(c, h, rs, M, carried_bits, slots, bj);
   uint32_t* present = R ? R->present.as<uint32_t>() : present_own.as<uint32_t>();
   int32_t* table = R ? R->table.as<int32_t>() : table_own.as<int32_t>();
   uint4* bitmap = R ? R->bitmap.as<uint4>() : bitmap_own.as<uint4>();
@@ -1666,6 +1711,38 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
     }
     const uint64_t total = host_apply(vs);
     if (total == 0 && !(round == 0 && plain_rules_done)) break;
+    if (bj.valid) {
+      // Every later round is  k_bm_plan -> one control read -> k_bm_expand : the plan kernel closes the round just joined
+      // (changed / new keys, bitmap cleared, snapshot of the changed units' tags) and lays out the next one's work items.
+      const uint32_t nwords = bm_quads * 4;
+      BmPlan P{reinterpret_cast<uint32_t*>(bitmap), present, nwords, table, bj.snap.as<int32_t>(), carried_bits - 5, bj.spec.inner_off,
+               (uint32_t)std::min<int64_t>(bj.spec.inner_domain, 0xffffffffll), bj.items.as<uint4>(), (unsigned long long*)(c->d_ctrl + kSlotBm)};
+      BmExpand E{bj.items.as<uint4>(), 0, bj.spec.inner_col[0], bj.spec.inner_tag, H.layout.mask[1], carried_bits, bj.snap.as<int32_t>(), table,
+                 reinterpret_cast<uint32_t*>(bitmap), ctrl_u32(c, kSlotErr)};
+      for (;;) {
+        zero_ctrl(c, kSlotBm, kBmTotals);
+        c->note_bytes = (int64_t)nwords * 4;
+        XLOG_LAUNCH(c, k_bm_plan, (nwords + kBmPlanTile - 1) / kBmPlanTile, kBmPlanBlock, 0, P);
+        sync_ctrl(c);
+        const uint64_t changed = c->h_ctrl[kSlotBm + kBmChanged], n_new = c->h_ctrl[kSlotBm + kBmNew], cand = c->h_ctrl[kSlotBm + kBmCandidates];
+        const uint64_t n_items = c->h_ctrl[kSlotBm + kBmItems], nbrs = c->h_ctrl[kSlotBm + kBmNeighbours];
+        total_new += n_new;
+        c->r_new += (int64_t)n_new; c->r_improved += (int64_t)changed - (int64_t)n_new;
+        if (changed == 0) break;
+        ++round;
+        if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
+        ++c->r_iterations;
+        if (cand == 0) break;
+        c->r_candidates += (int64_t)cand;
+        E.n_items = (uint32_t)n_items;
+        // per candidate its slot; per (unit, neighbour) the looked-up column and tag; per item its record and the unit's 32 snapshot tags
+        c->note_bytes = (int64_t)cand * 4 + (int64_t)nbrs * 8 + (int64_t)n_items * 144;
+        const unsigned grid = (unsigned)std::min<uint64_t>((n_items + 7) / 8, (uint64_t)kSMs * 8 * 16);
+        if (is_max) XLOG_LAUNCH(c, (k_bm_expand<kSinkMax>), grid, 256, 0, E);
+        else XLOG_LAUNCH(c, (k_bm_expand<kSinkMin>), grid, 256, 0, E);
+      }
+      break;
+    }
     launch_changed_count(c, reinterpret_cast<const uint32_t*>(bitmap), present, bm_quads * 4, ch_tiles, ch_sums, mr.n_new);
     XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, ch_sums, (int64_t)ch_tiles, ctrl_u32(c, kSlotMirChanged));
     sync_ctrl(c);
@@ -1705,7 +1782,7 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
     if (grouped && n_out > 1) {
       // rows came out in the mirror's order, (column 1, column 0) ascending: a stable sort on column 0's bits alone puts
       // them in the relation's key order
-      table_own.reset(); bitmap_own.reset(); present_own.reset();
+      table_own.reset(); bitmap_own.reset(); present_own.reset(); bj.snap.reset(); bj.items.reset();
       DevBuf ak(c, (size_t)n_out * 4), at(c, (size_t)n_out * 4);
       uint32_t* pk = full.keys.as<uint32_t>(); uint32_t* qk = ak.as<uint32_t>();
       float* pt = full.tags.as<float>(); float* qt = at.as<float>();

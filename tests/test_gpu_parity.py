@@ -39,10 +39,10 @@ def check_program(program, rel_tol=MINMAX_REL, abs_tol=0.0, expect_bit_equal=Tru
     o, oids, _, stats = oracle_run(program, mode)
     receipts, results = [], []
     # default (tag mirror, delta rounds resident in one graph) / the same rounds launched one by one / host-driven
-    # mirror rounds (with the grouped join where the rule has that shape) / the same with the row-wise join only / the
-    # sorting path
-    for extra in (0, xlog.FLAG_NO_GRAPH, xlog.FLAG_NO_RESIDENT_LOOP, xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_GROUPED_JOIN,
-                  xlog.FLAG_NO_TAG_MIRROR):
+    # mirror rounds (with the grouped join where the rule has that shape, driven by the changed bitmap where a unit of 32
+    # carried values exists) / the grouped join from a delta row list / the row-wise join only / the sorting path
+    for extra in (0, xlog.FLAG_NO_GRAPH, xlog.FLAG_NO_RESIDENT_LOOP, xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_BITMAP_JOIN,
+                  xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_GROUPED_JOIN, xlog.FLAG_NO_TAG_MIRROR):
         ctx, gids, _, receipt = gpu_run(program, **dict(kw, flags=kw.get("flags", xlog.FLAG_CHECK_INVARIANTS) | extra))
         got = {}
         for name in program.outputs:
@@ -274,7 +274,8 @@ def test_routes_agree_at_sizes_beyond_the_oracle():
     w = (1 + 9 * synth.uniform01(71, 3, 0, len(s))).astype(np.float32)
     for prog in (W.closure_program(s, t, w, W.MINPLUS, name="hubs"), W.config5(scale=16, n_sources=300)):
         base = None
-        for flags in (xlog.FLAG_NO_TAG_MIRROR, 0, xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_GROUPED_JOIN, xlog.FLAG_NO_RESIDENT_LOOP):
+        for flags in (xlog.FLAG_NO_TAG_MIRROR, 0, xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_GROUPED_JOIN, xlog.FLAG_NO_RESIDENT_LOOP,
+                      xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_BITMAP_JOIN):
             ctx, ids, _ = xlog.load_program(prog, arena_bytes=6 << 30, flags=flags)
             r = ctx.fixpoint()
             out = ctx.read(ids[prog.outputs[0]])
