@@ -43,7 +43,7 @@ typedef enum {
   XLOG_OK = 0,
   XLOG_ERR_INVALID_ARGUMENT = 1,
   XLOG_ERR_INVALID_VALUE = 2,        /* NaN tag, tag equal to the semiring zero, negative key */
-  XLOG_ERR_UNSUPPORTED = 3,          /* plan shape; non-idempotent oplus inside a recursive component */
+  XLOG_ERR_UNSUPPORTED = 3,          /* plan shape; a non-linear rule under logsumexp / sum inside a recursive component */
   XLOG_ERR_RESOURCE_EXHAUSTED = 4,   /* arena bytes */
   XLOG_ERR_CAPACITY_EXCEEDED = 5,    /* key bits > 64, count > INT32_MAX, head value outside [0, 2^31) */
   XLOG_ERR_CONVERGENCE_FAILURE = 6,  /* iteration cap reached */
@@ -92,9 +92,9 @@ typedef struct {
  *    Above 2^24 possible keys a rule of the shape h(a, c) :- h(a, b), r(b, c) is joined "grouped": the mirror is
  *    indexed with the probed column as the major part, the delta comes out grouped by b, and the delta rows of one b
  *    share the read of r's run of b and a line of the table (XLOG_FLAG_NO_GROUPED_JOIN switches this off).  With at
- *    least 32 possible values of a and one such rule, the rounds are driven by the changed bitmap itself: one kernel
- *    turns the bitmap into work items (no delta row list is written), one joins (XLOG_FLAG_NO_BITMAP_JOIN switches
- *    this off); it takes a second table of the mirror's size for the tags as they stood at the start of the round.
+ *    least 32 (and at most 1024) possible values of a and one such rule, the rounds are driven by the changed bitmap itself:
+ *    one kernel turns the bitmap into work items and a list of the changed keys' (tag, a) pairs grouped by b, one joins
+ *    (XLOG_FLAG_NO_BITMAP_JOIN switches this off); the pair list holds 8 bytes per possible key.
  *  - Resident rounds (tag mirror with <= 2^24 possible keys): the delta rounds run as one CUDA graph with a
  *    conditional WHILE node and fixed-capacity buffers (Section "GPU-Native Symbolic Substrate": resident
  *    conditional graph, no host reads inside the loop).  The buffers (about 36 bytes per possible key
@@ -156,9 +156,13 @@ xlog_status xlog_relation_view(xlog_ctx* ctx, xlog_rel rel, const int32_t** cols
  * xlog_receipt.triangle_plan reports the choice.  Both plans produce identical rows.
  * The four-cycle join  h(x,y,z,w) :- r(x,y), s(y,z), t(z,w), u(w,x)  (same sections: coverage
  * spans the triangle and 4-cycles) over up to four binary relations, head columns exactly
- * (x,y,z,w): the two-paths of r and s, then per two-path the intersection of t's out-list of
- * z with u's in-list of x, count -> scan -> write; rows come out sorted.  It must be the only
- * rule of its head, outside recursion; RESOURCE_EXHAUSTED if the two-paths do not fit the arena.
+ * (x,y,z,w): the two-paths of r and s, then either the multiway step (per two-path the
+ * intersection of t's out-list of z with u's in-list of x, count -> scan -> write) or the rest of
+ * the binary-join chain (every three-path of r, s, t written out, then a probe of u).  The same
+ * skew test chooses, on the exact three-path count; the same flags override it and
+ * xlog_receipt.triangle_plan reports the choice; both plans produce identical rows, sorted.  It
+ * must be the only rule of its head, outside recursion; RESOURCE_EXHAUSTED if the two-paths do
+ * not fit the arena.
  * Negation (Sections "Aggregations and constraints", "Completeness over finite domains":
  * explicit stratified negation-as-failure): a rule of one positive atom followed by one
  * negated atom,  h(..) :- a(..), not b(..).  The negated atom holds iff no row of b matches;
@@ -169,7 +173,15 @@ xlog_status xlog_relation_view(xlog_ctx* ctx, xlog_rel rel, const int32_t** cols
  * connected components of the relation dependency graph; a rule may have one or two
  * recursive atoms (p(x,z) :- p(x,y), p(y,z) is evaluated with one delta variant per
  * occurrence, Section "Semi-naive evaluation on GPU"), and a component may hold
- * several mutually recursive relations. */
+ * several mutually recursive relations.
+ * Tags inside recursion: a component of MAXPLUS / MINPLUS relations runs Algorithm 1 with tag
+ * improvement (a tuple re-enters the delta when its tag strictly improves).  A component of
+ * LOGSUMEXP or SUMPROD relations (Section "Aggregations and constraints" rejects aggregation
+ * inside a recursive component; this is the extension to acyclic derivations) must have at most
+ * one recursive atom per rule; the tag of a tuple is then the oplus over ALL its derivations
+ * (path counts, sums of path products), evaluated with deltas that carry tag differences, and
+ * recomputed from the loaded facts on every xlog_fixpoint.  If the derivations are cyclic the
+ * rounds never end: CONVERGENCE_FAILURE at max_iterations.  Mixed components: UNSUPPORTED. */
 typedef enum { XLOG_ARG_CONST = 0, XLOG_ARG_VAR = 1 } xlog_arg_kind;
 typedef struct { int32_t kind; int32_t var; int32_t mul; int32_t add; /* CONST: add is the value */ } xlog_arg;
 typedef struct { xlog_rel rel; xlog_arg args[XLOG_MAX_ARITY]; int32_t negated; /* 1: negation as failure, see below */ } xlog_atom;
@@ -204,8 +216,10 @@ typedef struct {
   int64_t  kernel_launches;
   int64_t  peak_arena_bytes;
   double   device_ms;              /* CUDA-event time of the whole call on the ctx stream */
-  int32_t  triangle_plan;          /* XLOG_PLAN_*: how the last materialised triangle join of this call was evaluated (a four-cycle join reports WCOJ) */
-  int32_t  reserved;
+  int32_t  triangle_plan;          /* XLOG_PLAN_*: how the last materialised triangle or four-cycle join of this call was evaluated */
+  int32_t  index_builds;           /* join indices (offsets over a column, permuted sorted copies) built during this call: indices
+                                      of relations that did not change since an earlier call are reused, not rebuilt
+                                      (Sections "Runtime optimization", "Index reuse and the chain scorer") */
 } xlog_receipt;
 #define XLOG_PLAN_NONE  0
 #define XLOG_PLAN_WCOJ  1          /* multiway join: per row of the first atom, intersect two sorted lists */
@@ -254,6 +268,19 @@ typedef struct {
 } xlog_kernel_stat;
 xlog_status xlog_profile_read(xlog_ctx* ctx, xlog_kernel_stat* out, int32_t capacity, int32_t* n_out);
 xlog_status xlog_profile_reset(xlog_ctx* ctx);
+
+/* ---- failure-path hooks (tests only) -----------------------------------------------------
+ * Two kernels wait for other thread blocks of their own launch: the sort pass and the resident count + scan look back
+ * through per-tile status words.  A tile only waits for tiles that already run, and every wait gives up after a number
+ * of polls, raises the device error flag, writes nothing more and lets the call fail with XLOG_ERR_INTERNAL (typed,
+ * fail-closed outcomes: Section "GPU residency model").  The default limit (2^22 polls) is never reached in a healthy run.
+ * xlog_debug_set_poll_limit lowers it for this context; xlog_debug_sort_pass_without_first_tile runs one 8-bit sort pass
+ * (keys / payload -> out_keys / out_payload, all DEVICE, n rows, at least two tiles of 4096) in which the first tile is
+ * deliberately not launched, so that every other tile's wait runs out: the call returns XLOG_ERR_INTERNAL, the outputs
+ * stay as they were, and the context remains usable. */
+xlog_status xlog_debug_set_poll_limit(xlog_ctx* ctx, uint32_t polls);
+xlog_status xlog_debug_sort_pass_without_first_tile(xlog_ctx* ctx, const void* keys, const void* payload, void* out_keys, void* out_payload,
+                                                    int64_t n, int32_t key_bytes);
 
 /* ---- reduce-by-key that allocates nothing --------------------------------------------
  * (The paper has no counterpart for this entry point.)

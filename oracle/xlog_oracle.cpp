@@ -233,9 +233,18 @@ struct Engine {
       for (const Rule* r : rs) for (const Atom& a : r->atoms) if (in.count(a.rel)) { recursive = true; if (a.neg) return status = ST_UNSUPPORTED; }
       if (!recursive) stratum_once(comp[0], rs);
       else {
-        for (int p : comp) if (rels[p].sr != SR_MAXPLUS && rels[p].sr != SR_MINPLUS) return status = ST_UNSUPPORTED;
+        int idem = 0, additive = 0;
+        for (int p : comp) { if (rels[p].sr == SR_MAXPLUS || rels[p].sr == SR_MINPLUS) ++idem; else ++additive; }
+        if (idem && additive) return status = ST_UNSUPPORTED;
         for (const Rule* r : rs) if (r->emit_count) return status = ST_UNSUPPORTED;
-        if (mode == 0) recursive_naive(in, rs, max_iter); else recursive_seminaive(in, rs, max_iter);
+        if (additive) {
+          if (mode == 0) additive_naive(in, rs, max_iter);
+          else {
+            // the delta form below needs T to be linear in the component's relations: at most one recursive atom per rule
+            for (const Rule* r : rs) { int k = 0; for (const Atom& a : r->atoms) if (in.count(a.rel)) ++k; if (k > 1) return status = ST_UNSUPPORTED; }
+            additive_seminaive(in, rs, max_iter);
+          }
+        } else if (mode == 0) recursive_naive(in, rs, max_iter); else recursive_seminaive(in, rs, max_iter);
       }
       if (status != ST_OK) return status;
     }
@@ -305,6 +314,77 @@ struct Engine {
           auto it = P.rows.find(e.first);
           if (it == P.rows.end()) { P.rows.emplace(e.first, e.second.best); nd[p].emplace(e.first, e.second.best); }
           else if (better(P.sr, e.second.best, it->second)) { it->second = e.second.best; nd[p].emplace(e.first, e.second.best); }
+        }
+        n += (int64_t)nd[p].size();
+      }
+      delta.swap(nd); delta_total += n; delta_trace.push_back(n);
+      return n;
+    };
+    {
+      std::map<int, AccTable> acc;
+      for (const Rule* r : rs) { auto s = full_sources(*r); contribute(*r, s.data(), acc[r->head]); if (status) return; }
+      ++iterations;
+      if (absorb(acc) == 0) return;
+    }
+    for (int64_t round = 1;; ++round) {
+      if (round >= max_iter) { status = ST_CONVERGENCE; return; }
+      std::map<int, AccTable> acc;
+      for (const Rule* r : rs)
+        for (size_t i = 0; i < r->atoms.size(); ++i) {
+          if (!in.count(r->atoms[i].rel) || r->atoms[i].neg) continue;
+          auto s = full_sources(*r);
+          s[i] = &delta[r->atoms[i].rel];
+          contribute(*r, s.data(), acc[r->head]);
+          if (status) return;
+        }
+      ++iterations;
+      if (absorb(acc) == 0) return;
+    }
+  }
+
+  // Non-idempotent oplus inside a recursive component, naive form:  I_0 = facts,  I_{k+1} = facts oplus T(I_k).
+  void additive_naive(const std::set<int>& in, const std::vector<const Rule*>& rs, int64_t max_iter) {
+    for (int p : in) rels[p].rows = rels[p].facts;
+    for (int64_t round = 0;; ++round) {
+      if (round >= max_iter) { status = ST_CONVERGENCE; return; }
+      std::map<int, AccTable> acc;
+      for (const Rule* r : rs) { auto s = full_sources(*r); contribute(*r, s.data(), acc[r->head]); if (status) return; }
+      bool changed = false;
+      for (int p : in) {
+        Rel& P = rels[p];
+        for (const auto& f : P.facts) acc[p][f.first].terms.push_back((double)f.second);
+        Table next;
+        for (const auto& e : acc[p]) next.emplace_hint(next.end(), e.first, finish(P.sr, e.second));
+        if (next.size() != P.rows.size()) changed = true;
+        else for (auto a = next.begin(), b = P.rows.begin(); a != next.end(); ++a, ++b)
+          if (a->first != b->first || std::memcmp(&a->second, &b->second, sizeof(float)) != 0) { changed = true; break; }
+        P.rows.swap(next);
+      }
+      ++iterations;
+      if (!changed) return;
+    }
+  }
+
+  // The same fixpoint in delta form (Algorithm 1 with the delta carrying tag DIFFERENCES).  T is linear in the
+  // component's relations (one recursive atom per rule), so  I_{k+1} - I_k = T_rec(I_k - I_{k-1}):
+  //   Delta_1 = T(facts)  (every atom reads the full relation),  Delta_{k+1} = T_rec(Delta_k),  I_{k+1} = I_k oplus Delta_{k+1},
+  // until a round derives nothing at all.  Each round's sums are taken in fp64 and rounded once; the running relation is fp32.
+  void additive_seminaive(const std::set<int>& in, const std::vector<const Rule*>& rs, int64_t max_iter) {
+    for (int p : in) rels[p].rows = rels[p].facts;
+    std::map<int, Table> delta;
+    auto absorb = [&](std::map<int, AccTable>& acc) {
+      std::map<int, Table> nd; int64_t n = 0;
+      for (int p : in) {
+        Rel& P = rels[p];
+        for (const auto& e : acc[p]) {
+          const float d = finish(P.sr, e.second);
+          nd[p].emplace_hint(nd[p].end(), e.first, d);
+          auto it = P.rows.find(e.first);
+          if (it == P.rows.end()) P.rows.emplace(e.first, d);
+          else {
+            Acc two; two.terms.push_back((double)it->second); two.terms.push_back((double)d);
+            it->second = finish(P.sr, two);
+          }
         }
         n += (int64_t)nd[p].size();
       }

@@ -229,4 +229,54 @@ __global__ void __launch_bounds__(256) k_cycle4_bitmap(Cycle4 P, const K2* __res
   }
 }
 
+// ---- the binary-join chain of the four-cycle ---------------------------------------------------------------------------
+// The plan a binary-join engine takes: every three-path (x,y,z,w) of r, s and t is written out (two-paths joined with t on
+// z), and u is then probed with (w, x) (k_chain_probe_* in triangle.cuh).  Chosen by the skew test when the three-paths
+// stay within a small multiple of the inputs; the multiway plan above never writes a three-path that u does not close.
+template <typename K2>
+__global__ void __launch_bounds__(256) k_c4_chain_count(Cycle4 P, const K2* __restrict__ keys2, uint64_t n, uint32_t* __restrict__ cnt) {
+  for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+    const int32_t z = key_col<K2>(P.L2, keys2[i], 2);
+    cnt[i] = z < P.t_domain ? P.t_off[z + 1] - P.t_off[z] : 0u;
+  }
+}
+
+// A warp takes 32 two-paths; each one's run of t is written by the whole warp (coalesced however long the run).
+template <typename K2, typename K>
+__global__ void __launch_bounds__(256) k_c4_chain_expand(Cycle4 P, const K2* __restrict__ keys2, const float* __restrict__ tags2, uint64_t n,
+                                                         const uint64_t* __restrict__ off, K* __restrict__ out_keys, float* __restrict__ out_tags) {
+  const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+  const unsigned lane = lane_id();
+  for (uint64_t base = warp * 32; base < n; base += nwarps * 32) {
+    const uint64_t i = base + lane;
+    uint32_t a0 = 0, a1 = 0;
+    K prefix = 0;
+    float tag = 0.f;
+    uint64_t pos = 0;
+    if (i < n) {
+      const K2 k2 = keys2[i];
+      const int32_t x = key_col<K2>(P.L2, k2, 0), y = key_col<K2>(P.L2, k2, 1), z = key_col<K2>(P.L2, k2, 2);
+      if (z < P.t_domain) { a0 = P.t_off[z]; a1 = P.t_off[z + 1]; }
+      prefix = ((K)(uint32_t)x << P.L.shift[0]) | ((K)(uint32_t)y << P.L.shift[1]) | ((K)(uint32_t)z << P.L.shift[2]);
+      tag = tags2[i];
+      pos = off[i];
+    }
+    unsigned todo = __ballot_sync(0xffffffffu, a1 > a0);
+    while (todo) {
+      const int src = __ffs(todo) - 1;
+      todo &= todo - 1;
+      const uint32_t A0 = __shfl_sync(0xffffffffu, a0, src), A1 = __shfl_sync(0xffffffffu, a1, src);
+      const K pre = (K)__shfl_sync(0xffffffffu, (unsigned long long)prefix, src);
+      const float tg = __shfl_sync(0xffffffffu, tag, src);
+      const uint64_t o = __shfl_sync(0xffffffffu, (unsigned long long)pos, src);
+      for (uint32_t j = lane; j < A1 - A0; j += 32) {
+        out_keys[o + j] = pre | ((K)(uint32_t)P.t_w[A0 + j] << P.L.shift[3]);
+        const float wt = P.t_tag[A0 + j];
+        out_tags[o + j] = P.times ? tg * wt : tg + wt;
+      }
+    }
+  }
+}
+
 }  // namespace xlog

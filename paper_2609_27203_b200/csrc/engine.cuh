@@ -158,7 +158,7 @@ struct Ctx {
   int64_t launches = 0, d2h_bytes = 0, h2d_bytes = 0;
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   // receipt counters of the running fixpoint
-  int64_t r_candidates = 0, r_unique = 0, r_new = 0, r_improved = 0, r_iterations = 0, r_strata = 0;
+  int64_t r_candidates = 0, r_unique = 0, r_new = 0, r_improved = 0, r_iterations = 0, r_strata = 0, r_index_builds = 0;
   // optional per-kernel timing (XLOG_FLAG_PROFILE): CUDA events around every launch
   struct ProfEntry { std::string name; int64_t launches = 0; double ms = 0; int64_t bytes = 0; };
   struct ProfPending { int entry; cudaEvent_t a, b; int big_entry; };      // big_entry >= 0: also counted under "<name> (large)"
@@ -169,6 +169,7 @@ struct Ctx {
   int64_t note_bytes = 0;                 // algorithmic bytes of the next launch (consumed by the launch macro)
   std::map<int, std::unique_ptr<Resident>> resident;   // by head relation
   int last_triangle_plan = 0;             // XLOG_PLAN_* of the last materialised triangle join
+  uint32_t spin_limit = kSpinLimit;      // polls of one status word before a look-back wait gives up (sort passes, resident scan)
   bool unique_untracked = false;          // a stratum went through the tag mirror, which does not count distinct candidate keys
   std::vector<char> stratum_done;         // per relation: its stratum has been evaluated in the running fixpoint
 };
@@ -326,7 +327,7 @@ inline void sort_pairs(Ctx* c, K*& keys, float*& tags, K*& keys_alt, float*& tag
 #define XLOG_SORT_PASS(B)                                                                                                          \
   XLOG_LAUNCH(c, (k_sort_pass<K, B>), ntiles, kSortBlock, sort_pass_smem<K>(), keys, reinterpret_cast<const uint32_t*>(tags), keys_alt, \
               reinterpret_cast<uint32_t*>(tags_alt), (uint32_t)n, P.shift[pass], hist + pass * kSortMaxBins, status, tickets + pass,  \
-              ctrl_u32(c, kSlotErr))
+              ctrl_u32(c, kSlotErr), c->spin_limit)
     switch (P.bits[pass]) {
       case 1: XLOG_SORT_PASS(1); break;
       case 2: XLOG_SORT_PASS(2); break;

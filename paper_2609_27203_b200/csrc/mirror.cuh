@@ -151,4 +151,80 @@ __global__ void __launch_bounds__(kMirBlock) k_mirror_full_emit(const int4* __re
   }
 }
 
+// ---- table -> relation when the mirror's minor column is the relation's major one ----------------------------------
+// A grouped mirror (group_join.cuh) is indexed (column 1, column 0), the relation is ordered (column 0, column 1).  With at
+// most 64 values of column 0 the rows can be written straight to their final places, no sort: a block takes kMtNodes
+// values c of column 1 (one per thread); k_mirror_t_count counts, per value a of column 0, the tile's present keys
+// (c, a); an exclusive scan over (a, tile) gives every (a, tile) run its place; k_mirror_t_emit stages the tile's tags in
+// shared memory with coalesced reads and writes each column's rows in order of c: a warp's rows of one a are contiguous.
+constexpr int kMtNodes = 128;
+
+__device__ __forceinline__ unsigned long long mt_mask(const uint32_t* __restrict__ present, uint32_t c, uint32_t n_nodes, int slots) {
+  if (c >= n_nodes) return 0ull;
+  if (slots == 64) return *reinterpret_cast<const unsigned long long*>(present + 2 * (size_t)c);
+  const uint32_t w = present[((size_t)c * slots) >> 5];          // slots is 1, 2, 4, 8, 16 or 32: a word holds 32 / slots values of c
+  return (unsigned long long)((w >> ((c * slots) & 31)) & (slots == 32 ? 0xffffffffu : ((1u << slots) - 1u)));
+}
+
+static __global__ void __launch_bounds__(kMtNodes) k_mirror_t_count(const uint32_t* __restrict__ present, uint32_t n_nodes, uint32_t ntiles, int slots,
+                                                                   uint32_t* __restrict__ cnt) {
+  __shared__ uint32_t s_cnt[64];
+  if (threadIdx.x < 64) s_cnt[threadIdx.x] = 0;
+  __syncthreads();
+  const unsigned long long mask = mt_mask(present, blockIdx.x * kMtNodes + threadIdx.x, n_nodes, slots);
+  for (int a = 0; a < slots; ++a) {
+    const unsigned bal = __ballot_sync(0xffffffffu, (mask >> a) & 1ull);
+    if (bal && lane_id() == 0) atomicAdd(&s_cnt[a], (uint32_t)__popc(bal));
+  }
+  __syncthreads();
+  if ((int)threadIdx.x < slots) cnt[(size_t)threadIdx.x * ntiles + blockIdx.x] = s_cnt[threadIdx.x];
+}
+
+template <typename K>
+__global__ void __launch_bounds__(kMtNodes) k_mirror_t_emit(const uint32_t* __restrict__ present, const int32_t* __restrict__ table, uint32_t n_nodes,
+                                                           uint32_t ntiles, int slots, const uint32_t* __restrict__ base, int shift0, int shift1,
+                                                           K* __restrict__ keys, float* __restrict__ tags) {
+  constexpr int NW = kMtNodes / 32;
+  __shared__ int32_t s_tag[kMtNodes * 65];
+  __shared__ uint32_t s_wcnt[NW][64];
+  __shared__ uint32_t s_base[64];
+  const uint32_t c = blockIdx.x * kMtNodes + threadIdx.x;
+  const int slots_log2 = 31 - __clz(slots);
+  if ((int)threadIdx.x < slots) s_base[threadIdx.x] = base[(size_t)threadIdx.x * ntiles + blockIdx.x];
+  const unsigned long long mask = mt_mask(present, c, n_nodes, slots);
+  for (int a = 0; a < slots; ++a) {
+    const unsigned bal = __ballot_sync(0xffffffffu, (mask >> a) & 1ull);
+    if (lane_id() == 0) s_wcnt[warp_id()][a] = __popc(bal);
+  }
+  __syncthreads();
+  if (__syncthreads_or(mask != 0ull) == 0) return;       // nothing present in this tile
+  // the tile's slots are contiguous in the table: a straight 16-byte-vector copy into the padded shared array, all of a
+  // thread's reads in flight together (empty slots come along; their values are never used)
+  const size_t tile_slot0 = (size_t)blockIdx.x * kMtNodes * slots;
+  const int4* __restrict__ src = reinterpret_cast<const int4*>(table + tile_slot0);
+  const uint32_t nvec = (uint32_t)min((size_t)(kMtNodes * slots / 4), ((size_t)n_nodes * slots - tile_slot0 + 3) / 4);
+#pragma unroll 8
+  for (uint32_t v = threadIdx.x; v < nvec; v += kMtNodes) {
+    const int4 x = __ldcs(src + v);
+    const int32_t e[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t i = v * 4 + j;
+      s_tag[(i >> slots_log2) * 65 + (i & (slots - 1))] = e[j];
+    }
+  }
+  __syncthreads();
+  for (int a = 0; a < slots; ++a) {
+    const unsigned bal = __ballot_sync(0xffffffffu, (mask >> a) & 1ull);
+    if (!bal) continue;
+    uint32_t pos = s_base[a];
+    for (unsigned w = 0; w < warp_id(); ++w) pos += s_wcnt[w][a];
+    if ((mask >> a) & 1ull) {
+      pos += __popc(bal & lanemask_lt());
+      keys[pos] = ((K)(uint32_t)a << shift0) | ((K)c << shift1);
+      tags[pos] = ord2f(s_tag[threadIdx.x * 65 + a]);
+    }
+  }
+}
+
 }  // namespace xlog

@@ -40,7 +40,6 @@ constexpr int kResMaxVariants = 16;
 constexpr int kResScanItems = 4;                       // rows per thread in the fused count + scan: short dependent chains
 constexpr int kResScanTile = kScanBlock * kResScanItems;
 constexpr uint64_t kScanFlagAgg = 1ull << 62, kScanFlagIncl = 2ull << 62, kScanValMask = (1ull << 62) - 1;
-constexpr uint32_t kResSpinLimit = 1u << 22;          // polls of one status word before giving up
 
 __device__ __forceinline__ unsigned long long ld_volatile_u64(const unsigned long long* p) { return *reinterpret_cast<const volatile unsigned long long*>(p); }
 __device__ __forceinline__ void st_volatile_u64(unsigned long long* p, unsigned long long v) { *reinterpret_cast<volatile unsigned long long*>(p) = v; }
@@ -70,12 +69,12 @@ static __global__ void __launch_bounds__(1024) k_res_init(ResState* st, ResScrat
 // before it (aggregate first, inclusive prefix once known: a chained scan), writes the rows' start offsets, and - since
 // a row knows which candidate positions it covers - the first / last row of every expand tile whose boundary it covers.
 // The last tile publishes the candidate total and the expand tile count.  Waits are bounded: a status word that stays
-// empty for kResSpinLimit polls raises the internal-error flag and stops the resident loop.
+// empty for spin_limit polls (a value of the context) raises the internal-error flag and stops the resident loop.
 template <typename KO>
 __global__ void __launch_bounds__(kScanBlock) k_res_count_scan(JoinSpec S, const KO* __restrict__ okeys, const float* __restrict__ otags,
                                                                ResState* __restrict__ st, uint4* __restrict__ rowinfo, uint64_t* __restrict__ start,
                                                                uint2* __restrict__ tile_rows, unsigned long long* __restrict__ status,
-                                                               uint32_t* __restrict__ ticket, uint32_t* __restrict__ err) {
+                                                               uint32_t* __restrict__ ticket, uint32_t* __restrict__ err, uint32_t spin_limit) {
   __shared__ uint64_t sh[kScanBlock / 32 + 1];
   __shared__ uint32_t sdeg[kResScanTile];
   __shared__ uint32_t s_tile;
@@ -120,7 +119,7 @@ __global__ void __launch_bounds__(kScanBlock) k_res_count_scan(JoinSpec S, const
             for (;;) {
               v = ld_volatile_u64(status + idx);
               if (v & ~kScanValMask) break;
-              if (++spins > kResSpinLimit) { timeout = true; v = kScanFlagIncl; break; }
+              if (++spins > spin_limit) { timeout = true; v = kScanFlagIncl; break; }
               if (spins > 64) __nanosleep(32);
             }
           }

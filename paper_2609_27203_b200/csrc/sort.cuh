@@ -32,7 +32,7 @@ constexpr int kSortMaxBins = 256;
 constexpr int kSortMaxPasses = 8;
 constexpr uint32_t kSortMaxN = (1u << 30) - 1;       // status words keep 30 bits of count
 constexpr uint32_t kFlagLocal = 1u << 30, kFlagGlobal = 2u << 30, kCountMask = (1u << 30) - 1;
-constexpr uint32_t kSpinLimit = 1u << 22;            // polls of one status word before giving up
+constexpr uint32_t kSpinLimit = 1u << 22;            // default number of polls of one status word before giving up (a context may lower it)
 
 template <typename K> struct SortCfg { static constexpr int items = XLOG_SORT_ITEMS; };
 template <typename K> constexpr int sort_tile() { return kSortBlock * SortCfg<K>::items; }
@@ -154,7 +154,7 @@ __device__ __forceinline__ void sort_tile_body(const K* __restrict__ keys_in, co
                                                K* __restrict__ keys_out, uint32_t* __restrict__ vals_out, const uint64_t base,
                                                const uint32_t valid, const uint32_t tile, const int shift,
                                                const uint32_t* __restrict__ digit_base, uint32_t* __restrict__ status,
-                                               uint32_t* __restrict__ err, K* skeys, uint32_t* svals, uint32_t* whist,
+                                               uint32_t* __restrict__ err, const uint32_t spin_limit, K* skeys, uint32_t* svals, uint32_t* whist,
                                                uint32_t* lbase, uint32_t* goff, uint32_t* scan_sh) {
   constexpr int ITEMS = SortCfg<K>::items;
   constexpr int TILE = kSortBlock * ITEMS;
@@ -229,7 +229,7 @@ __device__ __forceinline__ void sort_tile_body(const K* __restrict__ keys_in, co
         const uint32_t s = ld_volatile_u32(&status[(uint64_t)look * kSortMaxBins + d]);
         const uint32_t flag = s & ~kCountMask;
         if (flag == 0) {
-          if (++spins > kSpinLimit) { timeout = true; break; }
+          if (++spins > spin_limit) { timeout = true; break; }
           __nanosleep(64);
           continue;
         }
@@ -238,7 +238,8 @@ __device__ __forceinline__ void sort_tile_body(const K* __restrict__ keys_in, co
         --look;
         spins = 0;
       }
-      st_volatile_u32(&status[(uint64_t)tile * kSortMaxBins + d], kFlagGlobal | ((excl + total_d) & kCountMask));
+      // a wait that gave up publishes nothing: the tiles behind this one must run into the same gap, not past it
+      if (!timeout) st_volatile_u32(&status[(uint64_t)tile * kSortMaxBins + d], kFlagGlobal | ((excl + total_d) & kCountMask));
     }
     if (timeout) { atomicOr(err, kErrInternal); scan_sh[kSortBlock / 32 + 2] = 1u; }
     goff[d] = digit_base[d] + excl - lb;
@@ -264,7 +265,7 @@ __global__ void __launch_bounds__(kSortBlock, sizeof(K) == 4 ? XLOG_SORT_MINB : 
                                                           K* __restrict__ keys_out, uint32_t* __restrict__ vals_out, uint32_t n,
                                                           int shift, const uint32_t* __restrict__ digit_base,
                                                           uint32_t* __restrict__ status, uint32_t* __restrict__ ticket,
-                                                          uint32_t* __restrict__ err) {
+                                                          uint32_t* __restrict__ err, uint32_t spin_limit) {
   constexpr int ITEMS = SortCfg<K>::items;
   constexpr int TILE = kSortBlock * ITEMS;
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -282,10 +283,10 @@ __global__ void __launch_bounds__(kSortBlock, sizeof(K) == 4 ? XLOG_SORT_MINB : 
   const uint64_t base = (uint64_t)tile * TILE;
   const uint32_t valid = (uint32_t)min((uint64_t)TILE, (uint64_t)n - base);
   if (valid == (uint32_t)TILE)
-    sort_tile_body<K, BITS, true>(keys_in, vals_in, keys_out, vals_out, base, valid, tile, shift, digit_base, status, err, skeys, svals,
+    sort_tile_body<K, BITS, true>(keys_in, vals_in, keys_out, vals_out, base, valid, tile, shift, digit_base, status, err, spin_limit, skeys, svals,
                                   whist, lbase, goff, scan_sh);
   else
-    sort_tile_body<K, BITS, false>(keys_in, vals_in, keys_out, vals_out, base, valid, tile, shift, digit_base, status, err, skeys, svals,
+    sort_tile_body<K, BITS, false>(keys_in, vals_in, keys_out, vals_out, base, valid, tile, shift, digit_base, status, err, spin_limit, skeys, svals,
                                    whist, lbase, goff, scan_sh);
 }
 

@@ -245,11 +245,12 @@ __global__ void __launch_bounds__(256) k_tri_compact(const uint32_t* __restrict_
 
 // ---- the binary-join plan of the same query (paper: "WCOJ vs. the binary-join plan") -------------------------------
 // Step one materialises every two-path (x,y,z) of the first two atoms with the ordinary join kernels; step two, here,
-// keeps the two-paths that the third atom closes: one thread per two-path looks (z, x) up in the third relation's
+// keeps the paths that the closing atom closes: one thread per path looks (last column, x) up in the closing relation's
 // store (offsets over its column 0, then a binary search in the run's sorted column 1).  count -> scan -> emit, in
 // input order, so the output is sorted by (x,y,z) like the worst-case-optimal path's.
 struct ChainProbe {
-  KeyLayout L;                   // layout of the two-path keys (x,y,z): wide enough for everything r and s hold
+  int last;                      // index of the path's last column: 2 for the two-paths (x,y,z) of the triangle, 3 for the three-paths of the four-cycle
+  KeyLayout L;                   // layout of the path keys (x,y,z[,w]): wide enough for everything the joined atoms hold
   KeyLayout out;                 // layout of the head relation (its bounds take t into account as well)
   int64_t t_domain;
   const uint32_t* t_off;         // offsets over the third relation's column 0
@@ -260,7 +261,7 @@ struct ChainProbe {
 
 template <typename K>
 __device__ __forceinline__ bool chain_lookup(const ChainProbe& P, K key, uint32_t& pos) {
-  const int32_t x = key_col<K>(P.L, key, 0), z = key_col<K>(P.L, key, 2);
+  const int32_t x = key_col<K>(P.L, key, 0), z = key_col<K>(P.L, key, P.last);
   if (z >= P.t_domain) return false;
   uint32_t lo = P.t_off[z];
   const uint32_t end = P.t_off[z + 1];
@@ -289,7 +290,8 @@ __global__ void __launch_bounds__(256) k_chain_probe_emit(ChainProbe P, const K*
     const float w = P.t_w[pos];
     KH hk = 0;
 #pragma unroll
-    for (int col = 0; col < 3; ++col) hk |= (KH)(uint32_t)key_col<K>(P.L, keys[i], col) << P.out.shift[col];
+    for (int col = 0; col < kMaxArity; ++col)
+      if (col <= P.last) hk |= (KH)(uint32_t)key_col<K>(P.L, keys[i], col) << P.out.shift[col];
     out_keys[off[i]] = hk;
     out_tags[off[i]] = P.times ? tags[i] * w : tags[i] + w;
   }

@@ -318,6 +318,7 @@ void add_rule(Ctx* c, const xlog_plan* p, xlog_rule* out) {
 Index& ensure_index(Ctx* c, Relation& R, int col) {
   Index& ix = R.idx[col];
   if (ix.valid) return ix;
+  ++c->r_index_builds;
   ensure_soa(c, R);
   ix = Index();
   ix.domain = (int64_t)R.val_max[col] + 1;
@@ -945,6 +946,7 @@ void triangle_chain(Ctx* c, Relation& H, const Relation& H2, Counted& q, Relatio
   // step two: probe t with (z, x)
   Index& tix = ensure_index(c, T, 0);
   ChainProbe P{};
+  P.last = 2;
   P.L = H2.layout; P.out = H.layout;
   P.t_domain = tix.domain; P.t_off = tix.off.as<uint32_t>(); P.t_col1 = tix.other[0]; P.t_w = tix.tags; P.times = times;
   DevBuf hit(c, std::max<uint64_t>(n2, 1) * 4), off(c, std::max<uint64_t>(n2, 1) * 8);
@@ -1056,15 +1058,18 @@ void triangle_materialise(Ctx* c, Relation& H, const RuleC& r) {
   set_current(H, std::move(kt));
 }
 
-// c4(x,y,z,w) :- r(x,y), s(y,z), t(z,w), u(w,x): the two-paths of r and s through the ordinary join, then per two-path
-// the intersection of t's out-list of z with u's in-list of x (count -> scan -> write; see cycle4.cuh).
+// c4(x,y,z,w) :- r(x,y), s(y,z), t(z,w), u(w,x): the two-paths of r and s through the ordinary join, then either the
+// multiway step (per two-path the intersection of t's out-list of z with u's in-list of x: count -> scan -> write; see
+// cycle4.cuh) or the rest of the binary-join chain (every three-path written out, then a probe of u), as the skew test says.
 void cycle4_materialise(Ctx* c, Relation& H, const RuleC& r) {
   Relation& R = *c->rels[r.plan.atoms[0].rel];
   Relation& S = *c->rels[r.plan.atoms[1].rel];
   Relation& T = *c->rels[r.plan.atoms[2].rel];
   Relation& U = *c->rels[r.plan.atoms[3].rel];
   if (H.n_facts) fail(XLOG_ERR_UNSUPPORTED, "a materialised four-cycle relation cannot also hold loaded facts");
-  c->last_triangle_plan = XLOG_PLAN_WCOJ;
+  // empty inputs take the chain (nothing to intersect), as for the triangle
+  const int empty_plan = (c->flags & XLOG_FLAG_FORCE_WCOJ) ? XLOG_PLAN_WCOJ : XLOG_PLAN_CHAIN;
+  c->last_triangle_plan = empty_plan;
   if (R.n == 0 || S.n == 0 || T.n == 0 || U.n == 0) { KeyTags empty; set_current(H, std::move(empty)); return; }
   RuleC two;                                             // tmp(x,y,z) :- r(x,y), s(y,z)
   two.plan = r.plan;
@@ -1092,6 +1097,7 @@ void cycle4_materialise(Ctx* c, Relation& H, const RuleC& r) {
   if (need > c->arena.largest_free() / 2) fail(XLOG_ERR_RESOURCE_EXHAUSTED, "four-cycle: the two-paths do not fit the arena");
   c->r_candidates += (int64_t)n2;
   if (n2 == 0) { KeyTags empty; set_current(H, std::move(empty)); return; }
+  c->last_triangle_plan = XLOG_PLAN_WCOJ;
   DevBuf k0(c, n2 * ckb), t0(c, n2 * 4);
   c->note_bytes = (int64_t)n2 * (ckb + 4 + 8);
   launch_expand<false>(c, q, 0, n2, ckb, k0.p, t0.as<float>(), BwdArgs{});
@@ -1109,6 +1115,80 @@ void cycle4_materialise(Ctx* c, Relation& H, const RuleC& r) {
   zero_ctrl(c, kSlotTotals);
   const unsigned grid = (unsigned)std::min<uint64_t>((n2 + 255) / 256, (uint64_t)kSMs * 8);
   KeyTags kt;
+  // skew test (as for the triangle): count the three-paths of r, s and t exactly, the chain's intermediate; the chain is taken
+  // when they number at most kChainMaxBlowup per row of the largest input and fit the arena, the multiway plan otherwise
+  if (!(c->flags & XLOG_FLAG_FORCE_WCOJ)) {
+    int32_t mx3[kMaxArity] = {H2.col_max[0], H2.col_max[1], H2.col_max[2], T.val_max[1] ? T.val_max[1] : T.col_max[1]};
+    const KeyLayout L3 = make_layout(4, mx3);
+    const int kb3 = L3.total_bits <= 32 ? 4 : 8;
+    Cycle4 P3 = P;
+    P3.L = L3;
+    DISPATCH_K(ckb, XLOG_LAUNCH(c, (k_c4_chain_count<K>), grid, 256, 0, P3, (const K*)k0.p, n2, cnt.as<uint32_t>()));
+    XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)cnt.as<uint32_t>(), (int64_t)n2, sums.as<uint64_t>());
+    XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, sums.as<uint64_t>(), (int64_t)tiles, (uint64_t*)(c->d_ctrl + kSlotTotals));
+    XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint64_t>), tiles, kScanBlock, 0, (const uint32_t*)cnt.as<uint32_t>(), (int64_t)n2,
+                (const uint64_t*)sums.as<uint64_t>(), off.as<uint64_t>());
+    sync_ctrl(c);
+    const uint64_t n3 = c->h_ctrl[kSlotTotals];
+    const uint64_t biggest = std::max<uint64_t>(std::max<uint64_t>(R.n, S.n), std::max<uint64_t>(T.n, U.n));
+    const size_t need3 = (size_t)n3 * (kb3 + 4 + 12) + (16u << 20);
+    const bool fits = L3.total_bits <= 64 && n3 <= kSortMaxN && need3 <= c->arena.largest_free() / 2;
+    bool chain = fits && n3 <= kChainMaxBlowup * biggest;
+    if (c->flags & XLOG_FLAG_FORCE_CHAIN) {
+      if (!fits) fail(XLOG_ERR_RESOURCE_EXHAUSTED, "four-cycle chain: the three-path intermediate does not fit the arena");
+      chain = true;
+    }
+    if (chain) {
+      c->last_triangle_plan = XLOG_PLAN_CHAIN;
+      c->r_candidates += (int64_t)n3;
+      if (n3 == 0) { KeyTags empty; set_current(H, std::move(empty)); return; }
+      DevBuf k3(c, n3 * kb3), t3(c, n3 * 4);
+      c->note_bytes = (int64_t)n2 * (ckb + 4 + 8) + (int64_t)n3 * (kb3 + 4 + 8);
+#define XLOG_C4_CHAIN(K2, K3) \
+  XLOG_LAUNCH(c, (k_c4_chain_expand<K2, K3>), grid, 256, 0, P3, (const K2*)k0.p, (const float*)t0.as<float>(), n2, (const uint64_t*)off.as<uint64_t>(), k3.as<K3>(), t3.as<float>())
+      if (ckb == 4 && kb3 == 4) XLOG_C4_CHAIN(uint32_t, uint32_t);
+      else if (ckb == 4) XLOG_C4_CHAIN(uint32_t, uint64_t);
+      else if (kb3 == 4) XLOG_C4_CHAIN(uint64_t, uint32_t);
+      else XLOG_C4_CHAIN(uint64_t, uint64_t);
+#undef XLOG_C4_CHAIN
+      k0.reset(); t0.reset(); cnt.reset(); off.reset(); sums.reset();
+      // probe u with (w, x)
+      Index& ux = ensure_index(c, U, 0);
+      ChainProbe Q{};
+      Q.last = 3;
+      Q.L = L3; Q.out = H.layout;
+      Q.t_domain = ux.domain; Q.t_off = ux.off.as<uint32_t>(); Q.t_col1 = ux.other[0]; Q.t_w = ux.tags; Q.times = P.times;
+      DevBuf hit(c, n3 * 4), hoff(c, n3 * 8);
+      const unsigned tiles3 = (unsigned)((n3 + kScanTile - 1) / kScanTile);
+      DevBuf sums3(c, (size_t)tiles3 * 8);
+      zero_ctrl(c, kSlotTotals);
+      c->note_bytes = (int64_t)n3 * (kb3 + 4);
+      DISPATCH_K(kb3, XLOG_LAUNCH(c, (k_chain_probe_count<K>), grid_for(n3, 256), 256, 0, Q, (const K*)k3.p, n3, hit.as<uint32_t>()));
+      XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint64_t>), tiles3, kScanBlock, 0, (const uint32_t*)hit.as<uint32_t>(), (int64_t)n3, sums3.as<uint64_t>());
+      XLOG_LAUNCH(c, (k_scan_spine<uint64_t>), 1, 1024, 0, sums3.as<uint64_t>(), (int64_t)tiles3, (uint64_t*)(c->d_ctrl + kSlotTotals));
+      XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint64_t>), tiles3, kScanBlock, 0, (const uint32_t*)hit.as<uint32_t>(), (int64_t)n3,
+                  (const uint64_t*)sums3.as<uint64_t>(), hoff.as<uint64_t>());
+      sync_ctrl(c);
+      const uint64_t total = c->h_ctrl[kSlotTotals];
+      if (total > kSortMaxN) fail(XLOG_ERR_CAPACITY_EXCEEDED, "materialised four-cycle relation exceeds 2^30 - 1 rows");
+      c->r_unique += (int64_t)total;
+      kt.n = (uint32_t)total;
+      kt.keys = DevBuf(c, (size_t)std::max<uint64_t>(total, 1) * H.key_bytes);
+      kt.tags = DevBuf(c, (size_t)std::max<uint64_t>(total, 1) * 4);
+      c->note_bytes = (int64_t)n3 * (kb3 + 4 + 12) + (int64_t)total * (H.key_bytes + 4);
+#define XLOG_C4_EMIT(K3, KH) \
+  XLOG_LAUNCH(c, (k_chain_probe_emit<K3, KH>), grid_for(n3, 256), 256, 0, Q, (const K3*)k3.p, (const float*)t3.as<float>(), n3, \
+              (const uint32_t*)hit.as<uint32_t>(), (const uint64_t*)hoff.as<uint64_t>(), kt.keys.as<KH>(), kt.tags.as<float>())
+      if (kb3 == 4 && H.key_bytes == 4) XLOG_C4_EMIT(uint32_t, uint32_t);
+      else if (kb3 == 4) XLOG_C4_EMIT(uint32_t, uint64_t);
+      else if (H.key_bytes == 4) XLOG_C4_EMIT(uint64_t, uint32_t);
+      else XLOG_C4_EMIT(uint64_t, uint64_t);
+#undef XLOG_C4_EMIT
+      set_current(H, std::move(kt));
+      return;
+    }
+    zero_ctrl(c, kSlotTotals);
+  }
   // long runs of equal x and small w values: the bitmap kernel (see cycle4.cuh)
   const uint64_t w_max = (uint64_t)(U.val_max[0] ? U.val_max[0] : U.col_max[0]);
   const uint64_t x_values = std::min<uint64_t>(R.n, (uint64_t)(R.val_max[0] ? R.val_max[0] : R.col_max[0]) + 1);
@@ -1331,7 +1411,7 @@ void resident_body(Ctx* c, Resident& R, const std::vector<JoinSpec>& specs, bool
   for (size_t v = 0; v < specs.size(); ++v) {
     const JoinSpec& S = specs[v];
     XLOG_LAUNCH(c, (k_res_count_scan<uint32_t>), kSMs * 4, kScanBlock, 0, S, dk, (const float*)R.dtags.as<float>(), st, R.rowinfo.as<uint4>(),
-                R.start.as<uint64_t>(), R.tile_rows.as<uint2>(), sc.scan_status + v * R.scan_tiles_cap, sc.tickets + v, err);
+                R.start.as<uint64_t>(), R.tile_rows.as<uint2>(), sc.scan_status + v * R.scan_tiles_cap, sc.tickets + v, err, c->spin_limit);
 // four waves of blocks: the hardware hands a new block to whichever SM finishes first, which evens out skewed tiles
 #define XLOG_RES_EXPAND(MODE, SINK)                                                                                                         \
   XLOG_LAUNCH(c, (k_res_expand<uint32_t, MODE, SINK>), kSMs * kExpMirrorBlocksPerSM * 4, kExpBlock, 0, S, dk, (const ResState*)st, (const uint64_t*)R.start.as<uint64_t>(), \
@@ -1377,7 +1457,7 @@ ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*
     std::vector<char> sig;
     for (const JoinSpec& S : specs) sig_add(sig, S);
     sig_add(sig, mr.table); sig_add(sig, mr.changed); sig_add(sig, mr.n_new); sig_add(sig, mr.key_max); sig_add(sig, mr.err); sig_add(sig, R.present.p);
-    sig_add(sig, is_max); sig_add(sig, bm_quads); sig_add(sig, ch_tiles); sig_add(sig, c->d_ctrl);
+    sig_add(sig, is_max); sig_add(sig, bm_quads); sig_add(sig, ch_tiles); sig_add(sig, c->d_ctrl); sig_add(sig, c->spin_limit);
     if (!R.exec || sig != R.sig) {
       if (R.exec) { cudaGraphExecDestroy(R.exec); R.exec = nullptr; }
       if (R.graph) { cudaGraphDestroy(R.graph); R.graph = nullptr; }
@@ -1549,15 +1629,15 @@ static_assert(kSlotBm + kBmTotals <= kCtrlSlots, "control block too small");
 struct BitmapJoin {
   bool valid = false;
   JoinSpec spec;
-  DevBuf snap, items;
+  DevBuf pairs, items;
   int carried_bits = 0;
 };
 
 // Applicable when exactly one rule has an atom over h (so a round is one join), that rule has the grouped shape with the
-// linear-key form, a unit of 32 carried values fits one value of the probed column, and the snapshot table and the item
-// list (sized for every unit changing in one round) fit the arena.
+// linear-key form, a value of the probed column owns 1 to 32 whole bitmap words, and the pair list and the item list
+// (sized for every key changing in one round) fit the arena.
 void bitmap_join_setup(Ctx* c, int h, const std::vector<const RuleC*>& rs, const KeyLayout& M, int carried_bits, uint64_t slots, BitmapJoin& bj) {
-  if ((c->flags & XLOG_FLAG_NO_BITMAP_JOIN) || carried_bits < 5) return;
+  if ((c->flags & XLOG_FLAG_NO_BITMAP_JOIN) || carried_bits < 5 || carried_bits > 5 + kBmMaxWordsLog2) return;
   Relation& H = *c->rels[h];
   if (H.dict_n[1]) return;
   const RuleC* rule = nullptr; int pos = -1, n_over = 0;
@@ -1571,13 +1651,13 @@ void bitmap_join_setup(Ctx* c, int h, const std::vector<const RuleC*>& rs, const
       S.inner_mult[0] != ((uint64_t)1 << carried_bits))
     return;
   const Relation& RB = *c->rels[rule->plan.atoms[1 - pos].rel];
-  const uint64_t units_per_value = (uint64_t)1 << (carried_bits - 5);
+  const uint64_t passes = (uint64_t)1 << (carried_bits - 5);             // at most one pass per 32 carried values
   const uint64_t values = std::min<uint64_t>((uint64_t)S.inner_domain, slots >> carried_bits);
-  const uint64_t max_items = ((uint64_t)RB.n / kBmSlice + values + 1) * units_per_value;
+  const uint64_t max_items = ((uint64_t)RB.n / kBmSlice + values + 1) * passes;
   if (max_items >= ((uint64_t)1 << 32)) return;
-  const uint64_t need = slots * 4 + max_items * 16 + (1u << 20);
+  const uint64_t need = slots * 8 + max_items * 16 + (1u << 20);          // a round can change every key: one (tag, carried value) pair each
   if (need > c->arena.largest_free() / 2) return;
-  bj.snap = DevBuf(c, slots * 4);
+  bj.pairs = DevBuf(c, slots * 8);
   bj.items = DevBuf(c, max_items * 16);
   bj.spec = S;
   bj.carried_bits = carried_bits;
@@ -1713,21 +1793,23 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
     if (total == 0 && !(round == 0 && plain_rules_done)) break;
     if (bj.valid) {
       // Every later round is  k_bm_plan -> one control read -> k_bm_expand : the plan kernel closes the round just joined
-      // (changed / new keys, bitmap cleared, snapshot of the changed units' tags) and lays out the next one's work items.
+      // (changed / new keys, bitmap cleared, the changed keys' tags set aside) and lays out the next one's work items.
       const uint32_t nwords = bm_quads * 4;
-      BmPlan P{reinterpret_cast<uint32_t*>(bitmap), present, nwords, table, bj.snap.as<int32_t>(), carried_bits - 5, bj.spec.inner_off,
+      BmPlan P{reinterpret_cast<uint32_t*>(bitmap), present, nwords, table, bj.pairs.as<uint2>(), carried_bits - 5, bj.spec.inner_off,
                (uint32_t)std::min<int64_t>(bj.spec.inner_domain, 0xffffffffll), bj.items.as<uint4>(), (unsigned long long*)(c->d_ctrl + kSlotBm)};
-      BmExpand E{bj.items.as<uint4>(), 0, bj.spec.inner_col[0], bj.spec.inner_tag, H.layout.mask[1], carried_bits, bj.snap.as<int32_t>(), table,
-                 reinterpret_cast<uint32_t*>(bitmap), ctrl_u32(c, kSlotErr)};
+      BmExpand E{bj.items.as<uint4>(), 0, bj.spec.inner_col[0], bj.spec.inner_tag, H.layout.mask[1], carried_bits,
+                 bj.pairs.as<uint2>(), table, reinterpret_cast<uint32_t*>(bitmap), ctrl_u32(c, kSlotErr)};
       for (;;) {
         zero_ctrl(c, kSlotBm, kBmTotals);
-        c->note_bytes = (int64_t)nwords * 4;
+        c->note_bytes = (int64_t)nwords * 4;              // plus 12 bytes per changed key and 16 per item, not known yet
         XLOG_LAUNCH(c, k_bm_plan, (nwords + kBmPlanTile - 1) / kBmPlanTile, kBmPlanBlock, 0, P);
         sync_ctrl(c);
         const uint64_t changed = c->h_ctrl[kSlotBm + kBmChanged], n_new = c->h_ctrl[kSlotBm + kBmNew], cand = c->h_ctrl[kSlotBm + kBmCandidates];
-        const uint64_t n_items = c->h_ctrl[kSlotBm + kBmItems], nbrs = c->h_ctrl[kSlotBm + kBmNeighbours];
+        const uint64_t n_items = c->h_ctrl[kSlotBm + kBmReserve] >> 32, nbrs = c->h_ctrl[kSlotBm + kBmNeighbours];
         total_new += n_new;
         c->r_new += (int64_t)n_new; c->r_improved += (int64_t)changed - (int64_t)n_new;
+        if (getenv("XLOG_TRACE")) fprintf(stderr, "bm round %lld: changed %llu new %llu cand %llu items %llu nbrs %llu\n", (long long)round, (unsigned long long)changed,
+                                          (unsigned long long)n_new, (unsigned long long)cand, (unsigned long long)n_items, (unsigned long long)nbrs);
         if (changed == 0) break;
         ++round;
         if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
@@ -1735,8 +1817,8 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
         if (cand == 0) break;
         c->r_candidates += (int64_t)cand;
         E.n_items = (uint32_t)n_items;
-        // per candidate its slot; per (unit, neighbour) the looked-up column and tag; per item its record and the unit's 32 snapshot tags
-        c->note_bytes = (int64_t)cand * 4 + (int64_t)nbrs * 8 + (int64_t)n_items * 144;
+        // per candidate its slot; per (b, neighbour) the looked-up column and tag; per item its record; per changed key its pair
+        c->note_bytes = (int64_t)cand * 4 + (int64_t)nbrs * 8 + (int64_t)n_items * 16 + (int64_t)changed * 8;
         const unsigned grid = (unsigned)std::min<uint64_t>((n_items + 7) / 8, (uint64_t)kSMs * 8 * 16);
         if (is_max) XLOG_LAUNCH(c, (k_bm_expand<kSinkMax>), grid, 256, 0, E);
         else XLOG_LAUNCH(c, (k_bm_expand<kSinkMin>), grid, 256, 0, E);
@@ -1769,7 +1851,27 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
   full.n = (uint32_t)n_out;
   full.keys = DevBuf(c, (size_t)std::max<uint64_t>(n_out, 1) * 4);
   full.tags = DevBuf(c, (size_t)std::max<uint64_t>(n_out, 1) * 4);
-  if (n_out) {
+  bool counted_slots = false;              // kSlotA holds the number of occupied slots (for the invariant check)
+  if (n_out && grouped && carried_bits <= 6) {
+    // the mirror is ordered (column 1, column 0) and column 0 has at most 64 values: every row goes straight to its place
+    // in the relation's order (mirror.cuh), found from the bitmap of present keys; no pass over empty slots, no sort
+    const int per_node = 1 << carried_bits;
+    const uint32_t n_nodes = (uint32_t)(slots >> carried_bits);
+    const uint32_t ntiles = (n_nodes + kMtNodes - 1) / kMtNodes;
+    const int64_t len = (int64_t)per_node * ntiles;
+    const unsigned stiles = (unsigned)((len + kScanTile - 1) / kScanTile);
+    DevBuf cnt(c, (size_t)len * 4), base(c, (size_t)len * 4), sums(c, (size_t)stiles * 4);
+    c->note_bytes = (int64_t)slots / 8;
+    XLOG_LAUNCH(c, k_mirror_t_count, ntiles, kMtNodes, 0, (const uint32_t*)present, n_nodes, ntiles, per_node, cnt.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), stiles, kScanBlock, 0, (const uint32_t*)cnt.as<uint32_t>(), len, sums.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, sums.as<uint32_t>(), (int64_t)stiles, ctrl_u32(c, kSlotA));
+    XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), stiles, kScanBlock, 0, (const uint32_t*)cnt.as<uint32_t>(), len, (const uint32_t*)sums.as<uint32_t>(),
+                base.as<uint32_t>());
+    c->note_bytes = (int64_t)slots / 8 + (int64_t)n_out * 12;
+    XLOG_LAUNCH(c, (k_mirror_t_emit<uint32_t>), ntiles, kMtNodes, 0, (const uint32_t*)present, (const int32_t*)table, n_nodes, ntiles, per_node,
+                (const uint32_t*)base.as<uint32_t>(), H.layout.shift[0], H.layout.shift[1], full.keys.as<uint32_t>(), full.tags.as<float>());
+    counted_slots = true;
+  } else if (n_out) {
     const uint64_t nquads = slots / 4;
     const unsigned tiles = (unsigned)((slots + kMirSlotsPerTile - 1) / kMirSlotsPerTile);
     DevBuf sums(c, (size_t)tiles * 4);
@@ -1779,10 +1881,11 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
     c->note_bytes = (int64_t)slots * 4 + (int64_t)n_out * 8;
     XLOG_LAUNCH(c, (k_mirror_full_emit<uint32_t>), tiles, kMirBlock, 0, (const int4*)table, nquads, empty, (const uint32_t*)sums.as<uint32_t>(), M, H.layout,
                 full.keys.as<uint32_t>(), full.tags.as<float>());
+    counted_slots = true;
     if (grouped && n_out > 1) {
       // rows came out in the mirror's order, (column 1, column 0) ascending: a stable sort on column 0's bits alone puts
       // them in the relation's key order
-      table_own.reset(); bitmap_own.reset(); present_own.reset(); bj.snap.reset(); bj.items.reset();
+      table_own.reset(); bitmap_own.reset(); present_own.reset(); bj.pairs.reset(); bj.items.reset();
       DevBuf ak(c, (size_t)n_out * 4), at(c, (size_t)n_out * 4);
       uint32_t* pk = full.keys.as<uint32_t>(); uint32_t* qk = ak.as<uint32_t>();
       float* pt = full.tags.as<float>(); float* qt = at.as<float>();
@@ -1794,18 +1897,80 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
   if (c->flags & XLOG_FLAG_CHECK_INVARIANTS) {
     XLOG_LAUNCH(c, (k_check_sorted<uint32_t>), grid_for(H.n, 256), 256, 0, (const uint32_t*)H.keys(), (int64_t)H.n, ctrl_u32(c, kSlotErr));
     sync_ctrl(c);
-    if (n_out && (uint64_t)(uint32_t)c->h_ctrl[kSlotA] != n_out) fail(XLOG_ERR_INTERNAL, "tag mirror: occupied slots disagree with the tuple count");
+    if (n_out && counted_slots && (uint64_t)(uint32_t)c->h_ctrl[kSlotA] != n_out) fail(XLOG_ERR_INTERNAL, "tag mirror: occupied slots disagree with the tuple count");
+  }
+}
+
+// Recursive component under a non-idempotent oplus (logsumexp / sum): the tag of a tuple is the oplus over all of its
+// derivations, which is finite when the tuples' dependencies form a DAG (path counting, path-probability sums on an
+// acyclic graph).  Algorithm 1 with the delta carrying tag DIFFERENCES: the rules are linear in the component's relations
+// (one recursive atom each), so  I_{k+1} - I_k = T_rec(I_k - I_{k-1}):
+//   Delta_1 = T(facts) with every atom reading the full relation;  Delta_{k+1} = T_rec(Delta_k);  I_{k+1} = I_k oplus Delta_{k+1}
+// (sort -> reduce-by-key gives Delta, the merge kernel's union-with-oplus gives I), until a round derives nothing.  A cyclic
+// dependency never gets there and ends at the iteration cap.  The component is recomputed from its loaded facts on
+// every call: adding to an earlier result would count every derivation twice.
+void stratum_recursive_additive(Ctx* c, const std::vector<int>& comp, const std::vector<const RuleC*>& rs) {
+  for (const RuleC* r : rs) {
+    int in = 0;
+    for (int j = 0; j < r->plan.n_atoms; ++j) if (in_set(comp, r->plan.atoms[j].rel)) ++in;
+    if (in > 1) fail(XLOG_ERR_UNSUPPORTED, "a rule with two recursive atoms under a non-idempotent oplus (logsumexp / sum)");
+  }
+  for (int p : comp) drop_current(*c->rels[p]);
+  std::vector<KeyTags> delta(c->rels.size());
+  for (int64_t round = 0;; ++round) {
+    if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint (cyclic derivations under a non-idempotent oplus never end)");
+    ++c->r_iterations;
+    std::vector<std::pair<int, KeyTags>> produced;
+    for (int h : comp) {
+      Relation& H = *c->rels[h];
+      std::vector<Variant> vs;
+      for (const RuleC* r : rs) {
+        if (r->plan.head_rel != h) continue;
+        if (round == 0) {
+          const int outer = seed_outer(comp, r);
+          vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
+        } else {
+          for (int j = 0; j < r->plan.n_atoms; ++j) {
+            const int ar = r->plan.atoms[j].rel;
+            if (!in_set(comp, ar) || r->plan.atoms[j].negated || delta[ar].n == 0) continue;
+            const Relation& RA = *c->rels[ar];
+            vs.push_back(Variant{r, j, Source{delta[ar].keys.p, delta[ar].tags.as<float>(), delta[ar].n, RA.layout, RA.key_bytes}});
+          }
+        }
+      }
+      if (!vs.empty()) produced.emplace_back(h, evaluate(c, H, vs, nullptr, H.layout, false));
+    }
+    for (int p : comp) delta[p] = KeyTags();
+    uint64_t derived = 0;
+    for (auto& pr : produced) {
+      Relation& H = *c->rels[pr.first];
+      KeyTags& u = pr.second;
+      if (u.n == 0) continue;
+      derived += u.n;
+      MergeResult m;
+      DISPATCH_K(H.key_bytes, m = merge<K>(c, H.sr, u.keys.as<K>(), u.tags.as<float>(), u.n, -1, (const K*)H.keys(), H.tags(), H.n, false, false));
+      c->r_new += m.n_new; c->r_improved += (int64_t)u.n - m.n_new;
+      set_current(H, std::move(m.full));
+      delta[pr.first] = std::move(u);
+      if (c->flags & XLOG_FLAG_CHECK_INVARIANTS) {
+        DISPATCH_K(H.key_bytes, XLOG_LAUNCH(c, (k_check_sorted<K>), grid_for(H.n, 256), 256, 0, (const K*)H.keys(), (int64_t)H.n, ctrl_u32(c, kSlotErr)));
+        sync_ctrl(c);
+      }
+    }
+    if (derived == 0) break;
   }
 }
 
 // Recursive component: Algorithm 1 with tag improvement.
 void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<const RuleC*>& rs) {
-  for (int p : comp) if (c->rels[p]->sr != XLOG_SR_MAXPLUS && c->rels[p]->sr != XLOG_SR_MINPLUS)
-    fail(XLOG_ERR_UNSUPPORTED, "relation '" + c->rels[p]->name + "': only max/min tags may be aggregated inside a recursive component");
+  int idem = 0, additive = 0;
+  for (int p : comp) { if (c->rels[p]->sr == XLOG_SR_MAXPLUS || c->rels[p]->sr == XLOG_SR_MINPLUS) ++idem; else ++additive; }
+  if (idem && additive) fail(XLOG_ERR_UNSUPPORTED, "a recursive component mixes max/min relations with logsumexp/sum relations");
   for (const RuleC* r : rs) {
     if (r->plan.emit_count_column) fail(XLOG_ERR_UNSUPPORTED, "count inside a recursive component");
     if (r->kind == 3 || r->kind == 4 || r->kind == 6) fail(XLOG_ERR_UNSUPPORTED, "triangle or four-cycle rule inside a recursive component");
   }
+  if (additive) { stratum_recursive_additive(c, comp, rs); return; }
   if (mirror_applies(c, comp, rs)) { stratum_recursive_mirror(c, comp[0], rs); return; }
   std::vector<KeyTags> delta(c->rels.size());
   for (int64_t round = 0;; ++round) {
@@ -2033,7 +2198,7 @@ xlog_status xlog_fixpoint(xlog_ctx* c, xlog_receipt* receipt) {
   if (!c) return XLOG_ERR_INVALID_ARGUMENT;
   if (receipt && receipt->struct_size != sizeof(xlog_receipt)) return XLOG_ERR_INVALID_ARGUMENT;
   const int64_t l0 = c->launches, d0 = c->d2h_bytes, h0 = c->h2d_bytes;
-  c->r_candidates = c->r_unique = c->r_new = c->r_improved = c->r_iterations = c->r_strata = 0;
+  c->r_candidates = c->r_unique = c->r_new = c->r_improved = c->r_iterations = c->r_strata = c->r_index_builds = 0;
   c->unique_untracked = false;
   c->last_triangle_plan = XLOG_PLAN_NONE;
   c->arena.reset_peak();
@@ -2067,7 +2232,7 @@ xlog_status xlog_fixpoint(xlog_ctx* c, xlog_receipt* receipt) {
     receipt->peak_arena_bytes = (int64_t)c->arena.peak();
     receipt->device_ms = ms;
     receipt->triangle_plan = c->last_triangle_plan;
-    receipt->reserved = 0;
+    receipt->index_builds = (int32_t)std::min<int64_t>(c->r_index_builds, INT32_MAX);
   }
   return st;
 }
@@ -2088,6 +2253,41 @@ xlog_status xlog_sort_pairs(xlog_ctx* c, void* keys, void* payload, int64_t n, i
       }
     });
     sync_ctrl(c);
+  });
+}
+
+xlog_status xlog_debug_set_poll_limit(xlog_ctx* c, uint32_t polls) {
+  return guarded(c, [&] {
+    if (polls == 0) fail(XLOG_ERR_INVALID_ARGUMENT, "poll limit must be positive");
+    c->spin_limit = polls;
+  });
+}
+
+// One 8-bit sort pass whose first tile never runs: tiles 1 .. T-1 are launched (tickets start at 1), tile 0's status words
+// stay empty, and every look-back that reaches them gives up after the context's poll limit.
+xlog_status xlog_debug_sort_pass_without_first_tile(xlog_ctx* c, const void* keys, const void* payload, void* out_keys, void* out_payload, int64_t n,
+                                                    int32_t key_bytes) {
+  return guarded(c, [&] {
+    if (!keys || !payload || !out_keys || !out_payload || (key_bytes != 4 && key_bytes != 8) || n <= 0 || n > (int64_t)kSortMaxN)
+      fail(XLOG_ERR_INVALID_ARGUMENT, "xlog_debug_sort_pass_without_first_tile: bad argument");
+    DISPATCH_K(key_bytes, {
+      const uint32_t ntiles = (uint32_t)((n + sort_tile<K>() - 1) / sort_tile<K>());
+      if (ntiles < 2) fail(XLOG_ERR_INVALID_ARGUMENT, "xlog_debug_sort_pass_without_first_tile: needs at least two tiles of rows");
+      const SortPasses P = make_sort_passes(0, 8);
+      const size_t head_words = (size_t)kSortMaxPasses * kSortMaxBins + kSortMaxPasses + 8;
+      DevBuf scratch(c, (head_words + (size_t)ntiles * kSortMaxBins) * 4);
+      uint32_t* hist = scratch.as<uint32_t>();
+      uint32_t* tickets = hist + kSortMaxPasses * kSortMaxBins;
+      uint32_t* done = tickets + kSortMaxPasses;
+      XLOG_CUDA(cudaMemsetAsync(hist, 0, (head_words + (size_t)ntiles * kSortMaxBins) * 4, c->stream));
+      zero_ctrl(c, kSlotErr);
+      XLOG_LAUNCH(c, (k_sort_digit_hist<K>), grid_for(n, 256 * 8, kSMs * 8), 256, 0, (const K*)keys, (uint32_t)n, P, hist, done);
+      const uint32_t one = 1;
+      XLOG_CUDA(cudaMemcpyAsync(tickets, &one, 4, cudaMemcpyHostToDevice, c->stream));
+      XLOG_LAUNCH(c, (k_sort_pass<K, 8>), ntiles - 1, kSortBlock, sort_pass_smem<K>(), (const K*)keys, (const uint32_t*)payload, (K*)out_keys, (uint32_t*)out_payload,
+                  (uint32_t)n, 0, hist, hist + head_words, tickets, ctrl_u32(c, kSlotErr), c->spin_limit);
+    });
+    sync_ctrl(c);                          // raises INTERNAL when a wait gave up
   });
 }
 

@@ -33,7 +33,7 @@ PLAN_NONE, PLAN_WCOJ, PLAN_CHAIN = 0, 1, 2
 EXPORTS = ["xlog_ctx_create", "xlog_ctx_destroy", "xlog_last_error", "xlog_relation_create", "xlog_relation_load",
            "xlog_relation_size", "xlog_relation_read", "xlog_relation_view", "xlog_rule_add", "xlog_fixpoint",
            "xlog_ctx_reset_idb", "xlog_rule_backward", "xlog_profile_read", "xlog_profile_reset",
-           "xlog_reduce_by_key_static", "xlog_sort_pairs"]
+           "xlog_reduce_by_key_static", "xlog_sort_pairs", "xlog_debug_set_poll_limit", "xlog_debug_sort_pass_without_first_tile"]
 
 
 class XlogError(RuntimeError):
@@ -72,7 +72,7 @@ class Receipt(C.Structure):
                 ("derived_tuples", C.c_int64), ("candidates", C.c_int64), ("unique_candidates", C.c_int64),
                 ("new_tuples", C.c_int64), ("improved_tags", C.c_int64), ("h2d_bytes", C.c_int64),
                 ("d2h_bytes", C.c_int64), ("kernel_launches", C.c_int64), ("peak_arena_bytes", C.c_int64),
-                ("device_ms", C.c_double), ("triangle_plan", C.c_int32), ("reserved", C.c_int32)]
+                ("device_ms", C.c_double), ("triangle_plan", C.c_int32), ("index_builds", C.c_int32)]
 
     def as_dict(self) -> Dict[str, object]:
         return {k: getattr(self, k) for k, _ in self._fields_ if k != "struct_size"}
@@ -110,6 +110,8 @@ def lib():
         L.xlog_profile_read.argtypes = [vp, C.POINTER(KernelStat), i32, C.POINTER(i32)]
         L.xlog_profile_reset.argtypes = [vp]
         L.xlog_sort_pairs.argtypes = [vp, vp, vp, i64, i32, i32]
+        L.xlog_debug_set_poll_limit.argtypes = [vp, C.c_uint32]
+        L.xlog_debug_sort_pass_without_first_tile.argtypes = [vp, vp, vp, vp, vp, i64, i32]
         L.xlog_reduce_by_key_static.argtypes = [vp, i32, vp, vp, i64, vp, vp, C.POINTER(i64), C.c_char_p, C.c_size_t]
         for name in EXPORTS:
             if name != "xlog_last_error":
@@ -292,6 +294,15 @@ class Context:
         assert keys.is_contiguous() and payload.is_contiguous() and payload.element_size() == 4
         self._check(self._L.xlog_sort_pairs(self._h, keys.data_ptr(), payload.data_ptr(), keys.numel(),
                                             keys.element_size(), key_bits))
+
+    def debug_set_poll_limit(self, polls: int):
+        """Test hook: how many polls a look-back wait makes before it gives up (default 2^22)."""
+        self._check(self._L.xlog_debug_set_poll_limit(self._h, polls))
+
+    def debug_sort_pass_without_first_tile(self, keys, payload, out_keys, out_payload):
+        """Test hook: one sort pass whose first tile never runs; raises XlogError(INTERNAL) once the waits give up."""
+        self._check(self._L.xlog_debug_sort_pass_without_first_tile(self._h, keys.data_ptr(), payload.data_ptr(), out_keys.data_ptr(),
+                                                                    out_payload.data_ptr(), keys.numel(), keys.element_size()))
 
     def reset_idb(self):
         self._check(self._L.xlog_ctx_reset_idb(self._h))

@@ -338,22 +338,41 @@ def test_stratified_negation_matches_oracle():
     c2.close()
 
 
-def check_four_cycle(prog, what, **kw):
+def check_four_cycle(prog, what, expect_plan=None, **kw):
+    """Both plans of the four-cycle join (multiway step / binary-join chain) and the skew test's own choice against the
+    oracle: identical rows and tags on every path (the paper's gate for its WCOJ comparison)."""
     from paper_2609_27203_b200 import xlog
-    ctx, gids, _, o, oids, _, receipt = both(prog, **kw)
-    got, want = ctx.read(gids["c4"]), o.read(oids["c4"])
-    rep = H.compare_relations(got, want, what=what)
-    assert rep["bit_unequal"] == 0                # ((w_xy (x) w_yz) (x) w_zw) (x) w_wx in fp32 on both sides
-    assert receipt["derived_tuples"] == len(want[1]) and receipt["triangle_plan"] == xlog.PLAN_WCOJ
-    ctx.close()
+    o, oids, _ = oracle.load_program(prog)
+    o.run("naive")
+    want = o.read(oids["c4"])
+    chosen = None
+    for flags, plan in ((xlog.FLAG_FORCE_WCOJ, xlog.PLAN_WCOJ), (xlog.FLAG_FORCE_CHAIN, xlog.PLAN_CHAIN), (0, None)):
+        ctx, gids, _ = xlog.load_program(prog, **dict(dict(arena_bytes=1 << 30), **kw, flags=xlog.FLAG_CHECK_INVARIANTS | flags))
+        receipt = ctx.fixpoint()
+        rep = H.compare_relations(ctx.read(gids["c4"]), want, what=f"{what}, flags {flags}")
+        assert rep["bit_unequal"] == 0            # ((w_xy (x) w_yz) (x) w_zw) (x) w_wx in fp32 on every path
+        assert receipt["derived_tuples"] == len(want[1])
+        if plan is not None:
+            assert receipt["triangle_plan"] == plan
+        else:
+            chosen = receipt["triangle_plan"]
+        ctx.close()
+    assert chosen in (xlog.PLAN_WCOJ, xlog.PLAN_CHAIN)
+    if expect_plan is not None:
+        assert chosen == expect_plan, (what, chosen)
     return len(want[1])
 
 
 def test_four_cycle_join_matches_the_oracle():
     # dense small domain (every two-path has two long lists: the warp-cooperative walk), sparse (short lists: a thread
     # per two-path), sum-product tags, and a skewed graph used four times (hub two-paths next to empty ones)
-    assert check_four_cycle(W.uniform_four_cycle(3000, 70), "dense") > 100000
-    assert check_four_cycle(W.uniform_four_cycle(20000, 2500), "sparse") > 0
+    from paper_2609_27203_b200 import xlog
+    # 3000 rows over 70 values: 43 partners per value, 5.5 M three-paths against 3000 input rows -> the multiway step;
+    # 20000 rows over 2500 values: 8 partners per value, hence 8^2 three-paths per input row -> still the multiway step;
+    # 20000 rows over 12000 values: fewer than two partners per value -> the chain
+    assert check_four_cycle(W.uniform_four_cycle(3000, 70), "dense", xlog.PLAN_WCOJ) > 100000
+    assert check_four_cycle(W.uniform_four_cycle(20000, 2500), "sparse", xlog.PLAN_WCOJ) > 0
+    assert check_four_cycle(W.uniform_four_cycle(20000, 12000), "very sparse", xlog.PLAN_CHAIN) >= 0
     sp = W.uniform_four_cycle(2500, 90, W.SUMPROD)
     for name in ("r", "s", "t", "u"):
         (a, b), _ = sp.facts[name]

@@ -42,3 +42,39 @@ def test_sort_pairs_is_a_stable_sort_on_the_low_bits(n, bits, kb, skew):
     assert np.array_equal(dp.cpu().numpy(), payload[order])          # stable: ties keep input order
     assert np.array_equal(dk.cpu().numpy(), keys[order])
     ctx.close()
+
+
+def test_a_look_back_wait_that_runs_out_fails_the_call_and_leaves_the_context_usable():
+    # failure path of the bounded waits: one sort pass is launched without its first tile, so the status words every other
+    # tile looks back to stay empty; with a poll limit of a thousand each wait gives up within a millisecond or so
+    import time
+    import torch
+    from paper_2609_27203_b200 import xlog
+    n = 64 * 4096 + 777                                   # 65 tiles, the last one ragged
+    ctx = xlog.Context(arena_bytes=1 << 27)
+    ctx.debug_set_poll_limit(1000)
+    keys = torch.from_numpy(_keys(n, 20, 5, False).astype(np.int32)).cuda()
+    vals = torch.arange(n, dtype=torch.int32, device="cuda")
+    out_k = torch.full_like(keys, -7)
+    out_v = torch.full_like(vals, -9)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    with pytest.raises(xlog.XlogError) as e:
+        ctx.debug_sort_pass_without_first_tile(keys, vals, out_k, out_v)
+    dt = time.perf_counter() - t0
+    assert e.value.status == "INTERNAL"
+    assert dt < 1.0, dt                                   # the kernel gave up on its own, in milliseconds (first-launch overhead included)
+    assert bool((out_k == -7).all()) and bool((out_v == -9).all())          # no tile wrote anything
+    # the context still works: an ordinary sort of the same rows, then a fixpoint
+    k2, v2 = keys.clone(), vals.clone()
+    ctx.sort_pairs(k2, v2, 20)
+    order = np.argsort(keys.cpu().numpy(), kind="stable")
+    assert np.array_equal(k2.cpu().numpy(), keys.cpu().numpy()[order]) and np.array_equal(v2.cpu().numpy(), order.astype(np.int32))
+    ctx.reset_idb()
+    e_rel = ctx.relation(2, "minplus")
+    p_rel = ctx.relation(2, "minplus")
+    ctx.load(e_rel, [np.array([0, 1], np.int32), np.array([1, 2], np.int32)], np.array([1.0, 2.0], np.float32))
+    ctx.rule(p_rel, [(0, {0: 1}), (0, {1: 1})], [(e_rel, [("v", 0, 1, 0), ("v", 1, 1, 0)])])
+    ctx.rule(p_rel, [(0, {0: 1}), (0, {2: 1})], [(p_rel, [("v", 0, 1, 0), ("v", 1, 1, 0)]), (e_rel, [("v", 1, 1, 0), ("v", 2, 1, 0)])])
+    assert ctx.fixpoint()["derived_tuples"] == 3
+    ctx.close()

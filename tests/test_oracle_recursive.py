@@ -220,8 +220,11 @@ def test_typed_failures():
         with pytest.raises(oracle.OracleError) as e:
             o.run(mode, max_iterations=3)
         assert e.value.status == "CONVERGENCE_FAILURE"
-    # non-idempotent oplus inside a recursive component is rejected
-    o, ids, _r = oracle.load_program(W.closure_program([0, 1], [1, 2], None, W.LOGSUMEXP))
+    # a recursive component that mixes max/min relations with logsumexp relations is rejected
+    mixed = W.Program("mixed", {"e": (1, W.MAXPLUS), "a": (1, W.MAXPLUS), "b": (1, W.LOGSUMEXP)},
+                      [W.Rule("a", (W.V(0),), (W.Atom("e", (W.Var(0),)),)), W.Rule("a", (W.V(0),), (W.Atom("b", (W.Var(0),)),)),
+                       W.Rule("b", (W.V(0),), (W.Atom("a", (W.Var(0),)),))], {"e": ([np.array([1, 2], np.int32)], None)})
+    o, ids, _r = oracle.load_program(mixed)
     with pytest.raises(oracle.OracleError) as e:
         o.run("naive")
     assert e.value.status == "UNSUPPORTED"
