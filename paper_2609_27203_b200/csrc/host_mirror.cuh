@@ -1,0 +1,593 @@
+// Recursive components over a tag mirror: host-driven rounds, resident rounds (CUDA graph with a WHILE node), grouped and bitmap-driven joins.
+// Host-side driver code of the engine; included by xlog_api.cu only (one translation unit).
+#pragma once
+#include "host_eval.cuh"
+#include "bitmap_join.cuh"
+#include "group_join.cuh"
+#include "mirror.cuh"
+#include "resident.cuh"
+
+namespace xlog {
+namespace {
+
+constexpr int kSlotMirNew = 12, kSlotMirChanged = 13;
+constexpr int kMirrorMaxBits = 30;
+
+// The tag mirror serves a component of one max/min relation whose rules are all linear (at most one atom over the
+// relation itself, and that atom is the scanned side): then the relation is only ever read through its delta, and
+// its sorted form is needed again only after the last round.
+bool mirror_applies(Ctx* c, const std::vector<int>& comp, const std::vector<const RuleC*>& rs) {
+  if ((c->flags & XLOG_FLAG_NO_TAG_MIRROR) || comp.size() != 1) return false;
+  const Relation& H = *c->rels[comp[0]];
+  if (H.sr != XLOG_SR_MAXPLUS && H.sr != XLOG_SR_MINPLUS) return false;
+  if (H.layout.total_bits > kMirrorMaxBits || H.key_bytes != 4) return false;
+  for (const RuleC* r : rs) {
+    if (r->plan.emit_count_column || r->kind == 3 || r->kind == 4 || r->kind == 6) return false;
+    int in = 0, pos = 0;
+    for (int j = 0; j < r->plan.n_atoms; ++j)
+      if (r->plan.atoms[j].rel == comp[0]) { if (r->plan.atoms[j].negated) return false; ++in; pos = j; }
+    if (in > 1) return false;
+    if (in == 1 && r->kind == 2 && !r->shape[pos].ok) return false;
+    if (in == 1 && r->kind != 2 && pos != 0) return false;
+    if (in == 0 && r->kind == 2 && !r->shape[0].ok && !r->shape[1].ok) return false;
+  }
+  const uint64_t need = ((uint64_t)4 << H.layout.total_bits) + ((uint64_t)1 << H.layout.total_bits) / 4 + (1u << 20);
+  return need <= c->arena.largest_free() / 2;
+}
+
+// ---- resident rounds (resident.cuh) --------------------------------------------------------------------
+constexpr int kResidentMaxBits = 24;
+constexpr uint32_t kResidentMaxTiles = 1u << 20;
+
+ResState* res_state(Ctx* c) { return reinterpret_cast<ResState*>(c->d_ctrl + kSlotResState); }
+static_assert(sizeof(ResState) <= (kCtrlSlots - kSlotResState) * sizeof(uint64_t), "state block must fit the control words");
+
+// The persistent buffers of head relation h at their fixed capacities, or nullptr when the resident rounds do not
+// apply (domain too large for fixed-capacity buffers, not enough arena, or switched off).
+Resident* resident_for(Ctx* c, int h, int bits, uint64_t slots, uint32_t bm_quads, unsigned ch_tiles) {
+  if ((c->flags & XLOG_FLAG_NO_RESIDENT_LOOP) || bits > kResidentMaxBits) { c->resident.erase(h); return nullptr; }
+  uint32_t max_tiles = kResidentMaxTiles;
+  if (c->chunk_bytes) max_tiles = (uint32_t)std::max<uint64_t>(1, std::min<uint64_t>(max_tiles, c->chunk_bytes / 16 / kExpTileMirror));
+  auto it = c->resident.find(h);
+  if (it != c->resident.end() && it->second->slots == slots && it->second->max_tiles == max_tiles) return it->second.get();
+  c->resident.erase(h);
+  const uint64_t dom = (uint64_t)1 << bits;
+  const uint64_t need = slots * 4 + (uint64_t)bm_quads * 32 + dom * 32 + (uint64_t)max_tiles * 8 + (4u << 20);
+  if (need > c->arena.largest_free() / 3) return nullptr;
+  std::unique_ptr<Resident> R(new Resident());
+  R->slots = slots; R->max_tiles = max_tiles;
+  R->table = DevBuf(c, slots * 4);
+  R->bitmap = DevBuf(c, (size_t)bm_quads * 16);
+  R->present = DevBuf(c, (size_t)bm_quads * 16);
+  R->ch_sums = DevBuf(c, (size_t)ch_tiles * 4);
+  R->dkeys = DevBuf(c, dom * 4); R->dtags = DevBuf(c, dom * 4);
+  R->rowinfo = DevBuf(c, dom * 16); R->start = DevBuf(c, dom * 8);
+  R->scan_tiles_cap = (uint32_t)(dom / kResScanTile + 2);
+  R->scan_status = DevBuf(c, (size_t)kResMaxVariants * R->scan_tiles_cap * 8);
+  R->tickets = DevBuf(c, (kResMaxVariants + 2) * 4);
+  R->tile_rows = DevBuf(c, (size_t)max_tiles * 8);
+  Resident* out = R.get();
+  c->resident[h] = std::move(R);
+  return out;
+}
+
+// bitmap tiles: one sweep of 256 words per tile for domains up to 2^22 keys (so that small domains still give hundreds of
+// blocks), four sweeps above that
+int mirror_sweeps(uint32_t nwords) { return nwords <= (1u << 17) ? 1 : 4; }
+unsigned mirror_tiles(uint32_t nwords) { const uint32_t per = kMirBlock * mirror_sweeps(nwords); return (nwords + per - 1) / per; }
+void launch_changed_count(Ctx* c, const uint32_t* words, uint32_t* present, uint32_t nwords, unsigned tiles, uint32_t* sums, unsigned long long* new_total) {
+  if (mirror_sweeps(nwords) == 1) XLOG_LAUNCH(c, (k_mirror_changed_count<1>), tiles, kMirBlock, 0, words, present, nwords, sums, new_total);
+  else XLOG_LAUNCH(c, (k_mirror_changed_count<4>), tiles, kMirBlock, 0, words, present, nwords, sums, new_total);
+}
+void launch_changed_emit(Ctx* c, uint32_t* words, uint32_t nwords, unsigned tiles, const uint32_t* base, const int32_t* table, uint32_t* keys,
+                         float* tags, const uint32_t* skip) {
+  if (mirror_sweeps(nwords) == 1) XLOG_LAUNCH(c, (k_mirror_changed_emit<uint32_t, 1>), tiles, kMirBlock, 0, words, nwords, base, table, keys, tags, skip);
+  else XLOG_LAUNCH(c, (k_mirror_changed_emit<uint32_t, 4>), tiles, kMirBlock, 0, words, nwords, base, table, keys, tags, skip);
+}
+
+template <typename T> void sig_add(std::vector<char>& sig, const T& v) {
+  const char* p = reinterpret_cast<const char*>(&v);
+  sig.insert(sig.end(), p, p + sizeof(T));
+}
+
+// One round's launches.  Nothing here allocates, copies or waits: the same calls are either captured into the WHILE
+// body or issued directly (host-driven rounds, used when launches are being timed one by one).
+void resident_body(Ctx* c, Resident& R, const std::vector<JoinSpec>& specs, bool is_max, const MirrorArgs& mr, uint32_t bm_quads, unsigned ch_tiles,
+                   cudaGraphConditionalHandle handle, int use_handle) {
+  ResState* st = res_state(c);
+  uint32_t* err = ctrl_u32(c, kSlotErr);
+  const uint32_t* dk = R.dkeys.as<uint32_t>();
+  const ResScratch sc{R.scan_status.as<unsigned long long>(), R.scan_tiles_cap, R.tickets.as<uint32_t>()};
+  for (size_t v = 0; v < specs.size(); ++v) {
+    const JoinSpec& S = specs[v];
+    XLOG_LAUNCH(c, (k_res_count_scan<uint32_t>), kSMs * 4, kScanBlock, 0, S, dk, (const float*)R.dtags.as<float>(), st, R.rowinfo.as<uint4>(),
+                R.start.as<uint64_t>(), R.tile_rows.as<uint2>(), sc.scan_status + v * R.scan_tiles_cap, sc.tickets + v, err, c->spin_limit);
+// four waves of blocks: the hardware hands a new block to whichever SM finishes first, which evens out skewed tiles
+#define XLOG_RES_EXPAND(MODE, SINK)                                                                                                         \
+  XLOG_LAUNCH(c, (k_res_expand<uint32_t, MODE, SINK>), kSMs * kExpMirrorBlocksPerSM * 4, kExpBlock, 0, S, dk, (const ResState*)st, (const uint64_t*)R.start.as<uint64_t>(), \
+              (const uint4*)R.rowinfo.as<uint4>(), (const uint2*)R.tile_rows.as<uint2>(), err, mr)
+    if (S.fast) { if (is_max) XLOG_RES_EXPAND(kExpFast, kSinkMax); else XLOG_RES_EXPAND(kExpFast, kSinkMin); }
+    else { if (is_max) XLOG_RES_EXPAND(kExpGeneric, kSinkMax); else XLOG_RES_EXPAND(kExpGeneric, kSinkMin); }
+#undef XLOG_RES_EXPAND
+  }
+  uint32_t* ctr = sc.tickets + kResMaxVariants;
+#define XLOG_RES_EMIT(SW)                                                                                                                  \
+  XLOG_LAUNCH(c, (k_res_emit<SW>), ch_tiles, kMirBlock, 0, R.bitmap.as<uint32_t>(), R.present.as<uint32_t>(), bm_quads * 4, mr.n_new,        \
+              (const int32_t*)R.table.as<int32_t>(),                                                                                        \
+              R.dkeys.as<uint32_t>(), R.dtags.as<float>(), st, sc, (uint32_t)specs.size(), (const unsigned long long*)mr.n_new, ctr, handle, use_handle)
+  if (mirror_sweeps(bm_quads * 4) == 1) XLOG_RES_EMIT(1); else XLOG_RES_EMIT(4);
+#undef XLOG_RES_EMIT
+}
+
+// Run rounds on the device until the delta is empty, the round budget is used up or a round needs more tiles than
+// planned.  Returns the final state block (read once, after the loop).
+ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*>& rs, bool is_max, const MirrorArgs& mr_host, uint32_t bm_quads,
+                      unsigned ch_tiles, uint32_t n_delta, int64_t rounds_left, uint64_t new_seen) {
+  Relation& H = *c->rels[h];
+  std::vector<JoinSpec> specs;
+  for (const RuleC* r : rs)
+    for (int j = 0; j < r->plan.n_atoms; ++j)
+      if (r->plan.atoms[j].rel == h) {
+        const Variant v{r, j, Source{R.dkeys.p, R.dtags.as<float>(), n_delta, H.layout, H.key_bytes}};
+        specs.push_back(make_spec(c, v, H));              // builds the looked-up relation's index if it is missing
+      }
+  if (specs.size() > 16) fail(XLOG_ERR_UNSUPPORTED, "too many rule variants for one head");
+  const uint32_t budget = (uint32_t)std::min<int64_t>(rounds_left, 0x7fffffff);
+  const ResScratch sc{R.scan_status.as<unsigned long long>(), R.scan_tiles_cap, R.tickets.as<uint32_t>()};
+  XLOG_LAUNCH(c, k_res_init, 1, 1024, 0, res_state(c), sc, (uint32_t)specs.size(), n_delta, budget, R.max_tiles, (unsigned long long)new_seen);
+  const MirrorArgs& mr = mr_host;
+  const int64_t l0 = c->launches;
+  const bool use_graph = !(c->flags & (XLOG_FLAG_PROFILE | XLOG_FLAG_NO_GRAPH));
+  ResState out{};
+  auto read_state = [&]() {
+    sync_ctrl(c);
+    memcpy(&out, c->h_ctrl + kSlotResState, sizeof out);
+  };
+  if (use_graph) {
+    std::vector<char> sig;
+    for (const JoinSpec& S : specs) sig_add(sig, S);
+    sig_add(sig, mr.table); sig_add(sig, mr.changed); sig_add(sig, mr.n_new); sig_add(sig, mr.key_max); sig_add(sig, mr.err); sig_add(sig, R.present.p);
+    sig_add(sig, is_max); sig_add(sig, bm_quads); sig_add(sig, ch_tiles); sig_add(sig, c->d_ctrl); sig_add(sig, c->spin_limit);
+    if (!R.exec || sig != R.sig) {
+      if (R.exec) { cudaGraphExecDestroy(R.exec); R.exec = nullptr; }
+      if (R.graph) { cudaGraphDestroy(R.graph); R.graph = nullptr; }
+      XLOG_CUDA(cudaGraphCreate(&R.graph, 0));
+      cudaGraphConditionalHandle handle;
+      XLOG_CUDA(cudaGraphConditionalHandleCreate(&handle, R.graph, 1, cudaGraphCondAssignDefault));
+      cudaGraphNodeParams np = {};
+      np.type = cudaGraphNodeTypeConditional;
+      np.conditional.handle = handle;
+      np.conditional.type = cudaGraphCondTypeWhile;
+      np.conditional.size = 1;
+      cudaGraphNode_t node;
+      XLOG_CUDA(cudaGraphAddNode(&node, R.graph, nullptr, 0, &np));
+      cudaGraph_t body = np.conditional.phGraph_out[0];
+      // the body is recorded on a stream of the context's own (the caller's stream may be the legacy default stream,
+      // which cannot capture); the instantiated graph is launched on the caller's stream like everything else
+      if (!c->capture_stream) XLOG_CUDA(cudaStreamCreateWithFlags(&c->capture_stream, cudaStreamNonBlocking));
+      XLOG_CUDA(cudaStreamBeginCaptureToGraph(c->capture_stream, body, nullptr, nullptr, 0, cudaStreamCaptureModeThreadLocal));
+      cudaStream_t caller = c->stream;
+      c->stream = c->capture_stream;
+      const int64_t b0 = c->launches;
+      try {
+        resident_body(c, R, specs, is_max, mr, bm_quads, ch_tiles, handle, 1);
+      } catch (...) {
+        c->stream = caller;
+        cudaGraph_t dummy = nullptr;
+        cudaStreamEndCapture(c->capture_stream, &dummy);
+        throw;
+      }
+      c->stream = caller;
+      R.body_launches = c->launches - b0;
+      XLOG_CUDA(cudaStreamEndCapture(c->capture_stream, nullptr));
+      XLOG_CUDA(cudaGraphInstantiate(&R.exec, R.graph, 0));
+      R.sig = std::move(sig);
+    }
+    XLOG_CUDA(cudaGraphLaunch(R.exec, c->stream));
+    read_state();
+    c->launches = l0 + R.body_launches * (int64_t)out.rounds + (out.status == kResOverflow ? R.body_launches : 0);
+  } else {
+    unsigned long long seen = 0;
+    uint32_t rows = n_delta;
+    double expand_ms_seen = 0.0;
+    int64_t expand_launches_seen = 0;
+    {
+      auto it0 = c->prof_index.find("k_res_expand");
+      if (it0 != c->prof_index.end()) { expand_ms_seen = c->prof[it0->second].ms; expand_launches_seen = c->prof[it0->second].launches; }
+    }
+    for (;;) {
+      resident_body(c, R, specs, is_max, mr, bm_quads, ch_tiles, cudaGraphConditionalHandle{}, 0);
+      read_state();
+      if (c->flags & XLOG_FLAG_PROFILE) {
+        // per delta row and rule: key and tag read, two offsets probed, 16-byte row record and 8-byte start offset written
+        auto cs = c->prof_index.find("k_res_count_scan");
+        if (cs != c->prof_index.end()) c->prof[cs->second].bytes += (int64_t)rows * 40 * (int64_t)specs.size();
+        rows = out.n_delta;
+        // algorithmic bytes of the round's expand launches (per candidate: the looked-up columns and tag, and the slot)
+        auto it = c->prof_index.find("k_res_expand");
+        if (it != c->prof_index.end()) {
+          const int64_t bytes = (int64_t)(out.candidates - seen) * (4 + (specs[0].has_inner ? 4 * (specs[0].inner_free + 1) : 0));
+          Ctx::ProfEntry& pe = c->prof[it->second];
+          pe.bytes += bytes;
+          if (bytes >= kProfLargeBytes) {                // this round's launches, totalled on their own like any large launch
+            const double round_ms = pe.ms - expand_ms_seen;
+            const int64_t round_launches = pe.launches - expand_launches_seen;
+            auto bt = c->prof_index.find("k_res_expand (large)");
+            if (bt == c->prof_index.end()) {
+              bt = c->prof_index.emplace("k_res_expand (large)", (int)c->prof.size()).first;
+              c->prof.push_back(Ctx::ProfEntry{"k_res_expand (large)", 0, 0.0, 0});
+            }
+            Ctx::ProfEntry& be = c->prof[bt->second];
+            be.ms += round_ms; be.launches += round_launches; be.bytes += bytes;
+          }
+          expand_ms_seen = c->prof[it->second].ms; expand_launches_seen = c->prof[it->second].launches;
+        }
+        seen = out.candidates;
+      }
+      if (out.status != kResOk || out.n_delta == 0) break;
+    }
+  }
+  return out;
+}
+
+// ---- grouped join (group_join.cuh) -----------------------------------------------------------------------
+// The shape  h(a, c) :- h(a, b), r(b, c)  for every rule over h (binary h; a and b bare variables; c the looked-up
+// relation's other column).
+bool grouped_shape(Ctx* c, int h, const std::vector<const RuleC*>& rs) {
+  const Relation& H = *c->rels[h];
+  if (H.arity != 2) return false;
+  bool any = false;
+  for (const RuleC* r : rs) {
+    int j = -1;
+    for (int k = 0; k < r->plan.n_atoms; ++k) if (r->plan.atoms[k].rel == h) j = k;
+    if (j < 0) continue;
+    if (r->kind != 2 || !r->shape[j].ok) return false;
+    const xlog_plan& p = r->plan;
+    const xlog_atom& A = p.atoms[j];
+    const xlog_atom& B = p.atoms[1 - j];
+    if (!is_plain_var(A.args[0]) || !is_plain_var(A.args[1]) || A.args[0].var == A.args[1].var) return false;
+    if (c->rels[B.rel]->arity != 2 || r->shape[j].probe_col != 0 || r->shape[j].probe_var != A.args[1].var || r->shape[j].probe_mul != 1 ||
+        r->shape[j].probe_add != 0 || !is_plain_var(B.args[1]))
+      return false;
+    const int hv[2] = {A.args[0].var, B.args[1].var};
+    for (int col = 0; col < 2; ++col) {
+      if (p.head[col].c0 != 0) return false;
+      for (int v = 0; v < XLOG_MAX_VARS; ++v) if (p.head[col].coef[v] != (v == hv[col] ? 1 : 0)) return false;
+    }
+    any = true;
+  }
+  return any;
+}
+
+constexpr int kSlotSeg = 80;               // grouped join: segments, candidates, work items, neighbour rows read
+
+// One delta variant through the grouped join.  Returns the candidate total, or UINT64_MAX when the compiled rule turns
+// out not to have the linear-key form (the caller then takes the row-wise join).
+uint64_t grouped_apply(Ctx* c, const Variant& v, const Relation& H, const KeyLayout& M, int carried_bits, bool is_max, const MirrorArgs& mr) {
+  const JoinSpec S = make_spec(c, v, H, &M);
+  if (!S.fast || !S.has_inner || S.inner_free != 1 || v.outer.key_bytes != 4) return UINT64_MAX;
+  const uint32_t n = v.outer.n;
+  const unsigned tiles = (n + kScanTile - 1) / kScanTile;
+  DevBuf deg(c, (size_t)n * 4), rowinfo(c, (size_t)n * 16), flags(c, (size_t)n * 4), idx(c, (size_t)n * 4), sums(c, (size_t)tiles * 4);
+  zero_ctrl(c, kSlotSeg, 4);
+  XLOG_LAUNCH(c, (k_join_count_flags<uint32_t>), grid_for(n, 256, kSMs * 32), 256, 0, S, (const uint32_t*)v.outer.keys, v.outer.tags, n, carried_bits, deg.as<uint32_t>(),
+              rowinfo.as<uint4>(), flags.as<uint32_t>(), (unsigned long long*)(c->d_ctrl + kSlotSeg + 1), ctrl_u32(c, kSlotErr));
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), tiles, kScanBlock, 0, (const uint32_t*)flags.as<uint32_t>(), (int64_t)n, sums.as<uint32_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, sums.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotSeg));
+  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), tiles, kScanBlock, 0, (const uint32_t*)flags.as<uint32_t>(), (int64_t)n,
+              (const uint32_t*)sums.as<uint32_t>(), idx.as<uint32_t>());
+  sync_ctrl(c);
+  const uint32_t n_seg = (uint32_t)c->h_ctrl[kSlotSeg];
+  const uint64_t total = c->h_ctrl[kSlotSeg + 1];
+  if (total == 0) return 0;
+  if (total / n_seg < 128) return UINT64_MAX;            // small segments: the row-wise join does as well, with fewer passes
+  const uint32_t ns1 = n_seg + 1;
+  DevBuf seg_first(c, (size_t)ns1 * 4);
+  XLOG_LAUNCH(c, k_seg_first, grid_for((uint64_t)n + 1, 256), 256, 0, (const uint32_t*)flags.as<uint32_t>(), (const uint32_t*)idx.as<uint32_t>(), n, n_seg,
+              seg_first.as<uint32_t>());
+  flags.reset(); idx.reset(); sums.reset();
+  const unsigned ittiles = (ns1 + kScanTile - 1) / kScanTile;
+  DevBuf items(c, (size_t)ns1 * 4), item_off(c, (size_t)ns1 * 4), itsums(c, (size_t)ittiles * 4);
+  XLOG_LAUNCH(c, k_seg_items, grid_for(ns1, 256, kSMs * 16), 256, 0, (const uint32_t*)seg_first.as<uint32_t>(), n_seg, (const uint32_t*)deg.as<uint32_t>(), items.as<uint32_t>(),
+              (unsigned long long*)(c->d_ctrl + kSlotSeg + 3));
+  XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), ittiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ns1, itsums.as<uint32_t>());
+  XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, itsums.as<uint32_t>(), (int64_t)ittiles, ctrl_u32(c, kSlotSeg + 2));
+  XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), ittiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ns1,
+              (const uint32_t*)itsums.as<uint32_t>(), item_off.as<uint32_t>());
+  sync_ctrl(c);
+  const uint32_t n_items = (uint32_t)c->h_ctrl[kSlotSeg + 2];
+  items.reset(); itsums.reset();
+  DevBuf item_seg(c, (size_t)std::max(n_items, 1u) * 4);
+  XLOG_LAUNCH(c, k_seg_item_fill, grid_for(n_seg, 256), 256, 0, n_seg, (const uint32_t*)item_off.as<uint32_t>(), item_seg.as<uint32_t>());
+  // per candidate: its slot; per segment and neighbour: the looked-up column and tag, read once for all the segment's rows;
+  // per delta row: its count record
+  c->note_bytes = (int64_t)total * 4 + (int64_t)c->h_ctrl[kSlotSeg + 3] * 8 + (int64_t)n * 16;
+  const unsigned grid = (unsigned)std::min<uint64_t>(((uint64_t)n_items + 7) / 8, (uint64_t)kSMs * 8 * 16);
+  if (is_max)
+    XLOG_LAUNCH(c, (k_seg_expand<kSinkMax>), grid, 256, 0, S, n_items, (const uint32_t*)item_off.as<uint32_t>(), (const uint32_t*)item_seg.as<uint32_t>(),
+                (const uint32_t*)seg_first.as<uint32_t>(), (const uint32_t*)deg.as<uint32_t>(), (const uint4*)rowinfo.as<uint4>(), mr);
+  else
+    XLOG_LAUNCH(c, (k_seg_expand<kSinkMin>), grid, 256, 0, S, n_items, (const uint32_t*)item_off.as<uint32_t>(), (const uint32_t*)item_seg.as<uint32_t>(),
+                (const uint32_t*)seg_first.as<uint32_t>(), (const uint32_t*)deg.as<uint32_t>(), (const uint4*)rowinfo.as<uint4>(), mr);
+  return total;
+}
+
+constexpr int kSlotBm = 84;                // bitmap-driven grouped join: the kBmTotals counters of k_bm_plan
+static_assert(kSlotBm + kBmTotals <= kCtrlSlots, "control block too small");
+
+// What the bitmap-driven grouped join (bitmap_join.cuh) needs beyond the mirror itself; valid == false: not applicable.
+struct BitmapJoin {
+  bool valid = false;
+  JoinSpec spec;
+  DevBuf pairs, items;
+  int carried_bits = 0;
+};
+
+// Applicable when exactly one rule has an atom over h (so a round is one join), that rule has the grouped shape with the
+// linear-key form, a value of the probed column owns 1 to 32 whole bitmap words, and the pair list and the item list
+// (sized for every key changing in one round) fit the arena.
+void bitmap_join_setup(Ctx* c, int h, const std::vector<const RuleC*>& rs, const KeyLayout& M, int carried_bits, uint64_t slots, BitmapJoin& bj) {
+  if ((c->flags & XLOG_FLAG_NO_BITMAP_JOIN) || carried_bits < 5 || carried_bits > 5 + kBmMaxWordsLog2) return;
+  Relation& H = *c->rels[h];
+  if (H.dict_n[1]) return;
+  const RuleC* rule = nullptr; int pos = -1, n_over = 0;
+  for (const RuleC* r : rs)
+    for (int j = 0; j < r->plan.n_atoms; ++j)
+      if (r->plan.atoms[j].rel == h) { ++n_over; rule = r; pos = j; }
+  if (n_over != 1) return;
+  const Variant v{rule, pos, Source{nullptr, nullptr, 0, M, H.key_bytes}};
+  const JoinSpec S = make_spec(c, v, H, &M);               // builds the looked-up relation's index if it is missing
+  if (!S.fast || !S.has_inner || S.inner_free != 1 || S.outer_decode[0] || S.outer_decode[1] || S.head_encode[0] || S.head_encode[1] ||
+      S.inner_mult[0] != ((uint64_t)1 << carried_bits))
+    return;
+  const Relation& RB = *c->rels[rule->plan.atoms[1 - pos].rel];
+  const uint64_t passes = (uint64_t)1 << (carried_bits - 5);             // at most one pass per 32 carried values
+  const uint64_t values = std::min<uint64_t>((uint64_t)S.inner_domain, slots >> carried_bits);
+  const uint64_t max_items = ((uint64_t)RB.n / kBmSlice + values + 1) * passes;
+  if (max_items >= ((uint64_t)1 << 32)) return;
+  const uint64_t need = slots * 8 + max_items * 16 + (1u << 20);          // a round can change every key: one (tag, carried value) pair each
+  if (need > c->arena.largest_free() / 2) return;
+  bj.pairs = DevBuf(c, slots * 8);
+  bj.items = DevBuf(c, max_items * 16);
+  bj.spec = S;
+  bj.carried_bits = carried_bits;
+  bj.valid = true;
+}
+
+// Algorithm 1 over a tag mirror (mirror.cuh): per round  count -> scan -> join straight into the table -> compact the
+// changed bitmap into the next delta.  No candidate is ever written to memory.  The seed round is driven by the host
+// (its rules scan whole relations of known size); the delta rounds run resident where the fixed-capacity buffers fit.
+void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs) {
+  Relation& H = *c->rels[h];
+  const std::vector<int> comp{h};
+  const int bits = H.layout.total_bits;
+  const uint64_t dom = (uint64_t)1 << bits;
+  const bool is_max = H.sr == XLOG_SR_MAXPLUS;
+  const int32_t empty = is_max ? kMirrorEmptyMax : kMirrorEmptyMin;
+  const uint64_t slots = std::max<uint64_t>(dom, 4);
+  const uint32_t bm_quads = (uint32_t)((std::max<uint64_t>(dom / 32, 1) + 3) / 4);
+  const unsigned ch_tiles = mirror_tiles(bm_quads * 4);
+  Resident* R = resident_for(c, h, bits, slots, bm_quads, ch_tiles);
+  // the mirror's own column order: for the grouped join the probed column is the major part of the index (group_join.cuh)
+  KeyLayout M = H.layout;
+  const bool grouped = !R && !(c->flags & XLOG_FLAG_NO_GROUPED_JOIN) && grouped_shape(c, h, rs);
+  int carried_bits = 0;
+  if (grouped) {
+    carried_bits = bits - H.layout.shift[0];             // width of column 0
+    M.shift[0] = 0;
+    M.shift[1] = carried_bits;
+  }
+  const KeyLayout* ML = grouped ? &M : nullptr;
+  DevBuf table_own, bitmap_own, present_own, ch_sums_own;
+  if (!R) {
+    table_own = DevBuf(c, slots * 4); bitmap_own = DevBuf(c, (size_t)bm_quads * 16); present_own = DevBuf(c, (size_t)bm_quads * 16);
+    ch_sums_own = DevBuf(c, (size_t)ch_tiles * 4);
+  }
+  BitmapJoin bj;
+  if (grouped) bitmap_join_setup(c, h, rs, M, carried_bits, slots, bj);
+  uint32_t* present = R ? R->present.as<uint32_t>() : present_own.as<uint32_t>();
+  int32_t* table = R ? R->table.as<int32_t>() : table_own.as<int32_t>();
+  uint4* bitmap = R ? R->bitmap.as<uint4>() : bitmap_own.as<uint4>();
+  uint32_t* ch_sums = R ? R->ch_sums.as<uint32_t>() : ch_sums_own.as<uint32_t>();
+  XLOG_LAUNCH(c, k_fill_i32, grid_for(slots, 256 * 8), 256, 0, table, slots, empty);
+  XLOG_CUDA(cudaMemsetAsync(bitmap, 0, (size_t)bm_quads * 16, c->stream));
+  XLOG_CUDA(cudaMemsetAsync(present, 0, (size_t)bm_quads * 16, c->stream));
+  // what the relation holds now (its loaded facts, or the result of an earlier fixpoint) is the starting state
+  const uint32_t n_start = H.n;
+  if (n_start)
+    XLOG_LAUNCH(c, (k_mirror_scatter<uint32_t>), grid_for(n_start, 256, 1 << 30), 256, 0, (const uint32_t*)H.keys(), (const float*)H.tags(), n_start, H.layout, M, table, present);
+  zero_ctrl(c, kSlotMirNew, 2);
+  const MirrorArgs mr{table, reinterpret_cast<uint32_t*>(bitmap), (unsigned long long*)(c->d_ctrl + kSlotMirNew), (uint32_t)(dom - 1),
+                      ctrl_u32(c, kSlotErr)};
+  c->unique_untracked = true;
+  KeyTags delta_own;                       // host-driven rounds without persistent buffers keep their delta here
+  const void* dk = nullptr; const float* dt = nullptr; uint32_t dn = 0;
+  uint64_t total_new = 0;
+  // count -> scan -> one control read -> join into the table, for a list of rule variants; returns the candidate total
+  auto host_apply = [&](std::vector<Variant>& vs) -> uint64_t {
+    if (vs.size() > 16) fail(XLOG_ERR_UNSUPPORTED, "too many rule variants for one head");
+    std::vector<Counted> counted;
+    counted.reserve(vs.size());
+    uint64_t total = 0;
+    for (Variant& v : vs) {
+      if (v.outer.n == 0) continue;
+      if (grouped && v.outer.keys == dk && v.rule->plan.atoms[v.outer_atom].rel == h) {
+        // a delta variant of the grouped shape: the delta is ordered by the probed column
+        const uint64_t t = grouped_apply(c, v, H, M, carried_bits, is_max, mr);
+        if (t != UINT64_MAX) { total += t; c->r_candidates += (int64_t)t; continue; }
+      }
+      counted.emplace_back();
+      count_variant(c, v, H, counted.back(), kSlotTotals + (int)counted.size() - 1, ML);
+    }
+    if (!counted.empty()) {
+      sync_ctrl(c);
+      for (Counted& q : counted) { q.total = c->h_ctrl[q.slot]; total += q.total; q.deg.reset(); q.sums.reset(); }
+    }
+    for (Counted& q : counted) c->r_candidates += (int64_t)q.total;
+    for (Counted& q : counted) {
+      if (q.total) {
+        // per candidate: the looked-up atom's other columns and tag are read, and the key's slot is read (and now and then written)
+        c->note_bytes = (int64_t)q.total * (4 + (q.spec.has_inner ? 4 * (q.spec.inner_free + 1) : 0));
+        launch_expand_mirror(c, q, is_max, mr);
+      }
+      q.start.reset(); q.rowinfo.reset();
+    }
+    return total;
+  };
+  auto over_h = [&](const RuleC* r) {
+    for (int j = 0; j < r->plan.n_atoms; ++j) if (r->plan.atoms[j].rel == h) return true;
+    return false;
+  };
+
+  int64_t round = 0;
+  bool plain_rules_done = false;           // the rules without an atom over H have had their one evaluation
+  bool converged = false;
+  if (R) {
+    // Resident route.  Seed round, part one: rules without an atom over H are evaluated once, by the host (they scan whole
+    // relations of known size).  Part two and every later round run on the device: for the rules over H the seed round
+    // is a delta round whose delta is everything H holds now.
+    std::vector<Variant> plain;
+    for (const RuleC* r : rs)
+      if (!over_h(r)) { const int outer = seed_outer(comp, r); plain.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])}); }
+    host_apply(plain);
+    plain_rules_done = true;
+    if (n_start) {
+      XLOG_CUDA(cudaMemcpyAsync(R->dkeys.p, H.keys(), (size_t)n_start * 4, cudaMemcpyDeviceToDevice, c->stream));
+      XLOG_CUDA(cudaMemcpyAsync(R->dtags.p, H.tags(), (size_t)n_start * 4, cudaMemcpyDeviceToDevice, c->stream));
+    }
+    const ResState s = run_resident(c, *R, h, rs, is_max, mr, bm_quads, ch_tiles, n_start, c->max_iter, 0);
+    round = s.rounds;
+    c->r_iterations += s.rounds; c->r_candidates += (int64_t)s.candidates;
+    c->r_new += (int64_t)s.n_new; c->r_improved += (int64_t)s.n_improved;
+    total_new = s.new_seen;
+    dk = R->dkeys.p; dt = R->dtags.as<float>(); dn = s.n_delta;
+    if (s.status == kResCap) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
+    if (s.status == kResOk) converged = true;             // the delta ran empty
+    // kResOverflow: a round needs more expand tiles than planned; the host redoes that round and finishes the job
+  }
+  for (; !converged; ++round) {
+    if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
+    ++c->r_iterations;
+    std::vector<Variant> vs;
+    for (const RuleC* r : rs) {
+      if (round == 0) {
+        if (plain_rules_done && !over_h(r)) continue;
+        const int outer = seed_outer(comp, r);
+        vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
+      } else {
+        for (int j = 0; j < r->plan.n_atoms; ++j)
+          if (r->plan.atoms[j].rel == h && dn) vs.push_back(Variant{r, j, Source{dk, dt, dn, M, H.key_bytes}});
+      }
+    }
+    const uint64_t total = host_apply(vs);
+    if (total == 0 && !(round == 0 && plain_rules_done)) break;
+    if (bj.valid) {
+      // Every later round is  k_bm_plan -> one control read -> k_bm_expand : the plan kernel closes the round just joined
+      // (changed / new keys, bitmap cleared, the changed keys' tags set aside) and lays out the next one's work items.
+      const uint32_t nwords = bm_quads * 4;
+      BmPlan P{reinterpret_cast<uint32_t*>(bitmap), present, nwords, table, bj.pairs.as<uint2>(), carried_bits - 5, bj.spec.inner_off,
+               (uint32_t)std::min<int64_t>(bj.spec.inner_domain, 0xffffffffll), bj.items.as<uint4>(), (unsigned long long*)(c->d_ctrl + kSlotBm)};
+      BmExpand E{bj.items.as<uint4>(), 0, bj.spec.inner_col[0], bj.spec.inner_tag, H.layout.mask[1], carried_bits,
+                 bj.pairs.as<uint2>(), table, reinterpret_cast<uint32_t*>(bitmap), ctrl_u32(c, kSlotErr)};
+      for (;;) {
+        zero_ctrl(c, kSlotBm, kBmTotals);
+        c->note_bytes = (int64_t)nwords * 4;              // plus 12 bytes per changed key and 16 per item, not known yet
+        XLOG_LAUNCH(c, k_bm_plan, (nwords + kBmPlanTile - 1) / kBmPlanTile, kBmPlanBlock, 0, P);
+        sync_ctrl(c);
+        const uint64_t changed = c->h_ctrl[kSlotBm + kBmChanged], n_new = c->h_ctrl[kSlotBm + kBmNew], cand = c->h_ctrl[kSlotBm + kBmCandidates];
+        const uint64_t n_items = c->h_ctrl[kSlotBm + kBmReserve] >> 32, nbrs = c->h_ctrl[kSlotBm + kBmNeighbours];
+        total_new += n_new;
+        c->r_new += (int64_t)n_new; c->r_improved += (int64_t)changed - (int64_t)n_new;
+        if (changed == 0) break;
+        ++round;
+        if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
+        ++c->r_iterations;
+        if (cand == 0) break;
+        c->r_candidates += (int64_t)cand;
+        E.n_items = (uint32_t)n_items;
+        // per candidate its slot; per (b, neighbour) the looked-up column and tag; per item its record; per changed key its pair
+        c->note_bytes = (int64_t)cand * 4 + (int64_t)nbrs * 8 + (int64_t)n_items * 16 + (int64_t)changed * 8;
+        const unsigned grid = (unsigned)std::min<uint64_t>((n_items + 7) / 8, (uint64_t)kSMs * 8 * 16);
+        if (is_max) XLOG_LAUNCH(c, (k_bm_expand<kSinkMax>), grid, 256, 0, E);
+        else XLOG_LAUNCH(c, (k_bm_expand<kSinkMin>), grid, 256, 0, E);
+      }
+      break;
+    }
+    launch_changed_count(c, reinterpret_cast<const uint32_t*>(bitmap), present, bm_quads * 4, ch_tiles, ch_sums, mr.n_new);
+    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, ch_sums, (int64_t)ch_tiles, ctrl_u32(c, kSlotMirChanged));
+    sync_ctrl(c);
+    const uint32_t changed = (uint32_t)c->h_ctrl[kSlotMirChanged];
+    const uint64_t n_new = c->h_ctrl[kSlotMirNew] - total_new;
+    total_new += n_new;
+    c->r_new += (int64_t)n_new; c->r_improved += (int64_t)changed - (int64_t)n_new;
+    if (changed == 0) break;
+    uint32_t* ek; float* et;
+    if (R) { ek = R->dkeys.as<uint32_t>(); et = R->dtags.as<float>(); }
+    else {
+      delta_own = KeyTags();
+      delta_own.keys = DevBuf(c, (size_t)changed * 4);
+      delta_own.tags = DevBuf(c, (size_t)changed * 4);
+      ek = delta_own.keys.as<uint32_t>(); et = delta_own.tags.as<float>();
+    }
+    c->note_bytes = (int64_t)bm_quads * 16 + (int64_t)changed * 12;
+    launch_changed_emit(c, reinterpret_cast<uint32_t*>(bitmap), bm_quads * 4, ch_tiles, ch_sums, table, ek, et, nullptr);
+    dk = ek; dt = et; dn = changed;
+  }
+  // the relation in sorted form: every occupied slot, in slot order
+  const uint64_t n_out = (uint64_t)n_start + total_new;
+  KeyTags full;
+  full.n = (uint32_t)n_out;
+  full.keys = DevBuf(c, (size_t)std::max<uint64_t>(n_out, 1) * 4);
+  full.tags = DevBuf(c, (size_t)std::max<uint64_t>(n_out, 1) * 4);
+  bool counted_slots = false;              // kSlotA holds the number of occupied slots (for the invariant check)
+  if (n_out && grouped && carried_bits <= 6) {
+    // the mirror is ordered (column 1, column 0) and column 0 has at most 64 values: every row goes straight to its place
+    // in the relation's order (mirror.cuh), found from the bitmap of present keys; no pass over empty slots, no sort
+    const int per_node = 1 << carried_bits;
+    const uint32_t n_nodes = (uint32_t)(slots >> carried_bits);
+    const uint32_t ntiles = (n_nodes + kMtNodes - 1) / kMtNodes;
+    const int64_t len = (int64_t)per_node * ntiles;
+    const unsigned stiles = (unsigned)((len + kScanTile - 1) / kScanTile);
+    DevBuf cnt(c, (size_t)len * 4), base(c, (size_t)len * 4), sums(c, (size_t)stiles * 4);
+    c->note_bytes = (int64_t)slots / 8;
+    XLOG_LAUNCH(c, k_mirror_t_count, ntiles, kMtNodes, 0, (const uint32_t*)present, n_nodes, ntiles, per_node, cnt.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), stiles, kScanBlock, 0, (const uint32_t*)cnt.as<uint32_t>(), len, sums.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, sums.as<uint32_t>(), (int64_t)stiles, ctrl_u32(c, kSlotA));
+    XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), stiles, kScanBlock, 0, (const uint32_t*)cnt.as<uint32_t>(), len, (const uint32_t*)sums.as<uint32_t>(),
+                base.as<uint32_t>());
+    c->note_bytes = (int64_t)slots / 8 + (int64_t)n_out * 12;
+    XLOG_LAUNCH(c, (k_mirror_t_emit<uint32_t>), ntiles, kMtNodes, 0, (const uint32_t*)present, (const int32_t*)table, n_nodes, ntiles, per_node,
+                (const uint32_t*)base.as<uint32_t>(), H.layout.shift[0], H.layout.shift[1], full.keys.as<uint32_t>(), full.tags.as<float>());
+    counted_slots = true;
+  } else if (n_out) {
+    const uint64_t nquads = slots / 4;
+    const unsigned tiles = (unsigned)((slots + kMirSlotsPerTile - 1) / kMirSlotsPerTile);
+    DevBuf sums(c, (size_t)tiles * 4);
+    c->note_bytes = (int64_t)slots * 4;
+    XLOG_LAUNCH(c, k_mirror_full_count, tiles, kMirBlock, 0, (const int4*)table, nquads, empty, sums.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, sums.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotA));
+    c->note_bytes = (int64_t)slots * 4 + (int64_t)n_out * 8;
+    XLOG_LAUNCH(c, (k_mirror_full_emit<uint32_t>), tiles, kMirBlock, 0, (const int4*)table, nquads, empty, (const uint32_t*)sums.as<uint32_t>(), M, H.layout,
+                full.keys.as<uint32_t>(), full.tags.as<float>());
+    counted_slots = true;
+    if (grouped && n_out > 1) {
+      // rows came out in the mirror's order, (column 1, column 0) ascending: a stable sort on column 0's bits alone puts
+      // them in the relation's key order
+      table_own.reset(); bitmap_own.reset(); present_own.reset(); bj.pairs.reset(); bj.items.reset();
+      DevBuf ak(c, (size_t)n_out * 4), at(c, (size_t)n_out * 4);
+      uint32_t* pk = full.keys.as<uint32_t>(); uint32_t* qk = ak.as<uint32_t>();
+      float* pt = full.tags.as<float>(); float* qt = at.as<float>();
+      sort_pairs<uint32_t>(c, pk, pt, qk, qt, n_out, bits, H.layout.shift[0]);
+      if ((void*)pk != full.keys.p) { std::swap(full.keys, ak); std::swap(full.tags, at); }
+    }
+  }
+  set_current(H, std::move(full));
+  if (c->flags & XLOG_FLAG_CHECK_INVARIANTS) {
+    XLOG_LAUNCH(c, (k_check_sorted<uint32_t>), grid_for(H.n, 256), 256, 0, (const uint32_t*)H.keys(), (int64_t)H.n, ctrl_u32(c, kSlotErr));
+    sync_ctrl(c);
+    if (n_out && counted_slots && (uint64_t)(uint32_t)c->h_ctrl[kSlotA] != n_out) fail(XLOG_ERR_INTERNAL, "tag mirror: occupied slots disagree with the tuple count");
+  }
+}
+
+}  // namespace
+}  // namespace xlog
