@@ -74,6 +74,11 @@ def make_program(name: str, scale: int | None, sources: int | None = None):
         return W.uniform_four_cycle(n_rows=1 << s, domain=int(4 * 2 ** (s / 2))), 4 << 30
     if name == "digits":
         return W.config4(), 1 << 30
+    if name == "nonlinear":
+        # path doubling p(x,z) :- p(x,y), p(y,z): on configuration 1's graph, or (--scale) on a small R-MAT graph
+        return (W.nonlinear_rmat_config(scale) if scale else W.nonlinear_config()), 24 << 30
+    if name == "mutual":
+        return W.mutual_config(), 2 << 30
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -219,18 +224,15 @@ def roofline_of(program, prof_all, steps, sorting_route):
     mirror_kernel = dom in MIRROR_JOIN_KERNELS or (dom == "k_join_expand" and not sorting_route and "k_sort_pass" not in prof)
     ratio = traffic_ratios().get((dom, "mirror" if mirror_kernel else "sorting"))
     bound = "hbm"
-    alu = None
-    if dom.startswith("k_tri"):
-        bound = "alu"      # sorted-list intersections served from L1 / L2: compare and branch work, not an HBM-bound kernel
-        # unit of work: one probe (binary search of a walked entry in the other sorted list).  ncu: 6.5 warp instructions per probe at
-        # R-MAT scale 18, so the issue-rate ceiling is 148 SMs x 4 schedulers x 1.965e9 / 6.5 probes per second.
-        if dom == "k_tri_edges" and "n_edges" in program.info:
-            probes = (d["bytes"] - 12.0 * program.info["n_edges"] * d["launches"]) / 4.0
-            alu = {"achieved": probes / (d["ms"] / 1e3) / 1e9, "peak": 148 * 4 * 1.965 / 6.5, "unit": "Gprobe/s"}
+    l2 = None
+    probes = None
+    if dom == "k_tri_edges" and "n_edges" in program.info:
+        # sorted-list intersections served from L1 / L2 (both orientations of the graph fit L2): unit of work = one probe, a binary
+        # search of one walked entry in the other sorted list; the launch site declares 4 bytes per probe plus 12 per edge
+        probes = (d["bytes"] - 12.0 * program.info["n_edges"] * d["launches"]) / 4.0
     if dom in ("k_cycle4", "k_cycle4_bitmap") and program.info.get("domain", 1 << 30) <= 4096:
-        bound = "alu"      # sorted-list intersections served from L1 / L2 (DRAM 1 % busy under ncu), as for the triangles
-        # unit of work: one probe = one walked entry of the shorter list, searched in the other list; both launches (count, write)
-        # walk every two-path's list.  ncu at scale 16: 2.26e9 warp instructions for 5.0e8 probes = 4.5 per probe.
+        # one probe = one walked entry of the shorter list searched in the other (the bitmap kernel always walks t's out-list of z);
+        # both launches (count, write) walk every two-path's list
         nd = program.info["domain"]
         adj = {}
         for nm in ("r", "s", "t", "u"):
@@ -240,13 +242,25 @@ def roofline_of(program, prof_all, steps, sorting_route):
             adj[nm] = m
         two_paths = adj["r"] @ adj["s"]                                            # [x, z]
         walk = np.minimum(adj["t"].sum(axis=1)[None, :], adj["u"].sum(axis=0)[:, None])     # min(out_t(z), in_u(x))
-        per_probe = 4.5
         if dom == "k_cycle4_bitmap":
-            # the bitmap kernel always walks t's out-list of z; ncu at scale 16: 1.55e9 warp instructions for 5.37e8 probes = 2.9 per probe
             walk = np.broadcast_to(adj["t"].sum(axis=1)[None, :], two_paths.shape)
-            per_probe = 2.9
         probes = float((two_paths * walk).sum()) * d["launches"]
-        alu = {"achieved": probes / (d["ms"] / 1e3) / 1e9, "peak": 148 * 4 * 1.965 / per_probe, "unit": "Gprobe/s"}
+    if probes:
+        # L2 roofline: L2 bytes per probe from the ncu capture listed in profiles/ncu_traffic_ratios.md (lts__t_bytes.sum over the
+        # probes of the captured launch) times the probes per second measured here, against the L2 bandwidth measured here
+        # with the library's own copy kernel on a buffer pair that fits L2
+        per_probe = traffic_ratios().get((dom, "l2probe"))
+        instr = traffic_ratios().get((dom, "instr"))
+        if per_probe:
+            from paper_2609_27203_b200 import xlog
+            l2_peak = xlog.copy_bandwidth_gbs(32 << 20, 100)
+            rate = probes / (d["ms"] / 1e3)
+            l2 = {"achieved": rate * per_probe / 1e9, "peak": l2_peak, "probes_per_s": rate, "l2_bytes_per_probe": per_probe}
+            if instr:
+                # second figure, not a roofline: share of the issue slots the kernel's own instruction count takes at this rate
+                l2["issue"] = {"warp_instructions_per_probe": instr, "utilisation": rate * instr / (148 * 4 * 1.965e9),
+                               "what": "instructions per probe from the same ncu capture x probes/s over 148 SMs x 4 schedulers x 1.965 GHz"}
+            bound = "l2"
     roofline = {"bound": bound, "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "peak_source": peak_src,
                 "traffic": None if ratio is None else ratio * d["bytes"] / d["launches"],
@@ -263,9 +277,12 @@ def roofline_of(program, prof_all, steps, sorting_route):
         g = big["bytes"] / (big["ms"] / 1e3) / 1e9
         roofline["large_launches"] = {"launches_per_step": big["launches"] / steps, "ms_per_step": big["ms"] / steps,
                                       "achieved": g, "frac": g / peak, "what": "this kernel's launches of at least 48 MB algorithmic bytes (4 M candidates x 12 B) only"}
-    if alu:
-        roofline.update(achieved=alu["achieved"], peak=alu["peak"], unit=alu["unit"], frac=alu["achieved"] / alu["peak"], traffic=None,
-                        peak_source="derived: issue slots x clock / measured warp instructions per probe")
+    if l2:
+        roofline.update(achieved=l2["achieved"], peak=l2["peak"], unit="GB/s", frac=l2["achieved"] / l2["peak"], traffic=None,
+                        peak_source="measured here: xlog_device_copy on a 32 MB buffer pair (L2-resident), read + write bytes",
+                        probes_per_s=l2["probes_per_s"], l2_bytes_per_probe=l2["l2_bytes_per_probe"])
+        if "issue" in l2:
+            roofline["issue"] = l2["issue"]
     if mirror_kernel:
         # the tag-mirror joins move few bytes per candidate by construction; what limits them is said here
         roofline["limiter"] = ("instruction issue; the table, too large for L2, is read from HBM one 128-byte line per (changed unit of 32 keys, neighbour)"
@@ -433,7 +450,8 @@ def run_ours(args):
 # ------------------------------------------------------------------------------------------------
 FULL_SCALE = {"sssp": 20, "reach": 22, "triangles": 18, "wcoj": 16, "cycle4": 16}
 # seconds of one oracle fixpoint at the full size (host-core measurements of earlier runs; only used to size the sample)
-ORACLE_SECONDS_FULL = {"sssp": 12.0, "reach": 3400.0, "closure": 3.0, "triangles": 3200.0, "digits": 3.0, "wcoj": 60.0, "cycle4": 60.0}
+ORACLE_SECONDS_FULL = {"sssp": 12.0, "reach": 3400.0, "closure": 3.0, "triangles": 3200.0, "digits": 3.0, "wcoj": 60.0, "cycle4": 60.0,
+                       "nonlinear": 400.0, "mutual": 8.0}
 REFERENCE_BUDGET_S = 420.0
 
 
@@ -509,7 +527,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default=HEADLINE, choices=["sssp", "closure", "reach", "triangles", "digits", "wcoj", "cycle4"])
+    ap.add_argument("--workload", default=HEADLINE, choices=["sssp", "closure", "reach", "triangles", "digits", "wcoj", "cycle4", "nonlinear", "mutual"])
     ap.add_argument("--scale", type=int, default=None, help="R-MAT scale override (smaller cases for profiling)")
     ap.add_argument("--sources", type=int, default=None, help="reach: number of sources (fewer for a small profiling case)")
     ap.add_argument("--triangle-plan", default="auto", choices=["auto", "wcoj", "chain"], help="wcoj workload: force a join plan")

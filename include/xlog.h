@@ -269,6 +269,13 @@ typedef struct {
 xlog_status xlog_profile_read(xlog_ctx* ctx, xlog_kernel_stat* out, int32_t capacity, int32_t* n_out);
 xlog_status xlog_profile_reset(xlog_ctx* ctx);
 
+/* ---- a plain copy kernel, for measuring (The paper has no counterpart.) ----------------------------------------------
+ * Copies `bytes` (a multiple of 16; both pointers DEVICE, 16-byte aligned, not overlapping) from src to dst `repeats`
+ * times with the library's own grid-stride 16-byte-vector kernel, on `stream`, without waiting.  The benchmark times it
+ * on a buffer pair smaller than L2 to obtain the L2 bandwidth that cache-resident kernels (the sorted-list intersections
+ * of the triangle and four-cycle joins) are reported against, and on a large pair as a cross-check of the HBM figure. */
+xlog_status xlog_device_copy(void* stream, void* dst, const void* src, uint64_t bytes, int32_t repeats);
+
 /* ---- failure-path hooks (tests only) -----------------------------------------------------
  * Two kernels wait for other thread blocks of their own launch: the sort pass and the resident count + scan look back
  * through per-tile status words.  A tile only waits for tiles that already run, and every wait gives up after a number

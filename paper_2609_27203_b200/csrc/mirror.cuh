@@ -172,9 +172,13 @@ static __global__ void __launch_bounds__(kMtNodes) k_mirror_t_count(const uint32
   if (threadIdx.x < 64) s_cnt[threadIdx.x] = 0;
   __syncthreads();
   const unsigned long long mask = mt_mask(present, blockIdx.x * kMtNodes + threadIdx.x, n_nodes, slots);
-  for (int a = 0; a < slots; ++a) {
+  // only the columns some lane of the warp has
+  unsigned long long cols = ((unsigned long long)__reduce_or_sync(0xffffffffu, (uint32_t)(mask >> 32)) << 32) | __reduce_or_sync(0xffffffffu, (uint32_t)mask);
+  while (cols) {
+    const int a = __ffsll((long long)cols) - 1;
+    cols &= cols - 1;
     const unsigned bal = __ballot_sync(0xffffffffu, (mask >> a) & 1ull);
-    if (bal && lane_id() == 0) atomicAdd(&s_cnt[a], (uint32_t)__popc(bal));
+    if (lane_id() == 0) atomicAdd(&s_cnt[a], (uint32_t)__popc(bal));
   }
   __syncthreads();
   if ((int)threadIdx.x < slots) cnt[(size_t)threadIdx.x * ntiles + blockIdx.x] = s_cnt[threadIdx.x];
@@ -192,7 +196,12 @@ __global__ void __launch_bounds__(kMtNodes) k_mirror_t_emit(const uint32_t* __re
   const int slots_log2 = 31 - __clz(slots);
   if ((int)threadIdx.x < slots) s_base[threadIdx.x] = base[(size_t)threadIdx.x * ntiles + blockIdx.x];
   const unsigned long long mask = mt_mask(present, c, n_nodes, slots);
-  for (int a = 0; a < slots; ++a) {
+  const unsigned long long warp_cols = ((unsigned long long)__reduce_or_sync(0xffffffffu, (uint32_t)(mask >> 32)) << 32) | __reduce_or_sync(0xffffffffu, (uint32_t)mask);
+  for (int a = lane_id(); a < 64; a += 32) s_wcnt[warp_id()][a] = 0;
+  __syncwarp();
+  for (unsigned long long cols = warp_cols; cols;) {
+    const int a = __ffsll((long long)cols) - 1;
+    cols &= cols - 1;
     const unsigned bal = __ballot_sync(0xffffffffu, (mask >> a) & 1ull);
     if (lane_id() == 0) s_wcnt[warp_id()][a] = __popc(bal);
   }
@@ -207,22 +216,32 @@ __global__ void __launch_bounds__(kMtNodes) k_mirror_t_emit(const uint32_t* __re
   for (uint32_t v = threadIdx.x; v < nvec; v += kMtNodes) {
     const int4 x = __ldcs(src + v);
     const int32_t e[4] = {x.x, x.y, x.z, x.w};
+    const uint32_t i = v * 4;
+    if (slots >= 4) {
+      // the four slots of a vector belong to one c
+      int32_t* dst = s_tag + (i >> slots_log2) * 65 + (i & (slots - 1));
+      dst[0] = e[0]; dst[1] = e[1]; dst[2] = e[2]; dst[3] = e[3];
+    } else {
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const uint32_t i = v * 4 + j;
-      s_tag[(i >> slots_log2) * 65 + (i & (slots - 1))] = e[j];
+      for (int j = 0; j < 4; ++j) s_tag[((i + j) >> slots_log2) * 65 + ((i + j) & (slots - 1))] = e[j];
     }
   }
+  // where each warp's rows of column a begin: the (a, tile) base plus the earlier warps' counts
+  if (threadIdx.x < 64) {
+    uint32_t run = s_base[threadIdx.x];
+#pragma unroll
+    for (int w = 0; w < NW; ++w) { const uint32_t n = s_wcnt[w][threadIdx.x]; s_wcnt[w][threadIdx.x] = run; run += n; }
+  }
   __syncthreads();
-  for (int a = 0; a < slots; ++a) {
+  const int32_t* my_tags = s_tag + threadIdx.x * 65;
+  for (unsigned long long cols = warp_cols; cols;) {
+    const int a = __ffsll((long long)cols) - 1;
+    cols &= cols - 1;
     const unsigned bal = __ballot_sync(0xffffffffu, (mask >> a) & 1ull);
-    if (!bal) continue;
-    uint32_t pos = s_base[a];
-    for (unsigned w = 0; w < warp_id(); ++w) pos += s_wcnt[w][a];
     if ((mask >> a) & 1ull) {
-      pos += __popc(bal & lanemask_lt());
+      const uint32_t pos = s_wcnt[warp_id()][a] + __popc(bal & lanemask_lt());
       keys[pos] = ((K)(uint32_t)a << shift0) | ((K)c << shift1);
-      tags[pos] = ord2f(s_tag[threadIdx.x * 65 + a]);
+      tags[pos] = ord2f(my_tags[a]);
     }
   }
 }

@@ -189,6 +189,66 @@ def hot_domain_triangle(n_rows=65536, domain=406, seed=synth.SEED_BASE + 6) -> P
     return p
 
 
+def nonlinear_closure_program(src, dst, tag, semiring=MAXPLUS, name="nonlinear_closure") -> Program:
+    """p(x,y) :- e(x,y).  p(x,z) :- p(x,y), p(y,z): path doubling, two recursive atoms in one rule."""
+    return Program(
+        name=name,
+        relations={"e": (2, semiring), "p": (2, semiring)},
+        rules=[
+            Rule("p", (V(0), V(1)), (Atom("e", (Var(0), Var(1))),)),
+            Rule("p", (V(0), V(2)), (Atom("p", (Var(0), Var(1))), Atom("p", (Var(1), Var(2))))),
+        ],
+        facts={"e": ([np.ascontiguousarray(src, np.int32), np.ascontiguousarray(dst, np.int32)],
+                     None if tag is None else np.ascontiguousarray(tag, np.float32))},
+        outputs=("p",),
+    )
+
+
+def odd_even_program(src, dst, w, semiring=MINPLUS, name="odd_even") -> Program:
+    """odd(x,y) :- e(x,y).  even(x,z) :- odd(x,y), e(y,z).  odd(x,z) :- even(x,y), e(y,z): two mutually recursive heads
+    (best walks of odd / even length)."""
+    return Program(
+        name=name,
+        relations={"e": (2, semiring), "odd": (2, semiring), "even": (2, semiring)},
+        rules=[
+            Rule("odd", (V(0), V(1)), (Atom("e", (Var(0), Var(1))),)),
+            Rule("even", (V(0), V(2)), (Atom("odd", (Var(0), Var(1))), Atom("e", (Var(1), Var(2))))),
+            Rule("odd", (V(0), V(2)), (Atom("even", (Var(0), Var(1))), Atom("e", (Var(1), Var(2))))),
+        ],
+        facts={"e": ([np.ascontiguousarray(src, np.int32), np.ascontiguousarray(dst, np.int32)],
+                     np.ascontiguousarray(w, np.float32))},
+        outputs=("odd", "even"),
+    )
+
+
+def nonlinear_config(n_nodes=1000, n_edges=4000) -> Program:
+    """Path doubling on configuration 1's graph."""
+    seed = synth.SEED_BASE + 1
+    s, d = synth.uniform_digraph(n_nodes, n_edges, seed)
+    p = nonlinear_closure_program(s, d, synth.log_prob_tags(n_edges, seed), MAXPLUS, name=f"nonlinear_closure_n{n_nodes}_m{n_edges}")
+    p.info.update(n_nodes=n_nodes, n_edges=n_edges)
+    return p
+
+
+def nonlinear_rmat_config(scale=10, edge_factor=4) -> Program:
+    """Path doubling on a small R-MAT graph (hub-skewed: a few nodes reach and are reached by most of the others)."""
+    seed = synth.SEED_BASE + 8
+    s, d, w = synth.rmat_graph(scale, edge_factor, seed, "u1_10")
+    p = nonlinear_closure_program(s, d, w, MINPLUS, name=f"nonlinear_closure_rmat{scale}")
+    p.info.update(scale=scale, n_nodes=1 << scale, n_edges=int(s.size))
+    return p
+
+
+def mutual_config(n_nodes=1000, n_edges=4000) -> Program:
+    """Odd / even walks on configuration 1's graph with weights uniform in [1, 10]."""
+    seed = synth.SEED_BASE + 1
+    s, d = synth.uniform_digraph(n_nodes, n_edges, seed)
+    w = (1.0 + 9.0 * synth.uniform01(seed, 9, 0, n_edges)).astype(np.float32)
+    p = odd_even_program(s, d, w, MINPLUS, name=f"odd_even_n{n_nodes}_m{n_edges}")
+    p.info.update(n_nodes=n_nodes, n_edges=n_edges)
+    return p
+
+
 def digits_program(log_tags: np.ndarray, name="digits") -> Program:
     """sum(p, a+b) :- digit(2p, a), digit(2p+1, b), logsumexp per (p, a+b).
 

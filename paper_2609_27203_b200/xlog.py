@@ -33,7 +33,7 @@ PLAN_NONE, PLAN_WCOJ, PLAN_CHAIN = 0, 1, 2
 EXPORTS = ["xlog_ctx_create", "xlog_ctx_destroy", "xlog_last_error", "xlog_relation_create", "xlog_relation_load",
            "xlog_relation_size", "xlog_relation_read", "xlog_relation_view", "xlog_rule_add", "xlog_fixpoint",
            "xlog_ctx_reset_idb", "xlog_rule_backward", "xlog_profile_read", "xlog_profile_reset",
-           "xlog_reduce_by_key_static", "xlog_sort_pairs", "xlog_debug_set_poll_limit", "xlog_debug_sort_pass_without_first_tile"]
+           "xlog_reduce_by_key_static", "xlog_sort_pairs", "xlog_debug_set_poll_limit", "xlog_debug_sort_pass_without_first_tile", "xlog_device_copy"]
 
 
 class XlogError(RuntimeError):
@@ -110,6 +110,7 @@ def lib():
         L.xlog_profile_read.argtypes = [vp, C.POINTER(KernelStat), i32, C.POINTER(i32)]
         L.xlog_profile_reset.argtypes = [vp]
         L.xlog_sort_pairs.argtypes = [vp, vp, vp, i64, i32, i32]
+        L.xlog_device_copy.argtypes = [vp, vp, vp, C.c_uint64, i32]
         L.xlog_debug_set_poll_limit.argtypes = [vp, C.c_uint32]
         L.xlog_debug_sort_pass_without_first_tile.argtypes = [vp, vp, vp, vp, vp, i64, i32]
         L.xlog_reduce_by_key_static.argtypes = [vp, i32, vp, vp, i64, vp, vp, C.POINTER(i64), C.c_char_p, C.c_size_t]
@@ -326,6 +327,26 @@ class Context:
 
 
 STATIC_REDUCE_MAX_ROWS = 1 << 24
+
+
+def copy_bandwidth_gbs(n_bytes: int, repeats: int = 50, device: int = 0) -> float:
+    """GB/s (bytes read + bytes written) of the library's own copy kernel on a pair of n_bytes buffers: with a pair that
+    fits L2 this is the L2 bandwidth, with a large pair the HBM bandwidth.  CUDA events on torch's current stream."""
+    import torch
+    with torch.cuda.device(device):
+        a = torch.empty(n_bytes, dtype=torch.uint8, device=f"cuda:{device}").fill_(1)
+        b = torch.empty_like(a)
+        s = torch.cuda.current_stream(device)
+        L = lib()
+        if L.xlog_device_copy(s.cuda_stream, b.data_ptr(), a.data_ptr(), n_bytes, 5):
+            raise XlogError(9, "xlog_device_copy failed")
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(s)
+        if L.xlog_device_copy(s.cuda_stream, b.data_ptr(), a.data_ptr(), n_bytes, repeats):
+            raise XlogError(9, "xlog_device_copy failed")
+        e1.record(s)
+        e1.synchronize()
+        return 2.0 * n_bytes * repeats / (e0.elapsed_time(e1) * 1e-3) / 1e9
 
 
 def check_load_shapes(cols, tags, device) -> int:
