@@ -81,6 +81,7 @@ typedef struct {
 #define XLOG_FLAG_FORCE_CHAIN     64u  /* ... always the binary-join chain (fails with RESOURCE_EXHAUSTED if its intermediate does not fit) */
 #define XLOG_FLAG_NO_GROUPED_JOIN 128u  /* tag mirror: always the row-wise join, never the grouped one (see csrc/group_join.cuh) */
 #define XLOG_FLAG_NO_BITMAP_JOIN  256u  /* tag mirror, grouped join: always from a delta row list, never straight from the changed bitmap (see csrc/bitmap_join.cuh) */
+#define XLOG_FLAG_NO_DENSE_DOUBLING 512u /* tag mirror: the path-doubling rule h(x,z) :- h(x,y), h(y,z) goes through the sorting route, not the dense rounds */
 #define XLOG_FLAG_NO_GRAPH        16u  /* resident rounds are launched one by one instead of as one graph with a WHILE node */
 
 /* Evaluation routes of a recursive component (Algorithm 1).  All of them derive the same relation,
@@ -95,6 +96,10 @@ typedef struct {
  *    least 32 (and at most 1024) possible values of a and one such rule, the rounds are driven by the changed bitmap itself:
  *    one kernel turns the bitmap into work items and a list of the changed keys' (tag, a) pairs grouped by b, one joins
  *    (XLOG_FLAG_NO_BITMAP_JOIN switches this off); the pair list holds 8 bytes per possible key.
+ *    One rule shape with two atoms over the relation is served as well: path doubling  h(x,z) :- h(x,y), h(y,z)  as the
+ *    only rule over a binary h with at most 4096 values in its second column.  The mirror is then a matrix; a round copies
+ *    it (the state both delta variants read) and one thread block per row applies every candidate of both variants in
+ *    shared memory (csrc/dense_closure.cuh; XLOG_FLAG_NO_DENSE_DOUBLING sends the rule through the sorting route).
  *  - Resident rounds (tag mirror with <= 2^24 possible keys): the delta rounds run as one CUDA graph with a
  *    conditional WHILE node and fixed-capacity buffers (Section "GPU-Native Symbolic Substrate": resident
  *    conditional graph, no host reads inside the loop).  The buffers (about 36 bytes per possible key

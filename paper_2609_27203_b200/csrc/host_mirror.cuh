@@ -3,6 +3,7 @@
 #pragma once
 #include "host_eval.cuh"
 #include "bitmap_join.cuh"
+#include "dense_closure.cuh"
 #include "group_join.cuh"
 #include "mirror.cuh"
 #include "resident.cuh"
@@ -16,6 +17,42 @@ constexpr int kMirrorMaxBits = 30;
 // The tag mirror serves a component of one max/min relation whose rules are all linear (at most one atom over the
 // relation itself, and that atom is the scanned side): then the relation is only ever read through its delta, and
 // its sorted form is needed again only after the last round.
+// Path doubling  h(x,z) :- h(x,y), h(y,z)  (dense_closure.cuh): the one rule shape with two atoms over the relation that a
+// tag mirror serves, because both of its delta variants can read the looked-up side from the mirror itself.  It must be
+// the only rule with atoms over h, h binary without dictionaries, and a row of the matrix must fit shared memory.
+constexpr int kDenseMaxColumnBits = 12;
+constexpr int kSlotDense = 90;             // candidate counter of the dense path-doubling rounds
+
+bool is_doubling_rule(Ctx* c, int h, const RuleC* r) {
+  const xlog_plan& p = r->plan;
+  if (r->kind != 2 || p.n_atoms != 2 || p.atoms[0].rel != h || p.atoms[1].rel != h || p.atoms[0].negated || p.atoms[1].negated) return false;
+  const xlog_arg* a = p.atoms[0].args; const xlog_arg* b = p.atoms[1].args;
+  if (!is_plain_var(a[0]) || !is_plain_var(a[1]) || !is_plain_var(b[0]) || !is_plain_var(b[1])) return false;
+  const int x = a[0].var, y = a[1].var, z = b[1].var;
+  if (b[0].var != y || x == y || y == z || x == z || p.n_head_cols != 2 || p.emit_count_column) return false;
+  const int hv[2] = {x, z};
+  for (int col = 0; col < 2; ++col) {
+    if (p.head[col].c0 != 0) return false;
+    for (int v = 0; v < XLOG_MAX_VARS; ++v) if (p.head[col].coef[v] != (v == hv[col] ? 1 : 0)) return false;
+  }
+  return true;
+}
+const RuleC* doubling_rule_of(Ctx* c, int h, const std::vector<const RuleC*>& rs) {
+  if (c->flags & XLOG_FLAG_NO_DENSE_DOUBLING) return nullptr;
+  const Relation& H = *c->rels[h];
+  if (H.arity != 2 || H.dict_n[0] || H.dict_n[1] || H.layout.shift[1] != 0) return nullptr;
+  if (H.layout.shift[0] > kDenseMaxColumnBits) return nullptr;             // shift of column 0 = bits of column 1 = log2 of the row length
+  const RuleC* found = nullptr;
+  for (const RuleC* r : rs) {
+    int in = 0;
+    for (int j = 0; j < r->plan.n_atoms; ++j) if (r->plan.atoms[j].rel == h) ++in;
+    if (in == 0) continue;
+    if (found || !is_doubling_rule(c, h, r)) return nullptr;
+    found = r;
+  }
+  return found;
+}
+
 bool mirror_applies(Ctx* c, const std::vector<int>& comp, const std::vector<const RuleC*>& rs) {
   if ((c->flags & XLOG_FLAG_NO_TAG_MIRROR) || comp.size() != 1) return false;
   const Relation& H = *c->rels[comp[0]];
@@ -26,12 +63,13 @@ bool mirror_applies(Ctx* c, const std::vector<int>& comp, const std::vector<cons
     int in = 0, pos = 0;
     for (int j = 0; j < r->plan.n_atoms; ++j)
       if (r->plan.atoms[j].rel == comp[0]) { if (r->plan.atoms[j].negated) return false; ++in; pos = j; }
-    if (in > 1) return false;
+    if (in > 1 && !(c->rels[comp[0]]->layout.total_bits <= kMirrorMaxBits && doubling_rule_of(c, comp[0], rs) == r)) return false;
     if (in == 1 && r->kind == 2 && !r->shape[pos].ok) return false;
     if (in == 1 && r->kind != 2 && pos != 0) return false;
     if (in == 0 && r->kind == 2 && !r->shape[0].ok && !r->shape[1].ok) return false;
   }
-  const uint64_t need = ((uint64_t)4 << H.layout.total_bits) + ((uint64_t)1 << H.layout.total_bits) / 4 + (1u << 20);
+  uint64_t need = ((uint64_t)4 << H.layout.total_bits) + ((uint64_t)1 << H.layout.total_bits) / 4 + (1u << 20);
+  if (doubling_rule_of(c, comp[0], rs)) need += (uint64_t)4 << H.layout.total_bits;       // the snapshot of the matrix
   return need <= c->arena.largest_free() / 2;
 }
 
@@ -367,7 +405,9 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
   const uint64_t slots = std::max<uint64_t>(dom, 4);
   const uint32_t bm_quads = (uint32_t)((std::max<uint64_t>(dom / 32, 1) + 3) / 4);
   const unsigned ch_tiles = mirror_tiles(bm_quads * 4);
-  Resident* R = resident_for(c, h, bits, slots, bm_quads, ch_tiles);
+  const RuleC* doubling = doubling_rule_of(c, h, rs);
+  Resident* R = doubling ? nullptr : resident_for(c, h, bits, slots, bm_quads, ch_tiles);
+  if (doubling) c->resident.erase(h);
   // the mirror's own column order: for the grouped join the probed column is the major part of the index (group_join.cuh)
   KeyLayout M = H.layout;
   const bool grouped = !R && !(c->flags & XLOG_FLAG_NO_GROUPED_JOIN) && grouped_shape(c, h, rs);
@@ -385,6 +425,10 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
   }
   BitmapJoin bj;
   if (grouped) bitmap_join_setup(c, h, rs, M, carried_bits, slots, bj);
+  DevBuf snap_own, rowstart_own;
+  const int dense_bits1 = H.layout.shift[0];
+  const uint32_t dense_rows = (uint32_t)(slots >> dense_bits1);
+  if (doubling) { snap_own = DevBuf(c, slots * 4); rowstart_own = DevBuf(c, ((size_t)dense_rows + 2) * 4); }
   uint32_t* present = R ? R->present.as<uint32_t>() : present_own.as<uint32_t>();
   int32_t* table = R ? R->table.as<int32_t>() : table_own.as<int32_t>();
   uint4* bitmap = R ? R->bitmap.as<uint4>() : bitmap_own.as<uint4>();
@@ -475,11 +519,37 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
         const int outer = seed_outer(comp, r);
         vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
       } else {
+        if (r == doubling) continue;                      // both of its delta variants run in the dense round below
         for (int j = 0; j < r->plan.n_atoms; ++j)
           if (r->plan.atoms[j].rel == h && dn) vs.push_back(Variant{r, j, Source{dk, dt, dn, M, H.key_bytes}});
       }
     }
-    const uint64_t total = host_apply(vs);
+    uint64_t total = 0;
+    const bool dense_round = doubling && round > 0 && dn > 0;
+    if (dense_round) {
+      // path doubling: snapshot the matrix, then one block per row applies both delta variants (dense_closure.cuh)
+      XLOG_CUDA(cudaMemcpyAsync(snap_own.p, table, slots * 4, cudaMemcpyDeviceToDevice, c->stream));
+      zero_ctrl(c, kSlotDense);
+      XLOG_LAUNCH(c, k_dense_rowstart, (dense_rows + 1 + 255) / 256, 256, 0, (const uint32_t*)dk, dn, dense_bits1, dense_rows, rowstart_own.as<uint32_t>());
+      const DenseRound D{snap_own.as<int32_t>(), table, reinterpret_cast<uint32_t*>(bitmap), (const uint32_t*)dk, dt, rowstart_own.as<uint32_t>(), dense_rows,
+                         dense_bits1, (unsigned long long*)(c->d_ctrl + kSlotDense)};
+      c->note_bytes = (int64_t)slots * 8 + (int64_t)dn * 8;
+#define XLOG_DENSE_ROUND(COLS)                                                                                                  \
+  do {                                                                                                                          \
+    if (is_max) XLOG_LAUNCH(c, (k_dense_round<kSinkMax, COLS>), dense_rows, kDenseRoundBlock, dense_round_smem(dense_bits1), D); \
+    else XLOG_LAUNCH(c, (k_dense_round<kSinkMin, COLS>), dense_rows, kDenseRoundBlock, dense_round_smem(dense_bits1), D);        \
+  } while (0)
+      switch (std::max(dense_bits1 - 8, 0)) {              // columns per thread = row length / 256
+        case 0: XLOG_DENSE_ROUND(1); break;
+        case 1: XLOG_DENSE_ROUND(2); break;
+        case 2: XLOG_DENSE_ROUND(4); break;
+        case 3: XLOG_DENSE_ROUND(8); break;
+        default: XLOG_DENSE_ROUND(16); break;
+      }
+#undef XLOG_DENSE_ROUND
+      total = 1;                                         // the candidate count arrives with the round's control read
+    }
+    total += host_apply(vs);
     if (total == 0 && !(round == 0 && plain_rules_done)) break;
     if (bj.valid) {
       // Every later round is  k_bm_plan -> one control read -> k_bm_expand : the plan kernel closes the round just joined
@@ -517,6 +587,7 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
     XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, ch_sums, (int64_t)ch_tiles, ctrl_u32(c, kSlotMirChanged));
     sync_ctrl(c);
     const uint32_t changed = (uint32_t)c->h_ctrl[kSlotMirChanged];
+    if (dense_round) c->r_candidates += (int64_t)c->h_ctrl[kSlotDense];
     const uint64_t n_new = c->h_ctrl[kSlotMirNew] - total_new;
     total_new += n_new;
     c->r_new += (int64_t)n_new; c->r_improved += (int64_t)changed - (int64_t)n_new;

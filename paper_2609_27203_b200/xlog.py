@@ -28,6 +28,7 @@ FLAG_FORCE_WCOJ = 32
 FLAG_FORCE_CHAIN = 64
 FLAG_NO_GROUPED_JOIN = 128
 FLAG_NO_BITMAP_JOIN = 256
+FLAG_NO_DENSE_DOUBLING = 512
 PLAN_NONE, PLAN_WCOJ, PLAN_CHAIN = 0, 1, 2
 
 EXPORTS = ["xlog_ctx_create", "xlog_ctx_destroy", "xlog_last_error", "xlog_relation_create", "xlog_relation_load",

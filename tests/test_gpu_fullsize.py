@@ -202,3 +202,17 @@ def test_config5_reach_rmat22_full_four_sources_by_oracle():
         assert np.array_equal(rt[sel].view(np.int32), ot.view(np.int32))
         assert len(ot) > 2_000_000
     pool.shutdown()
+
+
+def test_mutual_recursion_full_size_against_the_oracle():
+    # odd / even walks on configuration 1's graph: two mutually recursive heads, 1.9 M derived tuples, every row by the oracle
+    prog = W.mutual_config()
+    ctx, ids, _, receipt = gpu_fixpoint(prog, 2 << 30)
+    o, oids, _ = oracle.load_program(prog)
+    stats = o.run("seminaive")
+    for name in ("odd", "even"):
+        rep = H.compare_relations(ctx.read(ids[name]), o.read(oids[name]), rel_tol=1e-5, what=name)
+        assert rep["bit_unequal"] == 0
+    assert receipt["derived_tuples"] == stats["derived_tuples"] and receipt["candidates"] == stats["contributions"]
+    assert receipt["iterations"] == stats["iterations"]
+    ctx.close()

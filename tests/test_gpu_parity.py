@@ -423,3 +423,36 @@ def test_join_indices_of_unchanged_relations_are_reused_across_fixpoints():
         assert third["index_builds"] == first["index_builds"]
         assert H.compare_relations(ctx.read(ids["path"]), want, what="after reload")["bit_unequal"] == 0
         ctx.close()
+
+
+def test_path_doubling_through_the_dense_rounds_at_scale():
+    # p(x,z) :- p(x,y), p(y,z) on graphs of 300 to 1000 nodes: the default route keeps p as a matrix and applies both delta
+    # variants of a round row by row (no sort, no index of p); it must agree bit for bit, relation and counters, with the
+    # sorting route, with the oracle where the oracle finishes in seconds, and (tuple set; tags to 1e-5) with the linear closure
+    from paper_2609_27203_b200 import xlog
+    small = W.nonlinear_config(300, 1200)
+    r, stats = check_program(small, expect_bit_equal=True)
+    assert r["candidates"] == stats["contributions"]                     # every binding of both delta variants, counted once each
+    # hub-skewed, min-plus, with loaded facts of p itself (the seed round then joins the full relation with itself)
+    rm = W.nonlinear_rmat_config(8)
+    (s, d), w = rm.facts["e"]
+    rm.facts["p"] = ([np.array([3, 200], np.int32), np.array([250, 7], np.int32)], np.array([0.5, 40.0], np.float32))
+    check_program(rm)
+    big = W.nonlinear_config()                                             # configuration 1's graph
+    res = {}
+    for flags in (0, xlog.FLAG_NO_DENSE_DOUBLING):
+        ctx, ids, _ = xlog.load_program(big, arena_bytes=16 << 30, flags=flags)
+        receipt = ctx.fixpoint()
+        res[flags] = (receipt, ctx.read(ids["p"]))
+        again = ctx.fixpoint()
+        assert again["new_tuples"] == 0 and again["improved_tags"] == 0   # idempotent on both routes
+        ctx.close()
+    a, b = res[0], res[xlog.FLAG_NO_DENSE_DOUBLING]
+    assert H.compare_relations(a[1], b[1], what="dense rounds vs sorting route")["bit_unequal"] == 0
+    for k in ("iterations", "candidates", "new_tuples", "improved_tags", "derived_tuples"):
+        assert a[0][k] == b[0][k], k
+    lin = W.config1()
+    ctx, ids, _ = xlog.load_program(lin, arena_bytes=1 << 28)
+    ctx.fixpoint()
+    H.compare_relations(a[1], ctx.read(ids["path"]), rel_tol=1e-5, what="path doubling vs linear closure")
+    ctx.close()
