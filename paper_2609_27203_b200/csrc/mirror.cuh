@@ -172,13 +172,15 @@ static __global__ void __launch_bounds__(kMtNodes) k_mirror_t_count(const uint32
   if (threadIdx.x < 64) s_cnt[threadIdx.x] = 0;
   __syncthreads();
   const unsigned long long mask = mt_mask(present, blockIdx.x * kMtNodes + threadIdx.x, n_nodes, slots);
-  // only the columns some lane of the warp has
-  unsigned long long cols = ((unsigned long long)__reduce_or_sync(0xffffffffu, (uint32_t)(mask >> 32)) << 32) | __reduce_or_sync(0xffffffffu, (uint32_t)mask);
-  while (cols) {
-    const int a = __ffsll((long long)cols) - 1;
-    cols &= cols - 1;
-    const unsigned bal = __ballot_sync(0xffffffffu, (mask >> a) & 1ull);
-    if (lane_id() == 0) atomicAdd(&s_cnt[a], (uint32_t)__popc(bal));
+  // only the columns some lane of the warp has; the two 32-bit halves of the mask one after the other
+#pragma unroll
+  for (int half = 0; half < 2; ++half) {
+    const uint32_t m32 = (uint32_t)(mask >> (32 * half));
+    for (uint32_t cols = __reduce_or_sync(0xffffffffu, m32); cols; cols &= cols - 1) {
+      const int a = __ffs(cols) - 1;
+      const unsigned bal = __ballot_sync(0xffffffffu, (m32 >> a) & 1u);
+      if (lane_id() == 0) atomicAdd(&s_cnt[32 * half + a], (uint32_t)__popc(bal));
+    }
   }
   __syncthreads();
   if ((int)threadIdx.x < slots) cnt[(size_t)threadIdx.x * ntiles + blockIdx.x] = s_cnt[threadIdx.x];
@@ -196,15 +198,17 @@ __global__ void __launch_bounds__(kMtNodes) k_mirror_t_emit(const uint32_t* __re
   const int slots_log2 = 31 - __clz(slots);
   if ((int)threadIdx.x < slots) s_base[threadIdx.x] = base[(size_t)threadIdx.x * ntiles + blockIdx.x];
   const unsigned long long mask = mt_mask(present, c, n_nodes, slots);
-  const unsigned long long warp_cols = ((unsigned long long)__reduce_or_sync(0xffffffffu, (uint32_t)(mask >> 32)) << 32) | __reduce_or_sync(0xffffffffu, (uint32_t)mask);
+  const uint32_t m32[2] = {(uint32_t)mask, (uint32_t)(mask >> 32)};
+  const uint32_t warp_cols[2] = {__reduce_or_sync(0xffffffffu, m32[0]), __reduce_or_sync(0xffffffffu, m32[1])};
   for (int a = lane_id(); a < 64; a += 32) s_wcnt[warp_id()][a] = 0;
   __syncwarp();
-  for (unsigned long long cols = warp_cols; cols;) {
-    const int a = __ffsll((long long)cols) - 1;
-    cols &= cols - 1;
-    const unsigned bal = __ballot_sync(0xffffffffu, (mask >> a) & 1ull);
-    if (lane_id() == 0) s_wcnt[warp_id()][a] = __popc(bal);
-  }
+#pragma unroll
+  for (int half = 0; half < 2; ++half)
+    for (uint32_t cols = warp_cols[half]; cols; cols &= cols - 1) {
+      const int a = __ffs(cols) - 1;
+      const unsigned bal = __ballot_sync(0xffffffffu, (m32[half] >> a) & 1u);
+      if (lane_id() == 0) s_wcnt[warp_id()][32 * half + a] = __popc(bal);
+    }
   __syncthreads();
   if (__syncthreads_or(mask != 0ull) == 0) return;       // nothing present in this tile
   // the tile's slots are contiguous in the table: a straight 16-byte-vector copy into the padded shared array, all of a
@@ -234,16 +238,20 @@ __global__ void __launch_bounds__(kMtNodes) k_mirror_t_emit(const uint32_t* __re
   }
   __syncthreads();
   const int32_t* my_tags = s_tag + threadIdx.x * 65;
-  for (unsigned long long cols = warp_cols; cols;) {
-    const int a = __ffsll((long long)cols) - 1;
-    cols &= cols - 1;
-    const unsigned bal = __ballot_sync(0xffffffffu, (mask >> a) & 1ull);
-    if ((mask >> a) & 1ull) {
-      const uint32_t pos = s_wcnt[warp_id()][a] + __popc(bal & lanemask_lt());
-      keys[pos] = ((K)(uint32_t)a << shift0) | ((K)c << shift1);
-      tags[pos] = ord2f(my_tags[a]);
+  const K ckey = (K)c << shift1;
+  const uint32_t* my_base = s_wcnt[warp_id()];
+#pragma unroll
+  for (int half = 0; half < 2; ++half)
+    for (uint32_t cols = warp_cols[half]; cols; cols &= cols - 1) {
+      const int a = __ffs(cols) - 1;
+      const bool mine = (m32[half] >> a) & 1u;
+      const unsigned bal = __ballot_sync(0xffffffffu, mine);
+      if (mine) {
+        const uint32_t pos = my_base[32 * half + a] + __popc(bal & lanemask_lt());
+        keys[pos] = ((K)(uint32_t)(32 * half + a) << shift0) | ckey;
+        tags[pos] = ord2f(my_tags[32 * half + a]);
+      }
     }
-  }
 }
 
 }  // namespace xlog
