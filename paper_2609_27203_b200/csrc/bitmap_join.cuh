@@ -11,9 +11,9 @@
 //                passes over the k changed keys of b.  A block reserves its list room with one atomic add, so the
 //                order of items and of pair runs varies from run to run; nothing derived depends on it.
 //                Totals (changed keys, new keys, candidates, items, neighbour rows read) go to counters.
-//   k_bm_expand  a warp per item.  Four steps of 32 lanes offer 128 lane slots; the pass's k pairs times floor(128 / k)
-//                neighbours fill them, so the lanes stay busy whatever k is.  32 neighbours at a time are read coalesced
-//                and handed round with shuffles; per candidate: two shuffles, an add for the slot, the slot read, an add,
+//   k_bm_expand  a warp per item.  The lanes take the pass's k keys (k rounded up to a power of two k'), so one step of
+//                the warp covers 32 / k' neighbours.  32 neighbours at a time are read coalesced and staged in shared
+//                memory; per candidate: one broadcast read of (neighbour's slot base, weight), the slot read, an add,
 //                the order map, a compare, and for the few that improve the atomic min / max and the bit in the changed
 //                bitmap.
 //
