@@ -102,7 +102,7 @@ Resident* resident_for(Ctx* c, int h, int bits, uint64_t slots, uint32_t bm_quad
   R->rowinfo = DevBuf(c, dom * 16); R->start = DevBuf(c, dom * 8);
   R->scan_tiles_cap = (uint32_t)(dom / kResScanTile + 2);
   R->scan_status = DevBuf(c, (size_t)kResMaxVariants * R->scan_tiles_cap * 8);
-  R->tickets = DevBuf(c, (kResMaxVariants + 2) * 4);
+  R->tickets = DevBuf(c, kResTickets * 4);
   R->tile_rows = DevBuf(c, (size_t)max_tiles * 8);
   Resident* out = R.get();
   c->resident[h] = std::move(R);
@@ -128,6 +128,13 @@ template <typename T> void sig_add(std::vector<char>& sig, const T& v) {
   sig.insert(sig.end(), p, p + sizeof(T));
 }
 
+// Count, scan and partition of rule v over the current delta (resident.cuh).
+void resident_count(Ctx* c, Resident& R, const JoinSpec& S, size_t v) {
+  XLOG_LAUNCH(c, (k_res_count_scan<uint32_t>), kSMs * 4, kScanBlock, 0, S, (const uint32_t*)R.dkeys.as<uint32_t>(), (const float*)R.dtags.as<float>(), res_state(c),
+              R.rowinfo.as<uint4>(), R.start.as<uint64_t>(), R.tile_rows.as<uint2>(), R.scan_status.as<unsigned long long>() + v * R.scan_tiles_cap,
+              R.tickets.as<uint32_t>() + v, ctrl_u32(c, kSlotErr), c->spin_limit);
+}
+
 // One round's launches.  Nothing here allocates, copies or waits: the same calls are either captured into the WHILE
 // body or issued directly (host-driven rounds, used when launches are being timed one by one).
 void resident_body(Ctx* c, Resident& R, const std::vector<JoinSpec>& specs, bool is_max, const MirrorArgs& mr, uint32_t bm_quads, unsigned ch_tiles,
@@ -136,10 +143,10 @@ void resident_body(Ctx* c, Resident& R, const std::vector<JoinSpec>& specs, bool
   uint32_t* err = ctrl_u32(c, kSlotErr);
   const uint32_t* dk = R.dkeys.as<uint32_t>();
   const ResScratch sc{R.scan_status.as<unsigned long long>(), R.scan_tiles_cap, R.tickets.as<uint32_t>()};
+  const bool fused = specs.size() == 1;                  // the count of the next round rides on the emit kernel; the first round's is launched before the loop
   for (size_t v = 0; v < specs.size(); ++v) {
     const JoinSpec& S = specs[v];
-    XLOG_LAUNCH(c, (k_res_count_scan<uint32_t>), kSMs * 4, kScanBlock, 0, S, dk, (const float*)R.dtags.as<float>(), st, R.rowinfo.as<uint4>(),
-                R.start.as<uint64_t>(), R.tile_rows.as<uint2>(), sc.scan_status + v * R.scan_tiles_cap, sc.tickets + v, err, c->spin_limit);
+    if (!fused) resident_count(c, R, S, v);
 // four waves of blocks: the hardware hands a new block to whichever SM finishes first, which evens out skewed tiles
 #define XLOG_RES_EXPAND(MODE, SINK)                                                                                                         \
   XLOG_LAUNCH(c, (k_res_expand<uint32_t, MODE, SINK>), kSMs * kExpMirrorBlocksPerSM * 4, kExpBlock, 0, S, dk, (const ResState*)st, (const uint64_t*)R.start.as<uint64_t>(), \
@@ -148,7 +155,16 @@ void resident_body(Ctx* c, Resident& R, const std::vector<JoinSpec>& specs, bool
     else { if (is_max) XLOG_RES_EXPAND(kExpGeneric, kSinkMax); else XLOG_RES_EXPAND(kExpGeneric, kSinkMin); }
 #undef XLOG_RES_EXPAND
   }
-  uint32_t* ctr = sc.tickets + kResMaxVariants;
+  uint32_t* ctr = sc.tickets + kResTkEmit;
+  if (fused) {
+#define XLOG_RES_EMIT_COUNT(SW)                                                                                                            \
+  XLOG_LAUNCH(c, (k_res_emit_count<SW>), (bm_quads * 4 + kResEcWords * SW - 1) / (kResEcWords * SW), kMirBlock, 0, R.bitmap.as<uint32_t>(), R.present.as<uint32_t>(), bm_quads * 4, mr.n_new,  \
+              (const int32_t*)R.table.as<int32_t>(), R.dkeys.as<uint32_t>(), R.dtags.as<float>(), st, sc, (const unsigned long long*)mr.n_new, \
+              ctr, handle, use_handle, specs[0], R.rowinfo.as<uint4>(), R.start.as<uint64_t>(), R.tile_rows.as<uint2>(), err)
+    if (mirror_sweeps(bm_quads * 4) == 1) XLOG_RES_EMIT_COUNT(1); else XLOG_RES_EMIT_COUNT(4);
+#undef XLOG_RES_EMIT_COUNT
+    return;
+  }
 #define XLOG_RES_EMIT(SW)                                                                                                                  \
   XLOG_LAUNCH(c, (k_res_emit<SW>), ch_tiles, kMirBlock, 0, R.bitmap.as<uint32_t>(), R.present.as<uint32_t>(), bm_quads * 4, mr.n_new,        \
               (const int32_t*)R.table.as<int32_t>(),                                                                                        \
@@ -174,6 +190,8 @@ ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*
   const ResScratch sc{R.scan_status.as<unsigned long long>(), R.scan_tiles_cap, R.tickets.as<uint32_t>()};
   XLOG_LAUNCH(c, k_res_init, 1, 1024, 0, res_state(c), sc, (uint32_t)specs.size(), n_delta, budget, R.max_tiles, (unsigned long long)new_seen);
   const MirrorArgs& mr = mr_host;
+  const bool fused = specs.size() == 1;
+  if (fused) resident_count(c, R, specs[0], 0);          // the first round's count; every later one rides on the emit kernel
   const int64_t l0 = c->launches;
   const bool use_graph = !(c->flags & (XLOG_FLAG_PROFILE | XLOG_FLAG_NO_GRAPH));
   ResState out{};
@@ -223,7 +241,7 @@ ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*
     }
     XLOG_CUDA(cudaGraphLaunch(R.exec, c->stream));
     read_state();
-    c->launches = l0 + R.body_launches * (int64_t)out.rounds + (out.status == kResOverflow ? R.body_launches : 0);
+    c->launches = l0 + R.body_launches * (int64_t)out.rounds + (out.status == kResOverflow && !fused ? R.body_launches : 0);
   } else {
     unsigned long long seen = 0;
     uint32_t rows = n_delta;
@@ -238,8 +256,8 @@ ResState run_resident(Ctx* c, Resident& R, int h, const std::vector<const RuleC*
       read_state();
       if (c->flags & XLOG_FLAG_PROFILE) {
         // per delta row and rule: key and tag read, two offsets probed, 16-byte row record and 8-byte start offset written
-        auto cs = c->prof_index.find("k_res_count_scan");
-        if (cs != c->prof_index.end()) c->prof[cs->second].bytes += (int64_t)rows * 40 * (int64_t)specs.size();
+        auto cs = c->prof_index.find(fused ? "k_res_emit_count" : "k_res_count_scan");
+        if (cs != c->prof_index.end()) c->prof[cs->second].bytes += (int64_t)(fused ? out.n_delta : rows) * 40 * (int64_t)specs.size() + (fused ? (int64_t)bm_quads * 16 : 0);
         rows = out.n_delta;
         // algorithmic bytes of the round's expand launches (per candidate: the looked-up columns and tag, and the slot)
         auto it = c->prof_index.find("k_res_expand");

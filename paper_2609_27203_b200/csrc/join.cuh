@@ -96,14 +96,15 @@ __device__ __forceinline__ bool bind_outer(const JoinSpec& S, KO key, int64_t* v
 // is linear in the inner columns, key = rowkey + sum_j inner_col_j * inner_mult[j], so everything that
 // depends on the outer row alone (constants, outer variables, dictionary ranks, range checks) is done
 // here once per row instead of once per candidate.
+// The row is given by value (its packed key and tag); rowinfo == nullptr: the degree only, nothing is written.
 template <typename KO>
-__device__ __forceinline__ uint32_t join_count_row(const JoinSpec& S, const KO* __restrict__ okeys, const float* __restrict__ otags, uint32_t i,
-                                                   uint4* __restrict__ rowinfo, uint32_t* __restrict__ err) {
+__device__ __forceinline__ uint32_t join_count_kv(const JoinSpec& S, const KO okey, const float otag, uint32_t i, uint4* __restrict__ rowinfo,
+                                                  uint32_t* __restrict__ err) {
   int64_t var[kMaxVars];
   uint32_t d = 0, lo = 0;
   uint64_t rowkey = 0;
   if (S.simple) {
-    const uint64_t k = (uint64_t)okeys[i];
+    const uint64_t k = (uint64_t)okey;
     if ((k & S.s_const_mask) == S.s_const_val) {
       d = 1;
       if (S.has_inner) {
@@ -126,7 +127,7 @@ __device__ __forceinline__ uint32_t join_count_row(const JoinSpec& S, const KO* 
         if (e) atomicOr(err, e);
       }
     }
-  } else if (bind_outer<KO>(S, okeys[i], var)) {
+  } else if (bind_outer<KO>(S, okey, var)) {
     if (S.neg_prefix) {
       int64_t val[2] = {0, 0};
 #pragma unroll
@@ -176,8 +177,14 @@ __device__ __forceinline__ uint32_t join_count_row(const JoinSpec& S, const KO* 
       if (e) atomicOr(err, e);
     }
   }
-  rowinfo[i] = make_uint4(lo, __float_as_uint(otags[i]), (uint32_t)rowkey, (uint32_t)(rowkey >> 32));
+  if (rowinfo) rowinfo[i] = make_uint4(lo, __float_as_uint(otag), (uint32_t)rowkey, (uint32_t)(rowkey >> 32));
   return d;
+}
+
+template <typename KO>
+__device__ __forceinline__ uint32_t join_count_row(const JoinSpec& S, const KO* __restrict__ okeys, const float* __restrict__ otags, uint32_t i,
+                                                   uint4* __restrict__ rowinfo, uint32_t* __restrict__ err) {
+  return join_count_kv<KO>(S, okeys[i], otags[i], i, rowinfo, err);
 }
 
 template <typename KO>
