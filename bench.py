@@ -277,6 +277,17 @@ def roofline_of(program, prof_all, steps, sorting_route):
         g = big["bytes"] / (big["ms"] / 1e3) / 1e9
         roofline["large_launches"] = {"launches_per_step": big["launches"] / steps, "ms_per_step": big["ms"] / steps,
                                       "achieved": g, "frac": g / peak, "what": "this kernel's launches of at least 48 MB algorithmic bytes (4 M candidates x 12 B) only"}
+    per_cand = traffic_ratios().get((dom, "l2cand"))
+    if big and big["ms"] > 0 and per_cand and mirror_kernel:
+        # second roofline of the large launches: the slots sit in L2 and every candidate reads one at random, so the bytes that
+        # count are L2's.  L2 bytes per candidate from the ncu capture listed in profiles/ncu_traffic_ratios.md (lts__t_bytes.sum of a
+        # large launch over its candidates) x candidates/s measured here, against the L2 bandwidth measured here.
+        from paper_2609_27203_b200 import xlog
+        l2_peak = xlog.copy_bandwidth_gbs(32 << 20, 100)
+        cps = big["bytes"] / 12.0 / (big["ms"] / 1e3)
+        roofline["large_launches"]["l2"] = {"achieved": cps * per_cand / 1e9, "peak": l2_peak, "frac": cps * per_cand / 1e9 / l2_peak, "unit": "GB/s",
+                                            "l2_bytes_per_candidate": per_cand, "candidates_per_s": cps,
+                                            "peak_source": "measured here: xlog_device_copy on a 32 MB buffer pair (L2-resident), read + write bytes"}
     if l2:
         roofline.update(achieved=l2["achieved"], peak=l2["peak"], unit="GB/s", frac=l2["achieved"] / l2["peak"], traffic=None,
                         peak_source="measured here: xlog_device_copy on a 32 MB buffer pair (L2-resident), read + write bytes",
