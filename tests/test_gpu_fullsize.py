@@ -204,6 +204,34 @@ def test_config5_reach_rmat22_full_four_sources_by_oracle():
     pool.shutdown()
 
 
+def test_resident_rounds_over_a_23_bit_key_space():
+    # 128 sources on R-MAT 16: 7 + 16 key bits, the largest class of key space the resident rounds take (up to 2^24) and the
+    # only one whose bitmap tiles are swept four times per block; the graph-driven rounds, the same launched one by one, and
+    # the sorting path must agree bit for bit, and three sources are checked row by row against the oracle
+    from paper_2609_27203_b200 import xlog
+    prog = W.config5(scale=16, n_sources=128)
+    (s, d), w = prog.facts["edge"]
+    srcs = prog.facts["src"][0][0]
+    deg = np.bincount(s, minlength=1 << 16)
+    live = srcs[deg[srcs] > 0]
+    ctx, ids, _, receipt = gpu_fixpoint(prog, 8 << 30)
+    rc, rt = ctx.read(ids["reach"])
+    ctx.close()
+    assert receipt["derived_tuples"] == len(rt) and receipt["kernel_launches"] < 60       # resident: a handful of launches outside the loop
+    ctx, ids, _, r1 = gpu_fixpoint(prog, 8 << 30, xlog.FLAG_NO_GRAPH)
+    c1, t1 = ctx.read(ids["reach"])
+    ctx.close()
+    assert all(np.array_equal(a, b) for a, b in zip(rc, c1)) and np.array_equal(rt.view(np.int32), t1.view(np.int32))
+    for k in ("iterations", "candidates", "new_tuples", "improved_tags", "derived_tuples"):
+        assert receipt[k] == r1[k], k
+    same_on_the_sorting_path(prog, 8 << 30, "reach", rc, rt, receipt)
+    chosen = [int(live[0]), int(live[len(live) // 2]), int(live[-1])]
+    oc, ot = _oracle_reach_rows(prog.facts["edge"], chosen)
+    sel = np.isin(rc[0], np.unique(oc[0]))
+    assert np.array_equal(rc[0][sel], oc[0]) and np.array_equal(rc[1][sel], oc[1])
+    assert np.array_equal(rt[sel].view(np.int32), ot.view(np.int32))
+
+
 def test_mutual_recursion_full_size_against_the_oracle():
     # odd / even walks on configuration 1's graph: two mutually recursive heads, 1.9 M derived tuples, every row by the oracle
     prog = W.mutual_config()
