@@ -439,6 +439,7 @@ def run_ours(args):
                                          "launches_per_fixpoint": o["launches"] / min(args.steps, 5),
                                          "dominant_kernel": r["kernel"], "bound": r["bound"], "achieved": r["achieved"], "unit": r["unit"],
                                          "frac": r["frac"], "large_launches_frac": (r.get("large_launches") or {}).get("frac"),
+                                         "large_launches_l2_frac": ((r.get("large_launches") or {}).get("l2") or {}).get("frac"),
                                          "clocks": o["clocks"]}
         out["configs"] = others
 
