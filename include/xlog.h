@@ -280,6 +280,17 @@ xlog_status xlog_profile_reset(xlog_ctx* ctx);
  * on a buffer pair smaller than L2 to obtain the L2 bandwidth that cache-resident kernels (the sorted-list intersections
  * of the triangle and four-cycle joins) are reported against, and on a large pair as a cross-check of the HBM figure. */
 xlog_status xlog_device_copy(void* stream, void* dst, const void* src, uint64_t bytes, int32_t repeats);
+/* The read-only counterpart: reads `bytes` (a multiple of 16; src DEVICE, 16-byte aligned) `repeats` times, eight 16-byte loads
+ * per thread in flight, and writes nothing (`sink`: 4 writable DEVICE bytes, 4-byte aligned, that keep the loads alive; they
+ * are stored to only if the XOR of a thread's words takes one particular value).  The join kernels that are held against the
+ * L2 rate mostly read, so the benchmark reports them against the higher of the two figures.  Same error behaviour as above:
+ * XLOG_ERR_INVALID_ARGUMENT for a null or misaligned pointer, a size that is not a multiple of 16 or repeats < 1. */
+xlog_status xlog_device_read(void* stream, const void* src, uint64_t bytes, int32_t repeats, void* sink);
+/* Random reads: at least `reads` 4-byte loads (rounded up to a multiple of 8 per thread of a fixed grid) at hashed word
+ * offsets of the `bytes`-byte table at src (DEVICE, 4-byte aligned, 4 <= bytes <= 2^34, a multiple of 4), eight per thread
+ * in flight; nothing is written (`sink` as above).  Each load touches one 32-byte sector: the rate is what the row-wise
+ * tag-mirror join (one table slot per candidate) is held against. */
+xlog_status xlog_device_gather(void* stream, const void* src, uint64_t bytes, uint64_t reads, void* sink);
 
 /* ---- failure-path hooks (tests only) -----------------------------------------------------
  * Two kernels wait for other thread blocks of their own launch: the sort pass and the resident count + scan look back

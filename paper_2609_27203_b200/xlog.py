@@ -34,7 +34,7 @@ PLAN_NONE, PLAN_WCOJ, PLAN_CHAIN = 0, 1, 2
 EXPORTS = ["xlog_ctx_create", "xlog_ctx_destroy", "xlog_last_error", "xlog_relation_create", "xlog_relation_load",
            "xlog_relation_size", "xlog_relation_read", "xlog_relation_view", "xlog_rule_add", "xlog_fixpoint",
            "xlog_ctx_reset_idb", "xlog_rule_backward", "xlog_profile_read", "xlog_profile_reset",
-           "xlog_reduce_by_key_static", "xlog_sort_pairs", "xlog_debug_set_poll_limit", "xlog_debug_sort_pass_without_first_tile", "xlog_device_copy"]
+           "xlog_reduce_by_key_static", "xlog_sort_pairs", "xlog_debug_set_poll_limit", "xlog_debug_sort_pass_without_first_tile", "xlog_device_copy", "xlog_device_read", "xlog_device_gather"]
 
 
 class XlogError(RuntimeError):
@@ -112,6 +112,8 @@ def lib():
         L.xlog_profile_reset.argtypes = [vp]
         L.xlog_sort_pairs.argtypes = [vp, vp, vp, i64, i32, i32]
         L.xlog_device_copy.argtypes = [vp, vp, vp, C.c_uint64, i32]
+        L.xlog_device_read.argtypes = [vp, vp, C.c_uint64, i32, vp]
+        L.xlog_device_gather.argtypes = [vp, vp, C.c_uint64, C.c_uint64, vp]
         L.xlog_debug_set_poll_limit.argtypes = [vp, C.c_uint32]
         L.xlog_debug_sort_pass_without_first_tile.argtypes = [vp, vp, vp, vp, vp, i64, i32]
         L.xlog_reduce_by_key_static.argtypes = [vp, i32, vp, vp, i64, vp, vp, C.POINTER(i64), C.c_char_p, C.c_size_t]
@@ -348,6 +350,47 @@ def copy_bandwidth_gbs(n_bytes: int, repeats: int = 50, device: int = 0) -> floa
         e1.record(s)
         e1.synchronize()
         return 2.0 * n_bytes * repeats / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+
+def read_bandwidth_gbs(n_bytes: int, repeats: int = 50, device: int = 0) -> float:
+    """GB/s (bytes read) of the library's own read-only kernel on a buffer of n_bytes: the L2 read rate when it fits L2."""
+    import torch
+    with torch.cuda.device(device):
+        a = torch.empty(n_bytes, dtype=torch.uint8, device=f"cuda:{device}").fill_(1)
+        sink = torch.zeros(1, dtype=torch.int32, device=f"cuda:{device}")
+        s = torch.cuda.current_stream(device)
+        L = lib()
+        if L.xlog_device_read(s.cuda_stream, a.data_ptr(), n_bytes, 5, sink.data_ptr()):
+            raise XlogError(9, "xlog_device_read failed")
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(s)
+        if L.xlog_device_read(s.cuda_stream, a.data_ptr(), n_bytes, repeats, sink.data_ptr()):
+            raise XlogError(9, "xlog_device_read failed")
+        e1.record(s)
+        e1.synchronize()
+        return 1.0 * n_bytes * repeats / (e0.elapsed_time(e1) * 1e-3) / 1e9
+
+
+def gather_rate(n_bytes: int, reads: int = 1 << 28, device: int = 0) -> float:
+    """Random 4-byte reads per second from a table of n_bytes with the library's own gather kernel (each read touches one
+    32-byte sector): with a table that fits L2, the rate a kernel that reads one table slot per unit of work can reach."""
+    import torch
+    with torch.cuda.device(device):
+        a = torch.empty(n_bytes, dtype=torch.uint8, device=f"cuda:{device}").fill_(1)
+        sink = torch.zeros(1, dtype=torch.int32, device=f"cuda:{device}")
+        s = torch.cuda.current_stream(device)
+        L = lib()
+        threads = 148 * 8 * 256
+        done = ((reads + threads - 1) // threads + 7) // 8 * 8 * threads
+        if L.xlog_device_gather(s.cuda_stream, a.data_ptr(), n_bytes, reads // 8, sink.data_ptr()):
+            raise XlogError(9, "xlog_device_gather failed")
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(s)
+        if L.xlog_device_gather(s.cuda_stream, a.data_ptr(), n_bytes, reads, sink.data_ptr()):
+            raise XlogError(9, "xlog_device_gather failed")
+        e1.record(s)
+        e1.synchronize()
+        return done / (e0.elapsed_time(e1) * 1e-3)
 
 
 def check_load_shapes(cols, tags, device) -> int:

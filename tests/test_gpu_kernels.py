@@ -78,3 +78,30 @@ def test_a_look_back_wait_that_runs_out_fails_the_call_and_leaves_the_context_us
     ctx.rule(p_rel, [(0, {0: 1}), (0, {2: 1})], [(p_rel, [("v", 0, 1, 0), ("v", 1, 1, 0)]), (e_rel, [("v", 1, 1, 0), ("v", 2, 1, 0)])])
     assert ctx.fixpoint()["derived_tuples"] == 3
     ctx.close()
+
+
+def test_bandwidth_probe_kernels_copy_exactly_and_write_nothing_else():
+    # the measuring kernels of the benchmark: the copy must copy, the two read-only probes must leave their sink untouched
+    import torch
+    from paper_2609_27203_b200 import xlog
+    L = xlog.lib()
+    s = torch.cuda.current_stream()
+    n = (3 << 20) + 48                                            # a ragged tail of three 16-byte words
+    src = torch.from_numpy(synth.randint(3, 1, 0, n // 4, 1 << 30).astype(np.int32)).cuda()
+    dst = torch.zeros_like(src)
+    assert L.xlog_device_copy(s.cuda_stream, dst.data_ptr(), src.data_ptr(), n, 2) == 0
+    torch.cuda.synchronize()
+    assert torch.equal(src, dst)
+    sink = torch.zeros(1, dtype=torch.int32, device="cuda")
+    assert L.xlog_device_read(s.cuda_stream, src.data_ptr(), n, 20, sink.data_ptr()) == 0
+    assert L.xlog_device_gather(s.cuda_stream, src.data_ptr(), n, 1 << 20, sink.data_ptr()) == 0
+    torch.cuda.synchronize()
+    assert int(sink.item()) == 0 and torch.equal(src, dst)
+    # bad arguments are refused before any launch
+    assert L.xlog_device_copy(s.cuda_stream, dst.data_ptr(), src.data_ptr(), n + 4, 1) == 1
+    assert L.xlog_device_read(s.cuda_stream, src.data_ptr() + 4, n - 16, 1, sink.data_ptr()) == 1
+    assert L.xlog_device_read(s.cuda_stream, src.data_ptr(), n, 0, sink.data_ptr()) == 1
+    assert L.xlog_device_gather(s.cuda_stream, src.data_ptr(), 0, 8, sink.data_ptr()) == 1
+    assert L.xlog_device_gather(s.cuda_stream, None, n, 8, sink.data_ptr()) == 1
+    for rate in (xlog.copy_bandwidth_gbs(8 << 20, 4), xlog.read_bandwidth_gbs(8 << 20, 16), xlog.gather_rate(8 << 20, 1 << 22)):
+        assert rate > 0
