@@ -178,7 +178,9 @@ xlog_status xlog_relation_view(xlog_ctx* ctx, xlog_rel rel, const int32_t** cols
  * connected components of the relation dependency graph; a rule may have one or two
  * recursive atoms (p(x,z) :- p(x,y), p(y,z) is evaluated with one delta variant per
  * occurrence, Section "Semi-naive evaluation on GPU"), and a component may hold
- * several mutually recursive relations.
+ * several mutually recursive relations (MAXPLUS / MINPLUS heads whose rules each read one
+ * relation of the component are evaluated over one tag mirror per head, see below; other
+ * shapes by sort, reduce-by-key and merge).
  * Tags inside recursion: a component of MAXPLUS / MINPLUS relations runs Algorithm 1 with tag
  * improvement (a tuple re-enters the delta when its tag strictly improves).  A component of
  * LOGSUMEXP or SUMPROD relations (Section "Aggregations and constraints" rejects aggregation

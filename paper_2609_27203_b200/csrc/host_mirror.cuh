@@ -678,5 +678,169 @@ void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs
   }
 }
 
+// ---- several heads in one component (mutual recursion) ----------------------------------------------------------------
+constexpr int kMultiMaxHeads = 8;
+constexpr int kSlotMultiChanged = 32, kSlotMultiNew = 40;     // per head: changed keys of the round, running count of new keys
+static_assert(kSlotMultiNew + kMultiMaxHeads <= kSlotResState, "control words overlap");
+
+// Mutually recursive max / min heads, each over its own tag mirror, when every rule reads at most one relation of the
+// component (so the looked-up side of every join is a relation of a lower stratum, indexed once).
+bool mirror_multi_applies(Ctx* c, const std::vector<int>& comp, const std::vector<const RuleC*>& rs) {
+  if ((c->flags & XLOG_FLAG_NO_TAG_MIRROR) || comp.size() < 2 || comp.size() > (size_t)kMultiMaxHeads) return false;
+  uint64_t need = 1u << 20;
+  for (int h : comp) {
+    const Relation& H = *c->rels[h];
+    if (H.sr != XLOG_SR_MAXPLUS && H.sr != XLOG_SR_MINPLUS) return false;
+    if (H.layout.total_bits > kMirrorMaxBits || H.key_bytes != 4) return false;
+    need += ((uint64_t)4 << H.layout.total_bits) + ((uint64_t)1 << H.layout.total_bits) / 4 + (1u << 16);
+  }
+  for (const RuleC* r : rs) {
+    if (r->plan.emit_count_column || (r->kind != 1 && r->kind != 2)) return false;
+    int in = 0, pos = 0;
+    for (int j = 0; j < r->plan.n_atoms; ++j)
+      if (in_set(comp, r->plan.atoms[j].rel)) { if (r->plan.atoms[j].negated) return false; ++in; pos = j; }
+    if (in > 1) return false;
+    if (in == 1 && r->kind == 2 && !r->shape[pos].ok) return false;
+    if (in == 1 && r->kind != 2 && pos != 0) return false;
+    if (in == 0 && r->kind == 2 && !r->shape[0].ok && !r->shape[1].ok) return false;
+  }
+  return need <= c->arena.largest_free() / 2;
+}
+
+// Algorithm 1 over one tag mirror per head.  A round applies every delta variant of every rule to its head's table (the
+// deltas are lists written at the end of the round before, so all heads see the same state), then each head's changed
+// bitmap becomes its next delta.  Two control reads per round: the variants' candidate totals, the heads' changed counts.
+void stratum_recursive_mirror_multi(Ctx* c, const std::vector<int>& comp, const std::vector<const RuleC*>& rs) {
+  struct Head {
+    int h; Relation* H; bool is_max; int32_t empty; uint64_t slots; uint32_t bm_quads; unsigned ch_tiles;
+    DevBuf table, bitmap, present, ch_sums;
+    KeyTags delta; uint32_t n_start; uint64_t total_new; MirrorArgs mr;
+  };
+  std::vector<Head> heads(comp.size());
+  zero_ctrl(c, kSlotMultiChanged, 2 * kMultiMaxHeads);
+  for (size_t i = 0; i < comp.size(); ++i) {
+    Head& X = heads[i];
+    X.h = comp[i]; X.H = c->rels[comp[i]];
+    Relation& H = *X.H;
+    const uint64_t dom = (uint64_t)1 << H.layout.total_bits;
+    X.is_max = H.sr == XLOG_SR_MAXPLUS;
+    X.empty = X.is_max ? kMirrorEmptyMax : kMirrorEmptyMin;
+    X.slots = std::max<uint64_t>(dom, 4);
+    X.bm_quads = (uint32_t)((std::max<uint64_t>(dom / 32, 1) + 3) / 4);
+    X.ch_tiles = mirror_tiles(X.bm_quads * 4);
+    X.table = DevBuf(c, X.slots * 4); X.bitmap = DevBuf(c, (size_t)X.bm_quads * 16); X.present = DevBuf(c, (size_t)X.bm_quads * 16);
+    X.ch_sums = DevBuf(c, (size_t)X.ch_tiles * 4);
+    X.n_start = H.n; X.total_new = 0;
+    XLOG_LAUNCH(c, k_fill_i32, grid_for(X.slots, 256 * 8), 256, 0, X.table.as<int32_t>(), X.slots, X.empty);
+    XLOG_CUDA(cudaMemsetAsync(X.bitmap.p, 0, (size_t)X.bm_quads * 16, c->stream));
+    XLOG_CUDA(cudaMemsetAsync(X.present.p, 0, (size_t)X.bm_quads * 16, c->stream));
+    if (X.n_start)
+      XLOG_LAUNCH(c, (k_mirror_scatter<uint32_t>), grid_for(X.n_start, 256, 1 << 30), 256, 0, (const uint32_t*)H.keys(), (const float*)H.tags(), X.n_start, H.layout,
+                  H.layout, X.table.as<int32_t>(), X.present.as<uint32_t>());
+    X.mr = MirrorArgs{X.table.as<int32_t>(), X.bitmap.as<uint32_t>(), (unsigned long long*)(c->d_ctrl + kSlotMultiNew + i), (uint32_t)(dom - 1),
+                      ctrl_u32(c, kSlotErr)};
+  }
+  c->unique_untracked = true;
+  auto head_of = [&](int rel) -> Head& { for (Head& X : heads) if (X.h == rel) return X; return heads[0]; };
+  for (int64_t round = 0;; ++round) {
+    if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
+    ++c->r_iterations;
+    std::vector<Variant> vs;
+    for (const RuleC* r : rs) {
+      if (round == 0) {                                     // seed: every atom reads the full relation
+        const int outer = seed_outer(comp, r);
+        vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])});
+      } else {
+        for (int j = 0; j < r->plan.n_atoms; ++j) {
+          const int ar = r->plan.atoms[j].rel;
+          if (!in_set(comp, ar)) continue;
+          const Head& D = head_of(ar);
+          if (D.delta.n) vs.push_back(Variant{r, j, Source{D.delta.keys.p, D.delta.tags.as<float>(), D.delta.n, D.H->layout, D.H->key_bytes}});
+        }
+      }
+    }
+    // the candidate totals of a round's variants are settled sixteen at a time, by one control read
+    uint64_t total = 0;
+    for (size_t v0 = 0; v0 < vs.size(); v0 += 16) {
+      std::vector<Counted> counted;
+      std::vector<Head*> target;
+      counted.reserve(16);
+      for (size_t v = v0; v < std::min(vs.size(), v0 + 16); ++v) {
+        if (vs[v].outer.n == 0) continue;
+        Head& T = head_of(vs[v].rule->plan.head_rel);
+        counted.emplace_back();
+        count_variant(c, vs[v], *T.H, counted.back(), kSlotTotals + (int)counted.size() - 1);
+        target.push_back(&T);
+      }
+      if (counted.empty()) continue;
+      sync_ctrl(c);
+      for (size_t i = 0; i < counted.size(); ++i) {
+        Counted& q = counted[i];
+        q.total = c->h_ctrl[q.slot];
+        q.deg.reset(); q.sums.reset();
+        total += q.total;
+        c->r_candidates += (int64_t)q.total;
+        if (q.total) {
+          c->note_bytes = (int64_t)q.total * (4 + (q.spec.has_inner ? 4 * (q.spec.inner_free + 1) : 0));
+          launch_expand_mirror(c, q, target[i]->is_max, target[i]->mr);
+        }
+      }
+    }
+    if (total == 0) break;
+    for (size_t i = 0; i < heads.size(); ++i) {
+      Head& X = heads[i];
+      launch_changed_count(c, X.bitmap.as<uint32_t>(), X.present.as<uint32_t>(), X.bm_quads * 4, X.ch_tiles, X.ch_sums.as<uint32_t>(), X.mr.n_new);
+      XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, X.ch_sums.as<uint32_t>(), (int64_t)X.ch_tiles, ctrl_u32(c, kSlotMultiChanged + (int)i));
+    }
+    sync_ctrl(c);
+    uint64_t changed_all = 0;
+    for (size_t i = 0; i < heads.size(); ++i) {
+      Head& X = heads[i];
+      const uint32_t changed = (uint32_t)c->h_ctrl[kSlotMultiChanged + i];
+      const uint64_t n_new = c->h_ctrl[kSlotMultiNew + i] - X.total_new;
+      X.total_new += n_new;
+      c->r_new += (int64_t)n_new; c->r_improved += (int64_t)changed - (int64_t)n_new;
+      changed_all += changed;
+      X.delta = KeyTags();
+      X.delta.n = changed;
+      if (changed == 0) continue;
+      X.delta.keys = DevBuf(c, (size_t)changed * 4);
+      X.delta.tags = DevBuf(c, (size_t)changed * 4);
+      c->note_bytes = (int64_t)X.bm_quads * 16 + (int64_t)changed * 12;
+      launch_changed_emit(c, X.bitmap.as<uint32_t>(), X.bm_quads * 4, X.ch_tiles, X.ch_sums.as<uint32_t>(), X.table.as<int32_t>(), X.delta.keys.as<uint32_t>(),
+                          X.delta.tags.as<float>(), nullptr);
+    }
+    if (changed_all == 0) break;
+  }
+  // every head in sorted form: the occupied slots in slot order
+  for (Head& X : heads) {
+    Relation& H = *X.H;
+    X.delta = KeyTags();
+    const uint64_t n_out = (uint64_t)X.n_start + X.total_new;
+    KeyTags full;
+    full.n = (uint32_t)n_out;
+    full.keys = DevBuf(c, (size_t)std::max<uint64_t>(n_out, 1) * 4);
+    full.tags = DevBuf(c, (size_t)std::max<uint64_t>(n_out, 1) * 4);
+    if (n_out) {
+      const uint64_t nquads = X.slots / 4;
+      const unsigned tiles = (unsigned)((X.slots + kMirSlotsPerTile - 1) / kMirSlotsPerTile);
+      DevBuf sums(c, (size_t)tiles * 4);
+      c->note_bytes = (int64_t)X.slots * 4;
+      XLOG_LAUNCH(c, k_mirror_full_count, tiles, kMirBlock, 0, (const int4*)X.table.as<int4>(), nquads, X.empty, sums.as<uint32_t>());
+      XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, sums.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotA));
+      c->note_bytes = (int64_t)X.slots * 4 + (int64_t)n_out * 8;
+      XLOG_LAUNCH(c, (k_mirror_full_emit<uint32_t>), tiles, kMirBlock, 0, (const int4*)X.table.as<int4>(), nquads, X.empty, (const uint32_t*)sums.as<uint32_t>(), H.layout,
+                  H.layout, full.keys.as<uint32_t>(), full.tags.as<float>());
+    }
+    set_current(H, std::move(full));
+    X.table.reset(); X.bitmap.reset(); X.present.reset(); X.ch_sums.reset();
+    if (c->flags & XLOG_FLAG_CHECK_INVARIANTS) {
+      XLOG_LAUNCH(c, (k_check_sorted<uint32_t>), grid_for(H.n, 256), 256, 0, (const uint32_t*)H.keys(), (int64_t)H.n, ctrl_u32(c, kSlotErr));
+      sync_ctrl(c);
+      if (n_out && (uint64_t)(uint32_t)c->h_ctrl[kSlotA] != n_out) fail(XLOG_ERR_INTERNAL, "tag mirror: occupied slots disagree with the tuple count");
+    }
+  }
+}
+
 }  // namespace
 }  // namespace xlog

@@ -106,6 +106,7 @@ void stratum_recursive(Ctx* c, const std::vector<int>& comp, const std::vector<c
   }
   if (additive) { stratum_recursive_additive(c, comp, rs); return; }
   if (mirror_applies(c, comp, rs)) { stratum_recursive_mirror(c, comp[0], rs); return; }
+  if (mirror_multi_applies(c, comp, rs)) { stratum_recursive_mirror_multi(c, comp, rs); return; }
   std::vector<KeyTags> delta(c->rels.size());
   for (int64_t round = 0;; ++round) {
     if (round >= c->max_iter) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
