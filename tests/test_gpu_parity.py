@@ -249,6 +249,44 @@ def test_non_linear_and_mutual_recursion():
     check_program(mut)
 
 
+def test_mutual_recursion_over_one_tag_mirror_per_head():
+    # three heads in one component, each rule reading one of them: a one-atom copy rule, heads of different arity, a head
+    # that starts with loaded facts (some better, some worse than what gets derived), and a MAXPLUS head beside MINPLUS ones
+    # (each head combines with its own oplus; the component has no cycle of positive max-plus weight)
+    from paper_2609_27203_b200 import xlog
+    n, m = 400, 1500
+    s, d = synth.uniform_digraph(n, m, 77)
+    w = (1 + 9 * synth.uniform01(77, 2, 0, m)).astype(np.float32)
+    seeds = np.array([0, 5, 9], np.int32)
+    start = np.array([3, 17, 200], np.int32)
+    prog = W.Program("three_heads", {"e": (2, W.MINPLUS), "src": (1, W.MINPLUS), "a": (2, W.MINPLUS), "b": (2, W.MINPLUS), "far": (1, W.MINPLUS)},
+                     [W.Rule("a", (W.V(0), W.V(0)), (W.Atom("src", (W.Var(0),)),)),
+                      W.Rule("b", (W.V(0), W.V(2)), (W.Atom("a", (W.Var(0), W.Var(1))), W.Atom("e", (W.Var(1), W.Var(2))))),
+                      W.Rule("a", (W.V(0), W.V(2)), (W.Atom("b", (W.Var(0), W.Var(1))), W.Atom("e", (W.Var(1), W.Var(2))))),
+                      W.Rule("far", (W.V(1),), (W.Atom("b", (W.Var(0), W.Var(1))),)),
+                      W.Rule("a", (W.Affine(0, ()), W.V(0)), (W.Atom("far", (W.Var(0),)),))],
+                     {"e": ([s, d], w), "src": ([seeds], None),
+                      "far": ([start], np.array([0.5, 1000.0, 2.0], np.float32))}, ("a", "b", "far"))
+    r, stats = check_program(prog)
+    assert r["iterations"] == stats["iterations"] and r["iterations"] > 3
+    # the default route took the mirrors (it does not count distinct candidate keys), the sorting route does
+    ctx, ids, _ = xlog.load_program(prog, arena_bytes=1 << 28)
+    assert ctx.fixpoint()["unique_candidates"] == -1
+    ctx.close()
+    # a max-plus head fed by a min-plus head, on a DAG (edges u < v only) so that the longest walk is finite
+    lo, hi = np.minimum(s, d), np.maximum(s, d)
+    keep = lo != hi
+    key = np.unique(lo[keep].astype(np.int64) * n + hi[keep])
+    s2, d2 = (key // n).astype(np.int32), (key % n).astype(np.int32)
+    w2 = (1 + 9 * synth.uniform01(78, 2, 0, len(s2))).astype(np.float32)
+    mixed = W.Program("min_and_max", {"e": (2, W.MINPLUS), "lo": (2, W.MINPLUS), "hi": (2, W.MAXPLUS)},
+                      [W.Rule("lo", (W.V(0), W.V(1)), (W.Atom("e", (W.Var(0), W.Var(1))),)),
+                       W.Rule("hi", (W.V(0), W.V(2)), (W.Atom("lo", (W.Var(0), W.Var(1))), W.Atom("e", (W.Var(1), W.Var(2))))),
+                       W.Rule("lo", (W.V(0), W.V(2)), (W.Atom("hi", (W.Var(0), W.Var(1))), W.Atom("e", (W.Var(1), W.Var(2)))))],
+                      {"e": ([s2, d2], w2)}, ("lo", "hi"))
+    check_program(mixed)
+
+
 def test_recursion_with_head_arithmetic_takes_the_general_join_path():
     # down(x - 1) :- down(x), pos(x): a negative head constant rules out the linear-key shape, so every route goes through
     # the general per-candidate evaluation (with the tag mirror as sink on the default routes)
