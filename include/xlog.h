@@ -82,6 +82,7 @@ typedef struct {
 #define XLOG_FLAG_NO_GROUPED_JOIN 128u  /* tag mirror: always the row-wise join, never the grouped one (see csrc/group_join.cuh) */
 #define XLOG_FLAG_NO_BITMAP_JOIN  256u  /* tag mirror, grouped join: always from a delta row list, never straight from the changed bitmap (see csrc/bitmap_join.cuh) */
 #define XLOG_FLAG_NO_DENSE_DOUBLING 512u /* tag mirror: the path-doubling rule h(x,z) :- h(x,y), h(y,z) goes through the sorting route, not the dense rounds */
+#define XLOG_FLAG_NO_TRIANGLE_BITMAP 1024u /* fused triangle aggregate: always search the longer list, never mark in(x) in a shared-memory bitmap (see csrc/triangle.cuh) */
 #define XLOG_FLAG_NO_GRAPH        16u  /* resident rounds are launched one by one instead of as one graph with a WHILE node */
 
 /* Evaluation routes of a recursive component (Algorithm 1).  All of them derive the same relation,

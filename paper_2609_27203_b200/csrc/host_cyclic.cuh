@@ -66,15 +66,38 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
   const unsigned it_tiles = (ne1 + kScanTile - 1) / kScanTile;
   DevBuf it_sums(c, (size_t)it_tiles * 4);
   zero_ctrl(c, kSlotA, 4);
-  XLOG_LAUNCH(c, k_tri_plan, grid_for(ne1, 256), 256, 0, G, items.as<uint32_t>(), (unsigned long long*)(c->d_ctrl + kSlotC));
+  // per x: search the longer list, or mark in(x) in a shared-memory bitmap and walk every out(y) against it (triangle.cuh)
+  const bool bitmap_ok = !(c->flags & XLOG_FLAG_NO_TRIANGLE_BITMAP) && in_ix.domain <= kTriBitmapMaxDomain;
+  const int64_t sum_n = std::max<int64_t>(in_ix.domain, 1);
+  DevBuf route_sums(c, bitmap_ok ? (size_t)sum_n * 16 : 16);
+  TriRoute RT{route_sums.as<unsigned long long>(), route_sums.as<unsigned long long>() + (bitmap_ok ? sum_n : 0), bitmap_ok ? 1 : 0};
+  if (bitmap_ok) {
+    XLOG_CUDA(cudaMemsetAsync(route_sums.p, 0, (size_t)sum_n * 16, c->stream));
+    XLOG_LAUNCH(c, k_tri_route_sums, grid_for(E.n, 256), 256, 0, G, route_sums.as<unsigned long long>(), route_sums.as<unsigned long long>() + sum_n);
+  }
+  XLOG_LAUNCH(c, k_tri_plan, grid_for(ne1, 256), 256, 0, G, RT, items.as<uint32_t>(), (unsigned long long*)(c->d_ctrl + kSlotC),
+              (unsigned long long*)(c->d_ctrl + kSlotD));
   XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), it_tiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ne1, it_sums.as<uint32_t>());
   XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, it_sums.as<uint32_t>(), (int64_t)it_tiles, ctrl_u32(c, kSlotB));
   XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), it_tiles, kScanBlock, 0, (const uint32_t*)items.as<uint32_t>(), (int64_t)ne1,
               (const uint32_t*)it_sums.as<uint32_t>(), item_off.as<uint32_t>());
+  // the bitmap kernel's units: the work items of one x in slices (count -> scan; the total arrives with the same control read)
+  const int64_t nd1 = domain + 1;
+  const unsigned un_tiles = (unsigned)((nd1 + kScanTile - 1) / kScanTile);
+  DevBuf units(c, bitmap_ok ? (size_t)nd1 * 4 : 4), unit_off(c, bitmap_ok ? (size_t)nd1 * 4 : 4), un_sums(c, (size_t)un_tiles * 4);
+  if (bitmap_ok) {
+    XLOG_LAUNCH(c, k_tri_unit_count, grid_for(nd1, 256), 256, 0, G, RT, G.out_off, domain, (const uint32_t*)item_off.as<uint32_t>(), units.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_scan_tile_sums<uint32_t, uint32_t>), un_tiles, kScanBlock, 0, (const uint32_t*)units.as<uint32_t>(), nd1, un_sums.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, un_sums.as<uint32_t>(), (int64_t)un_tiles, ctrl_u32(c, kSlotA));
+    XLOG_LAUNCH(c, (k_scan_apply<uint32_t, uint32_t>), un_tiles, kScanBlock, 0, (const uint32_t*)units.as<uint32_t>(), nd1, (const uint32_t*)un_sums.as<uint32_t>(),
+                unit_off.as<uint32_t>());
+  }
   sync_ctrl(c);
   const uint32_t n_items = (uint32_t)c->h_ctrl[kSlotB];
-  const uint64_t walked = c->h_ctrl[kSlotC];               // sorted-list probes of the whole join
-  items.reset(); it_sums.reset();
+  const uint32_t n_units = bitmap_ok ? (uint32_t)c->h_ctrl[kSlotA] : 0u;
+  const uint64_t walked = c->h_ctrl[kSlotC];               // list entries walked by the whole join (one probe each)
+  const uint64_t walked_bitmap = c->h_ctrl[kSlotD];        // those of them the bitmap kernel walks
+  items.reset(); it_sums.reset(); units.reset(); un_sums.reset();
   DevBuf item_edge(c, (size_t)std::max(n_items, 1u) * 4), ecnt(c, (size_t)std::max(n_items, 1u) * 4), eacc(c, (size_t)std::max(n_items, 1u) * sizeof(A));
   DevBuf gcnt(c, (size_t)domain * 4), gtag(c, (size_t)domain * 4), flag(c, (size_t)domain * 4);
   const unsigned scan_tiles = (unsigned)((domain + kScanTile - 1) / kScanTile);
@@ -82,10 +105,21 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
   zero_ctrl(c, kSlotA, 4);
   XLOG_LAUNCH(c, k_tri_item_edges, grid_for(E.n, 256), 256, 0, E.n, (const uint32_t*)item_off.as<uint32_t>(), item_edge.as<uint32_t>());
   // declared work: one 4-byte entry per probe (the walked lists) plus the edge rows; the searches themselves hit L1 / L2
-  c->note_bytes = (int64_t)walked * 4 + (int64_t)E.n * 12;
+  c->note_bytes = (int64_t)(walked - walked_bitmap) * 4 + (int64_t)E.n * 12;
   c->r_candidates += (int64_t)walked;
-  XLOG_LAUNCH(c, (k_tri_edges<Op>), kSMs * 8, 256, 0, G, H.sr == XLOG_SR_SUMPROD ? 1 : 0, n_items, (const uint32_t*)item_off.as<uint32_t>(),
+  XLOG_LAUNCH(c, (k_tri_edges<Op>), kSMs * 8, 256, 0, G, RT, H.sr == XLOG_SR_SUMPROD ? 1 : 0, n_items, (const uint32_t*)item_off.as<uint32_t>(),
               (const uint32_t*)item_edge.as<uint32_t>(), ecnt.as<uint32_t>(), eacc.as<A>());
+  if (n_units) {
+    DevBuf unit(c, (size_t)n_units * 8);
+    XLOG_LAUNCH(c, k_tri_unit_fill, grid_for(domain, 256), 256, 0, G.out_off, domain, (const uint32_t*)item_off.as<uint32_t>(), (const uint32_t*)unit_off.as<uint32_t>(),
+                unit.as<uint2>());
+    const uint32_t words = (uint32_t)((in_ix.domain + 31) / 32);
+    const size_t smem = (size_t)words * 8;
+    c->note_bytes = (int64_t)walked_bitmap * 4;
+    XLOG_CUDA(cudaFuncSetAttribute(k_tri_bitmap<Op>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kTriBitmapMaxDomain / 32 * 8)));
+    XLOG_LAUNCH(c, (k_tri_bitmap<Op>), std::min<unsigned>(n_units, kSMs * 16), 256, smem, G, H.sr == XLOG_SR_SUMPROD ? 1 : 0, n_units, (const uint2*)unit.as<uint2>(),
+                G.out_off, (const uint32_t*)item_off.as<uint32_t>(), (const uint32_t*)item_edge.as<uint32_t>(), words, ecnt.as<uint32_t>(), eacc.as<A>());
+  }
   XLOG_LAUNCH(c, (k_tri_groups<Op>), grid_for((uint64_t)domain * 32, 256, kSMs * 8), 256, 0, G.out_off, domain, (const uint32_t*)item_off.as<uint32_t>(),
               (const uint32_t*)ecnt.as<uint32_t>(), (const A*)eacc.as<A>(), gcnt.as<uint32_t>(), gtag.as<float>(), flag.as<uint32_t>(), ctrl_u32(c, kSlotD),
               ctrl_u32(c, kSlotErr));

@@ -29,12 +29,70 @@ struct TriGraph {
 
 constexpr uint32_t kTriChunk = 1024;     // walked entries per work item (32 sweeps of a warp)
 
+// Two ways to intersect out(y) with in(x).  Search: walk the shorter list, binary-search the longer one (about log2 of its
+// length dependent reads per walked entry).  Bitmap: a block marks in(x) in a shared-memory bitmap (one bit per node, plus
+// a running popcount per word, so that a hit's place in in(x) - needed for its tag - is one popcount away) and its warps
+// walk the out-lists of ALL of x's neighbours y against it: one load and one bit test per walked entry.  The bitmap way
+// walks out(y) even where in(x) is the shorter list, and it pays for building the bitmap, so it is taken per x, from two
+// sums over x's edges that depend on the graph alone: the entries either way would walk.
+constexpr int64_t kTriBitmapMaxDomain = (int64_t)1 << 19;      // nodes: 64 KB of bits and 64 KB of running counts
+constexpr int kTriBitmapUnroll = 8;                            // sweeps of 32 list entries a warp reads before it tests them
+#ifndef XLOG_TRI_UNIT_ITEMS
+#define XLOG_TRI_UNIT_ITEMS 512
+#endif
+constexpr uint32_t kTriUnitItems = XLOG_TRI_UNIT_ITEMS;        // work items per (x, slice) unit of the bitmap kernel
+
+struct TriRoute {
+  const unsigned long long* sum_out;   // per x: sum over its edges (x,y) of |out(y)|            (entries the bitmap way walks)
+  const unsigned long long* sum_min;   // per x: sum over its edges of min(|out(y)|, |in(x)|)    (entries the search way walks)
+  int enabled;
+};
+
+// Measured on R-MAT 18: a searched entry costs 10.2 ps of kernel time, an entry tested against the bitmap 3.9 ps; building
+// costs about the in-list's length plus a scan of the bitmap's words.  The bitmap way is taken where it walks at most
+// kTriBitmapRatioX2 / 2 times the entries of the search way.
+#ifndef XLOG_TRI_BITMAP_RATIO_X2
+#define XLOG_TRI_BITMAP_RATIO_X2 5
+#endif
+constexpr unsigned long long kTriBitmapRatioX2 = XLOG_TRI_BITMAP_RATIO_X2;
+__device__ __forceinline__ bool tri_bitmap_route(const TriGraph& G, const TriRoute& R, int32_t x, uint32_t lb) {
+  if (!R.enabled || lb < 32u) return false;
+  const unsigned long long so = R.sum_out[x], sm = R.sum_min[x];
+  return so >= 8192ull && 2ull * (so + 16ull * lb + 32768ull) < kTriBitmapRatioX2 * sm;
+}
+
+// Per-x sums for the choice above; sums must be zero on entry.  Edges are sorted by x, so a warp's 32 edges mostly share
+// one x: then one lane adds for all.
+static __global__ void __launch_bounds__(256) k_tri_route_sums(TriGraph G, unsigned long long* __restrict__ sum_out, unsigned long long* __restrict__ sum_min) {
+  const uint32_t n32 = (G.n_edges + 31u) & ~31u;
+  for (uint32_t e = blockIdx.x * blockDim.x + threadIdx.x; e < n32; e += gridDim.x * blockDim.x) {
+    int32_t x = -1;
+    uint32_t la = 0, lb = 0;
+    if (e < G.n_edges) {
+      x = G.src[e];
+      const int32_t y = G.dst[e];
+      if (y < G.out_domain) la = G.out_off[y + 1] - G.out_off[y];
+      if (x < G.in_domain) lb = G.in_off[x + 1] - G.in_off[x];
+      if (x >= G.in_domain) x = -1;
+    }
+    const int32_t x0 = __shfl_sync(0xffffffffu, x, 0);
+    if (__all_sync(0xffffffffu, x == x0)) {
+      const unsigned long long a = __reduce_add_sync(0xffffffffu, la), m = __reduce_add_sync(0xffffffffu, min(la, lb));
+      if (lane_id() == 0 && x0 >= 0 && a) { atomicAdd(sum_out + x0, a); atomicAdd(sum_min + x0, m); }
+    } else if (x >= 0 && la) {
+      atomicAdd(sum_out + x, (unsigned long long)la);
+      atomicAdd(sum_min + x, (unsigned long long)min(la, lb));
+    }
+  }
+}
+
 // Work items of the aggregate: an edge whose shorter list has n entries is cut into ceil(n / kTriChunk) items, so that a
 // hub edge (tens of thousands of entries to walk) is shared by many warps instead of serialising one; an edge with an
 // empty list gets none.  items[e] for e < n_edges, items[n_edges] = 0 (so that the exclusive scan has n_edges + 1 entries).
-// *walked accumulates the total number of entries to walk (one sorted-list probe each).
-static __global__ void __launch_bounds__(256) k_tri_plan(TriGraph G, uint32_t* __restrict__ items, unsigned long long* __restrict__ walked) {
-  unsigned long long mine = 0;
+// *walked accumulates the total number of entries to walk (one probe each), *walked_bitmap those of them the bitmap kernel walks.
+static __global__ void __launch_bounds__(256) k_tri_plan(TriGraph G, TriRoute R, uint32_t* __restrict__ items, unsigned long long* __restrict__ walked,
+                                                         unsigned long long* __restrict__ walked_bitmap) {
+  unsigned long long mine = 0, mine_bm = 0;
   for (uint32_t e = blockIdx.x * blockDim.x + threadIdx.x; e <= G.n_edges; e += gridDim.x * blockDim.x) {
     uint32_t n = 0;
     if (e < G.n_edges) {
@@ -42,14 +100,19 @@ static __global__ void __launch_bounds__(256) k_tri_plan(TriGraph G, uint32_t* _
       uint32_t la = 0, lb = 0;
       if (y < G.out_domain) la = G.out_off[y + 1] - G.out_off[y];
       if (x < G.in_domain) lb = G.in_off[x + 1] - G.in_off[x];
-      n = (min(la, lb) + kTriChunk - 1) / kTriChunk;
-      mine += min(la, lb);
+      // the bitmap way walks out(y) whichever list is shorter
+      const bool bm = lb && tri_bitmap_route(G, R, x, lb);
+      const uint32_t w = bm ? la : min(la, lb);
+      n = (w + kTriChunk - 1) / kTriChunk;
+      mine += w;
+      if (bm) mine_bm += w;
     }
     items[e] = n;
   }
 #pragma unroll
-  for (int d = 16; d; d >>= 1) mine += __shfl_down_sync(0xffffffffu, mine, d);
+  for (int d = 16; d; d >>= 1) { mine += __shfl_down_sync(0xffffffffu, mine, d); mine_bm += __shfl_down_sync(0xffffffffu, mine_bm, d); }
   if (lane_id() == 0 && mine) atomicAdd(walked, mine);
+  if (lane_id() == 0 && mine_bm) atomicAdd(walked_bitmap, mine_bm);
 }
 
 // item -> edge, written by the edge (item_off = exclusive scan of items)
@@ -60,7 +123,7 @@ static __global__ void __launch_bounds__(256) k_tri_item_edges(uint32_t n_edges,
 
 // One warp per work item: partial count and aggregate of its slice of the walked list.
 template <typename Op>
-__global__ void __launch_bounds__(256) k_tri_edges(TriGraph G, int times, uint32_t n_items, const uint32_t* __restrict__ item_off,
+__global__ void __launch_bounds__(256) k_tri_edges(TriGraph G, TriRoute R, int times, uint32_t n_items, const uint32_t* __restrict__ item_off,
                                                    const uint32_t* __restrict__ item_edge, uint32_t* __restrict__ item_cnt,
                                                    typename Op::A* __restrict__ item_acc) {
   typedef typename Op::A A;
@@ -75,6 +138,7 @@ __global__ void __launch_bounds__(256) k_tri_edges(TriGraph G, int times, uint32
     const uint32_t a0 = G.out_off[y], a1 = G.out_off[y + 1];                   // out(y): candidates z with s(y,z)
     const uint32_t b0 = G.in_off[x], b1 = G.in_off[x + 1];                     // in(x):  candidates z with t(z,x)
     const uint32_t la = a1 - a0, lb = b1 - b0;
+    if (tri_bitmap_route(G, R, x, lb)) continue;                               // k_tri_bitmap's item
     uint32_t cnt = 0;
     A acc = Op::identity();
     const bool walk_a = la <= lb;
@@ -108,6 +172,132 @@ __global__ void __launch_bounds__(256) k_tri_edges(TriGraph G, int times, uint32
       acc = Op::combine(acc, o);
     }
     if (lane == 0) { item_cnt[it] = cnt; item_acc[it] = acc; }
+  }
+}
+
+// Units of the bitmap kernel: the work items of one x in slices of kTriUnitItems.  units[x] for x < domain, units[domain] = 0.
+static __global__ void __launch_bounds__(256) k_tri_unit_count(TriGraph G, TriRoute R, const uint32_t* __restrict__ edge_off, int64_t domain,
+                                                               const uint32_t* __restrict__ item_off, uint32_t* __restrict__ units) {
+  for (int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; x <= domain; x += (int64_t)gridDim.x * blockDim.x) {
+    uint32_t n = 0;
+    if (x < domain && x < G.in_domain) {
+      const uint32_t lb = G.in_off[x + 1] - G.in_off[x];
+      if (lb && tri_bitmap_route(G, R, (int32_t)x, lb)) n = (item_off[edge_off[x + 1]] - item_off[edge_off[x]] + kTriUnitItems - 1) / kTriUnitItems;
+    }
+    units[x] = n;
+  }
+}
+
+// unit -> (x, first item), written by the x (unit_off = exclusive scan of units)
+static __global__ void __launch_bounds__(256) k_tri_unit_fill(const uint32_t* __restrict__ edge_off, int64_t domain, const uint32_t* __restrict__ item_off,
+                                                              const uint32_t* __restrict__ unit_off, uint2* __restrict__ unit) {
+  for (int64_t x = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; x < domain; x += (int64_t)gridDim.x * blockDim.x) {
+    const uint32_t u0 = unit_off[x], u1 = unit_off[x + 1];
+    const uint32_t first = item_off[edge_off[x]];
+    for (uint32_t u = u0; u < u1; ++u) unit[u] = make_uint2((uint32_t)x, first + (u - u0) * kTriUnitItems);
+  }
+}
+
+// One block per unit: mark in(x), then the block's warps walk the unit's work items (slices of the out-lists of x's
+// neighbours) against the bitmap, warp w taking items w, w + 8, ...  Hits are rare among the walked entries (one in ten),
+// so a warp does not combine them where they fall: it queues them in shared memory, in entry order, and reads their tags
+// and folds them 32 at a time, a lane each.  A warp's partial result covers all its items of the unit; it is written to the first of them, the
+// others get the identity (the per-x combination that follows reads every item of x anyway).  The assignment of entries to
+// lanes depends on the graph alone, so results repeat from run to run.  Dynamic shared memory: 2 * words * 4 bytes (bits,
+// then the running count of set bits before each word).
+template <typename Op>
+__global__ void __launch_bounds__(256) k_tri_bitmap(TriGraph G, int times, uint32_t n_units, const uint2* __restrict__ unit, const uint32_t* __restrict__ edge_off,
+                                                    const uint32_t* __restrict__ item_off, const uint32_t* __restrict__ item_edge, uint32_t words,
+                                                    uint32_t* __restrict__ item_cnt, typename Op::A* __restrict__ item_acc) {
+  typedef typename Op::A A;
+  extern __shared__ uint32_t tri_smem[];
+  __shared__ uint32_t sh[256 / 32 + 1];
+  __shared__ uint2 s_queue[8][64];
+  uint32_t* bits = tri_smem;
+  uint32_t* before = tri_smem + words;
+  const unsigned lane = lane_id(), wid = warp_id();
+  uint2* queue = s_queue[wid];
+  int32_t have = -1;                                                         // the x whose in-list the bitmap holds
+  for (uint32_t u = blockIdx.x; u < n_units; u += gridDim.x) {
+    const int32_t x = (int32_t)unit[u].x;
+    const uint32_t b0 = G.in_off[x], b1 = G.in_off[x + 1];
+    if (x != have) {
+      __syncthreads();
+      for (uint32_t i = threadIdx.x; i < words; i += 256) bits[i] = 0u;
+      __syncthreads();
+      for (uint32_t i = b0 + threadIdx.x; i < b1; i += 256) { const uint32_t z = (uint32_t)G.in_src[i]; atomicOr(bits + (z >> 5), 1u << (z & 31)); }
+      __syncthreads();
+      // running count of set bits before each word: 256 words per step (a thread a word: no bank conflicts), a block-wide prefix per step
+      uint32_t carry = 0;
+      for (uint32_t i0 = 0; i0 < words; i0 += 256) {
+        const uint32_t i = i0 + threadIdx.x;
+        const uint32_t v = i < words ? __popc(bits[i]) : 0u;
+        uint32_t total;
+        const uint32_t ex = block_scan_excl<256, uint32_t>(v, sh, total);
+        if (i < words) before[i] = carry + ex;
+        carry += total;
+      }
+      __syncthreads();
+      have = x;
+    }
+    const uint32_t it_lo = unit[u].y, it_end = min(it_lo + kTriUnitItems, item_off[edge_off[x + 1]]);
+    uint32_t cnt = 0;                                                          // hits so far (uniform across the warp)
+    A acc = Op::identity();
+    for (uint32_t it = it_lo + wid; it < it_end; it += 8) {
+      const uint32_t e = item_edge[it];
+      const uint32_t first = (it - item_off[e]) * kTriChunk;
+      const int32_t y = G.dst[e];
+      const float wxy = G.w[e];
+      const uint32_t a0 = G.out_off[y], a1 = G.out_off[y + 1];
+      const uint32_t last = min(first + kTriChunk, a1 - a0);
+      if (it != it_lo + wid && lane == 0) { item_cnt[it] = 0u; item_acc[it] = Op::identity(); }
+      uint32_t qn = 0;                                                         // queued hits of this item (uniform across the warp)
+      // kTriBitmapUnroll sweeps at a time: their list reads are in flight together
+      for (uint32_t i0 = first; i0 < last; i0 += 32 * kTriBitmapUnroll) {
+        uint32_t z[kTriBitmapUnroll];
+#pragma unroll
+        for (int k = 0; k < kTriBitmapUnroll; ++k) {
+          const uint32_t i = i0 + k * 32 + lane;
+          z[k] = i < last ? (uint32_t)__ldcs(G.s_dst + a0 + i) : 0xffffffffu;
+        }
+#pragma unroll
+        for (int k = 0; k < kTriBitmapUnroll; ++k) {
+          uint32_t wd = 0, bit = 0;
+          if (z[k] < (uint32_t)G.in_domain) { wd = bits[z[k] >> 5]; bit = 1u << (z[k] & 31); }
+          const bool hit = (wd & bit) != 0u;
+          const unsigned m = __ballot_sync(0xffffffffu, hit);
+          if (m == 0) continue;                                                // uniform
+          // a hit is queued as (place of the entry in out(y), place of z in in(x)): its two tags are read when the queue is folded
+          if (hit) queue[qn + __popc(m & lanemask_lt())] = make_uint2(a0 + i0 + k * 32 + lane, b0 + before[z[k] >> 5] + __popc(wd & (bit - 1u)));
+          qn += __popc(m);
+          __syncwarp();
+          if (qn >= 32) {                                                      // fold 32 queued hits, a lane each; the rest moves to the front
+            const uint2 h = queue[lane];
+            const float wyz = G.s_w[h.x], wzx = G.in_w[h.y];
+            acc = Op::combine(acc, Op::lift(times ? (wxy * wyz) * wzx : (wxy + wyz) + wzx));
+            const uint2 rest = queue[32 + lane];
+            __syncwarp();
+            queue[lane] = rest;
+            qn -= 32;
+            cnt += 32;
+            __syncwarp();
+          }
+        }
+      }
+      if (lane < qn) {                                                         // what is left of this item's hits (the tag of (x,y) changes with the item)
+        const uint2 h = queue[lane];
+        const float wyz = G.s_w[h.x], wzx = G.in_w[h.y];
+        acc = Op::combine(acc, Op::lift(times ? (wxy * wyz) * wzx : (wxy + wyz) + wzx));
+      }
+      cnt += qn;
+      __syncwarp();
+    }
+#pragma unroll
+    for (int d = 16; d; d >>= 1) {
+      const A o = shfl_down(acc, d);
+      acc = Op::combine(acc, o);
+    }
+    if (lane == 0 && it_lo + wid < it_end) { item_cnt[it_lo + wid] = cnt; item_acc[it_lo + wid] = acc; }
   }
 }
 

@@ -53,6 +53,44 @@ def test_triangle_aggregate_ladder(scale):
     ctx.close()
 
 
+def test_triangle_aggregate_bitmap_and_search_ways_agree():
+    # a graph with hubs: a dense core (every ordered pair among the first 96 nodes) plus R-MAT 12 edges, so that the core
+    # nodes' in-lists are marked in the shared-memory bitmap while the rest is searched; both ways against the oracle,
+    # counts equal to the bit, and the run with the bitmap way must really have launched its kernel
+    from paper_2609_27203_b200 import xlog
+    base = W.config3(scale=12)
+    (s, d), w = base.facts["e"]
+    core = 96
+    cs, cd = np.meshgrid(np.arange(core, dtype=np.int32), np.arange(core, dtype=np.int32), indexing="ij")
+    keep = cs != cd
+    s2 = np.concatenate([s, cs[keep]]); d2 = np.concatenate([d, cd[keep]])
+    key, first = np.unique(s2.astype(np.int64) << 32 | d2, return_index=True)
+    s2, d2 = s2[first], d2[first]
+    w2 = synth.normal(12, 5, len(s2)).astype(np.float32)
+    prog = W.triangle_program(s2, d2, w2, name="triangles_core96_rmat12")
+    o, oids, _ = oracle.load_program(prog)
+    o.run("seminaive")
+    want = o.read(oids["tri_agg"])
+    got = {}
+    for flags in (xlog.FLAG_PROFILE, xlog.FLAG_PROFILE | xlog.FLAG_NO_TRIANGLE_BITMAP):
+        ctx, ids, _ = xlog.load_program(prog, arena_bytes=1 << 28, flags=flags)
+        ctx.fixpoint()
+        got[flags] = ctx.read(ids["tri_agg"])
+        H.compare_relations(got[flags], want, abs_tol=LSE_ABS, what="tri_agg")
+        ran = "k_tri_bitmap" in ctx.profile()
+        assert ran == (not flags & xlog.FLAG_NO_TRIANGLE_BITMAP)
+        ctx.close()
+    a, b = got[xlog.FLAG_PROFILE], got[xlog.FLAG_PROFILE | xlog.FLAG_NO_TRIANGLE_BITMAP]
+    assert all(np.array_equal(x, y) for x, y in zip(a[0], b[0]))               # keys and counts
+    assert np.allclose(a[1], b[1], rtol=0, atol=LSE_ABS)
+    # run to run, the bitmap way repeats itself bit for bit
+    ctx, ids, _ = xlog.load_program(prog, arena_bytes=1 << 28)
+    ctx.fixpoint()
+    again = ctx.read(ids["tri_agg"])
+    ctx.close()
+    assert np.array_equal(again[1].view(np.int32), a[1].view(np.int32))
+
+
 @pytest.mark.parametrize("scale", [6, 10, 13])
 def test_materialised_triangles_match_oracle_and_the_fused_aggregate(scale):
     # count -> scan -> materialise over the sorted columns; rows come out sorted by (x,y,z)
