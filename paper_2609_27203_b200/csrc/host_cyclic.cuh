@@ -67,7 +67,9 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
   DevBuf it_sums(c, (size_t)it_tiles * 4);
   zero_ctrl(c, kSlotA, 4);
   // per x: search the longer list, or mark in(x) in a shared-memory bitmap and walk every out(y) against it (triangle.cuh)
-  const bool bitmap_ok = !(c->flags & XLOG_FLAG_NO_TRIANGLE_BITMAP) && in_ix.domain <= kTriBitmapMaxDomain;
+  // the bitmap holds sources of edges into x (values of column 0) and is probed with targets (values of column 1): both ranges must fit
+  const int64_t node_domain = std::max(in_ix.domain, out_ix.domain);
+  const bool bitmap_ok = !(c->flags & XLOG_FLAG_NO_TRIANGLE_BITMAP) && node_domain <= kTriBitmapMaxDomain;
   const int64_t sum_n = std::max<int64_t>(in_ix.domain, 1);
   DevBuf route_sums(c, bitmap_ok ? (size_t)sum_n * 16 : 16);
   TriRoute RT{route_sums.as<unsigned long long>(), route_sums.as<unsigned long long>() + (bitmap_ok ? sum_n : 0), bitmap_ok ? 1 : 0};
@@ -113,7 +115,7 @@ void triangle_aggregate_t(Ctx* c, Relation& H, const RuleC& r) {
     DevBuf unit(c, (size_t)n_units * 8);
     XLOG_LAUNCH(c, k_tri_unit_fill, grid_for(domain, 256), 256, 0, G.out_off, domain, (const uint32_t*)item_off.as<uint32_t>(), (const uint32_t*)unit_off.as<uint32_t>(),
                 unit.as<uint2>());
-    const uint32_t words = (uint32_t)((in_ix.domain + 31) / 32);
+    const uint32_t words = (uint32_t)((node_domain + 31) / 32);
     const size_t smem = (size_t)words * 8;
     c->note_bytes = (int64_t)walked_bitmap * 4;
     XLOG_CUDA(cudaFuncSetAttribute(k_tri_bitmap<Op>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(kTriBitmapMaxDomain / 32 * 8)));

@@ -35,7 +35,7 @@ constexpr uint32_t kTriChunk = 1024;     // walked entries per work item (32 swe
 // walk the out-lists of ALL of x's neighbours y against it: one load and one bit test per walked entry.  The bitmap way
 // walks out(y) even where in(x) is the shorter list, and it pays for building the bitmap, so it is taken per x, from two
 // sums over x's edges that depend on the graph alone: the entries either way would walk.
-constexpr int64_t kTriBitmapMaxDomain = (int64_t)1 << 19;      // nodes: 64 KB of bits and 64 KB of running counts
+constexpr int64_t kTriBitmapMaxDomain = (int64_t)1 << 19;      // nodes (sources and targets alike): 64 KB of bits and 64 KB of running counts
 constexpr int kTriBitmapUnroll = 8;                            // sweeps of 32 list entries a warp reads before it tests them
 #ifndef XLOG_TRI_UNIT_ITEMS
 #define XLOG_TRI_UNIT_ITEMS 512
@@ -165,6 +165,16 @@ __global__ void __launch_bounds__(256) k_tri_edges(TriGraph G, TriRoute R, int t
         ++cnt;
       }
     }
+    // most work items of a sparse graph end with no hit or with hits in one lane only: skip the combining tree for those
+    const unsigned with_hits = __ballot_sync(0xffffffffu, cnt != 0u);
+    if (with_hits == 0u) {
+      if (lane == 0) { item_cnt[it] = 0u; item_acc[it] = Op::identity(); }
+      continue;
+    }
+    if ((with_hits & (with_hits - 1u)) == 0u) {
+      if (cnt) { item_cnt[it] = cnt; item_acc[it] = acc; }
+      continue;
+    }
 #pragma unroll
     for (int d = 16; d; d >>= 1) {
       cnt += __shfl_down_sync(0xffffffffu, cnt, d);
@@ -263,7 +273,7 @@ __global__ void __launch_bounds__(256) k_tri_bitmap(TriGraph G, int times, uint3
 #pragma unroll
         for (int k = 0; k < kTriBitmapUnroll; ++k) {
           uint32_t wd = 0, bit = 0;
-          if (z[k] < (uint32_t)G.in_domain) { wd = bits[z[k] >> 5]; bit = 1u << (z[k] & 31); }
+          if (z[k] < words * 32u) { wd = bits[z[k] >> 5]; bit = 1u << (z[k] & 31); }
           const bool hit = (wd & bit) != 0u;
           const unsigned m = __ballot_sync(0xffffffffu, hit);
           if (m == 0) continue;                                                // uniform
