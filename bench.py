@@ -244,6 +244,9 @@ def roofline_of(program, prof_all, steps, sorting_route):
         # sorted-list intersections served from L1 / L2 (both orientations of the graph fit L2): unit of work = one probe, a binary
         # search of one walked entry in the other sorted list; the launch site declares 4 bytes per probe plus 12 per edge
         probes = (d["bytes"] - 12.0 * program.info["n_edges"] * d["launches"]) / 4.0
+    if dom == "k_tri_bitmap":
+        # the same intersections against a shared-memory bitmap: one probe = one walked entry tested; 4 bytes declared per probe
+        probes = d["bytes"] / 4.0
     if dom in ("k_cycle4", "k_cycle4_bitmap") and program.info.get("domain", 1 << 30) <= 4096:
         # one probe = one walked entry of the shorter list searched in the other (the bitmap kernel always walks t's out-list of z);
         # both launches (count, write) walk every two-path's list

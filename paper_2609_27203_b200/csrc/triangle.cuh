@@ -222,11 +222,11 @@ __global__ void __launch_bounds__(256) k_tri_bitmap(TriGraph G, int times, uint3
   typedef typename Op::A A;
   extern __shared__ uint32_t tri_smem[];
   __shared__ uint32_t sh[256 / 32 + 1];
-  __shared__ uint2 s_queue[8][64];
+  __shared__ uint32_t s_queue[8][32 * kTriBitmapUnroll + 32];      // a group's hits plus what an earlier group left
   uint32_t* bits = tri_smem;
   uint32_t* before = tri_smem + words;
   const unsigned lane = lane_id(), wid = warp_id();
-  uint2* queue = s_queue[wid];
+  uint32_t* queue = s_queue[wid];
   int32_t have = -1;                                                         // the x whose in-list the bitmap holds
   for (uint32_t u = blockIdx.x; u < n_units; u += gridDim.x) {
     const int32_t x = (int32_t)unit[u].x;
@@ -270,33 +270,40 @@ __global__ void __launch_bounds__(256) k_tri_bitmap(TriGraph G, int times, uint3
           const uint32_t i = i0 + k * 32 + lane;
           z[k] = i < last ? (uint32_t)__ldcs(G.s_dst + a0 + i) : 0xffffffffu;
         }
+        // bit tests of the eight sweeps without a branch; a lane's hits as a bit per sweep
+        uint32_t wd[kTriBitmapUnroll];
+        uint32_t hb = 0;
 #pragma unroll
         for (int k = 0; k < kTriBitmapUnroll; ++k) {
-          uint32_t wd = 0, bit = 0;
-          if (z[k] < words * 32u) { wd = bits[z[k] >> 5]; bit = 1u << (z[k] & 31); }
-          const bool hit = (wd & bit) != 0u;
-          const unsigned m = __ballot_sync(0xffffffffu, hit);
-          if (m == 0) continue;                                                // uniform
-          // a hit is queued as (place of the entry in out(y), place of z in in(x)): its two tags are read when the queue is folded
-          if (hit) queue[qn + __popc(m & lanemask_lt())] = make_uint2(a0 + i0 + k * 32 + lane, b0 + before[z[k] >> 5] + __popc(wd & (bit - 1u)));
-          qn += __popc(m);
-          __syncwarp();
-          if (qn >= 32) {                                                      // fold 32 queued hits, a lane each; the rest moves to the front
-            const uint2 h = queue[lane];
-            const float wyz = G.s_w[h.x], wzx = G.in_w[h.y];
-            acc = Op::combine(acc, Op::lift(times ? (wxy * wyz) * wzx : (wxy + wyz) + wzx));
-            const uint2 rest = queue[32 + lane];
-            __syncwarp();
-            queue[lane] = rest;
-            qn -= 32;
-            cnt += 32;
-            __syncwarp();
-          }
+          wd[k] = z[k] < words * 32u ? bits[z[k] >> 5] : 0u;
+          hb |= ((wd[k] >> (z[k] & 31)) & 1u) << k;
         }
+        if (__ballot_sync(0xffffffffu, hb != 0u) == 0u) continue;              // uniform: no hit in these sweeps
+        // queue places: a warp-wide prefix over the lanes' hit counts; a hit is queued as (place of z in in(x), place of the
+        // entry in this item's slice of out(y)) in one word: its two tags are read when the queue is folded
+        const uint32_t mine = __popc(hb);
+        uint32_t incl = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) { const uint32_t o = __shfl_up_sync(0xffffffffu, incl, d); if ((int)lane >= d) incl += o; }
+        uint32_t at = qn + incl - mine;
+        qn += __shfl_sync(0xffffffffu, incl, 31);
+#pragma unroll
+        for (int k = 0; k < kTriBitmapUnroll; ++k)
+          if ((hb >> k) & 1u)
+            queue[at++] = ((before[z[k] >> 5] + __popc(wd[k] & ((1u << (z[k] & 31)) - 1u))) << 10) | (i0 - first + k * 32 + lane);
+        __syncwarp();
+        while (qn >= 32) {                                                     // fold 32 queued hits, a lane each, from the queue's end
+          const uint32_t h = queue[qn - 32 + lane];
+          const float wyz = G.s_w[a0 + first + (h & 1023u)], wzx = G.in_w[b0 + (h >> 10)];
+          acc = Op::combine(acc, Op::lift(times ? (wxy * wyz) * wzx : (wxy + wyz) + wzx));
+          qn -= 32;
+          cnt += 32;
+        }
+        __syncwarp();
       }
       if (lane < qn) {                                                         // what is left of this item's hits (the tag of (x,y) changes with the item)
-        const uint2 h = queue[lane];
-        const float wyz = G.s_w[h.x], wzx = G.in_w[h.y];
+        const uint32_t h = queue[lane];
+        const float wyz = G.s_w[a0 + first + (h & 1023u)], wzx = G.in_w[b0 + (h >> 10)];
         acc = Op::combine(acc, Op::lift(times ? (wxy * wyz) * wzx : (wxy + wyz) + wzx));
       }
       cnt += qn;
