@@ -505,10 +505,22 @@ inline KeyTags sort_reduce(Ctx* c, int sr, DevBuf& k0, DevBuf& t0, DevBuf& k1, D
                                  : sort_dense_reduce<K, OpMin>(c, k0, t0, k1, t1, n, nbits, defer_slot, presorted_top);
   K* ka = k0.as<K>(); K* kb = k1.as<K>();
   float* ta = t0.as<float>(); float* tb = t1.as<float>();
-  sort_pairs<K>(c, ka, ta, kb, tb, n, nbits);
+  // Candidates that arrive ordered by their top key bits need only their low bits sorted for equal keys to become
+  // neighbours (a stable sort: rows end up ordered by (low, top), each key's candidates in their arrival order, so a
+  // floating-point oplus sees them as the full sort would show them); the groups, far fewer than the candidates,
+  // are then put in key order by a stable sort on the top bits.
+  const bool top_presorted = presorted_top > 0 && presorted_top < nbits && !want_head_pos && defer_slot < 0;
+  sort_pairs<K>(c, ka, ta, kb, tb, n, top_presorted ? nbits - presorted_top : nbits);
   const bool sorted_in_0 = (void*)ka == k0.p;
   KeyTags out = reduce_by_key<K>(c, sr, ka, ta, (uint32_t)n, sorted_in_0 ? &k1 : &k0, sorted_in_0 ? &t1 : &t0, want_head_pos, defer_slot);
   k0.reset(); t0.reset(); k1.reset(); t1.reset();
+  if (top_presorted && out.n > 1) {
+    DevBuf ak(c, (size_t)out.n * sizeof(K)), at(c, (size_t)out.n * 4);
+    K* pk = out.keys.as<K>(); K* qk = ak.as<K>();
+    float* pt = out.tags.as<float>(); float* qt = at.as<float>();
+    sort_pairs<K>(c, pk, pt, qk, qt, out.n, nbits, nbits - presorted_top);
+    if ((void*)pk != out.keys.p) { std::swap(out.keys, ak); std::swap(out.tags, at); }
+  }
   return out;
 }
 

@@ -166,19 +166,23 @@ void count_variant(Ctx* c, const Variant& v, const Relation& H, Counted& q, int 
   q.outer = v.outer;
   q.slot = slot;
   {
-    // Leading head columns that are the leading columns of the scanned atom, in the same order, are carried over
-    // unchanged; the scanned relation is sorted by them (dictionary codes keep the order of the values), so the
-    // candidate stream is already ordered by those key bits.
+    // Leading head columns that follow the leading columns of the scanned atom, in the same order, through strictly
+    // increasing maps (column = mul * v + add with mul >= 1 in the atom, c0 + coef * v with coef >= 1 in the head, v in no
+    // earlier column): the scanned relation is sorted by those columns (dictionary codes keep the order of the values),
+    // equal column values give equal head values and the other way round, so the candidate stream is already ordered by
+    // those key bits.  sum(p, a + b) :- digit(2p, a), digit(2p + 1, b) has its first head column of this kind.
     const xlog_plan& p = v.rule->plan;
     const xlog_atom& A = p.atoms[v.outer_atom];
     const int ka = c->rels[A.rel]->arity;
     int k = 0;
     for (; k < p.n_head_cols && k < ka; ++k) {
-      if (!is_plain_var(A.args[k])) break;
+      if (A.args[k].kind != XLOG_ARG_VAR || A.args[k].mul < 1) break;
       const int var = A.args[k].var;
-      bool id = p.head[k].c0 == 0;
-      for (int w = 0; w < kMaxVars; ++w) id = id && p.head[k].coef[w] == (w == var ? 1 : 0);
-      if (!id) break;
+      bool fresh = true;
+      for (int j = 0; j < k; ++j) fresh = fresh && A.args[j].var != var;
+      bool mono = fresh && p.head[k].coef[var] >= 1;
+      for (int w = 0; w < kMaxVars; ++w) mono = mono && (w == var || p.head[k].coef[w] == 0);
+      if (!mono) break;
     }
     q.presorted_top = k ? q.spec.head.total_bits - q.spec.head.shift[k - 1] : 0;
   }
