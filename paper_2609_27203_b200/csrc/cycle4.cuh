@@ -128,15 +128,21 @@ __global__ void __launch_bounds__(256) k_cycle4(Cycle4 P, const K2* __restrict__
 // The same join with u's in-list of x marked in a shared-memory bitmap.  The two-paths are sorted by x, so a block takes a
 // chunk of them and works through its runs of equal x: mark the in-list (w values below kC4BmWords * 32), then a warp per
 // two-path tests the entries of t's out-list of z against the bitmap (one load and a bit test per probe); only a hit, in
-// the writing launch, is looked up in the in-list by binary search for its tag.  Then the marked words are cleared again.
+// the writing launch, needs its place in the in-list (for its tag): the in-list ascends, so the entries that fall into one
+// bitmap word are neighbours, the entry that opens a word notes its place in a second shared-memory table, and a hit's
+// place is that plus the marked bits below it in its word (in-lists of 65,536 entries and more are searched instead).
+// Then the marked words are cleared again.  Dynamic shared memory: kC4BmSmem bytes.
 constexpr uint32_t kC4BmWords = 8192;    // 32 KB of shared memory: w < 2^18
 constexpr uint32_t kC4Chunk = 1024;      // two-paths per block step
+constexpr size_t kC4BmSmem = (size_t)kC4BmWords * 4 + (size_t)kC4BmWords * 2;
 
 template <typename K2, typename K, bool EMIT>
 __global__ void __launch_bounds__(256) k_cycle4_bitmap(Cycle4 P, const K2* __restrict__ keys2, const float* __restrict__ tags2, uint64_t n,
                                                        uint32_t* __restrict__ cnt, const uint64_t* __restrict__ off,
                                                        K* __restrict__ out_keys, float* __restrict__ out_tags) {
-  __shared__ uint32_t bm[kC4BmWords];
+  extern __shared__ uint32_t c4_smem[];
+  uint32_t* bm = c4_smem;
+  uint16_t* first = reinterpret_cast<uint16_t*>(c4_smem + kC4BmWords);      // per word: place in the in-list of the first entry marked in it
   __shared__ unsigned long long run_end_s;
   const unsigned lane = lane_id(), wid = threadIdx.x >> 5, nwarp = blockDim.x >> 5;
   for (uint32_t i = threadIdx.x; i < kC4BmWords; i += blockDim.x) bm[i] = 0u;
@@ -154,7 +160,12 @@ __global__ void __launch_bounds__(256) k_cycle4_bitmap(Cycle4 P, const K2* __res
       }
       uint32_t b0 = 0, b1 = 0;
       if (x < P.u_domain) { b0 = P.u_off[x]; b1 = P.u_off[x + 1]; }
-      for (uint32_t j = b0 + threadIdx.x; j < b1; j += blockDim.x) { const uint32_t w = (uint32_t)P.u_w[j]; atomicOr(&bm[w >> 5], 1u << (w & 31)); }
+      const bool ranked = EMIT && b1 - b0 < 65536u;
+      for (uint32_t j = b0 + threadIdx.x; j < b1; j += blockDim.x) {
+        const uint32_t w = (uint32_t)P.u_w[j];
+        atomicOr(&bm[w >> 5], 1u << (w & 31));
+        if (ranked && (j == b0 || ((uint32_t)P.u_w[j - 1] >> 5) != (w >> 5))) first[w >> 5] = (uint16_t)(j - b0);
+      }
       __syncthreads();
       const uint64_t rend = run_end_s;
       if (b1 > b0) {
@@ -206,7 +217,8 @@ __global__ void __launch_bounds__(256) k_cycle4_bitmap(Cycle4 P, const K2* __res
                 for (int u = 0; u < 2; ++u)
                   if (hit[u]) {
                     uint32_t lo = b0, hi = b1;             // where w sits in the in-list: its tag
-                    while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if ((uint32_t)P.u_w[mid] < w[u]) lo = mid + 1; else hi = mid; }
+                    if (ranked) lo = b0 + first[w[u] >> 5] + __popc(bm[w[u] >> 5] & ((1u << (w[u] & 31)) - 1u));
+                    else while (lo < hi) { const uint32_t mid = (lo + hi) >> 1; if ((uint32_t)P.u_w[mid] < w[u]) lo = mid + 1; else hi = mid; }
                     const uint64_t at = o + total + (u ? __popc(m0) : 0) + __popc((u ? m1 : m0) & lanemask_lt());
                     out_keys[at] = pre | ((K)w[u] << P.L.shift[3]);
                     out_tags[at] = P.times ? (tg * P.t_tag[j[u]]) * P.u_tag[lo] : (tg + P.t_tag[j[u]]) + P.u_tag[lo];

@@ -416,10 +416,11 @@ void cycle4_materialise(Ctx* c, Relation& H, const RuleC& r) {
   const unsigned bgrid = (unsigned)std::min<uint64_t>((n2 + kC4Chunk - 1) / kC4Chunk, (uint64_t)kSMs * 6);
 #define XLOG_C4(K2, KH, EMIT, KEYS, TAGS)                                                                                          \
   do {                                                                                                                             \
-    if (bitmap)                                                                                                                    \
-      XLOG_LAUNCH(c, (k_cycle4_bitmap<K2, KH, EMIT>), bgrid, 256, 0, P, (const K2*)k0.p, (const float*)t0.as<float>(), n2,         \
+    if (bitmap) {                                                                                                                  \
+      XLOG_CUDA(cudaFuncSetAttribute(k_cycle4_bitmap<K2, KH, EMIT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kC4BmSmem));   \
+      XLOG_LAUNCH(c, (k_cycle4_bitmap<K2, KH, EMIT>), bgrid, 256, kC4BmSmem, P, (const K2*)k0.p, (const float*)t0.as<float>(), n2,         \
                   cnt.as<uint32_t>(), (const uint64_t*)off.as<uint64_t>(), (KH*)(KEYS), (float*)(TAGS));                           \
-    else                                                                                                                           \
+    } else                                                                                                                         \
       XLOG_LAUNCH(c, (k_cycle4<K2, KH, EMIT>), grid, 256, 0, P, (const K2*)k0.p, (const float*)t0.as<float>(), n2,                 \
                   cnt.as<uint32_t>(), (const uint64_t*)off.as<uint64_t>(), (KH*)(KEYS), (float*)(TAGS));                           \
   } while (0)

@@ -214,38 +214,36 @@ static __global__ void __launch_bounds__(256) k_tri_unit_fill(const uint32_t* __
 // and folds them 32 at a time, a lane each.  A warp's partial result covers all its items of the unit; it is written to the first of them, the
 // others get the identity (the per-x combination that follows reads every item of x anyway).  The assignment of entries to
 // lanes depends on the graph alone, so results repeat from run to run.  Dynamic shared memory: 2 * words * 4 bytes (bits,
-// then the running count of set bits before each word).
+// then, per word, the place in in(x) of the first entry marked in it).
 template <typename Op>
 __global__ void __launch_bounds__(256) k_tri_bitmap(TriGraph G, int times, uint32_t n_units, const uint2* __restrict__ unit, const uint32_t* __restrict__ edge_off,
                                                     const uint32_t* __restrict__ item_off, const uint32_t* __restrict__ item_edge, uint32_t words,
                                                     uint32_t* __restrict__ item_cnt, typename Op::A* __restrict__ item_acc) {
   typedef typename Op::A A;
   extern __shared__ uint32_t tri_smem[];
-  __shared__ uint32_t sh[256 / 32 + 1];
   __shared__ uint32_t s_queue[8][32 * kTriBitmapUnroll + 32];      // a group's hits plus what an earlier group left
   uint32_t* bits = tri_smem;
   uint32_t* before = tri_smem + words;
   const unsigned lane = lane_id(), wid = warp_id();
   uint32_t* queue = s_queue[wid];
   int32_t have = -1;                                                         // the x whose in-list the bitmap holds
+  for (uint32_t i = threadIdx.x; i < words; i += 256) bits[i] = 0u;
   for (uint32_t u = blockIdx.x; u < n_units; u += gridDim.x) {
     const int32_t x = (int32_t)unit[u].x;
     const uint32_t b0 = G.in_off[x], b1 = G.in_off[x + 1];
     if (x != have) {
       __syncthreads();
-      for (uint32_t i = threadIdx.x; i < words; i += 256) bits[i] = 0u;
-      __syncthreads();
-      for (uint32_t i = b0 + threadIdx.x; i < b1; i += 256) { const uint32_t z = (uint32_t)G.in_src[i]; atomicOr(bits + (z >> 5), 1u << (z & 31)); }
-      __syncthreads();
-      // running count of set bits before each word: 256 words per step (a thread a word: no bank conflicts), a block-wide prefix per step
-      uint32_t carry = 0;
-      for (uint32_t i0 = 0; i0 < words; i0 += 256) {
-        const uint32_t i = i0 + threadIdx.x;
-        const uint32_t v = i < words ? __popc(bits[i]) : 0u;
-        uint32_t total;
-        const uint32_t ex = block_scan_excl<256, uint32_t>(v, sh, total);
-        if (i < words) before[i] = carry + ex;
-        carry += total;
+      if (have >= 0) {                                                         // unmark the previous in-list: only the words it touched
+        const uint32_t p0 = G.in_off[have], p1 = G.in_off[have + 1];
+        for (uint32_t i = p0 + threadIdx.x; i < p1; i += 256) bits[(uint32_t)G.in_src[i] >> 5] = 0u;
+        __syncthreads();
+      }
+      // in(x) ascends, so the entries that fall into one bitmap word are neighbours in the list: the entry that opens a word
+      // notes its place there, and the place of any marked z is that plus the marked bits below z in its word
+      for (uint32_t i = b0 + threadIdx.x; i < b1; i += 256) {
+        const uint32_t z = (uint32_t)G.in_src[i];
+        atomicOr(bits + (z >> 5), 1u << (z & 31));
+        if (i == b0 || ((uint32_t)G.in_src[i - 1] >> 5) != (z >> 5)) before[z >> 5] = i - b0;
       }
       __syncthreads();
       have = x;
