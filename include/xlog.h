@@ -83,6 +83,7 @@ typedef struct {
 #define XLOG_FLAG_NO_BITMAP_JOIN  256u  /* tag mirror, grouped join: always from a delta row list, never straight from the changed bitmap (see csrc/bitmap_join.cuh) */
 #define XLOG_FLAG_NO_DENSE_DOUBLING 512u /* tag mirror: the path-doubling rule h(x,z) :- h(x,y), h(y,z) goes through the sorting route, not the dense rounds */
 #define XLOG_FLAG_NO_TRIANGLE_BITMAP 1024u /* fused triangle aggregate: always search the longer list, never mark in(x) in a shared-memory bitmap (see csrc/triangle.cuh) */
+#define XLOG_FLAG_NO_ROW_FIXPOINT 2048u /* tag mirror, h(a,c) :- h(a,b), r(b,c): never run the rounds of each a on their own in shared memory (see csrc/row_fixpoint.cuh) */
 #define XLOG_FLAG_NO_GRAPH        16u  /* resident rounds are launched one by one instead of as one graph with a WHILE node */
 
 /* Evaluation routes of a recursive component (Algorithm 1).  All of them derive the same relation,
@@ -101,6 +102,10 @@ typedef struct {
  *    only rule over a binary h with at most 4096 values in its second column.  The mirror is then a matrix; a round copies
  *    it (the state both delta variants read) and one thread block per row applies every candidate of both variants in
  *    shared memory (csrc/dense_closure.cuh; XLOG_FLAG_NO_DENSE_DOUBLING sends the rule through the sorting route).
+ *  - Row-local fixpoint (tag mirror, one rule of the shape h(a, c) :- h(a, b), r(b, c) over h, at most 8192 possible values
+ *    of c): the rule never changes a, so the rounds of each a are independent; after the seed round one launch runs every
+ *    a's rounds to the end, a thread block per a with that a's slots in shared memory (csrc/row_fixpoint.cuh;
+ *    XLOG_FLAG_NO_ROW_FIXPOINT, and the flags that select the routes below, switch it off).
  *  - Resident rounds (tag mirror with <= 2^24 possible keys): the delta rounds run as one CUDA graph with a
  *    conditional WHILE node and fixed-capacity buffers (Section "GPU-Native Symbolic Substrate": resident
  *    conditional graph, no host reads inside the loop).  The buffers (about 36 bytes per possible key

@@ -7,6 +7,7 @@
 #include "group_join.cuh"
 #include "mirror.cuh"
 #include "resident.cuh"
+#include "row_fixpoint.cuh"
 
 namespace xlog {
 namespace {
@@ -410,10 +411,143 @@ void bitmap_join_setup(Ctx* c, int h, const std::vector<const RuleC*>& rs, const
   bj.valid = true;
 }
 
+// ---- row-local fixpoint (row_fixpoint.cuh) -------------------------------------------------------------------------
+constexpr int kSlotRow = kSlotBm;          // the kRowTotals counters of k_row_fixpoint (a stratum takes this route or the bitmap-driven one)
+static_assert(kSlotRow + kRowTotals <= kSlotDense, "control words overlap");
+
+// The one rule over h, h(a, c) :- h(a, b), r(b, c), when a value of a owns few enough keys for shared memory: fills `spec`
+// with the join in the relation's own key order.
+bool row_fixpoint_applies(Ctx* c, int h, const std::vector<const RuleC*>& rs, JoinSpec& spec) {
+  if (c->flags & (XLOG_FLAG_NO_ROW_FIXPOINT | XLOG_FLAG_NO_RESIDENT_LOOP | XLOG_FLAG_NO_GRAPH | XLOG_FLAG_NO_GROUPED_JOIN)) return false;
+  Relation& H = *c->rels[h];
+  if (!grouped_shape(c, h, rs) || H.dict_n[0] || H.dict_n[1] || H.layout.shift[1] != 0) return false;
+  const int c_bits = H.layout.shift[0];
+  if (c_bits < 5 || c_bits > kRowMaxBits) return false;
+  const RuleC* rule = nullptr; int pos = -1, n_over = 0;
+  for (const RuleC* r : rs)
+    for (int j = 0; j < r->plan.n_atoms; ++j)
+      if (r->plan.atoms[j].rel == h) { ++n_over; rule = r; pos = j; }
+  if (n_over != 1) return false;
+  const Variant v{rule, pos, Source{nullptr, nullptr, 0, H.layout, H.key_bytes}};
+  const JoinSpec S = make_spec(c, v, H);                   // builds the looked-up relation's index if it is missing
+  if (!S.fast || !S.has_inner || S.inner_free != 1 || S.outer_decode[0] || S.outer_decode[1] || S.head_encode[0] || S.head_encode[1] ||
+      S.inner_mult[0] != 1 || S.times)
+    return false;
+  spec = S;
+  return true;
+}
+
+// The stratum by the row-local route: the seed round from the host (every rule over the full relations, into the table),
+// then every row's rounds in one launch, then the table in key order is the relation.
+void stratum_row_fixpoint(Ctx* c, int h, const std::vector<const RuleC*>& rs, const JoinSpec& S) {
+  Relation& H = *c->rels[h];
+  const std::vector<int> comp{h};
+  const int bits = H.layout.total_bits, c_bits = H.layout.shift[0];
+  const uint64_t dom = (uint64_t)1 << bits;
+  const bool is_max = H.sr == XLOG_SR_MAXPLUS;
+  const int32_t empty = is_max ? kMirrorEmptyMax : kMirrorEmptyMin;
+  const uint64_t slots = dom;
+  const uint32_t nwords = (uint32_t)(dom / 32);
+  DevBuf table(c, slots * 4), bitmap(c, (size_t)nwords * 4), present(c, (size_t)nwords * 4);
+  XLOG_LAUNCH(c, k_fill_i32, grid_for(slots, 256 * 8), 256, 0, table.as<int32_t>(), slots, empty);
+  XLOG_CUDA(cudaMemsetAsync(bitmap.p, 0, (size_t)nwords * 4, c->stream));
+  XLOG_CUDA(cudaMemsetAsync(present.p, 0, (size_t)nwords * 4, c->stream));
+  const uint32_t n_start = H.n;
+  if (n_start)
+    XLOG_LAUNCH(c, (k_mirror_scatter<uint32_t>), grid_for(n_start, 256, 1 << 30), 256, 0, (const uint32_t*)H.keys(), (const float*)H.tags(), n_start, H.layout, H.layout,
+                table.as<int32_t>(), present.as<uint32_t>());
+  zero_ctrl(c, kSlotMirNew, 2);
+  zero_ctrl(c, kSlotRow, kRowTotals);
+  const MirrorArgs mr{table.as<int32_t>(), bitmap.as<uint32_t>(), (unsigned long long*)(c->d_ctrl + kSlotMirNew), (uint32_t)(dom - 1), ctrl_u32(c, kSlotErr)};
+  c->unique_untracked = true;
+  // seed round (Algorithm 1 lines 1-3)
+  if (c->max_iter < 1) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
+  ++c->r_iterations;
+  uint64_t seed_total = 0;
+  {
+    std::vector<Variant> vs;
+    for (const RuleC* r : rs) { const int outer = seed_outer(comp, r); vs.push_back(Variant{r, outer, full_source(*c->rels[r->plan.atoms[outer].rel])}); }
+    if (vs.size() > 16) fail(XLOG_ERR_UNSUPPORTED, "too many rule variants for one head");
+    std::vector<Counted> counted;
+    counted.reserve(vs.size());
+    for (Variant& v : vs) {
+      if (v.outer.n == 0) continue;
+      counted.emplace_back();
+      count_variant(c, v, H, counted.back(), kSlotTotals + (int)counted.size() - 1);
+    }
+    if (!counted.empty()) sync_ctrl(c);
+    for (Counted& q : counted) {
+      q.total = c->h_ctrl[q.slot];
+      q.deg.reset(); q.sums.reset();
+      seed_total += q.total;
+      c->r_candidates += (int64_t)q.total;
+      if (q.total) {
+        c->note_bytes = (int64_t)q.total * (4 + (q.spec.has_inner ? 4 * (q.spec.inner_free + 1) : 0));
+        launch_expand_mirror(c, q, is_max, mr);
+      }
+    }
+  }
+  uint64_t total_new = 0;
+  if (seed_total) {
+    RowFix P{};
+    P.table = table.as<int32_t>(); P.changed = bitmap.as<uint32_t>(); P.present = present.as<uint32_t>();
+    P.n_rows = (uint32_t)(slots >> c_bits); P.c_bits = c_bits;
+    P.off = S.inner_off; P.domain = (uint32_t)std::min<int64_t>(S.inner_domain, 0xffffffffll);
+    P.z = S.inner_col[0]; P.w = S.inner_tag; P.z_max = H.layout.mask[1];
+    P.max_rounds = (uint32_t)std::min<int64_t>(c->max_iter - 1, 0x7fffffff);
+    P.totals = (unsigned long long*)(c->d_ctrl + kSlotRow); P.err = ctrl_u32(c, kSlotErr);
+    const size_t smem = row_fix_smem(c_bits);
+    // per row: its slots read and written, its bitmap words; the candidates' reads of r are not known before the launch
+    c->note_bytes = (int64_t)slots * 8 + (int64_t)nwords * 12;
+    const unsigned grid = std::min<unsigned>(P.n_rows, kSMs * 16);
+    if (is_max) {
+      XLOG_CUDA(cudaFuncSetAttribute(k_row_fixpoint<kSinkMax>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)row_fix_smem(kRowMaxBits)));
+      XLOG_LAUNCH(c, (k_row_fixpoint<kSinkMax>), grid, kRowBlock, smem, P);
+    } else {
+      XLOG_CUDA(cudaFuncSetAttribute(k_row_fixpoint<kSinkMin>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)row_fix_smem(kRowMaxBits)));
+      XLOG_LAUNCH(c, (k_row_fixpoint<kSinkMin>), grid, kRowBlock, smem, P);
+    }
+    sync_ctrl(c);
+    const uint64_t cand = c->h_ctrl[kSlotRow + kRowCandidates], changed = c->h_ctrl[kSlotRow + kRowChanged], n_new = c->h_ctrl[kSlotRow + kRowNew];
+    c->r_candidates += (int64_t)cand;
+    c->r_new += (int64_t)n_new; c->r_improved += (int64_t)changed - (int64_t)n_new;
+    c->r_iterations += (int64_t)c->h_ctrl[kSlotRow + kRowRounds];
+    total_new = n_new;
+    if (c->h_ctrl[kSlotRow + kRowCapped]) fail(XLOG_ERR_CONVERGENCE_FAILURE, "iteration cap reached before the fixpoint");
+  }
+  // the relation in sorted form: every occupied slot, in slot order (the table is in key order)
+  const uint64_t n_out = (uint64_t)n_start + total_new;
+  KeyTags full;
+  full.n = (uint32_t)n_out;
+  full.keys = DevBuf(c, (size_t)std::max<uint64_t>(n_out, 1) * 4);
+  full.tags = DevBuf(c, (size_t)std::max<uint64_t>(n_out, 1) * 4);
+  if (n_out) {
+    const uint64_t nquads = slots / 4;
+    const unsigned tiles = (unsigned)((slots + kMirSlotsPerTile - 1) / kMirSlotsPerTile);
+    DevBuf sums(c, (size_t)tiles * 4);
+    c->note_bytes = (int64_t)slots * 4;
+    XLOG_LAUNCH(c, k_mirror_full_count, tiles, kMirBlock, 0, (const int4*)table.as<int4>(), nquads, empty, sums.as<uint32_t>());
+    XLOG_LAUNCH(c, (k_scan_spine<uint32_t>), 1, 1024, 0, sums.as<uint32_t>(), (int64_t)tiles, ctrl_u32(c, kSlotA));
+    c->note_bytes = (int64_t)slots * 4 + (int64_t)n_out * 8;
+    XLOG_LAUNCH(c, (k_mirror_full_emit<uint32_t>), tiles, kMirBlock, 0, (const int4*)table.as<int4>(), nquads, empty, (const uint32_t*)sums.as<uint32_t>(), H.layout,
+                H.layout, full.keys.as<uint32_t>(), full.tags.as<float>());
+  }
+  set_current(H, std::move(full));
+  if (c->flags & XLOG_FLAG_CHECK_INVARIANTS) {
+    XLOG_LAUNCH(c, (k_check_sorted<uint32_t>), grid_for(H.n, 256), 256, 0, (const uint32_t*)H.keys(), (int64_t)H.n, ctrl_u32(c, kSlotErr));
+    sync_ctrl(c);
+    if (n_out && (uint64_t)(uint32_t)c->h_ctrl[kSlotA] != n_out) fail(XLOG_ERR_INTERNAL, "tag mirror: occupied slots disagree with the tuple count");
+  }
+}
+
 // Algorithm 1 over a tag mirror (mirror.cuh): per round  count -> scan -> join straight into the table -> compact the
 // changed bitmap into the next delta.  No candidate is ever written to memory.  The seed round is driven by the host
 // (its rules scan whole relations of known size); the delta rounds run resident where the fixed-capacity buffers fit.
 void stratum_recursive_mirror(Ctx* c, int h, const std::vector<const RuleC*>& rs) {
+  {
+    JoinSpec row_spec;
+    if (row_fixpoint_applies(c, h, rs, row_spec)) { c->resident.erase(h); stratum_row_fixpoint(c, h, rs, row_spec); return; }
+  }
   Relation& H = *c->rels[h];
   const std::vector<int> comp{h};
   const int bits = H.layout.total_bits;

@@ -30,6 +30,7 @@ FLAG_NO_GROUPED_JOIN = 128
 FLAG_NO_BITMAP_JOIN = 256
 FLAG_NO_DENSE_DOUBLING = 512
 FLAG_NO_TRIANGLE_BITMAP = 1024
+FLAG_NO_ROW_FIXPOINT = 2048
 PLAN_NONE, PLAN_WCOJ, PLAN_CHAIN = 0, 1, 2
 
 EXPORTS = ["xlog_ctx_create", "xlog_ctx_destroy", "xlog_last_error", "xlog_relation_create", "xlog_relation_load",

@@ -38,10 +38,11 @@ def check_program(program, rel_tol=MINMAX_REL, abs_tol=0.0, expect_bit_equal=Tru
     from paper_2609_27203_b200 import xlog
     o, oids, _, stats = oracle_run(program, mode)
     receipts, results = [], []
-    # default (tag mirror, delta rounds resident in one graph) / the same rounds launched one by one / host-driven
+    # default (tag mirror; the rounds of each first-column value on their own in shared memory where the rule has that shape,
+    # else delta rounds resident in one graph) / resident in one graph always / the same rounds launched one by one / host-driven
     # mirror rounds (with the grouped join where the rule has that shape, driven by the changed bitmap where a unit of 32
     # carried values exists) / the grouped join from a delta row list / the row-wise join only / the sorting path
-    for extra in (0, xlog.FLAG_NO_GRAPH, xlog.FLAG_NO_RESIDENT_LOOP, xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_BITMAP_JOIN,
+    for extra in (0, xlog.FLAG_NO_ROW_FIXPOINT, xlog.FLAG_NO_GRAPH, xlog.FLAG_NO_RESIDENT_LOOP, xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_BITMAP_JOIN,
                   xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_GROUPED_JOIN, xlog.FLAG_NO_TAG_MIRROR):
         ctx, gids, _, receipt = gpu_run(program, **dict(kw, flags=kw.get("flags", xlog.FLAG_CHECK_INVARIANTS) | extra))
         got = {}

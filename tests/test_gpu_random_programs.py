@@ -17,7 +17,7 @@ SEEDS = sorted(set(range(80)) | {199, 214, 219})
 @pytest.mark.parametrize("chunk", range(4))
 def test_random_programs_agree_with_the_oracle_on_every_route(chunk):
     from paper_2609_27203_b200 import xlog
-    routes = (0, xlog.FLAG_NO_GRAPH, xlog.FLAG_NO_RESIDENT_LOOP, xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_BITMAP_JOIN,
+    routes = (0, xlog.FLAG_NO_ROW_FIXPOINT, xlog.FLAG_NO_GRAPH, xlog.FLAG_NO_RESIDENT_LOOP, xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_BITMAP_JOIN,
               xlog.FLAG_NO_RESIDENT_LOOP | xlog.FLAG_NO_GROUPED_JOIN, xlog.FLAG_NO_TAG_MIRROR)
     for seed in SEEDS[chunk::4]:
         p = random_program(seed)
