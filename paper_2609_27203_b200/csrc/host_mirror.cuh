@@ -420,7 +420,7 @@ static_assert(kSlotRow + kRowTotals <= kSlotDense, "control words overlap");
 bool row_fixpoint_applies(Ctx* c, int h, const std::vector<const RuleC*>& rs, JoinSpec& spec) {
   if (c->flags & (XLOG_FLAG_NO_ROW_FIXPOINT | XLOG_FLAG_NO_RESIDENT_LOOP | XLOG_FLAG_NO_GRAPH | XLOG_FLAG_NO_GROUPED_JOIN)) return false;
   Relation& H = *c->rels[h];
-  if (!grouped_shape(c, h, rs) || H.dict_n[0] || H.dict_n[1] || H.layout.shift[1] != 0) return false;
+  if (!grouped_shape(c, h, rs) || H.dict_n[1] || H.layout.shift[1] != 0) return false;   // a dictionary on column 0 is fine: its codes pass through the rule unchanged
   const int c_bits = H.layout.shift[0];
   if (c_bits < 5 || c_bits > kRowMaxBits) return false;
   const RuleC* rule = nullptr; int pos = -1, n_over = 0;

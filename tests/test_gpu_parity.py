@@ -374,6 +374,36 @@ def test_fixpoint_idempotent_and_reset():
     ctx.close()
 
 
+def test_row_local_fixpoint_route_edges():
+    # the route that runs each first-column value's rounds on its own in shared memory: (1) the iteration cap bites at
+    # exactly the round where the other routes stop, (2) rows of 8192 slots (the largest it takes) with a skewed graph,
+    # (3) a head that starts with loaded facts, some better and some worse than what the rule derives
+    from paper_2609_27203_b200 import xlog
+    chain = W.closure_program(np.arange(40), np.arange(1, 41), -np.ones(40, np.float32))
+    need = oracle_run(chain, "seminaive")[3]["iterations"]
+    for flags in (0, xlog.FLAG_NO_ROW_FIXPOINT):
+        ctx, ids, _ = xlog.load_program(chain, arena_bytes=1 << 26, max_iterations=need, flags=flags)
+        assert ctx.fixpoint()["iterations"] == need
+        ctx.close()
+        ctx, ids, _ = xlog.load_program(chain, arena_bytes=1 << 26, max_iterations=need - 1, flags=flags)
+        with pytest.raises(xlog.XlogError) as e:
+            ctx.fixpoint()
+        assert e.value.status == "CONVERGENCE_FAILURE"
+        ctx.close()
+    prog = W.config5(scale=13, n_sources=24)
+    r, _ = check_program(prog)
+    ctx, ids, _ = xlog.load_program(prog, arena_bytes=1 << 28, flags=xlog.FLAG_PROFILE)
+    ctx.fixpoint()
+    assert "k_row_fixpoint" in ctx.profile()
+    ctx.close()
+    s, d = synth.uniform_digraph(300, 1200, 91)
+    w = (1 + 9 * synth.uniform01(91, 2, 0, 1200)).astype(np.float32)
+    srcs = np.array([2, 50, 299], np.int32)
+    p2 = W.reach_program(s, d, w, srcs, W.MINPLUS, name="reach_with_facts")
+    p2.facts["reach"] = ([np.array([2, 2, 50, 7], np.int32), np.array([9, 10, 11, 12], np.int32)], np.array([0.25, 500.0, 3.0, 1.0], np.float32))
+    check_program(p2)
+
+
 def test_typed_failures_leave_the_context_usable():
     from paper_2609_27203_b200 import xlog
     chain = W.closure_program(np.arange(30), np.arange(1, 31), -np.ones(30, np.float32))
