@@ -104,7 +104,8 @@ typedef struct {
  *    shared memory (csrc/dense_closure.cuh; XLOG_FLAG_NO_DENSE_DOUBLING sends the rule through the sorting route).
  *  - Row-local fixpoint (tag mirror, one rule of the shape h(a, c) :- h(a, b), r(b, c) over h, at most 8192 possible values
  *    of c): the rule never changes a, so the rounds of each a are independent; after the seed round one launch runs every
- *    a's rounds to the end, a thread block per a with that a's slots in shared memory (csrc/row_fixpoint.cuh;
+ *    a's rounds to the end, a thread block per a with that a's slots in shared memory; several mutually recursive heads
+ *    whose rules all read h_i(a, c) :- h_j(a, b), r(b, c) and that share one key layout are handled alike (csrc/row_fixpoint.cuh;
  *    XLOG_FLAG_NO_ROW_FIXPOINT, and the flags that select the routes below, switch it off).
  *  - Resident rounds (tag mirror with <= 2^24 possible keys): the delta rounds run as one CUDA graph with a
  *    conditional WHILE node and fixed-capacity buffers (Section "GPU-Native Symbolic Substrate": resident
