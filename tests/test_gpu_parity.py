@@ -286,6 +286,14 @@ def test_mutual_recursion_over_one_tag_mirror_per_head():
                        W.Rule("lo", (W.V(0), W.V(2)), (W.Atom("hi", (W.Var(0), W.Var(1))), W.Atom("e", (W.Var(1), W.Var(2)))))],
                       {"e": ([s2, d2], w2)}, ("lo", "hi"))
     check_program(mixed)
+    # which route ran: two binary heads with one key layout and closure-shaped rules take the row-local fixpoint (a row per
+    # head in the block); the three heads above, one of them unary, take the host-driven rounds over one mirror per head
+    for program, row_local in ((mixed, True), (prog, False)):
+        ctx, ids, _ = xlog.load_program(program, arena_bytes=1 << 28, flags=xlog.FLAG_PROFILE)
+        ctx.fixpoint()
+        assert ("k_row_fixpoint" in ctx.profile()) == row_local
+        assert "k_sort_pass" not in ctx.profile() or not row_local
+        ctx.close()
 
 
 def test_recursion_with_head_arithmetic_takes_the_general_join_path():
