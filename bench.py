@@ -309,6 +309,9 @@ def roofline_of(program, prof_all, steps, sorting_route):
                         probes_per_s=l2["probes_per_s"], l2_bytes_per_probe=l2["l2_bytes_per_probe"])
         if "issue" in l2:
             roofline["issue"] = l2["issue"]
+    if dom in ("k_row_fixpoint", "k_dense_round"):
+        roofline["limiter"] = ("every round runs out of shared memory with the looked-up relation in L2; the rows cross HBM once, so the HBM "
+                               "fraction says nothing: read ms_per_step and the metric")
     if mirror_kernel:
         # the tag-mirror joins move few bytes per candidate by construction; what limits them is said here
         roofline["limiter"] = ("instruction issue; the table, too large for L2, is read from HBM one 128-byte line per (changed unit of 32 keys, neighbour)"
