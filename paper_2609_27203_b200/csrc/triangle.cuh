@@ -36,7 +36,10 @@ constexpr uint32_t kTriChunk = 1024;     // walked entries per work item (32 swe
 // walks out(y) even where in(x) is the shorter list, and it pays for building the bitmap, so it is taken per x, from two
 // sums over x's edges that depend on the graph alone: the entries either way would walk.
 constexpr int64_t kTriBitmapMaxDomain = (int64_t)1 << 19;      // nodes (sources and targets alike): 64 KB of bits and 64 KB of running counts
-constexpr int kTriBitmapUnroll = 8;                            // sweeps of 32 list entries a warp reads before it tests them
+#ifndef XLOG_TRI_UNROLL
+#define XLOG_TRI_UNROLL 8
+#endif
+constexpr int kTriBitmapUnroll = XLOG_TRI_UNROLL;                            // sweeps of 32 list entries a warp reads before it tests them
 #ifndef XLOG_TRI_UNIT_ITEMS
 #define XLOG_TRI_UNIT_ITEMS 512
 #endif
