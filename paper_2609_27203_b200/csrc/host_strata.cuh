@@ -3,7 +3,7 @@
 #pragma once
 #include "host_backward.cuh"
 #include "host_cyclic.cuh"
-#include "host_mirror.cuh"
+#include "host_mirror_strata.cuh"
 
 namespace xlog {
 namespace {
